@@ -1,0 +1,111 @@
+"""Workload definitions and seeded synthetic inputs.
+
+This module holds NONE of the method's arithmetic: only shapes, CKKS parameter literals and
+random-number recipes.  It is the one module both the CPU reference used by the tests and the CUDA
+library's callers draw inputs from.
+
+The synthetic layers stand in for the trained GPT-2 / Qwen3 / LLaMA-3 checkpoints the paper's
+evaluation (Sec. 5.1) runs on: only the layer shapes are kept; weights are fp32 N(0, 0.02^2),
+activations fp64 N(0, 1), everything derived from one base seed with a distinct stream per object.
+"""
+from __future__ import annotations
+
+import zlib
+from dataclasses import dataclass, field
+
+import numpy as np
+
+# ----------------------------------------------------------------------------- CKKS parameter sets
+# Largest primes = 1 (mod 2N) below 2^50 (base prime), below 2^40 (descending) and below 2^60
+# (special prime for key switching).
+Q40_N15 = [1099510054913, 1099507695617, 1099506515969, 1099504549889, 1099503894529, 1099503370241]
+
+PARAM_SETS = {
+    "n12": dict(N=1 << 12, primes=[1125899906826241, 1099511480321, 1099511390209],
+                special=1152921504606830593, scale=2.0 ** 40),
+    "n15": dict(N=1 << 15, primes=[1125899904679937] + Q40_N15,
+                special=1152921504606584833, scale=2.0 ** 40),
+    "n16": dict(N=1 << 16, primes=[1125899903827969] + Q40_N15 + [1099502714881, 1099500617729],
+                special=1152921504606584833, scale=2.0 ** 40),
+    # The prototype's own parameter set (Sec. 4.2): N = 8192, primes of [60, 30, 30, 30] bits,
+    # scale 2^30, one 60-bit special prime.
+    "paper_n13": dict(N=1 << 13, primes=[1152921504606830593, 1073692673, 1073643521, 1073479681],
+                      special=1152921504606748673, scale=2.0 ** 30),
+}
+
+
+@dataclass(frozen=True)
+class PlanSpec:
+    """Tile side D, replica split tau, baby steps b, giant steps g (b*g = D/tau)."""
+    D: int
+    tau: int
+    b: int
+    g: int
+
+
+@dataclass(frozen=True)
+class Layer:
+    name: str
+    d_in: int
+    d_out: int
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    params: str                 # key of PARAM_SETS
+    plan: PlanSpec
+    layers: tuple               # the distinct projections of one transformer layer
+    n_repeat: int = 1           # number of transformer layers in a decode step
+    cache_budget_bytes: int | None = None
+
+
+GPT2_LAYER = (Layer("qkv", 768, 2304), Layer("out_proj", 768, 768),
+              Layer("ffn_up", 768, 3072), Layer("ffn_down", 3072, 768))
+QWEN3_LAYER = (Layer("q", 1024, 2048), Layer("k", 1024, 1024), Layer("v", 1024, 1024),
+               Layer("o", 2048, 1024), Layer("gate", 1024, 3072), Layer("up", 1024, 3072),
+               Layer("down", 3072, 1024))
+LLAMA3_8B_LAYER = (Layer("q", 4096, 4096), Layer("k", 4096, 1024), Layer("v", 4096, 1024),
+                   Layer("o", 4096, 4096), Layer("gate", 4096, 14336), Layer("up", 4096, 14336),
+                   Layer("down", 14336, 4096))
+
+WORKLOADS = {
+    "tiny": Workload("tiny", "n12", PlanSpec(64, 1, 8, 8), (Layer("w", 64, 64),)),
+    "gpt2_qkv": Workload("gpt2_qkv", "n15", PlanSpec(1024, 16, 8, 8), (GPT2_LAYER[0],)),
+    "gpt2_step": Workload("gpt2_step", "n15", PlanSpec(1024, 16, 8, 8), GPT2_LAYER, n_repeat=12),
+    "qwen3_step": Workload("qwen3_step", "n15", PlanSpec(1024, 16, 8, 8), QWEN3_LAYER, n_repeat=28,
+                           cache_budget_bytes=60 * 10 ** 9),
+    "llama3_layer": Workload("llama3_layer", "n16", PlanSpec(1024, 32, 8, 4), LLAMA3_8B_LAYER),
+}
+CONFIG_ORDER = ["tiny", "gpt2_qkv", "gpt2_step", "qwen3_step", "llama3_layer"]
+
+
+# ----------------------------------------------------------------------------- seeded generators
+
+def _stream(seed: int, *tag) -> np.random.Generator:
+    words = [seed & 0xFFFFFFFF]
+    for t in tag:
+        words.append(zlib.crc32(str(t).encode()) if not isinstance(t, int) else t & 0xFFFFFFFF)
+    return np.random.Generator(np.random.PCG64(words))
+
+
+def gen_weights(seed: int, tag, d_out: int, d_in: int) -> np.ndarray:
+    """fp32 W[d_out][d_in] ~ N(0, 0.02^2)."""
+    return (_stream(seed, "W", tag).standard_normal((d_out, d_in)) * 0.02).astype(np.float32)
+
+
+def gen_activation(seed: int, tag, d_in: int) -> np.ndarray:
+    """fp64 x[d_in] ~ N(0, 1)."""
+    return _stream(seed, "x", tag).standard_normal(d_in)
+
+
+def gen_uniform_residues(seed: int, tag, moduli, shape_tail) -> np.ndarray:
+    """uint64 [len(moduli), *shape_tail], row i uniform in [0, moduli[i]).  A fresh ciphertext and a
+    switching key are computationally indistinguishable from this, so it serves as a stand-in
+    when only throughput is measured."""
+    rng = _stream(seed, "u", tag)
+    return np.stack([rng.integers(0, int(q), size=shape_tail, dtype=np.uint64) for q in moduli])
+
+
+def ceil_div(a: int, b: int) -> int:
+    return -(-a // b)
