@@ -1,0 +1,150 @@
+/*
+ * libbifrost: the accelerator-side CKKS linear layer of a hybrid TEE-FHE serving stack, for one
+ * NVIDIA B200 (sm_100a).  The trusted side (key generation, encryption, decryption, non-linear
+ * operators) is not here: callers hand in ciphertexts and rotation keys as plain arrays.
+ *
+ * Conventions shared by all entry points
+ *   - Every function returns BF_OK (0) or a negative BF_ERR_* code; nothing throws or aborts.
+ *     bf_strerror() names a code; bf_last_cuda_error() gives the CUDA message behind BF_ERR_CUDA.
+ *   - A context is bound to the CUDA device that was current at bf_ctx_create() and to one stream.
+ *     Calls only enqueue work on that stream (exceptions are stated); the caller synchronises.
+ *     Calls on one context must not overlap on the host.
+ *   - r = number of ciphertext primes q_0..q_{r-1}; P = special prime; N = ring degree.
+ *   - Ciphertext layout at the boundary: uint64 [2][r][N] = component (c0, c1), prime, coefficient,
+ *     in the COEFFICIENT domain with every residue in [0, q_i).  Arrays of ciphertexts are stored
+ *     back to back.  Decryption is c0 + c1*s.
+ *   - Rotation-key layout at the boundary: uint64 [r][2][r+1][N] = digit j, component (b, a),
+ *     prime of the extended basis {q_0..q_{r-1}, P}, coefficient; coefficient domain.
+ *   - "device" pointers are CUDA device memory owned by the caller; the library keeps no reference
+ *     to them after the enqueued work has run.  "host" pointers are ordinary host memory read or
+ *     written before the call returns, unless stated.
+ */
+#ifndef BIFROST_H
+#define BIFROST_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    BF_OK = 0,
+    BF_ERR_INVALID_ARG = -1,   /* null pointer, zero size, N not a power of two in [2^10, 2^16], ... */
+    BF_ERR_BAD_PRIME = -2,     /* not prime, not 1 mod 2N, duplicate, or not below 2^60 */
+    BF_ERR_SHAPE = -3,         /* n_in / n_out do not match d_in / d_out and the plan, or plan inconsistent */
+    BF_ERR_LEVEL = -4,         /* level outside [2, r] */
+    BF_ERR_MISSING_KEY = -5,   /* the plan needs a rotation whose key was not loaded */
+    BF_ERR_OOM = -6,           /* encoded weights exceed the cache budget, or device memory is exhausted */
+    BF_ERR_CUDA = -7,          /* a CUDA call failed; see bf_last_cuda_error() */
+    BF_ERR_RANGE = -8          /* an encoded coefficient does not fit 2^62 (scale too large for the data) */
+};
+
+typedef struct bf_ctx bf_ctx;          /* ring tables, rotation keys, scratch memory */
+typedef struct bf_weights bf_weights;  /* device-resident encoded diagonals of one projection */
+
+/* Tiling of a projection (the paper leaves packing open beyond "weight diagonals" kept as
+ * baby-step/giant-step objects, Sec. 4.2):  the weight matrix is cut into tile_D x tile_D tiles;
+ * slot s = (rho*tile_D + kappa)*tau + c of an input ciphertext holds x[(kappa + c*M) mod tile_D]
+ * of its chunk, M = tile_D/tau generalised diagonals per tile, split as M = bsgs_b * bsgs_g.
+ * All four are powers of two and tile_D*tau <= N/2. */
+typedef struct {
+    uint32_t tile_D, tau, bsgs_b, bsgs_g;
+} bf_plan;
+
+/* Create a context (Sec. 4.2: one CKKS context per projection shape, with its modulus chain and
+ * BSGS rotation parameters).
+ *   primes       host, n_ct_primes + 1 values: q_0..q_L then the special prime P
+ *   scale        Delta used when encoding weights (a power of two keeps the scaling exact)
+ *   cuda_stream  a cudaStream_t (0 = default stream)
+ * Allocates device tables; synchronises the device once.  Errors: INVALID_ARG, BAD_PRIME, SHAPE,
+ * CUDA. */
+int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, uint32_t n_ct_primes, double scale,
+                  const bf_plan* plan, void* cuda_stream);
+
+/* Frees everything the context owns, including weights not yet freed.  Synchronises. */
+void bf_ctx_destroy(bf_ctx* ctx);
+
+/* Load rotation (Galois) keys, replacing any loaded before (Sec. 4.1 "rotation material").
+ *   rot_steps  host, n_keys left-rotation amounts; key t switches from s(X^(5^rot_steps[t])) to s
+ *   keys       device, [n_keys][r][2][r+1][N] in the boundary layout
+ * The keys are transformed into the library's evaluation layout in its own memory.  Required
+ * amounts for a plan: k*tau for k = 1..b-1 and j*b*tau for j = 1..g-1.  Synchronises. */
+int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_t n_keys, const uint64_t* keys);
+
+/* Upper bound in bytes on the encoded weights kept resident by this context (Sec. 4.2: persistent
+ * cache vs fallback-encode modes).  0 = unlimited (default). */
+int bf_set_cache_budget(bf_ctx* ctx, uint64_t bytes);
+uint64_t bf_cache_bytes_used(const bf_ctx* ctx);
+
+/* Bytes bf_encode_weights would keep resident for a d_out x d_in projection under the plan. */
+uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in);
+
+/* EncodeWeights (Alg. 3, offline phase; Sec. 4.2): encode every generalised diagonal of
+ * W[d_out][d_in] (device, fp32, row-major) at scale Delta, reduce per prime and transform, keeping
+ * the result in device memory owned by the returned handle.  Returns BF_ERR_OOM without
+ * allocating when the cache budget would be exceeded: the caller then passes W itself to bf_linear.
+ * Synchronises. */
+int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, uint32_t d_in, bf_weights** out);
+void bf_weights_free(bf_ctx* ctx, bf_weights* w);
+
+/* FHE_Linear (Alg. 3, decode loop; Sec. 4.2 "BSGS matrix-vector multiply"):
+ *     ct_out[p] = sum_{j<g} rot( sum_q sum_{k<b} Pt[p][q][j][k] * rot(ct_in[q], k*tau), j*b*tau )
+ * for p < n_out = ceil(d_out/tile_D), q < n_in = ceil(d_in/tile_D).  Rotations are automorphisms
+ * followed by a key switch with one special prime (one prime per digit), each with its own
+ * division by P.
+ *   ct_in       device, n_in ciphertexts at full level, boundary layout
+ *   pt_weights  handle from bf_encode_weights for this (d_out, d_in); or NULL, in which case
+ *   W_raw       device fp32 [d_out][d_in] is encoded on the fly (fallback path)
+ *   ct_out      device, n_out ciphertexts, full level, scale = scale(ct_in) * Delta; must not
+ *               overlap ct_in
+ * Slot (0, kappa, c) of ct_out[p] decrypts to the partial dot product of row p*tile_D + kappa over
+ * column class c; the caller adds the tau partial sums.  Asynchronous on the context's stream,
+ * except that scratch memory may be grown (which synchronises) the first time a shape is seen.
+ * Errors: INVALID_ARG, SHAPE, MISSING_KEY, OOM, RANGE (fallback path only), CUDA. */
+int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
+              const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out);
+
+/* Rescale (Sec. 2.1): drop the last prime of n_ct ciphertexts that have `level` primes each,
+ *     c'_i = (c_i - centred(c_{level-1})) * q_{level-1}^{-1} mod q_i ,
+ * i.e. round(c / q_{level-1}).  ct_in: device [n_ct][2][level][N]; ct_out: device
+ * [n_ct][2][level-1][N]; ct_out may equal ct_in.  *scale_inout is divided by q_{level-1} when not
+ * NULL.  Asynchronous.  Errors: INVALID_ARG, LEVEL, CUDA. */
+int bf_rescale(bf_ctx* ctx, const uint64_t* ct_in, uint64_t* ct_out, uint32_t n_ct, uint32_t level,
+               double* scale_inout);
+
+/* bf_linear followed by bf_rescale with HOST buffers: copies n_in ciphertexts from host_ct_in to
+ * the device, runs the layer, rescales once and copies the n_out ciphertexts of level r-1 back to
+ * host_ct_out ([n_out][2][r-1][N]).  Pinned host memory makes the copies asynchronous; the call
+ * returns after the result has arrived (it synchronises the stream). */
+int bf_linear_host(bf_ctx* ctx, const uint64_t* host_ct_in, uint32_t n_in, const bf_weights* pt_weights,
+                   const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* host_ct_out, uint32_t n_out);
+
+/* One key-switched left rotation of a full-level ciphertext by `steps` slots (the primitive the
+ * baby and giant steps are made of).  ct_in, ct_out: device, boundary layout.  Asynchronous. */
+int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uint64_t* ct_out);
+
+/* Products in Z_q[X]/(X^N + 1): out[t] = a[t] * b[t] for n_polys polynomials, polynomial t modulo
+ * basis prime (t mod (r+1)); all device, [n_polys][N], coefficient domain.  Exercises the forward
+ * and inverse transforms.  Asynchronous. */
+int bf_negacyclic_mul(bf_ctx* ctx, const uint64_t* a, const uint64_t* b, uint64_t* out, uint32_t n_polys);
+
+/* Coefficient-domain residues [r][N] (device) of the encoded plaintext Pt[p][q][j][k] held by w. */
+int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, uint32_t q, uint32_t j, uint32_t k,
+                      uint64_t* out);
+
+/* Per-stage device time of the last bf_linear on this context, in milliseconds, when stage timing
+ * was switched on with bf_set_stage_timing(ctx, 1) (adds event records; off by default).
+ * stages: 0 input transforms + hoisted ModUp + baby steps, 1 multiply-accumulate (on the fallback
+ * path: with the on-the-fly encoding), 2 giant steps, 3 output transform.
+ * bf_get_stage_ms synchronises the stream. */
+int bf_set_stage_timing(bf_ctx* ctx, int on);
+int bf_get_stage_ms(bf_ctx* ctx, float* ms_out /* host, 4 values */);
+
+const char* bf_strerror(int code);
+const char* bf_last_cuda_error(const bf_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BIFROST_H */

@@ -1,0 +1,859 @@
+// C ABI of libbifrost: context and table set-up, key loading, weight encoding, and the launch
+// sequence of the encrypted linear layer (Alg. 3: EncodeWeights, FHE_Linear; Sec. 4.2).
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/bifrost.h"
+#include "bf_host.h"
+
+using namespace bf;
+
+typedef unsigned __int128 u128;
+
+// ------------------------------------------------------------------------------------------------
+// host number theory (table set-up only)
+static u64 h_mulmod(u64 a, u64 b, u64 q) { return (u64)((u128)a * b % q); }
+static u64 h_powmod(u64 a, u64 e, u64 q) {
+    u64 r = 1 % q;
+    a %= q;
+    for (; e; e >>= 1) {
+        if (e & 1) r = h_mulmod(r, a, q);
+        a = h_mulmod(a, a, q);
+    }
+    return r;
+}
+static u64 h_invmod(u64 a, u64 q) { return h_powmod(a % q, q - 2, q); }
+static u64 h_shoup(u64 w, u64 q) { return (u64)(((u128)w << 64) / q); }
+
+static bool h_is_prime(u64 n) {
+    if (n < 2) return false;
+    const u64 small[] = {2, 3, 5, 7, 11, 13, 17, 19, 23, 29, 31, 37};
+    for (u64 p : small) {
+        if (n % p == 0) return n == p;
+    }
+    u64 d = n - 1;
+    int s = 0;
+    while (!(d & 1)) { d >>= 1; ++s; }
+    for (u64 a : small) {              // these witnesses are conclusive below 2^64
+        u64 x = h_powmod(a, d, n);
+        if (x == 1 || x == n - 1) continue;
+        bool composite = true;
+        for (int i = 1; i < s && composite; ++i) {
+            x = h_mulmod(x, x, n);
+            if (x == n - 1) composite = false;
+        }
+        if (composite) return false;
+    }
+    return true;
+}
+
+static u32 h_brev(u32 x, int bits) {
+    u32 r = 0;
+    for (int i = 0; i < bits; ++i) { r = (r << 1) | (x & 1); x >>= 1; }
+    return r;
+}
+
+// a primitive 2N-th root of unity modulo q
+static u64 h_root_2n(u64 q, u32 N) {
+    const u64 e = (q - 1) / (2ull * N);
+    for (u64 x = 3; x < q; ++x) {
+        u64 psi = h_powmod(x, e, q);
+        if (h_powmod(psi, N, q) == q - 1) return psi;
+    }
+    return 0;
+}
+
+// ------------------------------------------------------------------------------------------------
+struct DevBuf {
+    void* p = nullptr;
+    size_t cap = 0;
+};
+
+struct bf_weights {
+    u32 d_out, d_in, n_in, n_out;
+    u64* pt;            // [g][n_out][n_in][b][r][N], NTT domain
+    size_t bytes;
+};
+
+struct bf_ctx {
+    RingHost ring;
+    u32 N, logN, r;
+    double scale;
+    bf_plan plan;
+    cudaStream_t stream;
+    int device;
+    ulonglong2 *tw_fwd = nullptr, *tw_inv = nullptr;
+    u32* slot_of_pos = nullptr;
+    double2 *T = nullptr, *Z = nullptr;
+    int* overflow_flag = nullptr;
+    // rotation keys
+    std::map<u32, int> key_of_steps;
+    u64* keys = nullptr;
+    u32* perms = nullptr;
+    u32 n_keys = 0;
+    // scratch (grow-only)
+    DevBuf X, Dig, U, Tc, Tn, Cc, A, Rres, Y, fft, coef, ptjit, stage_in, stage_out, nm_a, nm_b;
+    u64 cache_budget = 0, cache_used = 0;
+    std::vector<bf_weights*> weights;
+    std::string cuda_msg;
+    // stage timing
+    int timing = 0;
+    cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool ev_valid = false;
+};
+
+#define CK(call)                                                              \
+    do {                                                                      \
+        cudaError_t e__ = (call);                                             \
+        if (e__ != cudaSuccess) {                                             \
+            ctx->cuda_msg = std::string(#call) + ": " + cudaGetErrorString(e__); \
+            return BF_ERR_CUDA;                                               \
+        }                                                                     \
+    } while (0)
+
+static int ensure(bf_ctx* ctx, DevBuf& b, size_t bytes) {
+    if (b.cap >= bytes) return BF_OK;
+    CK(cudaStreamSynchronize(ctx->stream));
+    if (b.p) CK(cudaFree(b.p));
+    b.p = nullptr;
+    b.cap = 0;
+    cudaError_t e = cudaMalloc(&b.p, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        ctx->cuda_msg = std::string("cudaMalloc: ") + cudaGetErrorString(e);
+        return BF_ERR_OOM;
+    }
+    b.cap = bytes;
+    return BF_OK;
+}
+
+#define TRY(call)                     \
+    do {                              \
+        int s__ = (call);             \
+        if (s__ != BF_OK) return s__; \
+    } while (0)
+
+static bool is_pow2(u32 x) { return x && !(x & (x - 1)); }
+
+extern "C" const char* bf_strerror(int code) {
+    switch (code) {
+        case BF_OK: return "ok";
+        case BF_ERR_INVALID_ARG: return "invalid argument";
+        case BF_ERR_BAD_PRIME: return "bad prime (not prime, not 1 mod 2N, duplicate, or >= 2^60)";
+        case BF_ERR_SHAPE: return "shape does not match the plan";
+        case BF_ERR_LEVEL: return "bad level";
+        case BF_ERR_MISSING_KEY: return "rotation key not loaded";
+        case BF_ERR_OOM: return "out of memory or over the cache budget";
+        case BF_ERR_CUDA: return "CUDA error";
+        case BF_ERR_RANGE: return "encoded coefficient out of range";
+        default: return "unknown error";
+    }
+}
+
+extern "C" const char* bf_last_cuda_error(const bf_ctx* ctx) { return ctx ? ctx->cuda_msg.c_str() : ""; }
+
+// ------------------------------------------------------------------------------------------------
+extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, uint32_t n_ct_primes, double scale,
+                             const bf_plan* plan, void* cuda_stream) {
+    if (!out || !primes || !plan) return BF_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!is_pow2(N) || N < (1u << 10) || N > (1u << 16)) return BF_ERR_INVALID_ARG;
+    if (n_ct_primes < 2 || n_ct_primes + 1 > (u32)MAX_MODULI) return BF_ERR_INVALID_ARG;
+    if (!(scale >= 1.0) || !std::isfinite(scale)) return BF_ERR_INVALID_ARG;
+    const u32 nb = n_ct_primes + 1;
+    for (u32 i = 0; i < nb; ++i) {
+        const u64 q = primes[i];
+        if (q >= (1ull << 60) || q % (2ull * N) != 1 || !h_is_prime(q)) return BF_ERR_BAD_PRIME;
+        for (u32 k = 0; k < i; ++k)
+            if (primes[k] == q) return BF_ERR_BAD_PRIME;
+    }
+    const u32 n = N / 2;
+    if (!is_pow2(plan->tile_D) || !is_pow2(plan->tau) || !is_pow2(plan->bsgs_b) || !is_pow2(plan->bsgs_g))
+        return BF_ERR_SHAPE;
+    if ((u64)plan->tile_D * plan->tau > n || plan->tile_D % plan->tau != 0 ||
+        (u64)plan->bsgs_b * plan->bsgs_g != plan->tile_D / plan->tau)
+        return BF_ERR_SHAPE;
+    if (plan->bsgs_b - 1 > (u32)MAX_ROT_BATCH) return BF_ERR_SHAPE;
+
+    bf_ctx* ctx = new (std::nothrow) bf_ctx();
+    if (!ctx) return BF_ERR_OOM;
+    ctx->N = N;
+    ctx->logN = 0;
+    while ((1u << ctx->logN) < N) ctx->logN++;
+    ctx->r = n_ct_primes;
+    ctx->scale = scale;
+    ctx->plan = *plan;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    int status = BF_OK;
+    auto fail = [&](int s) {
+        bf_ctx_destroy(ctx);
+        return s;
+    };
+    if (cudaGetDevice(&ctx->device) != cudaSuccess) return fail(BF_ERR_CUDA);
+
+    RingDev& R = ctx->ring.dev;
+    memset(&R, 0, sizeof(R));
+    R.N = N;
+    R.logN = ctx->logN;
+    R.r = n_ct_primes;
+    ctx->ring.geom = ntt_geometry(ctx->logN);
+    ctx->ring.q.assign(primes, primes + nb);
+    const u64 P = primes[n_ct_primes];
+    std::vector<ulonglong2> twf((size_t)nb * N), twi((size_t)nb * N);
+    for (u32 m = 0; m < nb; ++m) {
+        const u64 q = primes[m];
+        R.q[m] = q;
+        R.mu[m] = (u64)((((u128)1) << 64) / q);
+        R.c64[m] = (u64)((((u128)1) << 64) % q);
+        R.c64s[m] = h_shoup(R.c64[m], q);
+        R.ninv[m] = h_invmod(N % q, q);
+        R.ninvs[m] = h_shoup(R.ninv[m], q);
+        if (m < n_ct_primes) {
+            R.pmod[m] = P % q;
+            R.pinv[m] = h_invmod(P % q, q);
+            R.pinvs[m] = h_shoup(R.pinv[m], q);
+        }
+        const u64 psi = h_root_2n(q, N);
+        if (!psi) return fail(BF_ERR_BAD_PRIME);
+        const u64 psi_inv = h_invmod(psi, q);
+        std::vector<u64> pw(N), pwi(N);
+        pw[0] = 1;
+        pwi[0] = 1;
+        for (u32 k = 1; k < N; ++k) {
+            pw[k] = h_mulmod(pw[k - 1], psi, q);
+            pwi[k] = h_mulmod(pwi[k - 1], psi_inv, q);
+        }
+        for (u32 k = 0; k < N; ++k) {
+            const u32 e = h_brev(k, (int)ctx->logN);
+            twf[(size_t)m * N + k] = make_ulonglong2(pw[e], h_shoup(pw[e], q));
+            twi[(size_t)m * N + k] = make_ulonglong2(pwi[e], h_shoup(pwi[e], q));
+        }
+    }
+    // encoder tables: twiddles from the host's libm so that results do not depend on the device's
+    // own sine and cosine
+    const int logn = (int)ctx->logN - 1;
+    std::vector<u32> sop(n);
+    {
+        u64 pw5 = 1;
+        for (u32 s = 0; s < n; ++s) {
+            const u32 idx = (u32)((pw5 - 1) / 4);
+            sop[h_brev(idx, logn)] = s;
+            pw5 = (pw5 * 5) % (2ull * N);
+        }
+    }
+    std::vector<double2> T(n / 2), Z(n);
+    {
+        const double PI = 3.14159265358979323846264338327950288;
+        const double two_pi_over_n = (2.0 * PI) / (double)n;
+        const double pi_over_N = PI / (double)N;
+        for (u32 t = 0; t < n / 2; ++t) {
+            const double ang = (double)t * two_pi_over_n;
+            T[t] = make_double2(cos(ang), -sin(ang));
+        }
+        for (u32 k = 0; k < n; ++k) {
+            const double ang = (double)k * pi_over_N;
+            Z[k] = make_double2(cos(ang), -sin(ang));
+        }
+    }
+#define CKC(call)                                                        \
+    do {                                                                 \
+        cudaError_t e__ = (call);                                        \
+        if (e__ != cudaSuccess) {                                        \
+            status = (e__ == cudaErrorMemoryAllocation) ? BF_ERR_OOM : BF_ERR_CUDA; \
+            cudaGetLastError();                                          \
+            return fail(status);                                         \
+        }                                                                \
+    } while (0)
+    CKC(cudaMalloc(&ctx->tw_fwd, twf.size() * sizeof(ulonglong2)));
+    CKC(cudaMalloc(&ctx->tw_inv, twi.size() * sizeof(ulonglong2)));
+    CKC(cudaMalloc(&ctx->slot_of_pos, sop.size() * sizeof(u32)));
+    CKC(cudaMalloc(&ctx->T, T.size() * sizeof(double2)));
+    CKC(cudaMalloc(&ctx->Z, Z.size() * sizeof(double2)));
+    CKC(cudaMalloc(&ctx->overflow_flag, sizeof(int)));
+    CKC(cudaMemcpy(ctx->tw_fwd, twf.data(), twf.size() * sizeof(ulonglong2), cudaMemcpyHostToDevice));
+    CKC(cudaMemcpy(ctx->tw_inv, twi.data(), twi.size() * sizeof(ulonglong2), cudaMemcpyHostToDevice));
+    CKC(cudaMemcpy(ctx->slot_of_pos, sop.data(), sop.size() * sizeof(u32), cudaMemcpyHostToDevice));
+    CKC(cudaMemcpy(ctx->T, T.data(), T.size() * sizeof(double2), cudaMemcpyHostToDevice));
+    CKC(cudaMemcpy(ctx->Z, Z.data(), Z.size() * sizeof(double2), cudaMemcpyHostToDevice));
+    CKC(cudaMemset(ctx->overflow_flag, 0, sizeof(int)));
+    CKC(cudaDeviceSynchronize());
+#undef CKC
+    R.tw_fwd = ctx->tw_fwd;
+    R.tw_inv = ctx->tw_inv;
+    *out = ctx;
+    return BF_OK;
+}
+
+static void free_buf(DevBuf& b) {
+    if (b.p) cudaFree(b.p);
+    b.p = nullptr;
+    b.cap = 0;
+}
+
+extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
+    if (!ctx) return;
+    cudaDeviceSynchronize();
+    for (bf_weights* w : ctx->weights) {
+        if (w) {
+            cudaFree(w->pt);
+            delete w;
+        }
+    }
+    DevBuf* bufs[] = {&ctx->X, &ctx->Dig, &ctx->U, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres, &ctx->Y,
+                      &ctx->fft, &ctx->coef, &ctx->ptjit, &ctx->stage_in, &ctx->stage_out, &ctx->nm_a, &ctx->nm_b};
+    for (DevBuf* b : bufs) free_buf(*b);
+    cudaFree(ctx->tw_fwd);
+    cudaFree(ctx->tw_inv);
+    cudaFree(ctx->slot_of_pos);
+    cudaFree(ctx->T);
+    cudaFree(ctx->Z);
+    cudaFree(ctx->overflow_flag);
+    cudaFree(ctx->keys);
+    cudaFree(ctx->perms);
+    for (cudaEvent_t& e : ctx->ev)
+        if (e) cudaEventDestroy(e);
+    cudaGetLastError();
+    delete ctx;
+}
+
+// ------------------------------------------------------------------------------------------------
+extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_t n_keys, const uint64_t* keys) {
+    if (!ctx || (n_keys && (!rot_steps || !keys))) return BF_ERR_INVALID_ARG;
+    const u32 N = ctx->N, r = ctx->r, nb = r + 1, n = N / 2;
+    CK(cudaStreamSynchronize(ctx->stream));
+    cudaFree(ctx->keys);
+    cudaFree(ctx->perms);
+    ctx->keys = nullptr;
+    ctx->perms = nullptr;
+    ctx->key_of_steps.clear();
+    ctx->n_keys = 0;
+    if (n_keys == 0) return BF_OK;
+    const size_t key_words = (size_t)r * 2 * nb * N;
+    cudaError_t e = cudaMalloc(&ctx->keys, key_words * n_keys * sizeof(u64));
+    if (e != cudaSuccess) { cudaGetLastError(); ctx->keys = nullptr; return BF_ERR_OOM; }
+    e = cudaMalloc(&ctx->perms, (size_t)n_keys * N * sizeof(u32));
+    if (e != cudaSuccess) { cudaGetLastError(); ctx->perms = nullptr; return BF_ERR_OOM; }
+    // permutation tables: position i of the transform holds the evaluation at psi^(2*brev(i)+1);
+    // a(X) -> a(X^g) maps it to the evaluation at exponent (2*brev(i)+1)*g mod 2N
+    std::vector<u32> perms((size_t)n_keys * N);
+    for (u32 t = 0; t < n_keys; ++t) {
+        const u32 steps = rot_steps[t] % n;
+        u64 g = 1;
+        for (u32 s = 0; s < steps; ++s) g = (g * 5) % (2ull * N);
+        for (u32 i = 0; i < N; ++i) {
+            const u64 ex = ((2ull * h_brev(i, (int)ctx->logN) + 1) * g) % (2ull * N);
+            perms[(size_t)t * N + i] = h_brev((u32)((ex - 1) / 2), (int)ctx->logN);
+        }
+        ctx->key_of_steps[steps] = (int)t;
+    }
+    CK(cudaMemcpy(ctx->perms, perms.data(), perms.size() * sizeof(u32), cudaMemcpyHostToDevice));
+    PolyBatch B;
+    memset(&B, 0, sizeof(B));
+    B.src = keys;
+    B.dst = ctx->keys;
+    B.src_so = B.dst_so = (long long)nb * N;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = nb;
+    B.mod0 = 0;
+    B.mod_step = 1;
+    CK(ntt_forward(ctx->ring, B, n_keys * r * 2, LOAD_REDUCE, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    ctx->n_keys = n_keys;
+    return BF_OK;
+}
+
+extern "C" int bf_set_cache_budget(bf_ctx* ctx, uint64_t bytes) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    ctx->cache_budget = bytes;
+    return BF_OK;
+}
+
+extern "C" uint64_t bf_cache_bytes_used(const bf_ctx* ctx) { return ctx ? ctx->cache_used : 0; }
+
+static u32 cdiv(u32 a, u32 b) { return (a + b - 1) / b; }
+
+extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
+    if (!ctx) return 0;
+    const u64 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = cdiv(d_out, ctx->plan.tile_D);
+    const u64 M = ctx->plan.tile_D / ctx->plan.tau;
+    return n_in * n_out * M * ctx->r * ctx->N * sizeof(u64);
+}
+
+// Encode diagonals [d0, d0 + count) of W (order [j][p][q][k]) into dst (NTT domain, [count][r][N]).
+static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0, u32 count, u64* dst) {
+    const u32 N = ctx->N, r = ctx->r, n = N / 2;
+    const u32 chunk = 64;
+    TRY(ensure(ctx, ctx->fft, (size_t)chunk * n * sizeof(double2)));
+    TRY(ensure(ctx, ctx->coef, (size_t)chunk * N * sizeof(i64)));
+    EncodeTables tab;
+    tab.slot_of_pos = ctx->slot_of_pos;
+    tab.T = ctx->T;
+    tab.Z = ctx->Z;
+    tab.scale_over_n = ctx->scale / (double)n;
+    for (u32 lo = 0; lo < count; lo += chunk) {
+        const u32 cnt = (count - lo < chunk) ? count - lo : chunk;
+        DiagBatch db;
+        db.W = W;
+        db.d_out = d_out;
+        db.d_in = d_in;
+        db.n_in = cdiv(d_in, ctx->plan.tile_D);
+        db.n_out = cdiv(d_out, ctx->plan.tile_D);
+        db.D = ctx->plan.tile_D;
+        db.tau = ctx->plan.tau;
+        db.b = ctx->plan.bsgs_b;
+        db.g = ctx->plan.bsgs_g;
+        db.d0 = d0 + lo;
+        db.count = cnt;
+        CK(launch_encode(ctx->ring, tab, db, (double2*)ctx->fft.p, (i64*)ctx->coef.p, ctx->overflow_flag, ctx->stream));
+        PolyBatch B;
+        memset(&B, 0, sizeof(B));
+        B.src = ctx->coef.p;
+        B.dst = dst + (size_t)lo * r * N;
+        B.src_so = N;
+        B.src_sm = 0;
+        B.dst_so = (long long)r * N;
+        B.dst_sm = N;
+        B.n_m = r;
+        B.mod0 = 0;
+        B.mod_step = 1;
+        CK(ntt_forward(ctx->ring, B, cnt, LOAD_I64, ctx->stream));
+    }
+    return BF_OK;
+}
+
+static int check_overflow(bf_ctx* ctx) {
+    int flag = 0;
+    CK(cudaMemcpyAsync(&flag, ctx->overflow_flag, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    if (flag) {
+        CK(cudaMemsetAsync(ctx->overflow_flag, 0, sizeof(int), ctx->stream));
+        return BF_ERR_RANGE;
+    }
+    return BF_OK;
+}
+
+extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, uint32_t d_in, bf_weights** out) {
+    if (!ctx || !W || !out || !d_out || !d_in) return BF_ERR_INVALID_ARG;
+    *out = nullptr;
+    const u64 bytes = bf_weights_bytes(ctx, d_out, d_in);
+    if (ctx->cache_budget && ctx->cache_used + bytes > ctx->cache_budget) return BF_ERR_OOM;
+    bf_weights* w = new (std::nothrow) bf_weights();
+    if (!w) return BF_ERR_OOM;
+    w->d_out = d_out;
+    w->d_in = d_in;
+    w->n_in = cdiv(d_in, ctx->plan.tile_D);
+    w->n_out = cdiv(d_out, ctx->plan.tile_D);
+    w->bytes = bytes;
+    cudaError_t e = cudaMalloc(&w->pt, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        delete w;
+        return BF_ERR_OOM;
+    }
+    const u32 n_diag = w->n_in * w->n_out * (ctx->plan.tile_D / ctx->plan.tau);
+    int s = encode_range(ctx, W, d_out, d_in, 0, n_diag, w->pt);
+    if (s == BF_OK) s = check_overflow(ctx);
+    if (s != BF_OK) {
+        cudaStreamSynchronize(ctx->stream);
+        cudaFree(w->pt);
+        delete w;
+        return s;
+    }
+    ctx->cache_used += bytes;
+    ctx->weights.push_back(w);
+    *out = w;
+    return BF_OK;
+}
+
+extern "C" void bf_weights_free(bf_ctx* ctx, bf_weights* w) {
+    if (!ctx || !w) return;
+    for (size_t i = 0; i < ctx->weights.size(); ++i) {
+        if (ctx->weights[i] == w) {
+            cudaStreamSynchronize(ctx->stream);
+            cudaFree(w->pt);
+            ctx->cache_used -= w->bytes;
+            delete w;
+            ctx->weights.erase(ctx->weights.begin() + i);
+            return;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Division by the special prime and assembly of rotated ciphertexts for the rotations listed in rb
+// (their inner products already sit in U): inverse transform of the P-residues, centred lift into
+// every q_i with a forward transform, then (u - t) * P^{-1} plus the permuted c0.
+static int moddown_batch(bf_ctx* ctx, const RotBatch& rb, const u64* c0_base, long long c0_stride, u64* out_base,
+                         long long out_stride) {
+    const u32 N = ctx->N, r = ctx->r, nb = r + 1;
+    PolyBatch B;
+    memset(&B, 0, sizeof(B));
+    B.src = (const u64*)ctx->U.p + (size_t)r * N;       // the P-residue of each (rotation, component)
+    B.dst = (u64*)ctx->Tc.p;
+    B.src_so = (long long)nb * N;
+    B.dst_so = N;
+    B.n_m = 1;
+    B.mod0 = r;
+    B.mod_step = 0;
+    CK(ntt_inverse(ctx->ring, B, (u32)rb.n * 2, ctx->stream));
+    memset(&B, 0, sizeof(B));
+    B.src = ctx->Tc.p;
+    B.dst = (u64*)ctx->Tn.p;
+    B.src_so = N;
+    B.src_sm = 0;
+    B.dst_so = (long long)r * N;
+    B.dst_sm = N;
+    B.n_m = r;
+    B.mod0 = 0;
+    B.mod_step = 1;
+    B.lift_mod = ctx->ring.q[r];
+    CK(ntt_forward(ctx->ring, B, (u32)rb.n * 2, LOAD_CENTRED, ctx->stream));
+    CK(launch_moddown_finish(ctx->ring, rb, (const u64*)ctx->U.p, (const u64*)ctx->Tn.p, c0_base, c0_stride,
+                             ctx->perms, out_base, out_stride, ctx->stream));
+    return BF_OK;
+}
+
+static int ensure_rot_scratch(bf_ctx* ctx, u32 n_dig_sets, u32 n_rot) {
+    const size_t N = ctx->N, r = ctx->r, nb = r + 1;
+    TRY(ensure(ctx, ctx->Dig, (size_t)n_dig_sets * r * nb * N * 8));
+    TRY(ensure(ctx, ctx->U, (size_t)n_rot * 2 * nb * N * 8));
+    TRY(ensure(ctx, ctx->Tc, (size_t)n_rot * 2 * N * 8));
+    TRY(ensure(ctx, ctx->Tn, (size_t)n_rot * 2 * r * N * 8));
+    return BF_OK;
+}
+
+static int find_key(bf_ctx* ctx, u32 steps, int* key) {
+    auto it = ctx->key_of_steps.find(steps % (ctx->N / 2));
+    if (it == ctx->key_of_steps.end()) return BF_ERR_MISSING_KEY;
+    *key = it->second;
+    return BF_OK;
+}
+
+// Digits of c1 (coefficient domain, [r][N] with stride N) reduced into every prime of the extended
+// basis and transformed: dig[set][j][m] = NTT_m( c1_j mod m ).
+static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_sets, u64* dig) {
+    const u32 N = ctx->N, r = ctx->r, nb = r + 1;
+    PolyBatch B;
+    memset(&B, 0, sizeof(B));
+    B.n_m = nb;
+    B.mod0 = 0;
+    B.mod_step = 1;
+    B.src_sm = 0;
+    B.dst_sm = N;
+    B.dst_so = (long long)nb * N;
+    if (set_stride == (long long)r * N || n_sets == 1) {
+        B.src = c1_coeff;
+        B.dst = dig;
+        B.src_so = N;
+        CK(ntt_forward(ctx->ring, B, n_sets * r, LOAD_REDUCE, ctx->stream));
+    } else {
+        for (u32 s = 0; s < n_sets; ++s) {
+            B.src = c1_coeff + (size_t)s * set_stride;
+            B.dst = dig + (size_t)s * r * nb * N;
+            B.src_so = N;
+            CK(ntt_forward(ctx->ring, B, r, LOAD_REDUCE, ctx->stream));
+        }
+    }
+    return BF_OK;
+}
+
+static void stamp(bf_ctx* ctx, int i) {
+    if (ctx->timing && ctx->ev[i]) cudaEventRecord(ctx->ev[i], ctx->stream);
+}
+
+static u32 giant_batch(const bf_ctx* ctx) {
+    // rotations per giant-step launch: keep the digit sets of one batch near the L2 capacity
+    const size_t per_rot = (size_t)ctx->r * (ctx->r + 1) * ctx->N * 8;
+    size_t nrot = ((size_t)96 << 20) / per_rot;
+    if (nrot < 1) nrot = 1;
+    if (nrot > (size_t)MAX_ROT_BATCH) nrot = MAX_ROT_BATCH;
+    return (u32)nrot;
+}
+
+extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
+                         const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out) {
+    if (!ctx || !ct_in || !ct_out || (!pt_weights && !W_raw) || !d_out || !d_in) return BF_ERR_INVALID_ARG;
+    const u32 N = ctx->N, r = ctx->r, nb = r + 1;
+    const u32 D = ctx->plan.tile_D, tau = ctx->plan.tau, b = ctx->plan.bsgs_b, g = ctx->plan.bsgs_g;
+    if (n_in != cdiv(d_in, D) || n_out != cdiv(d_out, D)) return BF_ERR_SHAPE;
+    if (pt_weights && (pt_weights->d_out != d_out || pt_weights->d_in != d_in)) return BF_ERR_SHAPE;
+    const size_t ctw = (size_t)2 * r * N;                 // words per ciphertext
+    // rotation keys the plan needs
+    std::vector<int> baby_key(b, -1), giant_key(g, -1);
+    for (u32 k = 1; k < b; ++k) TRY(find_key(ctx, k * tau, &baby_key[k]));
+    for (u32 j = 1; j < g; ++j) TRY(find_key(ctx, j * b * tau, &giant_key[j]));
+
+    const u32 gb = giant_batch(ctx);
+    const u32 n_giant = (g - 1) * n_out;
+    u32 n_dig_sets = n_giant < gb ? n_giant : gb;       // digit sets alive at once
+    if (n_dig_sets < 1) n_dig_sets = 1;
+    u32 rot_cap = b - 1 > n_dig_sets ? b - 1 : n_dig_sets;
+    if (rot_cap < 1) rot_cap = 1;
+    TRY(ensure(ctx, ctx->X, (size_t)n_in * b * ctw * 8));
+    TRY(ensure(ctx, ctx->A, (size_t)n_out * g * ctw * 8));
+    TRY(ensure(ctx, ctx->Rres, (size_t)(n_giant ? n_giant : 1) * ctw * 8));
+    TRY(ensure(ctx, ctx->Y, (size_t)n_out * ctw * 8));
+    TRY(ensure(ctx, ctx->Cc, (size_t)n_dig_sets * r * N * 8));
+    TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_cap));
+    u64* X = (u64*)ctx->X.p;
+    u64* A = (u64*)ctx->A.p;
+    u64* Rres = (u64*)ctx->Rres.p;
+    u64* Y = (u64*)ctx->Y.p;
+    u64* Dig = (u64*)ctx->Dig.p;
+    u64* U = (u64*)ctx->U.p;
+    u64* Cc = (u64*)ctx->Cc.p;
+    if (ctx->timing) {
+        for (cudaEvent_t& e : ctx->ev)
+            if (!e) CK(cudaEventCreate(&e));
+        ctx->ev_valid = true;
+    }
+    stamp(ctx, 0);
+
+    // ---- ingest, hoisted ModUp and baby steps, one input ciphertext at a time
+    PolyBatch B;
+    for (u32 q = 0; q < n_in; ++q) {
+        const u64* ct = ct_in + (size_t)q * ctw;
+        u64* X0 = X + (size_t)q * b * ctw;               // X[q][0] = NTT(ct_q)
+        memset(&B, 0, sizeof(B));
+        B.src = ct;
+        B.dst = X0;
+        B.src_so = B.dst_so = (long long)r * N;
+        B.src_sm = B.dst_sm = N;
+        B.n_m = r;
+        B.mod0 = 0;
+        B.mod_step = 1;
+        CK(ntt_forward(ctx->ring, B, 2, LOAD_PLAIN, ctx->stream));
+        if (b > 1) {
+            TRY(modup(ctx, ct + (size_t)r * N, (long long)r * N, 1, Dig));
+            RotBatch rb;
+            memset(&rb, 0, sizeof(rb));
+            rb.n = (int)(b - 1);
+            for (u32 k = 1; k < b; ++k) {
+                rb.key[k - 1] = baby_key[k];
+                rb.dig[k - 1] = 0;
+                rb.c0[k - 1] = (int)(q * b);
+                rb.out[k - 1] = (int)(q * b + k);
+            }
+            CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, ctx->perms, U, ctx->stream));
+            TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
+        }
+    }
+    stamp(ctx, 1);
+
+    // ---- multiply-accumulate over the encoded diagonals
+    const u32 n_terms = n_in * b, n_pj = n_out * g;
+    if (pt_weights) {
+        CK(launch_mac(ctx->ring, pt_weights->pt, X, A, n_pj, n_terms, ctx->stream));
+    } else {
+        // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them
+        const size_t group_bytes = (size_t)n_terms * r * N * 8;
+        u32 groups = (u32)(((size_t)1 << 30) / group_bytes);
+        if (groups < 1) groups = 1;
+        if (groups > n_pj) groups = n_pj;
+        TRY(ensure(ctx, ctx->ptjit, group_bytes * groups));
+        for (u32 pj0 = 0; pj0 < n_pj; pj0 += groups) {
+            const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
+            TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p));
+            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, X, A + (size_t)pj0 * ctw, cnt, n_terms, ctx->stream));
+        }
+    }
+    stamp(ctx, 2);
+
+    // ---- giant steps: rotate A[j][p] by j*b*tau (full key switch each), then sum over j
+    for (u32 rho0 = 0; rho0 < n_giant; rho0 += gb) {
+        const u32 cnt = (n_giant - rho0 < gb) ? n_giant - rho0 : gb;
+        const u64* Asrc = A + (size_t)(n_out + rho0) * ctw;      // ciphertexts with j >= 1 are contiguous
+        memset(&B, 0, sizeof(B));
+        B.src = Asrc + (size_t)r * N;                            // c1 of each
+        B.dst = Cc;
+        B.src_so = (long long)ctw;
+        B.src_sm = N;
+        B.dst_so = (long long)r * N;
+        B.dst_sm = N;
+        B.n_m = r;
+        B.mod0 = 0;
+        B.mod_step = 1;
+        CK(ntt_inverse(ctx->ring, B, cnt, ctx->stream));
+        TRY(modup(ctx, Cc, (long long)r * N, cnt, Dig));
+        RotBatch rb;
+        memset(&rb, 0, sizeof(rb));
+        rb.n = (int)cnt;
+        for (u32 t = 0; t < cnt; ++t) {
+            const u32 j = (rho0 + t) / n_out + 1;
+            rb.key[t] = giant_key[j];
+            rb.dig[t] = (int)t;
+            rb.c0[t] = (int)t;
+            rb.out[t] = (int)t;
+        }
+        CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, ctx->perms, U, ctx->stream));
+        TRY(moddown_batch(ctx, rb, Asrc, (long long)ctw, Rres + (size_t)rho0 * ctw, (long long)ctw));
+    }
+    const u64* Yfinal = A;
+    if (g > 1) {
+        CK(launch_giant_sum(ctx->ring, A, Rres, Y, n_out, g, ctx->stream));
+        Yfinal = Y;
+    }
+    stamp(ctx, 3);
+
+    // ---- back to the coefficient domain
+    memset(&B, 0, sizeof(B));
+    B.src = Yfinal;
+    B.dst = ct_out;
+    B.src_so = B.dst_so = (long long)r * N;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = r;
+    B.mod0 = 0;
+    B.mod_step = 1;
+    CK(ntt_inverse(ctx->ring, B, n_out * 2, ctx->stream));
+    stamp(ctx, 4);
+    if (!pt_weights) TRY(check_overflow(ctx));
+    (void)nb;
+    return BF_OK;
+}
+
+extern "C" int bf_rescale(bf_ctx* ctx, const uint64_t* ct_in, uint64_t* ct_out, uint32_t n_ct, uint32_t level,
+                          double* scale_inout) {
+    if (!ctx || !ct_in || !ct_out || !n_ct) return BF_ERR_INVALID_ARG;
+    if (level < 2 || level > ctx->r) return BF_ERR_LEVEL;
+    const u64 qL = ctx->ring.q[level - 1];
+    u64 inv[MAX_MODULI], invs[MAX_MODULI], qlmod[MAX_MODULI];
+    for (u32 i = 0; i + 1 < level; ++i) {
+        const u64 q = ctx->ring.q[i];
+        inv[i] = h_invmod(qL % q, q);
+        invs[i] = h_shoup(inv[i], q);
+        qlmod[i] = qL % q;
+    }
+    if (ct_in == ct_out && n_ct > 1) {
+        // packed output of ciphertext t overlaps the input of ciphertext t-1 only: in-order launches
+        for (u32 t = 0; t < n_ct; ++t)
+            CK(launch_rescale(ctx->ring, ct_in + (size_t)t * 2 * level * ctx->N,
+                              ct_out + (size_t)t * 2 * (level - 1) * ctx->N, 1, level, inv, invs, qlmod, ctx->stream));
+    } else {
+        CK(launch_rescale(ctx->ring, ct_in, ct_out, n_ct, level, inv, invs, qlmod, ctx->stream));
+    }
+    if (scale_inout) *scale_inout /= (double)qL;
+    return BF_OK;
+}
+
+extern "C" int bf_linear_host(bf_ctx* ctx, const uint64_t* host_ct_in, uint32_t n_in, const bf_weights* pt_weights,
+                              const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* host_ct_out,
+                              uint32_t n_out) {
+    if (!ctx || !host_ct_in || !host_ct_out) return BF_ERR_INVALID_ARG;
+    const size_t ctw = (size_t)2 * ctx->r * ctx->N;
+    TRY(ensure(ctx, ctx->stage_in, (size_t)n_in * ctw * 8));
+    TRY(ensure(ctx, ctx->stage_out, (size_t)n_out * ctw * 8));
+    CK(cudaMemcpyAsync(ctx->stage_in.p, host_ct_in, (size_t)n_in * ctw * 8, cudaMemcpyHostToDevice, ctx->stream));
+    TRY(bf_linear(ctx, (const u64*)ctx->stage_in.p, n_in, pt_weights, W_raw, d_out, d_in, (u64*)ctx->stage_out.p, n_out));
+    TRY(bf_rescale(ctx, (const u64*)ctx->stage_out.p, (u64*)ctx->stage_out.p, n_out, ctx->r, nullptr));
+    const size_t out_bytes = (size_t)n_out * 2 * (ctx->r - 1) * ctx->N * 8;
+    CK(cudaMemcpyAsync(host_ct_out, ctx->stage_out.p, out_bytes, cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    return BF_OK;
+}
+
+extern "C" int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uint64_t* ct_out) {
+    if (!ctx || !ct_in || !ct_out) return BF_ERR_INVALID_ARG;
+    const u32 N = ctx->N, r = ctx->r;
+    const size_t ctw = (size_t)2 * r * N;
+    int key = -1;
+    TRY(find_key(ctx, steps, &key));
+    TRY(ensure(ctx, ctx->X, 2 * ctw * 8));
+    TRY(ensure_rot_scratch(ctx, 1, 1));
+    u64* X = (u64*)ctx->X.p;
+    PolyBatch B;
+    memset(&B, 0, sizeof(B));
+    B.src = ct_in;
+    B.dst = X;
+    B.src_so = B.dst_so = (long long)r * N;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = r;
+    B.mod_step = 1;
+    CK(ntt_forward(ctx->ring, B, 2, LOAD_PLAIN, ctx->stream));
+    TRY(modup(ctx, ct_in + (size_t)r * N, (long long)r * N, 1, (u64*)ctx->Dig.p));
+    RotBatch rb;
+    memset(&rb, 0, sizeof(rb));
+    rb.n = 1;
+    rb.key[0] = key;
+    rb.out[0] = 1;
+    CK(launch_key_inner_product(ctx->ring, rb, (const u64*)ctx->Dig.p, ctx->keys, ctx->perms, (u64*)ctx->U.p, ctx->stream));
+    TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
+    memset(&B, 0, sizeof(B));
+    B.src = X + ctw;
+    B.dst = ct_out;
+    B.src_so = B.dst_so = (long long)r * N;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = r;
+    B.mod_step = 1;
+    CK(ntt_inverse(ctx->ring, B, 2, ctx->stream));
+    return BF_OK;
+}
+
+extern "C" int bf_negacyclic_mul(bf_ctx* ctx, const uint64_t* a, const uint64_t* b, uint64_t* out, uint32_t n_polys) {
+    if (!ctx || !a || !b || !out || !n_polys) return BF_ERR_INVALID_ARG;
+    const u32 N = ctx->N, nb = ctx->r + 1;
+    const u32 n_outer = cdiv(n_polys, nb);
+    // polynomial t uses basis prime t mod (r+1): pad the batch to whole groups of r+1
+    TRY(ensure(ctx, ctx->nm_a, (size_t)n_outer * nb * N * 8));
+    TRY(ensure(ctx, ctx->nm_b, (size_t)n_outer * nb * N * 8));
+    CK(cudaMemsetAsync(ctx->nm_a.p, 0, (size_t)n_outer * nb * N * 8, ctx->stream));
+    CK(cudaMemsetAsync(ctx->nm_b.p, 0, (size_t)n_outer * nb * N * 8, ctx->stream));
+    CK(cudaMemcpyAsync(ctx->nm_a.p, a, (size_t)n_polys * N * 8, cudaMemcpyDeviceToDevice, ctx->stream));
+    CK(cudaMemcpyAsync(ctx->nm_b.p, b, (size_t)n_polys * N * 8, cudaMemcpyDeviceToDevice, ctx->stream));
+    PolyBatch B;
+    memset(&B, 0, sizeof(B));
+    B.src_so = B.dst_so = (long long)nb * N;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = nb;
+    B.mod_step = 1;
+    B.src = ctx->nm_a.p;
+    B.dst = (u64*)ctx->nm_a.p;
+    CK(ntt_forward(ctx->ring, B, n_outer, LOAD_PLAIN, ctx->stream));
+    B.src = ctx->nm_b.p;
+    B.dst = (u64*)ctx->nm_b.p;
+    CK(ntt_forward(ctx->ring, B, n_outer, LOAD_PLAIN, ctx->stream));
+    CK(launch_pointwise_mul(ctx->ring, (const u64*)ctx->nm_a.p, (const u64*)ctx->nm_b.p, (u64*)ctx->nm_a.p,
+                            n_outer * nb, nb, 0, ctx->stream));
+    B.src = ctx->nm_a.p;
+    B.dst = (u64*)ctx->nm_a.p;
+    CK(ntt_inverse(ctx->ring, B, n_outer, ctx->stream));
+    CK(cudaMemcpyAsync(out, ctx->nm_a.p, (size_t)n_polys * N * 8, cudaMemcpyDeviceToDevice, ctx->stream));
+    return BF_OK;
+}
+
+extern "C" int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, uint32_t q, uint32_t j, uint32_t k,
+                                 uint64_t* out) {
+    if (!ctx || !w || !out) return BF_ERR_INVALID_ARG;
+    if (p >= w->n_out || q >= w->n_in || j >= ctx->plan.bsgs_g || k >= ctx->plan.bsgs_b) return BF_ERR_SHAPE;
+    const u32 N = ctx->N, r = ctx->r;
+    const size_t d = (((size_t)j * w->n_out + p) * w->n_in + q) * ctx->plan.bsgs_b + k;
+    PolyBatch B;
+    memset(&B, 0, sizeof(B));
+    B.src = w->pt + d * r * N;
+    B.dst = out;
+    B.src_so = B.dst_so = (long long)r * N;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = r;
+    B.mod_step = 1;
+    CK(ntt_inverse(ctx->ring, B, 1, ctx->stream));
+    return BF_OK;
+}
+
+extern "C" int bf_set_stage_timing(bf_ctx* ctx, int on) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    ctx->timing = on ? 1 : 0;
+    if (!on) ctx->ev_valid = false;
+    return BF_OK;
+}
+
+extern "C" int bf_get_stage_ms(bf_ctx* ctx, float* ms_out) {
+    if (!ctx || !ms_out) return BF_ERR_INVALID_ARG;
+    if (!ctx->ev_valid) return BF_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(ctx->stream));
+    for (int i = 0; i < 4; ++i) CK(cudaEventElapsedTime(&ms_out[i], ctx->ev[i], ctx->ev[i + 1]));
+    return BF_OK;
+}

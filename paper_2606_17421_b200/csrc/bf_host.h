@@ -1,0 +1,73 @@
+// Host-side structures and kernel launchers shared by the translation units of libbifrost.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <map>
+#include <vector>
+
+#include "bf_common.cuh"
+
+namespace bf {
+
+struct NttGeometry {
+    int log_r, log_c;                 // N = 2^log_r rows x 2^log_c columns
+    int strided_lanes, strided_threads;
+    int contig_lanes, contig_threads, contig_pad;
+};
+
+struct RingHost {
+    RingDev dev;
+    NttGeometry geom;
+    std::vector<u64> q;               // q_0..q_L, then P
+};
+
+// ---- ntt.cu
+NttGeometry ntt_geometry(u32 logN);
+cudaError_t ntt_forward(const RingHost& ring, const PolyBatch& B, u32 n_outer, int load, cudaStream_t stream);
+cudaError_t ntt_inverse(const RingHost& ring, const PolyBatch& B, u32 n_outer, cudaStream_t stream);
+
+// ---- kernels.cu : element-wise and streaming kernels of the linear layer
+struct RotBatch {                     // one key-switch launch over n rotations
+    int n;
+    int key[MAX_ROT_BATCH];           // index of the rotation key (and of its permutation table)
+    int dig[MAX_ROT_BATCH];           // which digit set the rotation reads
+    int c0[MAX_ROT_BATCH];            // which ciphertext supplies the c0 that is permuted and added
+    int out[MAX_ROT_BATCH];           // which output ciphertext slot receives the result
+};
+
+// out[t] = a[t] * b[t] pointwise, polynomial t modulo basis prime mod0 + t % n_m
+cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* b, u64* out, u32 n_polys, u32 n_m,
+                                 u32 mod0, cudaStream_t stream);
+// u[rot][comp][m][n] = sum_j dig[dig(rot)][j][m][perm[key(rot)][n]] * key[key(rot)][j][comp][m][n]
+cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys,
+                                     const u32* perms, u64* u, cudaStream_t stream);
+// out[out(rot)][comp][i][n] = (u[rot][comp][i][n] - tn[rot][comp][i][n]) * P^{-1}
+//                             + (comp == 0 ? c0[c0(rot)][0][i][perm[n]] : 0)
+cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, const u64* u, const u64* tn,
+                                  const u64* c0_base, long long c0_stride, const u32* perms, u64* out_base,
+                                  long long out_stride, cudaStream_t stream);
+// A[pj][comp][i][n] = sum_{t < n_terms} Pt[pj][t][i][n] * X[t][comp][i][n],  pj = j*n_out + p, t = q*b + k
+cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
+                       cudaStream_t stream);
+// y[p] = a[p] + sum_{j=1}^{g-1} rres[(j-1)*n_out + p]   (ciphertexts of [2][r][N] words)
+cudaError_t launch_giant_sum(const RingHost& ring, const u64* a, const u64* rres, u64* y, u32 n_out, u32 g,
+                             cudaStream_t stream);
+cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
+                           const u64* invs, const u64* qlmod, cudaStream_t stream);
+
+// ---- encode.cu : canonical-embedding encoder (fp64) for weight diagonals
+struct EncodeTables {
+    const u32* slot_of_pos;           // [n] slot index whose value sits at FFT input position a
+    const double2* T;                 // [n/2] (cos, -sin)(2 pi t / n)
+    const double2* Z;                 // [n]   (cos, -sin)(pi k / N)
+    double scale_over_n;
+};
+struct DiagBatch {                    // diagonals d0 .. d0+count-1 in [j][p][q][k] order
+    const float* W;
+    u32 d_out, d_in, n_in, n_out, D, tau, b, g;
+    u32 d0, count;
+};
+cudaError_t launch_encode(const RingHost& ring, const EncodeTables& tab, const DiagBatch& db, double2* fft_scratch,
+                          i64* coeff_out, int* overflow_flag, cudaStream_t stream);
+
+}  // namespace bf

@@ -1,0 +1,198 @@
+// CKKS weight encoding on the device (Sec. 4.2: weight-matrix diagonals are pre-encoded into
+// resident BSGS objects, or encoded per call on the fallback path).
+//
+// For every generalised diagonal of a tile the kernels build the slot vector straight from the
+// fp32 weight matrix, apply the inverse canonical embedding as an n-point complex FFT in fp64
+// (n = N/2), multiply by the twist exp(-i pi k / N) and by scale/n, and round to 64-bit integer
+// coefficients.  The per-prime reduction and the forward NTT happen in the NTT's load stage.
+//
+// The floating-point arithmetic is a fixed DAG so that results are reproducible bit for bit:
+// radix-2 decimation-in-time butterflies (a, b) -> (a + w b, a - w b) over a bit-reversed input,
+// the complex product formed as (br wr - bi wi, br wi + bi wr) with each product and each sum
+// rounded on its own (the _rn intrinsics are never contracted into fused multiply-adds), twiddles
+// taken from host-computed tables, and round-to-nearest-even at the end.  Register blocking only
+// regroups butterflies; it does not change any operand.
+#include "bf_host.h"
+
+namespace bf {
+
+struct FftCfg {
+    int log_len, lanes, n_groups, K[4], log_other, first, pad;
+};
+
+__device__ __forceinline__ double2 cmul_rn(double2 b, double2 w) {
+    double2 t;
+    t.x = __dsub_rn(__dmul_rn(b.x, w.x), __dmul_rn(b.y, w.y));
+    t.y = __dadd_rn(__dmul_rn(b.x, w.y), __dmul_rn(b.y, w.x));
+    return t;
+}
+
+// Slot value of plaintext Pt[p][q][j][k] at slot s: generalised diagonal i = j*b + k of tile (p, q),
+// pre-rotated right by j*b*tau.  Slot s' = (rho*D + kappa)*tau + c holds
+// W[p*D + kappa][q*D + ((kappa + i + c*M) mod D)], zero outside the matrix.
+__device__ __forceinline__ double diag_value(const DiagBatch& db, u32 dd, u32 s, u32 n) {
+    const u32 k = dd % db.b;
+    const u32 q = (dd / db.b) % db.n_in;
+    const u32 p = (dd / (db.b * db.n_in)) % db.n_out;
+    const u32 j = dd / (db.b * db.n_in * db.n_out);
+    const u32 sp = (s - j * db.b * db.tau) & (n - 1);
+    const u32 c = sp % db.tau;
+    const u32 kappa = (sp / db.tau) % db.D;
+    const u32 M = db.D / db.tau;
+    const u32 row = p * db.D + kappa;
+    const u32 col = q * db.D + ((kappa + j * db.b + k + c * M) % db.D);
+    if (row >= db.d_out || col >= db.d_in) return 0.0;
+    return (double)__ldg(&db.W[(size_t)row * db.d_in + col]);
+}
+
+// One pass of the batched FFT.  CONTIG = the first pass (chunks of adjacent points, small butterfly
+// distances, reads the weights); otherwise the strided second pass, which also applies twist,
+// scale and rounding.
+template <bool CONTIG>
+__global__ void __launch_bounds__(256) encode_fft_pass(const EncodeTables tab, const DiagBatch db, const FftCfg cfg,
+                                                       u32 logn, double2* __restrict__ scratch,
+                                                       i64* __restrict__ coeff, int* __restrict__ overflow) {
+    extern __shared__ double2 smc[];
+    const u32 n = 1u << logn;
+    const u32 diag = blockIdx.y;
+    double2* buf = scratch + (size_t)diag * n;
+    const int LEN = 1 << cfg.log_len;
+    const int lanes = cfg.lanes;
+    const int lane0 = blockIdx.x * lanes;
+    const int other = 1 << cfg.log_other;
+    const int pitch = LEN + cfg.pad;
+    const int unit = CONTIG ? 1 : other;              // global index distance of one local index step
+
+    int step = 1;
+    for (int gi = 0; gi < cfg.n_groups; ++gi) {
+        const int K = cfg.K[cfg.n_groups - 1 - gi];   // smallest distances first
+        const int t0 = step << (K - 1);
+        const int nsets = (LEN * lanes) >> K;
+        const int sets_per_lane = LEN >> K;
+        const bool g_first = (gi == 0), g_last = (gi == cfg.n_groups - 1);
+        for (int w = threadIdx.x; w < nsets; w += blockDim.x) {
+            int lane, u;
+            if (CONTIG) { u = w % sets_per_lane; lane = w / sets_per_lane; }
+            else { lane = w % lanes; u = w / lanes; }
+            const int blk = u / step, off = u % step;
+            const int base = blk * 2 * t0 + off;
+            double2 e[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (i < (1 << K)) {
+                    const int li = base + i * step;
+                    if (g_first) {
+                        const u32 gidx = CONTIG ? (u32)(lane0 + lane) * LEN + li : (u32)li * other + lane0 + lane;
+                        if (CONTIG) {
+                            e[i].x = diag_value(db, db.d0 + diag, __ldg(&tab.slot_of_pos[gidx]), n);
+                            e[i].y = 0.0;
+                        } else {
+                            e[i] = buf[gidx];
+                        }
+                    } else {
+                        e[i] = CONTIG ? smc[lane * pitch + li] : smc[li * lanes + lane];
+                    }
+                }
+            }
+            // stages with set-local distance d = 1, 2, 4 (times `step` in local index units)
+#pragma unroll
+            for (int s = 0; s < 3; ++s) {
+                if (s < K) {
+                    const int d = 1 << s;
+                    const u32 half_local = (u32)d * step;                  // butterfly distance, local units
+                    const u32 tw_stride = n / (2u * half_local * unit);    // n / len
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (i < (1 << K) && ((i & d) == 0)) {
+                            const u32 li = base + i * step;
+                            const u32 jj = (li % half_local) * unit + (CONTIG ? 0u : (u32)(lane0 + lane));
+                            const double2 wv = __ldg(&tab.T[(size_t)jj * tw_stride]);
+                            const double2 t = cmul_rn(e[i + d], wv);
+                            const double2 a = e[i];
+                            e[i].x = __dadd_rn(a.x, t.x);
+                            e[i].y = __dadd_rn(a.y, t.y);
+                            e[i + d].x = __dsub_rn(a.x, t.x);
+                            e[i + d].y = __dsub_rn(a.y, t.y);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (i < (1 << K)) {
+                    const int li = base + i * step;
+                    if (g_last) {
+                        const u32 gidx = CONTIG ? (u32)(lane0 + lane) * LEN + li : (u32)li * other + lane0 + lane;
+                        if (CONTIG) {
+                            buf[gidx] = e[i];
+                        } else {
+                            // twist by exp(-i pi k / N), scale by Delta / n, round to nearest even
+                            const double2 uu = cmul_rn(e[i], __ldg(&tab.Z[gidx]));
+                            const double cr = rint(__dmul_rn(uu.x, tab.scale_over_n));
+                            const double ci = rint(__dmul_rn(uu.y, tab.scale_over_n));
+                            const double lim = 4611686018427387904.0;      // 2^62
+                            if (!(fabs(cr) < lim) || !(fabs(ci) < lim)) {
+                                atomicExch(overflow, 1);
+                            } else {
+                                i64* cp = coeff + (size_t)diag * 2 * n;
+                                cp[gidx] = (i64)cr;
+                                cp[gidx + n] = (i64)ci;
+                            }
+                        }
+                    } else {
+                        if (CONTIG) smc[lane * pitch + li] = e[i];
+                        else smc[li * lanes + lane] = e[i];
+                    }
+                }
+            }
+        }
+        if (!g_last) __syncthreads();
+        step <<= K;
+    }
+}
+
+static void fft_groups(int s, int* K, int* n) {
+    static const int table[9][4] = {{0, 0, 0, 0}, {1, 0, 0, 0}, {2, 0, 0, 0}, {3, 0, 0, 0}, {2, 2, 0, 0},
+                                    {3, 2, 0, 0}, {3, 3, 0, 0}, {3, 2, 2, 0}, {3, 3, 2, 0}};
+    *n = 0;
+    for (int i = 0; i < 4; ++i) {
+        K[i] = table[s][i];
+        if (K[i]) (*n)++;
+    }
+}
+
+cudaError_t launch_encode(const RingHost& ring, const EncodeTables& tab, const DiagBatch& db, double2* fft_scratch,
+                          i64* coeff_out, int* overflow_flag, cudaStream_t stream) {
+    if (db.count == 0) return cudaSuccess;
+    const u32 logn = ring.dev.logN - 1;
+    const int log_a = 8;                        // first pass: chunks of 256 points
+    const int log_b = (int)logn - log_a;        // second pass: 2^log_b rows
+    FftCfg ca, cb;
+    ca.log_len = log_a; ca.log_other = log_b; ca.lanes = 8; ca.first = 1; ca.pad = 1;
+    fft_groups(ca.log_len, ca.K, &ca.n_groups);
+    cb.log_len = log_b; cb.log_other = log_a; cb.first = 0; cb.pad = 0;
+    int tc = 2048 / (1 << log_b);
+    if (tc < 16) tc = 16;
+    if (tc > 256) tc = 256;
+    cb.lanes = tc;
+    fft_groups(cb.log_len, cb.K, &cb.n_groups);
+    {
+        dim3 grid((1u << ca.log_other) / ca.lanes, db.count);
+        if ((1u << ca.log_other) < (u32)ca.lanes) { ca.lanes = 1 << ca.log_other; grid.x = 1; }
+        const size_t smem = (size_t)((1 << ca.log_len) + ca.pad) * ca.lanes * sizeof(double2);
+        encode_fft_pass<true><<<grid, 256, smem, stream>>>(tab, db, ca, logn, fft_scratch, coeff_out, overflow_flag);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    {
+        dim3 grid((1u << cb.log_other) / cb.lanes, db.count);
+        const size_t smem = (size_t)(1 << cb.log_len) * cb.lanes * sizeof(double2);
+        int threads = ((1 << cb.log_len) * cb.lanes) / 8;
+        if (threads < 32) threads = 32;
+        if (threads > 256) threads = 256;
+        encode_fft_pass<false><<<grid, threads, smem, stream>>>(tab, db, cb, logn, fft_scratch, coeff_out, overflow_flag);
+        return cudaGetLastError();
+    }
+}
+
+}  // namespace bf

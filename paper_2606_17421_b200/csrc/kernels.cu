@@ -1,0 +1,221 @@
+// Streaming and element-wise kernels of the encrypted linear layer: the ciphertext x plaintext
+// multiply-accumulate that streams encoded weight diagonals from HBM (the "ciphertext-plaintext
+// multiplication with pre-encoded weight diagonals" of Sec. 3.5 / Sec. 4.2), the key-switch inner
+// product, the division by the special prime, the giant-step sum and the rescale (Sec. 2.1).
+#include "bf_host.h"
+
+namespace bf {
+
+// ------------------------------------------------------------------------------------------------
+// Pointwise product of NTT-domain polynomials (parity helper for the transform).
+__global__ void pointwise_mul_kernel(const RingDev R, const u64* __restrict__ a, const u64* __restrict__ b,
+                                     u64* __restrict__ out, u32 n_m, u32 mod0) {
+    const u32 poly = blockIdx.y;
+    const u32 mod = mod0 + poly % n_m;
+    const size_t idx = (size_t)poly * R.N + blockIdx.x * blockDim.x + threadIdx.x;
+    u64 hi = 0, lo = 0;
+    mac128(hi, lo, a[idx], b[idx]);
+    out[idx] = reduce128(hi, lo, R.q[mod], R.mu[mod], R.c64[mod], R.c64s[mod]);
+}
+
+cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* b, u64* out, u32 n_polys, u32 n_m,
+                                 u32 mod0, cudaStream_t stream) {
+    if (n_polys == 0) return cudaSuccess;
+    dim3 grid(ring.dev.N / 256, n_polys);
+    pointwise_mul_kernel<<<grid, 256, 0, stream>>>(ring.dev, a, b, out, n_m, mod0);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Multiply-accumulate over encoded diagonals.
+//   A[pj][comp][i][n] = sum_{t < n_terms} Pt[pj][t][i][n] * X[t][comp][i][n]   (mod q_i)
+// Every plaintext word is read from HBM exactly once with 128-bit loads; the two ciphertext
+// components share it.  Products accumulate lazily in 128 bits; one reduction per output word.
+constexpr int MAC_THREADS = 256;
+constexpr int MAC_LAZY_TERMS = 128;   // 128 * (2^60)^2 < 2^128
+
+__global__ void __launch_bounds__(MAC_THREADS) mac_kernel(const RingDev R, const u64* __restrict__ pt,
+                                                          const u64* __restrict__ x, u64* __restrict__ a,
+                                                          u32 n_terms) {
+    const u32 i = blockIdx.y, pj = blockIdx.z;
+    const u32 N = R.N, r = R.r;
+    const u32 n = (blockIdx.x * MAC_THREADS + threadIdx.x) * 2;
+    const u64 q = R.q[i], mu = R.mu[i], c64 = R.c64[i], c64s = R.c64s[i];
+    const u64* ptp = pt + ((size_t)pj * n_terms * r + i) * N + n;
+    const u64* xp = x + (size_t)i * N + n;
+    const size_t pt_stride = (size_t)r * N, x_stride = (size_t)2 * r * N, comp_stride = (size_t)r * N;
+    u64 h00 = 0, l00 = 0, h01 = 0, l01 = 0, h10 = 0, l10 = 0, h11 = 0, l11 = 0;   // [comp][word]
+    for (u32 t0 = 0; t0 < n_terms; t0 += MAC_LAZY_TERMS) {
+        const u32 t1 = min(n_terms, t0 + MAC_LAZY_TERMS);
+#pragma unroll 4
+        for (u32 t = t0; t < t1; ++t) {
+            const ulonglong2 w = __ldcs((const ulonglong2*)(ptp + t * pt_stride));     // streamed once
+            const ulonglong2 x0 = __ldg((const ulonglong2*)(xp + t * x_stride));
+            const ulonglong2 x1 = __ldg((const ulonglong2*)(xp + t * x_stride + comp_stride));
+            mac128(h00, l00, w.x, x0.x);
+            mac128(h01, l01, w.y, x0.y);
+            mac128(h10, l10, w.x, x1.x);
+            mac128(h11, l11, w.y, x1.y);
+        }
+        if (t1 < n_terms) {   // keep the running sums below 2^64 before the next lazy stretch
+            l00 = reduce128(h00, l00, q, mu, c64, c64s); h00 = 0;
+            l01 = reduce128(h01, l01, q, mu, c64, c64s); h01 = 0;
+            l10 = reduce128(h10, l10, q, mu, c64, c64s); h10 = 0;
+            l11 = reduce128(h11, l11, q, mu, c64, c64s); h11 = 0;
+        }
+    }
+    u64* ap = a + ((size_t)pj * 2 * r + i) * N + n;
+    ulonglong2 o0, o1;
+    o0.x = reduce128(h00, l00, q, mu, c64, c64s);
+    o0.y = reduce128(h01, l01, q, mu, c64, c64s);
+    o1.x = reduce128(h10, l10, q, mu, c64, c64s);
+    o1.y = reduce128(h11, l11, q, mu, c64, c64s);
+    *(ulonglong2*)ap = o0;
+    *(ulonglong2*)(ap + comp_stride) = o1;
+}
+
+cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
+                       cudaStream_t stream) {
+    if (n_pj == 0) return cudaSuccess;
+    dim3 grid(ring.dev.N / (2 * MAC_THREADS), ring.dev.r, n_pj);
+    mac_kernel<<<grid, MAC_THREADS, 0, stream>>>(ring.dev, pt, x, a, n_terms);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Key-switch inner product over the extended basis, with the automorphism applied as a gather on
+// the digits:  u[rot][comp][m][n] = sum_j dig[.][j][m][perm[n]] * key[.][j][comp][m][n].
+__global__ void __launch_bounds__(256) key_inner_product_kernel(const RingDev R, const RotBatch rb,
+                                                                const u64* __restrict__ dig,
+                                                                const u64* __restrict__ keys,
+                                                                const u32* __restrict__ perms, u64* __restrict__ u) {
+    const u32 m = blockIdx.y, rot = blockIdx.z;
+    const u32 N = R.N, r = R.r, nb = r + 1;
+    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
+    const u32 key = rb.key[rot];
+    const u32 pn = perms[(size_t)key * N + n];
+    const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + pn;
+    const u64* kp = keys + ((size_t)key * r * 2 * nb + m) * N + n;
+    u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
+    for (u32 j = 0; j < r; ++j) {
+        const u64 d = dp[(size_t)j * nb * N];
+        const u64 k0 = __ldcs(kp + (size_t)(j * 2) * nb * N);
+        const u64 k1 = __ldcs(kp + (size_t)(j * 2 + 1) * nb * N);
+        mac128(h0, l0, d, k0);
+        mac128(h1, l1, d, k1);
+    }
+    const u64 q = R.q[m], mu = R.mu[m], c64 = R.c64[m], c64s = R.c64s[m];
+    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n;
+    up[0] = reduce128(h0, l0, q, mu, c64, c64s);
+    up[(size_t)nb * N] = reduce128(h1, l1, q, mu, c64, c64s);
+}
+
+cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys,
+                                     const u32* perms, u64* u, cudaStream_t stream) {
+    if (rb.n == 0) return cudaSuccess;
+    dim3 grid(ring.dev.N / 256, ring.dev.r + 1, rb.n);
+    key_inner_product_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, perms, u);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Last step of the division by P:  v = (u - NTT(centred lift of the P-residue)) * P^{-1} mod q_i,
+// plus the automorphism of c0 for component 0.
+__global__ void __launch_bounds__(256) moddown_finish_kernel(const RingDev R, const RotBatch rb,
+                                                             const u64* __restrict__ u, const u64* __restrict__ tn,
+                                                             const u64* __restrict__ c0_base, long long c0_stride,
+                                                             const u32* __restrict__ perms, u64* __restrict__ out_base,
+                                                             long long out_stride) {
+    const u32 i = blockIdx.y % R.r, comp = blockIdx.y / R.r, rot = blockIdx.z;
+    const u32 N = R.N, r = R.r, nb = r + 1;
+    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
+    const u64 q = R.q[i];
+    const u64 uv = u[(((size_t)rot * 2 + comp) * nb + i) * N + n];
+    const u64 tv = tn[(((size_t)rot * 2 + comp) * r + i) * N + n];
+    u64 v = mul_shoup(sub_mod(uv, tv, q), R.pinv[i], R.pinvs[i], q);
+    if (comp == 0) {
+        const u32 pn = perms[(size_t)rb.key[rot] * N + n];
+        v = add_mod(v, c0_base[(size_t)rb.c0[rot] * c0_stride + (size_t)i * N + pn], q);
+    }
+    out_base[(size_t)rb.out[rot] * out_stride + ((size_t)comp * r + i) * N + n] = v;
+}
+
+cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, const u64* u, const u64* tn,
+                                  const u64* c0_base, long long c0_stride, const u32* perms, u64* out_base,
+                                  long long out_stride, cudaStream_t stream) {
+    if (rb.n == 0) return cudaSuccess;
+    dim3 grid(ring.dev.N / 256, 2 * ring.dev.r, rb.n);
+    moddown_finish_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, u, tn, c0_base, c0_stride, perms, out_base,
+                                                    out_stride);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Y[p] = A[0][p] + sum_{j >= 1} (rotated A[j][p]);  a holds the j = 0 block, rres[(j-1)*n_out + p] the rest
+__global__ void __launch_bounds__(256) giant_sum_kernel(const RingDev R, const u64* __restrict__ a,
+                                                        const u64* __restrict__ rres, u64* __restrict__ y, u32 g) {
+    const u32 ci = blockIdx.y, p = blockIdx.z, n_out = gridDim.z;   // ci = comp * r + i
+    const u32 N = R.N, r = R.r;
+    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
+    const u64 q = R.q[ci % r];
+    const size_t ct = (size_t)2 * r * N;
+    u64 v = a[(size_t)p * ct + (size_t)ci * N + n];
+    for (u32 j = 1; j < g; ++j) v = add_mod(v, rres[((size_t)(j - 1) * n_out + p) * ct + (size_t)ci * N + n], q);
+    y[(size_t)p * ct + (size_t)ci * N + n] = v;
+}
+
+cudaError_t launch_giant_sum(const RingHost& ring, const u64* a, const u64* rres, u64* y, u32 n_out, u32 g,
+                             cudaStream_t stream) {
+    if (n_out == 0) return cudaSuccess;
+    dim3 grid(ring.dev.N / 256, 2 * ring.dev.r, n_out);
+    giant_sum_kernel<<<grid, 256, 0, stream>>>(ring.dev, a, rres, y, g);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rescale (Sec. 2.1): drop the last prime q_L of a level-`level` ciphertext in coefficient form,
+//   c'_i = (c_i - centred(c_L)) * q_L^{-1} mod q_i.
+// Every address a thread touches is congruent to its coefficient index modulo N, and it reads all
+// residues of that coefficient before writing, so one ciphertext can be rescaled in place even
+// though the output is packed more tightly ([2][level-1][N]).
+struct RescaleConsts {
+    u64 inv[MAX_MODULI], invs[MAX_MODULI], qlmod[MAX_MODULI];
+};
+
+__global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const RescaleConsts rc,
+                                                      const u64* __restrict__ in, u64* __restrict__ out, u32 level) {
+    const u32 ct = blockIdx.y;
+    const u32 N = R.N;
+    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
+    const u64 qL = R.q[level - 1];
+    const u64* ip = in + (size_t)ct * 2 * level * N + n;
+    u64* op = out + (size_t)ct * 2 * (level - 1) * N + n;
+    u64 res[2][MAX_MODULI];
+#pragma unroll
+    for (int comp = 0; comp < 2; ++comp) {
+        const u64 t = ip[((size_t)comp * level + (level - 1)) * N];
+        const bool high = t > (qL - 1) / 2;
+        for (u32 i = 0; i + 1 < level; ++i) {
+            const u64 q = R.q[i];
+            u64 tq = barrett64(t, q, R.mu[i]);
+            if (high) tq = sub_mod(tq, rc.qlmod[i], q);
+            const u64 c = ip[((size_t)comp * level + i) * N];
+            res[comp][i] = mul_shoup(sub_mod(c, tq, q), rc.inv[i], rc.invs[i], q);
+        }
+    }
+#pragma unroll
+    for (int comp = 0; comp < 2; ++comp)
+        for (u32 i = 0; i + 1 < level; ++i) op[((size_t)comp * (level - 1) + i) * N] = res[comp][i];
+}
+
+cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
+                           const u64* invs, const u64* qlmod, cudaStream_t stream) {
+    if (n_ct == 0) return cudaSuccess;
+    RescaleConsts rc;
+    for (u32 i = 0; i + 1 < level; ++i) { rc.inv[i] = inv[i]; rc.invs[i] = invs[i]; rc.qlmod[i] = qlmod[i]; }
+    dim3 grid(ring.dev.N / 256, n_ct);
+    rescale_kernel<<<grid, 256, 0, stream>>>(ring.dev, rc, in, out, level);
+    return cudaGetLastError();
+}
+
+}  // namespace bf
