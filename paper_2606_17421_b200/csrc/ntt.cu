@@ -182,7 +182,7 @@ NttGeometry ntt_geometry(u32 logN) {
     if (tc > 256) tc = 256;
     g.strided_lanes = tc;
     g.strided_threads = (Rr * tc) / 8 < 32 ? 32 : (Rr * tc) / 8;
-    g.contig_lanes = 8;                       // 8 chunks of 256 points per block
+    g.contig_lanes = Rr < 8 ? Rr : 8;         // up to 8 chunks of 256 points per block
     g.contig_threads = 256;
     g.contig_pad = 8;
     return g;

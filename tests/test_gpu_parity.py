@@ -79,7 +79,7 @@ def test_encode_weights_matches_oracle(pkey, plan_t, shape):
 @pytest.mark.parametrize("pkey", ["n12", "n15"])
 def test_rotate_matches_oracle(pkey):
     par = oracle_params(pkey)
-    plan = ckks.Plan(64, 1, 4, 2) if pkey == "n12" else ckks.Plan(1024, 16, 2, 32)
+    plan = ckks.Plan(64, 1, 8, 8) if pkey == "n12" else ckks.Plan(1024, 16, 4, 16)
     s = ckks.keygen(par, 3)
     keys = ckks.make_rotation_keys(par, s, plan, 3)
     g = GpuSide(par, plan)
@@ -89,7 +89,7 @@ def test_rotate_matches_oracle(pkey):
         z = rng.normal(size=par.n)
         ct = ckks.encrypt(par, s, ckks.encode_coeffs(z, par.N, par.scale), 4)
         out = g.empty_u64(2, par.r, par.N)
-        for st in steps:
+        for st in steps[:4] + steps[-2:]:
             g.bf.bf_rotate(g.ctx, g.to_dev(ct), st, out)
             expect = ckks.rotate(par, ct, st, keys)
             got = g.to_host_u64(out)
