@@ -141,6 +141,22 @@ int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, uint32_t q, 
 int bf_set_stage_timing(bf_ctx* ctx, int on);
 int bf_get_stage_ms(bf_ctx* ctx, float* ms_out /* host, 4 values */);
 
+/* Launch accounting.  The library counts its kernel launches per category; with
+ * bf_set_kernel_timing(ctx, 1) it also brackets every launch with a pair of CUDA events on the
+ * context's stream.  bf_get_kernel_stats synchronises the stream, writes for every category the
+ * launches since the previous call (launches_out, host, bf_kernel_categories() values) and the
+ * summed event time in ms of the timed ones (ms_out, host), and resets both. */
+int bf_set_kernel_timing(bf_ctx* ctx, int on);
+int bf_kernel_categories(void);
+const char* bf_kernel_category_name(int cat);
+int bf_get_kernel_stats(bf_ctx* ctx, uint64_t* launches_out, float* ms_out);
+
+/* Measured rate, in operations per second over the whole GPU, of the 32x32+64-bit integer
+ * multiply-add (mad.wide.u32) that the 64-bit modular arithmetic of the transforms and the key
+ * switch decomposes into: the denominator for the integer-bound kernels' roofline.  Runs a short
+ * probe kernel (a few ms) on the context's stream and synchronises. */
+int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out);
+
 const char* bf_strerror(int code);
 const char* bf_last_cuda_error(const bf_ctx* ctx);
 

@@ -463,6 +463,27 @@ def encode_weights(params: Params, plan: Plan, W: np.ndarray, blocks=None) -> di
     return out
 
 
+def baby_rotations(params: Params, plan: Plan, ct: np.ndarray, keys: dict, ks=None) -> dict:
+    """X[k] = rot(ct, k*tau) for the requested baby steps k (all of 0..b-1 by default)."""
+    ks = range(plan.b) if ks is None else ks
+    return {k: rotate(params, ct, k * plan.tau, keys) for k in ks}
+
+
+def inner_sum(params: Params, plan: Plan, Xh: list, encoded: dict, p: int, j: int) -> np.ndarray:
+    """A[p][j] = sum_q sum_{k<b} Pt[p][q][j][k] (*) X[q][k], both components, every ciphertext
+    prime; Xh[q][k] are the baby-step ciphertexts in the evaluation domain.  Returns the
+    coefficient-domain ciphertext [2][r][N]."""
+    N, r, primes = params.N, params.r, params.primes
+    acc = np.zeros((2, r, N), dtype=np.uint64)
+    for q in range(len(Xh)):
+        pts = np.stack([encoded[(p, q, j, k)] for k in range(plan.b)])
+        pth = ntt(pts, primes * plan.b, params)
+        for k in range(plan.b):
+            for comp in range(2):
+                mul_acc(acc[comp], pth[k], Xh[q][k][comp], primes, N)
+    return intt(acc, primes * 2, params)
+
+
 def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blocks=None, encoded=None) -> dict:
     """Encrypted matrix-vector product (Sec. 4.2 "BSGS matrix-vector multiply"; Alg. 3 FHE_Linear).
 
@@ -478,20 +499,13 @@ def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blo
     if encoded is None:
         encoded = encode_weights(params, plan, W, blocks)
     # baby steps: X[q][k] = rot(ct_q, k*tau), then to the evaluation domain for the products
-    X = [[rotate(params, cts[q], k * plan.tau, keys) for k in range(plan.b)] for q in range(n_in)]
+    X = [baby_rotations(params, plan, cts[q], keys) for q in range(n_in)]
     Xh = [[ntt(X[q][k], primes * 2, params) for k in range(plan.b)] for q in range(n_in)]
     out = {}
     for p in blocks:
         Y = np.zeros((2, r, N), dtype=np.uint64)
         for j in range(plan.g):
-            acc = np.zeros((2, r, N), dtype=np.uint64)
-            for q in range(n_in):
-                pts = np.stack([encoded[(p, q, j, k)] for k in range(plan.b)])
-                pth = ntt(pts, primes * plan.b, params)
-                for k in range(plan.b):
-                    for comp in range(2):
-                        mul_acc(acc[comp], pth[k], Xh[q][k][comp], primes, N)
-            A = intt(acc, primes * 2, params)
+            A = inner_sum(params, plan, Xh, encoded, p, j)
             A = rotate(params, A, j * plan.b * plan.tau, keys)
             for comp in range(2):
                 for i, qi in enumerate(primes):

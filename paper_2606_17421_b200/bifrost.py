@@ -57,6 +57,11 @@ _SIGNATURES = {
     "bf_weights_export": (ctypes.c_int, [_vp, _vp, _u32, _u32, _u32, _u32, _vp]),
     "bf_set_stage_timing": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_get_stage_ms": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float)]),
+    "bf_set_kernel_timing": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "bf_kernel_categories": (ctypes.c_int, []),
+    "bf_kernel_category_name": (ctypes.c_char_p, [ctypes.c_int]),
+    "bf_get_kernel_stats": (ctypes.c_int, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(ctypes.c_float)]),
+    "bf_measure_imad_rate": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "bf_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "bf_last_cuda_error": (ctypes.c_char_p, [_vp]),
 }
@@ -184,3 +189,30 @@ def bf_get_stage_ms(ctx) -> list[float]:
     arr = (ctypes.c_float * 4)()
     _check(load().bf_get_stage_ms(ctx, arr), "bf_get_stage_ms", ctx)
     return list(arr)
+
+
+def bf_set_kernel_timing(ctx, on: bool):
+    _check(load().bf_set_kernel_timing(ctx, 1 if on else 0), "bf_set_kernel_timing", ctx)
+
+
+def bf_kernel_categories() -> int:
+    return load().bf_kernel_categories()
+
+
+def bf_kernel_category_name(cat: int) -> str:
+    return load().bf_kernel_category_name(cat).decode()
+
+
+def bf_get_kernel_stats(ctx) -> dict:
+    """{category name: (launches, summed event ms)} since the previous call."""
+    n = bf_kernel_categories()
+    launches = (_u64 * n)()
+    ms = (ctypes.c_float * n)()
+    _check(load().bf_get_kernel_stats(ctx, launches, ms), "bf_get_kernel_stats", ctx)
+    return {bf_kernel_category_name(c): (int(launches[c]), float(ms[c])) for c in range(n)}
+
+
+def bf_measure_imad_rate(ctx) -> float:
+    out = ctypes.c_double(0.0)
+    _check(load().bf_measure_imad_rate(ctx, ctypes.byref(out)), "bf_measure_imad_rate", ctx)
+    return out.value

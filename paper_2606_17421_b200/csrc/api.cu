@@ -82,6 +82,7 @@ struct bf_weights {
 
 struct bf_ctx {
     RingHost ring;
+    Profiler prof;
     u32 N, logN, r;
     double scale;
     bf_plan plan;
@@ -189,6 +190,7 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
     ctx->scale = scale;
     ctx->plan = *plan;
     ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->ring.prof = &ctx->prof;
     int status = BF_OK;
     auto fail = [&](int s) {
         bf_ctx_destroy(ctx);
@@ -317,6 +319,8 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
     cudaFree(ctx->perms);
     for (cudaEvent_t& e : ctx->ev)
         if (e) cudaEventDestroy(e);
+    for (auto& rec : ctx->prof.recs) { cudaEventDestroy(rec.a); cudaEventDestroy(rec.b); }
+    for (cudaEvent_t e : ctx->prof.pool) cudaEventDestroy(e);
     cudaGetLastError();
     delete ctx;
 }
@@ -855,5 +859,65 @@ extern "C" int bf_get_stage_ms(bf_ctx* ctx, float* ms_out) {
     if (!ctx->ev_valid) return BF_ERR_INVALID_ARG;
     CK(cudaStreamSynchronize(ctx->stream));
     for (int i = 0; i < 4; ++i) CK(cudaEventElapsedTime(&ms_out[i], ctx->ev[i], ctx->ev[i + 1]));
+    return BF_OK;
+}
+
+extern "C" int bf_set_kernel_timing(bf_ctx* ctx, int on) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    ctx->prof.timing = on != 0;
+    return BF_OK;
+}
+
+extern "C" int bf_kernel_categories(void) { return (int)CAT_COUNT; }
+
+extern "C" const char* bf_kernel_category_name(int cat) {
+    static const char* names[CAT_COUNT] = {"ntt_fwd_strided", "ntt_fwd_contig", "ntt_inv_contig", "ntt_inv_strided",
+                                           "key_inner_product", "moddown_finish", "mac", "giant_sum", "rescale",
+                                           "encode_fft_a", "encode_fft_b", "pointwise_mul"};
+    return (cat >= 0 && cat < (int)CAT_COUNT) ? names[cat] : "";
+}
+
+extern "C" int bf_get_kernel_stats(bf_ctx* ctx, uint64_t* launches_out, float* ms_out) {
+    if (!ctx || !launches_out || !ms_out) return BF_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(ctx->stream));
+    for (int c = 0; c < (int)CAT_COUNT; ++c) {
+        launches_out[c] = ctx->prof.launches[c];
+        ms_out[c] = 0.f;
+        ctx->prof.launches[c] = 0;
+    }
+    for (auto& rec : ctx->prof.recs) {
+        float ms = 0.f;
+        CK(cudaEventElapsedTime(&ms, rec.a, rec.b));
+        ms_out[rec.cat] += ms;
+        ctx->prof.pool.push_back(rec.a);
+        ctx->prof.pool.push_back(rec.b);
+    }
+    ctx->prof.recs.clear();
+    return BF_OK;
+}
+
+extern "C" int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out) {
+    if (!ctx || !mad_per_second_out) return BF_ERR_INVALID_ARG;
+    TRY(ensure(ctx, ctx->nm_a, 4096));
+    cudaDeviceProp prop;
+    CK(cudaGetDeviceProperties(&prop, ctx->device));
+    const u32 blocks = (u32)prop.multiProcessorCount * 8, iters = 4096;
+    cudaEvent_t a, b;
+    CK(cudaEventCreate(&a));
+    CK(cudaEventCreate(&b));
+    double best = 0.0;
+    for (int rep = 0; rep < 5; ++rep) {
+        CK(cudaEventRecord(a, ctx->stream));
+        CK(launch_imad_probe((u64*)ctx->nm_a.p, blocks, iters, ctx->stream));
+        CK(cudaEventRecord(b, ctx->stream));
+        CK(cudaEventSynchronize(b));
+        float ms = 0.f;
+        CK(cudaEventElapsedTime(&ms, a, b));
+        const double rate = (double)blocks * 256.0 * iters * 64.0 / (ms * 1e-3);
+        if (rep > 0 && rate > best) best = rate;
+    }
+    cudaEventDestroy(a);
+    cudaEventDestroy(b);
+    *mad_per_second_out = best;
     return BF_OK;
 }

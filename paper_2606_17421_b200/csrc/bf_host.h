@@ -15,10 +15,34 @@ struct NttGeometry {
     int contig_lanes, contig_threads, contig_pad;
 };
 
+// Kernel categories for launch counting and optional per-launch event timing.
+enum KernelCat : int {
+    CAT_NTT_FWD_STRIDED = 0, CAT_NTT_FWD_CONTIG, CAT_NTT_INV_CONTIG, CAT_NTT_INV_STRIDED,
+    CAT_KEY_INNER, CAT_MODDOWN_FINISH, CAT_MAC, CAT_GIANT_SUM, CAT_RESCALE,
+    CAT_ENCODE_FFT_A, CAT_ENCODE_FFT_B, CAT_POINTWISE, CAT_COUNT
+};
+
+struct Profiler {
+    bool timing = false;
+    uint64_t launches[CAT_COUNT] = {0};
+    struct Rec { int cat; cudaEvent_t a, b; };
+    std::vector<Rec> recs;            // event pairs recorded since the last collection
+    std::vector<cudaEvent_t> pool;    // idle events
+    cudaEvent_t get();
+};
+
+// Counts a launch and, when timing is on, brackets it with two events on the launch stream.
+struct ProfScope {
+    Profiler* p; int cat; cudaStream_t s; cudaEvent_t a = nullptr;
+    ProfScope(Profiler* prof, int c, cudaStream_t st);
+    ~ProfScope();
+};
+
 struct RingHost {
     RingDev dev;
     NttGeometry geom;
     std::vector<u64> q;               // q_0..q_L, then P
+    Profiler* prof = nullptr;
 };
 
 // ---- ntt.cu
@@ -54,6 +78,8 @@ cudaError_t launch_giant_sum(const RingHost& ring, const u64* a, const u64* rres
                              cudaStream_t stream);
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
                            const u64* invs, const u64* qlmod, cudaStream_t stream);
+
+cudaError_t launch_imad_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream);   // 64 mad.wide per iteration and thread
 
 // ---- encode.cu : canonical-embedding encoder (fp64) for weight diagonals
 struct EncodeTables {

@@ -180,6 +180,7 @@ cudaError_t launch_encode(const RingHost& ring, const EncodeTables& tab, const D
         dim3 grid((1u << ca.log_other) / ca.lanes, db.count);
         if ((1u << ca.log_other) < (u32)ca.lanes) { ca.lanes = 1 << ca.log_other; grid.x = 1; }
         const size_t smem = (size_t)((1 << ca.log_len) + ca.pad) * ca.lanes * sizeof(double2);
+        ProfScope prof(ring.prof, CAT_ENCODE_FFT_A, stream);
         encode_fft_pass<true><<<grid, 256, smem, stream>>>(tab, db, ca, logn, fft_scratch, coeff_out, overflow_flag);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -190,6 +191,7 @@ cudaError_t launch_encode(const RingHost& ring, const EncodeTables& tab, const D
         int threads = ((1 << cb.log_len) * cb.lanes) / 8;
         if (threads < 32) threads = 32;
         if (threads > 256) threads = 256;
+        ProfScope prof(ring.prof, CAT_ENCODE_FFT_B, stream);
         encode_fft_pass<false><<<grid, threads, smem, stream>>>(tab, db, cb, logn, fft_scratch, coeff_out, overflow_flag);
         return cudaGetLastError();
     }

@@ -22,6 +22,7 @@ cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* 
                                  u32 mod0, cudaStream_t stream) {
     if (n_polys == 0) return cudaSuccess;
     dim3 grid(ring.dev.N / 256, n_polys);
+    ProfScope prof(ring.prof, CAT_POINTWISE, stream);
     pointwise_mul_kernel<<<grid, 256, 0, stream>>>(ring.dev, a, b, out, n_m, mod0);
     return cudaGetLastError();
 }
@@ -78,6 +79,7 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a
                        cudaStream_t stream) {
     if (n_pj == 0) return cudaSuccess;
     dim3 grid(ring.dev.N / (2 * MAC_THREADS), ring.dev.r, n_pj);
+    ProfScope prof(ring.prof, CAT_MAC, stream);
     mac_kernel<<<grid, MAC_THREADS, 0, stream>>>(ring.dev, pt, x, a, n_terms);
     return cudaGetLastError();
 }
@@ -114,6 +116,7 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
                                      const u32* perms, u64* u, cudaStream_t stream) {
     if (rb.n == 0) return cudaSuccess;
     dim3 grid(ring.dev.N / 256, ring.dev.r + 1, rb.n);
+    ProfScope prof(ring.prof, CAT_KEY_INNER, stream);
     key_inner_product_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, perms, u);
     return cudaGetLastError();
 }
@@ -145,6 +148,7 @@ cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, cons
                                   long long out_stride, cudaStream_t stream) {
     if (rb.n == 0) return cudaSuccess;
     dim3 grid(ring.dev.N / 256, 2 * ring.dev.r, rb.n);
+    ProfScope prof(ring.prof, CAT_MODDOWN_FINISH, stream);
     moddown_finish_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, u, tn, c0_base, c0_stride, perms, out_base,
                                                     out_stride);
     return cudaGetLastError();
@@ -168,6 +172,7 @@ cudaError_t launch_giant_sum(const RingHost& ring, const u64* a, const u64* rres
                              cudaStream_t stream) {
     if (n_out == 0) return cudaSuccess;
     dim3 grid(ring.dev.N / 256, 2 * ring.dev.r, n_out);
+    ProfScope prof(ring.prof, CAT_GIANT_SUM, stream);
     giant_sum_kernel<<<grid, 256, 0, stream>>>(ring.dev, a, rres, y, g);
     return cudaGetLastError();
 }
@@ -214,7 +219,36 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
     RescaleConsts rc;
     for (u32 i = 0; i + 1 < level; ++i) { rc.inv[i] = inv[i]; rc.invs[i] = invs[i]; rc.qlmod[i] = qlmod[i]; }
     dim3 grid(ring.dev.N / 256, n_ct);
+    ProfScope prof(ring.prof, CAT_RESCALE, stream);
     rescale_kernel<<<grid, 256, 0, stream>>>(ring.dev, rc, in, out, level);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Throughput probe for the 32x32+64-bit integer multiply-add the modular arithmetic is made of:
+// every thread runs 8 independent mad.wide.u32 chains.  Gives the measured denominator for the
+// integer-bound kernels (NTT, key switch).
+__global__ void __launch_bounds__(256) imad_probe_kernel(u64* __restrict__ sink, u32 iters) {
+    u32 b = threadIdx.x * 2654435761u + blockIdx.x * 40503u + 12345u;
+    u64 c0 = b, c1 = b + 1, c2 = b + 2, c3 = b + 3, c4 = b + 4, c5 = b + 5, c6 = b + 6, c7 = b + 7;
+    for (u32 i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            asm volatile("mad.wide.u32 %0, %8, %9, %0;\n\tmad.wide.u32 %1, %8, %10, %1;\n\t"
+                         "mad.wide.u32 %2, %8, %11, %2;\n\tmad.wide.u32 %3, %8, %12, %3;\n\t"
+                         "mad.wide.u32 %4, %8, %13, %4;\n\tmad.wide.u32 %5, %8, %14, %5;\n\t"
+                         "mad.wide.u32 %6, %8, %15, %6;\n\tmad.wide.u32 %7, %8, %16, %7;"
+                         : "+l"(c0), "+l"(c1), "+l"(c2), "+l"(c3), "+l"(c4), "+l"(c5), "+l"(c6), "+l"(c7)
+                         : "r"(b), "r"((u32)c1), "r"((u32)c2), "r"((u32)c3), "r"((u32)c4), "r"((u32)c5),
+                           "r"((u32)c6), "r"((u32)c7), "r"((u32)c0));
+        }
+    }
+    u64 v = c0 ^ c1 ^ c2 ^ c3 ^ c4 ^ c5 ^ c6 ^ c7;
+    if (v == 0x1234567ull) sink[0] = v;      // practically never true; keeps the chains alive
+}
+
+cudaError_t launch_imad_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream) {
+    imad_probe_kernel<<<blocks, 256, 0, stream>>>(sink, iters);
     return cudaGetLastError();
 }
 

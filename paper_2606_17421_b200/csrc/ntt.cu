@@ -15,15 +15,32 @@
 
 namespace bf {
 
-struct PassCfg {
-    int log_len;        // log2 of the local transform length
-    int lanes;          // independent local transforms per block (columns, or chunks)
-    int n_groups;       // stage groups, in forward order (largest butterfly distance first)
-    int K[4];           // stages per group (2 or 3, or 1 for tiny lengths)
-    int log_other;      // log2(N / local length): rows for the contiguous pass, columns for the strided
-    int first;          // 1: this pass reads the batch source through the load functor; 0: in place on dst
-    int pad;            // shared-memory padding per lane in the contiguous pass
-};
+cudaEvent_t Profiler::get() {
+    if (!pool.empty()) {
+        cudaEvent_t e = pool.back();
+        pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+ProfScope::ProfScope(Profiler* prof, int c, cudaStream_t st) : p(prof), cat(c), s(st) {
+    if (!p) return;
+    p->launches[cat]++;
+    if (p->timing) {
+        a = p->get();
+        cudaEventRecord(a, s);
+    }
+}
+
+ProfScope::~ProfScope() {
+    if (!p || !a) return;
+    cudaEvent_t b = p->get();
+    cudaEventRecord(b, s);
+    p->recs.push_back({cat, a, b});
+}
 
 template <int LOAD>
 __device__ __forceinline__ u64 load_src(const void* src, size_t idx, u64 q, u64 mu, u64 lift_mod, u64 lift_red) {
@@ -42,9 +59,12 @@ __device__ __forceinline__ u64 load_src(const void* src, size_t idx, u64 q, u64 
     return m;
 }
 
+// Butterflies of one register-resident set of 2^K points over K consecutive stages.
+// tw_base = (blocks at the group's first forward stage) * mult, so that stage st, sub-block sub
+// uses twiddle (tw_base << st) + (blk << st) + sub.
 template <int K, bool FWD>
-__device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* __restrict__ tw,
-                                                u32 m0mult, u32 blk, u64 q) {
+__device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
+                                                u64 q) {
     const u64 q2 = 2 * q;
 #pragma unroll
     for (int s = 0; s < K; ++s) {
@@ -52,7 +72,7 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
         const int d = (1 << K) >> (st + 1);
 #pragma unroll
         for (int sub = 0; sub < (1 << st); ++sub) {
-            const ulonglong2 w = __ldg(&tw[(m0mult << st) + (blk << st) + sub]);
+            const ulonglong2 w = __ldg(&tw[(tw_base << st) + (blk << st) + sub]);
 #pragma unroll
             for (int off = 0; off < d; ++off) {
                 const int i = sub * 2 * d + off;
@@ -74,12 +94,43 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
     }
 }
 
-// One pass of a batched transform.  FWD/STRIDED pick the direction and which half this is:
-//   forward  = strided pass (first), then contiguous pass (in place)
-//   inverse  = contiguous pass (first), then strided pass (in place, scales by N^{-1})
-template <bool FWD, bool STRIDED, int LOAD>
-__global__ void __launch_bounds__(512) ntt_pass(const RingDev R, const PolyBatch B, const PassCfg cfg) {
-    extern __shared__ u64 sm[];
+// Stage groups of a local transform of 2^LOG_LEN points, in forward order.
+__host__ __device__ constexpr int n_groups(int log_len) { return log_len <= 3 ? 1 : (log_len <= 6 ? 2 : 3); }
+__host__ __device__ constexpr int group_k(int log_len, int gi) {
+    // 1:{1} 2:{2} 3:{3} 4:{2,2} 5:{3,2} 6:{3,3} 7:{3,2,2} 8:{3,3,2}
+    return log_len <= 3 ? log_len
+         : log_len == 4 ? 2
+         : log_len == 5 ? (gi == 0 ? 3 : 2)
+         : log_len == 6 ? 3
+         : log_len == 7 ? (gi == 0 ? 3 : 2)
+         : (gi == 2 ? 2 : 3);
+}
+// log2 of the point spacing of group gi's sets (forward order index)
+__host__ __device__ constexpr int group_log_step(int log_len, int gi) {
+    int done = 0;
+    for (int i = 0; i <= gi; ++i) done += group_k(log_len, i);
+    return log_len - done;
+}
+
+// Shared-memory index swizzle for a 256-point chunk of 64-bit words: makes the three access
+// patterns of the contiguous pass (spacing 32, spacing 4 and 4 adjacent points per thread) free of
+// bank conflicts without padding.
+__device__ __forceinline__ int swz(int i) { return i ^ ((i >> 4) & 3) ^ (((i >> 5) & 3) << 2); }
+
+constexpr int LOG_C = 8;              // contiguous pass: chunks of 256 points, one warp each
+constexpr int CHUNKS_PER_BLOCK = 8;
+
+// Strided pass: transforms the 2^LOG_R rows (stride 256) of 2^LOG_LANES adjacent columns.
+// Forward: first pass (reads the batch source through the load functor).  Inverse: second pass
+// (in place, scales by N^{-1}).
+template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
+__global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8),
+                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
+ntt_strided(const RingDev R, const PolyBatch B) {
+    constexpr int LEN = 1 << LOG_R, LANES = 1 << LOG_LANES;
+    constexpr int NT = (LEN * LANES / 8) < 32 ? 32 : (LEN * LANES / 8);
+    constexpr int NG = n_groups(LOG_R);
+    __shared__ u64 sm[LEN * LANES];
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
     const u32 mod = B.mod0 + m * B.mod_step;
@@ -88,144 +139,213 @@ __global__ void __launch_bounds__(512) ntt_pass(const RingDev R, const PolyBatch
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
     const char* src = (const char*)B.src + ((size_t)o * B.src_so + (size_t)m * B.src_sm) * 8;
     const u64 lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu) : 0;
-
-    const int LEN = 1 << cfg.log_len;
-    const int lanes = cfg.lanes;
-    const int lane0 = blockIdx.x * lanes;            // first column (strided) or first chunk (contiguous)
-    const int other = 1 << cfg.log_other;
-    const int pitch = LEN + cfg.pad;                 // contiguous pass: shared-memory pitch per chunk
-    const bool from_src = cfg.first != 0;
-    const bool last_pass = !from_src;
-
-    // Forward walks the groups from the largest butterfly distance down, inverse the other way.
-    int t0 = FWD ? (LEN >> 1) : 0;
-    int step_inv = 1;
-    for (int gi = 0; gi < cfg.n_groups; ++gi) {
-        const int K = FWD ? cfg.K[gi] : cfg.K[cfg.n_groups - 1 - gi];
-        if (!FWD) t0 = step_inv << (K - 1);
-        const int step = t0 >> (K - 1);              // spacing of a set's points
-        const int m0 = LEN / (2 * t0);               // blocks at the group's first forward stage
-        const int nsets = (LEN * lanes) >> K;
-        const int sets_per_lane = LEN >> K;
-        const bool g_first = (gi == 0), g_last = (gi == cfg.n_groups - 1);
-        for (int w = threadIdx.x; w < nsets; w += blockDim.x) {
-            int lane, u;
-            if (STRIDED) { lane = w % lanes; u = w / lanes; }
-            else { u = w % sets_per_lane; lane = w / sets_per_lane; }
-            const int blk = u / step, off = u % step;
+    const int col0 = blockIdx.x * LANES;
+    const int tid = threadIdx.x;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+        const int fg = FWD ? gi : NG - 1 - gi;                 // group index in forward order
+        const int K = group_k(LOG_R, fg);
+        const int log_step = group_log_step(LOG_R, fg);
+        const int step = 1 << log_step, t0 = step << (K - 1);
+        const int m0 = LEN / (2 * t0);
+        const int nsets = (LEN * LANES) >> K;
+        const bool g_first = (gi == 0), g_last = (gi == NG - 1);
+#pragma unroll
+        for (int w0 = 0; w0 < nsets; w0 += NT) {
+            const int w = w0 + tid;
+            if (NT > nsets && w >= nsets) break;
+            const int lane = w & (LANES - 1), u = w >> LOG_LANES;
+            const int blk = u >> log_step, off = u & (step - 1);
             const int base = blk * 2 * t0 + off;
-            const u32 mult = STRIDED ? 1u : (u32)(other + lane0 + lane);
             u64 e[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (i < (1 << K)) {
-                    const int li = base + i * step;
-                    if (g_first) {
-                        const size_t gidx = STRIDED ? ((size_t)li * other + lane0 + lane)
-                                                    : ((size_t)(lane0 + lane) * LEN + li);
-                        e[i] = from_src ? load_src<LOAD>(src, gidx, q, mu, B.lift_mod, lift_red) : dst[gidx];
-                    } else {
-                        e[i] = STRIDED ? sm[li * lanes + lane] : sm[lane * pitch + li];
-                    }
+            for (int i = 0; i < (1 << K); ++i) {
+                const int row = base + i * step;
+                if (g_first) {
+                    const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
+                    e[i] = FWD ? load_src<LOAD>(src, gidx, q, mu, B.lift_mod, lift_red) : dst[gidx];
+                } else {
+                    e[i] = sm[row * LANES + lane];
                 }
             }
-            if (K == 3) set_butterflies<3, FWD>(e, tw, (u32)m0 * mult, (u32)blk, q);
-            else if (K == 2) set_butterflies<2, FWD>(e, tw, (u32)m0 * mult, (u32)blk, q);
-            else set_butterflies<1, FWD>(e, tw, (u32)m0 * mult, (u32)blk, q);
+            if (K == 3) set_butterflies<3, FWD>(e, tw, (u32)m0, (u32)blk, q);
+            else if (K == 2) set_butterflies<2, FWD>(e, tw, (u32)m0, (u32)blk, q);
+            else set_butterflies<1, FWD>(e, tw, (u32)m0, (u32)blk, q);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (i < (1 << K)) {
-                    const int li = base + i * step;
-                    if (g_last) {
-                        const size_t gidx = STRIDED ? ((size_t)li * other + lane0 + lane)
-                                                    : ((size_t)(lane0 + lane) * LEN + li);
-                        u64 v = e[i];
-                        if (last_pass) {
-                            if (FWD) {                       // [0, 4q) -> [0, q)
-                                if (v >= 2 * q) v -= 2 * q;
-                                if (v >= q) v -= q;
-                            } else {                         // scale by N^{-1}, [0, 2q) -> [0, q)
-                                v = mul_shoup(v, R.ninv[mod], R.ninvs[mod], q);
-                            }
-                        }
-                        dst[gidx] = v;
-                    } else {
-                        if (STRIDED) sm[li * lanes + lane] = e[i];
-                        else sm[lane * pitch + li] = e[i];
-                    }
+            for (int i = 0; i < (1 << K); ++i) {
+                const int row = base + i * step;
+                if (g_last) {
+                    const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
+                    u64 v = e[i];
+                    if (!FWD) v = mul_shoup(v, R.ninv[mod], R.ninvs[mod], q);   // scale by N^{-1}, to [0, q)
+                    dst[gidx] = v;                                              // forward: lazy, below 4q
+                } else {
+                    sm[row * LANES + lane] = e[i];
                 }
             }
         }
         if (!g_last) __syncthreads();
-        if (FWD) t0 >>= K; else step_inv <<= K;
     }
 }
 
-static void stage_groups(int s, int* K, int* n) {
-    // Split s butterfly stages into register-resident groups of 3 or 2 (1 only when s == 1).
-    static const int table[9][4] = {{0, 0, 0, 0}, {1, 0, 0, 0}, {2, 0, 0, 0}, {3, 0, 0, 0}, {2, 2, 0, 0},
-                                    {3, 2, 0, 0}, {3, 3, 0, 0}, {3, 2, 2, 0}, {3, 3, 2, 0}};
-    *n = 0;
-    for (int i = 0; i < 4; ++i) {
-        K[i] = table[s][i];
-        if (K[i]) (*n)++;
+// Contiguous pass: every warp transforms one chunk of 256 adjacent points (8 per thread) through
+// the groups {3,3,2}; the chunk lives in the warp's own swizzled slice of shared memory between
+// groups, so only warp-level synchronisation is needed.
+// Forward: second pass (in place, final reduction to [0, q)).  Inverse: first pass (reads the batch
+// source, plain residues).
+template <bool FWD>
+__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const RingDev R, const PolyBatch B,
+                                                                       u32 chunks_per_block) {
+    constexpr int LEN = 1 << LOG_C;
+    __shared__ u64 sm_all[CHUNKS_PER_BLOCK * LEN];
+    const u32 poly = blockIdx.y;
+    const u32 o = poly / B.n_m, m = poly % B.n_m;
+    const u32 mod = B.mod0 + m * B.mod_step;
+    const u64 q = R.q[mod];
+    const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
+    u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
+    const u64* src = FWD ? dst : (const u64*)B.src + (size_t)o * B.src_so + (size_t)m * B.src_sm;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if ((u32)warp >= chunks_per_block) return;
+    const u32 chunk = blockIdx.x * chunks_per_block + warp;
+    const u32 mult = (R.N >> LOG_C) + chunk;                   // twiddle index multiplier of this chunk
+    u64* sm = sm_all + warp * LEN;
+    const u64* gsrc = src + (size_t)chunk * LEN;
+    u64* gdst = dst + (size_t)chunk * LEN;
+    u64 e[8];
+    if (FWD) {
+        // group 0: K = 3, spacing 32
+#pragma unroll
+        for (int i = 0; i < 8; ++i) e[i] = gsrc[lane + 32 * i];
+        set_butterflies<3, true>(e, tw, 1u * mult, 0u, q);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sm[swz(lane + 32 * i)] = e[i];
+        __syncwarp();
+        // group 1: K = 3, spacing 4
+        {
+            const int blk = lane >> 2, base = blk * 32 + (lane & 3);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
+            set_butterflies<3, true>(e, tw, 8u * mult, (u32)blk, q);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
+        }
+        __syncwarp();
+        // group 2: K = 2, adjacent points; two sets per thread
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+            const int s = lane + 32 * it;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) e[i] = sm[swz(4 * s + i)];
+            set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {   // final reduction [0, 4q) -> [0, q)
+                u64 v = e[i];
+                if (v >= 2 * q) v -= 2 * q;
+                if (v >= q) v -= q;
+                e[i] = v;
+            }
+            ulonglong2* gp = (ulonglong2*)(gdst + 4 * s);
+            gp[0] = make_ulonglong2(e[0], e[1]);
+            gp[1] = make_ulonglong2(e[2], e[3]);
+        }
+    } else {
+        // inverse: groups in the opposite order
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+            const int s = lane + 32 * it;
+            const ulonglong2* gp = (const ulonglong2*)(gsrc + 4 * s);
+            const ulonglong2 a = gp[0], b = gp[1];
+            e[0] = a.x; e[1] = a.y; e[2] = b.x; e[3] = b.y;
+            set_butterflies<2, false>(e, tw, 64u * mult, (u32)s, q);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) sm[swz(4 * s + i)] = e[i];
+        }
+        __syncwarp();
+        {
+            const int blk = lane >> 2, base = blk * 32 + (lane & 3);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
+            set_butterflies<3, false>(e, tw, 8u * mult, (u32)blk, q);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
+        }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) e[i] = sm[swz(lane + 32 * i)];
+        set_butterflies<3, false>(e, tw, 1u * mult, 0u, q);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) gdst[lane + 32 * i] = e[i];      // lazy, below 2q; the strided pass finishes
     }
 }
 
 NttGeometry ntt_geometry(u32 logN) {
     NttGeometry g;
-    g.log_c = 8;                              // contiguous pass: chunks of 256 points
-    g.log_r = (int)logN - g.log_c;            // strided pass: 4 .. 256 rows
-    const int Rr = 1 << g.log_r;
-    int tc = 2048 / Rr;
-    if (tc < 16) tc = 16;
-    if (tc > 256) tc = 256;
-    g.strided_lanes = tc;
-    g.strided_threads = (Rr * tc) / 8 < 32 ? 32 : (Rr * tc) / 8;
-    g.contig_lanes = Rr < 8 ? Rr : 8;         // up to 8 chunks of 256 points per block
-    g.contig_threads = 256;
-    g.contig_pad = 8;
+    g.log_c = LOG_C;
+    g.log_r = (int)logN - LOG_C;
+    // strided tile: 2048 points (256 threads) unless the row count forces otherwise
+    int log_lanes = 11 - g.log_r;
+    if (log_lanes < 4) log_lanes = 4;
+    if (log_lanes > 8) log_lanes = 8;
+    g.strided_lanes = 1 << log_lanes;
+    g.strided_threads = ((1 << g.log_r) * g.strided_lanes) / 8 < 32 ? 32 : ((1 << g.log_r) * g.strided_lanes) / 8;
+    g.contig_lanes = (1 << g.log_r) < CHUNKS_PER_BLOCK ? (1 << g.log_r) : CHUNKS_PER_BLOCK;
+    g.contig_threads = 32 * CHUNKS_PER_BLOCK;
+    g.contig_pad = 0;
     return g;
 }
 
-template <bool FWD, bool STRIDED>
-static cudaError_t launch_pass(const RingHost& ring, const PolyBatch& B, u32 n_polys, int load, bool first,
-                               cudaStream_t stream) {
-    const NttGeometry& g = ring.geom;
-    PassCfg cfg;
-    cfg.log_len = STRIDED ? g.log_r : g.log_c;
-    cfg.log_other = STRIDED ? g.log_c : g.log_r;
-    cfg.lanes = STRIDED ? g.strided_lanes : g.contig_lanes;
-    cfg.first = first ? 1 : 0;
-    cfg.pad = STRIDED ? 0 : g.contig_pad;
-    stage_groups(cfg.log_len, cfg.K, &cfg.n_groups);
-    const int threads = STRIDED ? g.strided_threads : g.contig_threads;
-    const int LEN = 1 << cfg.log_len;
-    const size_t smem = STRIDED ? (size_t)LEN * cfg.lanes * 8 : (size_t)(LEN + cfg.pad) * cfg.lanes * 8;
-    dim3 grid((1u << cfg.log_other) / cfg.lanes, n_polys);
+template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
+static void launch_strided_t(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream) {
+    constexpr int NT = ((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8);
+    dim3 grid((1u << LOG_C) >> LOG_LANES, n_polys);
+    ntt_strided<FWD, LOAD, LOG_R, LOG_LANES><<<grid, NT, 0, stream>>>(ring.dev, B);
+}
+
+template <bool FWD, int LOAD>
+static cudaError_t launch_strided(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream) {
     if (n_polys == 0) return cudaSuccess;
-#define BF_LAUNCH(LM) ntt_pass<FWD, STRIDED, LM><<<grid, threads, smem, stream>>>(ring.dev, B, cfg)
-    if (!first) BF_LAUNCH(LOAD_PLAIN);
-    else if (load == LOAD_PLAIN) BF_LAUNCH(LOAD_PLAIN);
-    else if (load == LOAD_REDUCE) BF_LAUNCH(LOAD_REDUCE);
-    else if (load == LOAD_I64) BF_LAUNCH(LOAD_I64);
-    else BF_LAUNCH(LOAD_CENTRED);
-#undef BF_LAUNCH
+    ProfScope prof(ring.prof, FWD ? CAT_NTT_FWD_STRIDED : CAT_NTT_INV_STRIDED, stream);
+    switch (ring.geom.log_r) {
+        case 2: launch_strided_t<FWD, LOAD, 2, 8>(ring, B, n_polys, stream); break;
+        case 3: launch_strided_t<FWD, LOAD, 3, 8>(ring, B, n_polys, stream); break;
+        case 4: launch_strided_t<FWD, LOAD, 4, 7>(ring, B, n_polys, stream); break;
+        case 5: launch_strided_t<FWD, LOAD, 5, 6>(ring, B, n_polys, stream); break;
+        case 6: launch_strided_t<FWD, LOAD, 6, 5>(ring, B, n_polys, stream); break;
+        case 7: launch_strided_t<FWD, LOAD, 7, 4>(ring, B, n_polys, stream); break;
+        case 8: launch_strided_t<FWD, LOAD, 8, 4>(ring, B, n_polys, stream); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+template <bool FWD>
+static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream) {
+    if (n_polys == 0) return cudaSuccess;
+    ProfScope prof(ring.prof, FWD ? CAT_NTT_FWD_CONTIG : CAT_NTT_INV_CONTIG, stream);
+    const u32 chunks = 1u << ring.geom.log_r;
+    const u32 cpb = (u32)ring.geom.contig_lanes;
+    dim3 grid(chunks / cpb, n_polys);
+    ntt_contig<FWD><<<grid, 32 * CHUNKS_PER_BLOCK, 0, stream>>>(ring.dev, B, cpb);
     return cudaGetLastError();
 }
 
 cudaError_t ntt_forward(const RingHost& ring, const PolyBatch& B, u32 n_outer, int load, cudaStream_t stream) {
     const u32 n_polys = n_outer * B.n_m;
-    cudaError_t e = launch_pass<true, true>(ring, B, n_polys, load, true, stream);
+    cudaError_t e;
+    if (load == LOAD_PLAIN) e = launch_strided<true, LOAD_PLAIN>(ring, B, n_polys, stream);
+    else if (load == LOAD_REDUCE) e = launch_strided<true, LOAD_REDUCE>(ring, B, n_polys, stream);
+    else if (load == LOAD_I64) e = launch_strided<true, LOAD_I64>(ring, B, n_polys, stream);
+    else e = launch_strided<true, LOAD_CENTRED>(ring, B, n_polys, stream);
     if (e != cudaSuccess) return e;
-    return launch_pass<true, false>(ring, B, n_polys, LOAD_PLAIN, false, stream);
+    return launch_contig<true>(ring, B, n_polys, stream);
 }
 
 cudaError_t ntt_inverse(const RingHost& ring, const PolyBatch& B, u32 n_outer, cudaStream_t stream) {
     const u32 n_polys = n_outer * B.n_m;
-    cudaError_t e = launch_pass<false, false>(ring, B, n_polys, LOAD_PLAIN, true, stream);
+    cudaError_t e = launch_contig<false>(ring, B, n_polys, stream);
     if (e != cudaSuccess) return e;
-    return launch_pass<false, true>(ring, B, n_polys, LOAD_PLAIN, false, stream);
+    return launch_strided<false, LOAD_PLAIN>(ring, B, n_polys, stream);
 }
 
 }  // namespace bf

@@ -1,0 +1,116 @@
+"""Drive the library over a workload with synthetic inputs (benchmarks and demos).
+
+Holds no arithmetic of the method: it creates a context, fills rotation keys and ciphertexts with
+seeded uniform residues (a fresh ciphertext or a switching key is indistinguishable from that, and
+the kernels' work does not depend on the values), draws fp32 weights ~ N(0, 0.02^2), and calls the
+C ABI.  Correctness is established elsewhere (tests compare with the CPU reference).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import bifrost as bf
+from . import workloads as wl
+
+
+def _uniform_residues(gen: torch.Generator, moduli, lead_shape, N: int, device) -> torch.Tensor:
+    """int64 tensor [*lead_shape, len(moduli), N], slice m uniform in [0, moduli[m])."""
+    out = torch.empty((*lead_shape, len(moduli), N), dtype=torch.int64, device=device)
+    for m, q in enumerate(moduli):
+        out[..., m, :] = torch.randint(0, int(q), (*lead_shape, N), generator=gen, device=device, dtype=torch.int64)
+    return out
+
+
+class WorkloadRunner:
+    """One context per workload; per layer: weights (cached when the budget allows), input and
+    output ciphertext buffers."""
+
+    def __init__(self, name: str, seed: int = 0, device: str = "cuda:0", cache: bool = True,
+                 cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None):
+        self.w = wl.WORKLOADS[name]
+        ps = wl.PARAM_SETS[self.w.params]
+        self.N, self.primes, self.P, self.scale = ps["N"], list(ps["primes"]), ps["special"], ps["scale"]
+        self.r = len(self.primes)
+        self.plan = self.w.plan
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.stream = stream or torch.cuda.current_stream()
+        self.gen = torch.Generator(device=self.device)
+        self.gen.manual_seed(seed)
+        self.ctx = bf.bf_ctx_create(self.N, self.primes + [self.P], self.r, self.scale,
+                                    bf.bf_plan(self.plan.D, self.plan.tau, self.plan.b, self.plan.g),
+                                    self.stream.cuda_stream)
+        budget = cache_budget_bytes if cache_budget_bytes is not None else self.w.cache_budget_bytes
+        if budget:
+            bf.bf_set_cache_budget(self.ctx, int(budget))
+        # rotation keys: uniform residues over the extended basis
+        steps = [k * self.plan.tau for k in range(1, self.plan.b)] + \
+                [j * self.plan.b * self.plan.tau for j in range(1, self.plan.g)]
+        n = self.N // 2
+        self.rot_steps = sorted({s % n for s in steps if s % n})
+        basis = self.primes + [self.P]
+        if self.rot_steps:
+            keys = _uniform_residues(self.gen, basis, (len(self.rot_steps), self.r, 2), self.N, self.device)
+            bf.bf_load_eval_keys(self.ctx, self.rot_steps, len(self.rot_steps), keys)
+            del keys
+        self.key_bytes = len(self.rot_steps) * self.r * 2 * (self.r + 1) * self.N * 8
+        # layers
+        self.layers = []
+        D = self.plan.D
+        for rep in range(self.w.n_repeat):
+            for L in self.w.layers:
+                n_in, n_out = wl.ceil_div(L.d_in, D), wl.ceil_div(L.d_out, D)
+                W = torch.from_numpy(wl.gen_weights(seed, f"{L.name}.{rep}", L.d_out, L.d_in)).to(self.device)
+                handle = None
+                if cache:
+                    try:
+                        handle = bf.bf_encode_weights(self.ctx, W, L.d_out, L.d_in)
+                    except bf.BifrostError as e:
+                        if e.code != bf.BF_ERR_OOM:
+                            raise
+                ct_in = _uniform_residues(self.gen, self.primes, (n_in, 2), self.N, self.device)
+                ct_out = torch.empty((n_out, 2, self.r, self.N), dtype=torch.int64, device=self.device)
+                self.layers.append(dict(layer=L, rep=rep, n_in=n_in, n_out=n_out, W=W, handle=handle,
+                                        ct_in=ct_in, ct_out=ct_out,
+                                        pt_bytes=n_in * n_out * (D // self.plan.tau) * self.r * self.N * 8))
+        torch.cuda.synchronize()
+
+    # ------------------------------------------------------------------ one decode token
+    def step(self):
+        """All linear layers of the workload once: bf_linear + bf_rescale per layer (device buffers)."""
+        for e in self.layers:
+            L = e["layer"]
+            bf.bf_linear(self.ctx, e["ct_in"], e["n_in"], e["handle"], None if e["handle"] else e["W"],
+                         L.d_out, L.d_in, e["ct_out"], e["n_out"])
+            bf.bf_rescale(self.ctx, e["ct_out"], e["ct_out"], e["n_out"], self.r)
+
+    def make_host_buffers(self):
+        for e in self.layers:
+            e["h_in"] = e["ct_in"].cpu().pin_memory()
+            e["h_out"] = torch.empty((e["n_out"], 2, self.r - 1, self.N), dtype=torch.int64).pin_memory()
+
+    def step_host(self):
+        """The same through the host-buffer entry point: ciphertexts travel host -> device -> host."""
+        for e in self.layers:
+            L = e["layer"]
+            bf.bf_linear_host(self.ctx, e["h_in"], e["n_in"], e["handle"], None if e["handle"] else e["W"],
+                              L.d_out, L.d_in, e["h_out"], e["n_out"])
+
+    def host_bytes_per_step(self):
+        h2d = sum(e["n_in"] * 2 * self.r * self.N * 8 for e in self.layers)
+        d2h = sum(e["n_out"] * 2 * (self.r - 1) * self.N * 8 for e in self.layers)
+        return h2d, d2h
+
+    def cached_pt_bytes(self):
+        return sum(e["pt_bytes"] for e in self.layers if e["handle"])
+
+    def total_pt_bytes(self):
+        return sum(e["pt_bytes"] for e in self.layers)
+
+    def n_fallback_layers(self):
+        return sum(1 for e in self.layers if not e["handle"])
+
+    def close(self):
+        bf.bf_ctx_destroy(self.ctx)
+        self.layers = []
