@@ -76,7 +76,7 @@ struct DevBuf {
 
 struct bf_weights {
     u32 d_out, d_in, n_in, n_out;
-    u64* pt;            // [g][n_out][n_in][b][r][N], NTT domain
+    u64* pt;            // [g][n_out][n_in][b][r][N], NTT domain, Montgomery form (times 2^64 mod q_i)
     size_t bytes;
 };
 
@@ -91,7 +91,8 @@ struct bf_ctx {
     ulonglong2 *tw_fwd = nullptr, *tw_inv = nullptr;
     u32* slot_of_pos = nullptr;
     double2 *T = nullptr, *Z = nullptr;
-    int* overflow_flag = nullptr;
+    int* overflow_flag = nullptr;   // [0]: encoder range overflow; [1]: a bounded device-side wait gave up
+    int* device_error = nullptr;
     // rotation keys
     std::map<u32, int> key_of_steps;
     u64* keys = nullptr;
@@ -215,6 +216,14 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
         R.c64s[m] = h_shoup(R.c64[m], q);
         R.ninv[m] = h_invmod(N % q, q);
         R.ninvs[m] = h_shoup(R.ninv[m], q);
+        {
+            u64 inv = 1;                                   // q^{-1} mod 2^64 by Newton iteration
+            for (int it = 0; it < 6; ++it) inv *= 2 - q * inv;
+            R.qneg[m] = (u64)0 - inv;
+            const u64 two64_inv = h_invmod(R.c64[m], q);
+            R.ninv_m[m] = h_mulmod(R.ninv[m], two64_inv, q);
+            R.ninv_ms[m] = h_shoup(R.ninv_m[m], q);
+        }
         if (m < n_ct_primes) {
             R.pmod[m] = P % q;
             R.pinv[m] = h_invmod(P % q, q);
@@ -276,13 +285,14 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
     CKC(cudaMalloc(&ctx->slot_of_pos, sop.size() * sizeof(u32)));
     CKC(cudaMalloc(&ctx->T, T.size() * sizeof(double2)));
     CKC(cudaMalloc(&ctx->Z, Z.size() * sizeof(double2)));
-    CKC(cudaMalloc(&ctx->overflow_flag, sizeof(int)));
+    CKC(cudaMalloc(&ctx->overflow_flag, 2 * sizeof(int)));
+    ctx->device_error = ctx->overflow_flag + 1;
     CKC(cudaMemcpy(ctx->tw_fwd, twf.data(), twf.size() * sizeof(ulonglong2), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->tw_inv, twi.data(), twi.size() * sizeof(ulonglong2), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->slot_of_pos, sop.data(), sop.size() * sizeof(u32), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->T, T.data(), T.size() * sizeof(double2), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->Z, Z.data(), Z.size() * sizeof(double2), cudaMemcpyHostToDevice));
-    CKC(cudaMemset(ctx->overflow_flag, 0, sizeof(int)));
+    CKC(cudaMemset(ctx->overflow_flag, 0, 2 * sizeof(int)));
     CKC(cudaDeviceSynchronize());
 #undef CKC
     R.tw_fwd = ctx->tw_fwd;
@@ -425,7 +435,7 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
         B.n_m = r;
         B.mod0 = 0;
         B.mod_step = 1;
-        CK(ntt_forward(ctx->ring, B, cnt, LOAD_I64, ctx->stream));
+        CK(ntt_forward(ctx->ring, B, cnt, LOAD_I64_MONT, ctx->stream));   // cached form: NTT domain, times 2^64
     }
     return BF_OK;
 }
@@ -652,7 +662,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     // ---- multiply-accumulate over the encoded diagonals
     const u32 n_terms = n_in * b, n_pj = n_out * g;
     if (pt_weights) {
-        CK(launch_mac(ctx->ring, pt_weights->pt, X, A, n_pj, n_terms, ctx->stream));
+        CK(launch_mac(ctx->ring, pt_weights->pt, X, A, n_pj, n_terms, ctx->device_error, ctx->stream));
     } else {
         // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them
         const size_t group_bytes = (size_t)n_terms * r * N * 8;
@@ -663,7 +673,8 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         for (u32 pj0 = 0; pj0 < n_pj; pj0 += groups) {
             const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
             TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p));
-            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, X, A + (size_t)pj0 * ctw, cnt, n_terms, ctx->stream));
+            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, X, A + (size_t)pj0 * ctw, cnt, n_terms, ctx->device_error,
+                          ctx->stream));
         }
     }
     stamp(ctx, 2);
@@ -843,6 +854,7 @@ extern "C" int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, u
     B.src_sm = B.dst_sm = N;
     B.n_m = r;
     B.mod_step = 1;
+    B.from_mont = 1;
     CK(ntt_inverse(ctx->ring, B, 1, ctx->stream));
     return BF_OK;
 }

@@ -28,6 +28,9 @@ struct RingDev {
     u64 pinv[MAX_MODULI];        // P^{-1} mod q_i (i < r)
     u64 pinvs[MAX_MODULI];
     u64 pmod[MAX_MODULI];        // P mod q_i
+    u64 qneg[MAX_MODULI];        // -q^{-1} mod 2^64 (Montgomery reduction)
+    u64 ninv_m[MAX_MODULI];      // N^{-1} * 2^{-64} mod q: inverse transform that also leaves Montgomery form
+    u64 ninv_ms[MAX_MODULI];
     const ulonglong2* tw_fwd;    // [r+1][N]  (psi^brev(k), Shoup companion), merged Cooley-Tukey order
     const ulonglong2* tw_inv;    // [r+1][N]  inverses of the above, for the Gentleman-Sande inverse
 };
@@ -68,6 +71,70 @@ __device__ __forceinline__ void mac128(u64& hi, u64& lo, u64 a, u64 b) {
     hi += ph + (lo < pl ? 1ull : 0ull);
 }
 
+// Lazy sum of products of 64-bit words, kept as partial sums of 32-bit limb products so that one
+// term costs four 32x32->64 multiplies and no 64-bit high-product sequence:
+//   sum a*b = lo + mid * 2^32 + hi * 2^64,   lo = sum a0*b0,  mid = sum (a0*b1 + a1*b0),  hi = sum a1*b1.
+// lo and mid carry their overflow into 32-bit counters.  With words below 2^60 and at most 2^8 terms
+// hi stays below 2^64 and the total below 2^128.  SMALL drops the carry counter of mid: valid while
+// terms * 2 * 2^(bits-32) * 2^32 < 2^64, e.g. words below 2^50 and up to 2^13 terms.
+template <bool SMALL>
+struct LimbAcc {
+    u64 lo = 0, mid = 0, hi = 0;
+    u32 lo_c = 0, mid_c = 0;
+
+    __device__ __forceinline__ void mac(u64 a, u64 b) {
+        const u32 a0 = (u32)a, a1 = (u32)(a >> 32), b0 = (u32)b, b1 = (u32)(b >> 32);
+        if (SMALL) {
+            asm("{\n\t.reg .u64 p;\n\t"
+                "mul.wide.u32 p, %4, %6;\n\t"
+                "add.cc.u64 %0, %0, p;\n\t"
+                "addc.u32 %1, %1, 0;\n\t"
+                "mad.wide.u32 %2, %4, %7, %2;\n\t"
+                "mad.wide.u32 %2, %5, %6, %2;\n\t"
+                "mad.wide.u32 %3, %5, %7, %3;\n\t}"
+                : "+l"(lo), "+r"(lo_c), "+l"(mid), "+l"(hi)
+                : "r"(a0), "r"(a1), "r"(b0), "r"(b1));
+        } else {
+            asm("{\n\t.reg .u64 p;\n\t"
+                "mul.wide.u32 p, %5, %7;\n\t"
+                "add.cc.u64 %0, %0, p;\n\t"
+                "addc.u32 %1, %1, 0;\n\t"
+                "mul.wide.u32 p, %5, %8;\n\t"
+                "add.cc.u64 %2, %2, p;\n\t"
+                "addc.u32 %3, %3, 0;\n\t"
+                "mul.wide.u32 p, %6, %7;\n\t"
+                "add.cc.u64 %2, %2, p;\n\t"
+                "addc.u32 %3, %3, 0;\n\t"
+                "mad.wide.u32 %4, %6, %8, %4;\n\t}"
+                : "+l"(lo), "+r"(lo_c), "+l"(mid), "+r"(mid_c), "+l"(hi)
+                : "r"(a0), "r"(a1), "r"(b0), "r"(b1));
+        }
+    }
+
+    // the accumulated integer modulo q, in [0, q)
+    __device__ __forceinline__ u64 reduce(u64 q, u64 mu, u64 c64, u64 c64s) const {
+        const u64 L = lo + (mid << 32);
+        const u64 carry = L < lo ? 1ull : 0ull;
+        const u64 H = (u64)lo_c + (mid >> 32) + ((u64)mid_c << 32) + hi + carry;
+        return reduce128(H, L, q, mu, c64, c64s);
+    }
+
+    // Montgomery reduction of the accumulated integer V: V * 2^{-64} mod q, in [0, q).
+    // Requires V < q * 2^64 (number of terms times q below 2^64).  qneg = -q^{-1} mod 2^64.
+    __device__ __forceinline__ u64 reduce_mont(u64 q, u64 qneg) const {
+        const u64 L = lo + (mid << 32);
+        const u64 carry = L < lo ? 1ull : 0ull;
+        const u64 H = (u64)lo_c + (mid >> 32) + ((u64)mid_c << 32) + hi + carry;
+        const u64 m = L * qneg;
+        u64 t = H + __umul64hi(m, q) + (L != 0 ? 1ull : 0ull);   // L + lo(m*q) = 0 mod 2^64, carrying iff L != 0
+        return t >= q ? t - q : t;
+    }
+
+    __device__ __forceinline__ void reset_to(u64 v) {
+        lo = v; mid = 0; hi = 0; lo_c = 0; mid_c = 0;
+    }
+};
+
 __device__ __forceinline__ u64 add_mod(u64 a, u64 b, u64 q) {
     u64 v = a + b;
     return v >= q ? v - q : v;
@@ -83,6 +150,7 @@ enum LoadMode : int {
     LOAD_REDUCE = 1,    // any 64-bit non-negative integer (e.g. a residue of another prime): x mod q
     LOAD_I64 = 2,       // signed 64-bit integer coefficient: x mod q in [0, q)
     LOAD_CENTRED = 3,   // residue t in [0, M) of modulus M: centred lift to (-M/2, M/2], then mod q
+    LOAD_I64_MONT = 4,  // LOAD_I64, then times 2^64 mod q: the transform's output is in Montgomery form
 };
 
 // A batch of equally sized polynomials addressed as (outer index o, slot m):
@@ -95,6 +163,7 @@ struct PolyBatch {
     long long src_so, src_sm, dst_so, dst_sm;
     u32 n_m, mod0, mod_step;
     u64 lift_mod;                 // LOAD_CENTRED: the modulus M the source residues live in
+    u32 from_mont;                // inverse transform only: input is in Montgomery form, output is not
 };
 
 }  // namespace bf

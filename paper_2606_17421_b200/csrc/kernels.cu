@@ -28,60 +28,231 @@ cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Multiply-accumulate over encoded diagonals.
-//   A[pj][comp][i][n] = sum_{t < n_terms} Pt[pj][t][i][n] * X[t][comp][i][n]   (mod q_i)
-// Every plaintext word is read from HBM exactly once with 128-bit loads; the two ciphertext
-// components share it.  Products accumulate lazily in 128 bits; one reduction per output word.
-constexpr int MAC_THREADS = 256;
-constexpr int MAC_LAZY_TERMS = 128;   // 128 * (2^60)^2 < 2^128
+// Asynchronous bulk copies (TMA, untiled form) and transaction barriers.
+__device__ __forceinline__ u32 smem_addr(const void* p) { return (u32)__cvta_generic_to_shared(p); }
 
-__global__ void __launch_bounds__(MAC_THREADS) mac_kernel(const RingDev R, const u64* __restrict__ pt,
-                                                          const u64* __restrict__ x, u64* __restrict__ a,
-                                                          u32 n_terms) {
-    const u32 i = blockIdx.y, pj = blockIdx.z;
-    const u32 N = R.N, r = R.r;
-    const u32 n = (blockIdx.x * MAC_THREADS + threadIdx.x) * 2;
-    const u64 q = R.q[i], mu = R.mu[i], c64 = R.c64[i], c64s = R.c64s[i];
-    const u64* ptp = pt + ((size_t)pj * n_terms * r + i) * N + n;
-    const u64* xp = x + (size_t)i * N + n;
-    const size_t pt_stride = (size_t)r * N, x_stride = (size_t)2 * r * N, comp_stride = (size_t)r * N;
-    u64 h00 = 0, l00 = 0, h01 = 0, l01 = 0, h10 = 0, l10 = 0, h11 = 0, l11 = 0;   // [comp][word]
-    for (u32 t0 = 0; t0 < n_terms; t0 += MAC_LAZY_TERMS) {
-        const u32 t1 = min(n_terms, t0 + MAC_LAZY_TERMS);
-#pragma unroll 4
-        for (u32 t = t0; t < t1; ++t) {
-            const ulonglong2 w = __ldcs((const ulonglong2*)(ptp + t * pt_stride));     // streamed once
-            const ulonglong2 x0 = __ldg((const ulonglong2*)(xp + t * x_stride));
-            const ulonglong2 x1 = __ldg((const ulonglong2*)(xp + t * x_stride + comp_stride));
-            mac128(h00, l00, w.x, x0.x);
-            mac128(h01, l01, w.y, x0.y);
-            mac128(h10, l10, w.x, x1.x);
-            mac128(h11, l11, w.y, x1.y);
-        }
-        if (t1 < n_terms) {   // keep the running sums below 2^64 before the next lazy stretch
-            l00 = reduce128(h00, l00, q, mu, c64, c64s); h00 = 0;
-            l01 = reduce128(h01, l01, q, mu, c64, c64s); h01 = 0;
-            l10 = reduce128(h10, l10, q, mu, c64, c64s); h10 = 0;
-            l11 = reduce128(h11, l11, q, mu, c64, c64s); h11 = 0;
-        }
+__device__ __forceinline__ void mbar_init(u64* bar, u32 count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(u64* bar, u32 bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+// global -> shared copy of `bytes` (multiple of 16, both addresses 16-byte aligned); completion is
+// signalled on the barrier as transferred bytes
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, u64* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
+    u32 ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after a fixed number of polls (each poll may itself suspend for a while),
+// records the failure and lets the caller carry on so that the kernel always terminates.
+__device__ __forceinline__ void mbar_wait(u64* bar, u32 parity, int* error_flag) {
+    for (int it = 0; it < (1 << 22); ++it)
+        if (mbar_try_wait(bar, parity)) return;
+    atomicExch(error_flag, 1);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Multiply-accumulate over encoded diagonals (the ciphertext x plaintext product of Sec. 3.5 / 4.2).
+//   A[pj][comp][i][n] = sum_{t < n_terms} Pt[pj][t][i][n] * X[t][comp][i][n]   (mod q_i)
+//
+// A block owns one prime i and a tile of TN adjacent coefficients.  The rotated inputs X of that
+// tile, for every term and both components, are brought into shared memory once and stay there.
+// The encoded weights are then streamed from HBM through a ring of shared-memory stages filled by
+// bulk asynchronous copies (each plaintext word crosses HBM exactly once and is shared by both
+// ciphertext components).  The 256 threads are arranged as TN coefficients x PL "group lanes":
+// lane l accumulates output groups pj = l, l + PL, ...  Products accumulate lazily as limb partial
+// sums; one modular reduction per output word.
+constexpr int MAC_THREADS = 256;
+constexpr int MAC_TS = 8;                         // terms per stage
+constexpr int MAC_STAGES = 4;
+constexpr int MAC_STAGE_WORDS = MAC_TS * MAC_THREADS;   // 16 KB per stage whatever TN is
+
+template <bool SMALL, int LOG_TN>
+__global__ void __launch_bounds__(MAC_THREADS, 2)
+mac_kernel(const RingDev R, const u64* __restrict__ pt, const u64* __restrict__ x, u64* __restrict__ a, u32 n_terms,
+           u32 n_pj, u32 pj_per_block, u32 lazy_terms, int* __restrict__ error_flag) {
+    extern __shared__ __align__(128) unsigned char mac_smem[];
+    constexpr u32 TN = 1u << LOG_TN, PL = MAC_THREADS >> LOG_TN;
+    u64* ring = (u64*)mac_smem;                                    // [MAC_STAGES][PL][MAC_TS][TN]
+    u64* xs = ring + MAC_STAGES * MAC_STAGE_WORDS;                 // [n_terms][2][TN]
+    u64* bars = xs + (size_t)n_terms * 2 * TN;                     // [MAC_STAGES] full barriers + 1 for X
+    const u32 i = blockIdx.y, N = R.N, r = R.r;
+    const u32 n0 = blockIdx.x << LOG_TN;
+    const u32 tid = threadIdx.x, c = tid & (TN - 1), l = tid >> LOG_TN;
+    const u64 q = R.q[i], qneg = R.qneg[i];
+    const u32 pj_begin = blockIdx.z * pj_per_block;
+    const u32 pj_end = min(n_pj, pj_begin + pj_per_block);
+    const u32 n_groups = (pj_end - pj_begin + PL - 1) / PL;        // rounds of PL output groups
+    const u32 n_chunks = (n_terms + MAC_TS - 1) / MAC_TS;
+    const u32 n_items = n_groups * n_chunks;
+    const size_t pt_term = (size_t)r * N, pt_pj = (size_t)n_terms * r * N;
+
+    if (tid == 0) {
+        for (int s = 0; s <= MAC_STAGES; ++s) mbar_init(&bars[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    u64* ap = a + ((size_t)pj * 2 * r + i) * N + n;
-    ulonglong2 o0, o1;
-    o0.x = reduce128(h00, l00, q, mu, c64, c64s);
-    o0.y = reduce128(h01, l01, q, mu, c64, c64s);
-    o1.x = reduce128(h10, l10, q, mu, c64, c64s);
-    o1.y = reduce128(h11, l11, q, mu, c64, c64s);
-    *(ulonglong2*)ap = o0;
-    *(ulonglong2*)(ap + comp_stride) = o1;
+    __syncthreads();
+
+    // item (group round g, term chunk ch) -> ring slot: lane l' copies up to TS segments of TN words
+    // for output group pj = pj_begin + g*PL + l'.  Called by the 32 threads of warp 0.
+    auto issue = [&](u32 g, u32 ch, u32 slot) {
+        const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
+        const u32 first = pj_begin + g * PL;
+        const u32 lanes = min((u32)PL, pj_end - first);
+        if (tid == 0) mbar_expect_tx(&bars[slot], lanes * cnt * TN * 8);
+        __syncwarp();
+        for (u32 e = tid; e < lanes * MAC_TS; e += 32) {           // one copy per (lane, term)
+            const u32 ll = e / MAC_TS, ts = e % MAC_TS;
+            if (ts < cnt) {
+                const u64* src = pt + (size_t)(first + ll) * pt_pj + (size_t)(t0 + ts) * pt_term + (size_t)i * N + n0;
+                bulk_g2s(ring + (size_t)slot * MAC_STAGE_WORDS + ((size_t)ll * MAC_TS + ts) * TN, src, TN * 8,
+                         &bars[slot]);
+            }
+        }
+    };
+
+    u32 ig = 0, ich = 0, islot = 0, issued = 0;                     // next item to issue (warp 0 only)
+    auto issue_next = [&]() {
+        issue(ig, ich, islot);
+        ++issued;
+        if (++ich == n_chunks) { ich = 0; ++ig; }
+        if (++islot == MAC_STAGES) islot = 0;
+    };
+    if (tid < 32) {
+        if (tid == 0) mbar_expect_tx(&bars[MAC_STAGES], n_terms * 2 * TN * 8);
+        __syncwarp();
+        for (u32 e = tid; e < n_terms * 2; e += 32)                 // X tile: [term][component] segments
+            bulk_g2s(xs + (size_t)e * TN, x + ((size_t)e * r + i) * N + n0, TN * 8, &bars[MAC_STAGES]);
+        while (issued < (u32)MAC_STAGES - 1 && issued < n_items) issue_next();
+    }
+    mbar_wait(&bars[MAC_STAGES], 0, error_flag);
+
+    LimbAcc<SMALL> acc0, acc1;
+    u32 since_flush = 0, g = 0, ch = 0, slot = 0, phase = 0;
+    for (u32 k = 0; k < n_items; ++k) {
+        if (tid < 32 && issued < n_items) issue_next();   // into the slot everyone left at the end of item k-1
+        const u32 pj = pj_begin + g * PL + l;
+        const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
+        mbar_wait(&bars[slot], phase, error_flag);
+        if (pj < pj_end) {
+            const u64* ps = ring + (size_t)slot * MAC_STAGE_WORDS + (size_t)l * MAC_TS * TN + c;
+            const u64* xt = xs + (size_t)t0 * 2 * TN + c;
+            if (cnt == MAC_TS) {
+#pragma unroll
+                for (int ts = 0; ts < MAC_TS; ++ts) {
+                    const u64 w = ps[ts * TN];
+                    acc0.mac(w, xt[(ts * 2) * TN]);
+                    acc1.mac(w, xt[(ts * 2 + 1) * TN]);
+                }
+            } else {
+                for (u32 ts = 0; ts < cnt; ++ts) {
+                    const u64 w = ps[ts * TN];
+                    acc0.mac(w, xt[(ts * 2) * TN]);
+                    acc1.mac(w, xt[(ts * 2 + 1) * TN]);
+                }
+            }
+            since_flush += cnt;
+            if (ch + 1 == n_chunks) {
+                // the cached plaintexts carry a factor 2^64, which the Montgomery reduction removes
+                u64* ap = a + ((size_t)pj * 2 * r + i) * N + n0 + c;
+                ap[0] = acc0.reduce_mont(q, qneg);
+                ap[(size_t)r * N] = acc1.reduce_mont(q, qneg);
+                acc0.reset_to(0);
+                acc1.reset_to(0);
+                since_flush = 0;
+            } else if (since_flush + MAC_TS > lazy_terms) {   // keep the partial sums inside their words
+                acc0.reset_to(acc0.reduce(q, R.mu[i], R.c64[i], R.c64s[i]));
+                acc1.reset_to(acc1.reduce(q, R.mu[i], R.c64[i], R.c64s[i]));
+                since_flush = 1;
+            }
+        }
+        __syncthreads();       // the slot may now be overwritten
+        if (++ch == n_chunks) { ch = 0; ++g; }
+        if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
+    }
+}
+
+static int bits_of(u64 v) {
+    int b = 0;
+    while (v) { ++b; v >>= 1; }
+    return b;
+}
+
+template <bool SMALL, int LOG_TN>
+static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
+                                u32 lazy, int* error_flag, cudaStream_t stream) {
+    constexpr u32 TN = 1u << LOG_TN, PL = MAC_THREADS >> LOG_TN;
+    const size_t smem = (size_t)MAC_STAGES * MAC_STAGE_WORDS * 8 + (size_t)n_terms * 2 * TN * 8 + (MAC_STAGES + 1) * 8;
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    static bool attr_set = false;     // opt in once to the large dynamic shared-memory carve-out
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(mac_kernel<SMALL, LOG_TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             200 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    // slices over output groups: enough blocks to fill the machine several times over
+    const u32 tiles = (ring.dev.N >> LOG_TN) * ring.dev.r;
+    u32 slices = (148u * 2 * 6 + tiles - 1) / tiles;
+    const u32 max_slices = (n_pj + PL - 1) / PL;
+    if (slices > max_slices) slices = max_slices;
+    if (slices < 1) slices = 1;
+    u32 pj_per_block = (n_pj + slices - 1) / slices;
+    pj_per_block = (pj_per_block + PL - 1) / PL * PL;
+    slices = (n_pj + pj_per_block - 1) / pj_per_block;
+    dim3 grid(ring.dev.N >> LOG_TN, ring.dev.r, slices);
+    mac_kernel<SMALL, LOG_TN><<<grid, MAC_THREADS, smem, stream>>>(ring.dev, pt, x, a, n_terms, n_pj, pj_per_block, lazy,
+                                                                    error_flag);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
-                       cudaStream_t stream) {
+                       int* error_flag, cudaStream_t stream) {
     if (n_pj == 0) return cudaSuccess;
-    dim3 grid(ring.dev.N / (2 * MAC_THREADS), ring.dev.r, n_pj);
     ProfScope prof(ring.prof, CAT_MAC, stream);
-    mac_kernel<<<grid, MAC_THREADS, 0, stream>>>(ring.dev, pt, x, a, n_terms);
-    return cudaGetLastError();
+    u64 qmax = 0;
+    for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
+    const int qbits = bits_of(qmax);
+    // tile width: the resident X tile (n_terms * 2 * TN words) must stay within 48 KB
+    u32 log_tn = 8;
+    while (log_tn > 4 && (size_t)n_terms * 2 * (1u << log_tn) * 8 > 48 * 1024) --log_tn;
+    const bool small = qbits <= 50;
+    // terms the lazy sums can take: limb partial sums inside their words, and the total below q * 2^64
+    u32 lazy = small ? (1u << (63 - qbits)) : 128u;
+    const u64 by_q = (~(u64)0) / qmax;
+    if ((u64)lazy > by_q - 1) lazy = (u32)(by_q - 1);
+    if (lazy < MAC_TS) return cudaErrorInvalidValue;
+#define BF_MAC(S, L) launch_mac_t<S, L>(ring, pt, x, a, n_pj, n_terms, lazy, error_flag, stream)
+    if (small) {
+        switch (log_tn) {
+            case 8: return BF_MAC(true, 8);
+            case 7: return BF_MAC(true, 7);
+            case 6: return BF_MAC(true, 6);
+            case 5: return BF_MAC(true, 5);
+            default: return BF_MAC(true, 4);
+        }
+    }
+    switch (log_tn) {
+        case 8: return BF_MAC(false, 8);
+        case 7: return BF_MAC(false, 7);
+        case 6: return BF_MAC(false, 6);
+        case 5: return BF_MAC(false, 5);
+        default: return BF_MAC(false, 4);
+    }
+#undef BF_MAC
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -46,11 +46,13 @@ template <int LOAD>
 __device__ __forceinline__ u64 load_src(const void* src, size_t idx, u64 q, u64 mu, u64 lift_mod, u64 lift_red) {
     if (LOAD == LOAD_PLAIN) return ((const u64*)src)[idx];
     if (LOAD == LOAD_REDUCE) return barrett64(((const u64*)src)[idx], q, mu);
-    if (LOAD == LOAD_I64) {
+    if (LOAD == LOAD_I64 || LOAD == LOAD_I64_MONT) {
         i64 v = ((const i64*)src)[idx];
         u64 a = v < 0 ? (u64)(-v) : (u64)v;
         u64 m = barrett64(a, q, mu);
-        return (v < 0 && m != 0) ? q - m : m;
+        m = (v < 0 && m != 0) ? q - m : m;
+        if (LOAD == LOAD_I64_MONT) m = mul_shoup(m, lift_mod, lift_red, q);   // (2^64 mod q, its Shoup companion)
+        return m;
     }
     // LOAD_CENTRED
     u64 t = ((const u64*)src)[idx];
@@ -138,7 +140,11 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
     const char* src = (const char*)B.src + ((size_t)o * B.src_so + (size_t)m * B.src_sm) * 8;
-    const u64 lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu) : 0;
+    const u64 lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu)
+                       : (LOAD == LOAD_I64_MONT) ? R.c64s[mod] : 0;
+    const u64 lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
+    const u64 ninv = (!FWD && B.from_mont) ? R.ninv_m[mod] : R.ninv[mod];
+    const u64 ninvs = (!FWD && B.from_mont) ? R.ninv_ms[mod] : R.ninvs[mod];
     const int col0 = blockIdx.x * LANES;
     const int tid = threadIdx.x;
 #pragma unroll
@@ -163,7 +169,7 @@ ntt_strided(const RingDev R, const PolyBatch B) {
                 const int row = base + i * step;
                 if (g_first) {
                     const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
-                    e[i] = FWD ? load_src<LOAD>(src, gidx, q, mu, B.lift_mod, lift_red) : dst[gidx];
+                    e[i] = FWD ? load_src<LOAD>(src, gidx, q, mu, lift_mod, lift_red) : dst[gidx];
                 } else {
                     e[i] = sm[row * LANES + lane];
                 }
@@ -177,7 +183,7 @@ ntt_strided(const RingDev R, const PolyBatch B) {
                 if (g_last) {
                     const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
                     u64 v = e[i];
-                    if (!FWD) v = mul_shoup(v, R.ninv[mod], R.ninvs[mod], q);   // scale by N^{-1}, to [0, q)
+                    if (!FWD) v = mul_shoup(v, ninv, ninvs, q);                  // scale by N^{-1}, to [0, q)
                     dst[gidx] = v;                                              // forward: lazy, below 4q
                 } else {
                     sm[row * LANES + lane] = e[i];
@@ -336,6 +342,7 @@ cudaError_t ntt_forward(const RingHost& ring, const PolyBatch& B, u32 n_outer, i
     if (load == LOAD_PLAIN) e = launch_strided<true, LOAD_PLAIN>(ring, B, n_polys, stream);
     else if (load == LOAD_REDUCE) e = launch_strided<true, LOAD_REDUCE>(ring, B, n_polys, stream);
     else if (load == LOAD_I64) e = launch_strided<true, LOAD_I64>(ring, B, n_polys, stream);
+    else if (load == LOAD_I64_MONT) e = launch_strided<true, LOAD_I64_MONT>(ring, B, n_polys, stream);
     else e = launch_strided<true, LOAD_CENTRED>(ring, B, n_polys, stream);
     if (e != cudaSuccess) return e;
     return launch_contig<true>(ring, B, n_polys, stream);
