@@ -435,6 +435,7 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
         B.n_m = r;
         B.mod0 = 0;
         B.mod_step = 1;
+        B.split_bits = mac_split_bits(ctx->ring);
         CK(ntt_forward(ctx->ring, B, cnt, LOAD_I64_MONT, ctx->stream));   // cached form: NTT domain, times 2^64
     }
     return BF_OK;
@@ -855,6 +856,7 @@ extern "C" int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, u
     B.n_m = r;
     B.mod_step = 1;
     B.from_mont = 1;
+    B.split_bits = mac_split_bits(ctx->ring);
     CK(ntt_inverse(ctx->ring, B, 1, ctx->stream));
     return BF_OK;
 }

@@ -164,6 +164,59 @@ struct PolyBatch {
     u32 n_m, mod0, mod_step;
     u64 lift_mod;                 // LOAD_CENTRED: the modulus M the source residues live in
     u32 from_mont;                // inverse transform only: input is in Montgomery form, output is not
+    u32 split_bits;               // L > 0: the NTT-domain side of the transform is stored as two L-bit-aligned
+                                  // limbs per word, (v >> L) << 32 | (v & (2^L - 1)); forward writes, inverse reads it
 };
+
+__device__ __forceinline__ u64 limb_split(u64 v, u32 L) { return ((v >> L) << 32) | (v & ((1ull << L) - 1)); }
+__device__ __forceinline__ u64 limb_join(u64 s, u32 L) { return ((s >> 32) << L) | (s & 0xffffffffull); }
+
+// Karatsuba accumulator for products of words given as two L-bit limbs (low limb in the low 32-bit
+// half, high limb in the high half), L <= 25:  three 32x32->64 multiply-adds per product and no
+// carries.  sum v*x = lo + (mid - lo - hi) * 2^L + hi * 2^(2L), with lo = sum v0*x0, hi = sum v1*x1,
+// mid = sum (v0+v1)*(x0+x1); every term of mid is below 2^(2L+2), so 2^(62-2L) terms fit.
+struct KaraAcc {
+    u64 lo = 0, mid = 0, hi = 0;
+    __device__ __forceinline__ void mac(u32 v0, u32 v1, u32 vs, u64 xsplit) {
+        const u32 x0 = (u32)xsplit, x1 = (u32)(xsplit >> 32);
+        lo += (u64)v0 * x0;
+        hi += (u64)v1 * x1;
+        mid += (u64)vs * (x0 + x1);
+    }
+    // the accumulated integer V as (H, L64)
+    __device__ __forceinline__ void value(u32 L, u64& H, u64& L64) const {
+        const u64 m = mid - lo - hi;
+        u64 l = lo, h = 0;
+        const u64 a = m << L;
+        l += a; h += (l < a) ? 1ull : 0ull;
+        h += m >> (64 - L);
+        const u64 b = hi << (2 * L);
+        l += b; h += (l < b) ? 1ull : 0ull;
+        h += hi >> (64 - 2 * L);
+        H = h; L64 = l;
+    }
+};
+
+// Montgomery reduction by two 32-bit rounds: V * 2^{-64} mod q in [0, q), for V = (H, L) < q * 2^64.
+// qneg32 = -q^{-1} mod 2^32.  Six 32-bit multiplies instead of a 64x64 high product.
+__device__ __forceinline__ u64 redc_2x32(u64 H, u64 L, u64 q, u32 qneg32) {
+    const u32 q0 = (u32)q, q1 = (u32)(q >> 32);
+#pragma unroll
+    for (int round = 0; round < 2; ++round) {
+        const u32 m = (u32)L * qneg32;
+        const u64 p0 = (u64)m * q0, p1 = (u64)m * q1;
+        // (H, L) += p0 + (p1 << 32)
+        u64 l = L + p0;
+        u64 c = (l < p0) ? 1ull : 0ull;
+        const u64 p1s = p1 << 32;
+        l += p1s;
+        c += (l < p1s) ? 1ull : 0ull;
+        const u64 h = H + (p1 >> 32) + c;
+        // low 32 bits are now zero: shift right by 32
+        L = (l >> 32) | (h << 32);
+        H = h >> 32;
+    }
+    return L >= q ? L - q : L;
+}
 
 }  // namespace bf

@@ -71,6 +71,7 @@ cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, cons
                                   const u64* c0_base, long long c0_stride, const u32* perms, u64* out_base,
                                   long long out_stride, cudaStream_t stream);
 // A[pj][comp][i][n] = sum_{t < n_terms} Pt[pj][t][i][n] * X[t][comp][i][n],  pj = j*n_out + p, t = q*b + k
+u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintext format (0 = whole words)
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
                        int* error_flag, cudaStream_t stream);
 // y[p] = a[p] + sum_{j=1}^{g-1} rres[(j-1)*n_out + p]   (ciphertexts of [2][r][N] words)

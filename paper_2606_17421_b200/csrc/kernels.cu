@@ -64,89 +64,112 @@ __device__ __forceinline__ void mbar_wait(u64* bar, u32 parity, int* error_flag)
     atomicExch(error_flag, 1);
 }
 
+__device__ __forceinline__ void mbar_arrive(u64* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
 // ------------------------------------------------------------------------------------------------
 // Multiply-accumulate over encoded diagonals (the ciphertext x plaintext product of Sec. 3.5 / 4.2).
 //   A[pj][comp][i][n] = sum_{t < n_terms} Pt[pj][t][i][n] * X[t][comp][i][n]   (mod q_i)
 //
 // A block owns one prime i and a tile of TN adjacent coefficients.  The rotated inputs X of that
 // tile, for every term and both components, are brought into shared memory once and stay there.
-// The encoded weights are then streamed from HBM through a ring of shared-memory stages filled by
-// bulk asynchronous copies (each plaintext word crosses HBM exactly once and is shared by both
-// ciphertext components).  The 256 threads are arranged as TN coefficients x PL "group lanes":
-// lane l accumulates output groups pj = l, l + PL, ...  Products accumulate lazily as limb partial
-// sums; one modular reduction per output word.
-constexpr int MAC_THREADS = 256;
+// The encoded weights are streamed from HBM through a ring of shared-memory stages filled by bulk
+// asynchronous copies that a dedicated producer warp issues; full/empty transaction barriers
+// couple it to the eight consumer warps, so no block-wide barrier sits on the stream.  Each
+// plaintext word crosses HBM exactly once and is shared by both ciphertext components.  The 256
+// consumer threads are arranged as TN coefficients x PL "group lanes": lane l accumulates output
+// groups pj = l, l + PL, ...
+//
+// Arithmetic.  The cached plaintexts are in Montgomery form (times 2^64 mod q_i).  KARA (all
+// ciphertext primes below 2^50): they are stored as two 25-bit limbs per word, X is split the same
+// way once per block, and products accumulate by Karatsuba (3 multiplies, no carries).  Otherwise
+// words are whole and products accumulate as 32-bit limb partial sums with carries.  One Montgomery
+// reduction per output word removes the 2^64.
+constexpr int MAC_CONSUMERS = 256;
+constexpr int MAC_THREADS = MAC_CONSUMERS + 32;   // + one producer warp
 constexpr int MAC_TS = 8;                         // terms per stage
 constexpr int MAC_STAGES = 4;
-constexpr int MAC_STAGE_WORDS = MAC_TS * MAC_THREADS;   // 16 KB per stage whatever TN is
+constexpr int MAC_STAGE_WORDS = MAC_TS * MAC_CONSUMERS;   // 16 KB per stage whatever TN is
+constexpr u32 KARA_L = 25;
 
-template <bool SMALL, int LOG_TN>
+template <bool KARA, int LOG_TN>
 __global__ void __launch_bounds__(MAC_THREADS, 2)
 mac_kernel(const RingDev R, const u64* __restrict__ pt, const u64* __restrict__ x, u64* __restrict__ a, u32 n_terms,
            u32 n_pj, u32 pj_per_block, u32 lazy_terms, int* __restrict__ error_flag) {
     extern __shared__ __align__(128) unsigned char mac_smem[];
-    constexpr u32 TN = 1u << LOG_TN, PL = MAC_THREADS >> LOG_TN;
+    constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     u64* ring = (u64*)mac_smem;                                    // [MAC_STAGES][PL][MAC_TS][TN]
     u64* xs = ring + MAC_STAGES * MAC_STAGE_WORDS;                 // [n_terms][2][TN]
-    u64* bars = xs + (size_t)n_terms * 2 * TN;                     // [MAC_STAGES] full barriers + 1 for X
+    u64* full = xs + (size_t)n_terms * 2 * TN;                     // [MAC_STAGES]
+    u64* empty = full + MAC_STAGES;                                // [MAC_STAGES]
+    u64* xbar = empty + MAC_STAGES;
     const u32 i = blockIdx.y, N = R.N, r = R.r;
     const u32 n0 = blockIdx.x << LOG_TN;
-    const u32 tid = threadIdx.x, c = tid & (TN - 1), l = tid >> LOG_TN;
-    const u64 q = R.q[i], qneg = R.qneg[i];
+    const u32 tid = threadIdx.x;
     const u32 pj_begin = blockIdx.z * pj_per_block;
     const u32 pj_end = min(n_pj, pj_begin + pj_per_block);
     const u32 n_groups = (pj_end - pj_begin + PL - 1) / PL;        // rounds of PL output groups
     const u32 n_chunks = (n_terms + MAC_TS - 1) / MAC_TS;
     const u32 n_items = n_groups * n_chunks;
-    const size_t pt_term = (size_t)r * N, pt_pj = (size_t)n_terms * r * N;
 
     if (tid == 0) {
-        for (int s = 0; s <= MAC_STAGES; ++s) mbar_init(&bars[s], 1);
+        for (int s = 0; s < MAC_STAGES; ++s) {
+            mbar_init(&full[s], 1);                                // the producer's arrive.expect_tx
+            mbar_init(&empty[s], MAC_CONSUMERS / 32);              // one arrival per consumer warp
+        }
+        mbar_init(xbar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    // item (group round g, term chunk ch) -> ring slot: lane l' copies up to TS segments of TN words
-    // for output group pj = pj_begin + g*PL + l'.  Called by the 32 threads of warp 0.
-    auto issue = [&](u32 g, u32 ch, u32 slot) {
-        const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
-        const u32 first = pj_begin + g * PL;
-        const u32 lanes = min((u32)PL, pj_end - first);
-        if (tid == 0) mbar_expect_tx(&bars[slot], lanes * cnt * TN * 8);
+    if (tid >= MAC_CONSUMERS) {
+        // ---------------- producer warp
+        const u32 lane = tid - MAC_CONSUMERS;
+        const size_t pt_term = (size_t)r * N, pt_pj = (size_t)n_terms * r * N;
+        if (lane == 0) mbar_expect_tx(xbar, n_terms * 2 * TN * 8);
         __syncwarp();
-        for (u32 e = tid; e < lanes * MAC_TS; e += 32) {           // one copy per (lane, term)
-            const u32 ll = e / MAC_TS, ts = e % MAC_TS;
-            if (ts < cnt) {
-                const u64* src = pt + (size_t)(first + ll) * pt_pj + (size_t)(t0 + ts) * pt_term + (size_t)i * N + n0;
-                bulk_g2s(ring + (size_t)slot * MAC_STAGE_WORDS + ((size_t)ll * MAC_TS + ts) * TN, src, TN * 8,
-                         &bars[slot]);
+        for (u32 e = lane; e < n_terms * 2; e += 32)                // X tile: [term][component] segments
+            bulk_g2s(xs + (size_t)e * TN, x + ((size_t)e * r + i) * N + n0, TN * 8, xbar);
+        u32 g = 0, ch = 0, slot = 0, phase = 0;
+        for (u32 k = 0; k < n_items; ++k) {
+            if (k >= (u32)MAC_STAGES) mbar_wait(&empty[slot], phase ^ 1, error_flag);   // consumers left this slot
+            const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
+            const u32 first = pj_begin + g * PL;
+            const u32 lanes = min((u32)PL, pj_end - first);
+            if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * 8);
+            __syncwarp();
+            for (u32 e = lane; e < lanes * MAC_TS; e += 32) {        // one copy per (group lane, term)
+                const u32 ll = e / MAC_TS, ts = e % MAC_TS;
+                if (ts < cnt) {
+                    const u64* src = pt + (size_t)(first + ll) * pt_pj + (size_t)(t0 + ts) * pt_term + (size_t)i * N + n0;
+                    bulk_g2s(ring + (size_t)slot * MAC_STAGE_WORDS + ((size_t)ll * MAC_TS + ts) * TN, src, TN * 8,
+                             &full[slot]);
+                }
             }
+            if (++ch == n_chunks) { ch = 0; ++g; }
+            if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
         }
-    };
-
-    u32 ig = 0, ich = 0, islot = 0, issued = 0;                     // next item to issue (warp 0 only)
-    auto issue_next = [&]() {
-        issue(ig, ich, islot);
-        ++issued;
-        if (++ich == n_chunks) { ich = 0; ++ig; }
-        if (++islot == MAC_STAGES) islot = 0;
-    };
-    if (tid < 32) {
-        if (tid == 0) mbar_expect_tx(&bars[MAC_STAGES], n_terms * 2 * TN * 8);
-        __syncwarp();
-        for (u32 e = tid; e < n_terms * 2; e += 32)                 // X tile: [term][component] segments
-            bulk_g2s(xs + (size_t)e * TN, x + ((size_t)e * r + i) * N + n0, TN * 8, &bars[MAC_STAGES]);
-        while (issued < (u32)MAC_STAGES - 1 && issued < n_items) issue_next();
+        return;
     }
-    mbar_wait(&bars[MAC_STAGES], 0, error_flag);
 
-    LimbAcc<SMALL> acc0, acc1;
+    // ---------------- consumer warps
+    const u32 c = tid & (TN - 1), l = tid >> LOG_TN;
+    const u64 q = R.q[i];
+    const u32 qneg32 = (u32)R.qneg[i];
+    mbar_wait(xbar, 0, error_flag);
+    if (KARA) {
+        // split the resident X words into limbs, each exactly once, then let every consumer see them
+        for (u32 e = l; e < n_terms * 2; e += PL) xs[(size_t)e * TN + c] = limb_split(xs[(size_t)e * TN + c], KARA_L);
+        asm volatile("bar.sync 1, %0;" ::"n"(MAC_CONSUMERS) : "memory");
+    }
+    KaraAcc k0, k1;
+    LimbAcc<false> a0, a1;
     u32 since_flush = 0, g = 0, ch = 0, slot = 0, phase = 0;
     for (u32 k = 0; k < n_items; ++k) {
-        if (tid < 32 && issued < n_items) issue_next();   // into the slot everyone left at the end of item k-1
         const u32 pj = pj_begin + g * PL + l;
         const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
-        mbar_wait(&bars[slot], phase, error_flag);
+        mbar_wait(&full[slot], phase, error_flag);
         if (pj < pj_end) {
             const u64* ps = ring + (size_t)slot * MAC_STAGE_WORDS + (size_t)l * MAC_TS * TN + c;
             const u64* xt = xs + (size_t)t0 * 2 * TN + c;
@@ -154,32 +177,56 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const u64* __restrict__ 
 #pragma unroll
                 for (int ts = 0; ts < MAC_TS; ++ts) {
                     const u64 w = ps[ts * TN];
-                    acc0.mac(w, xt[(ts * 2) * TN]);
-                    acc1.mac(w, xt[(ts * 2 + 1) * TN]);
+                    if (KARA) {
+                        const u32 w0 = (u32)w, w1 = (u32)(w >> 32), ws = w0 + w1;
+                        k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
+                        k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
+                    } else {
+                        a0.mac(w, xt[(ts * 2) * TN]);
+                        a1.mac(w, xt[(ts * 2 + 1) * TN]);
+                    }
                 }
             } else {
                 for (u32 ts = 0; ts < cnt; ++ts) {
                     const u64 w = ps[ts * TN];
-                    acc0.mac(w, xt[(ts * 2) * TN]);
-                    acc1.mac(w, xt[(ts * 2 + 1) * TN]);
+                    if (KARA) {
+                        const u32 w0 = (u32)w, w1 = (u32)(w >> 32), ws = w0 + w1;
+                        k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
+                        k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
+                    } else {
+                        a0.mac(w, xt[(ts * 2) * TN]);
+                        a1.mac(w, xt[(ts * 2 + 1) * TN]);
+                    }
                 }
             }
+        }
+        __syncwarp();
+        if ((tid & 31) == 0) mbar_arrive(&empty[slot]);              // this warp is done with the slot
+        if (pj < pj_end) {
             since_flush += cnt;
             if (ch + 1 == n_chunks) {
-                // the cached plaintexts carry a factor 2^64, which the Montgomery reduction removes
                 u64* ap = a + ((size_t)pj * 2 * r + i) * N + n0 + c;
-                ap[0] = acc0.reduce_mont(q, qneg);
-                ap[(size_t)r * N] = acc1.reduce_mont(q, qneg);
-                acc0.reset_to(0);
-                acc1.reset_to(0);
+                if (KARA) {
+                    u64 H, L;
+                    k0.value(KARA_L, H, L);
+                    ap[0] = redc_2x32(H, L, q, qneg32);
+                    k1.value(KARA_L, H, L);
+                    ap[(size_t)r * N] = redc_2x32(H, L, q, qneg32);
+                    k0 = KaraAcc();
+                    k1 = KaraAcc();
+                } else {
+                    ap[0] = a0.reduce_mont(q, R.qneg[i]);
+                    ap[(size_t)r * N] = a1.reduce_mont(q, R.qneg[i]);
+                    a0.reset_to(0);
+                    a1.reset_to(0);
+                }
                 since_flush = 0;
-            } else if (since_flush + MAC_TS > lazy_terms) {   // keep the partial sums inside their words
-                acc0.reset_to(acc0.reduce(q, R.mu[i], R.c64[i], R.c64s[i]));
-                acc1.reset_to(acc1.reduce(q, R.mu[i], R.c64[i], R.c64s[i]));
+            } else if (!KARA && since_flush + MAC_TS > lazy_terms) {   // keep the partial sums inside their words
+                a0.reset_to(a0.reduce(q, R.mu[i], R.c64[i], R.c64s[i]));
+                a1.reset_to(a1.reduce(q, R.mu[i], R.c64[i], R.c64s[i]));
                 since_flush = 1;
             }
         }
-        __syncthreads();       // the slot may now be overwritten
         if (++ch == n_chunks) { ch = 0; ++g; }
         if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
     }
@@ -191,15 +238,21 @@ static int bits_of(u64 v) {
     return b;
 }
 
-template <bool SMALL, int LOG_TN>
+u32 mac_split_bits(const RingHost& ring) {
+    u64 qmax = 0;
+    for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
+    return bits_of(qmax) <= 50 ? KARA_L : 0;
+}
+
+template <bool KARA, int LOG_TN>
 static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
                                 u32 lazy, int* error_flag, cudaStream_t stream) {
-    constexpr u32 TN = 1u << LOG_TN, PL = MAC_THREADS >> LOG_TN;
-    const size_t smem = (size_t)MAC_STAGES * MAC_STAGE_WORDS * 8 + (size_t)n_terms * 2 * TN * 8 + (MAC_STAGES + 1) * 8;
+    constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
+    const size_t smem = (size_t)MAC_STAGES * MAC_STAGE_WORDS * 8 + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_STAGES + 1) * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
     static bool attr_set = false;     // opt in once to the large dynamic shared-memory carve-out
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(mac_kernel<SMALL, LOG_TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(mac_kernel<KARA, LOG_TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              200 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
@@ -214,8 +267,8 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const u64* 
     pj_per_block = (pj_per_block + PL - 1) / PL * PL;
     slices = (n_pj + pj_per_block - 1) / pj_per_block;
     dim3 grid(ring.dev.N >> LOG_TN, ring.dev.r, slices);
-    mac_kernel<SMALL, LOG_TN><<<grid, MAC_THREADS, smem, stream>>>(ring.dev, pt, x, a, n_terms, n_pj, pj_per_block, lazy,
-                                                                    error_flag);
+    mac_kernel<KARA, LOG_TN><<<grid, MAC_THREADS, smem, stream>>>(ring.dev, pt, x, a, n_terms, n_pj, pj_per_block, lazy,
+                                                                   error_flag);
     return cudaGetLastError();
 }
 
@@ -225,18 +278,22 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a
     ProfScope prof(ring.prof, CAT_MAC, stream);
     u64 qmax = 0;
     for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
-    const int qbits = bits_of(qmax);
     // tile width: the resident X tile (n_terms * 2 * TN words) must stay within 48 KB
     u32 log_tn = 8;
     while (log_tn > 4 && (size_t)n_terms * 2 * (1u << log_tn) * 8 > 48 * 1024) --log_tn;
-    const bool small = qbits <= 50;
-    // terms the lazy sums can take: limb partial sums inside their words, and the total below q * 2^64
-    u32 lazy = small ? (1u << (63 - qbits)) : 128u;
+    const bool kara = mac_split_bits(ring) != 0;
+    // terms a lazy sum can take: Karatsuba's middle sum grows by < 2^52 per term; the whole-word
+    // path is limited by its high partial sum and by the total staying below q * 2^64
+    u32 lazy = 128u;
     const u64 by_q = (~(u64)0) / qmax;
     if ((u64)lazy > by_q - 1) lazy = (u32)(by_q - 1);
-    if (lazy < MAC_TS) return cudaErrorInvalidValue;
+    if (kara) {
+        if (n_terms > 4000) return cudaErrorInvalidValue;
+    } else if (lazy < (u32)MAC_TS) {
+        return cudaErrorInvalidValue;
+    }
 #define BF_MAC(S, L) launch_mac_t<S, L>(ring, pt, x, a, n_pj, n_terms, lazy, error_flag, stream)
-    if (small) {
+    if (kara) {
         switch (log_tn) {
             case 8: return BF_MAC(true, 8);
             case 7: return BF_MAC(true, 7);

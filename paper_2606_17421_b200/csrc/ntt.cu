@@ -251,6 +251,10 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
                 if (v >= q) v -= q;
                 e[i] = v;
             }
+            if (B.split_bits) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) e[i] = limb_split(e[i], B.split_bits);
+            }
             ulonglong2* gp = (ulonglong2*)(gdst + 4 * s);
             gp[0] = make_ulonglong2(e[0], e[1]);
             gp[1] = make_ulonglong2(e[2], e[3]);
@@ -263,6 +267,10 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             const ulonglong2* gp = (const ulonglong2*)(gsrc + 4 * s);
             const ulonglong2 a = gp[0], b = gp[1];
             e[0] = a.x; e[1] = a.y; e[2] = b.x; e[3] = b.y;
+            if (B.split_bits) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) e[i] = limb_join(e[i], B.split_bits);
+            }
             set_butterflies<2, false>(e, tw, 64u * mult, (u32)s, q);
 #pragma unroll
             for (int i = 0; i < 4; ++i) sm[swz(4 * s + i)] = e[i];
