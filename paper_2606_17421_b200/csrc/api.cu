@@ -76,7 +76,9 @@ struct DevBuf {
 
 struct bf_weights {
     u32 d_out, d_in, n_in, n_out;
-    u64* pt;            // [g][n_out][n_in][b][r][N], NTT domain, Montgomery form (times 2^64 mod q_i)
+    u64* pt;            // groups pj = j*n_out + p of terms t = q*b + k in the tile-major layout `lay`;
+                        // NTT domain, Montgomery form (times 2^64 mod q_i), limbs split when the primes allow
+    TileLayout lay;
     size_t bytes;
 };
 
@@ -99,7 +101,7 @@ struct bf_ctx {
     u32* perms = nullptr;
     u32 n_keys = 0;
     // scratch (grow-only)
-    DevBuf X, Dig, U, Tc, Tn, Cc, A, Rres, Y, fft, coef, ptjit, stage_in, stage_out, nm_a, nm_b;
+    DevBuf X, Dig, U, Tc, Tn, Cc, A, Rres, Y, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
     u64 cache_budget = 0, cache_used = 0;
     std::vector<bf_weights*> weights;
     std::string cuda_msg;
@@ -317,7 +319,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
         }
     }
     DevBuf* bufs[] = {&ctx->X, &ctx->Dig, &ctx->U, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres, &ctx->Y,
-                      &ctx->fft, &ctx->coef, &ctx->ptjit, &ctx->stage_in, &ctx->stage_out, &ctx->nm_a, &ctx->nm_b};
+                      &ctx->fft, &ctx->coef, &ctx->ptnat, &ctx->ptjit, &ctx->stage_in, &ctx->stage_out, &ctx->nm_a, &ctx->nm_b};
     for (DevBuf* b : bufs) free_buf(*b);
     cudaFree(ctx->tw_fwd);
     cudaFree(ctx->tw_inv);
@@ -393,17 +395,20 @@ static u32 cdiv(u32 a, u32 b) { return (a + b - 1) / b; }
 
 extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
     if (!ctx) return 0;
-    const u64 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = cdiv(d_out, ctx->plan.tile_D);
-    const u64 M = ctx->plan.tile_D / ctx->plan.tau;
-    return n_in * n_out * M * ctx->r * ctx->N * sizeof(u64);
+    const u32 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = cdiv(d_out, ctx->plan.tile_D);
+    const TileLayout lay = mac_tile_layout(ctx->ring, n_out * ctx->plan.bsgs_g, n_in * ctx->plan.bsgs_b);
+    return mac_tile_words(ctx->ring, lay) * sizeof(u64);
 }
 
-// Encode diagonals [d0, d0 + count) of W (order [j][p][q][k]) into dst (NTT domain, [count][r][N]).
-static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0, u32 count, u64* dst) {
+// Encode diagonals [d0, d0 + count) of W (order [j][p][q][k], i.e. group pj = d / n_terms, term d % n_terms)
+// into dst in the tile-major layout `lay`, whose group 0 is group pj0 of W.
+static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0, u32 count, u64* dst,
+                        const TileLayout& lay, u32 pj0) {
     const u32 N = ctx->N, r = ctx->r, n = N / 2;
-    const u32 chunk = 64;
+    const u32 chunk = 32;
     TRY(ensure(ctx, ctx->fft, (size_t)chunk * n * sizeof(double2)));
     TRY(ensure(ctx, ctx->coef, (size_t)chunk * N * sizeof(i64)));
+    TRY(ensure(ctx, ctx->ptnat, (size_t)chunk * r * N * sizeof(u64)));
     EncodeTables tab;
     tab.slot_of_pos = ctx->slot_of_pos;
     tab.T = ctx->T;
@@ -427,7 +432,7 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
         PolyBatch B;
         memset(&B, 0, sizeof(B));
         B.src = ctx->coef.p;
-        B.dst = dst + (size_t)lo * r * N;
+        B.dst = (u64*)ctx->ptnat.p;                 // first pass lands here; the second writes the tiles
         B.src_so = N;
         B.src_sm = 0;
         B.dst_so = (long long)r * N;
@@ -436,6 +441,10 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
         B.mod0 = 0;
         B.mod_step = 1;
         B.split_bits = mac_split_bits(ctx->ring);
+        B.tile_ptr = dst;
+        B.tile = lay;
+        B.tile_pj0 = pj0;
+        B.o_base = d0 + lo;
         CK(ntt_forward(ctx->ring, B, cnt, LOAD_I64_MONT, ctx->stream));   // cached form: NTT domain, times 2^64
     }
     return BF_OK;
@@ -464,6 +473,7 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
     w->n_in = cdiv(d_in, ctx->plan.tile_D);
     w->n_out = cdiv(d_out, ctx->plan.tile_D);
     w->bytes = bytes;
+    w->lay = mac_tile_layout(ctx->ring, w->n_out * ctx->plan.bsgs_g, w->n_in * ctx->plan.bsgs_b);
     cudaError_t e = cudaMalloc(&w->pt, bytes);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -471,7 +481,12 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
         return BF_ERR_OOM;
     }
     const u32 n_diag = w->n_in * w->n_out * (ctx->plan.tile_D / ctx->plan.tau);
-    int s = encode_range(ctx, W, d_out, d_in, 0, n_diag, w->pt);
+    int s = BF_OK;
+    {   // padding words of the layout are never read, but keep the allocation defined
+        cudaError_t me = cudaMemsetAsync(w->pt, 0, bytes, ctx->stream);
+        if (me != cudaSuccess) s = BF_ERR_CUDA;
+    }
+    if (s == BF_OK) s = encode_range(ctx, W, d_out, d_in, 0, n_diag, w->pt, w->lay, 0);
     if (s == BF_OK) s = check_overflow(ctx);
     if (s != BF_OK) {
         cudaStreamSynchronize(ctx->stream);
@@ -663,19 +678,21 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     // ---- multiply-accumulate over the encoded diagonals
     const u32 n_terms = n_in * b, n_pj = n_out * g;
     if (pt_weights) {
-        CK(launch_mac(ctx->ring, pt_weights->pt, X, A, n_pj, n_terms, ctx->device_error, ctx->stream));
+        CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, A, n_pj, n_terms, ctx->device_error, ctx->stream));
     } else {
         // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them
         const size_t group_bytes = (size_t)n_terms * r * N * 8;
         u32 groups = (u32)(((size_t)1 << 30) / group_bytes);
         if (groups < 1) groups = 1;
         if (groups > n_pj) groups = n_pj;
-        TRY(ensure(ctx, ctx->ptjit, group_bytes * groups));
+        const TileLayout jl = mac_tile_layout(ctx->ring, groups, n_terms);
+        TRY(ensure(ctx, ctx->ptjit, mac_tile_words(ctx->ring, jl) * 8));
         for (u32 pj0 = 0; pj0 < n_pj; pj0 += groups) {
             const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
-            TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p));
-            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, X, A + (size_t)pj0 * ctw, cnt, n_terms, ctx->device_error,
-                          ctx->stream));
+            const TileLayout cl = mac_tile_layout(ctx->ring, cnt, n_terms);
+            TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p, cl, pj0));
+            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, cl, X, A + (size_t)pj0 * ctw, cnt, n_terms,
+                          ctx->device_error, ctx->stream));
         }
     }
     stamp(ctx, 2);
@@ -849,7 +866,7 @@ extern "C" int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, u
     const size_t d = (((size_t)j * w->n_out + p) * w->n_in + q) * ctx->plan.bsgs_b + k;
     PolyBatch B;
     memset(&B, 0, sizeof(B));
-    B.src = w->pt + d * r * N;
+    B.src = out;                                 // unused: the first pass reads the tiles
     B.dst = out;
     B.src_so = B.dst_so = (long long)r * N;
     B.src_sm = B.dst_sm = N;
@@ -857,6 +874,10 @@ extern "C" int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, u
     B.mod_step = 1;
     B.from_mont = 1;
     B.split_bits = mac_split_bits(ctx->ring);
+    B.tile_ptr = w->pt;
+    B.tile = w->lay;
+    B.tile_pj0 = 0;
+    B.o_base = (u32)d;
     CK(ntt_inverse(ctx->ring, B, 1, ctx->stream));
     return BF_OK;
 }

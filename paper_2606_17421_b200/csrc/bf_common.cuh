@@ -153,6 +153,26 @@ enum LoadMode : int {
     LOAD_I64_MONT = 4,  // LOAD_I64, then times 2^64 mod q: the transform's output is in Montgomery form
 };
 
+// Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks
+// each stream one contiguous region:  word (group pj, term t, prime i, coefficient n) lives at
+//   (((((i*ntiles + n/TN)*G + pj/PL)*C + t/TS)*PL + pj%PL)*TS + t%TS)*TN + n%TN
+// with TN = 2^log_tn coefficients per tile, PL = 256/TN group lanes, TS = 8 terms per stage,
+// G = ceil(n_pj/PL), C = ceil(n_terms/TS).  One stage (fixed i, tile, pj/PL, t/TS) is 16 KB.
+struct TileLayout {
+    u32 log_tn, n_terms, n_pj, G, C, ntiles;
+};
+constexpr u32 TILE_TS = 8;
+constexpr u32 TILE_STAGE_WORDS = 2048;
+
+__host__ __device__ __forceinline__ size_t tile_stage_offset(const TileLayout& t, u32 i, u32 tile, u32 g, u32 ch) {
+    return ((((size_t)i * t.ntiles + tile) * t.G + g) * t.C + ch) * TILE_STAGE_WORDS;
+}
+__host__ __device__ __forceinline__ size_t tile_word_offset(const TileLayout& t, u32 pj, u32 term, u32 i, u32 n) {
+    const u32 TN = 1u << t.log_tn, PL = 256u >> t.log_tn;
+    return tile_stage_offset(t, i, n >> t.log_tn, pj / PL, term / TILE_TS) +
+           ((size_t)(pj % PL) * TILE_TS + term % TILE_TS) * TN + (n & (TN - 1));
+}
+
 // A batch of equally sized polynomials addressed as (outer index o, slot m):
 //   source  = src + o*src_so + m*src_sm      destination = dst + o*dst_so + m*dst_sm
 //   modulus index of polynomial (o, m) = mod0 + m*mod_step
@@ -164,6 +184,9 @@ struct PolyBatch {
     u32 n_m, mod0, mod_step;
     u64 lift_mod;                 // LOAD_CENTRED: the modulus M the source residues live in
     u32 from_mont;                // inverse transform only: input is in Montgomery form, output is not
+    u64* tile_ptr;                // non-null: the NTT-domain side lives there in the tile-major layout `tile`
+    TileLayout tile;              //   (forward writes its final result there, inverse reads its input there);
+    u32 tile_pj0, o_base;         //   diagonal o_base + o = pj*n_terms + t; the layout's group 0 is group tile_pj0
     u32 split_bits;               // L > 0: the NTT-domain side of the transform is stored as two L-bit-aligned
                                   // limbs per word, (v >> L) << 32 | (v & (2^L - 1)); forward writes, inverse reads it
 };

@@ -72,8 +72,10 @@ cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, cons
                                   long long out_stride, cudaStream_t stream);
 // A[pj][comp][i][n] = sum_{t < n_terms} Pt[pj][t][i][n] * X[t][comp][i][n],  pj = j*n_out + p, t = q*b + k
 u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintext format (0 = whole words)
-cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
-                       int* error_flag, cudaStream_t stream);
+TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms);   // layout of n_pj groups of n_terms diagonals
+size_t mac_tile_words(const RingHost& ring, const TileLayout& t);           // words that layout occupies
+cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
+                       u32 n_terms, int* error_flag, cudaStream_t stream);
 // y[p] = a[p] + sum_{j=1}^{g-1} rres[(j-1)*n_out + p]   (ciphertexts of [2][r][N] words)
 cudaError_t launch_giant_sum(const RingHost& ring, const u64* a, const u64* rres, u64* y, u32 n_out, u32 g,
                              cudaStream_t stream);

@@ -88,15 +88,15 @@ __device__ __forceinline__ void mbar_arrive(u64* bar) {
 // reduction per output word removes the 2^64.
 constexpr int MAC_CONSUMERS = 256;
 constexpr int MAC_THREADS = MAC_CONSUMERS + 32;   // + one producer warp
-constexpr int MAC_TS = 8;                         // terms per stage
+constexpr int MAC_TS = (int)TILE_TS;              // terms per stage
 constexpr int MAC_STAGES = 4;
 constexpr int MAC_STAGE_WORDS = MAC_TS * MAC_CONSUMERS;   // 16 KB per stage whatever TN is
 constexpr u32 KARA_L = 25;
 
 template <bool KARA, int LOG_TN>
 __global__ void __launch_bounds__(MAC_THREADS, 2)
-mac_kernel(const RingDev R, const u64* __restrict__ pt, const u64* __restrict__ x, u64* __restrict__ a, u32 n_terms,
-           u32 n_pj, u32 pj_per_block, u32 lazy_terms, int* __restrict__ error_flag) {
+mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, const u64* __restrict__ x,
+           u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, int* __restrict__ error_flag) {
     extern __shared__ __align__(128) unsigned char mac_smem[];
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     u64* ring = (u64*)mac_smem;                                    // [MAC_STAGES][PL][MAC_TS][TN]
@@ -126,7 +126,6 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const u64* __restrict__ 
     if (tid >= MAC_CONSUMERS) {
         // ---------------- producer warp
         const u32 lane = tid - MAC_CONSUMERS;
-        const size_t pt_term = (size_t)r * N, pt_pj = (size_t)n_terms * r * N;
         if (lane == 0) mbar_expect_tx(xbar, n_terms * 2 * TN * 8);
         __syncwarp();
         for (u32 e = lane; e < n_terms * 2; e += 32)                // X tile: [term][component] segments
@@ -137,15 +136,16 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const u64* __restrict__ 
             const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
             const u32 first = pj_begin + g * PL;
             const u32 lanes = min((u32)PL, pj_end - first);
+            // the stage is one contiguous 16 KB block of the tile-major layout; when its tail is
+            // padding (last group round or last term chunk) copy the valid part of every lane only
+            const u64* stage = pt + tile_stage_offset(lay, i, blockIdx.x, first / PL, ch);
+            u64* sdst = ring + (size_t)slot * MAC_STAGE_WORDS;
             if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * 8);
             __syncwarp();
-            for (u32 e = lane; e < lanes * MAC_TS; e += 32) {        // one copy per (group lane, term)
-                const u32 ll = e / MAC_TS, ts = e % MAC_TS;
-                if (ts < cnt) {
-                    const u64* src = pt + (size_t)(first + ll) * pt_pj + (size_t)(t0 + ts) * pt_term + (size_t)i * N + n0;
-                    bulk_g2s(ring + (size_t)slot * MAC_STAGE_WORDS + ((size_t)ll * MAC_TS + ts) * TN, src, TN * 8,
-                             &full[slot]);
-                }
+            if (lanes == PL && cnt == (u32)MAC_TS) {
+                if (lane == 0) bulk_g2s(sdst, stage, MAC_STAGE_WORDS * 8, &full[slot]);
+            } else if (lane < lanes) {
+                bulk_g2s(sdst + (size_t)lane * MAC_TS * TN, stage + (size_t)lane * MAC_TS * TN, cnt * TN * 8, &full[slot]);
             }
             if (++ch == n_chunks) { ch = 0; ++g; }
             if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
@@ -238,6 +238,29 @@ static int bits_of(u64 v) {
     return b;
 }
 
+// tile width: the resident X tile (n_terms * 2 * TN words) must stay within 48 KB
+static u32 mac_log_tn(u32 n_terms) {
+    u32 log_tn = 8;
+    while (log_tn > 4 && (size_t)n_terms * 2 * (1u << log_tn) * 8 > 48 * 1024) --log_tn;
+    return log_tn;
+}
+
+TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms) {
+    TileLayout t;
+    t.log_tn = mac_log_tn(n_terms);
+    const u32 PL = 256u >> t.log_tn;
+    t.n_terms = n_terms;
+    t.n_pj = n_pj;
+    t.G = (n_pj + PL - 1) / PL;
+    t.C = (n_terms + TILE_TS - 1) / TILE_TS;
+    t.ntiles = ring.dev.N >> t.log_tn;
+    return t;
+}
+
+size_t mac_tile_words(const RingHost& ring, const TileLayout& t) {
+    return (size_t)ring.dev.r * t.ntiles * t.G * t.C * TILE_STAGE_WORDS;
+}
+
 u32 mac_split_bits(const RingHost& ring) {
     u64 qmax = 0;
     for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
@@ -245,8 +268,8 @@ u32 mac_split_bits(const RingHost& ring) {
 }
 
 template <bool KARA, int LOG_TN>
-static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
-                                u32 lazy, int* error_flag, cudaStream_t stream) {
+static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a,
+                                u32 n_pj, u32 n_terms, u32 lazy, int* error_flag, cudaStream_t stream) {
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     const size_t smem = (size_t)MAC_STAGES * MAC_STAGE_WORDS * 8 + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_STAGES + 1) * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
@@ -267,20 +290,19 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const u64* 
     pj_per_block = (pj_per_block + PL - 1) / PL * PL;
     slices = (n_pj + pj_per_block - 1) / pj_per_block;
     dim3 grid(ring.dev.N >> LOG_TN, ring.dev.r, slices);
-    mac_kernel<KARA, LOG_TN><<<grid, MAC_THREADS, smem, stream>>>(ring.dev, pt, x, a, n_terms, n_pj, pj_per_block, lazy,
-                                                                   error_flag);
+    mac_kernel<KARA, LOG_TN><<<grid, MAC_THREADS, smem, stream>>>(ring.dev, pt, lay, x, a, n_terms, n_pj, pj_per_block,
+                                                                   lazy, error_flag);
     return cudaGetLastError();
 }
 
-cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a, u32 n_pj, u32 n_terms,
-                       int* error_flag, cudaStream_t stream) {
+cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
+                       u32 n_terms, int* error_flag, cudaStream_t stream) {
     if (n_pj == 0) return cudaSuccess;
+    if (lay.n_pj != n_pj || lay.n_terms != n_terms) return cudaErrorInvalidValue;
     ProfScope prof(ring.prof, CAT_MAC, stream);
     u64 qmax = 0;
     for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
-    // tile width: the resident X tile (n_terms * 2 * TN words) must stay within 48 KB
-    u32 log_tn = 8;
-    while (log_tn > 4 && (size_t)n_terms * 2 * (1u << log_tn) * 8 > 48 * 1024) --log_tn;
+    const u32 log_tn = lay.log_tn;
     const bool kara = mac_split_bits(ring) != 0;
     // terms a lazy sum can take: Karatsuba's middle sum grows by < 2^52 per term; the whole-word
     // path is limited by its high partial sum and by the total staying below q * 2^64
@@ -292,7 +314,7 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const u64* x, u64* a
     } else if (lazy < (u32)MAC_TS) {
         return cudaErrorInvalidValue;
     }
-#define BF_MAC(S, L) launch_mac_t<S, L>(ring, pt, x, a, n_pj, n_terms, lazy, error_flag, stream)
+#define BF_MAC(S, L) launch_mac_t<S, L>(ring, pt, lay, x, a, n_pj, n_terms, lazy, error_flag, stream)
     if (kara) {
         switch (log_tn) {
             case 8: return BF_MAC(true, 8);

@@ -256,6 +256,9 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
                 for (int i = 0; i < 4; ++i) e[i] = limb_split(e[i], B.split_bits);
             }
             ulonglong2* gp = (ulonglong2*)(gdst + 4 * s);
+            if (B.tile_ptr)     // 4 adjacent coefficients never straddle a tile (tiles hold >= 16)
+                gp = (ulonglong2*)(B.tile_ptr + tile_word_offset(B.tile, (B.o_base + o) / B.tile.n_terms - B.tile_pj0,
+                                                                 (B.o_base + o) % B.tile.n_terms, mod, chunk * LEN + 4 * s));
             gp[0] = make_ulonglong2(e[0], e[1]);
             gp[1] = make_ulonglong2(e[2], e[3]);
         }
@@ -265,6 +268,10 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
             const ulonglong2* gp = (const ulonglong2*)(gsrc + 4 * s);
+            if (B.tile_ptr)
+                gp = (const ulonglong2*)(B.tile_ptr + tile_word_offset(B.tile, (B.o_base + o) / B.tile.n_terms - B.tile_pj0,
+                                                                       (B.o_base + o) % B.tile.n_terms, mod,
+                                                                       chunk * LEN + 4 * s));
             const ulonglong2 a = gp[0], b = gp[1];
             e[0] = a.x; e[1] = a.y; e[2] = b.x; e[3] = b.y;
             if (B.split_bits) {
