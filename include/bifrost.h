@@ -37,7 +37,8 @@ enum {
     BF_ERR_MISSING_KEY = -5,   /* the plan needs a rotation whose key was not loaded */
     BF_ERR_OOM = -6,           /* encoded weights exceed the cache budget, or device memory is exhausted */
     BF_ERR_CUDA = -7,          /* a CUDA call failed; see bf_last_cuda_error() */
-    BF_ERR_RANGE = -8          /* an encoded coefficient does not fit 2^62 (scale too large for the data) */
+    BF_ERR_RANGE = -8,         /* an encoded coefficient does not fit 2^62 (scale too large for the data) */
+    BF_ERR_TOO_LARGE = -9      /* more work than the fixed scratch of an allocation-free entry point holds */
 };
 
 typedef struct bf_ctx bf_ctx;          /* ring tables, rotation keys, scratch memory */
@@ -128,6 +129,25 @@ int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uint64_t* ct_o
  * basis prime (t mod (r+1)); all device, [n_polys][N], coefficient domain.  Exercises the forward
  * and inverse transforms.  Asynchronous. */
 int bf_negacyclic_mul(bf_ctx* ctx, const uint64_t* a, const uint64_t* b, uint64_t* out, uint32_t n_polys);
+
+/* bf_negacyclic_mul for callers that must not allocate.  (No counterpart in the paper: this is a
+ * deployment convenience of the library.)
+ * Who needs it: a host program that has handed all device memory to its own pool, or that calls
+ * from a latency-critical loop, cannot tolerate the cudaMalloc (and the device-wide
+ * synchronisation that comes with it) by which bf_negacyclic_mul grows its scratch on first use.
+ * This entry point performs no cudaMalloc, cudaFree or other allocating call.  Its two
+ * transform-domain temporaries live in a fixed array inside the library's device image, which
+ * every GPU that loads the library holds (8 MiB) until the process exits.
+ *   Limit: ceil(n_polys / (r+1)) * (r+1) * N <= bf_noalloc_max_words() (2^19 words); larger
+ *   requests return BF_ERR_TOO_LARGE and enqueue nothing.
+ *   The first call on a device resolves the array's device address (cudaGetSymbolAddress); make
+ *   that call with the context's device current and before starting any stream capture.
+ *   All calls, from any context, share the one array, which keeps the previous call's contents;
+ *   the part a call uses is overwritten or cleared by that call.  Two calls whose work overlaps on
+ *   the GPU (different streams) race on it: serialise them.
+ * Arguments, layout, results and asynchrony are those of bf_negacyclic_mul. */
+int bf_negacyclic_mul_noalloc(bf_ctx* ctx, const uint64_t* a, const uint64_t* b, uint64_t* out, uint32_t n_polys);
+uint64_t bf_noalloc_max_words(void);
 
 /* Coefficient-domain residues [r][N] (device) of the encoded plaintext Pt[p][q][j][k] held by w. */
 int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, uint32_t q, uint32_t j, uint32_t k,

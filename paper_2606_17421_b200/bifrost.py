@@ -21,6 +21,7 @@ BF_ERR_MISSING_KEY = -5
 BF_ERR_OOM = -6
 BF_ERR_CUDA = -7
 BF_ERR_RANGE = -8
+BF_ERR_TOO_LARGE = -9
 
 
 class bf_plan(ctypes.Structure):
@@ -54,6 +55,8 @@ _SIGNATURES = {
     "bf_linear_host": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
     "bf_rotate": (ctypes.c_int, [_vp, _vp, _u32, _vp]),
     "bf_negacyclic_mul": (ctypes.c_int, [_vp, _vp, _vp, _vp, _u32]),
+    "bf_negacyclic_mul_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _u32]),
+    "bf_noalloc_max_words": (_u64, []),
     "bf_weights_export": (ctypes.c_int, [_vp, _vp, _u32, _u32, _u32, _u32, _vp]),
     "bf_set_stage_timing": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_get_stage_ms": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float)]),
@@ -175,6 +178,15 @@ def bf_rotate(ctx, ct_in, steps: int, ct_out):
 
 def bf_negacyclic_mul(ctx, a, b, out, n_polys: int):
     _check(load().bf_negacyclic_mul(ctx, _ptr(a), _ptr(b), _ptr(out), n_polys), "bf_negacyclic_mul", ctx)
+
+
+def bf_negacyclic_mul_noalloc(ctx, a, b, out, n_polys: int):
+    """bf_negacyclic_mul without any device allocation: scratch is a fixed array in the library image."""
+    _check(load().bf_negacyclic_mul_noalloc(ctx, _ptr(a), _ptr(b), _ptr(out), n_polys), "bf_negacyclic_mul_noalloc", ctx)
+
+
+def bf_noalloc_max_words() -> int:
+    return load().bf_noalloc_max_words()
 
 
 def bf_weights_export(ctx, w, p: int, q: int, j: int, k: int, out):

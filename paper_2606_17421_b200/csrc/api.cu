@@ -155,6 +155,7 @@ extern "C" const char* bf_strerror(int code) {
         case BF_ERR_OOM: return "out of memory or over the cache budget";
         case BF_ERR_CUDA: return "CUDA error";
         case BF_ERR_RANGE: return "encoded coefficient out of range";
+        case BF_ERR_TOO_LARGE: return "request exceeds the fixed capacity of the allocation-free entry point";
         default: return "unknown error";
     }
 }
@@ -954,5 +955,77 @@ extern "C" int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out) {
     cudaEventDestroy(a);
     cudaEventDestroy(b);
     *mad_per_second_out = best;
+    return BF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of bf_negacyclic_mul.
+//
+// bf_negacyclic_mul keeps its two transform-domain operands in scratch memory that the context
+// obtains from cudaMalloc on first use.  A caller whose device memory is entirely owned by its own
+// pool (a serving engine that reserved the whole GPU up front), or that sits on a latency path
+// where the implicit device synchronisation of cudaMalloc is unacceptable, cannot afford that.
+// This variant uses a fixed array that lives in the library's device image instead: every GPU that
+// loads the library holds BF_NOALLOC_BYTES of it until the process exits.
+constexpr size_t BF_NOALLOC_WORDS = (size_t)1 << 19;          // per operand: 4 MiB; 8 MiB in total
+static __device__ __align__(256) unsigned long long g_noalloc_scratch[2 * BF_NOALLOC_WORDS];
+// The array's name is only a host-side handle.  Its device address is looked up once per device,
+// with that device current, and cached here.
+static u64* g_noalloc_addr[64] = {nullptr};
+
+extern "C" uint64_t bf_noalloc_max_words(void) { return (uint64_t)BF_NOALLOC_WORDS; }
+
+extern "C" int bf_negacyclic_mul_noalloc(bf_ctx* ctx, const uint64_t* a, const uint64_t* b, uint64_t* out,
+                                         uint32_t n_polys) {
+    if (!ctx || !a || !b || !out || !n_polys) return BF_ERR_INVALID_ARG;
+    const u32 N = ctx->N, nb = ctx->r + 1;
+    const u32 n_outer = cdiv(n_polys, nb);
+    const size_t words = (size_t)n_outer * nb * N;               // batch padded to whole groups of r+1 primes
+    if (words > BF_NOALLOC_WORDS) return BF_ERR_TOO_LARGE;
+    int dev = -1;
+    CK(cudaGetDevice(&dev));
+    if (dev != ctx->device || dev < 0 || dev >= 64) return BF_ERR_INVALID_ARG;
+    if (!g_noalloc_addr[dev]) {                                  // first call on this device: set-up
+        void* p = nullptr;
+        CK(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        g_noalloc_addr[dev] = (u64*)p;
+    }
+    u64* sa = g_noalloc_addr[dev];
+    u64* sb = sa + BF_NOALLOC_WORDS;
+    // The array keeps whatever the previous call left; the padding polynomials of this batch are
+    // transformed along with the real ones, so give them defined contents.
+    const size_t used = (size_t)n_polys * N;
+    if (words > used) {
+        CK(cudaMemsetAsync(sa + used, 0, (words - used) * 8, ctx->stream));
+        CK(cudaMemsetAsync(sb + used, 0, (words - used) * 8, ctx->stream));
+    }
+    CK(cudaMemcpyAsync(sa, a, used * 8, cudaMemcpyDeviceToDevice, ctx->stream));
+    CK(cudaMemcpyAsync(sb, b, used * 8, cudaMemcpyDeviceToDevice, ctx->stream));
+    Profiler* saved = ctx->ring.prof;      // launch timing would create events; keep this path free of that
+    ctx->ring.prof = nullptr;
+    PolyBatch B;
+    memset(&B, 0, sizeof(B));
+    B.src_so = B.dst_so = (long long)nb * N;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = nb;
+    B.mod_step = 1;
+    cudaError_t e;
+    B.src = sa;
+    B.dst = sa;
+    e = ntt_forward(ctx->ring, B, n_outer, LOAD_PLAIN, ctx->stream);
+    if (e == cudaSuccess) {
+        B.src = sb;
+        B.dst = sb;
+        e = ntt_forward(ctx->ring, B, n_outer, LOAD_PLAIN, ctx->stream);
+    }
+    if (e == cudaSuccess) e = launch_pointwise_mul(ctx->ring, sa, sb, sa, n_outer * nb, nb, 0, ctx->stream);
+    if (e == cudaSuccess) {
+        B.src = sa;
+        B.dst = sa;
+        e = ntt_inverse(ctx->ring, B, n_outer, ctx->stream);
+    }
+    ctx->ring.prof = saved;
+    CK(e);
+    CK(cudaMemcpyAsync(out, sa, used * 8, cudaMemcpyDeviceToDevice, ctx->stream));
     return BF_OK;
 }
