@@ -98,7 +98,7 @@ struct bf_ctx {
     // rotation keys
     std::map<u32, int> key_of_steps;
     u64* keys = nullptr;
-    u32* perms = nullptr;
+    u32* perms = nullptr;            // [n_keys][N] pinv: where position n goes under the key's automorphism
     u32 n_keys = 0;
     // scratch (grow-only)
     DevBuf X, Dig, U, Tc, Tn, Cc, A, Rres, Y, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
@@ -356,19 +356,28 @@ extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_
     e = cudaMalloc(&ctx->perms, (size_t)n_keys * N * sizeof(u32));
     if (e != cudaSuccess) { cudaGetLastError(); ctx->perms = nullptr; return BF_ERR_OOM; }
     // permutation tables: position i of the transform holds the evaluation at psi^(2*brev(i)+1);
-    // a(X) -> a(X^g) maps it to the evaluation at exponent (2*brev(i)+1)*g mod 2N
-    std::vector<u32> perms((size_t)n_keys * N);
+    // a(X) -> a(X^g) maps it to the evaluation at exponent (2*brev(i)+1)*g mod 2N, so the rotated
+    // polynomial is out[i] = in[perm[i]].  The keys are stored as key'[perm[i]] = key[i], which lets
+    // the inner product run in the un-rotated index space; the rotation is applied at the very end
+    // as the scatter out[pinv[i]] = v'[i], pinv = perm^{-1}.  Only pinv stays on the device.
+    std::vector<u32> perms((size_t)n_keys * N), pinvs((size_t)n_keys * N);
     for (u32 t = 0; t < n_keys; ++t) {
         const u32 steps = rot_steps[t] % n;
         u64 g = 1;
         for (u32 s = 0; s < steps; ++s) g = (g * 5) % (2ull * N);
         for (u32 i = 0; i < N; ++i) {
             const u64 ex = ((2ull * h_brev(i, (int)ctx->logN) + 1) * g) % (2ull * N);
-            perms[(size_t)t * N + i] = h_brev((u32)((ex - 1) / 2), (int)ctx->logN);
+            const u32 pi = h_brev((u32)((ex - 1) / 2), (int)ctx->logN);
+            perms[(size_t)t * N + i] = pi;
+            pinvs[(size_t)t * N + pi] = i;
         }
         ctx->key_of_steps[steps] = (int)t;
     }
-    CK(cudaMemcpy(ctx->perms, perms.data(), perms.size() * sizeof(u32), cudaMemcpyHostToDevice));
+    u32* perm_dev = nullptr;
+    e = cudaMalloc(&perm_dev, perms.size() * sizeof(u32));
+    if (e != cudaSuccess) { cudaGetLastError(); return BF_ERR_OOM; }
+    CK(cudaMemcpy(perm_dev, perms.data(), perms.size() * sizeof(u32), cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(ctx->perms, pinvs.data(), pinvs.size() * sizeof(u32), cudaMemcpyHostToDevice));
     PolyBatch B;
     memset(&B, 0, sizeof(B));
     B.src = keys;
@@ -378,8 +387,20 @@ extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_
     B.n_m = nb;
     B.mod0 = 0;
     B.mod_step = 1;
-    CK(ntt_forward(ctx->ring, B, n_keys * r * 2, LOAD_REDUCE, ctx->stream));
-    CK(cudaStreamSynchronize(ctx->stream));
+    // The in-place first pass would race with the permuted store of the second pass, so transform
+    // the caller's array out of place: first pass into our buffer, permuted store into it too is not
+    // possible either.  Use a staging buffer for the natural-order transform.
+    u64* stage = nullptr;
+    e = cudaMalloc(&stage, key_words * n_keys * sizeof(u64));
+    if (e != cudaSuccess) { cudaGetLastError(); cudaFree(perm_dev); return BF_ERR_OOM; }
+    B.dst = stage;
+    B.scatter = nullptr;
+    cudaError_t ne = ntt_forward_split(ctx->ring, B, n_keys * r * 2, LOAD_REDUCE, ctx->keys, perm_dev, 2 * r, ctx->stream);
+    cudaError_t se = cudaStreamSynchronize(ctx->stream);
+    cudaFree(stage);
+    cudaFree(perm_dev);
+    CK(ne);
+    CK(se);
     ctx->n_keys = n_keys;
     return BF_OK;
 }
@@ -567,7 +588,10 @@ static int find_key(bf_ctx* ctx, u32 steps, int* key) {
 
 // Digits of c1 (coefficient domain, [r][N] with stride N) reduced into every prime of the extended
 // basis and transformed: dig[set][j][m] = NTT_m( c1_j mod m ).
-static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_sets, u64* dig) {
+// The digit in its own prime is the transform of c1 itself, which the caller already has
+// (c1_ntt + set*c1_ntt_stride, [r][N]): it is copied, not recomputed.
+static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_sets, u64* dig, const u64* c1_ntt,
+                 long long c1_ntt_stride) {
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
     PolyBatch B;
     memset(&B, 0, sizeof(B));
@@ -577,6 +601,9 @@ static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_s
     B.src_sm = 0;
     B.dst_sm = N;
     B.dst_so = (long long)nb * N;
+    B.skip_diag = 1;
+    B.diag_src = c1_ntt;
+    B.diag_so = c1_ntt_stride;
     if (set_stride == (long long)r * N || n_sets == 1) {
         B.src = c1_coeff;
         B.dst = dig;
@@ -586,6 +613,7 @@ static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_s
         for (u32 s = 0; s < n_sets; ++s) {
             B.src = c1_coeff + (size_t)s * set_stride;
             B.dst = dig + (size_t)s * r * nb * N;
+            B.diag_src = c1_ntt + (size_t)s * c1_ntt_stride;
             B.src_so = N;
             CK(ntt_forward(ctx->ring, B, r, LOAD_REDUCE, ctx->stream));
         }
@@ -660,7 +688,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         B.mod_step = 1;
         CK(ntt_forward(ctx->ring, B, 2, LOAD_PLAIN, ctx->stream));
         if (b > 1) {
-            TRY(modup(ctx, ct + (size_t)r * N, (long long)r * N, 1, Dig));
+            TRY(modup(ctx, ct + (size_t)r * N, (long long)r * N, 1, Dig, X0 + (size_t)r * N, 0));
             RotBatch rb;
             memset(&rb, 0, sizeof(rb));
             rb.n = (int)(b - 1);
@@ -670,7 +698,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
                 rb.c0[k - 1] = (int)(q * b);
                 rb.out[k - 1] = (int)(q * b + k);
             }
-            CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, ctx->perms, U, ctx->stream));
+            CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->stream));
             TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
         }
     }
@@ -713,7 +741,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         B.mod0 = 0;
         B.mod_step = 1;
         CK(ntt_inverse(ctx->ring, B, cnt, ctx->stream));
-        TRY(modup(ctx, Cc, (long long)r * N, cnt, Dig));
+        TRY(modup(ctx, Cc, (long long)r * N, cnt, Dig, Asrc + (size_t)r * N, (long long)ctw));
         RotBatch rb;
         memset(&rb, 0, sizeof(rb));
         rb.n = (int)cnt;
@@ -724,7 +752,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
             rb.c0[t] = (int)t;
             rb.out[t] = (int)t;
         }
-        CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, ctx->perms, U, ctx->stream));
+        CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->stream));
         TRY(moddown_batch(ctx, rb, Asrc, (long long)ctw, Rres + (size_t)rho0 * ctw, (long long)ctw));
     }
     const u64* Yfinal = A;
@@ -808,13 +836,13 @@ extern "C" int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uin
     B.n_m = r;
     B.mod_step = 1;
     CK(ntt_forward(ctx->ring, B, 2, LOAD_PLAIN, ctx->stream));
-    TRY(modup(ctx, ct_in + (size_t)r * N, (long long)r * N, 1, (u64*)ctx->Dig.p));
+    TRY(modup(ctx, ct_in + (size_t)r * N, (long long)r * N, 1, (u64*)ctx->Dig.p, X + (size_t)r * N, 0));
     RotBatch rb;
     memset(&rb, 0, sizeof(rb));
     rb.n = 1;
     rb.key[0] = key;
     rb.out[0] = 1;
-    CK(launch_key_inner_product(ctx->ring, rb, (const u64*)ctx->Dig.p, ctx->keys, ctx->perms, (u64*)ctx->U.p, ctx->stream));
+    CK(launch_key_inner_product(ctx->ring, rb, (const u64*)ctx->Dig.p, ctx->keys, (u64*)ctx->U.p, ctx->stream));
     TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
     memset(&B, 0, sizeof(B));
     B.src = X + ctw;

@@ -187,6 +187,12 @@ struct PolyBatch {
     u64* tile_ptr;                // non-null: the NTT-domain side lives there in the tile-major layout `tile`
     TileLayout tile;              //   (forward writes its final result there, inverse reads its input there);
     u32 tile_pj0, o_base;         //   diagonal o_base + o = pj*n_terms + t; the layout's group 0 is group tile_pj0
+    u32 skip_diag;                // forward only: polynomial (o, m) with m < r and o % r == m (a digit in its own prime)
+    const u64* diag_src;          //   is not transformed but copied from diag_src + (o / r)*diag_so + m*N, where its
+    long long diag_so;            //   transform already exists
+    const u32* scatter;           // forward only: final store goes to scatter_dst[scatter[(o / scatter_div) * N + n]]
+    u32 scatter_div;              //   instead of dst[n] (same polynomial strides as dst)
+    u64* scatter_dst;
     u32 split_bits;               // L > 0: the NTT-domain side of the transform is stored as two L-bit-aligned
                                   // limbs per word, (v >> L) << 32 | (v & (2^L - 1)); forward writes, inverse reads it
 };

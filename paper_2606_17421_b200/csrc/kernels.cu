@@ -335,49 +335,95 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 }
 
 // ------------------------------------------------------------------------------------------------
-// Key-switch inner product over the extended basis, with the automorphism applied as a gather on
-// the digits:  u[rot][comp][m][n] = sum_j dig[.][j][m][perm[n]] * key[.][j][comp][m][n].
-__global__ void __launch_bounds__(256) key_inner_product_kernel(const RingDev R, const RotBatch rb,
-                                                                const u64* __restrict__ dig,
-                                                                const u64* __restrict__ keys,
-                                                                const u32* __restrict__ perms, u64* __restrict__ u) {
-    const u32 m = blockIdx.y, rot = blockIdx.z;
-    const u32 N = R.N, r = R.r, nb = r + 1;
-    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
-    const u32 key = rb.key[rot];
-    const u32 pn = perms[(size_t)key * N + n];
-    const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + pn;
-    const u64* kp = keys + ((size_t)key * r * 2 * nb + m) * N + n;
-    u64 h0 = 0, l0 = 0, h1 = 0, l1 = 0;
-    for (u32 j = 0; j < r; ++j) {
-        const u64 d = dp[(size_t)j * nb * N];
-        const u64 k0 = __ldcs(kp + (size_t)(j * 2) * nb * N);
-        const u64 k1 = __ldcs(kp + (size_t)(j * 2 + 1) * nb * N);
-        mac128(h0, l0, d, k0);
-        mac128(h1, l1, d, k1);
+// Key-switch inner product over the extended basis (Sec. 4.2 "key-switching primitives").
+// The rotation keys are stored pre-permuted by their automorphism, so the product runs in the
+// un-rotated index space with fully coalesced operands:
+//   u'[rot][comp][m][n] = sum_j digit_j[m][n] * key'[key(rot)][j][comp][m][n]
+// and the automorphism is applied once, as a scatter, when the rotated ciphertext is assembled.
+// digit_j in its own prime (m == j) is the transform of c1 itself and is read from the source
+// ciphertext instead of the digit buffer.  Two coefficients per thread, 128-bit loads; the key
+// stream is read once per rotation.
+template <bool SMALL, int RR>
+__device__ __forceinline__ void key_inner_body(const RingDev& R, u32 r, u32 m, const u64* __restrict__ dp,
+                                               const u64* __restrict__ kp, u64* __restrict__ up) {
+    const u32 N = R.N, nb = r + 1;
+    LimbAcc<SMALL> a00, a01, a10, a11;                  // [component][word]
+    if (RR > 0) {
+        // the number of digits is known at compile time: every load is issued before the first product
+        ulonglong2 d[RR > 0 ? RR : 1], k0[RR > 0 ? RR : 1], k1[RR > 0 ? RR : 1];
+#pragma unroll
+        for (int j = 0; j < RR; ++j) {
+            d[j] = *(const ulonglong2*)(dp + (size_t)j * nb * N);
+            k0[j] = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2) * nb * N));
+            k1[j] = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2 + 1) * nb * N));
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j) {
+            a00.mac(d[j].x, k0[j].x);
+            a01.mac(d[j].y, k0[j].y);
+            a10.mac(d[j].x, k1[j].x);
+            a11.mac(d[j].y, k1[j].y);
+        }
+    } else {
+#pragma unroll 4
+        for (u32 j = 0; j < r; ++j) {
+            const ulonglong2 d = *(const ulonglong2*)(dp + (size_t)j * nb * N);
+            const ulonglong2 k0 = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2) * nb * N));
+            const ulonglong2 k1 = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2 + 1) * nb * N));
+            a00.mac(d.x, k0.x);
+            a01.mac(d.y, k0.y);
+            a10.mac(d.x, k1.x);
+            a11.mac(d.y, k1.y);
+        }
     }
     const u64 q = R.q[m], mu = R.mu[m], c64 = R.c64[m], c64s = R.c64s[m];
-    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n;
-    up[0] = reduce128(h0, l0, q, mu, c64, c64s);
-    up[(size_t)nb * N] = reduce128(h1, l1, q, mu, c64, c64s);
+    *(ulonglong2*)up = make_ulonglong2(a00.reduce(q, mu, c64, c64s), a01.reduce(q, mu, c64, c64s));
+    *(ulonglong2*)(up + (size_t)nb * N) = make_ulonglong2(a10.reduce(q, mu, c64, c64s), a11.reduce(q, mu, c64, c64s));
 }
 
-cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys,
-                                     const u32* perms, u64* u, cudaStream_t stream) {
+// grid: x = rotation (fastest, so that rotations sharing a key or a digit set run side by side and
+// meet in L2), y = tile of 512 coefficients, z = modulus of the extended basis
+template <int RR>
+__global__ void __launch_bounds__(256) key_inner_product_kernel(const RingDev R, const RotBatch rb,
+                                                                const u64* __restrict__ dig,
+                                                                const u64* __restrict__ keys, u64* __restrict__ u,
+                                                                u32 small_ok) {
+    const u32 rot = blockIdx.x, m = blockIdx.z;
+    const u32 N = R.N, r = R.r, nb = r + 1;
+    const u32 n = (blockIdx.y * blockDim.x + threadIdx.x) * 2;
+    const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + n;
+    const u64* kp = keys + ((size_t)rb.key[rot] * r * 2 * nb + m) * N + n;
+    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n;
+    if (m < r && small_ok) key_inner_body<true, RR>(R, r, m, dp, kp, up);
+    else key_inner_body<false, RR>(R, r, m, dp, kp, up);
+}
+
+cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
+                                     cudaStream_t stream) {
     if (rb.n == 0) return cudaSuccess;
-    dim3 grid(ring.dev.N / 256, ring.dev.r + 1, rb.n);
+    u64 qmax = 0;
+    for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
+    // without a carry counter the middle partial sum takes r <= 15 terms below 2^51 each
+    const u32 small_ok = (qmax < ((u64)1 << 50)) ? 1u : 0u;
+    dim3 grid(rb.n, ring.dev.N / 512, ring.dev.r + 1);
     ProfScope prof(ring.prof, CAT_KEY_INNER, stream);
-    key_inner_product_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, perms, u);
+    switch (ring.dev.r) {
+        case 3: key_inner_product_kernel<3><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
+        case 7: key_inner_product_kernel<7><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
+        case 9: key_inner_product_kernel<9><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
+        default: key_inner_product_kernel<0><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
+    }
     return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
-// Last step of the division by P:  v = (u - NTT(centred lift of the P-residue)) * P^{-1} mod q_i,
-// plus the automorphism of c0 for component 0.
+// Last step of the division by P, in the un-rotated index space, and the automorphism as a scatter:
+//   v'[n] = (u'[n] - NTT(centred lift of the P-residue)[n]) * P^{-1} + (comp == 0 ? c0[n] : 0)   mod q_i
+//   out[pinv[n]] = v'[n]        (pinv = where position n goes under the rotation's automorphism)
 __global__ void __launch_bounds__(256) moddown_finish_kernel(const RingDev R, const RotBatch rb,
                                                              const u64* __restrict__ u, const u64* __restrict__ tn,
                                                              const u64* __restrict__ c0_base, long long c0_stride,
-                                                             const u32* __restrict__ perms, u64* __restrict__ out_base,
+                                                             const u32* __restrict__ pinv, u64* __restrict__ out_base,
                                                              long long out_stride) {
     const u32 i = blockIdx.y % R.r, comp = blockIdx.y / R.r, rot = blockIdx.z;
     const u32 N = R.N, r = R.r, nb = r + 1;
@@ -386,20 +432,18 @@ __global__ void __launch_bounds__(256) moddown_finish_kernel(const RingDev R, co
     const u64 uv = u[(((size_t)rot * 2 + comp) * nb + i) * N + n];
     const u64 tv = tn[(((size_t)rot * 2 + comp) * r + i) * N + n];
     u64 v = mul_shoup(sub_mod(uv, tv, q), R.pinv[i], R.pinvs[i], q);
-    if (comp == 0) {
-        const u32 pn = perms[(size_t)rb.key[rot] * N + n];
-        v = add_mod(v, c0_base[(size_t)rb.c0[rot] * c0_stride + (size_t)i * N + pn], q);
-    }
-    out_base[(size_t)rb.out[rot] * out_stride + ((size_t)comp * r + i) * N + n] = v;
+    if (comp == 0) v = add_mod(v, c0_base[(size_t)rb.c0[rot] * c0_stride + (size_t)i * N + n], q);
+    const u32 pn = pinv[(size_t)rb.key[rot] * N + n];
+    out_base[(size_t)rb.out[rot] * out_stride + ((size_t)comp * r + i) * N + pn] = v;
 }
 
 cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, const u64* u, const u64* tn,
-                                  const u64* c0_base, long long c0_stride, const u32* perms, u64* out_base,
+                                  const u64* c0_base, long long c0_stride, const u32* pinv, u64* out_base,
                                   long long out_stride, cudaStream_t stream) {
     if (rb.n == 0) return cudaSuccess;
     dim3 grid(ring.dev.N / 256, 2 * ring.dev.r, rb.n);
     ProfScope prof(ring.prof, CAT_MODDOWN_FINISH, stream);
-    moddown_finish_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, u, tn, c0_base, c0_stride, perms, out_base,
+    moddown_finish_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, u, tn, c0_base, c0_stride, pinv, out_base,
                                                     out_stride);
     return cudaGetLastError();
 }

@@ -136,6 +136,16 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
     const u32 mod = B.mod0 + m * B.mod_step;
+    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) {
+        // this digit's transform in its own prime exists already: copy the tile instead
+        const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
+        u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
+        for (int w = threadIdx.x; w < (1 << (LOG_R + LOG_LANES)); w += blockDim.x) {
+            const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * (1 << LOG_LANES) + (w & ((1 << LOG_LANES) - 1));
+            dd[gidx] = ds[gidx];
+        }
+        return;
+    }
     const u64 q = R.q[mod], mu = R.mu[mod];
     const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
@@ -207,6 +217,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
     const u32 mod = B.mod0 + m * B.mod_step;
+    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) return;
     const u64 q = R.q[mod];
     const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
@@ -254,6 +265,13 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             if (B.split_bits) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) e[i] = limb_split(e[i], B.split_bits);
+            }
+            if (B.scatter) {    // permuted store (keys are kept pre-permuted by their automorphism)
+                const u32* sc = B.scatter + (size_t)(o / B.scatter_div) * R.N + chunk * LEN + 4 * s;
+                u64* sd = B.scatter_dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sd[sc[i]] = e[i];
+                continue;
             }
             ulonglong2* gp = (ulonglong2*)(gdst + 4 * s);
             if (B.tile_ptr)     // 4 adjacent coefficients never straddle a tile (tiles hold >= 16)
@@ -360,6 +378,22 @@ cudaError_t ntt_forward(const RingHost& ring, const PolyBatch& B, u32 n_outer, i
     else if (load == LOAD_I64_MONT) e = launch_strided<true, LOAD_I64_MONT>(ring, B, n_polys, stream);
     else e = launch_strided<true, LOAD_CENTRED>(ring, B, n_polys, stream);
     if (e != cudaSuccess) return e;
+    return launch_contig<true>(ring, B, n_polys, stream);
+}
+
+// Forward transform whose final store is permuted: polynomial (o, m) ends up at
+// final[(o*dst_so + m*dst_sm) + scatter[(o / scatter_div)*N + n]].  B.dst is a staging buffer of the same shape.
+cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B0, u32 n_outer, int load, u64* final_dst,
+                              const u32* scatter, u32 scatter_div, cudaStream_t stream) {
+    PolyBatch B = B0;
+    const u32 n_polys = n_outer * B.n_m;
+    cudaError_t e;
+    if (load == LOAD_PLAIN) e = launch_strided<true, LOAD_PLAIN>(ring, B, n_polys, stream);
+    else e = launch_strided<true, LOAD_REDUCE>(ring, B, n_polys, stream);
+    if (e != cudaSuccess) return e;
+    B.scatter = scatter;
+    B.scatter_div = scatter_div;
+    B.scatter_dst = final_dst;
     return launch_contig<true>(ring, B, n_polys, stream);
 }
 
