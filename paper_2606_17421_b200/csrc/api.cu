@@ -1,6 +1,7 @@
 // C ABI of libbifrost: context and table set-up, key loading, weight encoding, and the launch
 // sequence of the encrypted linear layer (Alg. 3: EncodeWeights, FHE_Linear; Sec. 4.2).
 #include <cmath>
+#include <cstdlib>
 #include <cstdio>
 #include <cstring>
 #include <map>
@@ -101,7 +102,7 @@ struct bf_ctx {
     u32* perms = nullptr;            // [n_keys][N] pinv: where position n goes under the key's automorphism
     u32 n_keys = 0;
     // scratch (grow-only)
-    DevBuf X, Dig, U, Tc, Tn, Cc, A, Rres, Y, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
+    DevBuf X, Dig, U, Tc, Tn, Cc, A, Rres, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
     u64 cache_budget = 0, cache_used = 0;
     std::vector<bf_weights*> weights;
     std::string cuda_msg;
@@ -319,7 +320,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
             delete w;
         }
     }
-    DevBuf* bufs[] = {&ctx->X, &ctx->Dig, &ctx->U, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres, &ctx->Y,
+    DevBuf* bufs[] = {&ctx->X, &ctx->Dig, &ctx->U, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres,
                       &ctx->fft, &ctx->coef, &ctx->ptnat, &ctx->ptjit, &ctx->stage_in, &ctx->stage_out, &ctx->nm_a, &ctx->nm_b};
     for (DevBuf* b : bufs) free_buf(*b);
     cudaFree(ctx->tw_fwd);
@@ -539,7 +540,8 @@ extern "C" void bf_weights_free(bf_ctx* ctx, bf_weights* w) {
 // ------------------------------------------------------------------------------------------------
 // Division by the special prime and assembly of rotated ciphertexts for the rotations listed in rb
 // (their inner products already sit in U): inverse transform of the P-residues, centred lift into
-// every q_i with a forward transform, then (u - t) * P^{-1} plus the permuted c0.
+// every q_i with a forward transform whose last store computes (u - t) * P^{-1} + c0 and scatters
+// it through the rotation's permutation.
 static int moddown_batch(bf_ctx* ctx, const RotBatch& rb, const u64* c0_base, long long c0_stride, u64* out_base,
                          long long out_stride) {
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
@@ -555,7 +557,7 @@ static int moddown_batch(bf_ctx* ctx, const RotBatch& rb, const u64* c0_base, lo
     CK(ntt_inverse(ctx->ring, B, (u32)rb.n * 2, ctx->stream));
     memset(&B, 0, sizeof(B));
     B.src = ctx->Tc.p;
-    B.dst = (u64*)ctx->Tn.p;
+    B.dst = (u64*)ctx->Tn.p;                            // staging between the two passes of the transform
     B.src_so = N;
     B.src_sm = 0;
     B.dst_so = (long long)r * N;
@@ -564,9 +566,14 @@ static int moddown_batch(bf_ctx* ctx, const RotBatch& rb, const u64* c0_base, lo
     B.mod0 = 0;
     B.mod_step = 1;
     B.lift_mod = ctx->ring.q[r];
-    CK(ntt_forward(ctx->ring, B, (u32)rb.n * 2, LOAD_CENTRED, ctx->stream));
-    CK(launch_moddown_finish(ctx->ring, rb, (const u64*)ctx->U.p, (const u64*)ctx->Tn.p, c0_base, c0_stride,
-                             ctx->perms, out_base, out_stride, ctx->stream));
+    ModDownEpilogue epi;
+    epi.u = (const u64*)ctx->U.p;
+    epi.c0_base = c0_base;
+    epi.c0_stride = c0_stride;
+    epi.pinv = ctx->perms;
+    epi.out_base = out_base;
+    epi.out_stride = out_stride;
+    CK(ntt_forward_moddown(ctx->ring, B, (u32)rb.n * 2, rb, epi, ctx->stream));
     return BF_OK;
 }
 
@@ -586,10 +593,10 @@ static int find_key(bf_ctx* ctx, u32 steps, int* key) {
     return BF_OK;
 }
 
-// Digits of c1 (coefficient domain, [r][N] with stride N) reduced into every prime of the extended
-// basis and transformed: dig[set][j][m] = NTT_m( c1_j mod m ).
-// The digit in its own prime is the transform of c1 itself, which the caller already has
-// (c1_ntt + set*c1_ntt_stride, [r][N]): it is copied, not recomputed.
+// Digits of c1 (coefficient domain; set s at c1_coeff + s*set_stride, [r][N]) reduced into every prime
+// of the extended basis and transformed: dig[set][j][m] = NTT_m( c1_j mod m ).  The digit in its own
+// prime is the transform of c1 itself, which the caller already has (c1_ntt + s*c1_ntt_stride, [r][N]):
+// it is copied, not recomputed.
 static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_sets, u64* dig, const u64* c1_ntt,
                  long long c1_ntt_stride) {
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
@@ -598,26 +605,18 @@ static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_s
     B.n_m = nb;
     B.mod0 = 0;
     B.mod_step = 1;
+    B.src = c1_coeff;
+    B.o_div = r;                 // o = set*r + digit
+    B.src_so2 = set_stride;
+    B.src_so = N;
     B.src_sm = 0;
-    B.dst_sm = N;
+    B.dst = dig;
     B.dst_so = (long long)nb * N;
+    B.dst_sm = N;
     B.skip_diag = 1;
     B.diag_src = c1_ntt;
     B.diag_so = c1_ntt_stride;
-    if (set_stride == (long long)r * N || n_sets == 1) {
-        B.src = c1_coeff;
-        B.dst = dig;
-        B.src_so = N;
-        CK(ntt_forward(ctx->ring, B, n_sets * r, LOAD_REDUCE, ctx->stream));
-    } else {
-        for (u32 s = 0; s < n_sets; ++s) {
-            B.src = c1_coeff + (size_t)s * set_stride;
-            B.dst = dig + (size_t)s * r * nb * N;
-            B.diag_src = c1_ntt + (size_t)s * c1_ntt_stride;
-            B.src_so = N;
-            CK(ntt_forward(ctx->ring, B, r, LOAD_REDUCE, ctx->stream));
-        }
-    }
+    CK(ntt_forward(ctx->ring, B, n_sets * r, LOAD_REDUCE, ctx->stream));
     return BF_OK;
 }
 
@@ -626,9 +625,11 @@ static void stamp(bf_ctx* ctx, int i) {
 }
 
 static u32 giant_batch(const bf_ctx* ctx) {
-    // rotations per giant-step launch: keep the digit sets of one batch near the L2 capacity
+    // rotations per key-switch launch
     const size_t per_rot = (size_t)ctx->r * (ctx->r + 1) * ctx->N * 8;
-    size_t nrot = ((size_t)96 << 20) / per_rot;
+    // Measured: fewer, larger launches beat keeping a batch's digits L2-resident.  Cap the digit
+    // buffer at 1 GiB.
+    size_t nrot = ((size_t)1 << 30) / per_rot;
     if (nrot < 1) nrot = 1;
     if (nrot > (size_t)MAX_ROT_BATCH) nrot = MAX_ROT_BATCH;
     return (u32)nrot;
@@ -649,20 +650,24 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
 
     const u32 gb = giant_batch(ctx);
     const u32 n_giant = (g - 1) * n_out;
+    // input ciphertexts whose baby steps share one key-switch launch
+    u32 in_batch = b > 1 ? (u32)MAX_ROT_BATCH / (b - 1) : n_in;
+    if (in_batch > gb) in_batch = gb;
+    if (in_batch > n_in) in_batch = n_in;
+    if (in_batch < 1) in_batch = 1;
     u32 n_dig_sets = n_giant < gb ? n_giant : gb;       // digit sets alive at once
+    if (n_dig_sets < in_batch) n_dig_sets = in_batch;
     if (n_dig_sets < 1) n_dig_sets = 1;
-    u32 rot_cap = b - 1 > n_dig_sets ? b - 1 : n_dig_sets;
+    u32 rot_cap = in_batch * (b - 1) > n_dig_sets ? in_batch * (b - 1) : n_dig_sets;
     if (rot_cap < 1) rot_cap = 1;
     TRY(ensure(ctx, ctx->X, (size_t)n_in * b * ctw * 8));
     TRY(ensure(ctx, ctx->A, (size_t)n_out * g * ctw * 8));
     TRY(ensure(ctx, ctx->Rres, (size_t)(n_giant ? n_giant : 1) * ctw * 8));
-    TRY(ensure(ctx, ctx->Y, (size_t)n_out * ctw * 8));
     TRY(ensure(ctx, ctx->Cc, (size_t)n_dig_sets * r * N * 8));
     TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_cap));
     u64* X = (u64*)ctx->X.p;
     u64* A = (u64*)ctx->A.p;
     u64* Rres = (u64*)ctx->Rres.p;
-    u64* Y = (u64*)ctx->Y.p;
     u64* Dig = (u64*)ctx->Dig.p;
     u64* U = (u64*)ctx->U.p;
     u64* Cc = (u64*)ctx->Cc.p;
@@ -673,30 +678,34 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     }
     stamp(ctx, 0);
 
-    // ---- ingest, hoisted ModUp and baby steps, one input ciphertext at a time
+    // ---- ingest, hoisted ModUp and baby steps, batched over the input ciphertexts
     PolyBatch B;
-    for (u32 q = 0; q < n_in; ++q) {
-        const u64* ct = ct_in + (size_t)q * ctw;
-        u64* X0 = X + (size_t)q * b * ctw;               // X[q][0] = NTT(ct_q)
-        memset(&B, 0, sizeof(B));
-        B.src = ct;
-        B.dst = X0;
-        B.src_so = B.dst_so = (long long)r * N;
-        B.src_sm = B.dst_sm = N;
-        B.n_m = r;
-        B.mod0 = 0;
-        B.mod_step = 1;
-        CK(ntt_forward(ctx->ring, B, 2, LOAD_PLAIN, ctx->stream));
-        if (b > 1) {
-            TRY(modup(ctx, ct + (size_t)r * N, (long long)r * N, 1, Dig, X0 + (size_t)r * N, 0));
+    memset(&B, 0, sizeof(B));
+    B.src = ct_in;                                       // X[q][0] = NTT(ct_q): polynomial (q, component*r + prime)
+    B.dst = X;
+    B.src_so = (long long)ctw;
+    B.dst_so = (long long)b * ctw;
+    B.src_sm = B.dst_sm = N;
+    B.n_m = 2 * r;
+    B.mod_wrap = r;
+    B.mod0 = 0;
+    B.mod_step = 1;
+    CK(ntt_forward(ctx->ring, B, n_in, LOAD_PLAIN, ctx->stream));
+    if (b > 1) {
+        for (u32 q0 = 0; q0 < n_in; q0 += in_batch) {
+            const u32 qn = (n_in - q0 < in_batch) ? n_in - q0 : in_batch;
+            TRY(modup(ctx, ct_in + (size_t)q0 * ctw + (size_t)r * N, (long long)ctw, qn, Dig,
+                      X + (size_t)q0 * b * ctw + (size_t)r * N, (long long)b * ctw));
             RotBatch rb;
             memset(&rb, 0, sizeof(rb));
-            rb.n = (int)(b - 1);
-            for (u32 k = 1; k < b; ++k) {
-                rb.key[k - 1] = baby_key[k];
-                rb.dig[k - 1] = 0;
-                rb.c0[k - 1] = (int)(q * b);
-                rb.out[k - 1] = (int)(q * b + k);
+            for (u32 q = 0; q < qn; ++q) {
+                for (u32 k = 1; k < b; ++k) {
+                    const int t = rb.n++;
+                    rb.key[t] = baby_key[k];
+                    rb.dig[t] = (int)q;
+                    rb.c0[t] = (int)((q0 + q) * b);
+                    rb.out[t] = (int)((q0 + q) * b + k);
+                }
             }
             CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->stream));
             TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
@@ -755,23 +764,23 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->stream));
         TRY(moddown_batch(ctx, rb, Asrc, (long long)ctw, Rres + (size_t)rho0 * ctw, (long long)ctw));
     }
-    const u64* Yfinal = A;
-    if (g > 1) {
-        CK(launch_giant_sum(ctx->ring, A, Rres, Y, n_out, g, ctx->stream));
-        Yfinal = Y;
-    }
     stamp(ctx, 3);
 
-    // ---- back to the coefficient domain
+    // ---- back to the coefficient domain; the sum over giant steps happens in the transform's load:
+    // Y[p] = A[0][p] + sum_{j >= 1} (rotated A[j][p])
     memset(&B, 0, sizeof(B));
-    B.src = Yfinal;
+    B.src = A;
     B.dst = ct_out;
-    B.src_so = B.dst_so = (long long)r * N;
+    B.src_so = B.dst_so = (long long)ctw;
     B.src_sm = B.dst_sm = N;
-    B.n_m = r;
+    B.n_m = 2 * r;
+    B.mod_wrap = r;
     B.mod0 = 0;
     B.mod_step = 1;
-    CK(ntt_inverse(ctx->ring, B, n_out * 2, ctx->stream));
+    B.sum_src = Rres;
+    B.sum_terms = g - 1;
+    B.sum_stride = (long long)n_out * ctw;
+    CK(ntt_inverse(ctx->ring, B, n_out, ctx->stream));
     stamp(ctx, 4);
     if (!pt_weights) TRY(check_overflow(ctx));
     (void)nb;
@@ -790,14 +799,7 @@ extern "C" int bf_rescale(bf_ctx* ctx, const uint64_t* ct_in, uint64_t* ct_out, 
         invs[i] = h_shoup(inv[i], q);
         qlmod[i] = qL % q;
     }
-    if (ct_in == ct_out && n_ct > 1) {
-        // packed output of ciphertext t overlaps the input of ciphertext t-1 only: in-order launches
-        for (u32 t = 0; t < n_ct; ++t)
-            CK(launch_rescale(ctx->ring, ct_in + (size_t)t * 2 * level * ctx->N,
-                              ct_out + (size_t)t * 2 * (level - 1) * ctx->N, 1, level, inv, invs, qlmod, ctx->stream));
-    } else {
-        CK(launch_rescale(ctx->ring, ct_in, ct_out, n_ct, level, inv, invs, qlmod, ctx->stream));
-    }
+    CK(launch_rescale(ctx->ring, ct_in, ct_out, n_ct, level, inv, invs, qlmod, ctx->stream));
     if (scale_inout) *scale_inout /= (double)qL;
     return BF_OK;
 }
@@ -936,7 +938,7 @@ extern "C" int bf_kernel_categories(void) { return (int)CAT_COUNT; }
 
 extern "C" const char* bf_kernel_category_name(int cat) {
     static const char* names[CAT_COUNT] = {"ntt_fwd_strided", "ntt_fwd_contig", "ntt_inv_contig", "ntt_inv_strided",
-                                           "key_inner_product", "moddown_finish", "mac", "giant_sum", "rescale",
+                                           "key_inner_product", "mac", "rescale",
                                            "encode_fft_a", "encode_fft_b", "pointwise_mul"};
     return (cat >= 0 && cat < (int)CAT_COUNT) ? names[cat] : "";
 }

@@ -13,8 +13,6 @@ typedef int64_t i64;
 typedef uint32_t u32;
 
 constexpr int MAX_MODULI = 16;    // ciphertext primes + the special prime
-constexpr int MAX_ROT_BATCH = 64; // rotations handled by one key-switch launch
-
 // Per-ring constants handed to every kernel by value (lands in the constant bank).
 // Modulus index r is the special prime P; 0..r-1 are the ciphertext primes q_0..q_L.
 struct RingDev {
@@ -153,6 +151,29 @@ enum LoadMode : int {
     LOAD_I64_MONT = 4,  // LOAD_I64, then times 2^64 mod q: the transform's output is in Montgomery form
 };
 
+constexpr int MAX_ROT_BATCH = 64; // rotations handled by one key-switch launch
+
+struct RotBatch {                     // one key-switch launch over n rotations
+    int n;
+    int key[MAX_ROT_BATCH];           // index of the rotation key (and of its permutation table)
+    int dig[MAX_ROT_BATCH];           // which digit set the rotation reads
+    int c0[MAX_ROT_BATCH];            // which source ciphertext is being rotated (its c0 is added)
+    int out[MAX_ROT_BATCH];           // which output ciphertext slot receives the result
+};
+
+// Epilogue of the division by P, fused into the forward transform of the lifted P-residue
+// (polynomial (o, m) = (rotation*2 + component, prime i)):  instead of storing t = NTT(lift),
+//   v = (u[o][i][n] - t) * P^{-1} + (component == 0 ? c0[c0(rot)][i][n] : 0)
+// is scattered to out[out(rot)][component][i][pinv[key(rot)][n]].
+struct ModDownEpilogue {
+    const u64* u;                 // [rot][2][r+1][N]
+    const u64* c0_base;
+    long long c0_stride;
+    const u32* pinv;              // [n_keys][N]
+    u64* out_base;
+    long long out_stride;
+};
+
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks
 // each stream one contiguous region:  word (group pj, term t, prime i, coefficient n) lives at
 //   (((((i*ntiles + n/TN)*G + pj/PL)*C + t/TS)*PL + pj%PL)*TS + t%TS)*TN + n%TN
@@ -182,6 +203,13 @@ struct PolyBatch {
     u64* dst;
     long long src_so, src_sm, dst_so, dst_sm;
     u32 n_m, mod0, mod_step;
+    u32 mod_wrap;                 // > 0: modulus index = mod0 + (m % mod_wrap) * mod_step (e.g. m = component*r + prime)
+    u32 o_div;                    // > 0: source = src + (o / o_div)*src_so2 + (o % o_div)*src_so + m*src_sm
+    long long src_so2;
+    // inverse only: the input is a sum  src + sum_{t < sum_terms} (sum_src + t*sum_stride)  of residues in [0, q)
+    const u64* sum_src;
+    long long sum_stride;
+    u32 sum_terms;
     u64 lift_mod;                 // LOAD_CENTRED: the modulus M the source residues live in
     u32 from_mont;                // inverse transform only: input is in Montgomery form, output is not
     u64* tile_ptr;                // non-null: the NTT-domain side lives there in the tile-major layout `tile`

@@ -18,7 +18,7 @@ struct NttGeometry {
 // Kernel categories for launch counting and optional per-launch event timing.
 enum KernelCat : int {
     CAT_NTT_FWD_STRIDED = 0, CAT_NTT_FWD_CONTIG, CAT_NTT_INV_CONTIG, CAT_NTT_INV_STRIDED,
-    CAT_KEY_INNER, CAT_MODDOWN_FINISH, CAT_MAC, CAT_GIANT_SUM, CAT_RESCALE,
+    CAT_KEY_INNER, CAT_MAC, CAT_RESCALE,
     CAT_ENCODE_FFT_A, CAT_ENCODE_FFT_B, CAT_POINTWISE, CAT_COUNT
 };
 
@@ -49,36 +49,24 @@ struct RingHost {
 NttGeometry ntt_geometry(u32 logN);
 cudaError_t ntt_forward(const RingHost& ring, const PolyBatch& B, u32 n_outer, int load, cudaStream_t stream);
 cudaError_t ntt_inverse(const RingHost& ring, const PolyBatch& B, u32 n_outer, cudaStream_t stream);
+// Forward transform of the centred lifts of P-residues with the ModDown epilogue fused into its last store.
+cudaError_t ntt_forward_moddown(const RingHost& ring, const PolyBatch& B, u32 n_outer, const RotBatch& rb,
+                                const ModDownEpilogue& epi, cudaStream_t stream);
 cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B, u32 n_outer, int load, u64* final_dst,
                               const u32* scatter, u32 scatter_div, cudaStream_t stream);
 
 // ---- kernels.cu : element-wise and streaming kernels of the linear layer
-struct RotBatch {                     // one key-switch launch over n rotations
-    int n;
-    int key[MAX_ROT_BATCH];           // index of the rotation key (and of its permutation table)
-    int dig[MAX_ROT_BATCH];           // which digit set the rotation reads
-    int c0[MAX_ROT_BATCH];            // which source ciphertext is being rotated (its c0 is added, its c1 is digit j at prime j)
-    int out[MAX_ROT_BATCH];           // which output ciphertext slot receives the result
-};
-
 // out[t] = a[t] * b[t] pointwise, polynomial t modulo basis prime mod0 + t % n_m
 cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* b, u64* out, u32 n_polys, u32 n_m,
                                  u32 mod0, cudaStream_t stream);
 // u'[rot][comp][m][n] = sum_j dig[dig(rot)][j][m][n] * key'[key(rot)][j][comp][m][n]  (keys pre-permuted)
 cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
                                      cudaStream_t stream);
-// out[out(rot)][comp][i][pinv[n]] = (u'[rot][comp][i][n] - tn[rot][comp][i][n]) * P^{-1} + (comp == 0 ? c0[c0(rot)][0][i][n] : 0)
-cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, const u64* u, const u64* tn,
-                                  const u64* c0_base, long long c0_stride, const u32* pinv, u64* out_base,
-                                  long long out_stride, cudaStream_t stream);
 u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintext format (0 = whole words)
 TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms);   // layout of n_pj groups of n_terms diagonals
 size_t mac_tile_words(const RingHost& ring, const TileLayout& t);           // words that layout occupies
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
                        u32 n_terms, int* error_flag, cudaStream_t stream);
-// y[p] = a[p] + sum_{j=1}^{g-1} rres[(j-1)*n_out + p]   (ciphertexts of [2][r][N] words)
-cudaError_t launch_giant_sum(const RingHost& ring, const u64* a, const u64* rres, u64* y, u32 n_out, u32 g,
-                             cudaStream_t stream);
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
                            const u64* invs, const u64* qlmod, cudaStream_t stream);
 

@@ -417,61 +417,6 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
 }
 
 // ------------------------------------------------------------------------------------------------
-// Last step of the division by P, in the un-rotated index space, and the automorphism as a scatter:
-//   v'[n] = (u'[n] - NTT(centred lift of the P-residue)[n]) * P^{-1} + (comp == 0 ? c0[n] : 0)   mod q_i
-//   out[pinv[n]] = v'[n]        (pinv = where position n goes under the rotation's automorphism)
-__global__ void __launch_bounds__(256) moddown_finish_kernel(const RingDev R, const RotBatch rb,
-                                                             const u64* __restrict__ u, const u64* __restrict__ tn,
-                                                             const u64* __restrict__ c0_base, long long c0_stride,
-                                                             const u32* __restrict__ pinv, u64* __restrict__ out_base,
-                                                             long long out_stride) {
-    const u32 i = blockIdx.y % R.r, comp = blockIdx.y / R.r, rot = blockIdx.z;
-    const u32 N = R.N, r = R.r, nb = r + 1;
-    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
-    const u64 q = R.q[i];
-    const u64 uv = u[(((size_t)rot * 2 + comp) * nb + i) * N + n];
-    const u64 tv = tn[(((size_t)rot * 2 + comp) * r + i) * N + n];
-    u64 v = mul_shoup(sub_mod(uv, tv, q), R.pinv[i], R.pinvs[i], q);
-    if (comp == 0) v = add_mod(v, c0_base[(size_t)rb.c0[rot] * c0_stride + (size_t)i * N + n], q);
-    const u32 pn = pinv[(size_t)rb.key[rot] * N + n];
-    out_base[(size_t)rb.out[rot] * out_stride + ((size_t)comp * r + i) * N + pn] = v;
-}
-
-cudaError_t launch_moddown_finish(const RingHost& ring, const RotBatch& rb, const u64* u, const u64* tn,
-                                  const u64* c0_base, long long c0_stride, const u32* pinv, u64* out_base,
-                                  long long out_stride, cudaStream_t stream) {
-    if (rb.n == 0) return cudaSuccess;
-    dim3 grid(ring.dev.N / 256, 2 * ring.dev.r, rb.n);
-    ProfScope prof(ring.prof, CAT_MODDOWN_FINISH, stream);
-    moddown_finish_kernel<<<grid, 256, 0, stream>>>(ring.dev, rb, u, tn, c0_base, c0_stride, pinv, out_base,
-                                                    out_stride);
-    return cudaGetLastError();
-}
-
-// ------------------------------------------------------------------------------------------------
-// Y[p] = A[0][p] + sum_{j >= 1} (rotated A[j][p]);  a holds the j = 0 block, rres[(j-1)*n_out + p] the rest
-__global__ void __launch_bounds__(256) giant_sum_kernel(const RingDev R, const u64* __restrict__ a,
-                                                        const u64* __restrict__ rres, u64* __restrict__ y, u32 g) {
-    const u32 ci = blockIdx.y, p = blockIdx.z, n_out = gridDim.z;   // ci = comp * r + i
-    const u32 N = R.N, r = R.r;
-    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
-    const u64 q = R.q[ci % r];
-    const size_t ct = (size_t)2 * r * N;
-    u64 v = a[(size_t)p * ct + (size_t)ci * N + n];
-    for (u32 j = 1; j < g; ++j) v = add_mod(v, rres[((size_t)(j - 1) * n_out + p) * ct + (size_t)ci * N + n], q);
-    y[(size_t)p * ct + (size_t)ci * N + n] = v;
-}
-
-cudaError_t launch_giant_sum(const RingHost& ring, const u64* a, const u64* rres, u64* y, u32 n_out, u32 g,
-                             cudaStream_t stream) {
-    if (n_out == 0) return cudaSuccess;
-    dim3 grid(ring.dev.N / 256, 2 * ring.dev.r, n_out);
-    ProfScope prof(ring.prof, CAT_GIANT_SUM, stream);
-    giant_sum_kernel<<<grid, 256, 0, stream>>>(ring.dev, a, rres, y, g);
-    return cudaGetLastError();
-}
-
-// ------------------------------------------------------------------------------------------------
 // Rescale (Sec. 2.1): drop the last prime q_L of a level-`level` ciphertext in coefficient form,
 //   c'_i = (c_i - centred(c_L)) * q_L^{-1} mod q_i.
 // Every address a thread touches is congruent to its coefficient index modulo N, and it reads all
@@ -481,12 +426,15 @@ struct RescaleConsts {
     u64 inv[MAX_MODULI], invs[MAX_MODULI], qlmod[MAX_MODULI];
 };
 
-__global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const RescaleConsts rc,
-                                                      const u64* __restrict__ in, u64* __restrict__ out, u32 level) {
-    const u32 ct = blockIdx.y;
+// `in` and `out` may alias, hence no __restrict__.  When they do and several ciphertexts are
+// rescaled, the launch uses one thread per coefficient that walks the ciphertexts in order
+// (n_seq > 1): the packed output of ciphertext t never reaches the input of ciphertext t+1.
+__global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const RescaleConsts rc, const u64* in, u64* out,
+                                                      u32 level, u32 n_seq) {
     const u32 N = R.N;
     const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
     const u64 qL = R.q[level - 1];
+  for (u32 ct = blockIdx.y; ct < blockIdx.y + n_seq; ++ct) {
     const u64* ip = in + (size_t)ct * 2 * level * N + n;
     u64* op = out + (size_t)ct * 2 * (level - 1) * N + n;
     u64 res[2][MAX_MODULI];
@@ -505,6 +453,7 @@ __global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const Res
 #pragma unroll
     for (int comp = 0; comp < 2; ++comp)
         for (u32 i = 0; i + 1 < level; ++i) op[((size_t)comp * (level - 1) + i) * N] = res[comp][i];
+  }
 }
 
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
@@ -512,9 +461,14 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
     if (n_ct == 0) return cudaSuccess;
     RescaleConsts rc;
     for (u32 i = 0; i + 1 < level; ++i) { rc.inv[i] = inv[i]; rc.invs[i] = invs[i]; rc.qlmod[i] = qlmod[i]; }
-    dim3 grid(ring.dev.N / 256, n_ct);
     ProfScope prof(ring.prof, CAT_RESCALE, stream);
-    rescale_kernel<<<grid, 256, 0, stream>>>(ring.dev, rc, in, out, level);
+    if (in == out && n_ct > 1) {
+        dim3 grid(ring.dev.N / 64, 1);
+        rescale_kernel<<<grid, 64, 0, stream>>>(ring.dev, rc, in, out, level, n_ct);
+    } else {
+        dim3 grid(ring.dev.N / 256, n_ct);
+        rescale_kernel<<<grid, 256, 0, stream>>>(ring.dev, rc, in, out, level, 1);
+    }
     return cudaGetLastError();
 }
 

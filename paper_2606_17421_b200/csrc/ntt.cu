@@ -135,7 +135,7 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     __shared__ u64 sm[LEN * LANES];
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
-    const u32 mod = B.mod0 + m * B.mod_step;
+    const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
     if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) {
         // this digit's transform in its own prime exists already: copy the tile instead
         const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
@@ -149,7 +149,9 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     const u64 q = R.q[mod], mu = R.mu[mod];
     const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
-    const char* src = (const char*)B.src + ((size_t)o * B.src_so + (size_t)m * B.src_sm) * 8;
+    const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
+                                   : (size_t)o * B.src_so;
+    const char* src = (const char*)B.src + (src_off + (size_t)m * B.src_sm) * 8;
     const u64 lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu)
                        : (LOAD == LOAD_I64_MONT) ? R.c64s[mod] : 0;
     const u64 lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
@@ -209,14 +211,15 @@ ntt_strided(const RingDev R, const PolyBatch B) {
 // groups, so only warp-level synchronisation is needed.
 // Forward: second pass (in place, final reduction to [0, q)).  Inverse: first pass (reads the batch
 // source, plain residues).
-template <bool FWD>
+template <bool FWD, bool EPI>
 __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const RingDev R, const PolyBatch B,
-                                                                       u32 chunks_per_block) {
+                                                                       u32 chunks_per_block, const RotBatch rb,
+                                                                       const ModDownEpilogue epi) {
     constexpr int LEN = 1 << LOG_C;
     __shared__ u64 sm_all[CHUNKS_PER_BLOCK * LEN];
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
-    const u32 mod = B.mod0 + m * B.mod_step;
+    const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
     if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) return;
     const u64 q = R.q[mod];
     const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
@@ -262,6 +265,29 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
                 if (v >= q) v -= q;
                 e[i] = v;
             }
+            if (EPI) {
+                const u32 rot = o >> 1, comp = o & 1, i = mod, r = R.r, nb = r + 1;
+                const size_t n = (size_t)chunk * LEN + 4 * s;
+                const u64* up = epi.u + ((size_t)o * nb + i) * R.N + n;
+                const ulonglong2 u0 = *(const ulonglong2*)up, u1 = *(const ulonglong2*)(up + 2);
+                const u64 uu[4] = {u0.x, u0.y, u1.x, u1.y};
+                u64 cc[4] = {0, 0, 0, 0};
+                if (comp == 0) {
+                    const u64* cp = epi.c0_base + (size_t)rb.c0[rot] * epi.c0_stride + (size_t)i * R.N + n;
+                    const ulonglong2 c0 = *(const ulonglong2*)cp, c1 = *(const ulonglong2*)(cp + 2);
+                    cc[0] = c0.x; cc[1] = c0.y; cc[2] = c1.x; cc[3] = c1.y;
+                }
+                const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
+                const u32 pp[4] = {pv.x, pv.y, pv.z, pv.w};
+                u64* op = epi.out_base + (size_t)rb.out[rot] * epi.out_stride + ((size_t)comp * r + i) * R.N;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    u64 v = mul_shoup(sub_mod(uu[t], e[t], q), R.pinv[i], R.pinvs[i], q);
+                    v = add_mod(v, cc[t], q);
+                    op[pp[t]] = v;
+                }
+                continue;
+            }
             if (B.split_bits) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) e[i] = limb_split(e[i], B.split_bits);
@@ -292,6 +318,15 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
                                                                        chunk * LEN + 4 * s));
             const ulonglong2 a = gp[0], b = gp[1];
             e[0] = a.x; e[1] = a.y; e[2] = b.x; e[3] = b.y;
+            if (B.sum_terms) {      // the input is a sum of several arrays of the same shape
+                const u64* sp = B.sum_src + (size_t)o * B.src_so + (size_t)m * B.src_sm + (size_t)chunk * LEN + 4 * s;
+                for (u32 t = 0; t < B.sum_terms; ++t) {
+                    const ulonglong2 a2 = *(const ulonglong2*)(sp + (size_t)t * B.sum_stride);
+                    const ulonglong2 b2 = *(const ulonglong2*)(sp + (size_t)t * B.sum_stride + 2);
+                    e[0] = add_mod(e[0], a2.x, q); e[1] = add_mod(e[1], a2.y, q);
+                    e[2] = add_mod(e[2], b2.x, q); e[3] = add_mod(e[3], b2.y, q);
+                }
+            }
             if (B.split_bits) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) e[i] = limb_join(e[i], B.split_bits);
@@ -359,13 +394,20 @@ static cudaError_t launch_strided(const RingHost& ring, const PolyBatch& B, u32 
 }
 
 template <bool FWD>
-static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream) {
+static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream,
+                                 const RotBatch* rb = nullptr, const ModDownEpilogue* epi = nullptr) {
     if (n_polys == 0) return cudaSuccess;
     ProfScope prof(ring.prof, FWD ? CAT_NTT_FWD_CONTIG : CAT_NTT_INV_CONTIG, stream);
     const u32 chunks = 1u << ring.geom.log_r;
     const u32 cpb = (u32)ring.geom.contig_lanes;
     dim3 grid(chunks / cpb, n_polys);
-    ntt_contig<FWD><<<grid, 32 * CHUNKS_PER_BLOCK, 0, stream>>>(ring.dev, B, cpb);
+    if (FWD && epi) {
+        ntt_contig<FWD, true><<<grid, 32 * CHUNKS_PER_BLOCK, 0, stream>>>(ring.dev, B, cpb, *rb, *epi);
+    } else {
+        static const RotBatch no_rb = {};
+        static const ModDownEpilogue no_epi = {};
+        ntt_contig<FWD, false><<<grid, 32 * CHUNKS_PER_BLOCK, 0, stream>>>(ring.dev, B, cpb, no_rb, no_epi);
+    }
     return cudaGetLastError();
 }
 
@@ -379,6 +421,14 @@ cudaError_t ntt_forward(const RingHost& ring, const PolyBatch& B, u32 n_outer, i
     else e = launch_strided<true, LOAD_CENTRED>(ring, B, n_polys, stream);
     if (e != cudaSuccess) return e;
     return launch_contig<true>(ring, B, n_polys, stream);
+}
+
+cudaError_t ntt_forward_moddown(const RingHost& ring, const PolyBatch& B, u32 n_outer, const RotBatch& rb,
+                                const ModDownEpilogue& epi, cudaStream_t stream) {
+    const u32 n_polys = n_outer * B.n_m;
+    cudaError_t e = launch_strided<true, LOAD_CENTRED>(ring, B, n_polys, stream);
+    if (e != cudaSuccess) return e;
+    return launch_contig<true>(ring, B, n_polys, stream, &rb, &epi);
 }
 
 // Forward transform whose final store is permuted: polynomial (o, m) ends up at
