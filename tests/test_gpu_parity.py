@@ -203,6 +203,65 @@ def test_linear_gpt2_qkv_config_bit_exact():
     run_case(par, ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g), L.d_out, L.d_in, 0, 1e-3, L.name)
 
 
+def check_blocks(par, plan, layers, blocks_of, seed, keys=None, s=None):
+    """Full-size layers in the configuration the benchmark runs: the device computes every output
+    block, the oracle the sampled ones; those must agree on every residue, and decrypt correctly."""
+    if s is None:
+        s = ckks.keygen(par, seed)
+        keys = ckks.make_rotation_keys(par, s, plan, seed)
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys)
+        for L in layers:
+            W = wl.gen_weights(seed, L.name, L.d_out, L.d_in)
+            x = wl.gen_activation(seed, L.name, L.d_in)
+            cts = ckks.encrypt_vector(par, plan, s, x, seed)
+            n_out = -(-L.d_out // plan.D)
+            blocks = blocks_of(L, n_out)
+            expect = ckks.linear(par, plan, cts, W, keys, blocks=blocks)
+            w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), L.d_out, L.d_in)
+            out = g.linear(cts, W, L.d_out, L.d_in, weights=w)
+            low = g.empty_u64(n_out, 2, par.r - 1, par.N)
+            scale = g.bf.bf_rescale(g.ctx, out, low, n_out, par.r, par.scale * par.scale)
+            got, low = g.to_host_u64(out), g.to_host_u64(low)
+            g.bf.bf_weights_free(g.ctx, w)
+            y_ref = W.astype(np.float64) @ x
+            for p in blocks:
+                assert np.array_equal(got[p], expect[p]), (L.name, p)
+                assert np.array_equal(low[p], ckks.rescale(par, expect[p])), (L.name, p)
+                part = ckks.fold_output(ckks.decode(ckks.decrypt(par, s, low[p]), par.N, scale), plan, p, L.d_out)
+                err = np.abs(part - y_ref[p * plan.D:p * plan.D + len(part)]).max()
+                assert err < 1e-3, (L.name, p, err)
+    finally:
+        g.close()
+
+
+def test_gpt2_layer_shapes_sampled_blocks():
+    # one transformer layer of the GPT-2 decode-step workload (qkv is covered in full above)
+    w = wl.WORKLOADS["gpt2_step"]
+    par = oracle_params(w.params)
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
+    check_blocks(par, plan, w.layers[1:], lambda L, n_out: [n_out - 1], 11)
+
+
+def test_qwen3_layer_shapes_sampled_blocks():
+    w = wl.WORKLOADS["qwen3_step"]
+    par = oracle_params(w.params)
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
+    # distinct shapes of the layer: q (1024->2048), o (2048->1024), gate (1024->3072), down (3072->1024)
+    pick = [L for L in w.layers if L.name in ("q", "o", "gate", "down")]
+    check_blocks(par, plan, pick, lambda L, n_out: [(3 * n_out) // 4 if n_out > 1 else 0], 12)
+
+
+def test_llama3_layer_shapes_sampled_blocks():
+    w = wl.WORKLOADS["llama3_layer"]
+    par = oracle_params(w.params)
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
+    # k (4096->1024) in full, one block of gate (4096->14336)
+    pick = [L for L in w.layers if L.name in ("k", "gate")]
+    check_blocks(par, plan, pick, lambda L, n_out: [n_out - 1], 13)
+
+
 def test_structured_matrices_on_device():
     par = oracle_params("n12")
     plan = ckks.Plan(64, 4, 4, 4)
