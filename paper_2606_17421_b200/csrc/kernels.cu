@@ -477,21 +477,21 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
 // every thread runs 8 independent mad.wide.u32 chains.  Gives the measured denominator for the
 // integer-bound kernels (NTT, key switch).
 __global__ void __launch_bounds__(256) imad_probe_kernel(u64* __restrict__ sink, u32 iters) {
-    u32 b = threadIdx.x * 2654435761u + blockIdx.x * 40503u + 12345u;
-    u64 c0 = b, c1 = b + 1, c2 = b + 2, c3 = b + 3, c4 = b + 4, c5 = b + 5, c6 = b + 6, c7 = b + 7;
+    const u32 b = threadIdx.x * 2654435761u + blockIdx.x * 40503u + 12345u;
+    u64 c[8];
+    u32 d[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { c[k] = b + k; d[k] = b * 3 + k; }
     for (u32 i = 0; i < iters; ++i) {
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            asm volatile("mad.wide.u32 %0, %8, %9, %0;\n\tmad.wide.u32 %1, %8, %10, %1;\n\t"
-                         "mad.wide.u32 %2, %8, %11, %2;\n\tmad.wide.u32 %3, %8, %12, %3;\n\t"
-                         "mad.wide.u32 %4, %8, %13, %4;\n\tmad.wide.u32 %5, %8, %14, %5;\n\t"
-                         "mad.wide.u32 %6, %8, %15, %6;\n\tmad.wide.u32 %7, %8, %16, %7;"
-                         : "+l"(c0), "+l"(c1), "+l"(c2), "+l"(c3), "+l"(c4), "+l"(c5), "+l"(c6), "+l"(c7)
-                         : "r"(b), "r"((u32)c1), "r"((u32)c2), "r"((u32)c3), "r"((u32)c4), "r"((u32)c5),
-                           "r"((u32)c6), "r"((u32)c7), "r"((u32)c0));
+#pragma unroll
+            for (int k = 0; k < 8; ++k) asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(c[k]) : "r"(b), "r"(d[(k + 1) & 7]));
         }
     }
-    u64 v = c0 ^ c1 ^ c2 ^ c3 ^ c4 ^ c5 ^ c6 ^ c7;
+    u64 v = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v ^= c[k];
     if (v == 0x1234567ull) sink[0] = v;      // practically never true; keeps the chains alive
 }
 
