@@ -243,10 +243,18 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
             pw[k] = h_mulmod(pw[k - 1], psi, q);
             pwi[k] = h_mulmod(pwi[k - 1], psi_inv, q);
         }
+        R.fp_ok[m] = q < (1ull << 41) ? 1u : 0u;
+        auto companion = [&](u64 w) -> u64 {
+            if (!R.fp_ok[m]) return h_shoup(w, q);
+            const double wq = (double)w / (double)q;      // both exact in fp64; IEEE division rounds correctly
+            u64 bits;
+            memcpy(&bits, &wq, sizeof(bits));
+            return bits;
+        };
         for (u32 k = 0; k < N; ++k) {
             const u32 e = h_brev(k, (int)ctx->logN);
-            twf[(size_t)m * N + k] = make_ulonglong2(pw[e], h_shoup(pw[e], q));
-            twi[(size_t)m * N + k] = make_ulonglong2(pwi[e], h_shoup(pwi[e], q));
+            twf[(size_t)m * N + k] = make_ulonglong2(pw[e], companion(pw[e]));
+            twi[(size_t)m * N + k] = make_ulonglong2(pwi[e], companion(pwi[e]));
         }
     }
     // encoder tables: twiddles from the host's libm so that results do not depend on the device's
@@ -967,7 +975,7 @@ extern "C" int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out) {
     TRY(ensure(ctx, ctx->nm_a, 4096));
     cudaDeviceProp prop;
     CK(cudaGetDeviceProperties(&prop, ctx->device));
-    const u32 blocks = (u32)prop.multiProcessorCount * 8, iters = 4096;
+    const u32 blocks = (u32)prop.multiProcessorCount * 8, iters = 256;
     cudaEvent_t a, b;
     CK(cudaEventCreate(&a));
     CK(cudaEventCreate(&b));

@@ -29,7 +29,9 @@ struct RingDev {
     u64 qneg[MAX_MODULI];        // -q^{-1} mod 2^64 (Montgomery reduction)
     u64 ninv_m[MAX_MODULI];      // N^{-1} * 2^{-64} mod q: inverse transform that also leaves Montgomery form
     u64 ninv_ms[MAX_MODULI];
-    const ulonglong2* tw_fwd;    // [r+1][N]  (psi^brev(k), Shoup companion), merged Cooley-Tukey order
+    u32 fp_ok[MAX_MODULI];       // modulus below 2^41: twiddle products estimate their quotient on the fp64 pipe and
+                                 //   the twiddle tables hold (w, bits of (double)w / q) instead of (w, Shoup companion)
+    const ulonglong2* tw_fwd;    // [r+1][N]  (psi^brev(k), companion), merged Cooley-Tukey order
     const ulonglong2* tw_inv;    // [r+1][N]  inverses of the above, for the Gentleman-Sande inverse
 };
 
@@ -38,6 +40,19 @@ struct RingDev {
 __device__ __forceinline__ u64 mul_shoup_lazy(u64 x, u64 w, u64 ws, u64 q) {
     u64 hi = __umul64hi(x, ws);
     return x * w - hi * q;
+}
+
+// Modular multiplication by a constant w for primes q < 2^41 with the quotient estimated on the
+// fp64 pipe (B200 issues fp64 FMAs at the rate of 32-bit integer multiply-adds, on a pipe of its
+// own, while a 64x64 high product costs about ten integer multiply-add slots).
+// w_over_q = (double)w / (double)q, correctly rounded.  For x < 2^43, qhat = round(x * w_over_q) is
+// within 1/2 + 2^-9 of x*w/q, so x*w - qhat*q + q lies in (0.49 q, 1.51 q) and is congruent to x*w.
+__device__ __forceinline__ u64 mul_fp_lazy(u64 x, u64 w, double w_over_q, u64 q) {
+    const double magic = 4503599627370496.0;                                             // 2^52
+    const double xd = __longlong_as_double((long long)(x | 0x4330000000000000ull)) - magic;   // exact
+    const double t = __fma_rn(xd, w_over_q, magic);                                      // 2^52 + round(x * w/q)
+    const u64 qhat = (u64)__double_as_longlong(t) - 0x4330000000000000ull;
+    return x * w - qhat * q + q;
 }
 
 __device__ __forceinline__ u64 mul_shoup(u64 x, u64 w, u64 ws, u64 q) {
@@ -257,23 +272,29 @@ struct KaraAcc {
 // Montgomery reduction by two 32-bit rounds: V * 2^{-64} mod q in [0, q), for V = (H, L) < q * 2^64.
 // qneg32 = -q^{-1} mod 2^32.  Six 32-bit multiplies instead of a 64x64 high product.
 __device__ __forceinline__ u64 redc_2x32(u64 H, u64 L, u64 q, u32 qneg32) {
+    u32 l0 = (u32)L, l1 = (u32)(L >> 32), h0 = (u32)H, h1 = (u32)(H >> 32);
     const u32 q0 = (u32)q, q1 = (u32)(q >> 32);
-#pragma unroll
-    for (int round = 0; round < 2; ++round) {
-        const u32 m = (u32)L * qneg32;
-        const u64 p0 = (u64)m * q0, p1 = (u64)m * q1;
-        // (H, L) += p0 + (p1 << 32)
-        u64 l = L + p0;
-        u64 c = (l < p0) ? 1ull : 0ull;
-        const u64 p1s = p1 << 32;
-        l += p1s;
-        c += (l < p1s) ? 1ull : 0ull;
-        const u64 h = H + (p1 >> 32) + c;
-        // low 32 bits are now zero: shift right by 32
-        L = (l >> 32) | (h << 32);
-        H = h >> 32;
-    }
-    return L >= q ? L - q : L;
+    // round 1: m = l0 * qneg32; (h1 h0 l1 l0) += m * (q1 q0); l0 becomes 0 and is dropped
+    // round 2: the same one limb up; the result is (h1 h0)
+    asm("{\n\t.reg .u32 m;\n\t"
+        "mul.lo.u32 m, %0, %6;\n\t"
+        "mad.lo.cc.u32 %0, m, %4, %0;\n\t"
+        "madc.hi.cc.u32 %1, m, %4, %1;\n\t"
+        "addc.cc.u32 %2, %2, 0;\n\t"
+        "addc.u32 %3, %3, 0;\n\t"
+        "mad.lo.cc.u32 %1, m, %5, %1;\n\t"
+        "madc.hi.cc.u32 %2, m, %5, %2;\n\t"
+        "addc.u32 %3, %3, 0;\n\t"
+        "mul.lo.u32 m, %1, %6;\n\t"
+        "mad.lo.cc.u32 %1, m, %4, %1;\n\t"
+        "madc.hi.cc.u32 %2, m, %4, %2;\n\t"
+        "addc.u32 %3, %3, 0;\n\t"
+        "mad.lo.cc.u32 %2, m, %5, %2;\n\t"
+        "madc.hi.u32 %3, m, %5, %3;\n\t}"
+        : "+r"(l0), "+r"(l1), "+r"(h0), "+r"(h1)
+        : "r"(q0), "r"(q1), "r"(qneg32));
+    const u64 t = ((u64)h1 << 32) | h0;
+    return t >= q ? t - q : t;
 }
 
 }  // namespace bf

@@ -89,12 +89,12 @@ __device__ __forceinline__ void mbar_arrive(u64* bar) {
 constexpr int MAC_CONSUMERS = 256;
 constexpr int MAC_THREADS = MAC_CONSUMERS + 32;   // + one producer warp
 constexpr int MAC_TS = (int)TILE_TS;              // terms per stage
-constexpr int MAC_STAGES = 4;
+constexpr int MAC_STAGES = 2;
 constexpr int MAC_STAGE_WORDS = MAC_TS * MAC_CONSUMERS;   // 16 KB per stage whatever TN is
 constexpr u32 KARA_L = 25;
 
 template <bool KARA, int LOG_TN>
-__global__ void __launch_bounds__(MAC_THREADS, 2)
+__global__ void __launch_bounds__(MAC_THREADS, 3)
 mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, const u64* __restrict__ x,
            u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, int* __restrict__ error_flag) {
     extern __shared__ __align__(128) unsigned char mac_smem[];

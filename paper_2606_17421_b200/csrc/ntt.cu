@@ -64,9 +64,9 @@ __device__ __forceinline__ u64 load_src(const void* src, size_t idx, u64 q, u64 
 // Butterflies of one register-resident set of 2^K points over K consecutive stages.
 // tw_base = (blocks at the group's first forward stage) * mult, so that stage st, sub-block sub
 // uses twiddle (tw_base << st) + (blk << st) + sub.
-template <int K, bool FWD>
-__device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
-                                                u64 q) {
+template <int K, bool FWD, bool FP>
+__device__ __forceinline__ void set_butterflies_t(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
+                                                  u64 q) {
     const u64 q2 = 2 * q;
 #pragma unroll
     for (int s = 0; s < K; ++s) {
@@ -81,7 +81,8 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
                 if (FWD) {
                     u64 x = e[i];
                     if (x >= q2) x -= q2;
-                    u64 t = mul_shoup_lazy(e[i + d], w.x, w.y, q);
+                    u64 t = FP ? mul_fp_lazy(e[i + d], w.x, __longlong_as_double((long long)w.y), q)
+                               : mul_shoup_lazy(e[i + d], w.x, w.y, q);
                     e[i] = x + t;
                     e[i + d] = x - t + q2;
                 } else {
@@ -89,11 +90,20 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
                     u64 s2 = a + b;
                     if (s2 >= q2) s2 -= q2;
                     e[i] = s2;
-                    e[i + d] = mul_shoup_lazy(a - b + q2, w.x, w.y, q);
+                    e[i + d] = FP ? mul_fp_lazy(a - b + q2, w.x, __longlong_as_double((long long)w.y), q)
+                                  : mul_shoup_lazy(a - b + q2, w.x, w.y, q);
                 }
             }
         }
     }
+}
+
+// fp selects the fp64-assisted twiddle product (block-uniform: it depends on the modulus only)
+template <int K, bool FWD>
+__device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
+                                                u64 q, bool fp) {
+    if (fp) set_butterflies_t<K, FWD, true>(e, tw, tw_base, blk, q);
+    else set_butterflies_t<K, FWD, false>(e, tw, tw_base, blk, q);
 }
 
 // Stage groups of a local transform of 2^LOG_LEN points, in forward order.
@@ -155,6 +165,7 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     const u64 lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu)
                        : (LOAD == LOAD_I64_MONT) ? R.c64s[mod] : 0;
     const u64 lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
+    const bool fp = R.fp_ok[mod] != 0;
     const u64 ninv = (!FWD && B.from_mont) ? R.ninv_m[mod] : R.ninv[mod];
     const u64 ninvs = (!FWD && B.from_mont) ? R.ninv_ms[mod] : R.ninvs[mod];
     const int col0 = blockIdx.x * LANES;
@@ -186,9 +197,9 @@ ntt_strided(const RingDev R, const PolyBatch B) {
                     e[i] = sm[row * LANES + lane];
                 }
             }
-            if (K == 3) set_butterflies<3, FWD>(e, tw, (u32)m0, (u32)blk, q);
-            else if (K == 2) set_butterflies<2, FWD>(e, tw, (u32)m0, (u32)blk, q);
-            else set_butterflies<1, FWD>(e, tw, (u32)m0, (u32)blk, q);
+            if (K == 3) set_butterflies<3, FWD>(e, tw, (u32)m0, (u32)blk, q, fp);
+            else if (K == 2) set_butterflies<2, FWD>(e, tw, (u32)m0, (u32)blk, q, fp);
+            else set_butterflies<1, FWD>(e, tw, (u32)m0, (u32)blk, q, fp);
 #pragma unroll
             for (int i = 0; i < (1 << K); ++i) {
                 const int row = base + i * step;
@@ -227,6 +238,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
     const u64* src = FWD ? dst : (const u64*)B.src + (size_t)o * B.src_so + (size_t)m * B.src_sm;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if ((u32)warp >= chunks_per_block) return;
+    const bool fp = R.fp_ok[mod] != 0;
     const u32 chunk = blockIdx.x * chunks_per_block + warp;
     const u32 mult = (R.N >> LOG_C) + chunk;                   // twiddle index multiplier of this chunk
     u64* sm = sm_all + warp * LEN;
@@ -237,7 +249,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
         // group 0: K = 3, spacing 32
 #pragma unroll
         for (int i = 0; i < 8; ++i) e[i] = gsrc[lane + 32 * i];
-        set_butterflies<3, true>(e, tw, 1u * mult, 0u, q);
+        set_butterflies<3, true>(e, tw, 1u * mult, 0u, q, fp);
 #pragma unroll
         for (int i = 0; i < 8; ++i) sm[swz(lane + 32 * i)] = e[i];
         __syncwarp();
@@ -246,7 +258,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             const int blk = lane >> 2, base = blk * 32 + (lane & 3);
 #pragma unroll
             for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
-            set_butterflies<3, true>(e, tw, 8u * mult, (u32)blk, q);
+            set_butterflies<3, true>(e, tw, 8u * mult, (u32)blk, q, fp);
 #pragma unroll
             for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
         }
@@ -257,7 +269,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             const int s = lane + 32 * it;
 #pragma unroll
             for (int i = 0; i < 4; ++i) e[i] = sm[swz(4 * s + i)];
-            set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q);
+            set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, fp);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {   // final reduction [0, 4q) -> [0, q)
                 u64 v = e[i];
@@ -331,7 +343,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
 #pragma unroll
                 for (int i = 0; i < 4; ++i) e[i] = limb_join(e[i], B.split_bits);
             }
-            set_butterflies<2, false>(e, tw, 64u * mult, (u32)s, q);
+            set_butterflies<2, false>(e, tw, 64u * mult, (u32)s, q, fp);
 #pragma unroll
             for (int i = 0; i < 4; ++i) sm[swz(4 * s + i)] = e[i];
         }
@@ -340,14 +352,14 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             const int blk = lane >> 2, base = blk * 32 + (lane & 3);
 #pragma unroll
             for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
-            set_butterflies<3, false>(e, tw, 8u * mult, (u32)blk, q);
+            set_butterflies<3, false>(e, tw, 8u * mult, (u32)blk, q, fp);
 #pragma unroll
             for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
         }
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 8; ++i) e[i] = sm[swz(lane + 32 * i)];
-        set_butterflies<3, false>(e, tw, 1u * mult, 0u, q);
+        set_butterflies<3, false>(e, tw, 1u * mult, 0u, q, fp);
 #pragma unroll
         for (int i = 0; i < 8; ++i) gdst[lane + 32 * i] = e[i];      // lazy, below 2q; the strided pass finishes
     }
