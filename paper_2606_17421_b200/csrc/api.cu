@@ -244,17 +244,27 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
             pwi[k] = h_mulmod(pwi[k - 1], psi_inv, q);
         }
         R.fp_ok[m] = q < (1ull << 41) ? 1u : 0u;
-        auto companion = [&](u64 w) -> u64 {
-            if (!R.fp_ok[m]) return h_shoup(w, q);
-            const double wq = (double)w / (double)q;      // both exact in fp64; IEEE division rounds correctly
+        R.qd[m] = (double)q;
+        R.qinv_d[m] = 1.0 / (double)q;
+        R.ninv_d[m] = (double)R.ninv[m];
+        R.ninv_q[m] = (double)R.ninv[m] / (double)q;
+        R.ninvm_d[m] = (double)R.ninv_m[m];
+        R.ninvm_q[m] = (double)R.ninv_m[m] / (double)q;
+        auto dbits = [](double d) -> u64 {
             u64 bits;
-            memcpy(&bits, &wq, sizeof(bits));
+            memcpy(&bits, &d, sizeof(bits));
             return bits;
+        };
+        // integer path: (w, floor(w * 2^64 / q)); fp64 path: bits of ((double)w, (double)w / q) -- both
+        // operands are exact in fp64 and IEEE division rounds correctly
+        auto entry = [&](u64 w) -> ulonglong2 {
+            if (!R.fp_ok[m]) return make_ulonglong2(w, h_shoup(w, q));
+            return make_ulonglong2(dbits((double)w), dbits((double)w / (double)q));
         };
         for (u32 k = 0; k < N; ++k) {
             const u32 e = h_brev(k, (int)ctx->logN);
-            twf[(size_t)m * N + k] = make_ulonglong2(pw[e], companion(pw[e]));
-            twi[(size_t)m * N + k] = make_ulonglong2(pwi[e], companion(pwi[e]));
+            twf[(size_t)m * N + k] = entry(pw[e]);
+            twi[(size_t)m * N + k] = entry(pwi[e]);
         }
     }
     // encoder tables: twiddles from the host's libm so that results do not depend on the device's

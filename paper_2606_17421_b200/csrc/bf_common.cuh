@@ -29,8 +29,12 @@ struct RingDev {
     u64 qneg[MAX_MODULI];        // -q^{-1} mod 2^64 (Montgomery reduction)
     u64 ninv_m[MAX_MODULI];      // N^{-1} * 2^{-64} mod q: inverse transform that also leaves Montgomery form
     u64 ninv_ms[MAX_MODULI];
-    u32 fp_ok[MAX_MODULI];       // modulus below 2^41: twiddle products estimate their quotient on the fp64 pipe and
-                                 //   the twiddle tables hold (w, bits of (double)w / q) instead of (w, Shoup companion)
+    u32 fp_ok[MAX_MODULI];       // modulus below 2^41: its transforms run in fp64 (every value an exact integer below
+                                 //   2^53) and its twiddle tables hold the bits of ((double)w, (double)w / q)
+    double qd[MAX_MODULI];       // (double)q
+    double qinv_d[MAX_MODULI];   // 1.0 / q
+    double ninv_d[MAX_MODULI], ninv_q[MAX_MODULI];     // (double)N^{-1} and N^{-1} / q
+    double ninvm_d[MAX_MODULI], ninvm_q[MAX_MODULI];   // the same for N^{-1} * 2^{-64} (leaving Montgomery form)
     const ulonglong2* tw_fwd;    // [r+1][N]  (psi^brev(k), companion), merged Cooley-Tukey order
     const ulonglong2* tw_inv;    // [r+1][N]  inverses of the above, for the Gentleman-Sande inverse
 };
@@ -42,17 +46,33 @@ __device__ __forceinline__ u64 mul_shoup_lazy(u64 x, u64 w, u64 ws, u64 q) {
     return x * w - hi * q;
 }
 
-// Modular multiplication by a constant w for primes q < 2^41 with the quotient estimated on the
-// fp64 pipe (B200 issues fp64 FMAs at the rate of 32-bit integer multiply-adds, on a pipe of its
-// own, while a 64x64 high product costs about ten integer multiply-add slots).
-// w_over_q = (double)w / (double)q, correctly rounded.  For x < 2^43, qhat = round(x * w_over_q) is
-// within 1/2 + 2^-9 of x*w/q, so x*w - qhat*q + q lies in (0.49 q, 1.51 q) and is congruent to x*w.
-__device__ __forceinline__ u64 mul_fp_lazy(u64 x, u64 w, double w_over_q, u64 q) {
-    const double magic = 4503599627370496.0;                                             // 2^52
-    const double xd = __longlong_as_double((long long)(x | 0x4330000000000000ull)) - magic;   // exact
-    const double t = __fma_rn(xd, w_over_q, magic);                                      // 2^52 + round(x * w/q)
-    const u64 qhat = (u64)__double_as_longlong(t) - 0x4330000000000000ull;
-    return x * w - qhat * q + q;
+// ---- fp64 arithmetic for primes q < 2^41.  B200 issues fp64 FMAs at the rate of 32-bit integer
+// multiply-adds, on a pipe of its own, while a 64x64-bit high product costs about ten integer
+// multiply-add slots; and integers below 2^53 are exact in fp64.
+__device__ __forceinline__ double u2d(u64 x) {          // exact for x < 2^52
+    return __longlong_as_double((long long)(x | 0x4330000000000000ull)) - 4503599627370496.0;
+}
+__device__ __forceinline__ u64 d2u(double d) {          // d an integer in [0, 2^52)
+    return (u64)__double_as_longlong(d + 4503599627370496.0) - 0x4330000000000000ull;
+}
+// x * w - round(x * w / q) * q for integer-valued x (|x| < 2^46) and a constant 0 <= w < q given as
+// (double)w and wq = (double)w / q.  The result is an exact integer in (-0.51 q, 0.51 q) congruent to
+// x*w:  ph + pl = x*w exactly (FMA), the quotient estimate is off by less than 2^-6, ph - qh*q is an
+// integer below 2^42 in magnitude and therefore exact, and so is the final sum.
+__device__ __forceinline__ double fp_mul_centred(double x, double w, double wq, double q) {
+    const double magic = 4503599627370496.0;             // 2^52
+    const double ph = __dmul_rn(x, w);
+    const double pl = __fma_rn(x, w, -ph);
+    const double qh = __dsub_rn(__fma_rn(x, wq, magic), magic);
+    return __dadd_rn(__fma_rn(-qh, q, ph), pl);
+}
+// v mod q in [0, q) for an integer-valued 0 <= v < 2^46
+__device__ __forceinline__ double fp_reduce(double v, double q, double qinv) {
+    const double magic = 4503599627370496.0;
+    const double qh = __dsub_rn(__fma_rn(v, qinv, magic), magic);
+    double r = __fma_rn(-qh, q, v);
+    if (r < 0.0) r = __dadd_rn(r, q);
+    return r;
 }
 
 __device__ __forceinline__ u64 mul_shoup(u64 x, u64 w, u64 ws, u64 q) {

@@ -64,9 +64,11 @@ __device__ __forceinline__ u64 load_src(const void* src, size_t idx, u64 q, u64 
 // Butterflies of one register-resident set of 2^K points over K consecutive stages.
 // tw_base = (blocks at the group's first forward stage) * mult, so that stage st, sub-block sub
 // uses twiddle (tw_base << st) + (blk << st) + sub.
-template <int K, bool FWD, bool FP>
-__device__ __forceinline__ void set_butterflies_t(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
-                                                  u64 q) {
+// Integer version: Harvey's lazy butterflies with Shoup products; forward values stay in [0, 4q),
+// inverse values in [0, 2q).
+template <int K, bool FWD>
+__device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
+                                                u64 q, double) {
     const u64 q2 = 2 * q;
 #pragma unroll
     for (int s = 0; s < K; ++s) {
@@ -81,8 +83,7 @@ __device__ __forceinline__ void set_butterflies_t(u64 (&e)[8], const ulonglong2*
                 if (FWD) {
                     u64 x = e[i];
                     if (x >= q2) x -= q2;
-                    u64 t = FP ? mul_fp_lazy(e[i + d], w.x, __longlong_as_double((long long)w.y), q)
-                               : mul_shoup_lazy(e[i + d], w.x, w.y, q);
+                    u64 t = mul_shoup_lazy(e[i + d], w.x, w.y, q);
                     e[i] = x + t;
                     e[i + d] = x - t + q2;
                 } else {
@@ -90,21 +91,53 @@ __device__ __forceinline__ void set_butterflies_t(u64 (&e)[8], const ulonglong2*
                     u64 s2 = a + b;
                     if (s2 >= q2) s2 -= q2;
                     e[i] = s2;
-                    e[i + d] = FP ? mul_fp_lazy(a - b + q2, w.x, __longlong_as_double((long long)w.y), q)
-                                  : mul_shoup_lazy(a - b + q2, w.x, w.y, q);
+                    e[i + d] = mul_shoup_lazy(a - b + q2, w.x, w.y, q);
                 }
             }
         }
     }
 }
 
-// fp selects the fp64-assisted twiddle product (block-uniform: it depends on the modulus only)
+// fp64 version (primes below 2^41).  Forward: (X, Y) -> (X + q + s, X + q - s) with s = Y*w centred in
+// (-0.51q, 0.51q): values stay non-negative and grow by at most 1.51q per stage, so after all
+// log2 N <= 16 stages they are below 26q < 2^46 and need one reduction at the very end.
+// Inverse: (a, b) -> (a + b reduced below 2q, (a - b + 2q)*w + q in (0.49q, 1.51q)): values in [0, 2q).
 template <int K, bool FWD>
-__device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
-                                                u64 q, bool fp) {
-    if (fp) set_butterflies_t<K, FWD, true>(e, tw, tw_base, blk, q);
-    else set_butterflies_t<K, FWD, false>(e, tw, tw_base, blk, q);
+__device__ __forceinline__ void set_butterflies(double (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base,
+                                                u32 blk, u64, double q) {
+    const double q2 = __dadd_rn(q, q);
+#pragma unroll
+    for (int s = 0; s < K; ++s) {
+        const int st = FWD ? s : (K - 1 - s);
+        const int d = (1 << K) >> (st + 1);
+#pragma unroll
+        for (int sub = 0; sub < (1 << st); ++sub) {
+            const ulonglong2 wb = __ldg(&tw[(tw_base << st) + (blk << st) + sub]);
+            const double w = __longlong_as_double((long long)wb.x), wq = __longlong_as_double((long long)wb.y);
+#pragma unroll
+            for (int off = 0; off < d; ++off) {
+                const int i = sub * 2 * d + off;
+                if (FWD) {
+                    const double sv = fp_mul_centred(e[i + d], w, wq, q);
+                    const double xq = __dadd_rn(e[i], q);
+                    e[i] = __dadd_rn(xq, sv);
+                    e[i + d] = __dsub_rn(xq, sv);
+                } else {
+                    const double a = e[i], b = e[i + d];
+                    double s2 = __dadd_rn(a, b);
+                    if (s2 >= q2) s2 = __dsub_rn(s2, q2);
+                    e[i] = s2;
+                    e[i + d] = __dadd_rn(fp_mul_centred(__dadd_rn(__dsub_rn(a, b), q2), w, wq, q), q);
+                }
+            }
+        }
+    }
 }
+
+template <bool FP> struct Elem { typedef u64 T; };
+template <> struct Elem<true> { typedef double T; };
+__device__ __forceinline__ void from_u64(u64& dst, u64 v) { dst = v; }
+__device__ __forceinline__ void from_u64(double& dst, u64 v) { dst = u2d(v); }
 
 // Stage groups of a local transform of 2^LOG_LEN points, in forward order.
 __host__ __device__ constexpr int n_groups(int log_len) { return log_len <= 3 ? 1 : (log_len <= 6 ? 2 : 3); }
@@ -132,31 +165,22 @@ __device__ __forceinline__ int swz(int i) { return i ^ ((i >> 4) & 3) ^ (((i >> 
 constexpr int LOG_C = 8;              // contiguous pass: chunks of 256 points, one warp each
 constexpr int CHUNKS_PER_BLOCK = 8;
 
+// Between the two passes of a transform the data sit in dst as lazily reduced values: 64-bit
+// integers for the integer path, fp64 bit patterns for the fp64 path (the modulus decides, so both
+// passes agree).
+
 // Strided pass: transforms the 2^LOG_R rows (stride 256) of 2^LOG_LANES adjacent columns.
 // Forward: first pass (reads the batch source through the load functor).  Inverse: second pass
 // (in place, scales by N^{-1}).
-template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
-__global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8),
-                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
-ntt_strided(const RingDev R, const PolyBatch B) {
+template <bool FWD, int LOAD, int LOG_R, int LOG_LANES, bool FP>
+__device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, u32 o, u32 m, u32 mod) {
+    typedef typename Elem<FP>::T T;
     constexpr int LEN = 1 << LOG_R, LANES = 1 << LOG_LANES;
     constexpr int NT = (LEN * LANES / 8) < 32 ? 32 : (LEN * LANES / 8);
     constexpr int NG = n_groups(LOG_R);
-    __shared__ u64 sm[LEN * LANES];
-    const u32 poly = blockIdx.y;
-    const u32 o = poly / B.n_m, m = poly % B.n_m;
-    const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
-    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) {
-        // this digit's transform in its own prime exists already: copy the tile instead
-        const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
-        u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
-        for (int w = threadIdx.x; w < (1 << (LOG_R + LOG_LANES)); w += blockDim.x) {
-            const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * (1 << LOG_LANES) + (w & ((1 << LOG_LANES) - 1));
-            dd[gidx] = ds[gidx];
-        }
-        return;
-    }
+    T* sm = (T*)sm_raw;
     const u64 q = R.q[mod], mu = R.mu[mod];
+    const double qd = R.qd[mod];
     const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
     const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
@@ -165,9 +189,6 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     const u64 lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu)
                        : (LOAD == LOAD_I64_MONT) ? R.c64s[mod] : 0;
     const u64 lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
-    const bool fp = R.fp_ok[mod] != 0;
-    const u64 ninv = (!FWD && B.from_mont) ? R.ninv_m[mod] : R.ninv[mod];
-    const u64 ninvs = (!FWD && B.from_mont) ? R.ninv_ms[mod] : R.ninvs[mod];
     const int col0 = blockIdx.x * LANES;
     const int tid = threadIdx.x;
 #pragma unroll
@@ -186,28 +207,39 @@ ntt_strided(const RingDev R, const PolyBatch B) {
             const int lane = w & (LANES - 1), u = w >> LOG_LANES;
             const int blk = u >> log_step, off = u & (step - 1);
             const int base = blk * 2 * t0 + off;
-            u64 e[8];
+            T e[8];
 #pragma unroll
             for (int i = 0; i < (1 << K); ++i) {
                 const int row = base + i * step;
                 if (g_first) {
                     const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
-                    e[i] = FWD ? load_src<LOAD>(src, gidx, q, mu, lift_mod, lift_red) : dst[gidx];
+                    if (FWD) from_u64(e[i], load_src<LOAD>(src, gidx, q, mu, lift_mod, lift_red));
+                    else e[i] = ((const T*)dst)[gidx];
                 } else {
                     e[i] = sm[row * LANES + lane];
                 }
             }
-            if (K == 3) set_butterflies<3, FWD>(e, tw, (u32)m0, (u32)blk, q, fp);
-            else if (K == 2) set_butterflies<2, FWD>(e, tw, (u32)m0, (u32)blk, q, fp);
-            else set_butterflies<1, FWD>(e, tw, (u32)m0, (u32)blk, q, fp);
+            if (K == 3) set_butterflies<3, FWD>(e, tw, (u32)m0, (u32)blk, q, qd);
+            else if (K == 2) set_butterflies<2, FWD>(e, tw, (u32)m0, (u32)blk, q, qd);
+            else set_butterflies<1, FWD>(e, tw, (u32)m0, (u32)blk, q, qd);
 #pragma unroll
             for (int i = 0; i < (1 << K); ++i) {
                 const int row = base + i * step;
                 if (g_last) {
                     const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
-                    u64 v = e[i];
-                    if (!FWD) v = mul_shoup(v, ninv, ninvs, q);                  // scale by N^{-1}, to [0, q)
-                    dst[gidx] = v;                                              // forward: lazy, below 4q
+                    if (FWD) {
+                        ((T*)dst)[gidx] = e[i];                 // lazy; the contiguous pass finishes
+                    } else if (FP) {                            // scale by N^{-1}, to [0, q)
+                        const bool mont = B.from_mont != 0;
+                        double v = __dadd_rn(fp_mul_centred(*(double*)&e[i], mont ? R.ninvm_d[mod] : R.ninv_d[mod],
+                                                            mont ? R.ninvm_q[mod] : R.ninv_q[mod], qd), qd);
+                        if (v >= qd) v = __dsub_rn(v, qd);
+                        dst[gidx] = d2u(v);
+                    } else {
+                        const bool mont = B.from_mont != 0;
+                        dst[gidx] = mul_shoup(*(u64*)&e[i], mont ? R.ninv_m[mod] : R.ninv[mod],
+                                              mont ? R.ninv_ms[mod] : R.ninvs[mod], q);
+                    }
                 } else {
                     sm[row * LANES + lane] = e[i];
                 }
@@ -217,39 +249,53 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     }
 }
 
-// Contiguous pass: every warp transforms one chunk of 256 adjacent points (8 per thread) through
-// the groups {3,3,2}; the chunk lives in the warp's own swizzled slice of shared memory between
-// groups, so only warp-level synchronisation is needed.
-// Forward: second pass (in place, final reduction to [0, q)).  Inverse: first pass (reads the batch
-// source, plain residues).
-template <bool FWD, bool EPI>
-__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const RingDev R, const PolyBatch B,
-                                                                       u32 chunks_per_block, const RotBatch rb,
-                                                                       const ModDownEpilogue epi) {
-    constexpr int LEN = 1 << LOG_C;
-    __shared__ u64 sm_all[CHUNKS_PER_BLOCK * LEN];
+template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
+__global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8),
+                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
+ntt_strided(const RingDev R, const PolyBatch B) {
+    __shared__ u64 sm[1 << (LOG_R + LOG_LANES)];
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
     const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
-    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) return;
+    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) {
+        // this digit's transform in its own prime exists already: copy the tile instead
+        const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
+        u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
+        for (int w = threadIdx.x; w < (1 << (LOG_R + LOG_LANES)); w += blockDim.x) {
+            const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * (1 << LOG_LANES) + (w & ((1 << LOG_LANES) - 1));
+            dd[gidx] = ds[gidx];
+        }
+        return;
+    }
+    if (R.fp_ok[mod]) strided_body<FWD, LOAD, LOG_R, LOG_LANES, true>(R, B, sm, o, m, mod);
+    else strided_body<FWD, LOAD, LOG_R, LOG_LANES, false>(R, B, sm, o, m, mod);
+}
+
+// Contiguous pass: every warp transforms one chunk of 256 adjacent points (8 per thread) through
+// the groups {3,3,2}; the chunk lives in the warp's own swizzled slice of shared memory between
+// groups, so only warp-level synchronisation is needed.
+// Forward: second pass (final reduction to [0, q), then the store functors).  Inverse: first pass
+// (reads the batch source: plain residues, tiled/limb-split plaintexts, or a sum of arrays).
+template <bool FWD, bool EPI, bool FP>
+__device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, u32 o, u32 m, u32 mod,
+                                            u32 chunk, int lane, const RotBatch& rb, const ModDownEpilogue& epi) {
+    typedef typename Elem<FP>::T T;
+    constexpr int LEN = 1 << LOG_C;
+    T* sm = (T*)sm_raw;
     const u64 q = R.q[mod];
+    const double qd = R.qd[mod];
     const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
     const u64* src = FWD ? dst : (const u64*)B.src + (size_t)o * B.src_so + (size_t)m * B.src_sm;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if ((u32)warp >= chunks_per_block) return;
-    const bool fp = R.fp_ok[mod] != 0;
-    const u32 chunk = blockIdx.x * chunks_per_block + warp;
     const u32 mult = (R.N >> LOG_C) + chunk;                   // twiddle index multiplier of this chunk
-    u64* sm = sm_all + warp * LEN;
     const u64* gsrc = src + (size_t)chunk * LEN;
     u64* gdst = dst + (size_t)chunk * LEN;
-    u64 e[8];
+    T e[8];
     if (FWD) {
         // group 0: K = 3, spacing 32
 #pragma unroll
-        for (int i = 0; i < 8; ++i) e[i] = gsrc[lane + 32 * i];
-        set_butterflies<3, true>(e, tw, 1u * mult, 0u, q, fp);
+        for (int i = 0; i < 8; ++i) e[i] = ((const T*)gsrc)[lane + 32 * i];
+        set_butterflies<3, true>(e, tw, 1u * mult, 0u, q, qd);
 #pragma unroll
         for (int i = 0; i < 8; ++i) sm[swz(lane + 32 * i)] = e[i];
         __syncwarp();
@@ -258,7 +304,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             const int blk = lane >> 2, base = blk * 32 + (lane & 3);
 #pragma unroll
             for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
-            set_butterflies<3, true>(e, tw, 8u * mult, (u32)blk, q, fp);
+            set_butterflies<3, true>(e, tw, 8u * mult, (u32)blk, q, qd);
 #pragma unroll
             for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
         }
@@ -269,32 +315,37 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             const int s = lane + 32 * it;
 #pragma unroll
             for (int i = 0; i < 4; ++i) e[i] = sm[swz(4 * s + i)];
-            set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, fp);
+            set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, qd);
+            u64 v4[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {   // final reduction [0, 4q) -> [0, q)
-                u64 v = e[i];
-                if (v >= 2 * q) v -= 2 * q;
-                if (v >= q) v -= q;
-                e[i] = v;
+            for (int i = 0; i < 4; ++i) {   // final reduction to [0, q)
+                if (FP) {
+                    v4[i] = d2u(fp_reduce(*(double*)&e[i], qd, R.qinv_d[mod]));
+                } else {
+                    u64 v = *(u64*)&e[i];
+                    if (v >= 2 * q) v -= 2 * q;
+                    if (v >= q) v -= q;
+                    v4[i] = v;
+                }
             }
             if (EPI) {
-                const u32 rot = o >> 1, comp = o & 1, i = mod, r = R.r, nb = r + 1;
+                const u32 rot = o >> 1, comp = o & 1, ip = mod, r = R.r, nb = r + 1;
                 const size_t n = (size_t)chunk * LEN + 4 * s;
-                const u64* up = epi.u + ((size_t)o * nb + i) * R.N + n;
+                const u64* up = epi.u + ((size_t)o * nb + ip) * R.N + n;
                 const ulonglong2 u0 = *(const ulonglong2*)up, u1 = *(const ulonglong2*)(up + 2);
                 const u64 uu[4] = {u0.x, u0.y, u1.x, u1.y};
                 u64 cc[4] = {0, 0, 0, 0};
                 if (comp == 0) {
-                    const u64* cp = epi.c0_base + (size_t)rb.c0[rot] * epi.c0_stride + (size_t)i * R.N + n;
+                    const u64* cp = epi.c0_base + (size_t)rb.c0[rot] * epi.c0_stride + (size_t)ip * R.N + n;
                     const ulonglong2 c0 = *(const ulonglong2*)cp, c1 = *(const ulonglong2*)(cp + 2);
                     cc[0] = c0.x; cc[1] = c0.y; cc[2] = c1.x; cc[3] = c1.y;
                 }
                 const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
                 const u32 pp[4] = {pv.x, pv.y, pv.z, pv.w};
-                u64* op = epi.out_base + (size_t)rb.out[rot] * epi.out_stride + ((size_t)comp * r + i) * R.N;
+                u64* op = epi.out_base + (size_t)rb.out[rot] * epi.out_stride + ((size_t)comp * r + ip) * R.N;
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    u64 v = mul_shoup(sub_mod(uu[t], e[t], q), R.pinv[i], R.pinvs[i], q);
+                    u64 v = mul_shoup(sub_mod(uu[t], v4[t], q), R.pinv[ip], R.pinvs[ip], q);
                     v = add_mod(v, cc[t], q);
                     op[pp[t]] = v;
                 }
@@ -302,21 +353,21 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             }
             if (B.split_bits) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) e[i] = limb_split(e[i], B.split_bits);
+                for (int i = 0; i < 4; ++i) v4[i] = limb_split(v4[i], B.split_bits);
             }
             if (B.scatter) {    // permuted store (keys are kept pre-permuted by their automorphism)
                 const u32* sc = B.scatter + (size_t)(o / B.scatter_div) * R.N + chunk * LEN + 4 * s;
                 u64* sd = B.scatter_dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sd[sc[i]] = e[i];
+                for (int i = 0; i < 4; ++i) sd[sc[i]] = v4[i];
                 continue;
             }
             ulonglong2* gp = (ulonglong2*)(gdst + 4 * s);
             if (B.tile_ptr)     // 4 adjacent coefficients never straddle a tile (tiles hold >= 16)
                 gp = (ulonglong2*)(B.tile_ptr + tile_word_offset(B.tile, (B.o_base + o) / B.tile.n_terms - B.tile_pj0,
                                                                  (B.o_base + o) % B.tile.n_terms, mod, chunk * LEN + 4 * s));
-            gp[0] = make_ulonglong2(e[0], e[1]);
-            gp[1] = make_ulonglong2(e[2], e[3]);
+            gp[0] = make_ulonglong2(v4[0], v4[1]);
+            gp[1] = make_ulonglong2(v4[2], v4[3]);
         }
     } else {
         // inverse: groups in the opposite order
@@ -329,21 +380,23 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
                                                                        (B.o_base + o) % B.tile.n_terms, mod,
                                                                        chunk * LEN + 4 * s));
             const ulonglong2 a = gp[0], b = gp[1];
-            e[0] = a.x; e[1] = a.y; e[2] = b.x; e[3] = b.y;
+            u64 v4[4] = {a.x, a.y, b.x, b.y};
+            if (B.split_bits) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) v4[i] = limb_join(v4[i], B.split_bits);
+            }
             if (B.sum_terms) {      // the input is a sum of several arrays of the same shape
                 const u64* sp = B.sum_src + (size_t)o * B.src_so + (size_t)m * B.src_sm + (size_t)chunk * LEN + 4 * s;
                 for (u32 t = 0; t < B.sum_terms; ++t) {
                     const ulonglong2 a2 = *(const ulonglong2*)(sp + (size_t)t * B.sum_stride);
                     const ulonglong2 b2 = *(const ulonglong2*)(sp + (size_t)t * B.sum_stride + 2);
-                    e[0] = add_mod(e[0], a2.x, q); e[1] = add_mod(e[1], a2.y, q);
-                    e[2] = add_mod(e[2], b2.x, q); e[3] = add_mod(e[3], b2.y, q);
+                    v4[0] = add_mod(v4[0], a2.x, q); v4[1] = add_mod(v4[1], a2.y, q);
+                    v4[2] = add_mod(v4[2], b2.x, q); v4[3] = add_mod(v4[3], b2.y, q);
                 }
             }
-            if (B.split_bits) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) e[i] = limb_join(e[i], B.split_bits);
-            }
-            set_butterflies<2, false>(e, tw, 64u * mult, (u32)s, q, fp);
+            for (int i = 0; i < 4; ++i) from_u64(e[i], v4[i]);
+            set_butterflies<2, false>(e, tw, 64u * mult, (u32)s, q, qd);
 #pragma unroll
             for (int i = 0; i < 4; ++i) sm[swz(4 * s + i)] = e[i];
         }
@@ -352,17 +405,34 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
             const int blk = lane >> 2, base = blk * 32 + (lane & 3);
 #pragma unroll
             for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
-            set_butterflies<3, false>(e, tw, 8u * mult, (u32)blk, q, fp);
+            set_butterflies<3, false>(e, tw, 8u * mult, (u32)blk, q, qd);
 #pragma unroll
             for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
         }
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 8; ++i) e[i] = sm[swz(lane + 32 * i)];
-        set_butterflies<3, false>(e, tw, 1u * mult, 0u, q, fp);
+        set_butterflies<3, false>(e, tw, 1u * mult, 0u, q, qd);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) gdst[lane + 32 * i] = e[i];      // lazy, below 2q; the strided pass finishes
+        for (int i = 0; i < 8; ++i) ((T*)gdst)[lane + 32 * i] = e[i];      // lazy, below 2q; the strided pass finishes
     }
+}
+
+template <bool FWD, bool EPI>
+__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const RingDev R, const PolyBatch B,
+                                                                       u32 chunks_per_block, const RotBatch rb,
+                                                                       const ModDownEpilogue epi) {
+    __shared__ u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
+    const u32 poly = blockIdx.y;
+    const u32 o = poly / B.n_m, m = poly % B.n_m;
+    const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
+    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if ((u32)warp >= chunks_per_block) return;
+    const u32 chunk = blockIdx.x * chunks_per_block + warp;
+    u64* sm = sm_all + (warp << LOG_C);
+    if (R.fp_ok[mod]) contig_body<FWD, EPI, true>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
+    else contig_body<FWD, EPI, false>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
 }
 
 NttGeometry ntt_geometry(u32 logN) {
