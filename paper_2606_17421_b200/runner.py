@@ -27,7 +27,8 @@ class WorkloadRunner:
     output ciphertext buffers."""
 
     def __init__(self, name: str, seed: int = 0, device: str = "cuda:0", cache: bool = True,
-                 cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None):
+                 cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None,
+                 fuse_shared_inputs: bool = True):
         self.w = wl.WORKLOADS[name]
         ps = wl.PARAM_SETS[self.w.params]
         self.N, self.primes, self.P, self.scale = ps["N"], list(ps["primes"]), ps["special"], ps["scale"]
@@ -58,10 +59,19 @@ class WorkloadRunner:
         # layers
         self.layers = []
         D = self.plan.D
+        if fuse_shared_inputs:      # q/k/v and gate/up read the same activation: one call over the stacked matrix
+            units = [wl.Layer(nm, d_in, sum(m.d_out for m in members)) for nm, d_in, members in
+                     wl.fuse_shared_inputs(self.w.layers, D)]
+            members_of = {nm: members for nm, _, members in wl.fuse_shared_inputs(self.w.layers, D)}
+        else:
+            units = list(self.w.layers)
+            members_of = {L.name: [L] for L in units}
         for rep in range(self.w.n_repeat):
-            for L in self.w.layers:
+            for L in units:
                 n_in, n_out = wl.ceil_div(L.d_in, D), wl.ceil_div(L.d_out, D)
-                W = torch.from_numpy(wl.gen_weights(seed, f"{L.name}.{rep}", L.d_out, L.d_in)).to(self.device)
+                W = torch.from_numpy(np.concatenate(
+                    [wl.gen_weights(seed, f"{m.name}.{rep}", m.d_out, m.d_in) for m in members_of[L.name]], axis=0)
+                ).to(self.device)
                 handle = None
                 if cache:
                     try:

@@ -48,6 +48,9 @@ class Layer:
     name: str
     d_in: int
     d_out: int
+    input: str = ""             # projections of one transformer layer with the same non-empty tag read the same
+                                # activation: a caller may stack their weight matrices row-wise into one call
+                                # (output row blocks are independent, so every residue is unchanged)
 
 
 @dataclass(frozen=True)
@@ -62,12 +65,26 @@ class Workload:
 
 GPT2_LAYER = (Layer("qkv", 768, 2304), Layer("out_proj", 768, 768),
               Layer("ffn_up", 768, 3072), Layer("ffn_down", 3072, 768))
-QWEN3_LAYER = (Layer("q", 1024, 2048), Layer("k", 1024, 1024), Layer("v", 1024, 1024),
-               Layer("o", 2048, 1024), Layer("gate", 1024, 3072), Layer("up", 1024, 3072),
+QWEN3_LAYER = (Layer("q", 1024, 2048, "attn"), Layer("k", 1024, 1024, "attn"), Layer("v", 1024, 1024, "attn"),
+               Layer("o", 2048, 1024), Layer("gate", 1024, 3072, "ffn"), Layer("up", 1024, 3072, "ffn"),
                Layer("down", 3072, 1024))
-LLAMA3_8B_LAYER = (Layer("q", 4096, 4096), Layer("k", 4096, 1024), Layer("v", 4096, 1024),
-                   Layer("o", 4096, 4096), Layer("gate", 4096, 14336), Layer("up", 4096, 14336),
+LLAMA3_8B_LAYER = (Layer("q", 4096, 4096, "attn"), Layer("k", 4096, 1024, "attn"), Layer("v", 4096, 1024, "attn"),
+                   Layer("o", 4096, 4096), Layer("gate", 4096, 14336, "ffn"), Layer("up", 4096, 14336, "ffn"),
                    Layer("down", 14336, 4096))
+
+
+def fuse_shared_inputs(layers, D: int):
+    """Group consecutive projections that read the same activation: [(fused name, d_in, [member layers])].
+    Members must have d_out a multiple of the tile side D so that their row blocks stay aligned."""
+    groups = []
+    for L in layers:
+        if groups and L.input and groups[-1][2][-1].input == L.input and groups[-1][1] == L.d_in \
+                and all(m.d_out % D == 0 for m in groups[-1][2]):
+            groups[-1][2].append(L)
+            groups[-1][0] += "+" + L.name
+        else:
+            groups.append([L.name, L.d_in, [L]])
+    return [(name, d_in, members) for name, d_in, members in groups]
 
 WORKLOADS = {
     "tiny": Workload("tiny", "n12", PlanSpec(64, 1, 8, 8), (Layer("w", 64, 64),)),

@@ -262,6 +262,30 @@ def test_llama3_layer_shapes_sampled_blocks():
     check_blocks(par, plan, pick, lambda L, n_out: [n_out - 1], 13)
 
 
+def test_stacking_projections_that_share_an_input_changes_no_residue():
+    # q/k/v (or gate/up) read the same activation: one call over the row-stacked matrix must give
+    # exactly the ciphertexts of the separate calls
+    par = oracle_params("n12")
+    plan = ckks.Plan(64, 4, 4, 4)
+    s = ckks.keygen(par, 21)
+    keys = ckks.make_rotation_keys(par, s, plan, 21)
+    x = wl.gen_activation(21, "shared", 100)
+    cts = ckks.encrypt_vector(par, plan, s, x, 21)
+    W1 = wl.gen_weights(21, "w1", 128, 100)
+    W2 = wl.gen_weights(21, "w2", 64, 100)
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys)
+        o1 = g.to_host_u64(g.linear(cts, W1, 128, 100))
+        o2 = g.to_host_u64(g.linear(cts, W2, 64, 100))
+        both = g.to_host_u64(g.linear(cts, np.concatenate([W1, W2]), 192, 100))
+        assert np.array_equal(both[:2], o1) and np.array_equal(both[2:], o2)
+        expect = ckks.linear(par, plan, cts, W2, keys)
+        assert np.array_equal(o2[0], expect[0])
+    finally:
+        g.close()
+
+
 def test_structured_matrices_on_device():
     par = oracle_params("n12")
     plan = ckks.Plan(64, 4, 4, 4)
