@@ -33,9 +33,6 @@ NCU_TRAFFIC_BYTES = {
     "gpt2_qkv": {"mac": None, "ntt_fwd_strided": None},
 }
 
-# 32-bit multiply-adds that one butterfly (x*w mod q by Shoup's method: one 64x64 high product and
-# two 64x64 low products) cannot do without: 4 + 3 + 3.
-IMAD_PER_BUTTERFLY = 10
 
 
 def read_peaks():
@@ -96,21 +93,31 @@ class ClockSampler(threading.Thread):
 
 
 def butterflies_per_step(runner) -> dict:
-    """Butterfly counts of the transforms one step launches, by kernel category."""
+    """Transforms one step launches, by direction and by arithmetic path.  Moduli below 2^41 run in
+    fp64 (9 fp64 operations per forward butterfly), the others in integers (at least 10 32-bit
+    multiply-adds per butterfly); both pipes issue 64 lanes per clock per SM."""
     import math
     r, N = runner.r, runner.N
     b, g = runner.plan.b, runner.plan.g
     per = (N // 2) * int(math.log2(N))
-    fwd = inv = 0
+    fp = [q < (1 << 41) for q in runner.primes] + [runner.P < (1 << 41)]
+    fwd = [0] * (r + 1)
+    inv = [0] * (r + 1)
     for e in runner.layers:
         n_in, n_out = e["n_in"], e["n_out"]
         n_giant = (g - 1) * n_out
-        # input transforms, ModUp (a digit in its own prime is copied, not transformed), lifted P-residues
-        fwd += n_in * (2 * r + (r * r if b > 1 else 0) + (b - 1) * 2 * r)
-        inv += n_in * (b - 1) * 2
-        fwd += n_giant * (r * r + 2 * r)
-        inv += n_giant * (r + 2) + n_out * 2 * r
-    return {"fwd_polys": fwd, "inv_polys": inv, "per_poly": per}
+        sets = (n_in if b > 1 else 0) + n_giant            # ModUp digit sets
+        rots = n_in * (b - 1) + n_giant                    # key switches
+        for i in range(r):
+            fwd[i] += 2 * n_in + sets * (r - 1) + 2 * rots # inputs; digits of the other primes; lifted P-residues
+            inv[i] += n_giant + 2 * n_out                  # c1 of the giant-step inputs; outputs
+        fwd[r] += sets * r
+        inv[r] += 2 * rots                                 # P-residues of the inner products
+    def summary(cnt):
+        polys = sum(cnt)
+        ops = sum(c * (9 if f else 10) for c, f in zip(cnt, fp))
+        return {"polys": polys, "fp64_polys": sum(c for c, f in zip(cnt, fp) if f), "ops_per_butterfly": ops / max(1, polys)}
+    return {"fwd": summary(fwd), "inv": summary(inv), "per_poly": per}
 
 
 def time_extra_workload(name: str, steps: int, cache_budget_bytes=None) -> dict:
@@ -254,28 +261,23 @@ def run_ours(args):
                                           "frac": round(ach / hbm_peak, 4), "of": peak_kind, "traffic": None,
                                           "launches_per_step": ki_n, "avg_ms": round(ki_ms, 5),
                                           "note": "bytes = one key per rotation; rotations sharing a key hit L2"}
-    # transforms: integer multiply-add bound
-    for cats, polys, label in ((("ntt_fwd_strided", "ntt_fwd_contig"), bfly["fwd_polys"], "ntt_forward"),
-                               (("ntt_inv_contig", "ntt_inv_strided"), bfly["inv_polys"], "ntt_inverse")):
+    # transforms: bound by the arithmetic pipes (fp64 for the 40-bit primes, integer multiply-add for the rest)
+    sm_mhz = clocks.get("sm_mhz") or 1965.0
+    lanes_per_s = 148 * 64 * sm_mhz * 1e6                  # either pipe: 148 SMs x 64 lanes x clock
+    for cats, key, label in ((("ntt_fwd_strided", "ntt_fwd_contig"), "fwd", "ntt_forward"),
+                             (("ntt_inv_contig", "ntt_inv_strided"), "inv", "ntt_inverse")):
         ms_step = sum(kstats[c][1] for c in cats) / K
         if ms_step > 0:
-            mads = polys * bfly["per_poly"] * IMAD_PER_BUTTERFLY
-            ach = mads / (ms_step * 1e-3) / 1e12
-            rooflines[label] = {"bound": "alu", "achieved": round(ach, 3), "peak": round(imad_rate / 1e12, 3),
-                                "unit": "T mad.wide.u32/s", "frac": round(ach / (imad_rate / 1e12), 4),
-                                "of": "measured probe (bf_measure_imad_rate), 10 multiply-adds per butterfly",
+            info = bfly[key]
+            rate = info["polys"] * bfly["per_poly"] / (ms_step * 1e-3)
+            peak = lanes_per_s / info["ops_per_butterfly"]
+            rooflines[label] = {"bound": "alu", "achieved": round(rate / 1e9, 1), "peak": round(peak / 1e9, 1),
+                                "unit": "G butterflies/s", "frac": round(rate / peak, 4),
+                                "of": (f"derived: 148 SMs x 64 lanes x {sm_mhz:.0f} MHz / {info['ops_per_butterfly']:.2f} "
+                                       "pipe operations per butterfly (9 fp64 ops on the fp64 path, 10 multiply-adds on "
+                                       f"the integer path); bf_measure_imad_rate measured {imad_rate / 1e12:.2f} T multiply-adds/s"),
                                 "traffic": traffic.get(cats[0]), "ms_per_step": round(ms_step, 5),
-                                "polys_per_step": polys,
-                                "butterflies_per_s": round(polys * bfly["per_poly"] / (ms_step * 1e-3) / 1e9, 2)}
-    # integer multiply-add peak from unit counts and the clock held during the run: 148 SMs x 64 lanes
-    sm_mhz = clocks.get("sm_mhz") or 1965.0
-    imad_derived = 148 * 64 * sm_mhz * 1e6
-    for k in ("ntt_forward", "ntt_inverse"):
-        if k in rooflines:
-            rooflines[k]["peak"] = round(imad_derived / 1e12, 3)
-            rooflines[k]["frac"] = round(rooflines[k]["achieved"] / (imad_derived / 1e12), 4)
-            rooflines[k]["of"] = ("derived: 148 SMs x 64 multiply-add lanes x sampled SM clock; the probe "
-                                  f"bf_measure_imad_rate measured {imad_rate / 1e12:.2f} T/s; 10 multiply-adds per butterfly")
+                                "polys_per_step": info["polys"], "fp64_polys_per_step": info["fp64_polys"]}
     total_k_ms = sum(v[1] for v in kstats.values())
     shares = {k: round(v[1] / total_k_ms, 4) for k, v in kstats.items() if v[0]}
     dominant = max(shares, key=shares.get)

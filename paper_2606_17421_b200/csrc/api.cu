@@ -725,7 +725,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
                     rb.out[t] = (int)((q0 + q) * b + k);
                 }
             }
-            CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->stream));
+            CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->device_error, ctx->stream));
             TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
         }
     }
@@ -779,7 +779,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
             rb.c0[t] = (int)t;
             rb.out[t] = (int)t;
         }
-        CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->stream));
+        CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->device_error, ctx->stream));
         TRY(moddown_batch(ctx, rb, Asrc, (long long)ctw, Rres + (size_t)rho0 * ctw, (long long)ctw));
     }
     stamp(ctx, 3);
@@ -862,7 +862,8 @@ extern "C" int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uin
     rb.n = 1;
     rb.key[0] = key;
     rb.out[0] = 1;
-    CK(launch_key_inner_product(ctx->ring, rb, (const u64*)ctx->Dig.p, ctx->keys, (u64*)ctx->U.p, ctx->stream));
+    CK(launch_key_inner_product(ctx->ring, rb, (const u64*)ctx->Dig.p, ctx->keys, (u64*)ctx->U.p, ctx->device_error,
+                                ctx->stream));
     TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
     memset(&B, 0, sizeof(B));
     B.src = X + ctw;

@@ -61,7 +61,7 @@ cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* 
                                  u32 mod0, cudaStream_t stream);
 // u'[rot][comp][m][n] = sum_j dig[dig(rot)][j][m][n] * key'[key(rot)][j][comp][m][n]  (keys pre-permuted)
 cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
-                                     cudaStream_t stream);
+                                     int* error_flag, cudaStream_t stream);
 u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintext format (0 = whole words)
 TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms);   // layout of n_pj groups of n_terms diagonals
 size_t mac_tile_words(const RingHost& ring, const TileLayout& t);           // words that layout occupies

@@ -338,81 +338,90 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 // Key-switch inner product over the extended basis (Sec. 4.2 "key-switching primitives").
 // The rotation keys are stored pre-permuted by their automorphism, so the product runs in the
 // un-rotated index space with fully coalesced operands:
-//   u'[rot][comp][m][n] = sum_j digit_j[m][n] * key'[key(rot)][j][comp][m][n]
+//   u'[rot][comp][m][n] = sum_j dig[dig(rot)][j][m][n] * key'[key(rot)][j][comp][m][n]
 // and the automorphism is applied once, as a scatter, when the rotated ciphertext is assembled.
-// digit_j in its own prime (m == j) is the transform of c1 itself and is read from the source
-// ciphertext instead of the digit buffer.  Two coefficients per thread, 128-bit loads; the key
-// stream is read once per rotation.
-template <bool SMALL, int RR>
-__device__ __forceinline__ void key_inner_body(const RingDev& R, u32 r, u32 m, const u64* __restrict__ dp,
-                                               const u64* __restrict__ kp, u64* __restrict__ up) {
-    const u32 N = R.N, nb = r + 1;
-    LimbAcc<SMALL> a00, a01, a10, a11;                  // [component][word]
-    if (RR > 0) {
-        // the number of digits is known at compile time: every load is issued before the first product
-        ulonglong2 d[RR > 0 ? RR : 1], k0[RR > 0 ? RR : 1], k1[RR > 0 ? RR : 1];
-#pragma unroll
-        for (int j = 0; j < RR; ++j) {
-            d[j] = *(const ulonglong2*)(dp + (size_t)j * nb * N);
-            k0[j] = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2) * nb * N));
-            k1[j] = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2 + 1) * nb * N));
-        }
-#pragma unroll
-        for (int j = 0; j < RR; ++j) {
-            a00.mac(d[j].x, k0[j].x);
-            a01.mac(d[j].y, k0[j].y);
-            a10.mac(d[j].x, k1[j].x);
-            a11.mac(d[j].y, k1[j].y);
-        }
-    } else {
-#pragma unroll 4
-        for (u32 j = 0; j < r; ++j) {
-            const ulonglong2 d = *(const ulonglong2*)(dp + (size_t)j * nb * N);
-            const ulonglong2 k0 = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2) * nb * N));
-            const ulonglong2 k1 = __ldcs((const ulonglong2*)(kp + (size_t)(j * 2 + 1) * nb * N));
-            a00.mac(d.x, k0.x);
-            a01.mac(d.y, k0.y);
-            a10.mac(d.x, k1.x);
-            a11.mac(d.y, k1.y);
-        }
-    }
-    const u64 q = R.q[m], mu = R.mu[m], c64 = R.c64[m], c64s = R.c64s[m];
-    *(ulonglong2*)up = make_ulonglong2(a00.reduce(q, mu, c64, c64s), a01.reduce(q, mu, c64, c64s));
-    *(ulonglong2*)(up + (size_t)nb * N) = make_ulonglong2(a10.reduce(q, mu, c64, c64s), a11.reduce(q, mu, c64, c64s));
-}
-
+// The key stream is read once per rotation; products accumulate as 32-bit limb partial sums
+// (with carry counters where the 60-bit special prime needs them), one reduction per output word.
 // grid: x = rotation (fastest, so that rotations sharing a key or a digit set run side by side and
-// meet in L2), y = tile of 512 coefficients, z = modulus of the extended basis
-template <int RR>
-__global__ void __launch_bounds__(256) key_inner_product_kernel(const RingDev R, const RotBatch rb,
-                                                                const u64* __restrict__ dig,
-                                                                const u64* __restrict__ keys, u64* __restrict__ u,
-                                                                u32 small_ok) {
+// meet in L2), y = tile, z = modulus of the extended basis.
+//
+// Bulk-copy version: a block owns one (rotation, modulus, tile of 256 coefficients).  Its 3r operand
+// segments (digit, key.b, key.a for every digit j; 2 KB each) are fetched by asynchronous bulk
+// copies into shared memory in one go, so the number of bytes in flight does not depend on
+// registers; several blocks per SM overlap one block's arithmetic with the others' copies.
+constexpr int KI_TILE = 256;
+
+__global__ void __launch_bounds__(KI_TILE, 4) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
+                                                                    const u64* __restrict__ dig,
+                                                                    const u64* __restrict__ keys, u64* __restrict__ u,
+                                                                    u32 small_ok, int* __restrict__ error_flag) {
+    extern __shared__ __align__(128) unsigned char ki_smem[];
     const u32 rot = blockIdx.x, m = blockIdx.z;
     const u32 N = R.N, r = R.r, nb = r + 1;
-    const u32 n = (blockIdx.y * blockDim.x + threadIdx.x) * 2;
-    const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + n;
-    const u64* kp = keys + ((size_t)rb.key[rot] * r * 2 * nb + m) * N + n;
-    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n;
-    if (m < r && small_ok) key_inner_body<true, RR>(R, r, m, dp, kp, up);
-    else key_inner_body<false, RR>(R, r, m, dp, kp, up);
+    const u32 n0 = blockIdx.y * KI_TILE;
+    u64* sd = (u64*)ki_smem;                        // [r][KI_TILE] digits
+    u64* sk = sd + (size_t)r * KI_TILE;             // [r][2][KI_TILE] key components
+    u64* bar = sk + (size_t)2 * r * KI_TILE;
+    const u32 tid = threadIdx.x;
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid < 32) {
+        if (tid == 0) mbar_expect_tx(bar, 3 * r * KI_TILE * 8);
+        __syncwarp();
+        const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + n0;
+        const u64* kp = keys + ((size_t)rb.key[rot] * r * 2 * nb + m) * N + n0;
+        for (u32 e = tid; e < 3 * r; e += 32) {
+            const u32 j = e / 3, which = e % 3;
+            if (which == 0) bulk_g2s(sd + (size_t)j * KI_TILE, dp + (size_t)j * nb * N, KI_TILE * 8, bar);
+            else bulk_g2s(sk + ((size_t)j * 2 + (which - 1)) * KI_TILE, kp + (size_t)(j * 2 + (which - 1)) * nb * N,
+                          KI_TILE * 8, bar);
+        }
+    }
+    mbar_wait(bar, 0, error_flag);
+    const u64 q = R.q[m], mu = R.mu[m], c64 = R.c64[m], c64s = R.c64s[m];
+    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
+    if (m < r && small_ok) {
+        LimbAcc<true> a0, a1;
+        for (u32 j = 0; j < r; ++j) {
+            const u64 d = sd[j * KI_TILE + tid];
+            a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
+            a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+        }
+        up[0] = a0.reduce(q, mu, c64, c64s);
+        up[(size_t)nb * N] = a1.reduce(q, mu, c64, c64s);
+    } else {
+        LimbAcc<false> a0, a1;
+        for (u32 j = 0; j < r; ++j) {
+            const u64 d = sd[j * KI_TILE + tid];
+            a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
+            a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+        }
+        up[0] = a0.reduce(q, mu, c64, c64s);
+        up[(size_t)nb * N] = a1.reduce(q, mu, c64, c64s);
+    }
 }
 
 cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
-                                     cudaStream_t stream) {
+                                     int* error_flag, cudaStream_t stream) {
     if (rb.n == 0) return cudaSuccess;
     u64 qmax = 0;
     for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
     // without a carry counter the middle partial sum takes r <= 15 terms below 2^51 each
     const u32 small_ok = (qmax < ((u64)1 << 50)) ? 1u : 0u;
-    dim3 grid(rb.n, ring.dev.N / 512, ring.dev.r + 1);
     ProfScope prof(ring.prof, CAT_KEY_INNER, stream);
-    switch (ring.dev.r) {
-        case 3: key_inner_product_kernel<3><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
-        case 7: key_inner_product_kernel<7><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
-        case 9: key_inner_product_kernel<9><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
-        default: key_inner_product_kernel<0><<<grid, 256, 0, stream>>>(ring.dev, rb, dig, keys, u, small_ok); break;
+    const u32 r = ring.dev.r;
+    const size_t smem = (size_t)3 * r * KI_TILE * 8 + 16;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(key_inner_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
     }
+    dim3 grid(rb.n, ring.dev.N / KI_TILE, r + 1);
+    key_inner_bulk_kernel<<<grid, KI_TILE, smem, stream>>>(ring.dev, rb, dig, keys, u, small_ok, error_flag);
     return cudaGetLastError();
 }
 

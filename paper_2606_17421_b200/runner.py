@@ -81,8 +81,9 @@ class WorkloadRunner:
                             raise
                 ct_in = _uniform_residues(self.gen, self.primes, (n_in, 2), self.N, self.device)
                 ct_out = torch.empty((n_out, 2, self.r, self.N), dtype=torch.int64, device=self.device)
+                ct_low = torch.empty((n_out, 2, self.r - 1, self.N), dtype=torch.int64, device=self.device)
                 self.layers.append(dict(layer=L, rep=rep, n_in=n_in, n_out=n_out, W=W, handle=handle,
-                                        ct_in=ct_in, ct_out=ct_out,
+                                        ct_in=ct_in, ct_out=ct_out, ct_low=ct_low,
                                         pt_bytes=n_in * n_out * (D // self.plan.tau) * self.r * self.N * 8))
         torch.cuda.synchronize()
 
@@ -93,7 +94,7 @@ class WorkloadRunner:
             L = e["layer"]
             bf.bf_linear(self.ctx, e["ct_in"], e["n_in"], e["handle"], None if e["handle"] else e["W"],
                          L.d_out, L.d_in, e["ct_out"], e["n_out"])
-            bf.bf_rescale(self.ctx, e["ct_out"], e["ct_out"], e["n_out"], self.r)
+            bf.bf_rescale(self.ctx, e["ct_out"], e["ct_low"], e["n_out"], self.r)
 
     def make_host_buffers(self):
         for e in self.layers:
