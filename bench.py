@@ -172,7 +172,7 @@ def run_ours(args):
     bf.load()   # fails loudly when the CUDA library is missing
     # every rank decodes its own token stream (independent problems: no data-path collective)
     R = WorkloadRunner(args.workload, seed=rank, device=f"cuda:{local}")
-    stream = torch.cuda.current_stream()
+    stream = R.stream                       # the runner's own stream, made torch's current stream
 
     def barrier():
         torch.cuda.synchronize()

@@ -106,6 +106,13 @@ void bf_weights_free(bf_ctx* ctx, bf_weights* w);
 int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
               const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out);
 
+/* bf_linear replays a captured CUDA graph of its launch sequence from the third call with the same
+ * (ct_in, pt_weights, ct_out, d_out, d_in) on: the first call runs directly (and sizes the scratch),
+ * the second is captured.  Replay is skipped on the fallback path, while stage or kernel timing is
+ * on, and when the context's stream is itself being captured.  bf_set_graph_replay(ctx, 0) turns
+ * it off and drops the stored graphs (default: on). */
+int bf_set_graph_replay(bf_ctx* ctx, int on);
+
 /* Rescale (Sec. 2.1): drop the last prime of n_ct ciphertexts that have `level` primes each,
  *     c'_i = (c_i - centred(c_{level-1})) * q_{level-1}^{-1} mod q_i ,
  * i.e. round(c / q_{level-1}).  ct_in: device [n_ct][2][level][N]; ct_out: device

@@ -51,6 +51,7 @@ _SIGNATURES = {
     "bf_encode_weights": (ctypes.c_int, [_vp, _vp, _u32, _u32, ctypes.POINTER(_vp)]),
     "bf_weights_free": (None, [_vp, _vp]),
     "bf_linear": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
+    "bf_set_graph_replay": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_rescale": (ctypes.c_int, [_vp, _vp, _vp, _u32, _u32, ctypes.POINTER(ctypes.c_double)]),
     "bf_linear_host": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
     "bf_rotate": (ctypes.c_int, [_vp, _vp, _u32, _vp]),
@@ -157,6 +158,10 @@ def bf_weights_free(ctx, w):
 def bf_linear(ctx, ct_in, n_in: int, pt_weights, W_raw, d_out: int, d_in: int, ct_out, n_out: int):
     _check(load().bf_linear(ctx, _ptr(ct_in), n_in, pt_weights, _ptr(W_raw), d_out, d_in, _ptr(ct_out), n_out),
            "bf_linear", ctx)
+
+
+def bf_set_graph_replay(ctx, on: bool):
+    _check(load().bf_set_graph_replay(ctx, 1 if on else 0), "bf_set_graph_replay", ctx)
 
 
 def bf_rescale(ctx, ct_in, ct_out, n_ct: int, level: int, scale: float | None = None):

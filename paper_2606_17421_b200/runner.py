@@ -36,7 +36,10 @@ class WorkloadRunner:
         self.plan = self.w.plan
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
-        self.stream = stream or torch.cuda.current_stream()
+        # a stream of our own: the legacy default stream cannot be captured, which would keep the
+        # library from replaying its launch sequences as CUDA graphs
+        self.stream = stream or torch.cuda.Stream(device=self.device)
+        torch.cuda.set_stream(self.stream)
         self.gen = torch.Generator(device=self.device)
         self.gen.manual_seed(seed)
         self.ctx = bf.bf_ctx_create(self.N, self.primes + [self.P], self.r, self.scale,

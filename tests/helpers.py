@@ -24,6 +24,10 @@ class GpuSide:
         self.torch, self.bf = torch, bf
         self.par, self.plan = par, plan
         self.dev = torch.device("cuda:0")
+        # work on a stream of our own: the legacy default stream cannot be captured, and bf_linear
+        # replays captured launch sequences
+        self.stream = torch.cuda.Stream(device=self.dev)
+        torch.cuda.set_stream(self.stream)
         p = bf.bf_plan(plan.D, plan.tau, plan.b, plan.g)
         self.ctx = bf.bf_ctx_create(par.N, par.basis, par.r, par.scale, p,
                                     torch.cuda.current_stream().cuda_stream)

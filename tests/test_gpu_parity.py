@@ -269,6 +269,42 @@ def test_linear_with_the_papers_own_parameter_set():
     run_case(par, ckks.Plan(256, 16, 4, 4), 300, 520, 4, 1e-2, "paper_n13", tight=1e-3)   # scale 2^30: coarser
 
 
+def test_repeated_calls_replay_a_graph_and_still_read_fresh_inputs():
+    # from the third call with the same buffers on, bf_linear replays a captured launch sequence; the
+    # data in those buffers may change between calls and results must follow
+    par = oracle_params("n12")
+    plan = ckks.Plan(64, 4, 4, 4)
+    s = ckks.keygen(par, 31)
+    keys = ckks.make_rotation_keys(par, s, plan, 31)
+    W = wl.gen_weights(31, "graph", 100, 130)
+    xs = [wl.gen_activation(31, f"graph{t}", 130) for t in range(2)]
+    cts = [ckks.encrypt_vector(par, plan, s, x, 31 + t) for t, x in enumerate(xs)]
+    expect = [ckks.linear(par, plan, c, W, keys) for c in cts]
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys)
+        w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), 100, 130)
+        ct_in = g.to_dev(np.stack(cts[0]))
+        ct_out = g.empty_u64(2, 2, par.r, par.N)
+        g.bf.bf_get_kernel_stats(g.ctx)            # reset the launch counters
+        for call in range(6):
+            which = call % 2
+            ct_in.copy_(g.to_dev(np.stack(cts[which])))
+            g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
+            got = g.to_host_u64(ct_out)
+            for p in range(2):
+                assert np.array_equal(got[p], expect[which][p]), (call, p)
+        stats = g.bf.bf_get_kernel_stats(g.ctx)
+        per_call = sum(v[0] for v in stats.values()) / 6
+        assert per_call == int(per_call) and per_call > 5       # replays are counted like direct launches
+        # turning replay off gives the same results
+        g.bf.bf_set_graph_replay(g.ctx, False)
+        g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
+        assert np.array_equal(g.to_host_u64(ct_out)[0], expect[1][0])
+    finally:
+        g.close()
+
+
 def test_stacking_projections_that_share_an_input_changes_no_residue():
     # q/k/v (or gate/up) read the same activation: one call over the row-stacked matrix must give
     # exactly the ciphertexts of the separate calls
