@@ -168,6 +168,7 @@ def run_ours(args):
 
     from paper_2606_17421_b200 import bifrost as bf
     from paper_2606_17421_b200.runner import WorkloadRunner
+    from paper_2606_17421_b200.replicas import job_ms_per_token, max_over_ranks
 
     bf.load()   # fails loudly when the CUDA library is missing
     # every rank decodes its own token stream (independent problems: no data-path collective)
@@ -190,11 +191,7 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         t1 = time.time()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), device="cuda")
         return ms, t0, t1
 
     for _ in range(max(args.warmup, 3)):
@@ -288,7 +285,7 @@ def run_ours(args):
 
     h2d, d2h = R.host_bytes_per_step()
     line = {
-        "metric": METRIC, "value": round(ms_per_step / world, 5), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": round(job_ms_per_token(ms_per_step, world), 5), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5),
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
         "config": {"workload": args.workload, "ring_N": R.N, "ct_primes": R.r,
@@ -299,7 +296,7 @@ def run_ours(args):
                    "multi_gpu": "replicas: every rank decodes its own token, no data-path collective"},
         "tokens_per_s": round(world * 1e3 / ms_per_step, 3),
         "clocks": clocks,
-        "e2e": {"value": round(e2e_ms / world, 5), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": round(job_ms_per_token(e2e_ms, world), 5), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": gpu_launches,
         "roofline": roofline,

@@ -38,7 +38,8 @@ enum {
     BF_ERR_OOM = -6,           /* encoded weights exceed the cache budget, or device memory is exhausted */
     BF_ERR_CUDA = -7,          /* a CUDA call failed; see bf_last_cuda_error() */
     BF_ERR_RANGE = -8,         /* an encoded coefficient does not fit 2^62 (scale too large for the data) */
-    BF_ERR_TOO_LARGE = -9      /* more work than the fixed scratch of an allocation-free entry point holds */
+    BF_ERR_TOO_LARGE = -9,     /* more work than the fixed scratch of an allocation-free entry point holds */
+    BF_ERR_TIMEOUT = -10       /* a device-side wait on an asynchronous copy hit its poll limit */
 };
 
 typedef struct bf_ctx bf_ctx;          /* ring tables, rotation keys, scratch memory */
@@ -167,6 +168,13 @@ int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, uint32_t q, 
  * bf_get_stage_ms synchronises the stream. */
 int bf_set_stage_timing(bf_ctx* ctx, int on);
 int bf_get_stage_ms(bf_ctx* ctx, float* ms_out /* host, 4 values */);
+
+/* Kernels that wait on asynchronous copies poll with a limit; when a wait gives up the kernel
+ * records it and still terminates.  bf_device_status synchronises the stream and returns
+ * BF_ERR_TIMEOUT if that happened since the last check (the affected call's results are invalid),
+ * BF_ERR_RANGE for an encoder overflow on the fallback path, else BF_OK.  bf_linear_host performs
+ * this check itself. */
+int bf_device_status(bf_ctx* ctx);
 
 /* Launch accounting.  The library counts its kernel launches per category; with
  * bf_set_kernel_timing(ctx, 1) it also brackets every launch with a pair of CUDA events on the

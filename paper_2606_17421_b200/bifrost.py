@@ -22,6 +22,7 @@ BF_ERR_OOM = -6
 BF_ERR_CUDA = -7
 BF_ERR_RANGE = -8
 BF_ERR_TOO_LARGE = -9
+BF_ERR_TIMEOUT = -10
 
 
 class bf_plan(ctypes.Structure):
@@ -51,6 +52,7 @@ _SIGNATURES = {
     "bf_encode_weights": (ctypes.c_int, [_vp, _vp, _u32, _u32, ctypes.POINTER(_vp)]),
     "bf_weights_free": (None, [_vp, _vp]),
     "bf_linear": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
+    "bf_device_status": (ctypes.c_int, [_vp]),
     "bf_set_graph_replay": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_rescale": (ctypes.c_int, [_vp, _vp, _vp, _u32, _u32, ctypes.POINTER(ctypes.c_double)]),
     "bf_linear_host": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
@@ -158,6 +160,11 @@ def bf_weights_free(ctx, w):
 def bf_linear(ctx, ct_in, n_in: int, pt_weights, W_raw, d_out: int, d_in: int, ct_out, n_out: int):
     _check(load().bf_linear(ctx, _ptr(ct_in), n_in, pt_weights, _ptr(W_raw), d_out, d_in, _ptr(ct_out), n_out),
            "bf_linear", ctx)
+
+
+def bf_device_status(ctx):
+    """Synchronises; raises if a device-side wait gave up or the on-the-fly encoder overflowed."""
+    _check(load().bf_device_status(ctx), "bf_device_status", ctx)
 
 
 def bf_set_graph_replay(ctx, on: bool):

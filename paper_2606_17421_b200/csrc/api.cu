@@ -179,6 +179,7 @@ extern "C" const char* bf_strerror(int code) {
         case BF_ERR_OOM: return "out of memory or over the cache budget";
         case BF_ERR_CUDA: return "CUDA error";
         case BF_ERR_RANGE: return "encoded coefficient out of range";
+        case BF_ERR_TIMEOUT: return "a bounded device-side wait gave up (results of that call are invalid)";
         case BF_ERR_TOO_LARGE: return "request exceeds the fixed capacity of the allocation-free entry point";
         default: return "unknown error";
     }
@@ -518,15 +519,21 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
     return BF_OK;
 }
 
+// Reads the two device-side flags (encoder range overflow; a bounded wait that gave up).  Synchronises.
 static int check_overflow(bf_ctx* ctx) {
-    int flag = 0;
-    CK(cudaMemcpyAsync(&flag, ctx->overflow_flag, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    int flags[2] = {0, 0};
+    CK(cudaMemcpyAsync(flags, ctx->overflow_flag, 2 * sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
     CK(cudaStreamSynchronize(ctx->stream));
-    if (flag) {
-        CK(cudaMemsetAsync(ctx->overflow_flag, 0, sizeof(int), ctx->stream));
-        return BF_ERR_RANGE;
+    if (flags[0] || flags[1]) {
+        CK(cudaMemsetAsync(ctx->overflow_flag, 0, 2 * sizeof(int), ctx->stream));
+        return flags[1] ? BF_ERR_TIMEOUT : BF_ERR_RANGE;
     }
     return BF_OK;
+}
+
+extern "C" int bf_device_status(bf_ctx* ctx) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    return check_overflow(ctx);
 }
 
 extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, uint32_t d_in, bf_weights** out) {
@@ -947,8 +954,7 @@ extern "C" int bf_linear_host(bf_ctx* ctx, const uint64_t* host_ct_in, uint32_t 
     TRY(bf_rescale(ctx, (const u64*)ctx->stage_out.p, (u64*)ctx->stage_out.p, n_out, ctx->r, nullptr));
     const size_t out_bytes = (size_t)n_out * 2 * (ctx->r - 1) * ctx->N * 8;
     CK(cudaMemcpyAsync(host_ct_out, ctx->stage_out.p, out_bytes, cudaMemcpyDeviceToHost, ctx->stream));
-    CK(cudaStreamSynchronize(ctx->stream));
-    return BF_OK;
+    return check_overflow(ctx);          // synchronises; reports a device-side wait that gave up
 }
 
 extern "C" int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uint64_t* ct_out) {
