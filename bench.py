@@ -30,7 +30,10 @@ UNIT = "ms"
 # DRAM bytes (read + write) per launch of the named kernel from an ncu capture of this workload;
 # see profiles/ for the capture each figure comes from.  None = not captured yet.
 NCU_TRAFFIC_BYTES = {
-    "gpt2_qkv": {"mac": None, "ntt_fwd_strided": None},
+    # profiles/gpt2_qkv_kernels_ncu.md: dram__bytes_read.sum + dram__bytes_write.sum per launch
+    "gpt2_qkv": {"mac": 448.2e6,                       # 411.1 MB read + 37.1 MB written
+                 "key_inner_product": 379.8e6,         # mean of the baby (510.2 MB) and giant (249.4 MB) launches
+                 "ntt_fwd_strided": 4.8e6, "ntt_inv_contig": 47.9e6},
 }
 
 
@@ -255,7 +258,8 @@ def run_ours(args):
         key_bytes = n_rot * R.r * 2 * (R.r + 1) * R.N * 8 / max(1.0, ki_n)
         ach = key_bytes / (ki_ms * 1e-3) / 1e9
         rooflines["key_inner_product"] = {"bound": "hbm", "achieved": round(ach, 1), "peak": hbm_peak, "unit": "GB/s",
-                                          "frac": round(ach / hbm_peak, 4), "of": peak_kind, "traffic": None,
+                                          "frac": round(ach / hbm_peak, 4), "of": peak_kind,
+                                          "traffic": traffic.get("key_inner_product"),
                                           "launches_per_step": ki_n, "avg_ms": round(ki_ms, 5),
                                           "note": "bytes = one key per rotation; rotations sharing a key hit L2"}
     # transforms: bound by the arithmetic pipes (fp64 for the 40-bit primes, integer multiply-add for the rest)
@@ -490,7 +494,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="gpt2_qkv")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
