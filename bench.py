@@ -146,7 +146,10 @@ def time_extra_workload(name: str, steps: int, cache_budget_bytes=None) -> dict:
     st = bf.bf_get_kernel_stats(R.ctx)
     mac_n, mac_ms = st["mac"]
     enc_ms = (st["encode_fft_a"][1] + st["encode_fft_b"][1]) / steps
-    out = {"ms_per_token": round(ms, 3), "layers": len(R.layers), "fallback_layers": R.n_fallback_layers(),
+    h2d, d2h = R.host_bytes_per_step()
+    out = {"ms_per_token": round(ms, 4), "layers": len(R.layers),
+           "ciphertexts_in": sum(e["n_in"] for e in R.layers), "ciphertexts_out": sum(e["n_out"] for e in R.layers),
+           "boundary_bytes": h2d + d2h, "rotation_keys": len(R.rot_steps), "fallback_layers": R.n_fallback_layers(),
            "plan": {"D": R.plan.D, "tau": R.plan.tau, "b": R.plan.b, "g": R.plan.g},
            "encoded_weight_bytes_cached": R.cached_pt_bytes(), "encoded_weight_bytes_total": R.total_pt_bytes(),
            "mac_gbs": round(R.total_pt_bytes() * steps / (mac_ms * 1e-3) / 1e9, 1) if mac_ms else None,
@@ -505,6 +508,8 @@ def main():
     args = ap.parse_args()
     if args.extra == "all":
         args.extra = "gpt2_step,qwen3_step,llama3_layer"
+    elif args.extra == "tiles":     # tile-size study and the paper's own parameter set
+        args.extra = "gemm1024_D1024,gemm1024_D512,gemm1024_D256,gemm1024_D128,gpt2_qkv_paper_params"
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -96,6 +96,14 @@ WORKLOADS = {
                            cache_budget_bytes=60 * 10 ** 9),
     "llama3_layer": Workload("llama3_layer", "n16", PlanSpec(1024, 32, 8, 4), LLAMA3_8B_LAYER),
 }
+# Tile-size study (the paper's Sec. 5.3 experiment on a 1024 x 1024 product): smaller tiles need fewer or no
+# rotations but send more ciphertexts across the TEE boundary (1024/D in, 1024/D out).
+for _D, _tau, _b, _g in ((1024, 16, 16, 4), (512, 32, 4, 4), (256, 64, 2, 2), (128, 128, 1, 1)):
+    WORKLOADS[f"gemm1024_D{_D}"] = Workload(f"gemm1024_D{_D}", "n15", PlanSpec(_D, _tau, _b, _g),
+                                            (Layer("w", 1024, 1024),))
+# The GPT-2 QKV projection under the prototype's own CKKS parameters (Sec. 4.2): N = 8192, 4096 slots.
+WORKLOADS["gpt2_qkv_paper_params"] = Workload("gpt2_qkv_paper_params", "paper_n13", PlanSpec(1024, 4, 16, 16),
+                                              (GPT2_LAYER[0],))
 CONFIG_ORDER = ["tiny", "gpt2_qkv", "gpt2_step", "qwen3_step", "llama3_layer"]
 
 

@@ -55,6 +55,8 @@ class GpuSide:
         for s in steps:
             if s % self.par.n and s % self.par.n not in uniq:
                 uniq.append(s % self.par.n)
+        if not uniq:                     # a plan with a single diagonal per tile needs no rotation
+            return uniq
         arr = np.stack([keys[ckks.galois_element(s, self.par.N)] for s in uniq])
         self.bf.bf_load_eval_keys(self.ctx, uniq, len(uniq), self.to_dev(arr))
         return uniq

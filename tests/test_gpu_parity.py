@@ -190,6 +190,7 @@ def test_linear_tiny_config_bit_exact():
     ((64, 32, 2, 1), (64, 64)),       # fully dense packing, no giant step
     ((128, 1, 1, 128), (128, 128)),   # no baby step: every diagonal its own giant rotation
     ((32, 1, 32, 1), (40, 32)),       # all rotations hoisted from the input
+    ((32, 32, 1, 1), (70, 50)),       # one diagonal per tile: no rotation at all, 3 x 2 tiles
 ])
 def test_linear_small_ring_plans(plan_t, shape):
     par = oracle_params("n12")
