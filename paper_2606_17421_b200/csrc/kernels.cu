@@ -45,6 +45,20 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, 
                  "l"(src), "r"(bytes), "r"(smem_addr(bar))
                  : "memory");
 }
+// the same copy, with the lines marked "evict first" in L2: for streams that are read exactly once and must
+// not push reused operands (rotated inputs, digits, outputs) out of the cache
+__device__ __forceinline__ u64 l2_evict_first_policy() {
+    u64 pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s_stream(void* dst, const void* src, u32 bytes, u64* bar, u64 policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+            smem_addr(dst)),
+        "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
+        : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
     u32 ok;
     asm volatile(
@@ -126,6 +140,7 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
     if (tid >= MAC_CONSUMERS) {
         // ---------------- producer warp
         const u32 lane = tid - MAC_CONSUMERS;
+        const u64 stream_policy = l2_evict_first_policy();
         if (lane == 0) mbar_expect_tx(xbar, n_terms * 2 * TN * 8);
         __syncwarp();
         for (u32 e = lane; e < n_terms * 2; e += 32)                // X tile: [term][component] segments
@@ -143,9 +158,10 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
             if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * 8);
             __syncwarp();
             if (lanes == PL && cnt == (u32)MAC_TS) {
-                if (lane == 0) bulk_g2s(sdst, stage, MAC_STAGE_WORDS * 8, &full[slot]);
+                if (lane == 0) bulk_g2s_stream(sdst, stage, MAC_STAGE_WORDS * 8, &full[slot], stream_policy);
             } else if (lane < lanes) {
-                bulk_g2s(sdst + (size_t)lane * MAC_TS * TN, stage + (size_t)lane * MAC_TS * TN, cnt * TN * 8, &full[slot]);
+                bulk_g2s_stream(sdst + (size_t)lane * MAC_TS * TN, stage + (size_t)lane * MAC_TS * TN, cnt * TN * 8,
+                                &full[slot], stream_policy);
             }
             if (++ch == n_chunks) { ch = 0; ++g; }
             if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
