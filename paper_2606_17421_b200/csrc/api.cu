@@ -422,8 +422,13 @@ extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_
     u32* perm_dev = nullptr;
     e = cudaMalloc(&perm_dev, perms.size() * sizeof(u32));
     if (e != cudaSuccess) { cudaGetLastError(); return BF_ERR_OOM; }
-    CK(cudaMemcpy(perm_dev, perms.data(), perms.size() * sizeof(u32), cudaMemcpyHostToDevice));
-    CK(cudaMemcpy(ctx->perms, pinvs.data(), pinvs.size() * sizeof(u32), cudaMemcpyHostToDevice));
+    if (cudaMemcpy(perm_dev, perms.data(), perms.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(ctx->perms, pinvs.data(), pinvs.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess) {
+        ctx->cuda_msg = "cudaMemcpy of the permutation tables failed";
+        cudaGetLastError();
+        cudaFree(perm_dev);
+        return BF_ERR_CUDA;
+    }
     PolyBatch B;
     memset(&B, 0, sizeof(B));
     B.src = keys;
@@ -433,9 +438,9 @@ extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_
     B.n_m = nb;
     B.mod0 = 0;
     B.mod_step = 1;
-    // The in-place first pass would race with the permuted store of the second pass, so transform
-    // the caller's array out of place: first pass into our buffer, permuted store into it too is not
-    // possible either.  Use a staging buffer for the natural-order transform.
+    // The first pass of the transform lands in a staging buffer in natural order; the second pass
+    // reads it and stores, permuted, into the resident key array (a permuted store in place would
+    // overwrite points other blocks have not read yet).
     u64* stage = nullptr;
     e = cudaMalloc(&stage, key_words * n_keys * sizeof(u64));
     if (e != cudaSuccess) { cudaGetLastError(); cudaFree(perm_dev); return BF_ERR_OOM; }
