@@ -267,7 +267,7 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
             pw[k] = h_mulmod(pw[k - 1], psi, q);
             pwi[k] = h_mulmod(pwi[k - 1], psi_inv, q);
         }
-        R.fp_ok[m] = q < (1ull << 41) ? 1u : 0u;
+        R.fp_ok[m] = q < (1ull << 50) ? 1u : 0u;      // below 2^41: lazy fp64 path; up to 2^50: fp64 path in [0, 4q)
         R.qd[m] = (double)q;
         R.qinv_d[m] = 1.0 / (double)q;
         R.ninv_d[m] = (double)R.ninv[m];

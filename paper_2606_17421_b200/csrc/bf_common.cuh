@@ -29,7 +29,7 @@ struct RingDev {
     u64 qneg[MAX_MODULI];        // -q^{-1} mod 2^64 (Montgomery reduction)
     u64 ninv_m[MAX_MODULI];      // N^{-1} * 2^{-64} mod q: inverse transform that also leaves Montgomery form
     u64 ninv_ms[MAX_MODULI];
-    u32 fp_ok[MAX_MODULI];       // modulus below 2^41: its transforms run in fp64 (every value an exact integer below
+    u32 fp_ok[MAX_MODULI];       // modulus below 2^50: its transforms run in fp64 (every value an exact integer below
                                  //   2^53) and its twiddle tables hold the bits of ((double)w, (double)w / q)
     double qd[MAX_MODULI];       // (double)q
     double qinv_d[MAX_MODULI];   // 1.0 / q
@@ -55,10 +55,11 @@ __device__ __forceinline__ double u2d(u64 x) {          // exact for x < 2^52
 __device__ __forceinline__ u64 d2u(double d) {          // d an integer in [0, 2^52)
     return (u64)__double_as_longlong(d + 4503599627370496.0) - 0x4330000000000000ull;
 }
-// x * w - round(x * w / q) * q for integer-valued x (|x| < 2^46) and a constant 0 <= w < q given as
-// (double)w and wq = (double)w / q.  The result is an exact integer in (-0.51 q, 0.51 q) congruent to
-// x*w:  ph + pl = x*w exactly (FMA), the quotient estimate is off by less than 2^-6, ph - qh*q is an
-// integer below 2^42 in magnitude and therefore exact, and so is the final sum.
+// x * w - round(x * w / q) * q for a non-negative integer-valued x and a constant 0 <= w < q given as
+// (double)w and wq = (double)w / q.  ph + pl = x*w exactly (FMA); the quotient estimate is within
+// 1/2 + x * 2^-52 of x*w/q; ph - qh*q is an integer far below 2^53 and therefore exact, and so is the final
+// sum.  For q < 2^41 and x < 2^46 the result lies in (-0.51q, 0.51q); for q < 2^50 and x <= 4q < 2^52 in
+// (-0.75q, 0.75q).  Always congruent to x*w.
 __device__ __forceinline__ double fp_mul_centred(double x, double w, double wq, double q) {
     const double magic = 4503599627370496.0;             // 2^52
     const double ph = __dmul_rn(x, w);

@@ -102,9 +102,12 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
 // (-0.51q, 0.51q): values stay non-negative and grow by at most 1.51q per stage, so after all
 // log2 N <= 16 stages they are below 26q < 2^46 and need one reduction at the very end.
 // Inverse: (a, b) -> (a + b reduced below 2q, (a - b + 2q)*w + q in (0.49q, 1.51q)): values in [0, 2q).
-template <int K, bool FWD>
-__device__ __forceinline__ void set_butterflies(double (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base,
-                                                u32 blk, u64, double q) {
+// WIDE (primes from 2^41 up to 2^50): the centred product lies in (-0.75q, 0.75q) and values must stay below
+// 4q < 2^52, so the forward butterfly keeps Harvey's invariant [0, 4q) with one conditional subtraction:
+// (X, Y) -> (X~ + T, X~ - T + 2q), X~ = X reduced below 2q, T = Y*w + q in (0.25q, 1.75q).
+template <int K, bool FWD, bool WIDE>
+__device__ __forceinline__ void set_butterflies_fp(double (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base,
+                                                   u32 blk, double q) {
     const double q2 = __dadd_rn(q, q);
 #pragma unroll
     for (int s = 0; s < K; ++s) {
@@ -117,7 +120,13 @@ __device__ __forceinline__ void set_butterflies(double (&e)[8], const ulonglong2
 #pragma unroll
             for (int off = 0; off < d; ++off) {
                 const int i = sub * 2 * d + off;
-                if (FWD) {
+                if (FWD && WIDE) {
+                    double x = e[i];
+                    if (x >= q2) x = __dsub_rn(x, q2);
+                    const double t = __dadd_rn(fp_mul_centred(e[i + d], w, wq, q), q);
+                    e[i] = __dadd_rn(x, t);
+                    e[i + d] = __dadd_rn(__dsub_rn(x, t), q2);
+                } else if (FWD) {
                     const double sv = fp_mul_centred(e[i + d], w, wq, q);
                     const double xq = __dadd_rn(e[i], q);
                     e[i] = __dadd_rn(xq, sv);
@@ -132,6 +141,13 @@ __device__ __forceinline__ void set_butterflies(double (&e)[8], const ulonglong2
             }
         }
     }
+}
+
+template <int K, bool FWD>
+__device__ __forceinline__ void set_butterflies(double (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base,
+                                                u32 blk, u64 q_int, double q) {
+    if (q_int >> 41) set_butterflies_fp<K, FWD, true>(e, tw, tw_base, blk, q);    // block-uniform
+    else set_butterflies_fp<K, FWD, false>(e, tw, tw_base, blk, q);
 }
 
 template <bool FP> struct Elem { typedef u64 T; };
@@ -234,6 +250,7 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
                         double v = __dadd_rn(fp_mul_centred(*(double*)&e[i], mont ? R.ninvm_d[mod] : R.ninv_d[mod],
                                                             mont ? R.ninvm_q[mod] : R.ninv_q[mod], qd), qd);
                         if (v >= qd) v = __dsub_rn(v, qd);
+                        if (v >= qd) v = __dsub_rn(v, qd);      // (the product can touch 2q for the 50-bit prime)
                         dst[gidx] = d2u(v);
                     } else {
                         const bool mont = B.from_mont != 0;
