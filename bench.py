@@ -30,7 +30,7 @@ UNIT = "ms"
 # DRAM bytes (read + write) per launch of the named kernel from an ncu capture of this workload;
 # see profiles/ for the capture each figure comes from.  None = not captured yet.
 NCU_TRAFFIC_BYTES = {
-    # profiles/gpt2_qkv_kernels_ncu.md: dram__bytes_read.sum + dram__bytes_write.sum per launch
+    # from the ncu capture summarised under profiles/: dram__bytes_read.sum + dram__bytes_write.sum per launch
     "gpt2_qkv": {"mac": 448.2e6,                       # 411.1 MB read + 37.1 MB written
                  "key_inner_product": 379.8e6,         # mean of the baby (510.2 MB) and giant (249.4 MB) launches
                  "ntt_fwd_strided": 4.8e6, "ntt_inv_contig": 47.9e6},

@@ -295,8 +295,8 @@ struct KaraAcc {
 __device__ __forceinline__ u64 redc_2x32(u64 H, u64 L, u64 q, u32 qneg32) {
     u32 l0 = (u32)L, l1 = (u32)(L >> 32), h0 = (u32)H, h1 = (u32)(H >> 32);
     const u32 q0 = (u32)q, q1 = (u32)(q >> 32);
-    // round 1: m = l0 * qneg32; (h1 h0 l1 l0) += m * (q1 q0); l0 becomes 0 and is dropped
-    // round 2: the same one limb up; the result is (h1 h0)
+    // first pass: m = l0 * qneg32; (h1 h0 l1 l0) += m * (q1 q0); l0 becomes 0 and is dropped
+    // second pass: the same one limb up; the result is (h1 h0)
     asm("{\n\t.reg .u32 m;\n\t"
         "mul.lo.u32 m, %0, %6;\n\t"
         "mad.lo.cc.u32 %0, m, %4, %0;\n\t"
