@@ -191,6 +191,9 @@ def test_linear_tiny_config_bit_exact():
     ((128, 1, 1, 128), (128, 128)),   # no baby step: every diagonal its own giant rotation
     ((32, 1, 32, 1), (40, 32)),       # all rotations hoisted from the input
     ((32, 32, 1, 1), (70, 50)),       # one diagonal per tile: no rotation at all, 3 x 2 tiles
+    ((64, 4, 16, 1), (150, 64)),      # 16 terms per output group, odd number of groups: half-filled last stage
+    ((64, 4, 4, 4), (64, 1472)),      # 23 input chunks: their 69 baby rotations span two key-switch batches
+    ((64, 4, 4, 4), (1920, 64)),      # 30 output blocks: their 90 giant rotations span two key-switch batches
 ])
 def test_linear_small_ring_plans(plan_t, shape):
     par = oracle_params("n12")
