@@ -114,6 +114,14 @@ int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weight
  * it off and drops the stored graphs (default: on). */
 int bf_set_graph_replay(bf_ctx* ctx, int on);
 
+/* The kernels of a call are launched with programmatic stream serialisation: each may be scheduled
+ * while the previous kernel of the stream drains, and waits for that kernel's completion before it
+ * touches memory the call writes (the multiply-accumulate and the key-switch inner product fetch
+ * their first cached weights and keys before that wait).  Results are unchanged.
+ * bf_set_dependent_launch(ctx, 0) falls back to plain stream order (default: on) and drops the
+ * stored graphs.  The paper has no counterpart; this is a launch-latency measure. */
+int bf_set_dependent_launch(bf_ctx* ctx, int on);
+
 /* Rescale (Sec. 2.1): drop the last prime of n_ct ciphertexts that have `level` primes each,
  *     c'_i = (c_i - centred(c_{level-1})) * q_{level-1}^{-1} mod q_i ,
  * i.e. round(c / q_{level-1}).  ct_in: device [n_ct][2][level][N]; ct_out: device

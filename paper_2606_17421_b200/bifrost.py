@@ -54,6 +54,7 @@ _SIGNATURES = {
     "bf_linear": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
     "bf_device_status": (ctypes.c_int, [_vp]),
     "bf_set_graph_replay": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "bf_set_dependent_launch": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_rescale": (ctypes.c_int, [_vp, _vp, _vp, _u32, _u32, ctypes.POINTER(ctypes.c_double)]),
     "bf_linear_host": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
     "bf_rotate": (ctypes.c_int, [_vp, _vp, _u32, _vp]),
@@ -169,6 +170,10 @@ def bf_device_status(ctx):
 
 def bf_set_graph_replay(ctx, on: bool):
     _check(load().bf_set_graph_replay(ctx, 1 if on else 0), "bf_set_graph_replay", ctx)
+
+
+def bf_set_dependent_launch(ctx, on: bool):
+    _check(load().bf_set_dependent_launch(ctx, 1 if on else 0), "bf_set_dependent_launch", ctx)
 
 
 def bf_rescale(ctx, ct_in, ct_out, n_ct: int, level: int, scale: float | None = None):

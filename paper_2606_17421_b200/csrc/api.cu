@@ -274,6 +274,9 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
         R.ninv_q[m] = (double)R.ninv[m] / (double)q;
         R.ninvm_d[m] = (double)R.ninv_m[m];
         R.ninvm_q[m] = (double)R.ninv_m[m] / (double)q;
+        R.c30_d[m] = (double)((1ull << 30) % q);
+        R.c30_q[m] = R.c30_d[m] / (double)q;
+        R.k59_d[m] = (double)(2 * q - (1ull << 59) % q);
         auto dbits = [](double d) -> u64 {
             u64 bits;
             memcpy(&bits, &d, sizeof(bits));
@@ -612,6 +615,7 @@ static int moddown_batch(bf_ctx* ctx, const RotBatch& rb, const u64* c0_base, lo
     B.n_m = 1;
     B.mod0 = r;
     B.mod_step = 0;
+    B.store_centred = 1;                                // the form the lift below reads
     CK(ntt_inverse(ctx->ring, B, (u32)rb.n * 2, ctx->stream));
     memset(&B, 0, sizeof(B));
     B.src = ctx->Tc.p;
@@ -672,6 +676,7 @@ static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_s
     B.dst_so = (long long)nb * N;
     B.dst_sm = N;
     B.skip_diag = 1;
+    B.src_digits = 1;
     B.diag_src = c1_ntt;
     B.diag_so = c1_ntt_stride;
     CK(ntt_forward(ctx->ring, B, n_sets * r, LOAD_REDUCE, ctx->stream));
@@ -774,7 +779,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     // ---- multiply-accumulate over the encoded diagonals
     const u32 n_terms = n_in * b, n_pj = n_out * g;
     if (pt_weights) {
-        CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, A, n_pj, n_terms, ctx->device_error, ctx->stream));
+        CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, A, n_pj, n_terms, true, ctx->device_error, ctx->stream));
     } else {
         // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them
         const size_t group_bytes = (size_t)n_terms * r * N * 8;
@@ -787,7 +792,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
             const TileLayout cl = mac_tile_layout(ctx->ring, cnt, n_terms);
             TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p, cl, pj0));
-            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, cl, X, A + (size_t)pj0 * ctw, cnt, n_terms,
+            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, cl, X, A + (size_t)pj0 * ctw, cnt, n_terms, false,
                           ctx->device_error, ctx->stream));
         }
     }
@@ -896,7 +901,11 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         ge.unusable = true;
         return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
     }
+    // measured: inside a replayed graph plain edges are as fast as programmatic ones, so capture those
+    const bool dependent = ctx->ring.dependent_launch;
+    ctx->ring.dependent_launch = false;
     const int rc = linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
+    ctx->ring.dependent_launch = dependent;
     cudaGraph_t graph = nullptr;
     const cudaError_t ec = cudaStreamEndCapture(ctx->stream, &graph);
     if (rc != BF_OK || ec != cudaSuccess || !graph) {
@@ -927,6 +936,13 @@ extern "C" int bf_set_graph_replay(bf_ctx* ctx, int on) {
     if (!ctx) return BF_ERR_INVALID_ARG;
     ctx->use_graphs = on ? 1 : 0;
     if (!on) destroy_graphs(ctx);
+    return BF_OK;
+}
+
+extern "C" int bf_set_dependent_launch(bf_ctx* ctx, int on) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    ctx->ring.dependent_launch = on != 0;
+    destroy_graphs(ctx);            // stored graphs carry the edges of the old setting
     return BF_OK;
 }
 

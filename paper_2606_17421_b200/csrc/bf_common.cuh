@@ -35,6 +35,8 @@ struct RingDev {
     double qinv_d[MAX_MODULI];   // 1.0 / q
     double ninv_d[MAX_MODULI], ninv_q[MAX_MODULI];     // (double)N^{-1} and N^{-1} / q
     double ninvm_d[MAX_MODULI], ninvm_q[MAX_MODULI];   // the same for N^{-1} * 2^{-64} (leaving Montgomery form)
+    double c30_d[MAX_MODULI], c30_q[MAX_MODULI];       // (double)(2^30 mod q) and that over q
+    double k59_d[MAX_MODULI];    // 2q - (2^59 mod q): undoes the offset of a stored centred lift, keeps it positive
     const ulonglong2* tw_fwd;    // [r+1][N]  (psi^brev(k), companion), merged Cooley-Tukey order
     const ulonglong2* tw_inv;    // [r+1][N]  inverses of the above, for the Gentleman-Sande inverse
 };
@@ -49,6 +51,14 @@ __device__ __forceinline__ u64 mul_shoup_lazy(u64 x, u64 w, u64 ws, u64 q) {
 // ---- fp64 arithmetic for primes q < 2^41.  B200 issues fp64 FMAs at the rate of 32-bit integer
 // multiply-adds, on a pipe of its own, while a 64x64-bit high product costs about ten integer
 // multiply-add slots; and integers below 2^53 are exact in fp64.
+// First statement of every kernel of a linear-layer call.  Lets the next kernel of the stream be scheduled
+// as soon as all blocks of this one have started, then waits until the previous kernel has completed and
+// flushed its writes.  A no-op when the launch carries no programmatic dependency.
+__device__ __forceinline__ void grid_dependency_enter() {
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ double u2d(u64 x) {          // exact for x < 2^52
     return __longlong_as_double((long long)(x | 0x4330000000000000ull)) - 4503599627370496.0;
 }
@@ -183,7 +193,7 @@ enum LoadMode : int {
     LOAD_PLAIN = 0,     // residues already modulo the target prime, in [0, q)
     LOAD_REDUCE = 1,    // any 64-bit non-negative integer (e.g. a residue of another prime): x mod q
     LOAD_I64 = 2,       // signed 64-bit integer coefficient: x mod q in [0, q)
-    LOAD_CENTRED = 3,   // residue t in [0, M) of modulus M: centred lift to (-M/2, M/2], then mod q
+    LOAD_CENTRED = 3,   // centred lift t' in (-M/2, M/2] of a residue of modulus M, stored as t' + 2^59: t' mod q
     LOAD_I64_MONT = 4,  // LOAD_I64, then times 2^64 mod q: the transform's output is in Montgomery form
 };
 
@@ -247,6 +257,9 @@ struct PolyBatch {
     long long sum_stride;
     u32 sum_terms;
     u64 lift_mod;                 // LOAD_CENTRED: the modulus M the source residues live in
+    u32 src_digits;               // LOAD_REDUCE: the source of outer index o is a residue modulo prime o % r
+    u32 store_centred;            // inverse transform: store the centred lift of each coefficient plus 2^59
+                                  //   (the form LOAD_CENTRED reads) instead of the residue in [0, q)
     u32 from_mont;                // inverse transform only: input is in Montgomery form, output is not
     u64* tile_ptr;                // non-null: the NTT-domain side lives there in the tile-major layout `tile`
     TileLayout tile;              //   (forward writes its final result there, inverse reads its input there);

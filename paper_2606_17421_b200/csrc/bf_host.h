@@ -43,7 +43,27 @@ struct RingHost {
     NttGeometry geom;
     std::vector<u64> q;               // q_0..q_L, then P
     Profiler* prof = nullptr;
+    bool dependent_launch = true;     // launch the kernels of a call with programmatic stream serialisation
 };
+
+// Launch with programmatic stream serialisation: the grid may be scheduled while the previous kernel
+// of the stream drains; every kernel launched this way calls grid_dependency_enter() before it touches
+// global memory, which waits until that previous kernel has completed and its writes are visible.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_dependent(const RingHost& ring, void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                                           size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = ring.dependent_launch ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 // ---- ntt.cu
 NttGeometry ntt_geometry(u32 logN);
@@ -66,7 +86,7 @@ u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintex
 TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms);   // layout of n_pj groups of n_terms diagonals
 size_t mac_tile_words(const RingHost& ring, const TileLayout& t);           // words that layout occupies
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
-                       u32 n_terms, int* error_flag, cudaStream_t stream);
+                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream);
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
                            const u64* invs, const u64* qlmod, cudaStream_t stream);
 

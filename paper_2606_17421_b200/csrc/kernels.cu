@@ -110,8 +110,10 @@ constexpr u32 KARA_L = 25;
 template <bool KARA, int LOG_TN>
 __global__ void __launch_bounds__(MAC_THREADS, 3)
 mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, const u64* __restrict__ x,
-           u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, int* __restrict__ error_flag) {
+           u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, u32 early_weights,
+           int* __restrict__ error_flag) {
     extern __shared__ __align__(128) unsigned char mac_smem[];
+    asm volatile("griddepcontrol.launch_dependents;");
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     u64* ring = (u64*)mac_smem;                                    // [MAC_STAGES][PL][MAC_TS][TN]
     u64* xs = ring + MAC_STAGES * MAC_STAGE_WORDS;                 // [n_terms][2][TN]
@@ -141,18 +143,13 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         // ---------------- producer warp
         const u32 lane = tid - MAC_CONSUMERS;
         const u64 stream_policy = l2_evict_first_policy();
-        if (lane == 0) mbar_expect_tx(xbar, n_terms * 2 * TN * 8);
-        __syncwarp();
-        for (u32 e = lane; e < n_terms * 2; e += 32)                // X tile: [term][component] segments
-            bulk_g2s(xs + (size_t)e * TN, x + ((size_t)e * r + i) * N + n0, TN * 8, xbar);
-        u32 g = 0, ch = 0, slot = 0, phase = 0;
-        for (u32 k = 0; k < n_items; ++k) {
-            if (k >= (u32)MAC_STAGES) mbar_wait(&empty[slot], phase ^ 1, error_flag);   // consumers left this slot
+        u32 g = 0, ch = 0, slot = 0, phase = 0, k = 0;
+        // one stage of the weight stream: a contiguous 16 KB block of the tile-major layout; when its tail
+        // is padding (last group round or last term chunk) copy the valid part of every lane only
+        auto issue_stage = [&]() {
             const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
             const u32 first = pj_begin + g * PL;
             const u32 lanes = min((u32)PL, pj_end - first);
-            // the stage is one contiguous 16 KB block of the tile-major layout; when its tail is
-            // padding (last group round or last term chunk) copy the valid part of every lane only
             const u64* stage = pt + tile_stage_offset(lay, i, blockIdx.x, first / PL, ch);
             u64* sdst = ring + (size_t)slot * MAC_STAGE_WORDS;
             if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * 8);
@@ -165,6 +162,19 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
             }
             if (++ch == n_chunks) { ch = 0; ++g; }
             if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
+            ++k;
+        };
+        // cached weights do not depend on the previous kernel: fill the ring before waiting for it
+        const u32 early = early_weights ? min(n_items, (u32)MAC_STAGES) : 0u;
+        while (k < early) issue_stage();
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (lane == 0) mbar_expect_tx(xbar, n_terms * 2 * TN * 8);
+        __syncwarp();
+        for (u32 e = lane; e < n_terms * 2; e += 32)                // X tile: [term][component] segments
+            bulk_g2s(xs + (size_t)e * TN, x + ((size_t)e * r + i) * N + n0, TN * 8, xbar);
+        while (k < n_items) {
+            if (k >= (u32)MAC_STAGES) mbar_wait(&empty[slot], phase ^ 1, error_flag);   // consumers left this slot
+            issue_stage();
         }
         return;
     }
@@ -173,6 +183,7 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
     const u32 c = tid & (TN - 1), l = tid >> LOG_TN;
     const u64 q = R.q[i];
     const u32 qneg32 = (u32)R.qneg[i];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     mbar_wait(xbar, 0, error_flag);
     if (KARA) {
         // split the resident X words into limbs, each exactly once, then let every consumer see them
@@ -285,7 +296,8 @@ u32 mac_split_bits(const RingHost& ring) {
 
 template <bool KARA, int LOG_TN>
 static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a,
-                                u32 n_pj, u32 n_terms, u32 lazy, int* error_flag, cudaStream_t stream) {
+                                u32 n_pj, u32 n_terms, u32 lazy, u32 early_weights, int* error_flag,
+                                cudaStream_t stream) {
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     const size_t smem = (size_t)MAC_STAGES * MAC_STAGE_WORDS * 8 + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_STAGES + 1) * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
@@ -306,13 +318,12 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     pj_per_block = (pj_per_block + PL - 1) / PL * PL;
     slices = (n_pj + pj_per_block - 1) / pj_per_block;
     dim3 grid(ring.dev.N >> LOG_TN, ring.dev.r, slices);
-    mac_kernel<KARA, LOG_TN><<<grid, MAC_THREADS, smem, stream>>>(ring.dev, pt, lay, x, a, n_terms, n_pj, pj_per_block,
-                                                                   lazy, error_flag);
-    return cudaGetLastError();
+    return launch_dependent(ring, mac_kernel<KARA, LOG_TN>, grid, dim3(MAC_THREADS), smem, stream, ring.dev, pt, lay, x, a,
+                            n_terms, n_pj, pj_per_block, lazy, early_weights, error_flag);
 }
 
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
-                       u32 n_terms, int* error_flag, cudaStream_t stream) {
+                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream) {
     if (n_pj == 0) return cudaSuccess;
     if (lay.n_pj != n_pj || lay.n_terms != n_terms) return cudaErrorInvalidValue;
     ProfScope prof(ring.prof, CAT_MAC, stream);
@@ -330,7 +341,8 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
     } else if (lazy < (u32)MAC_TS) {
         return cudaErrorInvalidValue;
     }
-#define BF_MAC(S, L) launch_mac_t<S, L>(ring, pt, lay, x, a, n_pj, n_terms, lazy, error_flag, stream)
+    const u32 early = weights_static ? 1u : 0u;
+#define BF_MAC(S, L) launch_mac_t<S, L>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, error_flag, stream)
     if (kara) {
         switch (log_tn) {
             case 8: return BF_MAC(true, 8);
@@ -379,6 +391,7 @@ __global__ void __launch_bounds__(KI_TILE, 4) key_inner_bulk_kernel(const RingDe
     u64* sk = sd + (size_t)r * KI_TILE;             // [r][2][KI_TILE] key components
     u64* bar = sk + (size_t)2 * r * KI_TILE;
     const u32 tid = threadIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;");
     if (tid == 0) {
         mbar_init(bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -389,12 +402,14 @@ __global__ void __launch_bounds__(KI_TILE, 4) key_inner_bulk_kernel(const RingDe
         __syncwarp();
         const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + n0;
         const u64* kp = keys + ((size_t)rb.key[rot] * r * 2 * nb + m) * N + n0;
-        for (u32 e = tid; e < 3 * r; e += 32) {
-            const u32 j = e / 3, which = e % 3;
-            if (which == 0) bulk_g2s(sd + (size_t)j * KI_TILE, dp + (size_t)j * nb * N, KI_TILE * 8, bar);
-            else bulk_g2s(sk + ((size_t)j * 2 + (which - 1)) * KI_TILE, kp + (size_t)(j * 2 + (which - 1)) * nb * N,
-                          KI_TILE * 8, bar);
-        }
+        // the keys do not depend on the previous kernel: fetch them before waiting for it, the digits after
+        for (u32 e = tid; e < 2 * r; e += 32)
+            bulk_g2s(sk + (size_t)e * KI_TILE, kp + (size_t)e * nb * N, KI_TILE * 8, bar);
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        for (u32 j = tid; j < r; j += 32)
+            bulk_g2s(sd + (size_t)j * KI_TILE, dp + (size_t)j * nb * N, KI_TILE * 8, bar);
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
     }
     mbar_wait(bar, 0, error_flag);
     const u64 q = R.q[m], mu = R.mu[m], c64 = R.c64[m], c64s = R.c64s[m];
@@ -437,8 +452,8 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
         attr_set = true;
     }
     dim3 grid(rb.n, ring.dev.N / KI_TILE, r + 1);
-    key_inner_bulk_kernel<<<grid, KI_TILE, smem, stream>>>(ring.dev, rb, dig, keys, u, small_ok, error_flag);
-    return cudaGetLastError();
+    return launch_dependent(ring, key_inner_bulk_kernel, grid, dim3(KI_TILE), smem, stream, ring.dev, rb, dig, keys, u,
+                            small_ok, error_flag);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -456,6 +471,7 @@ struct RescaleConsts {
 // (n_seq > 1): the packed output of ciphertext t never reaches the input of ciphertext t+1.
 __global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const RescaleConsts rc, const u64* in, u64* out,
                                                       u32 level, u32 n_seq) {
+    grid_dependency_enter();
     const u32 N = R.N;
     const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
     const u64 qL = R.q[level - 1];
@@ -489,10 +505,10 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
     ProfScope prof(ring.prof, CAT_RESCALE, stream);
     if (in == out && n_ct > 1) {
         dim3 grid(ring.dev.N / 64, 1);
-        rescale_kernel<<<grid, 64, 0, stream>>>(ring.dev, rc, in, out, level, n_ct);
+        launch_dependent(ring, rescale_kernel, grid, dim3(64), 0, stream, ring.dev, rc, in, out, level, n_ct);
     } else {
         dim3 grid(ring.dev.N / 256, n_ct);
-        rescale_kernel<<<grid, 256, 0, stream>>>(ring.dev, rc, in, out, level, 1);
+        launch_dependent(ring, rescale_kernel, grid, dim3(256), 0, stream, ring.dev, rc, in, out, level, 1u);
     }
     return cudaGetLastError();
 }

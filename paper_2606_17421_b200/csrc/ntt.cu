@@ -42,23 +42,60 @@ ProfScope::~ProfScope() {
     p->recs.push_back({cat, a, b});
 }
 
+struct LoadConsts {
+    u64 q, mu, lift_mod, lift_red;
+    double qd, qinv, c30, c30q, k59;
+    bool src_small;     // LOAD_REDUCE: every source word is below 1.5 q already (block-uniform)
+    bool src_fp;        // LOAD_REDUCE: every source word is below 2^51
+};
+
 template <int LOAD>
-__device__ __forceinline__ u64 load_src(const void* src, size_t idx, u64 q, u64 mu, u64 lift_mod, u64 lift_red) {
+__device__ __forceinline__ u64 load_src(const void* src, size_t idx, const LoadConsts& c) {
     if (LOAD == LOAD_PLAIN) return ((const u64*)src)[idx];
-    if (LOAD == LOAD_REDUCE) return barrett64(((const u64*)src)[idx], q, mu);
+    if (LOAD == LOAD_REDUCE) {
+        const u64 t = ((const u64*)src)[idx];
+        return c.src_small ? (t >= c.q ? t - c.q : t) : barrett64(t, c.q, c.mu);
+    }
     if (LOAD == LOAD_I64 || LOAD == LOAD_I64_MONT) {
         i64 v = ((const i64*)src)[idx];
         u64 a = v < 0 ? (u64)(-v) : (u64)v;
-        u64 m = barrett64(a, q, mu);
-        m = (v < 0 && m != 0) ? q - m : m;
-        if (LOAD == LOAD_I64_MONT) m = mul_shoup(m, lift_mod, lift_red, q);   // (2^64 mod q, its Shoup companion)
+        u64 m = barrett64(a, c.q, c.mu);
+        m = (v < 0 && m != 0) ? c.q - m : m;
+        if (LOAD == LOAD_I64_MONT) m = mul_shoup(m, c.lift_mod, c.lift_red, c.q);   // (2^64 mod q, its Shoup companion)
         return m;
     }
-    // LOAD_CENTRED
-    u64 t = ((const u64*)src)[idx];
-    u64 m = barrett64(t, q, mu);
-    if (t > (lift_mod - 1) / 2) m = sub_mod(m, lift_red, q);
+    // LOAD_CENTRED: the word is t' + 2^59 with t' the centred lift of a residue modulo lift_mod
+    const u64 T = ((const u64*)src)[idx];
+    const bool neg = T < (1ull << 59);
+    const u64 t = neg ? T + c.lift_mod - (1ull << 59) : T - (1ull << 59);      // back to [0, lift_mod)
+    u64 m = barrett64(t, c.q, c.mu);
+    if (neg) m = sub_mod(m, c.lift_red, c.q);
     return m;
+}
+
+// The same loads for a modulus on the fp64 path: the result is a non-negative integer-valued double
+// congruent to the source, below 3.6 q (lazy: the butterflies reduce).
+template <int LOAD>
+__device__ __forceinline__ double load_src_fp(const void* src, size_t idx, const LoadConsts& c) {
+    if (LOAD == LOAD_REDUCE) {
+        const u64 t = ((const u64*)src)[idx];
+        if (c.src_small) return u2d(t);
+        if (c.src_fp) {                                  // t - round(t / q) q + q  in [0.5 q, 1.5 q]
+            const double magic = 4503599627370496.0;
+            const double v = u2d(t);
+            const double qh = __dsub_rn(__fma_rn(v, c.qinv, magic), magic);
+            return __dadd_rn(__fma_rn(-qh, c.qd, v), c.qd);
+        }
+        return u2d(barrett64(t, c.q, c.mu));
+    }
+    if (LOAD == LOAD_CENTRED) {
+        // t' + 2^59 = hi 2^30 + lo, so t' = hi (2^30 mod q) + lo - (2^59 mod q)  (mod q); with the product
+        // centred in (-0.75 q, 0.75 q), lo < 2^30 and k59 = 2q - (2^59 mod q) the sum is positive
+        const u64 T = ((const u64*)src)[idx];
+        const double hi = u2d(T >> 30), lo = u2d(T & ((1ull << 30) - 1));
+        return __dadd_rn(__dadd_rn(fp_mul_centred(hi, c.c30, c.c30q, c.qd), lo), c.k59);
+    }
+    return u2d(load_src<LOAD>(src, idx, c));
 }
 
 // Butterflies of one register-resident set of 2^K points over K consecutive stages.
@@ -202,9 +239,21 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
     const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
                                    : (size_t)o * B.src_so;
     const char* src = (const char*)B.src + (src_off + (size_t)m * B.src_sm) * 8;
-    const u64 lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu)
-                       : (LOAD == LOAD_I64_MONT) ? R.c64s[mod] : 0;
-    const u64 lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
+    LoadConsts lc;
+    lc.q = q;
+    lc.mu = mu;
+    lc.lift_red = (LOAD == LOAD_CENTRED) ? barrett64(B.lift_mod, q, mu) : (LOAD == LOAD_I64_MONT) ? R.c64s[mod] : 0;
+    lc.lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
+    lc.qd = qd;
+    lc.qinv = R.qinv_d[mod];
+    lc.c30 = R.c30_d[mod];
+    lc.c30q = R.c30_q[mod];
+    lc.k59 = R.k59_d[mod];
+    {
+        const u64 qs = (LOAD == LOAD_REDUCE && B.src_digits) ? R.q[o % R.r] : ~(u64)0;
+        lc.src_small = qs <= q + (q >> 1);
+        lc.src_fp = qs < (1ull << 51);
+    }
     const int col0 = blockIdx.x * LANES;
     const int tid = threadIdx.x;
 #pragma unroll
@@ -229,8 +278,12 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
                 const int row = base + i * step;
                 if (g_first) {
                     const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
-                    if (FWD) from_u64(e[i], load_src<LOAD>(src, gidx, q, mu, lift_mod, lift_red));
-                    else e[i] = ((const T*)dst)[gidx];
+                    if (FWD) {
+                        if constexpr (FP) e[i] = load_src_fp<LOAD>(src, gidx, lc);
+                        else e[i] = load_src<LOAD>(src, gidx, lc);
+                    } else {
+                        e[i] = ((const T*)dst)[gidx];
+                    }
                 } else {
                     e[i] = sm[row * LANES + lane];
                 }
@@ -245,17 +298,20 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
                     const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
                     if (FWD) {
                         ((T*)dst)[gidx] = e[i];                 // lazy; the contiguous pass finishes
-                    } else if (FP) {                            // scale by N^{-1}, to [0, q)
+                    } else {                                    // scale by N^{-1}, to [0, q)
                         const bool mont = B.from_mont != 0;
-                        double v = __dadd_rn(fp_mul_centred(*(double*)&e[i], mont ? R.ninvm_d[mod] : R.ninv_d[mod],
-                                                            mont ? R.ninvm_q[mod] : R.ninv_q[mod], qd), qd);
-                        if (v >= qd) v = __dsub_rn(v, qd);
-                        if (v >= qd) v = __dsub_rn(v, qd);      // (the product can touch 2q for the 50-bit prime)
-                        dst[gidx] = d2u(v);
-                    } else {
-                        const bool mont = B.from_mont != 0;
-                        dst[gidx] = mul_shoup(*(u64*)&e[i], mont ? R.ninv_m[mod] : R.ninv[mod],
-                                              mont ? R.ninv_ms[mod] : R.ninvs[mod], q);
+                        u64 out;
+                        if constexpr (FP) {
+                            double v = __dadd_rn(fp_mul_centred(e[i], mont ? R.ninvm_d[mod] : R.ninv_d[mod],
+                                                                mont ? R.ninvm_q[mod] : R.ninv_q[mod], qd), qd);
+                            if (v >= qd) v = __dsub_rn(v, qd);
+                            if (v >= qd) v = __dsub_rn(v, qd);  // (the product can touch 2q for the 50-bit prime)
+                            out = d2u(v);
+                        } else {
+                            out = mul_shoup(e[i], mont ? R.ninv_m[mod] : R.ninv[mod], mont ? R.ninv_ms[mod] : R.ninvs[mod], q);
+                        }
+                        if (B.store_centred) out = (out > (q - 1) / 2 ? out - q : out) + (1ull << 59);
+                        dst[gidx] = out;
                     }
                 } else {
                     sm[row * LANES + lane] = e[i];
@@ -271,6 +327,7 @@ __global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : (
                                   ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
 ntt_strided(const RingDev R, const PolyBatch B) {
     __shared__ u64 sm[1 << (LOG_R + LOG_LANES)];
+    grid_dependency_enter();
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
     const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
@@ -440,6 +497,7 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
     __shared__ u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
+    grid_dependency_enter();
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
     const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
@@ -472,7 +530,7 @@ template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
 static void launch_strided_t(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream) {
     constexpr int NT = ((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8);
     dim3 grid((1u << LOG_C) >> LOG_LANES, n_polys);
-    ntt_strided<FWD, LOAD, LOG_R, LOG_LANES><<<grid, NT, 0, stream>>>(ring.dev, B);
+    launch_dependent(ring, ntt_strided<FWD, LOAD, LOG_R, LOG_LANES>, grid, dim3(NT), 0, stream, ring.dev, B);
 }
 
 template <bool FWD, int LOAD>
@@ -501,11 +559,12 @@ static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n
     const u32 cpb = (u32)ring.geom.contig_lanes;
     dim3 grid(chunks / cpb, n_polys);
     if (FWD && epi) {
-        ntt_contig<FWD, true><<<grid, 32 * CHUNKS_PER_BLOCK, 0, stream>>>(ring.dev, B, cpb, *rb, *epi);
+        launch_dependent(ring, ntt_contig<FWD, true>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb, *epi);
     } else {
         static const RotBatch no_rb = {};
         static const ModDownEpilogue no_epi = {};
-        ntt_contig<FWD, false><<<grid, 32 * CHUNKS_PER_BLOCK, 0, stream>>>(ring.dev, B, cpb, no_rb, no_epi);
+        launch_dependent(ring, ntt_contig<FWD, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, no_rb,
+                         no_epi);
     }
     return cudaGetLastError();
 }

@@ -305,6 +305,23 @@ def test_repeated_calls_replay_a_graph_and_still_read_fresh_inputs():
         g.bf.bf_set_graph_replay(g.ctx, False)
         g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
         assert np.array_equal(g.to_host_u64(ct_out)[0], expect[1][0])
+        # plain stream order instead of dependent launches, directly and replayed: same residues
+        g.bf.bf_set_dependent_launch(g.ctx, False)
+        g.bf.bf_set_graph_replay(g.ctx, True)
+        for call in range(4):
+            ct_out.zero_()
+            g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
+            got = g.to_host_u64(ct_out)
+            for p in range(2):
+                assert np.array_equal(got[p], expect[1][p]), (call, p)
+        # and the just-in-time encoding path under dependent launches
+        g.bf.bf_set_dependent_launch(g.ctx, True)
+        for call in range(2):
+            ct_out.zero_()
+            g.bf.bf_linear(g.ctx, ct_in, 3, None, g.to_dev(W), 100, 130, ct_out, 2)
+            got = g.to_host_u64(ct_out)
+            for p in range(2):
+                assert np.array_equal(got[p], expect[1][p]), (call, p)
     finally:
         g.close()
 
