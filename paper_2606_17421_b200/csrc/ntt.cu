@@ -103,7 +103,15 @@ __device__ __forceinline__ double load_src_fp(const void* src, size_t idx, const
 // uses twiddle (tw_base << st) + (blk << st) + sub.
 // Integer version: Harvey's lazy butterflies with Shoup products; forward values stay in [0, 4q),
 // inverse values in [0, 2q).
-template <int K, bool FWD>
+// Twiddle (and companion) number idx: from the global table through the read-only path, or from a copy of
+// the table's head that the block staged in shared memory.
+template <bool TWSM>
+__device__ __forceinline__ ulonglong2 tw_fetch(const ulonglong2* tw, u32 idx) {
+    if (TWSM) return tw[idx];
+    return __ldg(&tw[idx]);
+}
+
+template <int K, bool FWD, bool TWSM = false>
 __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base, u32 blk,
                                                 u64 q, double) {
     const u64 q2 = 2 * q;
@@ -113,7 +121,7 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
         const int d = (1 << K) >> (st + 1);
 #pragma unroll
         for (int sub = 0; sub < (1 << st); ++sub) {
-            const ulonglong2 w = __ldg(&tw[(tw_base << st) + (blk << st) + sub]);
+            const ulonglong2 w = tw_fetch<TWSM>(tw, (tw_base << st) + (blk << st) + sub);
 #pragma unroll
             for (int off = 0; off < d; ++off) {
                 const int i = sub * 2 * d + off;
@@ -142,7 +150,7 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
 // WIDE (primes from 2^41 up to 2^50): the centred product lies in (-0.75q, 0.75q) and values must stay below
 // 4q < 2^52, so the forward butterfly keeps Harvey's invariant [0, 4q) with one conditional subtraction:
 // (X, Y) -> (X~ + T, X~ - T + 2q), X~ = X reduced below 2q, T = Y*w + q in (0.25q, 1.75q).
-template <int K, bool FWD, bool WIDE>
+template <int K, bool FWD, bool WIDE, bool TWSM>
 __device__ __forceinline__ void set_butterflies_fp(double (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base,
                                                    u32 blk, double q) {
     const double q2 = __dadd_rn(q, q);
@@ -152,7 +160,7 @@ __device__ __forceinline__ void set_butterflies_fp(double (&e)[8], const ulonglo
         const int d = (1 << K) >> (st + 1);
 #pragma unroll
         for (int sub = 0; sub < (1 << st); ++sub) {
-            const ulonglong2 wb = __ldg(&tw[(tw_base << st) + (blk << st) + sub]);
+            const ulonglong2 wb = tw_fetch<TWSM>(tw, (tw_base << st) + (blk << st) + sub);
             const double w = __longlong_as_double((long long)wb.x), wq = __longlong_as_double((long long)wb.y);
 #pragma unroll
             for (int off = 0; off < d; ++off) {
@@ -180,11 +188,11 @@ __device__ __forceinline__ void set_butterflies_fp(double (&e)[8], const ulonglo
     }
 }
 
-template <int K, bool FWD>
+template <int K, bool FWD, bool TWSM = false>
 __device__ __forceinline__ void set_butterflies(double (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base,
                                                 u32 blk, u64 q_int, double q) {
-    if (q_int >> 41) set_butterflies_fp<K, FWD, true>(e, tw, tw_base, blk, q);    // block-uniform
-    else set_butterflies_fp<K, FWD, false>(e, tw, tw_base, blk, q);
+    if (q_int >> 41) set_butterflies_fp<K, FWD, true, TWSM>(e, tw, tw_base, blk, q);    // block-uniform
+    else set_butterflies_fp<K, FWD, false, TWSM>(e, tw, tw_base, blk, q);
 }
 
 template <bool FP> struct Elem { typedef u64 T; };
@@ -225,8 +233,11 @@ constexpr int CHUNKS_PER_BLOCK = 8;
 // Strided pass: transforms the 2^LOG_R rows (stride 256) of 2^LOG_LANES adjacent columns.
 // Forward: first pass (reads the batch source through the load functor).  Inverse: second pass
 // (in place, scales by N^{-1}).
-template <bool FWD, int LOAD, int LOG_R, int LOG_LANES, bool FP>
-__device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, u32 o, u32 m, u32 mod) {
+// STAGED: the source tile already sits in shared memory (`staged`, [row][lane], raw words) because several
+// target primes of the same block read it.
+template <bool FWD, int LOAD, int LOG_R, int LOG_LANES, bool FP, bool STAGED = false>
+__device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, ulonglong2* tws, u32 o,
+                                             u32 m, u32 mod, const u64* staged = nullptr) {
     typedef typename Elem<FP>::T T;
     constexpr int LEN = 1 << LOG_R, LANES = 1 << LOG_LANES;
     constexpr int NT = (LEN * LANES / 8) < 32 ? 32 : (LEN * LANES / 8);
@@ -234,7 +245,12 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
     T* sm = (T*)sm_raw;
     const u64 q = R.q[mod], mu = R.mu[mod];
     const double qd = R.qd[mod];
-    const ulonglong2* __restrict__ tw = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
+    // the strided pass uses the first LEN twiddles of the prime only: the block stages them in shared
+    // memory (the load is in flight together with the first data loads)
+    const ulonglong2* __restrict__ tw_global = (FWD ? R.tw_fwd : R.tw_inv) + (size_t)mod * R.N;
+    const ulonglong2* tw = tws;
+    ulonglong2 tw_mine = make_ulonglong2(0, 0);
+    if (threadIdx.x < LEN) tw_mine = __ldg(&tw_global[threadIdx.x]);
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
     const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
                                    : (size_t)o * B.src_so;
@@ -279,8 +295,10 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
                 if (g_first) {
                     const size_t gidx = ((size_t)row << LOG_C) + col0 + lane;
                     if (FWD) {
-                        if constexpr (FP) e[i] = load_src_fp<LOAD>(src, gidx, lc);
-                        else e[i] = load_src<LOAD>(src, gidx, lc);
+                        const void* from = STAGED ? (const void*)staged : (const void*)src;
+                        const size_t at = STAGED ? (size_t)(row * LANES + lane) : gidx;
+                        if constexpr (FP) e[i] = load_src_fp<LOAD>(from, at, lc);
+                        else e[i] = load_src<LOAD>(from, at, lc);
                     } else {
                         e[i] = ((const T*)dst)[gidx];
                     }
@@ -288,9 +306,14 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
                     e[i] = sm[row * LANES + lane];
                 }
             }
-            if (K == 3) set_butterflies<3, FWD>(e, tw, (u32)m0, (u32)blk, q, qd);
-            else if (K == 2) set_butterflies<2, FWD>(e, tw, (u32)m0, (u32)blk, q, qd);
-            else set_butterflies<1, FWD>(e, tw, (u32)m0, (u32)blk, q, qd);
+            if (g_first && w0 == 0) {       // (the first sweep of the first group is full for every geometry)
+                static_assert(NT <= ((LEN * LANES) >> group_k(LOG_R, FWD ? 0 : NG - 1)), "first sweep must be full");
+                if (threadIdx.x < LEN) tws[threadIdx.x] = tw_mine;
+                __syncthreads();
+            }
+            if (K == 3) set_butterflies<3, FWD, true>(e, tw, (u32)m0, (u32)blk, q, qd);
+            else if (K == 2) set_butterflies<2, FWD, true>(e, tw, (u32)m0, (u32)blk, q, qd);
+            else set_butterflies<1, FWD, true>(e, tw, (u32)m0, (u32)blk, q, qd);
 #pragma unroll
             for (int i = 0; i < (1 << K); ++i) {
                 const int row = base + i * step;
@@ -327,6 +350,7 @@ __global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : (
                                   ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
 ntt_strided(const RingDev R, const PolyBatch B) {
     __shared__ u64 sm[1 << (LOG_R + LOG_LANES)];
+    __shared__ ulonglong2 tws[1 << LOG_R];
     grid_dependency_enter();
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
@@ -341,8 +365,51 @@ ntt_strided(const RingDev R, const PolyBatch B) {
         }
         return;
     }
-    if (R.fp_ok[mod]) strided_body<FWD, LOAD, LOG_R, LOG_LANES, true>(R, B, sm, o, m, mod);
-    else strided_body<FWD, LOAD, LOG_R, LOG_LANES, false>(R, B, sm, o, m, mod);
+    if (R.fp_ok[mod]) strided_body<FWD, LOAD, LOG_R, LOG_LANES, true>(R, B, sm, tws, o, m, mod);
+    else strided_body<FWD, LOAD, LOG_R, LOG_LANES, false>(R, B, sm, tws, o, m, mod);
+}
+
+// Forward strided pass of a batch whose n_m target primes all read the same source polynomial (ModUp digits,
+// the P-residues of ModDown): a block stages the source tile in shared memory once and transforms it
+// into targets m_begin .. m_begin + m_count - 1, so the source crosses L2 once per block instead of once per
+// target.  grid: x = tile, y = outer index o, z = slice of the targets.
+template <int LOAD, int LOG_R, int LOG_LANES>
+__global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8),
+                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
+ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
+    constexpr int LANES = 1 << LOG_LANES, POINTS = 1 << (LOG_R + LOG_LANES);
+    extern __shared__ __align__(16) u64 shared_src_smem[];
+    u64* staged = shared_src_smem;                  // [POINTS] raw source words
+    u64* sm = shared_src_smem + POINTS;             // [POINTS] exchange between stage groups
+    ulonglong2* tws = (ulonglong2*)(shared_src_smem + 2 * POINTS);     // [2^LOG_R] twiddles of the current target
+    grid_dependency_enter();
+    const u32 o = blockIdx.y;
+    const u32 m_begin = blockIdx.z * m_per_block;
+    const u32 m_end = min(B.n_m, m_begin + m_per_block);
+    {
+        const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
+                                       : (size_t)o * B.src_so;
+        const u64* src = (const u64*)B.src + src_off;
+        for (int w = threadIdx.x; w < POINTS; w += blockDim.x)
+            staged[w] = src[((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1))];
+    }
+    __syncthreads();
+    for (u32 m = m_begin; m < m_end; ++m) {
+        const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
+        if (B.skip_diag && mod < R.r && o % R.r == mod) {
+            // this digit's transform in its own prime exists already: copy the tile instead
+            const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
+            u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
+            for (int w = threadIdx.x; w < POINTS; w += blockDim.x) {
+                const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1));
+                dd[gidx] = ds[gidx];
+            }
+            continue;
+        }
+        if (R.fp_ok[mod]) strided_body<true, LOAD, LOG_R, LOG_LANES, true, true>(R, B, sm, tws, o, m, mod, staged);
+        else strided_body<true, LOAD, LOG_R, LOG_LANES, false, true>(R, B, sm, tws, o, m, mod, staged);
+        __syncthreads();            // the exchange buffer is free again
+    }
 }
 
 // Contiguous pass: every warp transforms one chunk of 256 adjacent points (8 per thread) through
@@ -533,10 +600,53 @@ static void launch_strided_t(const RingHost& ring, const PolyBatch& B, u32 n_pol
     launch_dependent(ring, ntt_strided<FWD, LOAD, LOG_R, LOG_LANES>, grid, dim3(NT), 0, stream, ring.dev, B);
 }
 
+template <int LOAD, int LOG_R, int LOG_LANES>
+static void launch_shared_src_t(const RingHost& ring, const PolyBatch& B, u32 n_outer, cudaStream_t stream) {
+    constexpr int NT = ((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8);
+    constexpr u32 S = (1u << LOG_C) >> LOG_LANES;
+    // targets per block: fewer blocks share the source better but quantise into waves; cost model =
+    // waves x (targets per block + half a unit for staging the source)
+    const u32 slots = 148u * (NT >= 512 ? 2 : 4);
+    u32 best = 1;
+    double best_cost = 1e30;
+    for (u32 per = 1; per <= B.n_m; ++per) {
+        const u32 slices = (B.n_m + per - 1) / per;
+        if ((B.n_m + slices - 1) / slices != per) continue;         // keep the slices balanced
+        const u32 blocks = S * n_outer * slices;
+        const double cost = (double)((blocks + slots - 1) / slots) * (per + 0.5);
+        if (cost <= best_cost) { best_cost = cost; best = per; }
+    }
+    dim3 grid(S, n_outer, (B.n_m + best - 1) / best);
+    constexpr size_t smem = (size_t)2 * 8 * (1u << (LOG_R + LOG_LANES)) + (size_t)16 * (1u << LOG_R);
+    static bool attr_set = false;     // opt in once to more than 48 KB of dynamic shared memory
+    if (smem > 48 * 1024 && !attr_set) {
+        cudaFuncSetAttribute(ntt_strided_shared_src<LOAD, LOG_R, LOG_LANES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem);
+        attr_set = true;
+    }
+    launch_dependent(ring, ntt_strided_shared_src<LOAD, LOG_R, LOG_LANES>, grid, dim3(NT), smem, stream, ring.dev, B, best);
+}
+
 template <bool FWD, int LOAD>
 static cudaError_t launch_strided(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream) {
     if (n_polys == 0) return cudaSuccess;
     ProfScope prof(ring.prof, FWD ? CAT_NTT_FWD_STRIDED : CAT_NTT_INV_STRIDED, stream);
+    if constexpr (FWD && (LOAD == LOAD_REDUCE || LOAD == LOAD_CENTRED)) {
+        const u32 n_outer = n_polys / B.n_m;
+        if (B.src_sm == 0 && B.n_m > 1 && n_outer <= 65535 && !B.tile_ptr) {
+            switch (ring.geom.log_r) {
+                case 2: launch_shared_src_t<LOAD, 2, 8>(ring, B, n_outer, stream); break;
+                case 3: launch_shared_src_t<LOAD, 3, 8>(ring, B, n_outer, stream); break;
+                case 4: launch_shared_src_t<LOAD, 4, 7>(ring, B, n_outer, stream); break;
+                case 5: launch_shared_src_t<LOAD, 5, 6>(ring, B, n_outer, stream); break;
+                case 6: launch_shared_src_t<LOAD, 6, 5>(ring, B, n_outer, stream); break;
+                case 7: launch_shared_src_t<LOAD, 7, 4>(ring, B, n_outer, stream); break;
+                case 8: launch_shared_src_t<LOAD, 8, 4>(ring, B, n_outer, stream); break;
+                default: return cudaErrorInvalidValue;
+            }
+            return cudaGetLastError();
+        }
+    }
     switch (ring.geom.log_r) {
         case 2: launch_strided_t<FWD, LOAD, 2, 8>(ring, B, n_polys, stream); break;
         case 3: launch_strided_t<FWD, LOAD, 3, 8>(ring, B, n_polys, stream); break;
