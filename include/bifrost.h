@@ -122,6 +122,14 @@ int bf_set_graph_replay(bf_ctx* ctx, int on);
  * stored graphs.  The paper has no counterpart; this is a launch-latency measure. */
 int bf_set_dependent_launch(bf_ctx* ctx, int on);
 
+/* The key switches of a call are independent per rotation.  bf_linear deals the baby rotations of a
+ * batch, and then the giant rotations, out to n_lanes chains (inner product, then division by the
+ * special prime) that run on streams of the library's own between a fork from and a join into the
+ * context's stream, so that one chain's HBM-bound inner product overlaps another chain's
+ * arithmetic-bound transforms.  Results do not depend on n_lanes.  1 <= n_lanes <= 4 (default 2);
+ * bf_set_lanes drops the stored graphs.  The paper has no counterpart. */
+int bf_set_lanes(bf_ctx* ctx, int n_lanes);
+
 /* Rescale (Sec. 2.1): drop the last prime of n_ct ciphertexts that have `level` primes each,
  *     c'_i = (c_i - centred(c_{level-1})) * q_{level-1}^{-1} mod q_i ,
  * i.e. round(c / q_{level-1}).  ct_in: device [n_ct][2][level][N]; ct_out: device

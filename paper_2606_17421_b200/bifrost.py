@@ -55,6 +55,7 @@ _SIGNATURES = {
     "bf_device_status": (ctypes.c_int, [_vp]),
     "bf_set_graph_replay": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_set_dependent_launch": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "bf_set_lanes": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_rescale": (ctypes.c_int, [_vp, _vp, _vp, _u32, _u32, ctypes.POINTER(ctypes.c_double)]),
     "bf_linear_host": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
     "bf_rotate": (ctypes.c_int, [_vp, _vp, _u32, _vp]),
@@ -170,6 +171,10 @@ def bf_device_status(ctx):
 
 def bf_set_graph_replay(ctx, on: bool):
     _check(load().bf_set_graph_replay(ctx, 1 if on else 0), "bf_set_graph_replay", ctx)
+
+
+def bf_set_lanes(ctx, n_lanes: int):
+    _check(load().bf_set_lanes(ctx, n_lanes), "bf_set_lanes", ctx)
 
 
 def bf_set_dependent_launch(ctx, on: bool):

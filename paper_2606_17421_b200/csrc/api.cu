@@ -128,6 +128,13 @@ struct bf_ctx {
     std::map<GraphKey, GraphEntry> graphs;
     u64 epoch = 1;                 // bumped whenever memory the graphs point into is replaced
     int use_graphs = 1;
+    // Independent key-switch chains of one call (groups of baby rotations; groups of giant rotations) run
+    // on side streams between a fork and a join, so that one chain's HBM-bound inner product overlaps
+    // another chain's arithmetic-bound transforms.  lane 0 is the context's stream.
+    static constexpr int MAX_LANES = 4;
+    int n_lanes = 2;                // measured: two chains overlap best (0.651 -> 0.625 ms on the 768 x 2304 layer)
+    cudaStream_t side[MAX_LANES - 1] = {nullptr, nullptr, nullptr};
+    cudaEvent_t ev_fork = nullptr, ev_join[MAX_LANES - 1] = {nullptr, nullptr, nullptr};
     // stage timing
     int timing = 0;
     cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -376,6 +383,11 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
     cudaFree(ctx->slot_of_pos);
     cudaFree(ctx->T);
     cudaFree(ctx->Z);
+    for (cudaStream_t& s : ctx->side)
+        if (s) { cudaStreamDestroy(s); s = nullptr; }
+    for (cudaEvent_t& e : ctx->ev_join)
+        if (e) { cudaEventDestroy(e); e = nullptr; }
+    if (ctx->ev_fork) { cudaEventDestroy(ctx->ev_fork); ctx->ev_fork = nullptr; }
     cudaFree(ctx->overflow_flag);
     cudaFree(ctx->keys);
     cudaFree(ctx->perms);
@@ -603,23 +615,58 @@ extern "C" void bf_weights_free(bf_ctx* ctx, bf_weights* w) {
 // (their inner products already sit in U): inverse transform of the P-residues, centred lift into
 // every q_i with a forward transform whose last store computes (u - t) * P^{-1} + c0 and scatters
 // it through the rotation's permutation.
-static int moddown_batch(bf_ctx* ctx, const RotBatch& rb, const u64* c0_base, long long c0_stride, u64* out_base,
-                         long long out_stride) {
+struct Lane {
+    cudaStream_t s;
+    u64 *Dig, *U, *Tc, *Tn, *Cc;     // this lane's share of the key-switch scratch
+};
+
+static Lane main_lane(bf_ctx* ctx) {
+    return Lane{ctx->stream, (u64*)ctx->Dig.p, (u64*)ctx->U.p, (u64*)ctx->Tc.p, (u64*)ctx->Tn.p, (u64*)ctx->Cc.p};
+}
+
+static int ensure_lanes(bf_ctx* ctx) {
+    if (!ctx->ev_fork) CK(cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
+    for (int i = 0; i + 1 < ctx->n_lanes; ++i) {
+        if (!ctx->side[i]) CK(cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking));
+        if (!ctx->ev_join[i]) CK(cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming));
+    }
+    return BF_OK;
+}
+
+// side streams wait for everything enqueued on the context's stream so far
+static int fork_lanes(bf_ctx* ctx, int used) {
+    if (used <= 1) return BF_OK;
+    CK(cudaEventRecord(ctx->ev_fork, ctx->stream));
+    for (int i = 0; i + 1 < used; ++i) CK(cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
+    return BF_OK;
+}
+
+// the context's stream waits for everything enqueued on the side streams
+static int join_lanes(bf_ctx* ctx, int used) {
+    for (int i = 0; i + 1 < used; ++i) {
+        CK(cudaEventRecord(ctx->ev_join[i], ctx->side[i]));
+        CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_join[i], 0));
+    }
+    return BF_OK;
+}
+
+static int moddown_batch(bf_ctx* ctx, const Lane& lane, const RotBatch& rb, const u64* c0_base, long long c0_stride,
+                         u64* out_base, long long out_stride) {
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
     PolyBatch B;
     memset(&B, 0, sizeof(B));
-    B.src = (const u64*)ctx->U.p + (size_t)r * N;       // the P-residue of each (rotation, component)
-    B.dst = (u64*)ctx->Tc.p;
+    B.src = (const u64*)lane.U + (size_t)r * N;       // the P-residue of each (rotation, component)
+    B.dst = lane.Tc;
     B.src_so = (long long)nb * N;
     B.dst_so = N;
     B.n_m = 1;
     B.mod0 = r;
     B.mod_step = 0;
     B.store_centred = 1;                                // the form the lift below reads
-    CK(ntt_inverse(ctx->ring, B, (u32)rb.n * 2, ctx->stream));
+    CK(ntt_inverse(ctx->ring, B, (u32)rb.n * 2, lane.s));
     memset(&B, 0, sizeof(B));
-    B.src = ctx->Tc.p;
-    B.dst = (u64*)ctx->Tn.p;                            // staging between the two passes of the transform
+    B.src = lane.Tc;
+    B.dst = lane.Tn;                            // staging between the two passes of the transform
     B.src_so = N;
     B.src_sm = 0;
     B.dst_so = (long long)r * N;
@@ -629,13 +676,13 @@ static int moddown_batch(bf_ctx* ctx, const RotBatch& rb, const u64* c0_base, lo
     B.mod_step = 1;
     B.lift_mod = ctx->ring.q[r];
     ModDownEpilogue epi;
-    epi.u = (const u64*)ctx->U.p;
+    epi.u = (const u64*)lane.U;
     epi.c0_base = c0_base;
     epi.c0_stride = c0_stride;
     epi.pinv = ctx->perms;
     epi.out_base = out_base;
     epi.out_stride = out_stride;
-    CK(ntt_forward_moddown(ctx->ring, B, (u32)rb.n * 2, rb, epi, ctx->stream));
+    CK(ntt_forward_moddown(ctx->ring, B, (u32)rb.n * 2, rb, epi, lane.s));
     return BF_OK;
 }
 
@@ -659,8 +706,8 @@ static int find_key(bf_ctx* ctx, u32 steps, int* key) {
 // of the extended basis and transformed: dig[set][j][m] = NTT_m( c1_j mod m ).  The digit in its own
 // prime is the transform of c1 itself, which the caller already has (c1_ntt + s*c1_ntt_stride, [r][N]):
 // it is copied, not recomputed.
-static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_sets, u64* dig, const u64* c1_ntt,
-                 long long c1_ntt_stride) {
+static int modup(bf_ctx* ctx, cudaStream_t stream, const u64* c1_coeff, long long set_stride, u32 n_sets, u64* dig,
+                 const u64* c1_ntt, long long c1_ntt_stride) {
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
     PolyBatch B;
     memset(&B, 0, sizeof(B));
@@ -679,7 +726,7 @@ static int modup(bf_ctx* ctx, const u64* c1_coeff, long long set_stride, u32 n_s
     B.src_digits = 1;
     B.diag_src = c1_ntt;
     B.diag_so = c1_ntt_stride;
-    CK(ntt_forward(ctx->ring, B, n_sets * r, LOAD_REDUCE, ctx->stream));
+    CK(ntt_forward(ctx->ring, B, n_sets * r, LOAD_REDUCE, stream));
     return BF_OK;
 }
 
@@ -713,27 +760,40 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
 
     const u32 gb = giant_batch(ctx);
     const u32 n_giant = (g - 1) * n_out;
-    // input ciphertexts whose baby steps share one key-switch launch
+    // input ciphertexts whose baby steps share one hoisted ModUp
     u32 in_batch = b > 1 ? (u32)MAX_ROT_BATCH / (b - 1) : n_in;
     if (in_batch > gb) in_batch = gb;
     if (in_batch > n_in) in_batch = n_in;
     if (in_batch < 1) in_batch = 1;
-    u32 n_dig_sets = n_giant < gb ? n_giant : gb;       // digit sets alive at once
+    // lanes: the rotations of a stage are dealt out to up to n_lanes independent chains
+    int lanes = ctx->n_lanes < 1 ? 1 : (ctx->n_lanes > bf_ctx::MAX_LANES ? bf_ctx::MAX_LANES : ctx->n_lanes);
+    TRY(ensure_lanes(ctx));
+    const u32 baby_rots = in_batch * (b - 1);
+    const u32 baby_per_lane = cdiv(baby_rots > 0 ? baby_rots : 1, (u32)lanes);
+    u32 giant_per_lane = cdiv(n_giant > 0 ? n_giant : 1, (u32)lanes);     // rotations a lane holds at once
+    if (giant_per_lane > cdiv(gb, (u32)lanes)) giant_per_lane = cdiv(gb, (u32)lanes);
+    if (giant_per_lane < 1) giant_per_lane = 1;
+    const u32 rot_per_lane = baby_per_lane > giant_per_lane ? baby_per_lane : giant_per_lane;
+    u32 n_dig_sets = giant_per_lane * (u32)lanes;       // digit sets alive at once
     if (n_dig_sets < in_batch) n_dig_sets = in_batch;
-    if (n_dig_sets < 1) n_dig_sets = 1;
-    u32 rot_cap = in_batch * (b - 1) > n_dig_sets ? in_batch * (b - 1) : n_dig_sets;
-    if (rot_cap < 1) rot_cap = 1;
     TRY(ensure(ctx, ctx->X, (size_t)n_in * b * ctw * 8));
     TRY(ensure(ctx, ctx->A, (size_t)n_out * g * ctw * 8));
     TRY(ensure(ctx, ctx->Rres, (size_t)(n_giant ? n_giant : 1) * ctw * 8));
     TRY(ensure(ctx, ctx->Cc, (size_t)n_dig_sets * r * N * 8));
-    TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_cap));
+    TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_per_lane * (u32)lanes));
+    Lane lane[bf_ctx::MAX_LANES];
+    for (int c = 0; c < lanes; ++c) {
+        lane[c].s = c == 0 ? ctx->stream : ctx->side[c - 1];
+        lane[c].Dig = (u64*)ctx->Dig.p + (size_t)c * giant_per_lane * r * nb * N;
+        lane[c].U = (u64*)ctx->U.p + (size_t)c * rot_per_lane * 2 * nb * N;
+        lane[c].Tc = (u64*)ctx->Tc.p + (size_t)c * rot_per_lane * 2 * N;
+        lane[c].Tn = (u64*)ctx->Tn.p + (size_t)c * rot_per_lane * 2 * r * N;
+        lane[c].Cc = (u64*)ctx->Cc.p + (size_t)c * giant_per_lane * r * N;
+    }
     u64* X = (u64*)ctx->X.p;
     u64* A = (u64*)ctx->A.p;
     u64* Rres = (u64*)ctx->Rres.p;
     u64* Dig = (u64*)ctx->Dig.p;
-    u64* U = (u64*)ctx->U.p;
-    u64* Cc = (u64*)ctx->Cc.p;
     if (ctx->timing) {
         for (cudaEvent_t& e : ctx->ev)
             if (!e) CK(cudaEventCreate(&e));
@@ -757,21 +817,29 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     if (b > 1) {
         for (u32 q0 = 0; q0 < n_in; q0 += in_batch) {
             const u32 qn = (n_in - q0 < in_batch) ? n_in - q0 : in_batch;
-            TRY(modup(ctx, ct_in + (size_t)q0 * ctw + (size_t)r * N, (long long)ctw, qn, Dig,
+            TRY(modup(ctx, ctx->stream, ct_in + (size_t)q0 * ctw + (size_t)r * N, (long long)ctw, qn, Dig,
                       X + (size_t)q0 * b * ctw + (size_t)r * N, (long long)b * ctw));
-            RotBatch rb;
-            memset(&rb, 0, sizeof(rb));
-            for (u32 q = 0; q < qn; ++q) {
-                for (u32 k = 1; k < b; ++k) {
-                    const int t = rb.n++;
-                    rb.key[t] = baby_key[k];
-                    rb.dig[t] = (int)q;
-                    rb.c0[t] = (int)((q0 + q) * b);
-                    rb.out[t] = (int)((q0 + q) * b + k);
+            // the rotations of the batch, dealt out to the lanes in contiguous runs
+            const u32 n_rot = qn * (b - 1);
+            const u32 per = cdiv(n_rot, (u32)lanes);
+            const int used = (int)cdiv(n_rot, per);
+            TRY(fork_lanes(ctx, used));
+            for (int c = 0; c < used; ++c) {
+                RotBatch rb;
+                memset(&rb, 0, sizeof(rb));
+                const u32 t_end = (u32)(c + 1) * per < n_rot ? (u32)(c + 1) * per : n_rot;
+                for (u32 t = (u32)c * per; t < t_end; ++t) {
+                    const u32 q = t / (b - 1), k = t % (b - 1) + 1;
+                    const int i = rb.n++;
+                    rb.key[i] = baby_key[k];
+                    rb.dig[i] = (int)q;
+                    rb.c0[i] = (int)((q0 + q) * b);
+                    rb.out[i] = (int)((q0 + q) * b + k);
                 }
+                CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, lane[c].U, ctx->device_error, lane[c].s));
+                TRY(moddown_batch(ctx, lane[c], rb, X, (long long)ctw, X, (long long)ctw));
             }
-            CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->device_error, ctx->stream));
-            TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
+            TRY(join_lanes(ctx, used));
         }
     }
     stamp(ctx, 1);
@@ -799,33 +867,42 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     stamp(ctx, 2);
 
     // ---- giant steps: rotate A[j][p] by j*b*tau (full key switch each), then sum over j
-    for (u32 rho0 = 0; rho0 < n_giant; rho0 += gb) {
-        const u32 cnt = (n_giant - rho0 < gb) ? n_giant - rho0 : gb;
-        const u64* Asrc = A + (size_t)(n_out + rho0) * ctw;      // ciphertexts with j >= 1 are contiguous
-        memset(&B, 0, sizeof(B));
-        B.src = Asrc + (size_t)r * N;                            // c1 of each
-        B.dst = Cc;
-        B.src_so = (long long)ctw;
-        B.src_sm = N;
-        B.dst_so = (long long)r * N;
-        B.dst_sm = N;
-        B.n_m = r;
-        B.mod0 = 0;
-        B.mod_step = 1;
-        CK(ntt_inverse(ctx->ring, B, cnt, ctx->stream));
-        TRY(modup(ctx, Cc, (long long)r * N, cnt, Dig, Asrc + (size_t)r * N, (long long)ctw));
-        RotBatch rb;
-        memset(&rb, 0, sizeof(rb));
-        rb.n = (int)cnt;
-        for (u32 t = 0; t < cnt; ++t) {
-            const u32 j = (rho0 + t) / n_out + 1;
-            rb.key[t] = giant_key[j];
-            rb.dig[t] = (int)t;
-            rb.c0[t] = (int)t;
-            rb.out[t] = (int)t;
+    if (n_giant) {
+        const u32 per = cdiv(n_giant, (u32)lanes);
+        const int used = (int)cdiv(n_giant, per);
+        TRY(fork_lanes(ctx, used));
+        for (int c = 0; c < used; ++c) {
+            const u32 lane_end = (u32)(c + 1) * per < n_giant ? (u32)(c + 1) * per : n_giant;
+            for (u32 rho0 = (u32)c * per; rho0 < lane_end; rho0 += giant_per_lane) {
+                const u32 cnt = (lane_end - rho0 < giant_per_lane) ? lane_end - rho0 : giant_per_lane;
+                const u64* Asrc = A + (size_t)(n_out + rho0) * ctw;      // ciphertexts with j >= 1 are contiguous
+                memset(&B, 0, sizeof(B));
+                B.src = Asrc + (size_t)r * N;                            // c1 of each
+                B.dst = lane[c].Cc;
+                B.src_so = (long long)ctw;
+                B.src_sm = N;
+                B.dst_so = (long long)r * N;
+                B.dst_sm = N;
+                B.n_m = r;
+                B.mod0 = 0;
+                B.mod_step = 1;
+                CK(ntt_inverse(ctx->ring, B, cnt, lane[c].s));
+                TRY(modup(ctx, lane[c].s, lane[c].Cc, (long long)r * N, cnt, lane[c].Dig, Asrc + (size_t)r * N, (long long)ctw));
+                RotBatch rb;
+                memset(&rb, 0, sizeof(rb));
+                rb.n = (int)cnt;
+                for (u32 t = 0; t < cnt; ++t) {
+                    const u32 j = (rho0 + t) / n_out + 1;
+                    rb.key[t] = giant_key[j];
+                    rb.dig[t] = (int)t;
+                    rb.c0[t] = (int)t;
+                    rb.out[t] = (int)t;
+                }
+                CK(launch_key_inner_product(ctx->ring, rb, lane[c].Dig, ctx->keys, lane[c].U, ctx->device_error, lane[c].s));
+                TRY(moddown_batch(ctx, lane[c], rb, Asrc, (long long)ctw, Rres + (size_t)rho0 * ctw, (long long)ctw));
+            }
         }
-        CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, U, ctx->device_error, ctx->stream));
-        TRY(moddown_batch(ctx, rb, Asrc, (long long)ctw, Rres + (size_t)rho0 * ctw, (long long)ctw));
+        TRY(join_lanes(ctx, used));
     }
     stamp(ctx, 3);
 
@@ -939,6 +1016,13 @@ extern "C" int bf_set_graph_replay(bf_ctx* ctx, int on) {
     return BF_OK;
 }
 
+extern "C" int bf_set_lanes(bf_ctx* ctx, int n_lanes) {
+    if (!ctx || n_lanes < 1 || n_lanes > bf_ctx::MAX_LANES) return BF_ERR_INVALID_ARG;
+    ctx->n_lanes = n_lanes;
+    destroy_graphs(ctx);            // stored graphs have the old shape
+    return BF_OK;
+}
+
 extern "C" int bf_set_dependent_launch(bf_ctx* ctx, int on) {
     if (!ctx) return BF_ERR_INVALID_ARG;
     ctx->ring.dependent_launch = on != 0;
@@ -996,7 +1080,7 @@ extern "C" int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uin
     B.n_m = r;
     B.mod_step = 1;
     CK(ntt_forward(ctx->ring, B, 2, LOAD_PLAIN, ctx->stream));
-    TRY(modup(ctx, ct_in + (size_t)r * N, (long long)r * N, 1, (u64*)ctx->Dig.p, X + (size_t)r * N, 0));
+    TRY(modup(ctx, ctx->stream, ct_in + (size_t)r * N, (long long)r * N, 1, (u64*)ctx->Dig.p, X + (size_t)r * N, 0));
     RotBatch rb;
     memset(&rb, 0, sizeof(rb));
     rb.n = 1;
@@ -1004,7 +1088,7 @@ extern "C" int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uin
     rb.out[0] = 1;
     CK(launch_key_inner_product(ctx->ring, rb, (const u64*)ctx->Dig.p, ctx->keys, (u64*)ctx->U.p, ctx->device_error,
                                 ctx->stream));
-    TRY(moddown_batch(ctx, rb, X, (long long)ctw, X, (long long)ctw));
+    TRY(moddown_batch(ctx, main_lane(ctx), rb, X, (long long)ctw, X, (long long)ctw));
     memset(&B, 0, sizeof(B));
     B.src = X + ctw;
     B.dst = ct_out;

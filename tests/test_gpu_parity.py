@@ -314,8 +314,17 @@ def test_repeated_calls_replay_a_graph_and_still_read_fresh_inputs():
             got = g.to_host_u64(ct_out)
             for p in range(2):
                 assert np.array_equal(got[p], expect[1][p]), (call, p)
-        # and the just-in-time encoding path under dependent launches
+        # any number of concurrent key-switch chains, directly and replayed
         g.bf.bf_set_dependent_launch(g.ctx, True)
+        for lanes in (1, 3, 4, 2):
+            g.bf.bf_set_lanes(g.ctx, lanes)
+            for call in range(3):
+                ct_out.zero_()
+                g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
+                got = g.to_host_u64(ct_out)
+                for p in range(2):
+                    assert np.array_equal(got[p], expect[1][p]), (lanes, call, p)
+        # and the just-in-time encoding path under dependent launches
         for call in range(2):
             ct_out.zero_()
             g.bf.bf_linear(g.ctx, ct_in, 3, None, g.to_dev(W), 100, 130, ct_out, 2)
