@@ -111,7 +111,7 @@ template <bool KARA, int LOG_TN>
 __global__ void __launch_bounds__(MAC_THREADS, 3)
 mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, const u64* __restrict__ x,
            u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, u32 early_weights,
-           int* __restrict__ error_flag) {
+           u32 n_whole, u32 tail_split, int* __restrict__ error_flag) {
     extern __shared__ __align__(128) unsigned char mac_smem[];
     asm volatile("griddepcontrol.launch_dependents;");
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
@@ -120,11 +120,29 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
     u64* full = xs + (size_t)n_terms * 2 * TN;                     // [MAC_STAGES]
     u64* empty = full + MAC_STAGES;                                // [MAC_STAGES]
     u64* xbar = empty + MAC_STAGES;
-    const u32 i = blockIdx.y, N = R.N, r = R.r;
-    const u32 n0 = blockIdx.x << LOG_TN;
+    // Work units (tile, prime, slice of the output groups) are numbered tile-fastest.  The first n_whole
+    // blocks take one unit each; the units after them (the part that would be a thin last wave) are each
+    // cut into tail_split blocks over their output groups, so that the last wave is short instead.
+    const u32 N = R.N, r = R.r;
     const u32 tid = threadIdx.x;
-    const u32 pj_begin = blockIdx.z * pj_per_block;
-    const u32 pj_end = min(n_pj, pj_begin + pj_per_block);
+    u32 unit = blockIdx.x, sub = 0, n_sub = 1;
+    if (unit >= n_whole) {
+        sub = (unit - n_whole) % tail_split;
+        unit = n_whole + (unit - n_whole) / tail_split;
+        n_sub = tail_split;
+    }
+    const u32 tile_x = unit % (N >> LOG_TN);
+    const u32 i = (unit / (N >> LOG_TN)) % r;
+    const u32 n0 = tile_x << LOG_TN;
+    u32 pj_begin = (unit / (N >> LOG_TN) / r) * pj_per_block;
+    u32 pj_end = min(n_pj, pj_begin + pj_per_block);
+    if (n_sub > 1) {
+        const u32 groups = (pj_end - pj_begin + PL - 1) / PL;
+        const u32 per = (groups + n_sub - 1) / n_sub * PL;
+        pj_begin = min(pj_end, pj_begin + sub * per);
+        pj_end = min(pj_end, pj_begin + per);
+        if (pj_begin >= pj_end) return;                            // (uniform for the block)
+    }
     const u32 n_groups = (pj_end - pj_begin + PL - 1) / PL;        // rounds of PL output groups
     const u32 n_chunks = (n_terms + MAC_TS - 1) / MAC_TS;
     const u32 n_items = n_groups * n_chunks;
@@ -150,7 +168,7 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
             const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
             const u32 first = pj_begin + g * PL;
             const u32 lanes = min((u32)PL, pj_end - first);
-            const u64* stage = pt + tile_stage_offset(lay, i, blockIdx.x, first / PL, ch);
+            const u64* stage = pt + tile_stage_offset(lay, i, tile_x, first / PL, ch);
             u64* sdst = ring + (size_t)slot * MAC_STAGE_WORDS;
             if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * 8);
             __syncwarp();
@@ -317,9 +335,36 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     u32 pj_per_block = (n_pj + slices - 1) / slices;
     pj_per_block = (pj_per_block + PL - 1) / PL * PL;
     slices = (n_pj + pj_per_block - 1) / pj_per_block;
-    dim3 grid(ring.dev.N >> LOG_TN, ring.dev.r, slices);
+    // blocks resident at once; when the units leave a thin last wave, cut those units into shorter blocks
+    static int sm_count = 0, per_sm = 0;
+    static size_t per_sm_smem = 0;
+    if (!sm_count) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (sm_count <= 0) sm_count = 148;
+    }
+    if (per_sm_smem != smem) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mac_kernel<KARA, LOG_TN>, MAC_THREADS, smem) != cudaSuccess ||
+            per_sm < 1) {
+            cudaGetLastError();
+            per_sm = 1;
+        }
+        per_sm_smem = smem;
+    }
+    const u32 slots = (u32)sm_count * (u32)per_sm;
+    const u32 units = tiles * slices;
+    const u32 rem = units % slots;
+    u32 tail_split = 1;
+    if (units > slots && rem && rem * 2 < slots) {
+        tail_split = slots / rem;
+        if (tail_split > pj_per_block / PL) tail_split = pj_per_block / PL;
+        if (tail_split < 1) tail_split = 1;
+    }
+    const u32 n_whole = tail_split > 1 ? units - rem : units;
+    dim3 grid(n_whole + (units - n_whole) * tail_split);
     return launch_dependent(ring, mac_kernel<KARA, LOG_TN>, grid, dim3(MAC_THREADS), smem, stream, ring.dev, pt, lay, x, a,
-                            n_terms, n_pj, pj_per_block, lazy, early_weights, error_flag);
+                            n_terms, n_pj, pj_per_block, lazy, early_weights, n_whole, tail_split, error_flag);
 }
 
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
