@@ -77,6 +77,21 @@ __device__ __forceinline__ double fp_mul_centred(double x, double w, double wq, 
     const double qh = __dsub_rn(__fma_rn(x, wq, magic), magic);
     return __dadd_rn(__fma_rn(-qh, q, ph), pl);
 }
+// The same product for a signed integer-valued |x| < 2^47 and q < 2^41 (rounding constant 1.5 * 2^52, which
+// is exact for quotients of either sign): congruent to x*w, |result| <= 0.532 q.
+__device__ __forceinline__ double fp_mul_centred_signed(double x, double w, double wq, double q) {
+    const double magic = 6755399441055744.0;             // 1.5 * 2^52
+    const double ph = __dmul_rn(x, w);
+    const double pl = __fma_rn(x, w, -ph);
+    const double qh = __dsub_rn(__fma_rn(x, wq, magic), magic);
+    return __dadd_rn(__fma_rn(-qh, q, ph), pl);
+}
+// v - round(v / q) q for a signed integer-valued |v| < 2^50: congruent to v, |result| <= q / 2
+__device__ __forceinline__ double fp_centre(double v, double q, double qinv) {
+    const double magic = 6755399441055744.0;
+    const double qh = __dsub_rn(__fma_rn(v, qinv, magic), magic);
+    return __fma_rn(-qh, q, v);
+}
 // v mod q in [0, q) for an integer-valued 0 <= v < 2^46
 __device__ __forceinline__ double fp_reduce(double v, double q, double qinv) {
     const double magic = 4503599627370496.0;

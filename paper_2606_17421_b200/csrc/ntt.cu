@@ -45,6 +45,7 @@ ProfScope::~ProfScope() {
 struct LoadConsts {
     u64 q, mu, lift_mod, lift_red;
     double qd, qinv, c30, c30q, k59;
+    bool wide;          // target prime of 2^41 or more: values must stay in [0, 4q); otherwise they are signed
     bool src_small;     // LOAD_REDUCE: every source word is below 1.5 q already (block-uniform)
     bool src_fp;        // LOAD_REDUCE: every source word is below 2^51
 };
@@ -80,11 +81,9 @@ __device__ __forceinline__ double load_src_fp(const void* src, size_t idx, const
     if (LOAD == LOAD_REDUCE) {
         const u64 t = ((const u64*)src)[idx];
         if (c.src_small) return u2d(t);
-        if (c.src_fp) {                                  // t - round(t / q) q + q  in [0.5 q, 1.5 q]
-            const double magic = 4503599627370496.0;
-            const double v = u2d(t);
-            const double qh = __dsub_rn(__fma_rn(v, c.qinv, magic), magic);
-            return __dadd_rn(__fma_rn(-qh, c.qd, v), c.qd);
+        if (c.src_fp) {                                  // t - round(t / q) q, plus q where values must not be negative
+            const double v = fp_centre(u2d(t), c.qd, c.qinv);
+            return c.wide ? __dadd_rn(v, c.qd) : v;
         }
         return u2d(barrett64(t, c.q, c.mu));
     }
@@ -93,7 +92,7 @@ __device__ __forceinline__ double load_src_fp(const void* src, size_t idx, const
         // centred in (-0.75 q, 0.75 q), lo < 2^30 and k59 = 2q - (2^59 mod q) the sum is positive
         const u64 T = ((const u64*)src)[idx];
         const double hi = u2d(T >> 30), lo = u2d(T & ((1ull << 30) - 1));
-        return __dadd_rn(__dadd_rn(fp_mul_centred(hi, c.c30, c.c30q, c.qd), lo), c.k59);
+        return __dadd_rn(__dadd_rn(fp_mul_centred(hi, c.c30, c.c30q, c.qd), lo), c.k59);   // (k59: see LoadConsts)
     }
     return u2d(load_src<LOAD>(src, idx, c));
 }
@@ -143,13 +142,19 @@ __device__ __forceinline__ void set_butterflies(u64 (&e)[8], const ulonglong2* _
     }
 }
 
-// fp64 version (primes below 2^41).  Forward: (X, Y) -> (X + q + s, X + q - s) with s = Y*w centred in
-// (-0.51q, 0.51q): values stay non-negative and grow by at most 1.51q per stage, so after all
-// log2 N <= 16 stages they are below 26q < 2^46 and need one reduction at the very end.
-// Inverse: (a, b) -> (a + b reduced below 2q, (a - b + 2q)*w + q in (0.49q, 1.51q)): values in [0, 2q).
+// fp64 version.  Primes below 2^41: values are signed integer-valued doubles, reduced lazily.
+//   Forward: (X, Y) -> (X + s, X - s), s = Y*w centred in (-0.54q, 0.54q): magnitudes grow by at most 0.54q
+//   per stage, from at most 3.6q after the load functors to below 13q after log2 N <= 16 stages; one
+//   reduction at the very end.
+//   Inverse: (a, b) -> (a + b, (a - b)*w centred): the sums double per stage and the product takes
+//   |a - b| < 2^47, i.e. magnitudes below 32q going into a stage.  From [0, q) the contiguous pass runs its
+//   first two groups (5 stages, sums up to 32q), centres the sums, and leaves at most 4.4q after its last
+//   group; the strided pass centres the sums after its first group when more groups follow, which keeps
+//   every later stage below 18q going in and the values handed to the final scaling below 35q.
 // WIDE (primes from 2^41 up to 2^50): the centred product lies in (-0.75q, 0.75q) and values must stay below
 // 4q < 2^52, so the forward butterfly keeps Harvey's invariant [0, 4q) with one conditional subtraction:
-// (X, Y) -> (X~ + T, X~ - T + 2q), X~ = X reduced below 2q, T = Y*w + q in (0.25q, 1.75q).
+// (X, Y) -> (X~ + T, X~ - T + 2q), X~ = X reduced below 2q, T = Y*w + q in (0.25q, 1.75q); the inverse is
+// (a, b) -> (a + b reduced below 2q, (a - b + 2q)*w + q in (0.25q, 1.75q)): values in [0, 2q).
 template <int K, bool FWD, bool WIDE, bool TWSM>
 __device__ __forceinline__ void set_butterflies_fp(double (&e)[8], const ulonglong2* __restrict__ tw, u32 tw_base,
                                                    u32 blk, double q) {
@@ -172,16 +177,20 @@ __device__ __forceinline__ void set_butterflies_fp(double (&e)[8], const ulonglo
                     e[i] = __dadd_rn(x, t);
                     e[i + d] = __dadd_rn(__dsub_rn(x, t), q2);
                 } else if (FWD) {
-                    const double sv = fp_mul_centred(e[i + d], w, wq, q);
-                    const double xq = __dadd_rn(e[i], q);
-                    e[i] = __dadd_rn(xq, sv);
-                    e[i + d] = __dsub_rn(xq, sv);
-                } else {
+                    const double sv = fp_mul_centred_signed(e[i + d], w, wq, q);
+                    const double x = e[i];
+                    e[i] = __dadd_rn(x, sv);
+                    e[i + d] = __dsub_rn(x, sv);
+                } else if (WIDE) {
                     const double a = e[i], b = e[i + d];
                     double s2 = __dadd_rn(a, b);
                     if (s2 >= q2) s2 = __dsub_rn(s2, q2);
                     e[i] = s2;
                     e[i + d] = __dadd_rn(fp_mul_centred(__dadd_rn(__dsub_rn(a, b), q2), w, wq, q), q);
+                } else {
+                    const double a = e[i], b = e[i + d];
+                    e[i] = __dadd_rn(a, b);
+                    e[i + d] = fp_mul_centred_signed(__dsub_rn(a, b), w, wq, q);
                 }
             }
         }
@@ -194,6 +203,17 @@ __device__ __forceinline__ void set_butterflies(double (&e)[8], const ulonglong2
     if (q_int >> 41) set_butterflies_fp<K, FWD, true, TWSM>(e, tw, tw_base, blk, q);    // block-uniform
     else set_butterflies_fp<K, FWD, false, TWSM>(e, tw, tw_base, blk, q);
 }
+
+// After an inverse group of K stages the first 2^(K-1) values of a set are sums (they doubled per stage),
+// the others fresh centred products: bring the sums back to |v| <= q/2.  Signed fp64 path only.
+template <int K>
+__device__ __forceinline__ void centre_sums(double (&e)[8], u64 q_int, double q, double qinv) {
+    if (q_int >> 41) return;
+#pragma unroll
+    for (int i = 0; i < (1 << K) / 2; ++i) e[i] = fp_centre(e[i], q, qinv);
+}
+template <int K>
+__device__ __forceinline__ void centre_sums(u64 (&)[8], u64, double, double) {}
 
 template <bool FP> struct Elem { typedef u64 T; };
 template <> struct Elem<true> { typedef double T; };
@@ -264,7 +284,9 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
     lc.qinv = R.qinv_d[mod];
     lc.c30 = R.c30_d[mod];
     lc.c30q = R.c30_q[mod];
-    lc.k59 = R.k59_d[mod];
+    lc.wide = (q >> 41) != 0;
+    // wide: 2q - (2^59 mod q) keeps the lifted value positive; otherwise the offset is just -(2^59 mod q)
+    lc.k59 = lc.wide ? R.k59_d[mod] : __dsub_rn(R.k59_d[mod], __dadd_rn(qd, qd));
     {
         const u64 qs = (LOAD == LOAD_REDUCE && B.src_digits) ? R.q[o % R.r] : ~(u64)0;
         lc.src_small = qs <= q + (q >> 1);
@@ -314,6 +336,11 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
             if (K == 3) set_butterflies<3, FWD, true>(e, tw, (u32)m0, (u32)blk, q, qd);
             else if (K == 2) set_butterflies<2, FWD, true>(e, tw, (u32)m0, (u32)blk, q, qd);
             else set_butterflies<1, FWD, true>(e, tw, (u32)m0, (u32)blk, q, qd);
+            if (!FWD && g_first && NG > 1) {
+                if (K == 3) centre_sums<3>(e, q, qd, R.qinv_d[mod]);
+                else if (K == 2) centre_sums<2>(e, q, qd, R.qinv_d[mod]);
+                else centre_sums<1>(e, q, qd, R.qinv_d[mod]);
+            }
 #pragma unroll
             for (int i = 0; i < (1 << K); ++i) {
                 const int row = base + i * step;
@@ -325,10 +352,17 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
                         const bool mont = B.from_mont != 0;
                         u64 out;
                         if constexpr (FP) {
-                            double v = __dadd_rn(fp_mul_centred(e[i], mont ? R.ninvm_d[mod] : R.ninv_d[mod],
-                                                                mont ? R.ninvm_q[mod] : R.ninv_q[mod], qd), qd);
-                            if (v >= qd) v = __dsub_rn(v, qd);
-                            if (v >= qd) v = __dsub_rn(v, qd);  // (the product can touch 2q for the 50-bit prime)
+                            const double nv = mont ? R.ninvm_d[mod] : R.ninv_d[mod];
+                            const double nq = mont ? R.ninvm_q[mod] : R.ninv_q[mod];
+                            double v;
+                            if (q >> 41) {
+                                v = __dadd_rn(fp_mul_centred(e[i], nv, nq, qd), qd);
+                                if (v >= qd) v = __dsub_rn(v, qd);
+                                if (v >= qd) v = __dsub_rn(v, qd);  // (the product can touch 2q for the 50-bit prime)
+                            } else {
+                                v = fp_mul_centred_signed(e[i], nv, nq, qd);
+                                if (v < 0.0) v = __dadd_rn(v, qd);
+                            }
                             out = d2u(v);
                         } else {
                             out = mul_shoup(e[i], mont ? R.ninv_m[mod] : R.ninv[mod], mont ? R.ninv_ms[mod] : R.ninvs[mod], q);
@@ -461,7 +495,13 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 #pragma unroll
             for (int i = 0; i < 4; ++i) {   // final reduction to [0, q)
                 if (FP) {
-                    v4[i] = d2u(fp_reduce(*(double*)&e[i], qd, R.qinv_d[mod]));
+                    if (q >> 41) {
+                        v4[i] = d2u(fp_reduce(*(double*)&e[i], qd, R.qinv_d[mod]));
+                    } else {
+                        double v = fp_centre(*(double*)&e[i], qd, R.qinv_d[mod]);
+                        if (v < 0.0) v = __dadd_rn(v, qd);
+                        v4[i] = d2u(v);
+                    }
                 } else {
                     u64 v = *(u64*)&e[i];
                     if (v >= 2 * q) v -= 2 * q;
@@ -547,6 +587,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 #pragma unroll
             for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
             set_butterflies<3, false>(e, tw, 8u * mult, (u32)blk, q, qd);
+            centre_sums<3>(e, q, qd, R.qinv_d[mod]);
 #pragma unroll
             for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
         }
