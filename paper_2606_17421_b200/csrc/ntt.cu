@@ -241,7 +241,48 @@ __host__ __device__ constexpr int group_log_step(int log_len, int gi) {
 // Shared-memory index swizzle for a 256-point chunk of 64-bit words: makes the three access
 // patterns of the contiguous pass (spacing 32, spacing 4 and 4 adjacent points per thread) free of
 // bank conflicts without padding.
-__device__ __forceinline__ int swz(int i) { return i ^ ((i >> 4) & 3) ^ (((i >> 5) & 3) << 2); }
+__host__ __device__ constexpr int swz(int i) { return i ^ ((i >> 4) & 3) ^ (((i >> 5) & 3) << 2); }
+
+// The swizzle is linear over GF(2): swz(t ^ k) = swz(t) ^ swz(k).  Every access of the contiguous pass has
+// index t ^ k with t depending on the thread and k on the unrolled loop counter, in disjoint bit fields, so
+// its byte address is (A ^ 8 * (swz(k) & 15)) + 8 * (swz(k) & ~15) with A = slice base + 8 * swz(t) computed
+// once per group: one logic operation and an immediate offset per access.  (The swizzle only changes the low
+// four index bits, and t has no bits where swz(k) & ~15 has any.)  The slice base is 128-byte aligned.
+template <int K_INDEX>
+__device__ __forceinline__ void swz_store(u32 a_thread, u64 v) {
+    constexpr int S = swz(K_INDEX);
+    asm volatile("st.shared.b64 [%0+%1], %2;" ::"r"(a_thread ^ (u32)(8 * (S & 15))), "n"(8 * (S & ~15)), "l"(v));
+}
+template <int K_INDEX>
+__device__ __forceinline__ void swz_store(u32 a_thread, double v) {
+    swz_store<K_INDEX>(a_thread, (u64)__double_as_longlong(v));
+}
+template <int K_INDEX>
+__device__ __forceinline__ void swz_load(u32 a_thread, u64& v) {
+    constexpr int S = swz(K_INDEX);
+    asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(v) : "r"(a_thread ^ (u32)(8 * (S & 15))), "n"(8 * (S & ~15)));
+}
+template <int K_INDEX>
+__device__ __forceinline__ void swz_load(u32 a_thread, double& v) {
+    u64 bits;
+    swz_load<K_INDEX>(a_thread, bits);
+    v = __longlong_as_double((long long)bits);
+}
+// e[i] <-> slice[swz(t ^ (i << SHIFT))] for i < COUNT
+template <int COUNT, int SHIFT, typename T, int I = 0>
+__device__ __forceinline__ void swz_store_set(u32 a_thread, const T (&e)[8]) {
+    if constexpr (I < COUNT) {
+        swz_store<(I << SHIFT)>(a_thread, e[I]);
+        swz_store_set<COUNT, SHIFT, T, I + 1>(a_thread, e);
+    }
+}
+template <int COUNT, int SHIFT, typename T, int I = 0>
+__device__ __forceinline__ void swz_load_set(u32 a_thread, T (&e)[8]) {
+    if constexpr (I < COUNT) {
+        swz_load<(I << SHIFT)>(a_thread, e[I]);
+        swz_load_set<COUNT, SHIFT, T, I + 1>(a_thread, e);
+    }
+}
 
 constexpr int LOG_C = 8;              // contiguous pass: chunks of 256 points, one warp each
 constexpr int CHUNKS_PER_BLOCK = 8;
@@ -465,31 +506,32 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
     const u32 mult = (R.N >> LOG_C) + chunk;                   // twiddle index multiplier of this chunk
     const u64* gsrc = src + (size_t)chunk * LEN;
     u64* gdst = dst + (size_t)chunk * LEN;
+    // byte addresses (shared window) of the thread's base point in each of the three access patterns
+    const u32 slice = (u32)__cvta_generic_to_shared(sm);
+    const u32 a_far = slice + 8u * (u32)swz(lane);                                    // points lane + 32 i
+    const u32 a_mid = slice + 8u * (u32)swz((lane >> 2) * 32 + (lane & 3));           // points base + 4 i
+    const u32 a_near = slice + 8u * (u32)swz(4 * lane);                               // points 4 (lane + 32 it) + i
     T e[8];
     if (FWD) {
         // group 0: K = 3, spacing 32
 #pragma unroll
         for (int i = 0; i < 8; ++i) e[i] = ((const T*)gsrc)[lane + 32 * i];
         set_butterflies<3, true>(e, tw, 1u * mult, 0u, q, qd);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) sm[swz(lane + 32 * i)] = e[i];
+        swz_store_set<8, 5>(a_far, e);
         __syncwarp();
         // group 1: K = 3, spacing 4
         {
-            const int blk = lane >> 2, base = blk * 32 + (lane & 3);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
+            const int blk = lane >> 2;
+            swz_load_set<8, 2>(a_mid, e);
             set_butterflies<3, true>(e, tw, 8u * mult, (u32)blk, q, qd);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
+            swz_store_set<8, 2>(a_mid, e);
         }
         __syncwarp();
         // group 2: K = 2, adjacent points; two sets per thread
 #pragma unroll
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) e[i] = sm[swz(4 * s + i)];
+            swz_load_set<4, 0>(a_near + (u32)(it * 8 * swz(128)), e);      // (swz(128) = 128: above the bits of 4 * lane)
             set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, qd);
             u64 v4[4];
 #pragma unroll
@@ -578,22 +620,18 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 #pragma unroll
             for (int i = 0; i < 4; ++i) from_u64(e[i], v4[i]);
             set_butterflies<2, false>(e, tw, 64u * mult, (u32)s, q, qd);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) sm[swz(4 * s + i)] = e[i];
+            swz_store_set<4, 0>(a_near + (u32)(it * 8 * swz(128)), e);
         }
         __syncwarp();
         {
-            const int blk = lane >> 2, base = blk * 32 + (lane & 3);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) e[i] = sm[swz(base + 4 * i)];
+            const int blk = lane >> 2;
+            swz_load_set<8, 2>(a_mid, e);
             set_butterflies<3, false>(e, tw, 8u * mult, (u32)blk, q, qd);
             centre_sums<3>(e, q, qd, R.qinv_d[mod]);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) sm[swz(base + 4 * i)] = e[i];
+            swz_store_set<8, 2>(a_mid, e);
         }
         __syncwarp();
-#pragma unroll
-        for (int i = 0; i < 8; ++i) e[i] = sm[swz(lane + 32 * i)];
+        swz_load_set<8, 5>(a_far, e);
         set_butterflies<3, false>(e, tw, 1u * mult, 0u, q, qd);
 #pragma unroll
         for (int i = 0; i < 8; ++i) ((T*)gdst)[lane + 32 * i] = e[i];      // lazy, below 2q; the strided pass finishes
@@ -604,7 +642,7 @@ template <bool FWD, bool EPI>
 __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
-    __shared__ u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
+    __shared__ __align__(128) u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
     grid_dependency_enter();
     const u32 poly = blockIdx.y;
     const u32 o = poly / B.n_m, m = poly % B.n_m;
