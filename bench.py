@@ -31,9 +31,11 @@ UNIT = "ms"
 # see profiles/ for the capture each figure comes from.  None = not captured yet.
 NCU_TRAFFIC_BYTES = {
     # from the ncu capture summarised under profiles/: dram__bytes_read.sum + dram__bytes_write.sum per launch
-    "gpt2_qkv": {"mac": 448.2e6,                       # 411.1 MB read + 37.1 MB written
-                 "key_inner_product": 379.8e6,         # mean of the baby (510.2 MB) and giant (249.4 MB) launches
-                 "ntt_fwd_strided": 4.8e6, "ntt_inv_contig": 47.9e6},
+    "gpt2_qkv": {"mac": 423.8e6,                       # 411.1 MB read + 12.7 MB written
+                 "key_inner_product": 395.0e6,         # baby 517.5 MB + giant 272.6 MB per step, over the two launches
+                                                       #   of the serialised timing pass
+                 "ntt_fwd_strided": 23.0e6,            # mean of the eight captured forward launches (both passes)
+                 "ntt_inv_contig": 21.0e6},            # mean of the six captured inverse launches (both passes)
 }
 
 
@@ -100,15 +102,15 @@ DEFAULT_LANES = 2       # the library's default number of concurrent key-switch 
 
 def butterflies_per_step(runner) -> dict:
     """Transforms one step launches, by direction and by arithmetic path.  Moduli below 2^41 run in
-    fp64 with 9 fp64 operations per butterfly, moduli from 2^41 up to 2^50 in fp64 with one more
-    conditional subtraction and offset (12 operations), the 60-bit special prime in integers (at
-    least 10 32-bit multiply-adds per butterfly); both pipes issue 64 lanes per clock per SM."""
+    fp64 with 8 fp64 operations per butterfly (signed lazy values), moduli from 2^41 up to 2^50 in fp64
+    with a conditional subtraction and offsets (12 operations), the 60-bit special prime in integers
+    (at least 10 32-bit multiply-adds per butterfly); both pipes issue 64 lanes per clock per SM."""
     import math
     r, N = runner.r, runner.N
     b, g = runner.plan.b, runner.plan.g
     per = (N // 2) * int(math.log2(N))
     moduli = list(runner.primes) + [runner.P]
-    cost = [9 if q < (1 << 41) else 12 if q < (1 << 50) else 10 for q in moduli]
+    cost = [8 if q < (1 << 41) else 12 if q < (1 << 50) else 10 for q in moduli]
     fp = [q < (1 << 50) for q in moduli]
     fwd = [0] * (r + 1)
     inv = [0] * (r + 1)
@@ -289,7 +291,7 @@ def run_ours(args):
             rooflines[label] = {"bound": "alu", "achieved": round(rate / 1e9, 1), "peak": round(peak / 1e9, 1),
                                 "unit": "G butterflies/s", "frac": round(rate / peak, 4),
                                 "of": (f"derived: 148 SMs x 64 lanes x {sm_mhz:.0f} MHz / {info['ops_per_butterfly']:.2f} "
-                                       "pipe operations per butterfly (9 fp64 ops below 2^41, 12 up to 2^50, 10 multiply-adds on "
+                                       "pipe operations per butterfly (8 fp64 ops below 2^41, 12 up to 2^50, 10 multiply-adds on "
                                        f"the integer path); bf_measure_imad_rate measured {imad_rate / 1e12:.2f} T multiply-adds/s"),
                                 "traffic": traffic.get(cats[0]), "ms_per_step": round(ms_step, 5),
                                 "polys_per_step": info["polys"], "fp64_polys_per_step": info["fp64_polys"]}
