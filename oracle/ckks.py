@@ -398,9 +398,14 @@ def required_rotations(plan: Plan) -> list[int]:
     return [k * plan.tau for k in range(1, plan.b)] + [j * plan.b * plan.tau for j in range(1, plan.g)]
 
 
-def make_rotation_keys(params: Params, s: np.ndarray, plan: Plan, seed: int) -> dict:
+def fold_rotations(plan: Plan) -> list[int]:
+    """Rotation amounts of the in-ciphertext fold of the tau partial sums: 1, 2, ..., tau/2."""
+    return [1 << i for i in range(plan.tau.bit_length() - 1)]
+
+
+def make_rotation_keys(params: Params, s: np.ndarray, plan: Plan, seed: int, extra_steps=()) -> dict:
     keys = {}
-    for steps in required_rotations(plan):
+    for steps in list(required_rotations(plan)) + list(extra_steps):
         g = galois_element(steps, params.N)
         if g not in keys:
             keys[g] = galois_key(params, s, g, seed)
@@ -540,6 +545,31 @@ def fold_output(slots: np.ndarray, plan: Plan, p: int, d_out: int) -> np.ndarray
     """Host-side fold of the tau partial sums: y[p*D + kappa] = sum_c slot((0, kappa, c))."""
     D, tau = plan.D, plan.tau
     part = np.asarray(slots).real[:D * tau].reshape(D, tau).sum(axis=1)
+    rows = min(D, d_out - p * D)
+    return part[:rows]
+
+
+def fold_in_ciphertext(params: Params, plan: Plan, ct: np.ndarray, keys: dict) -> np.ndarray:
+    """The variant of the output stage that sums the tau partial results inside the ciphertext (the
+    packing of Sec. 4.2 leaves slot (rho, kappa, c) with the partial dot product over column class c):
+        for i = 0 .. log2(tau) - 1:  ct <- ct + rot(ct, 2^i)
+    after which slot (0, kappa, 0) holds the sum over all c, i.e. the complete dot product of row kappa.
+    Costs log2(tau) key switches per output ciphertext; level and scale are unchanged.  The default path
+    leaves this sum to the host after decryption (fold_output)."""
+    assert plan.tau & (plan.tau - 1) == 0, "the fold needs a power-of-two tau"
+    q = np.array(params.primes, dtype=np.uint64).reshape(1, -1, 1)
+    out = ct.copy()
+    for steps in fold_rotations(plan):
+        rot = rotate(params, out, steps, keys)
+        t = out + rot                       # residues are below 2^60: no wrap-around in 64 bits
+        out = np.where(t >= q, t - q, t).astype(np.uint64)
+    return out
+
+
+def folded_output(slots: np.ndarray, plan: Plan, p: int, d_out: int) -> np.ndarray:
+    """Reads the complete dot products of a ciphertext folded by fold_in_ciphertext: slot (0, kappa, 0)."""
+    D, tau = plan.D, plan.tau
+    part = np.asarray(slots).real[:D * tau:tau]
     rows = min(D, d_out - p * D)
     return part[:rows]
 

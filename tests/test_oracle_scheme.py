@@ -229,3 +229,45 @@ def test_end_to_end_tiny_config():
     x = wl.gen_activation(0, "tiny", 64)
     err = run_linear(par, plan, W, x, 0, 1e-2)
     assert err < 1e-6      # the stated tolerance is 1e-2; a scale-bookkeeping slip would sit near 1e-5
+
+
+# ------------------------------------------------------------------ in-ciphertext fold of the tau partial sums
+
+def test_fold_in_ciphertext_sums_each_group_of_tau_slots(ring64):
+    # expected values come straight from the slot vector: slot kappa*tau of the folded ciphertext must
+    # hold z[kappa*tau] + ... + z[kappa*tau + tau - 1]
+    par, s = ring64
+    plan = Plan(8, 4, 2, 1)                 # n = 32 slots = D * tau
+    rng = np.random.default_rng(21)
+    z = rng.normal(size=par.n)
+    ct = ckks.encrypt(par, s, ckks.encode_coeffs(z, par.N, par.scale), 22)
+    keys = {ckks.galois_element(t, par.N): ckks.galois_key(par, s, ckks.galois_element(t, par.N), 23)
+            for t in ckks.fold_rotations(plan)}
+    assert ckks.fold_rotations(plan) == [1, 2]
+    folded = ckks.fold_in_ciphertext(par, plan, ct, keys)
+    slots = ckks.decode(ckks.decrypt(par, s, folded), par.N, par.scale)
+    expect = z.reshape(plan.D, plan.tau).sum(axis=1)
+    assert np.abs(ckks.folded_output(slots, plan, 0, plan.D) - expect).max() < 1e-8
+    # tau = 1: nothing to fold
+    assert ckks.fold_rotations(Plan(32, 1, 2, 2)) == []
+    assert np.array_equal(ckks.fold_in_ciphertext(par, Plan(32, 1, 2, 2), ct, {}), ct)
+
+
+def test_linear_then_fold_in_ciphertext_gives_the_product():
+    N = 256
+    primes, P = ckks.prime_chain(N, 2)
+    par = Params(N, primes, P, 2.0 ** 40)
+    plan = Plan(16, 4, 2, 2)
+    W = wl.gen_weights(3, "f", 37, 41)
+    x = wl.gen_activation(3, "f", 41)
+    s = ckks.keygen(par, 3)
+    keys = ckks.make_rotation_keys(par, s, plan, 3, extra_steps=ckks.fold_rotations(plan))
+    cts = ckks.encrypt_vector(par, plan, s, x, 3)
+    out = ckks.linear(par, plan, cts, W, keys)
+    y = np.zeros(37)
+    out_scale = par.scale * par.scale / par.primes[-1]
+    for p, ct in out.items():
+        low = ckks.rescale(par, ckks.fold_in_ciphertext(par, plan, ct, keys))
+        part = ckks.folded_output(ckks.decode(ckks.decrypt(par, s, low), par.N, out_scale), plan, p, 37)
+        y[p * plan.D:p * plan.D + len(part)] = part
+    assert np.abs(y - W.astype(np.float64) @ x).max() < 1e-6
