@@ -131,12 +131,12 @@ def butterflies_per_step(runner) -> dict:
     return {"fwd": summary(fwd), "inv": summary(inv), "per_poly": per}
 
 
-def time_extra_workload(name: str, steps: int, cache_budget_bytes=None) -> dict:
+def time_extra_workload(name: str, steps: int, cache_budget_bytes=None, fold_in_ciphertext=False) -> dict:
     """ms per decode token of another workload (device-resident inputs), with the weight stream's rate."""
     import torch
     from paper_2606_17421_b200 import bifrost as bf
     from paper_2606_17421_b200.runner import WorkloadRunner
-    R = WorkloadRunner(name, cache_budget_bytes=cache_budget_bytes)
+    R = WorkloadRunner(name, cache_budget_bytes=cache_budget_bytes, fold_in_ciphertext=fold_in_ciphertext)
     for _ in range(3):
         R.step()
     torch.cuda.synchronize()
@@ -342,6 +342,9 @@ def run_ours(args):
             elif name == "llama3_layer":
                 extras[name + "@cached"] = time_extra_workload(name, 5)
                 extras[name + "@on_the_fly"] = time_extra_workload(name, 3, cache_budget_bytes=1)
+            elif name == "gpt2_qkv@fold_in_ciphertext":
+                # the variant that sums the tau partial results on the device (log2 tau more key switches)
+                extras[name] = time_extra_workload("gpt2_qkv", 50, fold_in_ciphertext=True)
             else:
                 extras[name] = time_extra_workload(name, 10)
         line["other_workloads"] = extras
@@ -524,7 +527,8 @@ def main():
     if args.extra == "all":
         args.extra = "gpt2_step,qwen3_step,llama3_layer"
     elif args.extra == "tiles":     # tile-size study and the paper's own parameter set
-        args.extra = "gemm1024_D1024,gemm1024_D512,gemm1024_D256,gemm1024_D128,gpt2_qkv_paper_params"
+        args.extra = ("gemm1024_D1024,gemm1024_D512,gemm1024_D256,gemm1024_D128,gpt2_qkv_paper_params,"
+                      "gpt2_qkv@fold_in_ciphertext")
     if args.impl == "reference":
         run_reference(args)
     else:

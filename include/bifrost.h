@@ -138,6 +138,17 @@ int bf_set_lanes(bf_ctx* ctx, int n_lanes);
 int bf_rescale(bf_ctx* ctx, const uint64_t* ct_in, uint64_t* ct_out, uint32_t n_ct, uint32_t level,
                double* scale_inout);
 
+/* In-ciphertext fold of the tau partial sums (a variant of the output stage; the packing of Sec. 4.2
+ * leaves slot (rho, kappa, c) of an output ciphertext with the partial dot product of row kappa over
+ * column class c, and by default the caller adds the tau of them after decryption):
+ *     for i = 0 .. log2(tau) - 1:  ct <- ct + rot(ct, 2^i)
+ * after which slot (0, kappa, 0) holds the complete dot product.  In place on n_ct full-level
+ * ciphertexts (device, boundary layout); level and scale are unchanged, so bf_rescale follows as
+ * usual.  Needs the rotation keys for 1, 2, ..., tau/2 slots (MISSING_KEY otherwise) and a
+ * power-of-two tau (INVALID_ARG otherwise); costs log2(tau) key switches per ciphertext.
+ * Asynchronous. */
+int bf_fold(bf_ctx* ctx, uint64_t* ct, uint32_t n_ct);
+
 /* bf_linear followed by bf_rescale with HOST buffers: copies n_in ciphertexts from host_ct_in to
  * the device, runs the layer, rescales once and copies the n_out ciphertexts of level r-1 back to
  * host_ct_out ([n_out][2][r-1][N]).  Pinned host memory makes the copies asynchronous; the call

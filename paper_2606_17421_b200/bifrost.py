@@ -57,6 +57,7 @@ _SIGNATURES = {
     "bf_set_dependent_launch": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_set_lanes": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_rescale": (ctypes.c_int, [_vp, _vp, _vp, _u32, _u32, ctypes.POINTER(ctypes.c_double)]),
+    "bf_fold": (ctypes.c_int, [_vp, _vp, _u32]),
     "bf_linear_host": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
     "bf_rotate": (ctypes.c_int, [_vp, _vp, _u32, _vp]),
     "bf_negacyclic_mul": (ctypes.c_int, [_vp, _vp, _vp, _vp, _u32]),
@@ -196,6 +197,11 @@ def bf_linear_host(ctx, host_ct_in, n_in: int, pt_weights, W_raw, d_out: int, d_
 
 def bf_rotate(ctx, ct_in, steps: int, ct_out):
     _check(load().bf_rotate(ctx, _ptr(ct_in), steps, _ptr(ct_out)), "bf_rotate", ctx)
+
+
+def bf_fold(ctx, ct, n_ct: int):
+    """Sums the tau partial results inside n_ct full-level ciphertexts, in place."""
+    _check(load().bf_fold(ctx, _ptr(ct), n_ct), "bf_fold", ctx)
 
 
 def bf_negacyclic_mul(ctx, a, b, out, n_polys: int):

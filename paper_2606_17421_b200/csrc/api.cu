@@ -1100,6 +1100,74 @@ extern "C" int bf_rotate(bf_ctx* ctx, const uint64_t* ct_in, uint32_t steps, uin
     return BF_OK;
 }
 
+// In-ciphertext fold of the tau partial sums: ct <- ct + rot(ct, 2^i) for i = 0 .. log2(tau) - 1, batched
+// over the ciphertexts.  Every round is one key switch per ciphertext: transform, hoisted ModUp of c1, inner
+// product with the key of 2^i, division by P with the automorphism as a scatter, then the sum of the
+// ciphertext and its rotation goes back to the coefficient domain (the next round decomposes its c1 again).
+extern "C" int bf_fold(bf_ctx* ctx, uint64_t* ct, uint32_t n_ct) {
+    if (!ctx || !ct || !n_ct) return BF_ERR_INVALID_ARG;
+    const u32 N = ctx->N, r = ctx->r, tau = ctx->plan.tau;
+    if (tau & (tau - 1)) return BF_ERR_INVALID_ARG;
+    const size_t ctw = (size_t)2 * r * N;
+    std::vector<int> keys;
+    for (u32 steps = 1; steps < tau; steps <<= 1) {
+        int key = -1;
+        TRY(find_key(ctx, steps, &key));
+        keys.push_back(key);
+    }
+    if (keys.empty()) return BF_OK;
+    u32 batch = giant_batch(ctx);
+    if (batch > n_ct) batch = n_ct;
+    TRY(ensure(ctx, ctx->X, (size_t)batch * 2 * ctw * 8));
+    TRY(ensure_rot_scratch(ctx, batch, batch));
+    u64* X = (u64*)ctx->X.p;                             // [t][0] = NTT(ct_t), [t][1] = its rotation
+    const Lane lane = main_lane(ctx);
+    for (u32 t0 = 0; t0 < n_ct; t0 += batch) {
+        const u32 cnt = (n_ct - t0 < batch) ? n_ct - t0 : batch;
+        u64* cts = ct + (size_t)t0 * ctw;
+        for (int key : keys) {
+            PolyBatch B;
+            memset(&B, 0, sizeof(B));
+            B.src = cts;
+            B.dst = X;
+            B.src_so = (long long)ctw;
+            B.dst_so = (long long)2 * ctw;
+            B.src_sm = B.dst_sm = N;
+            B.n_m = 2 * r;
+            B.mod_wrap = r;
+            B.mod_step = 1;
+            CK(ntt_forward(ctx->ring, B, cnt, LOAD_PLAIN, ctx->stream));
+            TRY(modup(ctx, ctx->stream, cts + (size_t)r * N, (long long)ctw, cnt, lane.Dig, X + (size_t)r * N,
+                      (long long)2 * ctw));
+            RotBatch rb;
+            memset(&rb, 0, sizeof(rb));
+            rb.n = (int)cnt;
+            for (u32 t = 0; t < cnt; ++t) {
+                rb.key[t] = key;
+                rb.dig[t] = (int)t;
+                rb.c0[t] = (int)(2 * t);
+                rb.out[t] = (int)(2 * t + 1);
+            }
+            CK(launch_key_inner_product(ctx->ring, rb, lane.Dig, ctx->keys, lane.U, ctx->device_error, ctx->stream));
+            TRY(moddown_batch(ctx, lane, rb, X, (long long)ctw, X, (long long)ctw));
+            memset(&B, 0, sizeof(B));
+            B.src = X;
+            B.dst = cts;
+            B.src_so = (long long)2 * ctw;
+            B.dst_so = (long long)ctw;
+            B.src_sm = B.dst_sm = N;
+            B.n_m = 2 * r;
+            B.mod_wrap = r;
+            B.mod_step = 1;
+            B.sum_src = X + ctw;
+            B.sum_terms = 1;
+            B.sum_stride = 0;
+            CK(ntt_inverse(ctx->ring, B, cnt, ctx->stream));
+        }
+    }
+    return BF_OK;
+}
+
 extern "C" int bf_negacyclic_mul(bf_ctx* ctx, const uint64_t* a, const uint64_t* b, uint64_t* out, uint32_t n_polys) {
     if (!ctx || !a || !b || !out || !n_polys) return BF_ERR_INVALID_ARG;
     const u32 N = ctx->N, nb = ctx->r + 1;

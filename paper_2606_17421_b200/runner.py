@@ -28,7 +28,7 @@ class WorkloadRunner:
 
     def __init__(self, name: str, seed: int = 0, device: str = "cuda:0", cache: bool = True,
                  cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None,
-                 fuse_shared_inputs: bool = True):
+                 fuse_shared_inputs: bool = True, fold_in_ciphertext: bool = False):
         self.w = wl.WORKLOADS[name]
         ps = wl.PARAM_SETS[self.w.params]
         self.N, self.primes, self.P, self.scale = ps["N"], list(ps["primes"]), ps["special"], ps["scale"]
@@ -51,6 +51,9 @@ class WorkloadRunner:
         # rotation keys: uniform residues over the extended basis
         steps = [k * self.plan.tau for k in range(1, self.plan.b)] + \
                 [j * self.plan.b * self.plan.tau for j in range(1, self.plan.g)]
+        self.fold_in_ciphertext = fold_in_ciphertext
+        if fold_in_ciphertext:      # the variant that sums the tau partial results on the device
+            steps += [1 << i for i in range(self.plan.tau.bit_length() - 1)]
         n = self.N // 2
         self.rot_steps = sorted({s % n for s in steps if s % n})
         basis = self.primes + [self.P]
@@ -97,6 +100,8 @@ class WorkloadRunner:
             L = e["layer"]
             bf.bf_linear(self.ctx, e["ct_in"], e["n_in"], e["handle"], None if e["handle"] else e["W"],
                          L.d_out, L.d_in, e["ct_out"], e["n_out"])
+            if self.fold_in_ciphertext:
+                bf.bf_fold(self.ctx, e["ct_out"], e["n_out"])
             bf.bf_rescale(self.ctx, e["ct_out"], e["ct_low"], e["n_out"], self.r)
 
     def make_host_buffers(self):

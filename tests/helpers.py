@@ -48,9 +48,9 @@ class GpuSide:
     def empty_u64(self, *shape):
         return self.torch.empty(shape, dtype=self.torch.int64, device=self.dev)
 
-    def load_keys(self, keys: dict):
+    def load_keys(self, keys: dict, extra_steps=()):
         """keys: {galois element: array [r][2][r+1][N]} from the oracle, plus the rotation amounts."""
-        steps = ckks.required_rotations(self.plan)
+        steps = list(ckks.required_rotations(self.plan)) + list(extra_steps)
         uniq = []
         for s in steps:
             if s % self.par.n and s % self.par.n not in uniq:

@@ -345,6 +345,55 @@ def test_repeated_calls_replay_a_graph_and_still_read_fresh_inputs():
         g.close()
 
 
+@pytest.mark.parametrize("pkey,plan_t,shape", [
+    ("n12", (64, 4, 4, 4), (100, 130)),          # tau = 4: rotations by 1 and 2, two output ciphertexts
+    ("n12", (32, 32, 1, 1), (70, 50)),           # tau = 32, no other rotation in the plan, three outputs
+    ("n15", (1024, 16, 16, 4), (1100, 300)),     # the headline plan: rotations by 1, 2, 4, 8
+])
+def test_fold_in_ciphertext_matches_oracle(pkey, plan_t, shape):
+    par = oracle_params(pkey)
+    plan = ckks.Plan(*plan_t)
+    d_out, d_in = shape
+    s = ckks.keygen(par, 41)
+    fold_steps = ckks.fold_rotations(plan)
+    keys = ckks.make_rotation_keys(par, s, plan, 41, extra_steps=fold_steps)
+    W = wl.gen_weights(41, "fold", d_out, d_in)
+    x = wl.gen_activation(41, "fold", d_in)
+    cts = ckks.encrypt_vector(par, plan, s, x, 41)
+    n_out = -(-d_out // plan.D)
+    lin = ckks.linear(par, plan, cts, W, keys)
+    expect = [ckks.fold_in_ciphertext(par, plan, lin[p], keys) for p in range(n_out)]
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys, extra_steps=fold_steps)
+        out = g.linear(cts, W, d_out, d_in, weights=g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in))
+        g.bf.bf_fold(g.ctx, out, n_out)
+        got = g.to_host_u64(out)
+        for p in range(n_out):
+            assert np.array_equal(got[p], expect[p]), p
+        # rescale, decrypt: slot (0, kappa, 0) is the complete dot product
+        low = g.empty_u64(n_out, 2, par.r - 1, par.N)
+        scale = g.bf.bf_rescale(g.ctx, out, low, n_out, par.r, par.scale * par.scale)
+        low = g.to_host_u64(low)
+        y = np.zeros(d_out)
+        for p in range(n_out):
+            part = ckks.folded_output(ckks.decode(ckks.decrypt(par, s, low[p]), par.N, scale), plan, p, d_out)
+            y[p * plan.D:p * plan.D + len(part)] = part
+        assert np.abs(y - W.astype(np.float64) @ x).max() < 1e-3
+        # without the keys of the fold the call is refused before anything is launched
+        g2 = GpuSide(par, plan)
+        try:
+            g2.load_keys(keys)
+            if fold_steps and not set(fold_steps) <= set(ckks.required_rotations(plan)):
+                with pytest.raises(g2.bf.BifrostError) as ei:
+                    g2.bf.bf_fold(g2.ctx, out, n_out)
+                assert ei.value.code == g2.bf.BF_ERR_MISSING_KEY
+        finally:
+            g2.close()
+    finally:
+        g.close()
+
+
 def test_stacking_projections_that_share_an_input_changes_no_residue():
     # q/k/v (or gate/up) read the same activation: one call over the row-stacked matrix must give
     # exactly the ciphertexts of the separate calls
