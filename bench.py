@@ -131,12 +131,14 @@ def butterflies_per_step(runner) -> dict:
     return {"fwd": summary(fwd), "inv": summary(inv), "per_poly": per}
 
 
-def time_extra_workload(name: str, steps: int, cache_budget_bytes=None, fold_in_ciphertext=False) -> dict:
+def time_extra_workload(name: str, steps: int, cache_budget_bytes=None, fold_in_ciphertext=False,
+                        compact_cache=False) -> dict:
     """ms per decode token of another workload (device-resident inputs), with the weight stream's rate."""
     import torch
     from paper_2606_17421_b200 import bifrost as bf
     from paper_2606_17421_b200.runner import WorkloadRunner
-    R = WorkloadRunner(name, cache_budget_bytes=cache_budget_bytes, fold_in_ciphertext=fold_in_ciphertext)
+    R = WorkloadRunner(name, cache_budget_bytes=cache_budget_bytes, fold_in_ciphertext=fold_in_ciphertext,
+                       compact_cache=compact_cache)
     for _ in range(3):
         R.step()
     torch.cuda.synchronize()
@@ -339,6 +341,9 @@ def run_ours(args):
                 part["fallback_share_of_step"] = round(1.0 - full["ms_per_token"] / part["ms_per_token"], 4)
                 extras[name + "@60GB"] = full
                 extras[name + "@40.5GB"] = part
+                # the same budget with the compact cache format: every layer fits, nothing falls back
+                extras[name + "@40.5GB_compact_cache"] = time_extra_workload(name, 5, cache_budget_bytes=int(40.5 * 10 ** 9),
+                                                                             compact_cache=True)
             elif name == "llama3_layer":
                 extras[name + "@cached"] = time_extra_workload(name, 5)
                 extras[name + "@on_the_fly"] = time_extra_workload(name, 3, cache_budget_bytes=1)

@@ -107,6 +107,16 @@ void bf_weights_free(bf_ctx* ctx, bf_weights* w);
 int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
               const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out);
 
+/* Cache compression (Sec. 6.1 names the encoded-weight cache as the memory wall).  With
+ * bf_set_compact_cache(ctx, 1) every weight encoded afterwards, cached or on the fallback path, is
+ * held in the narrowest word format its prime allows: 4 bytes per word for primes below 2^32, 5
+ * (low 32 bits and high bytes stored apart) below 2^40, 8 otherwise, instead of 8 throughout: with a
+ * 50-bit and six 40-bit primes 38 of 56 bytes, i.e. 68 % of the resident size and of the
+ * multiply-accumulate's HBM stream.  Results are identical; handles of both kinds can be used side by
+ * side.  Default: off (the multiply-accumulate is no faster for it on B200, see the design notes;
+ * the gain is capacity).  bf_weights_bytes reports sizes for the current setting. */
+int bf_set_compact_cache(bf_ctx* ctx, int on);
+
 /* bf_linear replays a captured CUDA graph of its launch sequence from the third call with the same
  * (ct_in, pt_weights, ct_out, d_out, d_in) on: the first call runs directly (and sizes the scratch),
  * the second is captured.  Replay is skipped on the fallback path, while stage or kernel timing is

@@ -486,7 +486,7 @@ extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t
     if (!ctx) return 0;
     const u32 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = cdiv(d_out, ctx->plan.tile_D);
     const TileLayout lay = mac_tile_layout(ctx->ring, n_out * ctx->plan.bsgs_g, n_in * ctx->plan.bsgs_b);
-    return mac_tile_words(ctx->ring, lay) * sizeof(u64);
+    return mac_tile_bytes(ctx->ring, lay);
 }
 
 // Encode diagonals [d0, d0 + count) of W (order [j][p][q][k], i.e. group pj = d / n_terms, term d % n_terms)
@@ -855,7 +855,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
         if (groups < 1) groups = 1;
         if (groups > n_pj) groups = n_pj;
         const TileLayout jl = mac_tile_layout(ctx->ring, groups, n_terms);
-        TRY(ensure(ctx, ctx->ptjit, mac_tile_words(ctx->ring, jl) * 8));
+        TRY(ensure(ctx, ctx->ptjit, mac_tile_bytes(ctx->ring, jl)));
         for (u32 pj0 = 0; pj0 < n_pj; pj0 += groups) {
             const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
             const TileLayout cl = mac_tile_layout(ctx->ring, cnt, n_terms);
@@ -1013,6 +1013,12 @@ extern "C" int bf_set_graph_replay(bf_ctx* ctx, int on) {
     if (!ctx) return BF_ERR_INVALID_ARG;
     ctx->use_graphs = on ? 1 : 0;
     if (!on) destroy_graphs(ctx);
+    return BF_OK;
+}
+
+extern "C" int bf_set_compact_cache(bf_ctx* ctx, int on) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    ctx->ring.compact_cache = on != 0;     // weights encoded from now on (and the fallback path's scratch) use it
     return BF_OK;
 }
 

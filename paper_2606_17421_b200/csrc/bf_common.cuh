@@ -236,23 +236,39 @@ struct ModDownEpilogue {
 };
 
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks
-// each stream one contiguous region:  word (group pj, term t, prime i, coefficient n) lives at
-//   (((((i*ntiles + n/TN)*G + pj/PL)*C + t/TS)*PL + pj%PL)*TS + t%TS)*TN + n%TN
+// each stream one contiguous region:  word (group pj, term t, prime i, coefficient n) has index
+//   ((pj%PL)*TS + t%TS)*TN + n%TN   inside stage   ((i, n/TN), pj/PL, t/TS)
 // with TN = 2^log_tn coefficients per tile, PL = 256/TN group lanes, TS = 8 terms per stage,
-// G = ceil(n_pj/PL), C = ceil(n_terms/TS).  One stage (fixed i, tile, pj/PL, t/TS) is 16 KB.
+// G = ceil(n_pj/PL), C = ceil(n_terms/TS); a stage holds 2048 words.  The stages of one prime are
+// contiguous, ordered (tile, pj/PL, t/TS), and every prime stores its words in the narrowest of three
+// formats its size allows, because the kernel that reads them is bound by HBM bytes:
+//   TILE_W64  8 bytes per word (16 KB per stage)
+//   TILE_W40  primes below 2^40: the low 32 bits of all 2048 words, then their high bytes (10 KB per stage)
+//   TILE_W32  primes below 2^32: 32-bit words (8 KB per stage)
+enum TileFormat : u32 { TILE_W64 = 0, TILE_W40 = 1, TILE_W32 = 2 };
 struct TileLayout {
     u32 log_tn, n_terms, n_pj, G, C, ntiles;
+    u32 fmt[MAX_MODULI];                    // TileFormat of every ciphertext prime
+    unsigned long long base[MAX_MODULI];    // byte offset of the prime's first stage; base[r] = total bytes
 };
 constexpr u32 TILE_TS = 8;
 constexpr u32 TILE_STAGE_WORDS = 2048;
 
-__host__ __device__ __forceinline__ size_t tile_stage_offset(const TileLayout& t, u32 i, u32 tile, u32 g, u32 ch) {
-    return ((((size_t)i * t.ntiles + tile) * t.G + g) * t.C + ch) * TILE_STAGE_WORDS;
+__host__ __device__ __forceinline__ u32 tile_stage_bytes(u32 fmt) {
+    return TILE_STAGE_WORDS * (fmt == TILE_W64 ? 8u : fmt == TILE_W40 ? 5u : 4u);
 }
-__host__ __device__ __forceinline__ size_t tile_word_offset(const TileLayout& t, u32 pj, u32 term, u32 i, u32 n) {
+// byte offset of a stage
+__host__ __device__ __forceinline__ size_t tile_stage_offset(const TileLayout& t, u32 i, u32 tile, u32 g, u32 ch) {
+    return (size_t)t.base[i] + (((size_t)tile * t.G + g) * t.C + ch) * tile_stage_bytes(t.fmt[i]);
+}
+// index of a word inside its stage
+__host__ __device__ __forceinline__ u32 tile_word_index(const TileLayout& t, u32 pj, u32 term, u32 n) {
     const u32 TN = 1u << t.log_tn, PL = 256u >> t.log_tn;
-    return tile_stage_offset(t, i, n >> t.log_tn, pj / PL, term / TILE_TS) +
-           ((size_t)(pj % PL) * TILE_TS + term % TILE_TS) * TN + (n & (TN - 1));
+    return ((pj % PL) * TILE_TS + term % TILE_TS) * TN + (n & (TN - 1));
+}
+__host__ __device__ __forceinline__ size_t tile_stage_of_word(const TileLayout& t, u32 pj, u32 term, u32 i, u32 n) {
+    const u32 PL = 256u >> t.log_tn;
+    return tile_stage_offset(t, i, n >> t.log_tn, pj / PL, term / TILE_TS);
 }
 
 // A batch of equally sized polynomials addressed as (outer index o, slot m):

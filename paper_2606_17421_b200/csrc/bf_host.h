@@ -44,6 +44,7 @@ struct RingHost {
     std::vector<u64> q;               // q_0..q_L, then P
     Profiler* prof = nullptr;
     bool dependent_launch = true;     // launch the kernels of a call with programmatic stream serialisation
+    bool compact_cache = false;       // encode plaintexts in the narrowest word format each prime allows
 };
 
 // Launch with programmatic stream serialisation: the grid may be scheduled while the previous kernel
@@ -84,7 +85,7 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
                                      int* error_flag, cudaStream_t stream);
 u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintext format (0 = whole words)
 TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms);   // layout of n_pj groups of n_terms diagonals
-size_t mac_tile_words(const RingHost& ring, const TileLayout& t);           // words that layout occupies
+size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t);           // bytes that layout occupies
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
                        u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream);
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,

@@ -4,6 +4,8 @@
 // product, the division by the special prime, the giant-step sum and the rescale (Sec. 2.1).
 #include "bf_host.h"
 
+#include <cstring>
+
 namespace bf {
 
 // ------------------------------------------------------------------------------------------------
@@ -103,8 +105,11 @@ __device__ __forceinline__ void mbar_arrive(u64* bar) {
 constexpr int MAC_CONSUMERS = 256;
 constexpr int MAC_THREADS = MAC_CONSUMERS + 32;   // + one producer warp
 constexpr int MAC_TS = (int)TILE_TS;              // terms per stage
-constexpr int MAC_STAGES = 2;
-constexpr int MAC_STAGE_WORDS = MAC_TS * MAC_CONSUMERS;   // 16 KB per stage whatever TN is
+constexpr int MAC_STAGES = 2;                             // (measured: three narrower stages in the same ring are slower)
+constexpr int MAC_STAGE_WORDS = MAC_TS * MAC_CONSUMERS;   // 2048 words per stage whatever TN is
+constexpr int MAC_SLOT_BYTES = MAC_STAGE_WORDS * 8;       // ring slot: room for the widest word format
+constexpr int MAC_RING_BYTES = MAC_STAGES * MAC_SLOT_BYTES;
+constexpr int MAC_MAX_STAGES = MAC_STAGES;
 constexpr u32 KARA_L = 25;
 
 template <bool KARA, int LOG_TN>
@@ -115,11 +120,11 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
     extern __shared__ __align__(128) unsigned char mac_smem[];
     asm volatile("griddepcontrol.launch_dependents;");
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
-    u64* ring = (u64*)mac_smem;                                    // [MAC_STAGES][PL][MAC_TS][TN]
-    u64* xs = ring + MAC_STAGES * MAC_STAGE_WORDS;                 // [n_terms][2][TN]
-    u64* full = xs + (size_t)n_terms * 2 * TN;                     // [MAC_STAGES]
-    u64* empty = full + MAC_STAGES;                                // [MAC_STAGES]
-    u64* xbar = empty + MAC_STAGES;
+    unsigned char* ring = mac_smem;                                // [stages][stage bytes of this block's prime]
+    u64* xs = (u64*)(mac_smem + MAC_RING_BYTES);                   // [n_terms][2][TN]
+    u64* full = xs + (size_t)n_terms * 2 * TN;                     // [MAC_MAX_STAGES]
+    u64* empty = full + MAC_MAX_STAGES;                            // [MAC_MAX_STAGES]
+    u64* xbar = empty + MAC_MAX_STAGES;
     // Work units (tile, prime, slice of the output groups) are numbered tile-fastest.  The first n_whole
     // blocks take one unit each; the units after them (the part that would be a thin last wave) are each
     // cut into tail_split blocks over their output groups, so that the last wave is short instead.
@@ -143,12 +148,15 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         pj_end = min(pj_end, pj_begin + per);
         if (pj_begin >= pj_end) return;                            // (uniform for the block)
     }
+    const u32 fmt = lay.fmt[i];                                    // this prime's word format decides the stage size
+    const u32 stage_bytes = tile_stage_bytes(fmt);
+    constexpr u32 n_stages = MAC_STAGES;
     const u32 n_groups = (pj_end - pj_begin + PL - 1) / PL;        // rounds of PL output groups
     const u32 n_chunks = (n_terms + MAC_TS - 1) / MAC_TS;
     const u32 n_items = n_groups * n_chunks;
 
     if (tid == 0) {
-        for (int s = 0; s < MAC_STAGES; ++s) {
+        for (int s = 0; s < MAC_MAX_STAGES; ++s) {
             mbar_init(&full[s], 1);                                // the producer's arrive.expect_tx
             mbar_init(&empty[s], MAC_CONSUMERS / 32);              // one arrival per consumer warp
         }
@@ -164,26 +172,33 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         u32 g = 0, ch = 0, slot = 0, phase = 0, k = 0;
         // one stage of the weight stream: a contiguous 16 KB block of the tile-major layout; when its tail
         // is padding (last group round or last term chunk) copy the valid part of every lane only
+        const u32 word_lo = fmt == TILE_W64 ? 8u : 4u;                 // bytes per word of the stage's first part
+        const u32 hi_at = TILE_STAGE_WORDS * 4u;                       // TILE_W40: where the high bytes start
         auto issue_stage = [&]() {
             const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
             const u32 first = pj_begin + g * PL;
             const u32 lanes = min((u32)PL, pj_end - first);
-            const u64* stage = pt + tile_stage_offset(lay, i, tile_x, first / PL, ch);
-            u64* sdst = ring + (size_t)slot * MAC_STAGE_WORDS;
-            if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * 8);
+            const unsigned char* stage = (const unsigned char*)pt + tile_stage_offset(lay, i, tile_x, first / PL, ch);
+            unsigned char* sdst = ring + (size_t)slot * MAC_SLOT_BYTES;
+            const u32 bytes_per_word = fmt == TILE_W64 ? 8u : fmt == TILE_W40 ? 5u : 4u;
+            if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * bytes_per_word);
             __syncwarp();
             if (lanes == PL && cnt == (u32)MAC_TS) {
-                if (lane == 0) bulk_g2s_stream(sdst, stage, MAC_STAGE_WORDS * 8, &full[slot], stream_policy);
+                if (lane == 0) bulk_g2s_stream(sdst, stage, stage_bytes, &full[slot], stream_policy);
             } else if (lane < lanes) {
-                bulk_g2s_stream(sdst + (size_t)lane * MAC_TS * TN, stage + (size_t)lane * MAC_TS * TN, cnt * TN * 8,
-                                &full[slot], stream_policy);
+                // the valid part of every lane: cnt terms of TN words (and their high bytes)
+                const u32 at = lane * MAC_TS * TN;
+                bulk_g2s_stream(sdst + (size_t)at * word_lo, stage + (size_t)at * word_lo, cnt * TN * word_lo, &full[slot],
+                                stream_policy);
+                if (fmt == TILE_W40)
+                    bulk_g2s_stream(sdst + hi_at + at, stage + hi_at + at, cnt * TN, &full[slot], stream_policy);
             }
             if (++ch == n_chunks) { ch = 0; ++g; }
-            if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
+            if (++slot == n_stages) { slot = 0; phase ^= 1; }
             ++k;
         };
         // cached weights do not depend on the previous kernel: fill the ring before waiting for it
-        const u32 early = early_weights ? min(n_items, (u32)MAC_STAGES) : 0u;
+        const u32 early = early_weights ? min(n_items, n_stages) : 0u;
         while (k < early) issue_stage();
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if (lane == 0) mbar_expect_tx(xbar, n_terms * 2 * TN * 8);
@@ -191,7 +206,7 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         for (u32 e = lane; e < n_terms * 2; e += 32)                // X tile: [term][component] segments
             bulk_g2s(xs + (size_t)e * TN, x + ((size_t)e * r + i) * N + n0, TN * 8, xbar);
         while (k < n_items) {
-            if (k >= (u32)MAC_STAGES) mbar_wait(&empty[slot], phase ^ 1, error_flag);   // consumers left this slot
+            if (k >= n_stages) mbar_wait(&empty[slot], phase ^ 1, error_flag);   // consumers left this slot
             issue_stage();
         }
         return;
@@ -216,32 +231,54 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
         mbar_wait(&full[slot], phase, error_flag);
         if (pj < pj_end) {
-            const u64* ps = ring + (size_t)slot * MAC_STAGE_WORDS + (size_t)l * MAC_TS * TN + c;
+            const unsigned char* sbase = ring + (size_t)slot * MAC_SLOT_BYTES;
+            const u32 at = l * MAC_TS * TN + c;                        // index of this thread's first word of the stage
             const u64* xt = xs + (size_t)t0 * 2 * TN + c;
-            if (cnt == MAC_TS) {
+            // one streamed word times both components of its X word
+            auto mac_word = [&](u64 w, u32 w0, u32 w1, u32 ts) {
+                if (KARA) {
+                    const u32 ws = w0 + w1;
+                    k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
+                    k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
+                } else {
+                    a0.mac(w, xt[(ts * 2) * TN]);
+                    a1.mac(w, xt[(ts * 2 + 1) * TN]);
+                }
+            };
+            if (fmt == TILE_W64) {              // whole words; limbs already split when KARA
+                const u64* ps = (const u64*)sbase + at;
+                if (cnt == MAC_TS) {
 #pragma unroll
-                for (int ts = 0; ts < MAC_TS; ++ts) {
-                    const u64 w = ps[ts * TN];
-                    if (KARA) {
-                        const u32 w0 = (u32)w, w1 = (u32)(w >> 32), ws = w0 + w1;
-                        k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
-                        k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
-                    } else {
-                        a0.mac(w, xt[(ts * 2) * TN]);
-                        a1.mac(w, xt[(ts * 2 + 1) * TN]);
+                    for (int ts = 0; ts < MAC_TS; ++ts) {
+                        const u64 w = ps[ts * TN];
+                        mac_word(w, (u32)w, (u32)(w >> 32), ts);
+                    }
+                } else {
+                    for (u32 ts = 0; ts < cnt; ++ts) {
+                        const u64 w = ps[ts * TN];
+                        mac_word(w, (u32)w, (u32)(w >> 32), ts);
                     }
                 }
-            } else {
-                for (u32 ts = 0; ts < cnt; ++ts) {
-                    const u64 w = ps[ts * TN];
-                    if (KARA) {
-                        const u32 w0 = (u32)w, w1 = (u32)(w >> 32), ws = w0 + w1;
-                        k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
-                        k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
-                    } else {
-                        a0.mac(w, xt[(ts * 2) * TN]);
-                        a1.mac(w, xt[(ts * 2 + 1) * TN]);
+            } else if (fmt == TILE_W40) {       // low 32 bits and high byte, limbs cut here
+                const u32* pl = (const u32*)sbase + at;
+                const unsigned char* ph = sbase + TILE_STAGE_WORDS * 4u + at;
+                if (cnt == MAC_TS) {
+#pragma unroll
+                    for (int ts = 0; ts < MAC_TS; ++ts) {
+                        const u32 lo = pl[ts * TN], hi = ph[ts * TN];
+                        mac_word(((u64)hi << 32) | lo, lo & ((1u << KARA_L) - 1), (lo >> KARA_L) | (hi << (32 - KARA_L)), ts);
                     }
+                } else {
+                    for (u32 ts = 0; ts < cnt; ++ts) {
+                        const u32 lo = pl[ts * TN], hi = ph[ts * TN];
+                        mac_word(((u64)hi << 32) | lo, lo & ((1u << KARA_L) - 1), (lo >> KARA_L) | (hi << (32 - KARA_L)), ts);
+                    }
+                }
+            } else {                            // 32-bit words
+                const u32* pl = (const u32*)sbase + at;
+                for (u32 ts = 0; ts < cnt; ++ts) {
+                    const u32 lo = pl[ts * TN];
+                    mac_word((u64)lo, lo & ((1u << KARA_L) - 1), lo >> KARA_L, ts);
                 }
             }
         }
@@ -273,7 +310,7 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
             }
         }
         if (++ch == n_chunks) { ch = 0; ++g; }
-        if (++slot == MAC_STAGES) { slot = 0; phase ^= 1; }
+        if (++slot == n_stages) { slot = 0; phase ^= 1; }
     }
 }
 
@@ -292,6 +329,7 @@ static u32 mac_log_tn(u32 n_terms) {
 
 TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms) {
     TileLayout t;
+    memset(&t, 0, sizeof(t));
     t.log_tn = mac_log_tn(n_terms);
     const u32 PL = 256u >> t.log_tn;
     t.n_terms = n_terms;
@@ -299,12 +337,18 @@ TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms) {
     t.G = (n_pj + PL - 1) / PL;
     t.C = (n_terms + TILE_TS - 1) / TILE_TS;
     t.ntiles = ring.dev.N >> t.log_tn;
+    unsigned long long at = 0;
+    for (u32 i = 0; i < ring.dev.r; ++i) {
+        t.fmt[i] = !ring.compact_cache ? TILE_W64
+                 : ring.q[i] < (1ull << 32) ? TILE_W32 : ring.q[i] < (1ull << 40) ? TILE_W40 : TILE_W64;
+        t.base[i] = at;
+        at += (unsigned long long)t.ntiles * t.G * t.C * tile_stage_bytes(t.fmt[i]);
+    }
+    t.base[ring.dev.r] = at;
     return t;
 }
 
-size_t mac_tile_words(const RingHost& ring, const TileLayout& t) {
-    return (size_t)ring.dev.r * t.ntiles * t.G * t.C * TILE_STAGE_WORDS;
-}
+size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t) { return (size_t)t.base[ring.dev.r]; }
 
 u32 mac_split_bits(const RingHost& ring) {
     u64 qmax = 0;
@@ -317,7 +361,7 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
                                 u32 n_pj, u32 n_terms, u32 lazy, u32 early_weights, int* error_flag,
                                 cudaStream_t stream) {
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
-    const size_t smem = (size_t)MAC_STAGES * MAC_STAGE_WORDS * 8 + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_STAGES + 1) * 8;
+    const size_t smem = (size_t)MAC_RING_BYTES + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_MAX_STAGES + 1) * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
     static bool attr_set = false;     // opt in once to the large dynamic shared-memory carve-out
     if (!attr_set) {

@@ -574,6 +574,28 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 }
                 continue;
             }
+            if (B.tile_ptr) {   // tile-major plaintext cache; 4 adjacent coefficients never straddle a tile (tiles hold >= 16)
+                const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
+                const u32 n = chunk * LEN + 4 * s;
+                unsigned char* stage = (unsigned char*)B.tile_ptr + tile_stage_of_word(B.tile, pj, term, mod, n);
+                const u32 at = tile_word_index(B.tile, pj, term, n);
+                const u32 fmt = B.tile.fmt[mod];
+                if (fmt == TILE_W64) {
+                    if (B.split_bits) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) v4[i] = limb_split(v4[i], B.split_bits);
+                    }
+                    ulonglong2* gp = (ulonglong2*)(stage + (size_t)at * 8);
+                    gp[0] = make_ulonglong2(v4[0], v4[1]);
+                    gp[1] = make_ulonglong2(v4[2], v4[3]);
+                } else {
+                    *(uint4*)(stage + (size_t)at * 4) = make_uint4((u32)v4[0], (u32)v4[1], (u32)v4[2], (u32)v4[3]);
+                    if (fmt == TILE_W40)
+                        *(u32*)(stage + TILE_STAGE_WORDS * 4u + at) = (u32)(v4[0] >> 32) | ((u32)(v4[1] >> 32) << 8) |
+                                                                     ((u32)(v4[2] >> 32) << 16) | ((u32)(v4[3] >> 32) << 24);
+                }
+                continue;
+            }
             if (B.split_bits) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) v4[i] = limb_split(v4[i], B.split_bits);
@@ -586,9 +608,6 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 continue;
             }
             ulonglong2* gp = (ulonglong2*)(gdst + 4 * s);
-            if (B.tile_ptr)     // 4 adjacent coefficients never straddle a tile (tiles hold >= 16)
-                gp = (ulonglong2*)(B.tile_ptr + tile_word_offset(B.tile, (B.o_base + o) / B.tile.n_terms - B.tile_pj0,
-                                                                 (B.o_base + o) % B.tile.n_terms, mod, chunk * LEN + 4 * s));
             gp[0] = make_ulonglong2(v4[0], v4[1]);
             gp[1] = make_ulonglong2(v4[2], v4[3]);
         }
@@ -597,16 +616,37 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 #pragma unroll
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
-            const ulonglong2* gp = (const ulonglong2*)(gsrc + 4 * s);
-            if (B.tile_ptr)
-                gp = (const ulonglong2*)(B.tile_ptr + tile_word_offset(B.tile, (B.o_base + o) / B.tile.n_terms - B.tile_pj0,
-                                                                       (B.o_base + o) % B.tile.n_terms, mod,
-                                                                       chunk * LEN + 4 * s));
-            const ulonglong2 a = gp[0], b = gp[1];
-            u64 v4[4] = {a.x, a.y, b.x, b.y};
-            if (B.split_bits) {
+            u64 v4[4];
+            if (B.tile_ptr) {       // read back from the tile-major plaintext cache
+                const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
+                const u32 n = chunk * LEN + 4 * s;
+                const unsigned char* stage = (const unsigned char*)B.tile_ptr + tile_stage_of_word(B.tile, pj, term, mod, n);
+                const u32 at = tile_word_index(B.tile, pj, term, n);
+                const u32 fmt = B.tile.fmt[mod];
+                if (fmt == TILE_W64) {
+                    const ulonglong2* gp = (const ulonglong2*)(stage + (size_t)at * 8);
+                    const ulonglong2 a = gp[0], b = gp[1];
+                    v4[0] = a.x; v4[1] = a.y; v4[2] = b.x; v4[3] = b.y;
+                    if (B.split_bits) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) v4[i] = limb_join(v4[i], B.split_bits);
+                        for (int i = 0; i < 4; ++i) v4[i] = limb_join(v4[i], B.split_bits);
+                    }
+                } else {
+                    const uint4 lo = *(const uint4*)(stage + (size_t)at * 4);
+                    const u32 hi = fmt == TILE_W40 ? *(const u32*)(stage + TILE_STAGE_WORDS * 4u + at) : 0u;
+                    v4[0] = lo.x | ((u64)(hi & 255u) << 32);
+                    v4[1] = lo.y | ((u64)((hi >> 8) & 255u) << 32);
+                    v4[2] = lo.z | ((u64)((hi >> 16) & 255u) << 32);
+                    v4[3] = lo.w | ((u64)(hi >> 24) << 32);
+                }
+            } else {
+                const ulonglong2* gp = (const ulonglong2*)(gsrc + 4 * s);
+                const ulonglong2 a = gp[0], b = gp[1];
+                v4[0] = a.x; v4[1] = a.y; v4[2] = b.x; v4[3] = b.y;
+                if (B.split_bits) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) v4[i] = limb_join(v4[i], B.split_bits);
+                }
             }
             if (B.sum_terms) {      // the input is a sum of several arrays of the same shape
                 const u64* sp = B.sum_src + (size_t)o * B.src_so + (size_t)m * B.src_sm + (size_t)chunk * LEN + 4 * s;

@@ -46,19 +46,29 @@ ENCODE_CASES = [
 ]
 
 
+@pytest.mark.parametrize("compact", [False, True])
 @pytest.mark.parametrize("pkey,plan_t,shape", ENCODE_CASES)
-def test_encode_weights_matches_oracle(pkey, plan_t, shape):
+def test_encode_weights_matches_oracle(pkey, plan_t, shape, compact):
     par = oracle_params(pkey)
     plan = ckks.Plan(*plan_t)
     d_out, d_in = shape
     W = wl.gen_weights(1, f"enc{pkey}{plan_t}", d_out, d_in)
     g = GpuSide(par, plan)
     try:
+        g.bf.bf_set_compact_cache(g.ctx, compact)
         w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in)
         n_in, n_out = -(-d_in // plan.D), -(-d_out // plan.D)
         used = g.bf.bf_cache_bytes_used(g.ctx)
         assert used == g.bf.bf_weights_bytes(g.ctx, d_out, d_in)
-        assert used >= n_in * n_out * plan.M * par.r * par.N * 8        # the encoded words, plus layout padding
+        # every encoded word is resident once: 8 bytes, or in the compact cache the narrowest format its
+        # prime allows (4, 5 or 8 bytes); layout padding comes on top
+        word_bytes = sum(4 if q < 2 ** 32 else 5 if q < 2 ** 40 else 8 for q in par.primes) if compact else 8 * par.r
+        words = n_in * n_out * plan.M * par.N
+        assert words * word_bytes <= used
+        if compact and word_bytes < 8 * par.r:
+            g.bf.bf_set_compact_cache(g.ctx, False)
+            assert used < g.bf.bf_weights_bytes(g.ctx, d_out, d_in)
+            g.bf.bf_set_compact_cache(g.ctx, True)
         idx = [(p, q, j, k) for p in range(n_out) for q in range(n_in) for j in range(plan.g) for k in range(plan.b)]
         if len(idx) > 48:                         # sample, always keeping the corners
             rng = np.random.default_rng(0)
@@ -166,6 +176,18 @@ def run_case(par, plan, d_out, d_in, seed, tol, tag, tight=1e-5):
         got_replayed = g.to_host_u64(ct_out)
         for p in range(n_out):
             assert np.array_equal(got_replayed[p], expect[p]), ("replayed", p)
+        # the compact cache format (narrower words per prime) changes no residue, cached or on the fly
+        g.bf.bf_set_compact_cache(g.ctx, True)
+        w_compact = g.bf.bf_encode_weights(g.ctx, Wd, d_out, d_in)
+        got_compact = g.to_host_u64(g.linear(cts, W, d_out, d_in, weights=w_compact))
+        got_compact_fallback = g.to_host_u64(g.linear(cts, W, d_out, d_in, weights=None))
+        got_mixed = g.to_host_u64(g.linear(cts, W, d_out, d_in, weights=w))        # the older handle still works
+        g.bf.bf_set_compact_cache(g.ctx, False)
+        for p in range(n_out):
+            assert np.array_equal(got_compact[p], expect[p]), ("compact", p)
+            assert np.array_equal(got_compact_fallback[p], expect[p]), ("compact fallback", p)
+            assert np.array_equal(got_mixed[p], expect[p]), ("mixed", p)
+        g.bf.bf_weights_free(g.ctx, w_compact)
         # rescale on the device, decrypt on the host, compare with the fp64 product
         d_ct = g.to_dev(got_cached)
         low = g.empty_u64(n_out, 2, par.r - 1, par.N)
