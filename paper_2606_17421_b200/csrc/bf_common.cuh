@@ -248,18 +248,27 @@ struct ModDownEpilogue {
 enum TileFormat : u32 { TILE_W64 = 0, TILE_W40 = 1, TILE_W32 = 2 };
 struct TileLayout {
     u32 log_tn, n_terms, n_pj, G, C, ntiles;
-    u32 fmt[MAX_MODULI];                    // TileFormat of every ciphertext prime
-    unsigned long long base[MAX_MODULI];    // byte offset of the prime's first stage; base[r] = total bytes
+    u32 fmt_bits;                           // TileFormat of ciphertext prime i in bits 2i, 2i+1
 };
 constexpr u32 TILE_TS = 8;
 constexpr u32 TILE_STAGE_WORDS = 2048;
 
+__host__ __device__ __forceinline__ u32 tile_format(const TileLayout& t, u32 i) { return (t.fmt_bits >> (2 * i)) & 3u; }
 __host__ __device__ __forceinline__ u32 tile_stage_bytes(u32 fmt) {
     return TILE_STAGE_WORDS * (fmt == TILE_W64 ? 8u : fmt == TILE_W40 ? 5u : 4u);
 }
+// byte offset of prime i's first stage (i = r: total size): the primes' regions follow one another
+__host__ __device__ __forceinline__ size_t tile_prime_base(const TileLayout& t, u32 i) {
+    size_t words8 = 0;                      // in units of 2048 bytes: a stage is 8, 5 or 4 of them
+    for (u32 k = 0; k < i; ++k) {
+        const u32 f = tile_format(t, k);
+        words8 += f == TILE_W64 ? 8u : f == TILE_W40 ? 5u : 4u;
+    }
+    return words8 * TILE_STAGE_WORDS * (size_t)t.ntiles * t.G * t.C;
+}
 // byte offset of a stage
 __host__ __device__ __forceinline__ size_t tile_stage_offset(const TileLayout& t, u32 i, u32 tile, u32 g, u32 ch) {
-    return (size_t)t.base[i] + (((size_t)tile * t.G + g) * t.C + ch) * tile_stage_bytes(t.fmt[i]);
+    return tile_prime_base(t, i) + (((size_t)tile * t.G + g) * t.C + ch) * tile_stage_bytes(tile_format(t, i));
 }
 // index of a word inside its stage
 __host__ __device__ __forceinline__ u32 tile_word_index(const TileLayout& t, u32 pj, u32 term, u32 n) {

@@ -112,7 +112,8 @@ constexpr int MAC_RING_BYTES = MAC_STAGES * MAC_SLOT_BYTES;
 constexpr int MAC_MAX_STAGES = MAC_STAGES;
 constexpr u32 KARA_L = 25;
 
-template <bool KARA, int LOG_TN>
+// COMPACT = false: every prime of the layout uses 8-byte words (the default), and the format tests fold away.
+template <bool KARA, int LOG_TN, bool COMPACT>
 __global__ void __launch_bounds__(MAC_THREADS, 3)
 mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, const u64* __restrict__ x,
            u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, u32 early_weights,
@@ -148,7 +149,7 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         pj_end = min(pj_end, pj_begin + per);
         if (pj_begin >= pj_end) return;                            // (uniform for the block)
     }
-    const u32 fmt = lay.fmt[i];                                    // this prime's word format decides the stage size
+    const u32 fmt = COMPACT ? tile_format(lay, i) : (u32)TILE_W64;          // this prime's word format decides the stage size
     const u32 stage_bytes = tile_stage_bytes(fmt);
     constexpr u32 n_stages = MAC_STAGES;
     const u32 n_groups = (pj_end - pj_begin + PL - 1) / PL;        // rounds of PL output groups
@@ -173,25 +174,41 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         // one stage of the weight stream: a contiguous 16 KB block of the tile-major layout; when its tail
         // is padding (last group round or last term chunk) copy the valid part of every lane only
         const u32 word_lo = fmt == TILE_W64 ? 8u : 4u;                 // bytes per word of the stage's first part
+        const unsigned char* prime_base = (const unsigned char*)pt + tile_prime_base(lay, i);
         const u32 hi_at = TILE_STAGE_WORDS * 4u;                       // TILE_W40: where the high bytes start
         auto issue_stage = [&]() {
             const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
             const u32 first = pj_begin + g * PL;
             const u32 lanes = min((u32)PL, pj_end - first);
-            const unsigned char* stage = (const unsigned char*)pt + tile_stage_offset(lay, i, tile_x, first / PL, ch);
-            unsigned char* sdst = ring + (size_t)slot * MAC_SLOT_BYTES;
-            const u32 bytes_per_word = fmt == TILE_W64 ? 8u : fmt == TILE_W40 ? 5u : 4u;
-            if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * bytes_per_word);
-            __syncwarp();
-            if (lanes == PL && cnt == (u32)MAC_TS) {
-                if (lane == 0) bulk_g2s_stream(sdst, stage, stage_bytes, &full[slot], stream_policy);
-            } else if (lane < lanes) {
-                // the valid part of every lane: cnt terms of TN words (and their high bytes)
-                const u32 at = lane * MAC_TS * TN;
-                bulk_g2s_stream(sdst + (size_t)at * word_lo, stage + (size_t)at * word_lo, cnt * TN * word_lo, &full[slot],
-                                stream_policy);
-                if (fmt == TILE_W40)
-                    bulk_g2s_stream(sdst + hi_at + at, stage + hi_at + at, cnt * TN, &full[slot], stream_policy);
+            if constexpr (!COMPACT) {
+                // the stage is one contiguous 16 KB block of the tile-major layout; when its tail is
+                // padding (last group round or last term chunk) copy the valid part of every lane only
+                const u64* stage = (const u64*)(prime_base + (((size_t)tile_x * lay.G + first / PL) * lay.C + ch) * (MAC_STAGE_WORDS * 8));
+                u64* sdst = (u64*)ring + (size_t)slot * MAC_STAGE_WORDS;
+                if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * 8);
+                __syncwarp();
+                if (lanes == PL && cnt == (u32)MAC_TS) {
+                    if (lane == 0) bulk_g2s_stream(sdst, stage, MAC_STAGE_WORDS * 8, &full[slot], stream_policy);
+                } else if (lane < lanes) {
+                    bulk_g2s_stream(sdst + (size_t)lane * MAC_TS * TN, stage + (size_t)lane * MAC_TS * TN, cnt * TN * 8,
+                                    &full[slot], stream_policy);
+                }
+            } else {
+                const unsigned char* stage = prime_base + (((size_t)tile_x * lay.G + first / PL) * lay.C + ch) * stage_bytes;
+                unsigned char* sdst = ring + (size_t)slot * MAC_SLOT_BYTES;
+                const u32 bytes_per_word = fmt == TILE_W64 ? 8u : fmt == TILE_W40 ? 5u : 4u;
+                if (lane == 0) mbar_expect_tx(&full[slot], lanes * cnt * TN * bytes_per_word);
+                __syncwarp();
+                if (lanes == PL && cnt == (u32)MAC_TS) {
+                    if (lane == 0) bulk_g2s_stream(sdst, stage, stage_bytes, &full[slot], stream_policy);
+                } else if (lane < lanes) {
+                    // the valid part of every lane: cnt terms of TN words (and their high bytes)
+                    const u32 at = lane * MAC_TS * TN;
+                    bulk_g2s_stream(sdst + (size_t)at * word_lo, stage + (size_t)at * word_lo, cnt * TN * word_lo, &full[slot],
+                                    stream_policy);
+                    if (fmt == TILE_W40)
+                        bulk_g2s_stream(sdst + hi_at + at, stage + hi_at + at, cnt * TN, &full[slot], stream_policy);
+                }
             }
             if (++ch == n_chunks) { ch = 0; ++g; }
             if (++slot == n_stages) { slot = 0; phase ^= 1; }
@@ -231,54 +248,76 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         const u32 t0 = ch * MAC_TS, cnt = min((u32)MAC_TS, n_terms - t0);
         mbar_wait(&full[slot], phase, error_flag);
         if (pj < pj_end) {
-            const unsigned char* sbase = ring + (size_t)slot * MAC_SLOT_BYTES;
-            const u32 at = l * MAC_TS * TN + c;                        // index of this thread's first word of the stage
             const u64* xt = xs + (size_t)t0 * 2 * TN + c;
-            // one streamed word times both components of its X word
-            auto mac_word = [&](u64 w, u32 w0, u32 w1, u32 ts) {
-                if (KARA) {
-                    const u32 ws = w0 + w1;
-                    k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
-                    k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
-                } else {
-                    a0.mac(w, xt[(ts * 2) * TN]);
-                    a1.mac(w, xt[(ts * 2 + 1) * TN]);
-                }
-            };
-            if (fmt == TILE_W64) {              // whole words; limbs already split when KARA
-                const u64* ps = (const u64*)sbase + at;
+            if constexpr (!COMPACT) {           // whole words; limbs already split when KARA
+                const u64* ps = (const u64*)ring + (size_t)slot * MAC_STAGE_WORDS + (size_t)l * MAC_TS * TN + c;
                 if (cnt == MAC_TS) {
 #pragma unroll
                     for (int ts = 0; ts < MAC_TS; ++ts) {
                         const u64 w = ps[ts * TN];
-                        mac_word(w, (u32)w, (u32)(w >> 32), ts);
+                        if (KARA) {
+                            const u32 w0 = (u32)w, w1 = (u32)(w >> 32), ws = w0 + w1;
+                            k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
+                            k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
+                        } else {
+                            a0.mac(w, xt[(ts * 2) * TN]);
+                            a1.mac(w, xt[(ts * 2 + 1) * TN]);
+                        }
                     }
                 } else {
                     for (u32 ts = 0; ts < cnt; ++ts) {
                         const u64 w = ps[ts * TN];
+                        if (KARA) {
+                            const u32 w0 = (u32)w, w1 = (u32)(w >> 32), ws = w0 + w1;
+                            k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
+                            k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
+                        } else {
+                            a0.mac(w, xt[(ts * 2) * TN]);
+                            a1.mac(w, xt[(ts * 2 + 1) * TN]);
+                        }
+                    }
+                }
+            } else {
+                const unsigned char* sbase = ring + (size_t)slot * MAC_SLOT_BYTES;
+                const u32 at = l * MAC_TS * TN + c;                    // index of this thread's first word of the stage
+                // one streamed word times both components of its X word
+                auto mac_word = [&](u64 w, u32 w0, u32 w1, u32 ts) {
+                    if (KARA) {
+                        const u32 ws = w0 + w1;
+                        k0.mac(w0, w1, ws, xt[(ts * 2) * TN]);
+                        k1.mac(w0, w1, ws, xt[(ts * 2 + 1) * TN]);
+                    } else {
+                        a0.mac(w, xt[(ts * 2) * TN]);
+                        a1.mac(w, xt[(ts * 2 + 1) * TN]);
+                    }
+                };
+                if (fmt == TILE_W64) {          // whole words; limbs already split when KARA
+                    const u64* ps = (const u64*)sbase + at;
+                    for (u32 ts = 0; ts < cnt; ++ts) {
+                        const u64 w = ps[ts * TN];
                         mac_word(w, (u32)w, (u32)(w >> 32), ts);
                     }
-                }
-            } else if (fmt == TILE_W40) {       // low 32 bits and high byte, limbs cut here
-                const u32* pl = (const u32*)sbase + at;
-                const unsigned char* ph = sbase + TILE_STAGE_WORDS * 4u + at;
-                if (cnt == MAC_TS) {
+                } else if (fmt == TILE_W40) {   // low 32 bits and high byte, limbs cut here
+                    const u32* pl = (const u32*)sbase + at;
+                    const unsigned char* ph = sbase + TILE_STAGE_WORDS * 4u + at;
+                    if (cnt == MAC_TS) {
 #pragma unroll
-                    for (int ts = 0; ts < MAC_TS; ++ts) {
-                        const u32 lo = pl[ts * TN], hi = ph[ts * TN];
-                        mac_word(((u64)hi << 32) | lo, lo & ((1u << KARA_L) - 1), (lo >> KARA_L) | (hi << (32 - KARA_L)), ts);
+                        for (int ts = 0; ts < MAC_TS; ++ts) {
+                            const u32 lo = pl[ts * TN], hi = ph[ts * TN];
+                            mac_word(((u64)hi << 32) | lo, lo & ((1u << KARA_L) - 1), (lo >> KARA_L) | (hi << (32 - KARA_L)), ts);
+                        }
+                    } else {
+                        for (u32 ts = 0; ts < cnt; ++ts) {
+                            const u32 lo = pl[ts * TN], hi = ph[ts * TN];
+                            mac_word(((u64)hi << 32) | lo, lo & ((1u << KARA_L) - 1), (lo >> KARA_L) | (hi << (32 - KARA_L)), ts);
+                        }
                     }
-                } else {
+                } else {                        // 32-bit words
+                    const u32* pl = (const u32*)sbase + at;
                     for (u32 ts = 0; ts < cnt; ++ts) {
-                        const u32 lo = pl[ts * TN], hi = ph[ts * TN];
-                        mac_word(((u64)hi << 32) | lo, lo & ((1u << KARA_L) - 1), (lo >> KARA_L) | (hi << (32 - KARA_L)), ts);
+                        const u32 lo = pl[ts * TN];
+                        mac_word((u64)lo, lo & ((1u << KARA_L) - 1), lo >> KARA_L, ts);
                     }
-                }
-            } else {                            // 32-bit words
-                const u32* pl = (const u32*)sbase + at;
-                for (u32 ts = 0; ts < cnt; ++ts) {
-                    const u32 lo = pl[ts * TN];
-                    mac_word((u64)lo, lo & ((1u << KARA_L) - 1), lo >> KARA_L, ts);
                 }
             }
         }
@@ -337,18 +376,15 @@ TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms) {
     t.G = (n_pj + PL - 1) / PL;
     t.C = (n_terms + TILE_TS - 1) / TILE_TS;
     t.ntiles = ring.dev.N >> t.log_tn;
-    unsigned long long at = 0;
     for (u32 i = 0; i < ring.dev.r; ++i) {
-        t.fmt[i] = !ring.compact_cache ? TILE_W64
-                 : ring.q[i] < (1ull << 32) ? TILE_W32 : ring.q[i] < (1ull << 40) ? TILE_W40 : TILE_W64;
-        t.base[i] = at;
-        at += (unsigned long long)t.ntiles * t.G * t.C * tile_stage_bytes(t.fmt[i]);
+        const u32 f = !ring.compact_cache ? TILE_W64
+                    : ring.q[i] < (1ull << 32) ? TILE_W32 : ring.q[i] < (1ull << 40) ? TILE_W40 : TILE_W64;
+        t.fmt_bits |= f << (2 * i);
     }
-    t.base[ring.dev.r] = at;
     return t;
 }
 
-size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t) { return (size_t)t.base[ring.dev.r]; }
+size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t) { return tile_prime_base(t, ring.dev.r); }
 
 u32 mac_split_bits(const RingHost& ring) {
     u64 qmax = 0;
@@ -356,7 +392,7 @@ u32 mac_split_bits(const RingHost& ring) {
     return bits_of(qmax) <= 50 ? KARA_L : 0;
 }
 
-template <bool KARA, int LOG_TN>
+template <bool KARA, int LOG_TN, bool COMPACT>
 static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a,
                                 u32 n_pj, u32 n_terms, u32 lazy, u32 early_weights, int* error_flag,
                                 cudaStream_t stream) {
@@ -365,7 +401,7 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
     static bool attr_set = false;     // opt in once to the large dynamic shared-memory carve-out
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(mac_kernel<KARA, LOG_TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(mac_kernel<KARA, LOG_TN, COMPACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              200 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
@@ -389,7 +425,7 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
         if (sm_count <= 0) sm_count = 148;
     }
     if (per_sm_smem != smem) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mac_kernel<KARA, LOG_TN>, MAC_THREADS, smem) != cudaSuccess ||
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mac_kernel<KARA, LOG_TN, COMPACT>, MAC_THREADS, smem) != cudaSuccess ||
             per_sm < 1) {
             cudaGetLastError();
             per_sm = 1;
@@ -407,7 +443,7 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     }
     const u32 n_whole = tail_split > 1 ? units - rem : units;
     dim3 grid(n_whole + (units - n_whole) * tail_split);
-    return launch_dependent(ring, mac_kernel<KARA, LOG_TN>, grid, dim3(MAC_THREADS), smem, stream, ring.dev, pt, lay, x, a,
+    return launch_dependent(ring, mac_kernel<KARA, LOG_TN, COMPACT>, grid, dim3(MAC_THREADS), smem, stream, ring.dev, pt, lay, x, a,
                             n_terms, n_pj, pj_per_block, lazy, early_weights, n_whole, tail_split, error_flag);
 }
 
@@ -431,7 +467,11 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
         return cudaErrorInvalidValue;
     }
     const u32 early = weights_static ? 1u : 0u;
-#define BF_MAC(S, L) launch_mac_t<S, L>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, error_flag, stream)
+    bool compact = false;
+    for (u32 i = 0; i < ring.dev.r; ++i) compact = compact || tile_format(lay, i) != TILE_W64;
+#define BF_MAC(S, L)                                                                                             \
+    (compact ? launch_mac_t<S, L, true>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, error_flag, stream)     \
+             : launch_mac_t<S, L, false>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, error_flag, stream))
     if (kara) {
         switch (log_tn) {
             case 8: return BF_MAC(true, 8);

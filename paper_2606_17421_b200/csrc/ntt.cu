@@ -492,7 +492,8 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
 // groups, so only warp-level synchronisation is needed.
 // Forward: second pass (final reduction to [0, q), then the store functors).  Inverse: first pass
 // (reads the batch source: plain residues, tiled/limb-split plaintexts, or a sum of arrays).
-template <bool FWD, bool EPI, bool FP>
+// TILED: the transform-domain side of the batch lives in the tile-major plaintext cache (B.tile_ptr).
+template <bool FWD, bool EPI, bool FP, bool TILED>
 __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, u32 o, u32 m, u32 mod,
                                             u32 chunk, int lane, const RotBatch& rb, const ModDownEpilogue& epi) {
     typedef typename Elem<FP>::T T;
@@ -574,12 +575,12 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 }
                 continue;
             }
-            if (B.tile_ptr) {   // tile-major plaintext cache; 4 adjacent coefficients never straddle a tile (tiles hold >= 16)
+            if constexpr (TILED) {   // tile-major plaintext cache; 4 adjacent coefficients never straddle a tile (tiles hold >= 16)
                 const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
                 const u32 n = chunk * LEN + 4 * s;
                 unsigned char* stage = (unsigned char*)B.tile_ptr + tile_stage_of_word(B.tile, pj, term, mod, n);
                 const u32 at = tile_word_index(B.tile, pj, term, n);
-                const u32 fmt = B.tile.fmt[mod];
+                const u32 fmt = tile_format(B.tile, mod);
                 if (fmt == TILE_W64) {
                     if (B.split_bits) {
 #pragma unroll
@@ -617,12 +618,12 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
             u64 v4[4];
-            if (B.tile_ptr) {       // read back from the tile-major plaintext cache
+            if constexpr (TILED) {  // read back from the tile-major plaintext cache
                 const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
                 const u32 n = chunk * LEN + 4 * s;
                 const unsigned char* stage = (const unsigned char*)B.tile_ptr + tile_stage_of_word(B.tile, pj, term, mod, n);
                 const u32 at = tile_word_index(B.tile, pj, term, n);
-                const u32 fmt = B.tile.fmt[mod];
+                const u32 fmt = tile_format(B.tile, mod);
                 if (fmt == TILE_W64) {
                     const ulonglong2* gp = (const ulonglong2*)(stage + (size_t)at * 8);
                     const ulonglong2 a = gp[0], b = gp[1];
@@ -678,7 +679,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
     }
 }
 
-template <bool FWD, bool EPI>
+template <bool FWD, bool EPI, bool TILED>
 __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
@@ -692,8 +693,8 @@ __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const Rin
     if ((u32)warp >= chunks_per_block) return;
     const u32 chunk = blockIdx.x * chunks_per_block + warp;
     u64* sm = sm_all + (warp << LOG_C);
-    if (R.fp_ok[mod]) contig_body<FWD, EPI, true>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
-    else contig_body<FWD, EPI, false>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
+    if (R.fp_ok[mod]) contig_body<FWD, EPI, true, TILED>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
+    else contig_body<FWD, EPI, false, TILED>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
 }
 
 NttGeometry ntt_geometry(u32 logN) {
@@ -788,12 +789,17 @@ static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n
     const u32 cpb = (u32)ring.geom.contig_lanes;
     dim3 grid(chunks / cpb, n_polys);
     if (FWD && epi) {
-        launch_dependent(ring, ntt_contig<FWD, true>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb, *epi);
+        launch_dependent(ring, ntt_contig<FWD, true, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
+                         *epi);
     } else {
         static const RotBatch no_rb = {};
         static const ModDownEpilogue no_epi = {};
-        launch_dependent(ring, ntt_contig<FWD, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, no_rb,
-                         no_epi);
+        if (B.tile_ptr)
+            launch_dependent(ring, ntt_contig<FWD, false, true>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
+                             no_rb, no_epi);
+        else
+            launch_dependent(ring, ntt_contig<FWD, false, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
+                             no_rb, no_epi);
     }
     return cudaGetLastError();
 }
