@@ -651,7 +651,22 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
             }
             if (B.sum_terms) {      // the input is a sum of several arrays of the same shape
                 const u64* sp = B.sum_src + (size_t)o * B.src_so + (size_t)m * B.src_sm + (size_t)chunk * LEN + 4 * s;
-                for (u32 t = 0; t < B.sum_terms; ++t) {
+                // three arrays at a time, all their loads in flight together (g - 1 = 3 is the common case)
+                u32 t = 0;
+                for (; t + 3 <= B.sum_terms; t += 3) {
+                    ulonglong2 a2[3], b2[3];
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) {
+                        a2[j] = *(const ulonglong2*)(sp + (size_t)(t + j) * B.sum_stride);
+                        b2[j] = *(const ulonglong2*)(sp + (size_t)(t + j) * B.sum_stride + 2);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) {
+                        v4[0] = add_mod(v4[0], a2[j].x, q); v4[1] = add_mod(v4[1], a2[j].y, q);
+                        v4[2] = add_mod(v4[2], b2[j].x, q); v4[3] = add_mod(v4[3], b2[j].y, q);
+                    }
+                }
+                for (; t < B.sum_terms; ++t) {
                     const ulonglong2 a2 = *(const ulonglong2*)(sp + (size_t)t * B.sum_stride);
                     const ulonglong2 b2 = *(const ulonglong2*)(sp + (size_t)t * B.sum_stride + 2);
                     v4[0] = add_mod(v4[0], a2.x, q); v4[1] = add_mod(v4[1], a2.y, q);
