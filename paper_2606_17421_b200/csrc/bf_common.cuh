@@ -48,9 +48,6 @@ __device__ __forceinline__ u64 mul_shoup_lazy(u64 x, u64 w, u64 ws, u64 q) {
     return x * w - hi * q;
 }
 
-// ---- fp64 arithmetic for primes q < 2^41.  B200 issues fp64 FMAs at the rate of 32-bit integer
-// multiply-adds, on a pipe of its own, while a 64x64-bit high product costs about ten integer
-// multiply-add slots; and integers below 2^53 are exact in fp64.
 // First statement of every kernel of a linear-layer call.  Lets the next kernel of the stream be scheduled
 // as soon as all blocks of this one have started, then waits until the previous kernel has completed and
 // flushed its writes.  A no-op when the launch carries no programmatic dependency.
@@ -59,6 +56,9 @@ __device__ __forceinline__ void grid_dependency_enter() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// ---- fp64 arithmetic for primes q < 2^50.  B200 issues fp64 FMAs at the rate of 32-bit integer
+// multiply-adds, on a pipe of its own, while a 64x64-bit high product costs about ten integer
+// multiply-add slots; and integers below 2^53 are exact in fp64.
 __device__ __forceinline__ double u2d(u64 x) {          // exact for x < 2^52
     return __longlong_as_double((long long)(x | 0x4330000000000000ull)) - 4503599627370496.0;
 }

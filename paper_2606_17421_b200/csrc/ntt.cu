@@ -74,8 +74,8 @@ __device__ __forceinline__ u64 load_src(const void* src, size_t idx, const LoadC
     return m;
 }
 
-// The same loads for a modulus on the fp64 path: the result is a non-negative integer-valued double
-// congruent to the source, below 3.6 q (lazy: the butterflies reduce).
+// The same loads for a modulus on the fp64 path: the result is an integer-valued double congruent to the
+// source, of magnitude below 3.6 q (lazy: the butterflies reduce); non-negative for primes of 2^41 or more.
 template <int LOAD>
 __device__ __forceinline__ double load_src_fp(const void* src, size_t idx, const LoadConsts& c) {
     if (LOAD == LOAD_REDUCE) {
