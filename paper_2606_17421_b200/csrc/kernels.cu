@@ -533,8 +533,9 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
         const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + n0;
         const u64* kp = keys + ((size_t)rb.key[rot] * r * 2 * nb + m) * N + n0;
         // the keys do not depend on the previous kernel: fetch them before waiting for it, the digits after
+        const u64 stream_policy = l2_evict_first_policy();      // keys stream through; digits and outputs stay in L2
         for (u32 e = tid; e < 2 * r; e += 32)
-            bulk_g2s(sk + (size_t)e * KI_TILE, kp + (size_t)e * nb * N, KI_TILE * 8, bar);
+            bulk_g2s_stream(sk + (size_t)e * KI_TILE, kp + (size_t)e * nb * N, KI_TILE * 8, bar, stream_policy);
         asm volatile("griddepcontrol.wait;" ::: "memory");
         for (u32 j = tid; j < r; j += 32)
             bulk_g2s(sd + (size_t)j * KI_TILE, dp + (size_t)j * nb * N, KI_TILE * 8, bar);
