@@ -285,7 +285,7 @@ __device__ __forceinline__ void swz_load_set(u32 a_thread, T (&e)[8]) {
 }
 
 constexpr int LOG_C = 8;              // contiguous pass: chunks of 256 points, one warp each
-constexpr int CHUNKS_PER_BLOCK = 8;
+constexpr int CHUNKS_PER_BLOCK = 4;      // measured: 4 beats 8 by 4 % of the pass, 2 is no better
 
 // Between the two passes of a transform the data sit in dst as lazily reduced values: 64-bit
 // integers for the integer path, fp64 bit patterns for the fp64 path (the modulus decides, so both
@@ -695,7 +695,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 }
 
 template <bool FWD, bool EPI, bool TILED>
-__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 4) ntt_contig(const RingDev R, const PolyBatch B,
+__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 8) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
     __shared__ __align__(128) u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
