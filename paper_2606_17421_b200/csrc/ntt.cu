@@ -422,7 +422,7 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
 
 template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
 __global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8),
-                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
+                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : ((1 << (LOG_R + LOG_LANES)) / 8) >= 256 ? 4 : 8)
 ntt_strided(const RingDev R, const PolyBatch B) {
     __shared__ u64 sm[1 << (LOG_R + LOG_LANES)];
     __shared__ ulonglong2 tws[1 << LOG_R];
@@ -450,7 +450,7 @@ ntt_strided(const RingDev R, const PolyBatch B) {
 // target.  grid: x = tile, y = outer index o, z = slice of the targets.
 template <int LOAD, int LOG_R, int LOG_LANES>
 __global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8),
-                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : 4)
+                                  ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : ((1 << (LOG_R + LOG_LANES)) / 8) >= 256 ? 4 : 8)
 ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
     constexpr int LANES = 1 << LOG_LANES, POINTS = 1 << (LOG_R + LOG_LANES);
     extern __shared__ __align__(16) u64 shared_src_smem[];
@@ -741,7 +741,7 @@ static void launch_shared_src_t(const RingHost& ring, const PolyBatch& B, u32 n_
     constexpr u32 S = (1u << LOG_C) >> LOG_LANES;
     // targets per block: fewer blocks share the source better but quantise into waves; cost model =
     // waves x (targets per block + half a unit for staging the source)
-    const u32 slots = 148u * (NT >= 512 ? 2 : 4);
+    const u32 slots = 148u * (NT >= 512 ? 2 : NT >= 256 ? 4 : 8);
     u32 best = 1;
     double best_cost = 1e30;
     for (u32 per = 1; per <= B.n_m; ++per) {
@@ -775,7 +775,7 @@ static cudaError_t launch_strided(const RingHost& ring, const PolyBatch& B, u32 
                 case 4: launch_shared_src_t<LOAD, 4, 7>(ring, B, n_outer, stream); break;
                 case 5: launch_shared_src_t<LOAD, 5, 6>(ring, B, n_outer, stream); break;
                 case 6: launch_shared_src_t<LOAD, 6, 5>(ring, B, n_outer, stream); break;
-                case 7: launch_shared_src_t<LOAD, 7, 4>(ring, B, n_outer, stream); break;
+                case 7: launch_shared_src_t<LOAD, 7, 3>(ring, B, n_outer, stream); break;
                 case 8: launch_shared_src_t<LOAD, 8, 4>(ring, B, n_outer, stream); break;
                 default: return cudaErrorInvalidValue;
             }
