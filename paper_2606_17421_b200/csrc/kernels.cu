@@ -628,6 +628,24 @@ __global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const Res
   }
 }
 
+// Out-of-place form: one thread per output word (coefficient, ciphertext, component, prime), so the launch is
+// wide enough to hide its loads; the dropped prime's residue is read once per output prime (an L2 hit).
+// grid: x = coefficients / 256, y = ciphertext, z = component * (level - 1) + prime.
+__global__ void __launch_bounds__(256) rescale_wide_kernel(const RingDev R, const RescaleConsts rc, const u64* __restrict__ in,
+                                                           u64* __restrict__ out, u32 level) {
+    grid_dependency_enter();
+    const u32 N = R.N;
+    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
+    const u32 ct = blockIdx.y, comp = blockIdx.z / (level - 1), i = blockIdx.z % (level - 1);
+    const u64* ip = in + ((size_t)ct * 2 + comp) * level * N + n;
+    const u64 qL = R.q[level - 1], q = R.q[i];
+    const u64 t = ip[(size_t)(level - 1) * N];
+    const u64 c = ip[(size_t)i * N];
+    u64 tq = barrett64(t, q, R.mu[i]);
+    if (t > (qL - 1) / 2) tq = sub_mod(tq, rc.qlmod[i], q);
+    out[(((size_t)ct * 2 + comp) * (level - 1) + i) * N + n] = mul_shoup(sub_mod(c, tq, q), rc.inv[i], rc.invs[i], q);
+}
+
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
                            const u64* invs, const u64* qlmod, cudaStream_t stream) {
     if (n_ct == 0) return cudaSuccess;
@@ -637,9 +655,12 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
     if (in == out && n_ct > 1) {
         dim3 grid(ring.dev.N / 64, 1);
         launch_dependent(ring, rescale_kernel, grid, dim3(64), 0, stream, ring.dev, rc, in, out, level, n_ct);
-    } else {
+    } else if (in == out || n_ct > 65535) {
         dim3 grid(ring.dev.N / 256, n_ct);
         launch_dependent(ring, rescale_kernel, grid, dim3(256), 0, stream, ring.dev, rc, in, out, level, 1u);
+    } else {
+        dim3 grid(ring.dev.N / 256, n_ct, 2 * (level - 1));
+        launch_dependent(ring, rescale_wide_kernel, grid, dim3(256), 0, stream, ring.dev, rc, in, out, level);
     }
     return cudaGetLastError();
 }
