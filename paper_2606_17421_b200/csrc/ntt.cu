@@ -533,6 +533,23 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
             swz_load_set<4, 0>(a_near + (u32)(it * 8 * swz(128)), e);      // (swz(128) = 128: above the bits of 4 * lane)
+            // the epilogue's operands do not depend on the transform: ask for them before the last butterflies
+            u64 uu[4] = {0, 0, 0, 0}, cc[4] = {0, 0, 0, 0};
+            u32 pp[4] = {0, 0, 0, 0};
+            if (EPI) {
+                const u32 rot = o >> 1, comp = o & 1, ip = mod, nb = R.r + 1;
+                const size_t n = (size_t)chunk * LEN + 4 * s;
+                const u64* up = epi.u + ((size_t)o * nb + ip) * R.N + n;
+                const ulonglong2 u0 = *(const ulonglong2*)up, u1 = *(const ulonglong2*)(up + 2);
+                uu[0] = u0.x; uu[1] = u0.y; uu[2] = u1.x; uu[3] = u1.y;
+                if (comp == 0) {
+                    const u64* cp = epi.c0_base + (size_t)rb.c0[rot] * epi.c0_stride + (size_t)ip * R.N + n;
+                    const ulonglong2 c0 = *(const ulonglong2*)cp, c1 = *(const ulonglong2*)(cp + 2);
+                    cc[0] = c0.x; cc[1] = c0.y; cc[2] = c1.x; cc[3] = c1.y;
+                }
+                const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
+                pp[0] = pv.x; pp[1] = pv.y; pp[2] = pv.z; pp[3] = pv.w;
+            }
             set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, qd);
             u64 v4[4];
 #pragma unroll
@@ -553,19 +570,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 }
             }
             if (EPI) {
-                const u32 rot = o >> 1, comp = o & 1, ip = mod, r = R.r, nb = r + 1;
-                const size_t n = (size_t)chunk * LEN + 4 * s;
-                const u64* up = epi.u + ((size_t)o * nb + ip) * R.N + n;
-                const ulonglong2 u0 = *(const ulonglong2*)up, u1 = *(const ulonglong2*)(up + 2);
-                const u64 uu[4] = {u0.x, u0.y, u1.x, u1.y};
-                u64 cc[4] = {0, 0, 0, 0};
-                if (comp == 0) {
-                    const u64* cp = epi.c0_base + (size_t)rb.c0[rot] * epi.c0_stride + (size_t)ip * R.N + n;
-                    const ulonglong2 c0 = *(const ulonglong2*)cp, c1 = *(const ulonglong2*)(cp + 2);
-                    cc[0] = c0.x; cc[1] = c0.y; cc[2] = c1.x; cc[3] = c1.y;
-                }
-                const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
-                const u32 pp[4] = {pv.x, pv.y, pv.z, pv.w};
+                const u32 rot = o >> 1, comp = o & 1, ip = mod, r = R.r;
                 u64* op = epi.out_base + (size_t)rb.out[rot] * epi.out_stride + ((size_t)comp * r + ip) * R.N;
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
