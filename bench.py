@@ -31,11 +31,11 @@ UNIT = "ms"
 # see profiles/ for the capture each figure comes from.  None = not captured yet.
 NCU_TRAFFIC_BYTES = {
     # from the ncu capture summarised under profiles/: dram__bytes_read.sum + dram__bytes_write.sum per launch
-    "gpt2_qkv": {"mac": 423.8e6,                       # 411.1 MB read + 12.7 MB written
-                 "key_inner_product": 395.0e6,         # baby 517.5 MB + giant 272.6 MB per step, over the two launches
-                                                       #   of the serialised timing pass
-                 "ntt_fwd_strided": 23.0e6,            # mean of the eight captured forward launches (both passes)
-                 "ntt_inv_contig": 21.0e6},            # mean of the six captured inverse launches (both passes)
+    "gpt2_qkv": {"mac": 422.9e6,                       # 411.1 MB read + 11.8 MB written
+                 "key_inner_product": 373.5e6,         # 747 MB per step (two lanes' launches), over the two launches of
+                                                       #   the serialised timing pass
+                 "ntt_fwd_strided": 23.8e6,            # mean of the eight captured forward launches (both passes)
+                 "ntt_inv_contig": 11.0e6},            # mean of the eight captured inverse launches (both passes)
 }
 
 
