@@ -416,6 +416,29 @@ def test_fold_in_ciphertext_matches_oracle(pkey, plan_t, shape):
         g.close()
 
 
+def test_fold_of_more_ciphertexts_than_one_key_switch_batch():
+    # 70 ciphertexts: the rounds run in two batches (64 + 6); sampled ones are compared with the oracle
+    par = oracle_params("n12")
+    plan = ckks.Plan(64, 4, 4, 4)
+    s = ckks.keygen(par, 43)
+    fold_steps = ckks.fold_rotations(plan)
+    keys = ckks.make_rotation_keys(par, s, plan, 43, extra_steps=fold_steps)
+    n_ct = 70
+    # [r][2][N] uniform residues per ciphertext, rearranged to the boundary layout [2][r][N]
+    cts = np.stack([np.ascontiguousarray(wl.gen_uniform_residues(43, f"fold{t}", par.primes, (2, par.N)).transpose(1, 0, 2))
+                    for t in range(n_ct)])
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys, extra_steps=fold_steps)
+        d = g.to_dev(cts)
+        g.bf.bf_fold(g.ctx, d, n_ct)
+        got = g.to_host_u64(d)
+        for t in (0, 1, 63, 64, 69):
+            assert np.array_equal(got[t], ckks.fold_in_ciphertext(par, plan, cts[t], keys)), t
+    finally:
+        g.close()
+
+
 def test_stacking_projections_that_share_an_input_changes_no_residue():
     # q/k/v (or gate/up) read the same activation: one call over the row-stacked matrix must give
     # exactly the ciphertexts of the separate calls
