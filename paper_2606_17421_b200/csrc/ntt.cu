@@ -44,7 +44,8 @@ ProfScope::~ProfScope() {
 
 struct LoadConsts {
     u64 q, mu, lift_mod, lift_red;
-    double qd, qinv, c30, c30q, k59;
+    double qd, qinv, c30, c30q, k59;      // (LOAD_I64_MONT: c30 = 2^96 mod q, k59 = the offset for -2^127)
+    double c64d, c64q;                     // LOAD_I64_MONT: 2^64 mod q
     bool wide;          // target prime of 2^41 or more: values must stay in [0, 4q); otherwise they are signed
     bool src_small;     // LOAD_REDUCE: every source word is below 1.5 q already (block-uniform)
     bool src_fp;        // LOAD_REDUCE: every source word is below 2^51
@@ -93,6 +94,14 @@ __device__ __forceinline__ double load_src_fp(const void* src, size_t idx, const
         const u64 T = ((const u64*)src)[idx];
         const double hi = u2d(T >> 30), lo = u2d(T & ((1ull << 30) - 1));
         return __dadd_rn(__dadd_rn(fp_mul_centred(hi, c.c30, c.c30q, c.qd), lo), c.k59);   // (k59: see LoadConsts)
+    }
+    if (LOAD == LOAD_I64_MONT) {
+        // v = (hi' - 2^31) 2^32 + lo with hi' = (v >> 32) + 2^31 in [0, 2^32); two centred products (each
+        // within 0.75 q, 0.51 q for primes below 2^41) plus the offset: magnitude below 1.6 q, or within
+        // (0, 4q) for the primes whose values must stay non-negative
+        const uint2 w = ((const uint2*)src)[idx];
+        const double hi = __uint2double_rn(w.y ^ 0x80000000u), lo = __uint2double_rn(w.x);
+        return __dadd_rn(__dadd_rn(fp_mul_centred(hi, c.c30, c.c30q, c.qd), fp_mul_centred(lo, c.c64d, c.c64q, c.qd)), c.k59);
     }
     return u2d(load_src<LOAD>(src, idx, c));
 }
@@ -323,11 +332,13 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
     lc.lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
     lc.qd = qd;
     lc.qinv = R.qinv_d[mod];
-    lc.c30 = R.c30_d[mod];
-    lc.c30q = R.c30_q[mod];
+    lc.c30 = (LOAD == LOAD_I64_MONT) ? R.c96_d[mod] : R.c30_d[mod];
+    lc.c30q = (LOAD == LOAD_I64_MONT) ? R.c96_q[mod] : R.c30_q[mod];
+    lc.c64d = R.c64_d[mod];
+    lc.c64q = R.c64_q[mod];
     lc.wide = (q >> 41) != 0;
     // wide: 2q - (2^59 mod q) keeps the lifted value positive; otherwise the offset is just -(2^59 mod q)
-    lc.k59 = lc.wide ? R.k59_d[mod] : __dsub_rn(R.k59_d[mod], __dadd_rn(qd, qd));
+    lc.k59 = (LOAD == LOAD_I64_MONT) ? R.k127_d[mod] : lc.wide ? R.k59_d[mod] : __dsub_rn(R.k59_d[mod], __dadd_rn(qd, qd));
     {
         const u64 qs = (LOAD == LOAD_REDUCE && B.src_digits) ? R.q[o % R.r] : ~(u64)0;
         lc.src_small = qs <= q + (q >> 1);
