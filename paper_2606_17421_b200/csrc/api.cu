@@ -94,6 +94,7 @@ struct bf_ctx {
     ulonglong2 *tw_fwd = nullptr, *tw_inv = nullptr;
     u32* slot_of_pos = nullptr;
     double2 *T = nullptr, *Z = nullptr;
+    double* enc_consts = nullptr;   // per-prime constants of the encoder's fp64 load
     int* overflow_flag = nullptr;   // [0]: encoder range overflow; [1]: a bounded device-side wait gave up
     int* device_error = nullptr;
     // rotation keys
@@ -234,6 +235,7 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
     };
     if (cudaGetDevice(&ctx->device) != cudaSuccess) return fail(BF_ERR_CUDA);
 
+    std::vector<double> enc_consts((size_t)MAX_MODULI * ENC_CONSTS, 0.0);
     RingDev& R = ctx->ring.dev;
     memset(&R, 0, sizeof(R));
     R.N = N;
@@ -284,17 +286,18 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
         R.c30_d[m] = (double)((1ull << 30) % q);
         R.c30_q[m] = R.c30_d[m] / (double)q;
         R.k59_d[m] = (double)(2 * q - (1ull << 59) % q);
-        {
+        {   // constants of the encoder's fp64 load (see RingDev::enc_consts)
             const u64 c96 = h_mulmod(R.c64[m], (1ull << 32) % q, q);
             const u64 c127 = h_mulmod(R.c64[m], (1ull << 63) % q, q);
-            R.c96_d[m] = (double)c96;
-            R.c96_q[m] = R.c96_d[m] / (double)q;
-            R.c64_d[m] = (double)R.c64[m];
-            R.c64_q[m] = R.c64_d[m] / (double)q;
             const u64 neg = c127 ? q - c127 : 0;                         // -2^127 mod q in [0, q)
             double k = neg > q / 2 ? -(double)(q - neg) : (double)neg;    // centred
             if (q >> 41) k += 2.0 * (double)q;
-            R.k127_d[m] = k;
+            double* ec = &enc_consts[(size_t)m * ENC_CONSTS];
+            ec[0] = (double)c96;
+            ec[1] = ec[0] / (double)q;
+            ec[2] = (double)R.c64[m];
+            ec[3] = ec[2] / (double)q;
+            ec[4] = k;
         }
         auto dbits = [](double d) -> u64 {
             u64 bits;
@@ -354,17 +357,20 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
     CKC(cudaMalloc(&ctx->T, T.size() * sizeof(double2)));
     CKC(cudaMalloc(&ctx->Z, Z.size() * sizeof(double2)));
     CKC(cudaMalloc(&ctx->overflow_flag, 2 * sizeof(int)));
+    CKC(cudaMalloc(&ctx->enc_consts, enc_consts.size() * sizeof(double)));
     ctx->device_error = ctx->overflow_flag + 1;
     CKC(cudaMemcpy(ctx->tw_fwd, twf.data(), twf.size() * sizeof(ulonglong2), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->tw_inv, twi.data(), twi.size() * sizeof(ulonglong2), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->slot_of_pos, sop.data(), sop.size() * sizeof(u32), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->T, T.data(), T.size() * sizeof(double2), cudaMemcpyHostToDevice));
     CKC(cudaMemcpy(ctx->Z, Z.data(), Z.size() * sizeof(double2), cudaMemcpyHostToDevice));
+    CKC(cudaMemcpy(ctx->enc_consts, enc_consts.data(), enc_consts.size() * sizeof(double), cudaMemcpyHostToDevice));
     CKC(cudaMemset(ctx->overflow_flag, 0, 2 * sizeof(int)));
     CKC(cudaDeviceSynchronize());
 #undef CKC
     R.tw_fwd = ctx->tw_fwd;
     R.tw_inv = ctx->tw_inv;
+    R.enc_consts = ctx->enc_consts;
     *out = ctx;
     return BF_OK;
 }
@@ -395,6 +401,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
     cudaFree(ctx->slot_of_pos);
     cudaFree(ctx->T);
     cudaFree(ctx->Z);
+    cudaFree(ctx->enc_consts);
     for (cudaStream_t& s : ctx->side)
         if (s) { cudaStreamDestroy(s); s = nullptr; }
     for (cudaEvent_t& e : ctx->ev_join)

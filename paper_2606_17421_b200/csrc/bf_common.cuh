@@ -13,6 +13,7 @@ typedef int64_t i64;
 typedef uint32_t u32;
 
 constexpr int MAX_MODULI = 16;    // ciphertext primes + the special prime
+constexpr int ENC_CONSTS = 5;
 // Per-ring constants handed to every kernel by value (lands in the constant bank).
 // Modulus index r is the special prime P; 0..r-1 are the ciphertext primes q_0..q_L.
 struct RingDev {
@@ -38,10 +39,11 @@ struct RingDev {
     double c30_d[MAX_MODULI], c30_q[MAX_MODULI];       // (double)(2^30 mod q) and that over q
     double k59_d[MAX_MODULI];    // 2q - (2^59 mod q): undoes the offset of a stored centred lift, keeps it positive
     // encoder output (signed 64-bit coefficients) into Montgomery form on the fp64 path: the word is
-    // (hi' - 2^31) 2^32 + lo, so times 2^64 it is  hi' (2^96 mod q) + lo (2^64 mod q) - (2^127 mod q)
-    double c96_d[MAX_MODULI], c96_q[MAX_MODULI];       // (double)(2^96 mod q) and that over q
-    double c64_d[MAX_MODULI], c64_q[MAX_MODULI];       // (double)(2^64 mod q) and that over q
-    double k127_d[MAX_MODULI];   // the centred residue of -2^127, plus 2q for primes of 2^41 or more (values stay >= 0)
+    // (hi' - 2^31) 2^32 + lo, so times 2^64 it is  hi' (2^96 mod q) + lo (2^64 mod q) - (2^127 mod q).
+    // Five doubles per prime, in device memory (kernel parameters stay small): (double)(2^96 mod q), that
+    // over q, (double)(2^64 mod q), that over q, and the centred residue of -2^127 (plus 2q for primes of
+    // 2^41 or more, whose values stay non-negative)
+    const double* enc_consts;    // [r+1][ENC_CONSTS]
     const ulonglong2* tw_fwd;    // [r+1][N]  (psi^brev(k), companion), merged Cooley-Tukey order
     const ulonglong2* tw_inv;    // [r+1][N]  inverses of the above, for the Gentleman-Sande inverse
 };

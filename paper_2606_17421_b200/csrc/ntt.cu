@@ -332,13 +332,20 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
     lc.lift_mod = (LOAD == LOAD_I64_MONT) ? R.c64[mod] : B.lift_mod;
     lc.qd = qd;
     lc.qinv = R.qinv_d[mod];
-    lc.c30 = (LOAD == LOAD_I64_MONT) ? R.c96_d[mod] : R.c30_d[mod];
-    lc.c30q = (LOAD == LOAD_I64_MONT) ? R.c96_q[mod] : R.c30_q[mod];
-    lc.c64d = R.c64_d[mod];
-    lc.c64q = R.c64_q[mod];
+    lc.c30 = R.c30_d[mod];
+    lc.c30q = R.c30_q[mod];
+    lc.c64d = lc.c64q = 0.0;
     lc.wide = (q >> 41) != 0;
     // wide: 2q - (2^59 mod q) keeps the lifted value positive; otherwise the offset is just -(2^59 mod q)
-    lc.k59 = (LOAD == LOAD_I64_MONT) ? R.k127_d[mod] : lc.wide ? R.k59_d[mod] : __dsub_rn(R.k59_d[mod], __dadd_rn(qd, qd));
+    lc.k59 = lc.wide ? R.k59_d[mod] : __dsub_rn(R.k59_d[mod], __dadd_rn(qd, qd));
+    if (LOAD == LOAD_I64_MONT) {
+        const double* ec = R.enc_consts + (size_t)mod * ENC_CONSTS;
+        lc.c30 = __ldg(ec);
+        lc.c30q = __ldg(ec + 1);
+        lc.c64d = __ldg(ec + 2);
+        lc.c64q = __ldg(ec + 3);
+        lc.k59 = __ldg(ec + 4);
+    }
     {
         const u64 qs = (LOAD == LOAD_REDUCE && B.src_digits) ? R.q[o % R.r] : ~(u64)0;
         lc.src_small = qs <= q + (q >> 1);
