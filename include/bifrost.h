@@ -117,6 +117,14 @@ int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weight
  * the gain is capacity).  bf_weights_bytes reports sizes for the current setting. */
 int bf_set_compact_cache(bf_ctx* ctx, int on);
 
+/* Fallback path of bf_linear (W_raw given, Sec. 4.2 "fallback encode"): output groups are encoded
+ * in rounds into a scratch buffer and consumed by the multiply-accumulate; `bytes` bounds that
+ * buffer (default 4 GiB; one output group, n_in * b encoded diagonals, is the minimum whatever the
+ * bound).  A larger bound means fewer rounds, and every round re-reads the rotated inputs.  Results
+ * do not depend on it.  Takes effect from the next call; the buffer only ever grows.  No counterpart
+ * in the paper.  Errors: INVALID_ARG (null context or zero bytes). */
+int bf_set_encode_scratch(bf_ctx* ctx, uint64_t bytes);
+
 /* bf_linear replays a captured CUDA graph of its launch sequence from the third call with the same
  * (ct_in, pt_weights, ct_out, d_out, d_in) on: the first call runs directly (and sizes the scratch),
  * the second is captured.  Replay is skipped on the fallback path, while stage or kernel timing is

@@ -239,7 +239,7 @@ def test_linear_gpt2_qkv_config_bit_exact():
     run_case(par, ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g), L.d_out, L.d_in, 0, 1e-3, L.name)
 
 
-def check_blocks(par, plan, layers, blocks_of, seed, keys=None, s=None):
+def check_blocks(par, plan, layers, blocks_of, seed, keys=None, s=None, on_the_fly=()):
     """Full-size layers in the configuration the benchmark runs: the device computes every output
     block, the oracle the sampled ones; those must agree on every residue, and decrypt correctly."""
     if s is None:
@@ -257,6 +257,11 @@ def check_blocks(par, plan, layers, blocks_of, seed, keys=None, s=None):
             expect = ckks.linear(par, plan, cts, W, keys, blocks=blocks)
             w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), L.d_out, L.d_in)
             out = g.linear(cts, W, L.d_out, L.d_in, weights=w)
+            if L.name in on_the_fly:      # the same call with the weights encoded on the fly
+                fly = g.to_host_u64(g.linear(cts, W, L.d_out, L.d_in))
+                for p in blocks:
+                    assert np.array_equal(fly[p], expect[p]), (L.name, p, "on the fly")
+                del fly
             low = g.empty_u64(n_out, 2, par.r - 1, par.N)
             scale = g.bf.bf_rescale(g.ctx, out, low, n_out, par.r, par.scale * par.scale)
             got, low = g.to_host_u64(out), g.to_host_u64(low)
@@ -286,7 +291,7 @@ def test_qwen3_layer_shapes_sampled_blocks():
     plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
     # distinct shapes of the layer: q (1024->2048), o (2048->1024), gate (1024->3072), down (3072->1024)
     pick = [L for L in w.layers if L.name in ("q", "o", "gate", "down")]
-    check_blocks(par, plan, pick, lambda L, n_out: [(3 * n_out) // 4 if n_out > 1 else 0], 12)
+    check_blocks(par, plan, pick, lambda L, n_out: [(3 * n_out) // 4 if n_out > 1 else 0], 12, on_the_fly=("o",))
 
 
 def test_llama3_layer_shapes_sampled_blocks():
@@ -295,7 +300,7 @@ def test_llama3_layer_shapes_sampled_blocks():
     plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
     # k (4096->1024) in full, one block of gate (4096->14336)
     pick = [L for L in w.layers if L.name in ("k", "gate")]
-    check_blocks(par, plan, pick, lambda L, n_out: [n_out - 1], 13)
+    check_blocks(par, plan, pick, lambda L, n_out: [n_out - 1], 13, on_the_fly=("k",))
 
 
 def test_linear_with_the_papers_own_parameter_set():
@@ -435,6 +440,33 @@ def test_fold_of_more_ciphertexts_than_one_key_switch_batch():
         got = g.to_host_u64(d)
         for t in (0, 1, 63, 64, 69):
             assert np.array_equal(got[t], ckks.fold_in_ciphertext(par, plan, cts[t], keys)), t
+    finally:
+        g.close()
+
+
+def test_fallback_path_in_several_rounds_of_its_scratch():
+    # the on-the-fly path encodes output groups in rounds bounded by a scratch size: one group per round,
+    # two per round with a ragged last round, and everything in one round must give the oracle's residues
+    par = oracle_params("n12")
+    plan = ckks.Plan(64, 4, 4, 4)
+    d_out, d_in = 150, 130                        # 3 output blocks x 4 giant steps = 12 groups of 3 x 4 terms
+    s = ckks.keygen(par, 31)
+    keys = ckks.make_rotation_keys(par, s, plan, 31)
+    W = wl.gen_weights(31, "rounds", d_out, d_in)
+    x = wl.gen_activation(31, "rounds", d_in)
+    cts = ckks.encrypt_vector(par, plan, s, x, 31)
+    expect = ckks.linear(par, plan, cts, W, keys)
+    group_bytes = 3 * 4 * par.r * par.N * 8
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys)
+        for bound in (1, 5 * group_bytes + 17, 2 * group_bytes, 1 << 32):
+            g.bf.bf_set_encode_scratch(g.ctx, bound)
+            got = g.to_host_u64(g.linear(cts, W, d_out, d_in))
+            for p in range(3):
+                assert np.array_equal(got[p], expect[p]), (bound, p)
+        with pytest.raises(g.bf.BifrostError):
+            g.bf.bf_set_encode_scratch(g.ctx, 0)
     finally:
         g.close()
 
