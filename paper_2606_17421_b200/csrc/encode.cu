@@ -202,6 +202,13 @@ __device__ __forceinline__ double diag_value_at(const DiagBatch& db, const DiagP
     return (double)__ldg(&db.W[(size_t)row * db.d_in + col]);
 }
 
+// Shared-memory slot of point li of chunk `lane` in the contiguous pass: 16-byte elements, eight to a row
+// of banks; XOR-ing the column with the row number keeps the stride-4 and stride-32 sets of a quarter
+// warp on distinct columns (with plain or padded indexing the first two groups conflict 4- and 2-way).
+__device__ __forceinline__ int fft_swz(int lane, int li, int log_len) {
+    return (lane << log_len) + (li ^ ((li >> 3) & 7));
+}
+
 template <bool CONTIG, int LOG_LEN, int LOG_LANES, int LOG_OTHER, int GI>
 __device__ __forceinline__ void fft_group(const EncodeTables& tab, const DiagBatch& db, const DiagPos& dp, double2* smc,
                                           double2* __restrict__ buf, i64* __restrict__ cp, int* __restrict__ overflow,
@@ -213,7 +220,6 @@ __device__ __forceinline__ void fft_group(const EncodeTables& tab, const DiagBat
     constexpr u32 n = 1u << (LOG_LEN + LOG_OTHER);
     constexpr int STEP = 1 << LOG_STEP;
     constexpr int NSETS = (LEN * LANES) >> K;
-    constexpr int PITCH = LEN + (CONTIG ? 1 : 0);
     constexpr bool FIRST = GI == 0, LAST = GI == NG - 1;
     constexpr int LOG_UNIT = CONTIG ? 0 : LOG_OTHER;      // global index distance of one local index step
     for (int w = threadIdx.x; w < NSETS; w += blockDim.x) {
@@ -235,7 +241,7 @@ __device__ __forceinline__ void fft_group(const EncodeTables& tab, const DiagBat
                     e[i] = buf[gidx];
                 }
             } else {
-                e[i] = CONTIG ? smc[lane * PITCH + li] : smc[li * LANES + lane];
+                e[i] = CONTIG ? smc[fft_swz(lane, li, LOG_LEN)] : smc[li * LANES + lane];
             }
         }
 #pragma unroll
@@ -279,7 +285,7 @@ __device__ __forceinline__ void fft_group(const EncodeTables& tab, const DiagBat
                     }
                 }
             } else {
-                if (CONTIG) smc[lane * PITCH + li] = e[i];
+                if (CONTIG) smc[fft_swz(lane, li, LOG_LEN)] = e[i];
                 else smc[li * LANES + lane] = e[i];
             }
         }
@@ -313,7 +319,7 @@ static cudaError_t launch_encode_fixed(const RingHost& ring, const EncodeTables&
     constexpr int LOG_A = 8, LOG_LANES_A = 3, LOG_LANES_B = 11 - LOG_B;
     {
         dim3 grid((1u << LOG_B) >> LOG_LANES_A, db.count);
-        constexpr size_t smem = (size_t)((1 << LOG_A) + 1) * (1 << LOG_LANES_A) * sizeof(double2);
+        constexpr size_t smem = (size_t)(1 << LOG_A) * (1 << LOG_LANES_A) * sizeof(double2);
         ProfScope prof(ring.prof, CAT_ENCODE_FFT_A, stream);
         encode_fft_fixed<true, LOG_A, LOG_LANES_A, LOG_B><<<grid, 256, smem, stream>>>(tab, db, fft_scratch, coeff_out,
                                                                                       overflow_flag);
