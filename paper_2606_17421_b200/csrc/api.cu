@@ -879,9 +879,8 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     } else {
         // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them
         const size_t group_bytes = (size_t)n_terms * r * N * 8;
-        u32 groups = (u32)(ctx->encode_scratch_bytes / group_bytes);
-        if (groups < 1) groups = 1;
-        if (groups > n_pj) groups = n_pj;
+        const size_t fit = ctx->encode_scratch_bytes / group_bytes;
+        const u32 groups = fit < 1 ? 1u : fit > (size_t)n_pj ? n_pj : (u32)fit;
         const TileLayout jl = mac_tile_layout(ctx->ring, groups, n_terms);
         TRY(ensure(ctx, ctx->ptjit, mac_tile_bytes(ctx->ring, jl)));
         for (u32 pj0 = 0; pj0 < n_pj; pj0 += groups) {
