@@ -125,7 +125,6 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
     u64* xs = (u64*)(mac_smem + MAC_RING_BYTES);                   // [n_terms][2][TN]
     u64* full = xs + (size_t)n_terms * 2 * TN;                     // [MAC_MAX_STAGES]
     u64* empty = full + MAC_MAX_STAGES;                            // [MAC_MAX_STAGES]
-    u64* xbar = empty + MAC_MAX_STAGES;
     // Work units (tile, prime, slice of the output groups) are numbered tile-fastest.  The first n_whole
     // blocks take one unit each; the units after them (the part that would be a thin last wave) are each
     // cut into tail_split blocks over their output groups, so that the last wave is short instead.
@@ -161,7 +160,6 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
             mbar_init(&full[s], 1);                                // the producer's arrive.expect_tx
             mbar_init(&empty[s], MAC_CONSUMERS / 32);              // one arrival per consumer warp
         }
-        mbar_init(xbar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -217,11 +215,7 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         // cached weights do not depend on the previous kernel: fill the ring before waiting for it
         const u32 early = early_weights ? min(n_items, n_stages) : 0u;
         while (k < early) issue_stage();
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (lane == 0) mbar_expect_tx(xbar, n_terms * 2 * TN * 8);
-        __syncwarp();
-        for (u32 e = lane; e < n_terms * 2; e += 32)                // X tile: [term][component] segments
-            bulk_g2s(xs + (size_t)e * TN, x + ((size_t)e * r + i) * N + n0, TN * 8, xbar);
+        asm volatile("griddepcontrol.wait;" ::: "memory");     // weights encoded on the fly come from the previous kernel
         while (k < n_items) {
             if (k >= n_stages) mbar_wait(&empty[slot], phase ^ 1, error_flag);   // consumers left this slot
             issue_stage();
@@ -234,10 +228,32 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
     const u64 q = R.q[i];
     const u32 qneg32 = (u32)R.qneg[i];
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    mbar_wait(xbar, 0, error_flag);
-    if (KARA) {
-        // split the resident X words into limbs, each exactly once, then let every consumer see them
-        for (u32 e = l; e < n_terms * 2; e += PL) xs[(size_t)e * TN + c] = limb_split(xs[(size_t)e * TN + c], KARA_L);
+    {
+        // X tile: [term][component] segments of TN words.  Its latency is exposed at the start of every block
+        // (measured: 2 to 4 us of a 17 us block), so all of a thread's words are requested in one batch of
+        // plain coalesced loads (one round trip; 32 bulk copies of 1 KB took 3.5 us and a separate split pass
+        // 0.9 us), split into limbs on the way, each word exactly once, then made visible to all consumers
+        const u64* xg = x + (size_t)i * N + n0 + c;
+        const u32 n_seg = n_terms * 2;
+        u32 e = l;
+        for (; e + 15 * PL < n_seg; e += 16 * PL) {
+            u64 v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = __ldg(xg + (size_t)(e + j * PL) * r * N);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) xs[(size_t)(e + j * PL) * TN + c] = KARA ? limb_split(v[j], KARA_L) : v[j];
+        }
+        for (; e + 3 * PL < n_seg; e += 4 * PL) {
+            u64 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = __ldg(xg + (size_t)(e + j * PL) * r * N);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) xs[(size_t)(e + j * PL) * TN + c] = KARA ? limb_split(v[j], KARA_L) : v[j];
+        }
+        for (; e < n_seg; e += PL) {
+            const u64 v = __ldg(xg + (size_t)e * r * N);
+            xs[(size_t)e * TN + c] = KARA ? limb_split(v, KARA_L) : v;
+        }
         asm volatile("bar.sync 1, %0;" ::"n"(MAC_CONSUMERS) : "memory");
     }
     KaraAcc k0, k1;
