@@ -196,6 +196,9 @@ struct LimbAcc {
         return t >= q ? t - q : t;
     }
 
+    // The same by two 32-bit rounds (redc_2x32 below): no 64-bit high product.
+    __device__ __forceinline__ u64 reduce_mont32(u64 q, u32 qneg32) const;
+
     __device__ __forceinline__ void reset_to(u64 v) {
         lo = v; mid = 0; hi = 0; lo_c = 0; mid_c = 0;
     }
@@ -317,6 +320,8 @@ struct PolyBatch {
     const u32* scatter;           // forward only: final store goes to scatter_dst[scatter[(o / scatter_div) * N + n]]
     u32 scatter_div;              //   instead of dst[n] (same polynomial strides as dst)
     u64* scatter_dst;
+    u32 scatter_mont;             //   and the stored value is the result times 2^64 mod q (rotation keys: the inner
+                                  //   product ends in a Montgomery reduction)
     u32 split_bits;               // L > 0: the NTT-domain side of the transform is stored as two L-bit-aligned
                                   // limbs per word, (v >> L) << 32 | (v & (2^L - 1)); forward writes, inverse reads it
 };
@@ -376,6 +381,14 @@ __device__ __forceinline__ u64 redc_2x32(u64 H, u64 L, u64 q, u32 qneg32) {
         : "r"(q0), "r"(q1), "r"(qneg32));
     const u64 t = ((u64)h1 << 32) | h0;
     return t >= q ? t - q : t;
+}
+
+template <bool SMALL>
+__device__ __forceinline__ u64 LimbAcc<SMALL>::reduce_mont32(u64 q, u32 qneg32) const {
+    const u64 L = lo + (mid << 32);
+    const u64 carry = L < lo ? 1ull : 0ull;
+    const u64 H = (u64)lo_c + (mid >> 32) + ((u64)mid_c << 32) + hi + carry;
+    return redc_2x32(H, L, q, qneg32);
 }
 
 }  // namespace bf

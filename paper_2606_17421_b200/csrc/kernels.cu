@@ -525,7 +525,7 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 // tiles beat 256 by 3 %, 64 lose 4 %).
 constexpr int KI_TILE = 128;
 
-__global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
+__global__ void __launch_bounds__(KI_TILE, 10) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
                                                                     const u64* __restrict__ dig,
                                                                     const u64* __restrict__ keys, u64* __restrict__ u,
                                                                     u32 small_ok, int* __restrict__ error_flag) {
@@ -559,7 +559,8 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
     mbar_wait(bar, 0, error_flag);
-    const u64 q = R.q[m], mu = R.mu[m], c64 = R.c64[m], c64s = R.c64s[m];
+    const u64 q = R.q[m];
+    const u32 qneg32 = (u32)R.qneg[m];
     u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
     if (m < r && small_ok) {
         LimbAcc<true> a0, a1;
@@ -568,8 +569,8 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
             a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
             a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
         }
-        up[0] = a0.reduce(q, mu, c64, c64s);
-        up[(size_t)nb * N] = a1.reduce(q, mu, c64, c64s);
+        up[0] = a0.reduce_mont32(q, qneg32);             // the keys carry a factor 2^64
+        up[(size_t)nb * N] = a1.reduce_mont32(q, qneg32);
     } else {
         LimbAcc<false> a0, a1;
         for (u32 j = 0; j < r; ++j) {
@@ -577,8 +578,8 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
             a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
             a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
         }
-        up[0] = a0.reduce(q, mu, c64, c64s);
-        up[(size_t)nb * N] = a1.reduce(q, mu, c64, c64s);
+        up[0] = a0.reduce_mont32(q, qneg32);             // the keys carry a factor 2^64
+        up[(size_t)nb * N] = a1.reduce_mont32(q, qneg32);
     }
 }
 

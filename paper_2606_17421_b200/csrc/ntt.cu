@@ -628,7 +628,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 const u32* sc = B.scatter + (size_t)(o / B.scatter_div) * R.N + chunk * LEN + 4 * s;
                 u64* sd = B.scatter_dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sd[sc[i]] = v4[i];
+                for (int i = 0; i < 4; ++i) sd[sc[i]] = B.scatter_mont ? mul_shoup(v4[i], R.c64[mod], R.c64s[mod], q) : v4[i];
                 continue;
             }
             ulonglong2* gp = (ulonglong2*)(gdst + 4 * s);
@@ -875,6 +875,7 @@ cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B0, u32 n_o
     B.scatter = scatter;
     B.scatter_div = scatter_div;
     B.scatter_dst = final_dst;
+    B.scatter_mont = 1;           // (the only permuted store is that of the rotation keys)
     return launch_contig<true>(ring, B, n_polys, stream);
 }
 
