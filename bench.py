@@ -31,8 +31,8 @@ UNIT = "ms"
 # see profiles/ for the capture each figure comes from.  None = not captured yet.
 NCU_TRAFFIC_BYTES = {
     # from the ncu capture summarised under profiles/: dram__bytes_read.sum + dram__bytes_write.sum per launch
-    "gpt2_qkv": {"mac": 422.9e6,                       # 411.1 MB read + 11.8 MB written
-                 "key_inner_product": 373.5e6,         # 747 MB per step (two lanes' launches), over the two launches of
+    "gpt2_qkv": {"mac": 423.7e6,                       # 411.1 MB read + 12.6 MB written
+                 "key_inner_product": 373.1e6,         # 746 MB per step (two lanes' launches), over the two launches of
                                                        #   the serialised timing pass
                  "ntt_fwd_strided": 23.8e6,            # mean of the eight captured forward launches (both passes)
                  "ntt_inv_contig": 11.0e6},            # mean of the eight captured inverse launches (both passes)

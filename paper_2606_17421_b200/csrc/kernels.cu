@@ -521,8 +521,10 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 // Bulk-copy version: a block owns one (rotation, modulus, tile of 128 coefficients).  Its 3r operand
 // segments (digit, key.b, key.a for every digit j; 1 KB each) are fetched by asynchronous bulk
 // copies into shared memory in one go, so the number of bytes in flight does not depend on
-// registers; eight blocks per SM overlap one block's arithmetic with the others' copies (measured: 128-coefficient
-// tiles beat 256 by 3 %, 64 lose 4 %).
+// registers; ten blocks per SM overlap one block's arithmetic with the others' copies (measured: 128-coefficient
+// tiles beat 256 by 3 %, 64 lose 2 to 4 %).  The keys are resident in Montgomery form (times 2^64 mod q), so the
+// sum of the r products ends in the two-round 32-bit Montgomery reduction: r * max digit < 2^64 keeps it below
+// q * 2^64.
 constexpr int KI_TILE = 128;
 
 __global__ void __launch_bounds__(KI_TILE, 10) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
