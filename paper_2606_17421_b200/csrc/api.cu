@@ -796,6 +796,12 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     // lanes: the rotations of a stage are dealt out to up to n_lanes independent chains
     int lanes = ctx->n_lanes < 1 ? 1 : (ctx->n_lanes > bf_ctx::MAX_LANES ? bf_ctx::MAX_LANES : ctx->n_lanes);
     TRY(ensure_lanes(ctx));
+    // per stage: splitting pays when a stage's kernels are too small to fill the GPU by themselves and there is
+    // enough to split (measured side by side per layer shape at N = 2^15: with 3 giant rotations, or with 30 and
+    // more baby rotations, the stage runs 1 to 2 % faster as one chain; 9 to 18 giant rotations and 15 baby
+    // rotations run 1.5 to 3 % faster as two)
+    const int lanes_giant = (lanes > 1 && n_giant >= 6) ? lanes : 1;
+    const int lanes_baby = (lanes > 1 && in_batch * (b - 1) <= 24) ? lanes : 1;
     const u32 baby_rots = in_batch * (b - 1);
     const u32 baby_per_lane = cdiv(baby_rots > 0 ? baby_rots : 1, (u32)lanes);
     u32 giant_per_lane = cdiv(n_giant > 0 ? n_giant : 1, (u32)lanes);     // rotations a lane holds at once
@@ -849,7 +855,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
                       X + (size_t)q0 * b * ctw + (size_t)r * N, (long long)b * ctw));
             // the rotations of the batch, dealt out to the lanes in contiguous runs
             const u32 n_rot = qn * (b - 1);
-            const u32 per = cdiv(n_rot, (u32)lanes);
+            const u32 per = cdiv(n_rot, (u32)lanes_baby);
             const int used = (int)cdiv(n_rot, per);
             TRY(fork_lanes(ctx, used));
             for (int c = 0; c < used; ++c) {
@@ -895,13 +901,15 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
 
     // ---- giant steps: rotate A[j][p] by j*b*tau (full key switch each), then sum over j
     if (n_giant) {
-        const u32 per = cdiv(n_giant, (u32)lanes);
+        const u32 per = cdiv(n_giant, (u32)lanes_giant);
         const int used = (int)cdiv(n_giant, per);
+        // a single chain may use the buffers of all lanes (they are contiguous)
+        const u32 giant_chunk = lanes_giant == 1 ? giant_per_lane * (u32)lanes : giant_per_lane;
         TRY(fork_lanes(ctx, used));
         for (int c = 0; c < used; ++c) {
             const u32 lane_end = (u32)(c + 1) * per < n_giant ? (u32)(c + 1) * per : n_giant;
-            for (u32 rho0 = (u32)c * per; rho0 < lane_end; rho0 += giant_per_lane) {
-                const u32 cnt = (lane_end - rho0 < giant_per_lane) ? lane_end - rho0 : giant_per_lane;
+            for (u32 rho0 = (u32)c * per; rho0 < lane_end; rho0 += giant_chunk) {
+                const u32 cnt = (lane_end - rho0 < giant_chunk) ? lane_end - rho0 : giant_chunk;
                 const u64* Asrc = A + (size_t)(n_out + rho0) * ctw;      // ciphertexts with j >= 1 are contiguous
                 memset(&B, 0, sizeof(B));
                 B.src = Asrc + (size_t)r * N;                            // c1 of each
