@@ -144,7 +144,9 @@ int bf_set_dependent_launch(bf_ctx* ctx, int on);
  * batch, and then the giant rotations, out to n_lanes chains (inner product, then division by the
  * special prime) that run on streams of the library's own between a fork from and a join into the
  * context's stream, so that one chain's HBM-bound inner product overlaps another chain's
- * arithmetic-bound transforms.  Results do not depend on n_lanes.  1 <= n_lanes <= 4 (default 2);
+ * arithmetic-bound transforms.  n_lanes is an upper bound: a stage is split only where that was
+ * measured to pay (at most 24 baby rotations in the batch; at least 6 giant rotations), otherwise it
+ * runs as one chain.  Results do not depend on n_lanes.  1 <= n_lanes <= 4 (default 2);
  * bf_set_lanes drops the stored graphs.  The paper has no counterpart. */
 int bf_set_lanes(bf_ctx* ctx, int n_lanes);
 
