@@ -145,7 +145,8 @@ int bf_set_dependent_launch(bf_ctx* ctx, int on);
  * special prime) that run on streams of the library's own between a fork from and a join into the
  * context's stream, so that one chain's HBM-bound inner product overlaps another chain's
  * arithmetic-bound transforms.  n_lanes is an upper bound: a stage is split only where that was
- * measured to pay (at most 24 baby rotations in the batch; at least 6 giant rotations), otherwise it
+ * measured to pay (at most 24 baby rotations in the batch; 6 to 20 giant rotations; counts weighted
+ * by N / 2^15 above that ring size), otherwise it
  * runs as one chain.  Results do not depend on n_lanes.  1 <= n_lanes <= 4 (default 2);
  * bf_set_lanes drops the stored graphs.  The paper has no counterpart. */
 int bf_set_lanes(bf_ctx* ctx, int n_lanes);

@@ -799,9 +799,12 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     // per stage: splitting pays when a stage's kernels are too small to fill the GPU by themselves and there is
     // enough to split (measured side by side per layer shape at N = 2^15: with 3 giant rotations, or with 30 and
     // more baby rotations, the stage runs 1 to 2 % faster as one chain; 9 to 18 giant rotations and 15 baby
-    // rotations run 1.5 to 3 % faster as two)
-    const int lanes_giant = (lanes > 1 && n_giant >= 6) ? lanes : 1;
-    const int lanes_baby = (lanes > 1 && in_batch * (b - 1) <= 24) ? lanes : 1;
+    // rotations run 1.5 to 3 % faster as two; more than 18 giant rotations were not measured and stay one chain)
+    // (rotation counts weighted by the ring size relative to 2^15: at N = 2^16 a LLaMA-3-8B layer ran 0.8 % faster
+    // with its 12 giant rotations per call as one chain)
+    const u32 ring_weight = N > (1u << 15) ? N >> 15 : 1u;
+    const int lanes_giant = (lanes > 1 && n_giant >= 6 && n_giant * ring_weight <= 20) ? lanes : 1;
+    const int lanes_baby = (lanes > 1 && in_batch * (b - 1) * ring_weight <= 24) ? lanes : 1;
     const u32 baby_rots = in_batch * (b - 1);
     const u32 baby_per_lane = cdiv(baby_rots > 0 ? baby_rots : 1, (u32)lanes);
     u32 giant_per_lane = cdiv(n_giant > 0 ? n_giant : 1, (u32)lanes);     // rotations a lane holds at once
