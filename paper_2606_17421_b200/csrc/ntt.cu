@@ -799,7 +799,7 @@ static cudaError_t launch_strided(const RingHost& ring, const PolyBatch& B, u32 
                 case 5: launch_shared_src_t<LOAD, 5, 6>(ring, B, n_outer, stream); break;
                 case 6: launch_shared_src_t<LOAD, 6, 5>(ring, B, n_outer, stream); break;
                 case 7: launch_shared_src_t<LOAD, 7, 3>(ring, B, n_outer, stream); break;
-                case 8: launch_shared_src_t<LOAD, 8, 4>(ring, B, n_outer, stream); break;
+                case 8: launch_shared_src_t<LOAD, 8, 3>(ring, B, n_outer, stream); break;
                 default: return cudaErrorInvalidValue;
             }
             return cudaGetLastError();
