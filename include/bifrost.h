@@ -195,7 +195,9 @@ int bf_negacyclic_mul(bf_ctx* ctx, const uint64_t* a, const uint64_t* b, uint64_
  * transform-domain temporaries live in a fixed array inside the library's device image, which
  * every GPU that loads the library holds (8 MiB) until the process exits.
  *   Limit: ceil(n_polys / (r+1)) * (r+1) * N <= bf_noalloc_max_words() (2^19 words); larger
- *   requests return BF_ERR_TOO_LARGE and enqueue nothing.
+ *   requests return BF_ERR_TOO_LARGE and enqueue nothing.  With N = 2^15 and r = 7 that is two
+ *   groups of 8 polynomials; a context with N = 2^16 and r = 9 (10 x 65536 words per group) never
+ *   fits, whatever n_polys is.
  *   The first call on a device resolves the array's device address (cudaGetSymbolAddress); make
  *   that call with the context's device current and before starting any stream capture.
  *   All calls, from any context, share the one array, which keeps the previous call's contents;

@@ -341,14 +341,6 @@ int orc_encode_real_batch(const double* z, u32 count, u32 N, double scale, i64* 
     return status;
 }
 
-/* Signed coefficients -> residues in [0, q). */
-void orc_reduce_i64(const i64* m, u64* out, u32 N, u64 q) {
-    for (u32 k = 0; k < N; k++) {
-        i64 v = m[k] % (i64)q; /* C remainder has the sign of the dividend */
-        out[k] = v < 0 ? (u64)(v + (i64)q) : (u64)v;
-    }
-}
-
 int orc_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

@@ -238,6 +238,7 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
         return s;
     };
     if (cudaGetDevice(&ctx->device) != cudaSuccess) return fail(BF_ERR_CUDA);
+    ctx->ring.device = ctx->device;
 
     std::vector<double> enc_consts((size_t)MAX_MODULI * ENC_CONSTS, 0.0);
     RingDev& R = ctx->ring.dev;
@@ -423,28 +424,42 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
 }
 
 // ------------------------------------------------------------------------------------------------
-extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_t n_keys, const uint64_t* keys) {
-    if (!ctx || (n_keys && (!rot_steps || !keys))) return BF_ERR_INVALID_ARG;
-    const u32 N = ctx->N, r = ctx->r, nb = r + 1, n = N / 2;
-    CK(cudaStreamSynchronize(ctx->stream));
+// Drops the resident keys and everything that refers to them: the step -> key map, the permutation tables and
+// the captured launch sequences (they hold the addresses of the freed arrays).
+static void drop_eval_keys(bf_ctx* ctx) {
+    destroy_graphs(ctx);
+    ctx->epoch++;
     cudaFree(ctx->keys);
     cudaFree(ctx->perms);
     ctx->keys = nullptr;
     ctx->perms = nullptr;
     ctx->key_of_steps.clear();
     ctx->n_keys = 0;
+}
+
+extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_t n_keys, const uint64_t* keys) {
+    if (!ctx || (n_keys && (!rot_steps || !keys))) return BF_ERR_INVALID_ARG;
+    const u32 N = ctx->N, r = ctx->r, nb = r + 1, n = N / 2;
+    CK(cudaStreamSynchronize(ctx->stream));
+    drop_eval_keys(ctx);
     if (n_keys == 0) return BF_OK;
+    // every failure below leaves the context without keys (BF_ERR_MISSING_KEY on the next rotation), never
+    // with a half-built set
+    auto fail = [&](int code) {
+        cudaGetLastError();
+        drop_eval_keys(ctx);
+        return code;
+    };
     const size_t key_words = (size_t)r * 2 * nb * N;
-    cudaError_t e = cudaMalloc(&ctx->keys, key_words * n_keys * sizeof(u64));
-    if (e != cudaSuccess) { cudaGetLastError(); ctx->keys = nullptr; return BF_ERR_OOM; }
-    e = cudaMalloc(&ctx->perms, (size_t)n_keys * N * sizeof(u32));
-    if (e != cudaSuccess) { cudaGetLastError(); ctx->perms = nullptr; return BF_ERR_OOM; }
+    if (cudaMalloc(&ctx->keys, key_words * n_keys * sizeof(u64)) != cudaSuccess) { ctx->keys = nullptr; return fail(BF_ERR_OOM); }
+    if (cudaMalloc(&ctx->perms, (size_t)n_keys * N * sizeof(u32)) != cudaSuccess) { ctx->perms = nullptr; return fail(BF_ERR_OOM); }
     // permutation tables: position i of the transform holds the evaluation at psi^(2*brev(i)+1);
     // a(X) -> a(X^g) maps it to the evaluation at exponent (2*brev(i)+1)*g mod 2N, so the rotated
     // polynomial is out[i] = in[perm[i]].  The keys are stored as key'[perm[i]] = key[i], which lets
     // the inner product run in the un-rotated index space; the rotation is applied at the very end
     // as the scatter out[pinv[i]] = v'[i], pinv = perm^{-1}.  Only pinv stays on the device.
     std::vector<u32> perms((size_t)n_keys * N), pinvs((size_t)n_keys * N);
+    std::map<u32, int> key_of_steps;
     for (u32 t = 0; t < n_keys; ++t) {
         const u32 steps = rot_steps[t] % n;
         u64 g = 1;
@@ -455,22 +470,19 @@ extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_
             perms[(size_t)t * N + i] = pi;
             pinvs[(size_t)t * N + pi] = i;
         }
-        ctx->key_of_steps[steps] = (int)t;
+        key_of_steps[steps] = (int)t;
     }
     u32* perm_dev = nullptr;
-    e = cudaMalloc(&perm_dev, perms.size() * sizeof(u32));
-    if (e != cudaSuccess) { cudaGetLastError(); return BF_ERR_OOM; }
+    if (cudaMalloc(&perm_dev, perms.size() * sizeof(u32)) != cudaSuccess) return fail(BF_ERR_OOM);
     if (cudaMemcpy(perm_dev, perms.data(), perms.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(ctx->perms, pinvs.data(), pinvs.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess) {
         ctx->cuda_msg = "cudaMemcpy of the permutation tables failed";
-        cudaGetLastError();
         cudaFree(perm_dev);
-        return BF_ERR_CUDA;
+        return fail(BF_ERR_CUDA);
     }
     PolyBatch B;
     memset(&B, 0, sizeof(B));
     B.src = keys;
-    B.dst = ctx->keys;
     B.src_so = B.dst_so = (long long)nb * N;
     B.src_sm = B.dst_sm = N;
     B.n_m = nb;
@@ -480,16 +492,18 @@ extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_
     // reads it and stores, permuted, into the resident key array (a permuted store in place would
     // overwrite points other blocks have not read yet).
     u64* stage = nullptr;
-    e = cudaMalloc(&stage, key_words * n_keys * sizeof(u64));
-    if (e != cudaSuccess) { cudaGetLastError(); cudaFree(perm_dev); return BF_ERR_OOM; }
+    if (cudaMalloc(&stage, key_words * n_keys * sizeof(u64)) != cudaSuccess) { cudaFree(perm_dev); return fail(BF_ERR_OOM); }
     B.dst = stage;
     B.scatter = nullptr;
     cudaError_t ne = ntt_forward_split(ctx->ring, B, n_keys * r * 2, LOAD_REDUCE, ctx->keys, perm_dev, 2 * r, ctx->stream);
     cudaError_t se = cudaStreamSynchronize(ctx->stream);
     cudaFree(stage);
     cudaFree(perm_dev);
-    CK(ne);
-    CK(se);
+    if (ne != cudaSuccess || se != cudaSuccess) {
+        ctx->cuda_msg = std::string("key transform: ") + cudaGetErrorString(ne != cudaSuccess ? ne : se);
+        return fail(BF_ERR_CUDA);
+    }
+    ctx->key_of_steps.swap(key_of_steps);
     ctx->n_keys = n_keys;
     ctx->epoch++;
     return BF_OK;
@@ -503,7 +517,7 @@ extern "C" int bf_set_cache_budget(bf_ctx* ctx, uint64_t bytes) {
 
 extern "C" uint64_t bf_cache_bytes_used(const bf_ctx* ctx) { return ctx ? ctx->cache_used : 0; }
 
-static u32 cdiv(u32 a, u32 b) { return (a + b - 1) / b; }
+static u32 cdiv(u32 a, u32 b) { return (u32)(((u64)a + b - 1) / b); }
 
 extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
     if (!ctx) return 0;
@@ -808,7 +822,9 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     const u32 baby_rots = in_batch * (b - 1);
     const u32 baby_per_lane = cdiv(baby_rots > 0 ? baby_rots : 1, (u32)lanes);
     u32 giant_per_lane = cdiv(n_giant > 0 ? n_giant : 1, (u32)lanes);     // rotations a lane holds at once
-    if (giant_per_lane > cdiv(gb, (u32)lanes)) giant_per_lane = cdiv(gb, (u32)lanes);
+    // (rounded down: a single chain uses the buffers of all lanes, giant_per_lane * lanes rotations per launch,
+    // and a launch takes at most MAX_ROT_BATCH)
+    if (giant_per_lane > gb / (u32)lanes) giant_per_lane = gb / (u32)lanes;
     if (giant_per_lane < 1) giant_per_lane = 1;
     const u32 rot_per_lane = baby_per_lane > giant_per_lane ? baby_per_lane : giant_per_lane;
     u32 n_dig_sets = giant_per_lane * (u32)lanes;       // digit sets alive at once
@@ -913,6 +929,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             const u32 lane_end = (u32)(c + 1) * per < n_giant ? (u32)(c + 1) * per : n_giant;
             for (u32 rho0 = (u32)c * per; rho0 < lane_end; rho0 += giant_chunk) {
                 const u32 cnt = (lane_end - rho0 < giant_chunk) ? lane_end - rho0 : giant_chunk;
+                if (cnt > (u32)MAX_ROT_BATCH) return BF_ERR_INVALID_ARG;   // (cannot happen: see giant_per_lane)
                 const u64* Asrc = A + (size_t)(n_out + rho0) * ctw;      // ciphertexts with j >= 1 are contiguous
                 memset(&B, 0, sizeof(B));
                 B.src = Asrc + (size_t)r * N;                            // c1 of each
@@ -1370,6 +1387,7 @@ extern "C" int bf_negacyclic_mul_noalloc(bf_ctx* ctx, const uint64_t* a, const u
                                          uint32_t n_polys) {
     if (!ctx || !a || !b || !out || !n_polys) return BF_ERR_INVALID_ARG;
     const u32 N = ctx->N, nb = ctx->r + 1;
+    if ((u64)n_polys * N > BF_NOALLOC_WORDS) return BF_ERR_TOO_LARGE;   // (before any 32-bit rounding of the count)
     const u32 n_outer = cdiv(n_polys, nb);
     const size_t words = (size_t)n_outer * nb * N;               // batch padded to whole groups of r+1 primes
     if (words > BF_NOALLOC_WORDS) return BF_ERR_TOO_LARGE;

@@ -45,7 +45,10 @@ struct RingHost {
     Profiler* prof = nullptr;
     bool dependent_launch = true;     // launch the kernels of a call with programmatic stream serialisation
     bool compact_cache = false;       // encode plaintexts in the narrowest word format each prime allows
+    int device = 0;                   // the CUDA device of the context (kernel attributes are set once per device)
 };
+constexpr int MAX_DEVICES = 64;
+inline int device_slot(const RingHost& ring) { return ring.device >= 0 && ring.device < MAX_DEVICES ? ring.device : 0; }
 
 // Launch with programmatic stream serialisation: the grid may be scheduled while the previous kernel
 // of the stream drains; every kernel launched this way calls grid_dependency_enter() before it touches

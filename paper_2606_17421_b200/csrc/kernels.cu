@@ -415,12 +415,13 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     const size_t smem = (size_t)MAC_RING_BYTES + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_MAX_STAGES + 1) * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
-    static bool attr_set = false;     // opt in once to the large dynamic shared-memory carve-out
-    if (!attr_set) {
+    const int ds = device_slot(ring);
+    static bool attr_set[MAX_DEVICES] = {false};     // opt in once per device to the large dynamic shared-memory carve-out
+    if (!attr_set[ds]) {
         cudaError_t e = cudaFuncSetAttribute(mac_kernel<KARA, LOG_TN, COMPACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              200 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[ds] = true;
     }
     // slices over output groups: enough blocks to fill the machine several times over
     const u32 tiles = (ring.dev.N >> LOG_TN) * ring.dev.r;
@@ -432,21 +433,20 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     pj_per_block = (pj_per_block + PL - 1) / PL * PL;
     slices = (n_pj + pj_per_block - 1) / pj_per_block;
     // blocks resident at once; when the units leave a thin last wave, cut those units into shorter blocks
-    static int sm_count = 0, per_sm = 0;
-    static size_t per_sm_smem = 0;
+    static int sm_counts[MAX_DEVICES] = {0}, per_sms[MAX_DEVICES] = {0};
+    static size_t per_sm_smems[MAX_DEVICES] = {0};
+    int &sm_count = sm_counts[ds], &per_sm = per_sms[ds];
     if (!sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, ring.device);
         if (sm_count <= 0) sm_count = 148;
     }
-    if (per_sm_smem != smem) {
+    if (per_sm_smems[ds] != smem) {
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mac_kernel<KARA, LOG_TN, COMPACT>, MAC_THREADS, smem) != cudaSuccess ||
             per_sm < 1) {
             cudaGetLastError();
             per_sm = 1;
         }
-        per_sm_smem = smem;
+        per_sm_smems[ds] = smem;
     }
     const u32 slots = (u32)sm_count * (u32)per_sm;
     const u32 units = tiles * slices;
@@ -595,11 +595,11 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
     ProfScope prof(ring.prof, CAT_KEY_INNER, stream);
     const u32 r = ring.dev.r;
     const size_t smem = (size_t)3 * r * KI_TILE * 8 + 16;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[MAX_DEVICES] = {false};     // per device: the attribute belongs to the device's copy of the kernel
+    if (!attr_set[device_slot(ring)]) {
         cudaError_t e = cudaFuncSetAttribute(key_inner_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[device_slot(ring)] = true;
     }
     dim3 grid(rb.n, ring.dev.N / KI_TILE, r + 1);
     return launch_dependent(ring, key_inner_bulk_kernel, grid, dim3(KI_TILE), smem, stream, ring.dev, rb, dig, keys, u,

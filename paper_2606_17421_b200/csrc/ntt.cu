@@ -776,11 +776,11 @@ static void launch_shared_src_t(const RingHost& ring, const PolyBatch& B, u32 n_
     }
     dim3 grid(S, n_outer, (B.n_m + best - 1) / best);
     constexpr size_t smem = (size_t)2 * 8 * (1u << (LOG_R + LOG_LANES)) + (size_t)16 * (1u << LOG_R);
-    static bool attr_set = false;     // opt in once to more than 48 KB of dynamic shared memory
-    if (smem > 48 * 1024 && !attr_set) {
+    static bool attr_set[MAX_DEVICES] = {false};     // opt in once per device to more than 48 KB of dynamic shared memory
+    if (smem > 48 * 1024 && !attr_set[device_slot(ring)]) {
         cudaFuncSetAttribute(ntt_strided_shared_src<LOAD, LOG_R, LOG_LANES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem);
-        attr_set = true;
+        attr_set[device_slot(ring)] = true;
     }
     launch_dependent(ring, ntt_strided_shared_src<LOAD, LOG_R, LOG_LANES>, grid, dim3(NT), smem, stream, ring.dev, B, best);
 }

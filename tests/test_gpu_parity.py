@@ -372,6 +372,71 @@ def test_repeated_calls_replay_a_graph_and_still_read_fresh_inputs():
         g.close()
 
 
+def test_unloading_keys_invalidates_replayed_launch_sequences():
+    # after the keys are dropped, a call that was being replayed from its captured graph must be refused
+    # (the graph holds the addresses of the freed key arrays), and reloading the keys must make it work again
+    par = oracle_params("n12")
+    plan = ckks.Plan(64, 4, 4, 4)
+    s = ckks.keygen(par, 51)
+    keys = ckks.make_rotation_keys(par, s, plan, 51)
+    W = wl.gen_weights(51, "unload", 100, 130)
+    cts = ckks.encrypt_vector(par, plan, s, wl.gen_activation(51, "unload", 130), 51)
+    expect = ckks.linear(par, plan, cts, W, keys)
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys)
+        w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), 100, 130)
+        ct_in = g.to_dev(np.stack(cts))
+        ct_out = g.empty_u64(2, 2, par.r, par.N)
+        for call in range(4):                       # direct, captured, replayed, replayed
+            g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
+        assert np.array_equal(g.to_host_u64(ct_out)[1], expect[1])
+        g.bf.bf_get_kernel_stats(g.ctx)
+        g.bf.bf_load_eval_keys(g.ctx, [], 0, None)
+        with pytest.raises(g.bf.BifrostError) as ei:
+            g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
+        assert ei.value.code == g.bf.BF_ERR_MISSING_KEY
+        assert sum(v[0] for v in g.bf.bf_get_kernel_stats(g.ctx).values()) == 0     # nothing was launched
+        g.load_keys(keys)
+        for call in range(3):
+            ct_out.zero_()
+            g.bf.bf_linear(g.ctx, ct_in, 3, w, None, 100, 130, ct_out, 2)
+        got = g.to_host_u64(ct_out)
+        assert np.array_equal(got[0], expect[0]) and np.array_equal(got[1], expect[1])
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("lanes", [3, 4])
+def test_more_giant_rotations_than_one_launch_holds_with_three_and_four_lanes(lanes):
+    # 30 output blocks x 3 giant steps = 90 rotations: as one chain they go in launches of lanes * floor(64 / lanes)
+    # rotations, which must not exceed the 64 a launch holds (with 3 lanes: 63)
+    par = oracle_params("n12")
+    plan = ckks.Plan(64, 4, 4, 4)
+    d_out, d_in = 1920, 64
+    s = ckks.keygen(par, 52)
+    keys = ckks.make_rotation_keys(par, s, plan, 52)
+    W = wl.gen_weights(52, "lanes", d_out, d_in)
+    cts = ckks.encrypt_vector(par, plan, s, wl.gen_activation(52, "lanes", d_in), 52)
+    blocks = [0, 20, 21, 29]
+    expect = ckks.linear(par, plan, cts, W, keys, blocks=blocks)
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys)
+        g.bf.bf_set_lanes(g.ctx, lanes)
+        w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in)
+        ct_in = g.to_dev(np.stack(cts))
+        ct_out = g.empty_u64(30, 2, par.r, par.N)
+        for call in range(3):                       # direct, captured, replayed
+            ct_out.zero_()
+            g.bf.bf_linear(g.ctx, ct_in, 1, w, None, d_out, d_in, ct_out, 30)
+            got = g.to_host_u64(ct_out)
+            for p in blocks:
+                assert np.array_equal(got[p], expect[p]), (call, p)
+    finally:
+        g.close()
+
+
 @pytest.mark.parametrize("pkey,plan_t,shape", [
     ("n12", (64, 4, 4, 4), (100, 130)),          # tau = 4: rotations by 1 and 2, two output ciphertexts
     ("n12", (32, 32, 1, 1), (70, 50)),           # tau = 32, no other rotation in the plan, three outputs

@@ -147,7 +147,10 @@ def test_rotation_composes(ring64):
 
 # ------------------------------------------------------------------ packing / BSGS (slot level, no crypto)
 
-PLANS = [(64, 1, 8, 8, 2048), (64, 4, 4, 4, 512), (1024, 16, 8, 8, 16384), (1024, 32, 8, 4, 32768), (8, 2, 2, 2, 32)]
+PLANS = [(64, 1, 8, 8, 2048), (64, 4, 4, 4, 512), (1024, 16, 8, 8, 16384), (1024, 32, 8, 4, 32768), (8, 2, 2, 2, 32),
+         # the plans the workloads ship with (ring sizes of their parameter sets)
+         (1024, 16, 16, 4, 16384), (512, 32, 4, 4, 16384), (256, 64, 2, 2, 16384), (128, 128, 1, 1, 16384),
+         (1024, 4, 16, 16, 4096)]
 
 
 @pytest.mark.parametrize("D,tau,b,g,n", PLANS)
