@@ -489,13 +489,16 @@ def inner_sum(params: Params, plan: Plan, Xh: list, encoded: dict, p: int, j: in
     return intt(acc, primes * 2, params)
 
 
-def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blocks=None, encoded=None) -> dict:
+def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blocks=None, encoded=None,
+           X=None) -> dict:
     """Encrypted matrix-vector product (Sec. 4.2 "BSGS matrix-vector multiply"; Alg. 3 FHE_Linear).
 
     cts[q] encrypts pack_input(x[q*D:(q+1)*D]).  For output block p:
         Y_p = sum_{j<g} rot( sum_q sum_{k<b} Pt[p][q][j][k] (*) rot(ct_q, k*tau), j*b*tau )
     where (*) multiplies both ciphertext components by the plaintext in R_{q_i}.  Output level is
-    unchanged, scale multiplies.  Returns {p: ciphertext}."""
+    unchanged, scale multiplies.  Returns {p: ciphertext}.  X, when given, is the list over q of
+    baby_rotations(params, plan, cts[q], keys) computed by an earlier call for the same inputs (several
+    projections that read the same ciphertexts need them only once)."""
     N, r, primes = params.N, params.r, params.primes
     d_out, d_in = W.shape
     n_in, n_out = -(-d_in // plan.D), -(-d_out // plan.D)
@@ -504,7 +507,9 @@ def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blo
     if encoded is None:
         encoded = encode_weights(params, plan, W, blocks)
     # baby steps: X[q][k] = rot(ct_q, k*tau), then to the evaluation domain for the products
-    X = [baby_rotations(params, plan, cts[q], keys) for q in range(n_in)]
+    if X is None:
+        X = [baby_rotations(params, plan, cts[q], keys) for q in range(n_in)]
+    assert len(X) == n_in
     Xh = [[ntt(X[q][k], primes * 2, params) for k in range(plan.b)] for q in range(n_in)]
     out = {}
     for p in blocks:

@@ -239,28 +239,41 @@ def test_linear_gpt2_qkv_config_bit_exact():
     run_case(par, ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g), L.d_out, L.d_in, 0, 1e-3, L.name)
 
 
-def check_blocks(par, plan, layers, blocks_of, seed, keys=None, s=None, on_the_fly=()):
-    """Full-size layers in the configuration the benchmark runs: the device computes every output
-    block, the oracle the sampled ones; those must agree on every residue, and decrypt correctly."""
-    if s is None:
-        s = ckks.keygen(par, seed)
-        keys = ckks.make_rotation_keys(par, s, plan, seed)
+def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=()):
+    """Full-size calls exactly as the benchmark's runner issues them (projections that read the same
+    activation stacked row-wise into one call, repeated on the same buffers so that the third call is the
+    replayed graph with its concurrent key-switch chains): the device computes every output block, the
+    oracle the listed ones; those must agree on every residue, before and after the rescale, and decrypt
+    to the fp64 product.  Calls with the same d_in share one set of input ciphertexts, so that the
+    oracle rotates them only once."""
+    s = ckks.keygen(par, seed)
+    keys = ckks.make_rotation_keys(par, s, plan, seed)
+    units = wl.fuse_shared_inputs(layers, plan.D)
+    inputs = {}                      # d_in -> (x, ciphertexts, the oracle's baby rotations)
     g = GpuSide(par, plan)
     try:
         g.load_keys(keys)
-        for L in layers:
-            W = wl.gen_weights(seed, L.name, L.d_out, L.d_in)
-            x = wl.gen_activation(seed, L.name, L.d_in)
-            cts = ckks.encrypt_vector(par, plan, s, x, seed)
-            n_out = -(-L.d_out // plan.D)
-            blocks = blocks_of(L, n_out)
-            expect = ckks.linear(par, plan, cts, W, keys, blocks=blocks)
-            w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), L.d_out, L.d_in)
-            out = g.linear(cts, W, L.d_out, L.d_in, weights=w)
-            if L.name in on_the_fly:      # the same call with the weights encoded on the fly
-                fly = g.to_host_u64(g.linear(cts, W, L.d_out, L.d_in))
+        for name, d_in, members in units:
+            d_out = sum(m.d_out for m in members)
+            W = np.concatenate([wl.gen_weights(seed, m.name, m.d_out, m.d_in) for m in members], axis=0)
+            if d_in not in inputs:
+                x = wl.gen_activation(seed, f"x{d_in}", d_in)
+                cts = ckks.encrypt_vector(par, plan, s, x, seed)
+                inputs[d_in] = (x, cts, [ckks.baby_rotations(par, plan, ct, keys) for ct in cts])
+            x, cts, X = inputs[d_in]
+            n_in, n_out = len(cts), -(-d_out // plan.D)
+            blocks = list(blocks_of(name, n_out))
+            expect = ckks.linear(par, plan, cts, W, keys, blocks=blocks, X=X)
+            w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in)
+            ct_in = g.to_dev(np.stack(cts))
+            out = g.empty_u64(n_out, 2, par.r, par.N)
+            for call in range(3):               # direct, captured, replayed
+                out.zero_()
+                g.bf.bf_linear(g.ctx, ct_in, n_in, w, None, d_out, d_in, out, n_out)
+            if name in on_the_fly:          # the same call with the weights encoded on the fly
+                fly = g.to_host_u64(g.linear(cts, W, d_out, d_in))
                 for p in blocks:
-                    assert np.array_equal(fly[p], expect[p]), (L.name, p, "on the fly")
+                    assert np.array_equal(fly[p], expect[p]), (name, p, "on the fly")
                 del fly
             low = g.empty_u64(n_out, 2, par.r - 1, par.N)
             scale = g.bf.bf_rescale(g.ctx, out, low, n_out, par.r, par.scale * par.scale)
@@ -268,39 +281,48 @@ def check_blocks(par, plan, layers, blocks_of, seed, keys=None, s=None, on_the_f
             g.bf.bf_weights_free(g.ctx, w)
             y_ref = W.astype(np.float64) @ x
             for p in blocks:
-                assert np.array_equal(got[p], expect[p]), (L.name, p)
-                assert np.array_equal(low[p], ckks.rescale(par, expect[p])), (L.name, p)
-                part = ckks.fold_output(ckks.decode(ckks.decrypt(par, s, low[p]), par.N, scale), plan, p, L.d_out)
+                assert np.array_equal(got[p], expect[p]), (name, p)
+                assert np.array_equal(low[p], ckks.rescale(par, expect[p])), (name, p)
+                part = ckks.fold_output(ckks.decode(ckks.decrypt(par, s, low[p]), par.N, scale), plan, p, d_out)
                 err = np.abs(part - y_ref[p * plan.D:p * plan.D + len(part)]).max()
-                assert err < 1e-3, (L.name, p, err)
+                assert err < 1e-3, (name, p, err)
     finally:
         g.close()
 
 
-def test_gpt2_layer_shapes_sampled_blocks():
-    # one transformer layer of the GPT-2 decode-step workload (qkv is covered in full above)
+def test_gpt2_step_one_whole_layer_every_block():
+    # config 2: one transformer layer of the GPT-2 decode step, all four calls, every output block
+    # (qkv 3 blocks, out_proj 1, ffn_up 3, ffn_down 1 with three input ciphertexts)
     w = wl.WORKLOADS["gpt2_step"]
     par = oracle_params(w.params)
     plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
-    check_blocks(par, plan, w.layers[1:], lambda L, n_out: [n_out - 1], 11)
+    check_blocks(par, plan, w.layers, lambda name, n_out: range(n_out), 11)
 
 
-def test_qwen3_layer_shapes_sampled_blocks():
+def test_qwen3_step_the_calls_of_one_layer():
+    # config 3: the four calls the runner issues per layer.  q+k+v (1024 -> 4096) in full; o (2048 -> 1024, two
+    # input ciphertexts) in full, also on the fly; gate+up (1024 -> 6144): its 18 giant rotations run as two
+    # chains of 9 -- blocks 0 and 2 lie in the first chain for j = 1, 2 and in the second for j = 3, blocks 3
+    # and 5 in the first for j = 1 and in the second for j = 2, 3; down (3072 -> 1024) in full
     w = wl.WORKLOADS["qwen3_step"]
     par = oracle_params(w.params)
     plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
-    # distinct shapes of the layer: q (1024->2048), o (2048->1024), gate (1024->3072), down (3072->1024)
-    pick = [L for L in w.layers if L.name in ("q", "o", "gate", "down")]
-    check_blocks(par, plan, pick, lambda L, n_out: [(3 * n_out) // 4 if n_out > 1 else 0], 12, on_the_fly=("o",))
+    pick = {"q+k+v": [0, 1, 2, 3], "o": [0], "gate+up": [0, 2, 3, 5], "down": [0]}
+    check_blocks(par, plan, w.layers, lambda name, n_out: pick[name], 12, on_the_fly=("o",))
 
 
-def test_llama3_layer_shapes_sampled_blocks():
+def test_llama3_layer_the_calls_the_benchmark_times():
+    # config 4 at N = 2^16: q+k+v (4096 -> 6144): first block, the k block and the v block; o (4096 -> 4096):
+    # first and last; gate+up (4096 -> 28672): 84 giant rotations in four launches of 22, 22, 22 and 18 --
+    # rotation (j - 1) * 28 + p of block p, so block 0 meets launches 1, 2, 3; block 14 (first of up) 1, 2, 4;
+    # blocks 21 and 22 the end of launch 1 and the start of launch 2; block 27 launches 2, 3 and the very last
+    # rotation; down (14336 -> 4096): 14 input ciphertexts whose 98 baby rotations share two hoisted ModUps
+    # (9 + 5 ciphertexts), every output block, and once more with the weights encoded on the fly
     w = wl.WORKLOADS["llama3_layer"]
     par = oracle_params(w.params)
     plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
-    # k (4096->1024) in full, one block of gate (4096->14336)
-    pick = [L for L in w.layers if L.name in ("k", "gate")]
-    check_blocks(par, plan, pick, lambda L, n_out: [n_out - 1], 13, on_the_fly=("k",))
+    pick = {"q+k+v": [0, 4, 5], "o": [0, 3], "gate+up": [0, 14, 21, 22, 27], "down": [0, 1, 2, 3]}
+    check_blocks(par, plan, w.layers, lambda name, n_out: pick[name], 13, on_the_fly=("down",))
 
 
 def test_linear_with_the_papers_own_parameter_set():
