@@ -3,11 +3,13 @@
 replicas, one process per GPU), with the roofline of the dominant kernels and the CPU oracle
 timed beside it.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload gpt2_qkv] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload qwen3_step@budget=60] [--impl reference]
 
 A step = one decode token's worth of the workload: bf_linear + bf_rescale for every linear layer
-of the workload, cached encoded weights streamed from HBM (352 MB per step for gpt2_qkv, larger
-than L2, so consecutive steps cannot be served from cache).  Inputs are seeded and synthetic.
+of the workload, cached encoded weights streamed from HBM (49 GB per step for the Qwen3-0.6B-shaped
+default, 352 MB for the single GPT-2 projection: always larger than L2, so consecutive steps cannot
+be served from cache).  The other configurations are timed after the main one and reported under
+"other_workloads", each with its own rooflines.  Inputs are seeded and synthetic.
 """
 from __future__ import annotations
 
@@ -28,7 +30,7 @@ METRIC = "encrypted linear-layer ms per decode token"
 UNIT = "ms"
 
 # DRAM bytes (read + write) per launch of the named kernel from an ncu capture of this workload;
-# see profiles/ for the capture each figure comes from.  None = not captured yet.
+# see profiles/ for the capture each figure comes from.  None = not captured.
 NCU_TRAFFIC_BYTES = {
     # from the ncu capture summarised under profiles/: dram__bytes_read.sum + dram__bytes_write.sum per launch
     "gpt2_qkv": {"mac": 423.7e6,                       # 411.1 MB read + 12.6 MB written
@@ -37,7 +39,9 @@ NCU_TRAFFIC_BYTES = {
                  "ntt_fwd_strided": 23.8e6,            # mean of the eight captured forward launches (both passes)
                  "ntt_inv_contig": 11.0e6},            # mean of the eight captured inverse launches (both passes)
 }
-
+# Executed instructions per butterfly by pipe, from ncu captures of the transform kernels (profiles/), to set
+# beside the modelled 8 / 12 / 10 operations.  None = not captured.
+NCU_PIPE_INSTR = {}
 
 
 def read_peaks():
@@ -98,13 +102,50 @@ class ClockSampler(threading.Thread):
 
 
 DEFAULT_LANES = 2       # the library's default number of concurrent key-switch chains
+MIN_REGION_S = 0.5      # every timed region lasts at least this long (steps are repeated inside it)
+
+# Workload specifications: "<workload>[@option[,option...]]".  Options: budget=<GB> (cache budget, so that
+# overflow layers take the on-the-fly path), on_the_fly (budget of one byte: nothing is cached), compact
+# (compact cache format), fold (in-ciphertext fold of the tau partial sums).
+DEFAULT_WORKLOAD = "qwen3_step@budget=60"
+DEFAULT_EXTRA = ("gpt2_qkv,gpt2_step,qwen3_step@budget=40.5,qwen3_step@budget=40.5,compact,"
+                 "llama3_layer,llama3_layer@on_the_fly,tiny")
 
 
-def butterflies_per_step(runner) -> dict:
+def parse_spec(spec: str):
+    name, _, opts = spec.partition("@")
+    kw = {}
+    for o in filter(None, opts.split(",")):
+        if o.startswith("budget="):
+            kw["cache_budget_bytes"] = int(float(o[7:]) * 10 ** 9)
+        elif o == "on_the_fly":
+            kw["cache_budget_bytes"] = 1
+        elif o == "compact":
+            kw["compact_cache"] = True
+        elif o == "fold":
+            kw["fold_in_ciphertext"] = True
+        else:
+            raise ValueError(f"unknown workload option {o!r}")
+    return name, kw
+
+
+def split_specs(text: str):
+    """Comma-separated specs; an item without a workload name in front is an option of the previous spec."""
+    from paper_2606_17421_b200 import workloads as wl
+    out = []
+    for item in filter(None, text.split(",")):
+        if item.split("@")[0] in wl.WORKLOADS:
+            out.append(item)
+        else:
+            out[-1] += ("," if "@" in out[-1] else "@") + item
+    return out
+
+
+def transform_counts(runner) -> dict:
     """Transforms one step launches, by direction and by arithmetic path.  Moduli below 2^41 run in
     fp64 with 8 fp64 operations per butterfly (signed lazy values), moduli from 2^41 up to 2^50 in fp64
     with a conditional subtraction and offsets (12 operations), the 60-bit special prime in integers
-    (at least 10 32-bit multiply-adds per butterfly); both pipes issue 64 lanes per clock per SM."""
+    (at least 10 32-bit multiply-adds per butterfly)."""
     import math
     r, N = runner.r, runner.N
     b, g = runner.plan.b, runner.plan.g
@@ -119,57 +160,186 @@ def butterflies_per_step(runner) -> dict:
         n_giant = (g - 1) * n_out
         sets = (n_in if b > 1 else 0) + n_giant            # ModUp digit sets
         rots = n_in * (b - 1) + n_giant                    # key switches
+        n_lift = 2 * rots                                  # divisions by P: one per rotation and component
         for i in range(r):
-            fwd[i] += 2 * n_in + sets * (r - 1) + 2 * rots # inputs; digits of the other primes; lifted P-residues
+            fwd[i] += 2 * n_in + sets * (r - 1) + n_lift   # inputs; digits of the other primes; lifted P-residues
             inv[i] += n_giant + 2 * n_out                  # c1 of the giant-step inputs; outputs
         fwd[r] += sets * r
-        inv[r] += 2 * rots                                 # P-residues of the inner products
+        inv[r] += n_lift                                   # P-residues of the inner products
     def summary(cnt):
-        polys = sum(cnt)
-        ops = sum(c * k for c, k in zip(cnt, cost))
-        return {"polys": polys, "fp64_polys": sum(c for c, f in zip(cnt, fp) if f), "ops_per_butterfly": ops / max(1, polys)}
+        return {"polys": sum(cnt), "fp64_polys": sum(c for c, f in zip(cnt, fp) if f),
+                "fp64_ops": sum(c * k for c, k, f in zip(cnt, cost, fp) if f),
+                "int_ops": sum(c * k for c, k, f in zip(cnt, cost, fp) if not f)}
     return {"fwd": summary(fwd), "inv": summary(inv), "per_poly": per}
 
 
-def time_extra_workload(name: str, steps: int, cache_budget_bytes=None, fold_in_ciphertext=False,
-                        compact_cache=False) -> dict:
-    """ms per decode token of another workload (device-resident inputs), with the weight stream's rate."""
-    import torch
-    from paper_2606_17421_b200 import bifrost as bf
-    from paper_2606_17421_b200.runner import WorkloadRunner
-    R = WorkloadRunner(name, cache_budget_bytes=cache_budget_bytes, fold_in_ciphertext=fold_in_ciphertext,
-                       compact_cache=compact_cache)
-    for _ in range(3):
-        R.step()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        R.step()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / steps
-    bf.bf_get_kernel_stats(R.ctx)
-    bf.bf_set_kernel_timing(R.ctx, True)
-    bf.bf_set_lanes(R.ctx, 1)              # one chain: every kernel runs alone, so its event pair times it alone
-    for _ in range(steps):
-        R.step()
-    st = bf.bf_get_kernel_stats(R.ctx)
-    bf.bf_set_lanes(R.ctx, DEFAULT_LANES)
-    mac_n, mac_ms = st["mac"]
-    enc_ms = (st["encode_fft_a"][1] + st["encode_fft_b"][1]) / steps
-    h2d, d2h = R.host_bytes_per_step()
-    out = {"ms_per_token": round(ms, 4), "layers": len(R.layers),
-           "ciphertexts_in": sum(e["n_in"] for e in R.layers), "ciphertexts_out": sum(e["n_out"] for e in R.layers),
-           "boundary_bytes": h2d + d2h, "rotation_keys": len(R.rot_steps), "fallback_layers": R.n_fallback_layers(),
-           "plan": {"D": R.plan.D, "tau": R.plan.tau, "b": R.plan.b, "g": R.plan.g},
-           "encoded_weight_bytes_cached": R.cached_pt_bytes(), "encoded_weight_bytes_total": R.total_pt_bytes(),
-           "mac_gbs": round(R.total_pt_bytes() * steps / (mac_ms * 1e-3) / 1e9, 1) if mac_ms else None,
-           "kernel_ms_per_token": {k: round(v[1] / steps, 3) for k, v in st.items() if v[0]},
-           "encode_fft_ms_per_token": round(enc_ms, 3)}
-    R.close()
-    torch.cuda.empty_cache()
-    return out
+class Measurement:
+    """Times one workload on the current device: K steps (repeated so that the region lasts at least
+    MIN_REGION_S) with the default launch configuration, then the same steps with an event pair around
+    every launch and the key-switch chains serialised, from which the per-kernel rooflines follow."""
+
+    def __init__(self, spec: str, seed: int = 0, device: str = "cuda:0", world: int = 1):
+        from paper_2606_17421_b200.runner import WorkloadRunner
+        self.spec = spec
+        name, kw = parse_spec(spec)
+        self.name = name
+        self.world = world
+        self.R = WorkloadRunner(name, seed=seed, device=device, **kw)
+
+    def barrier(self):
+        import torch
+        import torch.distributed as dist
+        torch.cuda.synchronize()
+        if self.world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(self, fn, count):
+        """count calls of fn between two events on the runner's stream; (max-over-ranks ms, wall t0, wall t1)"""
+        import torch
+        from paper_2606_17421_b200.replicas import max_over_ranks
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.barrier()
+        t0 = time.time()
+        e0.record(self.R.stream)
+        for _ in range(count):
+            fn()
+        e1.record(self.R.stream)
+        self.barrier()
+        t1 = time.time()
+        return max_over_ranks(e0.elapsed_time(e1), device="cuda"), t0, t1
+
+    def repeats_for(self, fn, steps):
+        """How often a step is repeated inside the timed region so that it lasts MIN_REGION_S (same on all ranks)."""
+        import math
+        ms, _, _ = self.timed(fn, 1)
+        return max(1, math.ceil(MIN_REGION_S * 1e3 / max(1e-3, ms * steps)))
+
+    def run(self, steps: int, warmup: int, e2e: bool = False) -> dict:
+        from paper_2606_17421_b200 import bifrost as bf
+        R = self.R
+        for _ in range(max(warmup, 3)):
+            R.step()
+        reps = self.repeats_for(R.step, steps)
+        self.barrier()
+        bf.bf_get_kernel_stats(R.ctx)   # reset launch counters
+        ms_total, t0, t1 = self.timed(R.step, steps * reps)
+        stats = bf.bf_get_kernel_stats(R.ctx)
+        out = {"ms_per_step": ms_total / (steps * reps), "repeats_per_step": reps, "t0": t0, "t1": t1,
+               "gpu_launches": sum(v[0] for v in stats.values()),
+               "launches_per_step": sum(v[0] for v in stats.values()) / (steps * reps)}
+        # per-kernel durations: an event pair around every launch, chains serialised (one lane) so that no other
+        # kernel of the step runs beside the timed one
+        k_steps = max(1, min(steps * reps, max(3, int(0.3 * steps * reps))))
+        bf.bf_set_kernel_timing(R.ctx, True)
+        bf.bf_set_lanes(R.ctx, 1)
+        bf.bf_get_key_stream_bytes(R.ctx)
+        self.timed(R.step, k_steps)
+        out["kstats"] = bf.bf_get_kernel_stats(R.ctx)
+        out["key_bytes"] = bf.bf_get_key_stream_bytes(R.ctx)
+        out["k_steps"] = k_steps
+        bf.bf_set_kernel_timing(R.ctx, False)
+        bf.bf_set_lanes(R.ctx, DEFAULT_LANES)
+        if e2e:
+            # end to end through the host-buffer entry point (pinned host ciphertexts in and out)
+            R.make_host_buffers()
+            for _ in range(2):
+                R.step_host()
+            e_reps = self.repeats_for(R.step_host, 3)
+            e_steps = 3 * e_reps
+            e_total, _, _ = self.timed(R.step_host, e_steps)
+            out["e2e_ms"] = e_total / e_steps
+            out["e2e_steps"] = e_steps
+        return out
+
+    def rooflines(self, m: dict, hbm_peak: float, peak_kind: str, fma_rate: float, imad_rate: float) -> dict:
+        R, kstats, K = self.R, m["kstats"], m["k_steps"]
+        traffic = NCU_TRAFFIC_BYTES.get(self.spec, {})
+        counts = transform_counts(R)
+
+        def avg_ms(cat):
+            n, ms = kstats[cat]
+            return (ms / n) if n else None, n / K
+
+        rl = {}
+        # weight-streaming multiply-accumulate: algorithmic bytes = every encoded word once
+        mac_ms, mac_n = avg_ms("mac")
+        if mac_ms:
+            mac_bytes = R.total_pt_bytes() / max(1.0, mac_n)
+            ach = mac_bytes / (mac_ms * 1e-3) / 1e9
+            rl["mac"] = {"bound": "hbm", "achieved": round(ach, 1), "peak": hbm_peak, "unit": "GB/s",
+                         "frac": round(ach / hbm_peak, 4), "of": peak_kind, "traffic": traffic.get("mac"),
+                         "launches_per_step": mac_n, "avg_ms": round(mac_ms, 5),
+                         "bytes_per_launch": round(mac_bytes), "frac_of_nominal_8000": round(ach / 8000.0, 4)}
+        # key-switch inner product: algorithmic bytes = every distinct key of a launch once
+        ki_ms, ki_n = avg_ms("key_inner_product")
+        if ki_ms:
+            distinct, per_rot = m["key_bytes"]
+            n_launch = kstats["key_inner_product"][0]
+            ach = distinct / n_launch / (ki_ms * 1e-3) / 1e9
+            ach_rot = per_rot / n_launch / (ki_ms * 1e-3) / 1e9
+            rl["key_inner_product"] = {"bound": "hbm", "achieved": round(ach, 1), "peak": hbm_peak, "unit": "GB/s",
+                                       "frac": round(ach / hbm_peak, 4), "of": peak_kind,
+                                       "traffic": traffic.get("key_inner_product"),
+                                       "launches_per_step": ki_n, "avg_ms": round(ki_ms, 5),
+                                       "bytes_per_launch": round(distinct / n_launch),
+                                       "achieved_counting_a_key_per_rotation": round(ach_rot, 1),
+                                       "note": "bytes = the distinct keys of a launch, each once; the second figure "
+                                               "counts a key once per rotation (repeats are L2 hits)"}
+        # transforms: bound by the arithmetic pipes (fp64 for the ciphertext primes, integer multiply-add for the
+        # special prime); the peak uses the two rates measured in this run
+        for cats, key, label in ((("ntt_fwd_strided", "ntt_fwd_contig"), "fwd", "ntt_forward"),
+                                 (("ntt_inv_contig", "ntt_inv_strided"), "inv", "ntt_inverse")):
+            ms_step = sum(kstats[c][1] for c in cats) / K
+            if ms_step > 0:
+                info = counts[key]
+                rate = info["polys"] * counts["per_poly"] / (ms_step * 1e-3)
+                t_poly = (info["fp64_ops"] / fma_rate + info["int_ops"] / imad_rate) / max(1, info["polys"])
+                peak = 1.0 / t_poly
+                rl[label] = {"bound": "alu", "achieved": round(rate / 1e9, 1), "peak": round(peak / 1e9, 1),
+                             "unit": "G butterflies/s", "frac": round(rate / peak, 4),
+                             "of": (f"measured in this run: {fma_rate / 1e12:.2f} T fp64 multiply-adds/s and "
+                                    f"{imad_rate / 1e12:.2f} T 32-bit integer multiply-adds/s over the GPU; modelled "
+                                    "operations per butterfly: 8 fp64 below 2^41, 12 fp64 up to 2^50, 10 integer for the "
+                                    "special prime"),
+                             "pipe_instructions_per_butterfly_ncu": NCU_PIPE_INSTR.get(label),
+                             "traffic": traffic.get(cats[0]), "ms_per_step": round(ms_step, 5),
+                             "polys_per_step": info["polys"], "fp64_polys_per_step": info["fp64_polys"]}
+        total_k_ms = sum(v[1] for v in kstats.values())
+        shares = {k: round(v[1] / total_k_ms, 4) for k, v in kstats.items() if v[0]}
+        return {"rooflines": rl, "kernel_time_share": shares,
+                "kernel_ms_per_step": {k: round(v[1] / K, 4) for k, v in kstats.items() if v[0]}}
+
+    def describe(self) -> dict:
+        R = self.R
+        h2d, d2h = R.host_bytes_per_step()
+        whole_step = R.w.n_repeat > 1 or len(R.w.layers) > 1
+        return {"layers": len(R.layers), "unit_of_work": "decode token (all linear layers)" if whole_step else "one projection call",
+                "ring_N": R.N, "ct_primes": R.r,
+                "plan": {"D": R.plan.D, "tau": R.plan.tau, "b": R.plan.b, "g": R.plan.g},
+                "ciphertexts_in": sum(e["n_in"] for e in R.layers), "ciphertexts_out": sum(e["n_out"] for e in R.layers),
+                "boundary_bytes": h2d + d2h, "rotation_keys": len(R.rot_steps), "fallback_layers": R.n_fallback_layers(),
+                "encoded_weight_bytes_cached": R.cached_pt_bytes(), "encoded_weight_bytes_total": R.total_pt_bytes()}
+
+    def close(self):
+        import torch
+        self.R.close()
+        torch.cuda.empty_cache()
+
+
+def measure_extra(spec: str, steps: int, peaks) -> dict:
+    M = Measurement(spec)
+    try:
+        m = M.run(steps, 3)
+        out = M.describe()
+        key = "ms_per_token" if out["unit_of_work"].startswith("decode token") else "ms_per_call"
+        out[key] = round(m["ms_per_step"], 4)
+        out["repeats_per_step"] = m["repeats_per_step"]
+        out["launches_per_step"] = m["launches_per_step"]
+        out.update(M.rooflines(m, *peaks))
+        return out
+    finally:
+        M.close()
 
 
 def run_ours(args):
@@ -185,179 +355,86 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     from paper_2606_17421_b200 import bifrost as bf
-    from paper_2606_17421_b200.runner import WorkloadRunner
-    from paper_2606_17421_b200.replicas import job_ms_per_token, max_over_ranks
+    from paper_2606_17421_b200.replicas import job_ms_per_token
 
     bf.load()   # fails loudly when the CUDA library is missing
     # every rank decodes its own token stream (independent problems: no data-path collective)
-    R = WorkloadRunner(args.workload, seed=rank, device=f"cuda:{local}")
-    stream = R.stream                       # the runner's own stream, made torch's current stream
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        t0 = time.time()
-        e0.record(stream)
-        for _ in range(steps):
-            fn()
-        e1.record(stream)
-        barrier()
-        t1 = time.time()
-        ms = max_over_ranks(e0.elapsed_time(e1), device="cuda")
-        return ms, t0, t1
-
-    for _ in range(max(args.warmup, 3)):
-        R.step()
-    barrier()
-    bf.bf_get_kernel_stats(R.ctx)   # reset launch counters
-
+    M = Measurement(args.workload, seed=rank, device=f"cuda:{local}", world=world)
+    R = M.R
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.15)
-    ms_total, t0, t1 = timed(R.step, args.steps)
-    stats = bf.bf_get_kernel_stats(R.ctx)
-    gpu_launches = sum(v[0] for v in stats.values())
-    ms_per_step = ms_total / args.steps
-
-    # per-kernel durations: the same K steps again with an event pair around every launch, and with the
-    # key-switch chains serialised (one lane) so that no other kernel of the step runs beside the timed one
-    bf.bf_set_kernel_timing(R.ctx, True)
-    bf.bf_set_lanes(R.ctx, 1)
-    timed(R.step, args.steps)
-    kstats = bf.bf_get_kernel_stats(R.ctx)
-    bf.bf_set_kernel_timing(R.ctx, False)
-    bf.bf_set_lanes(R.ctx, DEFAULT_LANES)
-
-    # end to end through the host-buffer entry point (pinned host ciphertexts in and out)
-    R.make_host_buffers()
-    for _ in range(3):
-        R.step_host()
-    e2e_steps = max(3, min(args.steps, 50))
-    e2e_total, _, _ = timed(R.step_host, e2e_steps)
-    e2e_ms = e2e_total / e2e_steps
+    m = M.run(args.steps, args.warmup, e2e=True)
     sampler.stop()
-    clocks = sampler.summary(t0, t1)
+    clocks = sampler.summary(m["t0"], m["t1"])
+    ms_per_step = m["ms_per_step"]
 
     if rank != 0:
+        M.close()
         if world > 1:
             dist.destroy_process_group()
         return
 
     hbm_peak, peak_kind = read_peaks()
     imad_rate = bf.bf_measure_imad_rate(R.ctx)
-    bfly = butterflies_per_step(R)
-    K = args.steps
-    traffic = NCU_TRAFFIC_BYTES.get(args.workload, {})
-
-    def avg_ms(cat):
-        n, ms = kstats[cat]
-        return (ms / n) if n else None, n / K
-
-    rooflines = {}
-    # weight-streaming multiply-accumulate: algorithmic bytes = every encoded word once
-    mac_ms, mac_n = avg_ms("mac")
-    if mac_ms:
-        mac_bytes = R.cached_pt_bytes() / max(1.0, mac_n)
-        ach = mac_bytes / (mac_ms * 1e-3) / 1e9
-        rooflines["mac"] = {"bound": "hbm", "achieved": round(ach, 1), "peak": hbm_peak, "unit": "GB/s",
-                            "frac": round(ach / hbm_peak, 4), "of": peak_kind, "traffic": traffic.get("mac"),
-                            "launches_per_step": mac_n, "avg_ms": round(mac_ms, 5),
-                            "frac_of_nominal_8000": round(ach / 8000.0, 4)}
-    # key-switch inner product: algorithmic bytes = the key stream of each rotation once
-    ki_ms, ki_n = avg_ms("key_inner_product")
-    if ki_ms:
-        n_rot = sum(e["n_in"] * (R.plan.b - 1) + e["n_out"] * (R.plan.g - 1) for e in R.layers)
-        key_bytes = n_rot * R.r * 2 * (R.r + 1) * R.N * 8 / max(1.0, ki_n)
-        ach = key_bytes / (ki_ms * 1e-3) / 1e9
-        rooflines["key_inner_product"] = {"bound": "hbm", "achieved": round(ach, 1), "peak": hbm_peak, "unit": "GB/s",
-                                          "frac": round(ach / hbm_peak, 4), "of": peak_kind,
-                                          "traffic": traffic.get("key_inner_product"),
-                                          "launches_per_step": ki_n, "avg_ms": round(ki_ms, 5),
-                                          "note": "bytes = one key per rotation; rotations sharing a key hit L2"}
-    # transforms: bound by the arithmetic pipes (fp64 for the ciphertext primes, integer multiply-add for the special prime)
-    sm_mhz = clocks.get("sm_mhz") or 1965.0
-    lanes_per_s = 148 * 64 * sm_mhz * 1e6                  # either pipe: 148 SMs x 64 lanes x clock
-    for cats, key, label in ((("ntt_fwd_strided", "ntt_fwd_contig"), "fwd", "ntt_forward"),
-                             (("ntt_inv_contig", "ntt_inv_strided"), "inv", "ntt_inverse")):
-        ms_step = sum(kstats[c][1] for c in cats) / K
-        if ms_step > 0:
-            info = bfly[key]
-            rate = info["polys"] * bfly["per_poly"] / (ms_step * 1e-3)
-            peak = lanes_per_s / info["ops_per_butterfly"]
-            rooflines[label] = {"bound": "alu", "achieved": round(rate / 1e9, 1), "peak": round(peak / 1e9, 1),
-                                "unit": "G butterflies/s", "frac": round(rate / peak, 4),
-                                "of": (f"derived: 148 SMs x 64 lanes x {sm_mhz:.0f} MHz / {info['ops_per_butterfly']:.2f} "
-                                       "pipe operations per butterfly (8 fp64 ops below 2^41, 12 up to 2^50, 10 multiply-adds on "
-                                       f"the integer path); bf_measure_imad_rate measured {imad_rate / 1e12:.2f} T multiply-adds/s"),
-                                "traffic": traffic.get(cats[0]), "ms_per_step": round(ms_step, 5),
-                                "polys_per_step": info["polys"], "fp64_polys_per_step": info["fp64_polys"]}
-    total_k_ms = sum(v[1] for v in kstats.values())
-    shares = {k: round(v[1] / total_k_ms, 4) for k, v in kstats.items() if v[0]}
+    fma_rate = bf.bf_measure_fma64_rate(R.ctx)
+    peaks = (hbm_peak, peak_kind, fma_rate, imad_rate)
+    info = M.rooflines(m, *peaks)
+    rooflines, shares = info["rooflines"], info["kernel_time_share"]
     dominant = max(shares, key=shares.get)
     dom_key = {"ntt_fwd_strided": "ntt_forward", "ntt_fwd_contig": "ntt_forward", "ntt_inv_contig": "ntt_inverse",
                "ntt_inv_strided": "ntt_inverse"}.get(dominant, dominant)
     roofline = dict(rooflines.get(dom_key, rooflines.get("mac", {})))
     roofline["kernel"] = dom_key
 
+    desc = M.describe()
     h2d, d2h = R.host_bytes_per_step()
+    sm_mhz = clocks.get("sm_mhz") or 1965.0
     line = {
         "metric": METRIC, "value": round(job_ms_per_token(ms_per_step, world), 5), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5),
+        "repeats_per_step": m["repeats_per_step"],
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": args.workload, "ring_N": R.N, "ct_primes": R.r,
-                   "plan": {"D": R.plan.D, "tau": R.plan.tau, "b": R.plan.b, "g": R.plan.g},
-                   "layers": len(R.layers), "encoded_weight_bytes_per_step": R.cached_pt_bytes(),
-                   "fallback_layers": R.n_fallback_layers(),
+        "config": {"workload": args.workload, "unit_of_work": desc["unit_of_work"], "ring_N": R.N, "ct_primes": R.r,
+                   "plan": desc["plan"], "layers": len(R.layers),
+                   "encoded_weight_bytes_per_step": R.total_pt_bytes(),
+                   "encoded_weight_bytes_cached": R.cached_pt_bytes(), "fallback_layers": R.n_fallback_layers(),
                    "l2": "inputs larger than L2: the encoded weights streamed each step exceed 126 MB",
+                   "timed_region": f"{args.steps} steps x {m['repeats_per_step']} repeats, at least {MIN_REGION_S} s",
                    "multi_gpu": "replicas: every rank decodes its own token, no data-path collective"},
         "tokens_per_s": round(world * 1e3 / ms_per_step, 3),
         "clocks": clocks,
-        "e2e": {"value": round(job_ms_per_token(e2e_ms, world), 5), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": gpu_launches,
+        "e2e": {"value": round(job_ms_per_token(m["e2e_ms"], world), 5), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": m["e2e_steps"]},
+        "gpu_launches": m["gpu_launches"],
         "roofline": roofline,
         "rooflines": rooflines,
         "kernel_time_share": shares,
+        "kernel_ms_per_step": info["kernel_ms_per_step"],
         "kernel_timing": "event pair around every launch with the key-switch chains serialised (1 lane); "
                          f"value and e2e are timed with {DEFAULT_LANES} concurrent chains and no per-launch events",
-        "imad_rate_per_sm_clk": round(imad_rate / 148 / ((clocks.get("sm_mhz") or 1965.0) * 1e6), 2),
+        "measured_rates": {"imad_per_sm_clk": round(imad_rate / 148 / (sm_mhz * 1e6), 2),
+                           "fma64_per_sm_clk": round(fma_rate / 148 / (sm_mhz * 1e6), 2),
+                           "imad_per_s": imad_rate, "fma64_per_s": fma_rate},
     }
-    R.close()
-    torch.cuda.empty_cache()
+    M.close()
     if world == 1 and args.extra:
         extras = {}
-        for name in args.extra.split(","):
-            if name == "qwen3_step":
-                # 60 GB keeps every layer resident; 40.5 GB = 23/28 of the encoded size reproduces the
-                # partially cached regime (Sec. 6.1, table "FHE decode cost breakdown"): the overflow layers are encoded on every call
-                full = time_extra_workload(name, 5, cache_budget_bytes=60 * 10 ** 9)
-                part = time_extra_workload(name, 3, cache_budget_bytes=int(40.5 * 10 ** 9))
-                part["fallback_share_of_step"] = round(1.0 - full["ms_per_token"] / part["ms_per_token"], 4)
-                extras[name + "@60GB"] = full
-                extras[name + "@40.5GB"] = part
-                # the same budget with the compact cache format: every layer fits, nothing falls back
-                extras[name + "@40.5GB_compact_cache"] = time_extra_workload(name, 5, cache_budget_bytes=int(40.5 * 10 ** 9),
-                                                                             compact_cache=True)
-            elif name == "llama3_layer":
-                extras[name + "@cached"] = time_extra_workload(name, 5)
-                extras[name + "@on_the_fly"] = time_extra_workload(name, 3, cache_budget_bytes=1)
-            elif name == "gpt2_qkv@on_the_fly":
-                # the headline call with its weights encoded inside the call (fallback path)
-                extras[name] = time_extra_workload("gpt2_qkv", 50, cache_budget_bytes=1)
-            elif name == "gpt2_qkv@fold_in_ciphertext":
-                # the variant that sums the tau partial results on the device (log2 tau more key switches)
-                extras[name] = time_extra_workload("gpt2_qkv", 50, fold_in_ciphertext=True)
-            else:
-                extras[name] = time_extra_workload(name, 10)
+        for spec in split_specs(args.extra):
+            name, _ = parse_spec(spec)
+            steps = 200 if name in ("tiny", "gpt2_qkv", "gpt2_qkv_paper_params") or name.startswith("gemm1024") else 5
+            extras[spec] = measure_extra(spec, steps, peaks)
+        full, part = line["value"], extras.get("qwen3_step@budget=40.5")
+        if args.workload == DEFAULT_WORKLOAD and part:
+            # 60 GB keeps every layer resident; 40.5 GB = 23/28 of the encoded size reproduces the partially cached
+            # regime (Sec. 6.1, table "FHE decode cost breakdown"): the overflow layers are encoded on every call
+            part["fallback_share_of_step"] = round(1.0 - full / part["ms_per_token"], 4)
+        a, b = extras.get("llama3_layer"), extras.get("llama3_layer@on_the_fly")
+        if a and b:
+            b["on_the_fly_over_cached"] = round(b["ms_per_token"] / a["ms_per_token"], 3)
         line["other_workloads"] = extras
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=20.0)
+        line["cpu_baseline"] = cpu_baseline(parse_spec(args.workload)[0], budget_s=20.0)
     elif world == 1:
         line["cpu_baseline"] = None
     print(json.dumps(line))
@@ -494,7 +571,7 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import ckks
-    S = OracleSample(args.workload)
+    S = OracleSample(parse_spec(args.workload)[0])
     cores = ckks.lib().orc_num_threads()
     # size the per-step sample so that the whole run stays near two minutes
     S.size_sample(max(0.3, 120.0 / max(1, args.steps + args.warmup)))
@@ -523,20 +600,19 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="gpt2_qkv")
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD,
+                    help="workload[@option,...]: see parse_spec; default = the largest single-GPU configuration")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--extra", default="gpt2_step",
-                    help="comma-separated further workloads timed after the main one (N=1 only); '' for none; "
-                         "all = gpt2_qkv@on_the_fly,gpt2_step,qwen3_step,llama3_layer")
+    ap.add_argument("--extra", default=DEFAULT_EXTRA,
+                    help="comma-separated further workload specs timed after the main one (N=1 only); '' for none; "
+                         "tiles = the tile-size study and the paper's own parameter set")
     args = ap.parse_args()
-    if args.extra == "all":
-        args.extra = "gpt2_qkv@on_the_fly,gpt2_step,qwen3_step,llama3_layer"
-    elif args.extra == "tiles":     # tile-size study and the paper's own parameter set
+    if args.extra == "tiles":     # tile-size study and the paper's own parameter set
         args.extra = ("gemm1024_D1024,gemm1024_D512,gemm1024_D256,gemm1024_D128,gpt2_qkv_paper_params,"
-                      "gpt2_qkv@fold_in_ciphertext")
+                      "gpt2_qkv@fold")
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -242,6 +242,16 @@ int bf_get_kernel_stats(bf_ctx* ctx, uint64_t* launches_out, float* ms_out);
  * probe kernel (a few ms) on the context's stream and synchronises. */
 int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out);
 
+/* The same for the fp64 fused multiply-add (fma.rn.f64) that the transforms of the ciphertext primes
+ * (below 2^50) are made of: the denominator for their roofline. */
+int bf_measure_fma64_rate(bf_ctx* ctx, double* fma_per_second_out);
+
+/* Bytes of rotation keys the key-switch inner products launched since the previous call had to stream:
+ * counted once per distinct key of each launch (distinct_out, host: what must come from HBM; Sec. 4.2
+ * "key-switching primitives") and once per rotation (per_rotation_out, host: what the launches read,
+ * L2 hits included).  Resets both counters.  Does not synchronise. */
+int bf_get_key_stream_bytes(bf_ctx* ctx, uint64_t* distinct_out, uint64_t* per_rotation_out);
+
 const char* bf_strerror(int code);
 const char* bf_last_cuda_error(const bf_ctx* ctx);
 

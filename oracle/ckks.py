@@ -21,6 +21,16 @@ evaluation strategy (packing, BSGS split, key-switch variant, rounding points):
   BSGS                  diagonal i = j*b + k; Y_p = sum_j rot( sum_q sum_k Pt[p][q][j][k] * rot(ct_q, k*tau), j*b*tau )
   rescale               c'_i = (c_i - centred(c_L)) * q_L^{-1} mod q_i
 
+Two variants change residues and are therefore modes of the plan, evaluated here step by step as well
+(the paper leaves both open: Sec. 4.2 speaks of "key-switching primitives" and of weight diagonals kept
+as BSGS objects, and Sec. 6.1 names the encoded-weight cache as the memory wall):
+  pack = "complex"      two output row blocks share a plaintext: block 2P in the real parts of the slots,
+                        block 2P+1 in the imaginary parts; the input ciphertexts stay real, so output
+                        ciphertext P decrypts to (block 2P) + i (block 2P+1); half the diagonals
+  moddown = "per_output"  the giant-step key switches of an output are summed in the extended basis
+                        {q_0..q_L, P} and divided by P once per output ciphertext and component,
+                        instead of once per rotation
+
 Array conventions (all numpy, C order):
   ciphertext  uint64 [2][r][N]   component, prime, coefficient; coefficient domain, residues in [0, q_i)
   plaintext   uint64 [r][N]      coefficient domain
@@ -76,6 +86,8 @@ def lib():
         L.orc_encode_slots.argtypes = [_f64p, _f64p, ctypes.c_uint32, ctypes.c_double, _i64p]
         L.orc_encode_real_batch.restype = ctypes.c_int
         L.orc_encode_real_batch.argtypes = [_f64p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_double, _i64p]
+        L.orc_encode_complex_batch.restype = ctypes.c_int
+        L.orc_encode_complex_batch.argtypes = [_f64p, _f64p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_double, _i64p]
         L.orc_num_threads.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -140,14 +152,26 @@ class Plan:
     tau: int
     b: int
     g: int
+    pack: str = "real"                 # "real" | "complex": see the module docstring
+    moddown: str = "per_rotation"      # "per_rotation" | "per_output"
 
     @property
     def M(self) -> int:
         return self.D // self.tau
 
+    @property
+    def rows_per_ct(self) -> int:
+        """Output rows one output ciphertext carries."""
+        return self.D * (2 if self.pack == "complex" else 1)
+
+    def n_out(self, d_out: int) -> int:
+        """Number of output ciphertexts of a projection with d_out rows."""
+        return -(-d_out // self.rows_per_ct)
+
     def check(self, n: int):
         assert self.D * self.tau <= n and n % (self.D * self.tau) == 0
         assert self.D % self.tau == 0 and self.b * self.g == self.M
+        assert self.pack in ("real", "complex") and self.moddown in ("per_rotation", "per_output")
 
 
 def galois_element(steps: int, N: int) -> int:
@@ -226,6 +250,18 @@ def encode_real_batch(z: np.ndarray, N: int, scale: float) -> np.ndarray:
     z = np.ascontiguousarray(z, dtype=np.float64)
     m = np.zeros((z.shape[0], N), dtype=np.int64)
     st = lib().orc_encode_real_batch(_p(z, _f64p), z.shape[0], N, scale, _p(m, _i64p))
+    if st != 0:
+        raise OverflowError("encoded coefficient out of range")
+    return m
+
+
+def encode_complex_batch(z: np.ndarray, N: int, scale: float) -> np.ndarray:
+    """z[count][N/2] complex -> int64 [count][N]."""
+    z = np.asarray(z, dtype=np.complex128)
+    zre = np.ascontiguousarray(z.real, dtype=np.float64)
+    zim = np.ascontiguousarray(z.imag, dtype=np.float64)
+    m = np.zeros((z.shape[0], N), dtype=np.int64)
+    st = lib().orc_encode_complex_batch(_p(zre, _f64p), _p(zim, _f64p), z.shape[0], N, scale, _p(m, _i64p))
     if st != 0:
         raise OverflowError("encoded coefficient out of range")
     return m
@@ -355,19 +391,18 @@ def mod_down(u: np.ndarray, params: Params) -> np.ndarray:
     return v
 
 
-def rotate_galois(params: Params, ct: np.ndarray, g: int, key: np.ndarray, key_ntt=None) -> np.ndarray:
-    """Apply X -> X^g to a full-level ciphertext and switch back to the secret key s.
-
-    1. digit j = residues of c1 mod q_j as integers in [0, q_j), reduced into every modulus of
-       the extended basis;  2. automorphism of each reduced digit;  3. (u0, u1) = sum_j digit_j *
-       (key_j.b, key_j.a) in R_m for every m of the basis;  4. divide both by P (mod_down);
-       5. result = (phi_g(c0) + v0, v1)."""
+def key_switch_ext(params: Params, c1: np.ndarray, g: int, key: np.ndarray, key_ntt=None) -> np.ndarray:
+    """The key switch of phi_g(c1) from phi_g(s) to s, before the division by P:
+    1. digit j = residues of c1 mod q_j as integers in [0, q_j), reduced into every modulus of the
+       extended basis;  2. automorphism of each reduced digit;  3. (u0, u1) = sum_j digit_j *
+       (key_j.b, key_j.a) in R_m for every m of the basis.  c1: [r][N]; returns u [2][r+1][N],
+       coefficient domain, with u0 + u1*s = P * phi_g(c1) * phi_g(s) + small."""
     N, r, basis = params.N, params.r, params.basis
-    assert ct.shape == (2, r, N)
+    assert c1.shape == (r, N)
     digits = np.zeros((r, r + 1, N), dtype=np.uint64)
     for j in range(r):
         for mi, m in enumerate(basis):
-            digits[j, mi] = automorphism(ct[1, j] % np.uint64(m), g, m)
+            digits[j, mi] = automorphism(c1[j] % np.uint64(m), g, m)
     moduli_d = basis * r
     dig_ntt = ntt(digits, moduli_d, params)
     if key_ntt is None:
@@ -376,7 +411,17 @@ def rotate_galois(params: Params, ct: np.ndarray, g: int, key: np.ndarray, key_n
     for comp in range(2):
         for j in range(r):
             mul_acc(u[comp], dig_ntt[j], key_ntt[j, comp], basis, N)
-    u = intt(u, basis * 2, params)
+    return intt(u, basis * 2, params)
+
+
+def rotate_galois(params: Params, ct: np.ndarray, g: int, key: np.ndarray, key_ntt=None) -> np.ndarray:
+    """Apply X -> X^g to a full-level ciphertext and switch back to the secret key s.
+
+    Steps 1-3: (u0, u1) = key_switch_ext(c1);  4. divide both by P (mod_down);
+    5. result = (phi_g(c0) + v0, v1)."""
+    N, r = params.N, params.r
+    assert ct.shape == (2, r, N)
+    u = key_switch_ext(params, ct[1], g, key, key_ntt)
     out = np.zeros_like(ct)
     v0, v1 = mod_down(u[0], params), mod_down(u[1], params)
     for i, q in enumerate(params.primes):
@@ -447,21 +492,33 @@ def bsgs_plain_slots(W: np.ndarray, plan: Plan, p: int, q: int, j: int, k: int, 
     return np.roll(d, j * plan.b * plan.tau)
 
 
+def plain_slots(W: np.ndarray, plan: Plan, p: int, q: int, j: int, k: int, n: int) -> np.ndarray:
+    """Slot vector of the plaintext Pt[p][q][j][k] that output ciphertext p multiplies into rot(ct_q, k*tau).
+    Real packing: the pre-rotated diagonal of row block p.  Complex packing: row block 2p in the real parts
+    and row block 2p+1 in the imaginary parts (zero where that block lies outside the matrix)."""
+    if plan.pack == "complex":
+        return bsgs_plain_slots(W, plan, 2 * p, q, j, k, n) + 1j * bsgs_plain_slots(W, plan, 2 * p + 1, q, j, k, n)
+    return bsgs_plain_slots(W, plan, p, q, j, k, n)
+
+
 def encode_weights(params: Params, plan: Plan, W: np.ndarray, blocks=None) -> dict:
     """Encoded diagonals of a projection W[d_out][d_in] (Sec. 4.2: pre-encoded weight diagonals kept
     as BSGS objects).  Returns {(p, q, j, k): uint64 [r][N] coefficient-domain plaintext} for the
-    requested output blocks (all by default)."""
+    requested output ciphertexts p (all by default)."""
     plan.check(params.n)
     d_out, d_in = W.shape
-    n_in, n_out = -(-d_in // plan.D), -(-d_out // plan.D)
+    n_in, n_out = -(-d_in // plan.D), plan.n_out(d_out)
     blocks = range(n_out) if blocks is None else blocks
     idx = [(p, q, j, k) for p in blocks for q in range(n_in) for j in range(plan.g) for k in range(plan.b)]
     out = {}
     step = 256
     for lo in range(0, len(idx), step):
         part = idx[lo:lo + step]
-        z = np.stack([bsgs_plain_slots(W, plan, *t, params.n) for t in part])
-        m = encode_real_batch(z, params.N, params.scale)
+        z = np.stack([plain_slots(W, plan, *t, params.n) for t in part])
+        if plan.pack == "complex":
+            m = encode_complex_batch(z, params.N, params.scale)
+        else:
+            m = encode_real_batch(z, params.N, params.scale)
         res = to_residues(m, params.primes)
         for t, pt in zip(part, res):
             out[t] = pt
@@ -499,9 +556,9 @@ def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blo
     unchanged, scale multiplies.  Returns {p: ciphertext}.  X, when given, is the list over q of
     baby_rotations(params, plan, cts[q], keys) computed by an earlier call for the same inputs (several
     projections that read the same ciphertexts need them only once)."""
-    N, r, primes = params.N, params.r, params.primes
+    N, r, primes, basis = params.N, params.r, params.primes, params.basis
     d_out, d_in = W.shape
-    n_in, n_out = -(-d_in // plan.D), -(-d_out // plan.D)
+    n_in, n_out = -(-d_in // plan.D), plan.n_out(d_out)
     assert len(cts) == n_in
     blocks = list(range(n_out) if blocks is None else blocks)
     if encoded is None:
@@ -514,12 +571,38 @@ def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blo
     out = {}
     for p in blocks:
         Y = np.zeros((2, r, N), dtype=np.uint64)
-        for j in range(plan.g):
-            A = inner_sum(params, plan, Xh, encoded, p, j)
-            A = rotate(params, A, j * plan.b * plan.tau, keys)
-            for comp in range(2):
+        if plan.moddown == "per_output":
+            # giant steps j >= 1: key-switch results summed over j in the extended basis, the rotated c0
+            # parts summed beside them; one division by P per component at the end
+            U = np.zeros((2, r + 1, N), dtype=np.uint64)
+            for j in range(plan.g):
+                A = inner_sum(params, plan, Xh, encoded, p, j)
+                steps = j * plan.b * plan.tau
+                if steps % params.n == 0:
+                    rot_c0, u = A[0], None
+                    for i, qi in enumerate(primes):
+                        Y[1, i] = _add(Y[1, i], A[1, i], qi)
+                else:
+                    g = galois_element(steps, N)
+                    u = key_switch_ext(params, A[1], g, keys[g])
+                    rot_c0 = np.stack([automorphism(A[0, i], g, qi) for i, qi in enumerate(primes)])
+                    for comp in range(2):
+                        for mi, m in enumerate(basis):
+                            U[comp, mi] = _add(U[comp, mi], u[comp, mi], m)
                 for i, qi in enumerate(primes):
-                    Y[comp, i] = _add(Y[comp, i], A[comp, i], qi)
+                    Y[0, i] = _add(Y[0, i], rot_c0[i], qi)
+            if plan.g > 1:
+                v0, v1 = mod_down(U[0], params), mod_down(U[1], params)
+                for i, qi in enumerate(primes):
+                    Y[0, i] = _add(Y[0, i], v0[i], qi)
+                    Y[1, i] = _add(Y[1, i], v1[i], qi)
+        else:
+            for j in range(plan.g):
+                A = inner_sum(params, plan, Xh, encoded, p, j)
+                A = rotate(params, A, j * plan.b * plan.tau, keys)
+                for comp in range(2):
+                    for i, qi in enumerate(primes):
+                        Y[comp, i] = _add(Y[comp, i], A[comp, i], qi)
         out[p] = Y
     return out
 
@@ -547,10 +630,15 @@ def rescale(params: Params, ct: np.ndarray) -> np.ndarray:
 
 
 def fold_output(slots: np.ndarray, plan: Plan, p: int, d_out: int) -> np.ndarray:
-    """Host-side fold of the tau partial sums: y[p*D + kappa] = sum_c slot((0, kappa, c))."""
+    """Host-side fold of the tau partial sums of output ciphertext p: y[p*D + kappa] = sum_c slot((0, kappa, c)).
+    Complex packing: the real parts give rows 2p*D + kappa, the imaginary parts rows (2p+1)*D + kappa; the
+    result is the rows_per_ct rows of ciphertext p in order (cut at d_out)."""
     D, tau = plan.D, plan.tau
-    part = np.asarray(slots).real[:D * tau].reshape(D, tau).sum(axis=1)
-    rows = min(D, d_out - p * D)
+    s = np.asarray(slots)[:D * tau]
+    part = s.real.reshape(D, tau).sum(axis=1)
+    if plan.pack == "complex":
+        part = np.concatenate([part, s.imag.reshape(D, tau).sum(axis=1)])
+    rows = min(plan.rows_per_ct, d_out - p * plan.rows_per_ct)
     return part[:rows]
 
 
@@ -574,8 +662,9 @@ def fold_in_ciphertext(params: Params, plan: Plan, ct: np.ndarray, keys: dict) -
 def folded_output(slots: np.ndarray, plan: Plan, p: int, d_out: int) -> np.ndarray:
     """Reads the complete dot products of a ciphertext folded by fold_in_ciphertext: slot (0, kappa, 0)."""
     D, tau = plan.D, plan.tau
-    part = np.asarray(slots).real[:D * tau:tau]
-    rows = min(D, d_out - p * D)
+    s = np.asarray(slots)[:D * tau:tau]
+    part = np.concatenate([s.real, s.imag]) if plan.pack == "complex" else s.real
+    rows = min(plan.rows_per_ct, d_out - p * plan.rows_per_ct)
     return part[:rows]
 
 

@@ -341,6 +341,21 @@ int orc_encode_real_batch(const double* z, u32 count, u32 N, double scale, i64* 
     return status;
 }
 
+/* Batch of complex slot vectors (zre[count][n], zim[count][n]) -> coefficients m[count][N]. */
+int orc_encode_complex_batch(const double* zre, const double* zim, u32 count, u32 N, double scale, i64* m) {
+    int status = 0;
+    u32 n = N / 2;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (u32 b = 0; b < count; b++) {
+        int s = orc_encode_slots(zre + (size_t)b * n, zim + (size_t)b * n, N, scale, m + (size_t)b * N);
+        if (s) {
+#pragma omp atomic write
+            status = s;
+        }
+    }
+    return status;
+}
+
 int orc_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

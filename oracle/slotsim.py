@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from .ckks import Plan, bsgs_plain_slots, fold_output, pack_input
+from .ckks import Plan, fold_output, pack_input, plain_slots
 
 
 def rot_left(v: np.ndarray, steps: int) -> np.ndarray:
@@ -21,19 +21,19 @@ def linear_slots(W: np.ndarray, x: np.ndarray, plan: Plan, n: int) -> np.ndarray
     plan.check(n)
     d_out, d_in = W.shape
     D = plan.D
-    n_in, n_out = -(-d_in // D), -(-d_out // D)
+    n_in, n_out = -(-d_in // D), plan.n_out(d_out)
     xp = np.zeros(n_in * D)
     xp[:d_in] = x
     packed = [pack_input(xp[q * D:(q + 1) * D], plan, n) for q in range(n_in)]
     y = np.zeros(d_out)
     for p in range(n_out):
-        Y = np.zeros(n)
+        Y = np.zeros(n, dtype=np.complex128 if plan.pack == "complex" else np.float64)
         for j in range(plan.g):
-            inner = np.zeros(n)
+            inner = np.zeros_like(Y)
             for q in range(n_in):
                 for k in range(plan.b):
-                    inner += bsgs_plain_slots(W, plan, p, q, j, k, n) * rot_left(packed[q], k * plan.tau)
+                    inner += plain_slots(W, plan, p, q, j, k, n) * rot_left(packed[q], k * plan.tau)
             Y += rot_left(inner, j * plan.b * plan.tau)
-        rows = min(D, d_out - p * D)
-        y[p * D:p * D + rows] = fold_output(Y, plan, p, d_out)
+        part = fold_output(Y, plan, p, d_out)
+        y[p * plan.rows_per_ct:p * plan.rows_per_ct + len(part)] = part
     return y

@@ -73,6 +73,8 @@ _SIGNATURES = {
     "bf_kernel_category_name": (ctypes.c_char_p, [ctypes.c_int]),
     "bf_get_kernel_stats": (ctypes.c_int, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(ctypes.c_float)]),
     "bf_measure_imad_rate": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
+    "bf_measure_fma64_rate": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
+    "bf_get_key_stream_bytes": (ctypes.c_int, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(_u64)]),
     "bf_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "bf_last_cuda_error": (ctypes.c_char_p, [_vp]),
 }
@@ -266,3 +268,16 @@ def bf_measure_imad_rate(ctx) -> float:
     out = ctypes.c_double(0.0)
     _check(load().bf_measure_imad_rate(ctx, ctypes.byref(out)), "bf_measure_imad_rate", ctx)
     return out.value
+
+
+def bf_measure_fma64_rate(ctx) -> float:
+    out = ctypes.c_double(0.0)
+    _check(load().bf_measure_fma64_rate(ctx, ctypes.byref(out)), "bf_measure_fma64_rate", ctx)
+    return out.value
+
+
+def bf_get_key_stream_bytes(ctx) -> tuple[int, int]:
+    """(bytes counted once per distinct key of each launch, bytes counted once per rotation) since the previous call."""
+    a, b = _u64(0), _u64(0)
+    _check(load().bf_get_key_stream_bytes(ctx, ctypes.byref(a), ctypes.byref(b)), "bf_get_key_stream_bytes", ctx)
+    return int(a.value), int(b.value)

@@ -118,6 +118,7 @@ struct bf_ctx {
         u32 seen = 0;
         bool unusable = false;
         uint64_t launches[CAT_COUNT] = {0};
+        uint64_t key_bytes_distinct = 0, key_bytes_per_rotation = 0;
     };
     struct GraphKey {
         const void *ct_in, *weights, *ct_out;
@@ -1011,6 +1012,8 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     if (ge.exec && ge.epoch == ctx->epoch) {
         CK(cudaGraphLaunch(ge.exec, ctx->stream));
         for (int c = 0; c < (int)CAT_COUNT; ++c) ctx->prof.launches[c] += ge.launches[c];
+        ctx->prof.key_bytes_distinct += ge.key_bytes_distinct;
+        ctx->prof.key_bytes_per_rotation += ge.key_bytes_per_rotation;
         return BF_OK;
     }
     if (ge.exec) {                       // stale: buffers, keys or weights changed since the capture
@@ -1028,6 +1031,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     // second call: capture, instantiate, launch
     uint64_t before[CAT_COUNT];
     for (int c = 0; c < (int)CAT_COUNT; ++c) before[c] = ctx->prof.launches[c];
+    const uint64_t kd_before = ctx->prof.key_bytes_distinct, kr_before = ctx->prof.key_bytes_per_rotation;
     if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         cudaGetLastError();
         ge.unusable = true;
@@ -1044,6 +1048,8 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         cudaGetLastError();
         if (graph) cudaGraphDestroy(graph);
         for (int c = 0; c < (int)CAT_COUNT; ++c) ctx->prof.launches[c] = before[c];
+        ctx->prof.key_bytes_distinct = kd_before;
+        ctx->prof.key_bytes_per_rotation = kr_before;
         ge.unusable = true;
         if (rc != BF_OK) return rc;      // argument errors are reported as usual
         return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
@@ -1054,10 +1060,14 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     if (ei != cudaSuccess || !exec) {
         cudaGetLastError();
         for (int c = 0; c < (int)CAT_COUNT; ++c) ctx->prof.launches[c] = before[c];
+        ctx->prof.key_bytes_distinct = kd_before;
+        ctx->prof.key_bytes_per_rotation = kr_before;
         ge.unusable = true;
         return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
     }
     for (int c = 0; c < (int)CAT_COUNT; ++c) ge.launches[c] = ctx->prof.launches[c] - before[c];
+    ge.key_bytes_distinct = ctx->prof.key_bytes_distinct - kd_before;
+    ge.key_bytes_per_rotation = ctx->prof.key_bytes_per_rotation - kr_before;
     ge.exec = exec;
     ge.epoch = ctx->epoch;
     CK(cudaGraphLaunch(ge.exec, ctx->stream));
@@ -1340,8 +1350,16 @@ extern "C" int bf_get_kernel_stats(bf_ctx* ctx, uint64_t* launches_out, float* m
     return BF_OK;
 }
 
-extern "C" int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out) {
-    if (!ctx || !mad_per_second_out) return BF_ERR_INVALID_ARG;
+extern "C" int bf_get_key_stream_bytes(bf_ctx* ctx, uint64_t* distinct_out, uint64_t* per_rotation_out) {
+    if (!ctx || !distinct_out || !per_rotation_out) return BF_ERR_INVALID_ARG;
+    *distinct_out = ctx->prof.key_bytes_distinct;
+    *per_rotation_out = ctx->prof.key_bytes_per_rotation;
+    ctx->prof.key_bytes_distinct = ctx->prof.key_bytes_per_rotation = 0;
+    return BF_OK;
+}
+
+static int measure_rate(bf_ctx* ctx, bool fp64, double* out) {
+    if (!ctx || !out) return BF_ERR_INVALID_ARG;
     TRY(ensure(ctx, ctx->nm_a, 4096));
     cudaDeviceProp prop;
     CK(cudaGetDeviceProperties(&prop, ctx->device));
@@ -1352,7 +1370,8 @@ extern "C" int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out) {
     double best = 0.0;
     for (int rep = 0; rep < 5; ++rep) {
         CK(cudaEventRecord(a, ctx->stream));
-        CK(launch_imad_probe((u64*)ctx->nm_a.p, blocks, iters, ctx->stream));
+        CK(fp64 ? launch_fma64_probe((u64*)ctx->nm_a.p, blocks, iters, ctx->stream)
+                : launch_imad_probe((u64*)ctx->nm_a.p, blocks, iters, ctx->stream));
         CK(cudaEventRecord(b, ctx->stream));
         CK(cudaEventSynchronize(b));
         float ms = 0.f;
@@ -1362,8 +1381,16 @@ extern "C" int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out) {
     }
     cudaEventDestroy(a);
     cudaEventDestroy(b);
-    *mad_per_second_out = best;
+    *out = best;
     return BF_OK;
+}
+
+extern "C" int bf_measure_imad_rate(bf_ctx* ctx, double* mad_per_second_out) {
+    return measure_rate(ctx, false, mad_per_second_out);
+}
+
+extern "C" int bf_measure_fma64_rate(bf_ctx* ctx, double* fma_per_second_out) {
+    return measure_rate(ctx, true, fma_per_second_out);
 }
 
 // ------------------------------------------------------------------------------------------------

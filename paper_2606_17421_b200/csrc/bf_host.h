@@ -25,6 +25,9 @@ enum KernelCat : int {
 struct Profiler {
     bool timing = false;
     uint64_t launches[CAT_COUNT] = {0};
+    // key-switch inner products: bytes of rotation keys counted once per distinct key of a launch (what must come
+    // from HBM) and once per rotation (what the launch reads, L2 hits included)
+    uint64_t key_bytes_distinct = 0, key_bytes_per_rotation = 0;
     struct Rec { int cat; cudaEvent_t a, b; };
     std::vector<Rec> recs;            // event pairs recorded since the last collection
     std::vector<cudaEvent_t> pool;    // idle events
@@ -95,6 +98,7 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
                            const u64* invs, const u64* qlmod, cudaStream_t stream);
 
 cudaError_t launch_imad_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream);   // 64 mad.wide per iteration and thread
+cudaError_t launch_fma64_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream);  // 64 fma.rn.f64 per iteration and thread
 
 // ---- encode.cu : canonical-embedding encoder (fp64) for weight diagonals
 struct EncodeTables {

@@ -594,6 +594,17 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
     const u32 small_ok = (qmax < ((u64)1 << 50)) ? 1u : 0u;
     ProfScope prof(ring.prof, CAT_KEY_INNER, stream);
     const u32 r = ring.dev.r;
+    if (ring.prof) {
+        const u64 key_bytes = (u64)r * 2 * (r + 1) * ring.dev.N * 8;
+        u32 distinct = 0;
+        for (int t = 0; t < rb.n; ++t) {
+            bool seen = false;
+            for (int k = 0; k < t && !seen; ++k) seen = rb.key[k] == rb.key[t];
+            distinct += seen ? 0u : 1u;
+        }
+        ring.prof->key_bytes_distinct += distinct * key_bytes;
+        ring.prof->key_bytes_per_rotation += (u64)rb.n * key_bytes;
+    }
     const size_t smem = (size_t)3 * r * KI_TILE * 8 + 16;
     static bool attr_set[MAX_DEVICES] = {false};     // per device: the attribute belongs to the device's copy of the kernel
     if (!attr_set[device_slot(ring)]) {
@@ -709,6 +720,31 @@ __global__ void __launch_bounds__(256) imad_probe_kernel(u64* __restrict__ sink,
 
 cudaError_t launch_imad_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream) {
     imad_probe_kernel<<<blocks, 256, 0, stream>>>(sink, iters);
+    return cudaGetLastError();
+}
+
+// The same probe for the fp64 fused multiply-add that the transforms of the ciphertext primes are made of:
+// every thread runs 8 independent fma.rn.f64 chains.
+__global__ void __launch_bounds__(256) fma64_probe_kernel(u64* __restrict__ sink, u32 iters) {
+    const double b = 1.0 + (double)(threadIdx.x + blockIdx.x * 256u) * 1e-9;
+    double c[8], d[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { c[k] = b + k; d[k] = 1e-3 * (k + 1); }
+    for (u32 i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) asm volatile("fma.rn.f64 %0, %1, %0, %2;" : "+d"(c[k]) : "d"(b), "d"(d[(k + 1) & 7]));
+        }
+    }
+    double v = 0.0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v += c[k];
+    if (v == 0.1234567) sink[0] = (u64)__double_as_longlong(v);      // practically never true; keeps the chains alive
+}
+
+cudaError_t launch_fma64_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream) {
+    fma64_probe_kernel<<<blocks, 256, 0, stream>>>(sink, iters);
     return cudaGetLastError();
 }
 

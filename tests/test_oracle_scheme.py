@@ -274,3 +274,173 @@ def test_linear_then_fold_in_ciphertext_gives_the_product():
         part = ckks.folded_output(ckks.decode(ckks.decrypt(par, s, low), par.N, out_scale), plan, p, 37)
         y[p * plan.D:p * plan.D + len(part)] = part
     assert np.abs(y - W.astype(np.float64) @ x).max() < 1e-6
+
+
+# ------------------------------------------------------------------ key switch before the division by P
+
+def negacyclic_int(a, b, N):
+    """Schoolbook product of two integer polynomials modulo X^N + 1 (Python integers)."""
+    out = [0] * N
+    for i in range(N):
+        if a[i] == 0:
+            continue
+        for j in range(N):
+            if b[j] == 0:
+                continue
+            k = i + j
+            if k < N:
+                out[k] += a[i] * b[j]
+            else:
+                out[k - N] -= a[i] * b[j]
+    return out
+
+
+def test_key_switch_ext_is_P_times_the_rotated_product_plus_small_noise(ring64):
+    # Over the full basis {q_i, P}: u0 + u1*s = P * (phi_g(c1) * phi_g(s) mod Q) + sum_j digit_j * e_j, with the
+    # last term below r * N * q_max * 6 sigma.  Checked with Python integers through the CRT.
+    par, s = ring64
+    N = par.N
+    rng = np.random.default_rng(31)
+    c1 = ckks.sample_uniform(rng, par.primes, N)
+    g = ckks.galois_element(3, N)
+    key = ckks.galois_key(par, s, g, 32)
+    u = ckks.key_switch_ext(par, c1, g, key)
+    assert u.shape == (2, par.r + 1, N)
+    Q = reduce(lambda a, b: a * b, par.primes)
+    QP = Q * par.P
+    u0 = [crt(u[0, :, k], par.basis)[0] for k in range(N)]
+    u1 = [crt(u[1, :, k], par.basis)[0] for k in range(N)]
+    lhs = [(a + b) % QP for a, b in zip(u0, negacyclic_int(u1, [int(v) for v in s], N))]
+    # phi_g of c1 (as the integer in [0, Q)) and of s, by the definition i -> i*g mod 2N with X^N = -1
+    def phi(poly):
+        out = [0] * N
+        for i, v in enumerate(poly):
+            k = (i * g) % (2 * N)
+            if k < N:
+                out[k] = v
+            else:
+                out[k - N] = -v
+        return out
+    c1_int = [crt(c1[:, k], par.primes)[0] for k in range(N)]
+    prod = [v % Q for v in negacyclic_int(phi(c1_int), phi([int(v) for v in s]), N)]
+    bound = par.r * N * max(par.primes) * 6 * 3.2
+    for k in range(N):
+        diff = centred((lhs[k] - par.P * prod[k]) % QP, QP)
+        assert abs(diff) <= bound
+
+
+def test_rotate_galois_is_key_switch_ext_then_mod_down(ring64):
+    par, s = ring64
+    rng = np.random.default_rng(33)
+    ct = np.stack([ckks.sample_uniform(rng, par.primes, par.N) for _ in range(2)])
+    g = ckks.galois_element(5, par.N)
+    key = ckks.galois_key(par, s, g, 34)
+    u = ckks.key_switch_ext(par, ct[1], g, key)
+    rot = ckks.rotate_galois(par, ct, g, key)
+    for i, q in enumerate(par.primes):
+        c0g = ckks.automorphism(ct[0, i], g, q)
+        assert np.array_equal(rot[0, i], (c0g + ckks.mod_down(u[0], par)[i]) % np.uint64(q))
+        assert np.array_equal(rot[1, i], ckks.mod_down(u[1], par)[i])
+
+
+# ------------------------------------------------------------------ plan modes: complex packing, one division by P per output
+
+COMPLEX_PLANS = [(64, 1, 8, 8, 2048), (64, 4, 4, 4, 512), (8, 2, 2, 2, 32), (1024, 16, 16, 4, 16384),
+                 (1024, 32, 8, 4, 32768)]
+
+
+@pytest.mark.parametrize("D,tau,b,g,n", COMPLEX_PLANS)
+def test_slot_simulator_with_complex_packing_equals_matvec(D, tau, b, g, n):
+    # two row blocks per output ciphertext (real and imaginary parts); shapes with an even and an odd number of
+    # row blocks (the last ciphertext then carries one block only) and ragged edges
+    rng = np.random.default_rng(D + tau + 1)
+    plan = Plan(D, tau, b, g, pack="complex")
+    for d_out, d_in in ((2 * D, D), (3 * D, D + 5), (D + 3, 2 * D - 5), (3 * D // 4, D)):
+        W = rng.normal(size=(d_out, d_in))
+        x = rng.normal(size=d_in)
+        assert plan.n_out(d_out) == -(-d_out // (2 * D))
+        y = slotsim.linear_slots(W, x, plan, n)
+        assert np.abs(y - W @ x).max() < 1e-10
+
+
+def test_complex_plaintext_is_the_two_real_ones_combined():
+    # encode is linear up to rounding: the coefficients of (block 2p) + i (block 2p+1) differ from
+    # enc(block 2p) + enc(i * block 2p+1) by at most one unit per coefficient (two roundings against one)
+    N, n = 256, 128
+    plan_r, plan_c = Plan(16, 4, 2, 2), Plan(16, 4, 2, 2, pack="complex")
+    W = wl.gen_weights(5, "c", 40, 20)
+    for (p, q, j, k) in ((0, 0, 0, 0), (0, 1, 1, 1), (1, 0, 1, 0)):
+        zc = ckks.plain_slots(W, plan_c, p, q, j, k, n)
+        za = ckks.plain_slots(W, plan_r, 2 * p, q, j, k, n)
+        zb = ckks.plain_slots(W, plan_r, 2 * p + 1, q, j, k, n)
+        assert np.array_equal(zc, za + 1j * zb)
+        mc = ckks.encode_coeffs(zc, N, 2.0 ** 40)
+        ma = ckks.encode_coeffs(za, N, 2.0 ** 40)
+        mb = ckks.encode_coeffs(1j * zb, N, 2.0 ** 40)
+        assert np.abs(mc - (ma + mb)).max() <= 1
+        assert np.array_equal(ckks.encode_complex_batch(zc[None], N, 2.0 ** 40)[0], mc)
+    # block 3 of a 40-row matrix with D = 16 does not exist: the imaginary part of ciphertext 1 is empty
+    assert not ckks.plain_slots(W, plan_c, 1, 0, 0, 0, n).imag.any()
+
+
+def run_linear_modes(par, plan, W, x, seed, tol):
+    s = ckks.keygen(par, seed)
+    keys = ckks.make_rotation_keys(par, s, plan, seed)
+    cts = ckks.encrypt_vector(par, plan, s, x, seed)
+    out = ckks.linear(par, plan, cts, W, keys)
+    d_out = W.shape[0]
+    assert sorted(out) == list(range(plan.n_out(d_out)))
+    y = np.zeros(d_out)
+    out_scale = par.scale * par.scale / par.primes[-1]
+    for p, ct in out.items():
+        low = ckks.rescale(par, ct)
+        part = ckks.fold_output(ckks.decode(ckks.decrypt(par, s, low), par.N, out_scale), plan, p, d_out)
+        y[p * plan.rows_per_ct:p * plan.rows_per_ct + len(part)] = part
+    err = np.abs(y - W.astype(np.float64) @ x).max()
+    assert err < tol, err
+    return out, s, keys, cts
+
+
+@pytest.mark.parametrize("pack,moddown", [("complex", "per_rotation"), ("real", "per_output"), ("complex", "per_output")])
+def test_end_to_end_plan_modes_small_ring(pack, moddown):
+    N = 256
+    primes, P = ckks.prime_chain(N, 2)
+    par = Params(N, primes, P, 2.0 ** 40)
+    W = wl.gen_weights(0, "m", 37, 41)            # 3 row blocks of 16: with complex packing two ciphertexts
+    x = wl.gen_activation(0, "m", 41)
+    run_linear_modes(par, Plan(16, 4, 2, 2, pack=pack, moddown=moddown), W, x, 1, 1e-6)
+    run_linear_modes(par, Plan(16, 1, 4, 4, pack=pack, moddown=moddown), W, x, 2, 1e-6)
+    run_linear_modes(par, Plan(16, 8, 2, 1, pack=pack, moddown=moddown), W, x, 3, 1e-6)     # no giant step
+
+
+def test_per_output_moddown_differs_from_per_rotation_only_by_rounding():
+    # the two modes divide by P at different points, so residues differ, but only by the rounding of the g - 1
+    # divisions: centred difference at most g - 1 units per coefficient (both are within 1/2 of the same real
+    # quotient per rotation, summed), and the decrypted results agree to far below the tolerance
+    N = 256
+    primes, P = ckks.prime_chain(N, 2)
+    par = Params(N, primes, P, 2.0 ** 40)
+    W = wl.gen_weights(7, "pm", 30, 33)
+    x = wl.gen_activation(7, "pm", 33)
+    plan_a = Plan(16, 1, 4, 4)
+    plan_b = Plan(16, 1, 4, 4, moddown="per_output")
+    out_a, s, keys, cts = run_linear_modes(par, plan_a, W, x, 7, 1e-6)
+    out_b = ckks.linear(par, plan_b, cts, W, keys)
+    Q = reduce(lambda a, b: a * b, par.primes)
+    differs = False
+    for p in out_a:
+        assert out_a[p].shape == out_b[p].shape
+        differs = differs or not np.array_equal(out_a[p], out_b[p])
+        for comp in range(2):
+            for k in range(0, N, 3):
+                a, _ = crt(out_a[p][comp, :, k], par.primes)
+                b, _ = crt(out_b[p][comp, :, k], par.primes)
+                assert abs(centred((a - b) % Q, Q)) <= plan_a.g - 1
+    assert differs                                  # the mode is really read
+    # with a single giant step there is nothing to merge: identical residues
+    plan_c, plan_d = Plan(16, 4, 4, 1), Plan(16, 4, 4, 1, moddown="per_output")
+    s2 = ckks.keygen(par, 8)
+    keys2 = ckks.make_rotation_keys(par, s2, plan_c, 8)
+    cts2 = ckks.encrypt_vector(par, plan_c, s2, x, 8)
+    o_c, o_d = ckks.linear(par, plan_c, cts2, W, keys2), ckks.linear(par, plan_d, cts2, W, keys2)
+    assert all(np.array_equal(o_c[p], o_d[p]) for p in o_c)
