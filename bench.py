@@ -106,7 +106,9 @@ MIN_REGION_S = 0.5      # every timed region lasts at least this long (steps are
 
 # Workload specifications: "<workload>[@option[,option...]]".  Options: budget=<GB> (cache budget, so that
 # overflow layers take the on-the-fly path), on_the_fly (budget of one byte: nothing is cached), compact
-# (compact cache format), fold (in-ciphertext fold of the tau partial sums).
+# (compact cache format), fold (in-ciphertext fold of the tau partial sums), complex (two output row blocks per
+# plaintext, in the real and imaginary parts of the slots), per_output (one division by the special prime per
+# output ciphertext instead of one per giant rotation).
 DEFAULT_WORKLOAD = "qwen3_step@budget=60"
 DEFAULT_EXTRA = ("gpt2_qkv,gpt2_step,qwen3_step@budget=40.5,qwen3_step@budget=40.5,compact,"
                  "llama3_layer,llama3_layer@on_the_fly,tiny")
@@ -124,6 +126,10 @@ def parse_spec(spec: str):
             kw["compact_cache"] = True
         elif o == "fold":
             kw["fold_in_ciphertext"] = True
+        elif o == "complex":
+            kw["pack"] = "complex"
+        elif o == "per_output":
+            kw["moddown"] = "per_output"
         else:
             raise ValueError(f"unknown workload option {o!r}")
     return name, kw

@@ -49,9 +49,25 @@ typedef struct bf_weights bf_weights;  /* device-resident encoded diagonals of o
  * baby-step/giant-step objects, Sec. 4.2):  the weight matrix is cut into tile_D x tile_D tiles;
  * slot s = (rho*tile_D + kappa)*tau + c of an input ciphertext holds x[(kappa + c*M) mod tile_D]
  * of its chunk, M = tile_D/tau generalised diagonals per tile, split as M = bsgs_b * bsgs_g.
- * All four are powers of two and tile_D*tau <= N/2. */
+ * All four are powers of two and tile_D*tau <= N/2.
+ * flags select variants of the evaluation that change the output residues (each is mirrored by a mode
+ * of the CPU reference the tests compare with); 0 = the plain evaluation:
+ *   BF_PLAN_COMPLEX_PACK       two output row blocks share one plaintext, block 2P in the real parts
+ *       of the slots and block 2P+1 in the imaginary parts (the input ciphertexts stay real), so
+ *       that output ciphertext P decrypts to (rows of block 2P) + i (rows of block 2P+1): half the
+ *       diagonals, half the encoded-weight bytes (the memory wall of Sec. 6.1), half the giant
+ *       rotations.  n_out = ceil(ceil(d_out / tile_D) / 2) output ciphertexts.
+ *   BF_PLAN_MODDOWN_PER_OUTPUT the key-switch results of an output's giant rotations are summed in
+ *       the extended basis {q_i, P} and divided by P once per output ciphertext and component
+ *       instead of once per rotation (Sec. 4.2 leaves the key-switching primitive open).  Needs
+ *       bsgs_g - 1 <= 64. */
+enum {
+    BF_PLAN_COMPLEX_PACK = 1,
+    BF_PLAN_MODDOWN_PER_OUTPUT = 2
+};
 typedef struct {
     uint32_t tile_D, tau, bsgs_b, bsgs_g;
+    uint32_t flags;                        /* BF_PLAN_* bits */
 } bf_plan;
 
 /* Create a context (Sec. 4.2: one CKKS context per projection shape, with its modulus chain and
@@ -92,7 +108,8 @@ void bf_weights_free(bf_ctx* ctx, bf_weights* w);
 
 /* FHE_Linear (Alg. 3, decode loop; Sec. 4.2 "BSGS matrix-vector multiply"):
  *     ct_out[p] = sum_{j<g} rot( sum_q sum_{k<b} Pt[p][q][j][k] * rot(ct_in[q], k*tau), j*b*tau )
- * for p < n_out = ceil(d_out/tile_D), q < n_in = ceil(d_in/tile_D).  Rotations are automorphisms
+ * for p < n_out = ceil(d_out/tile_D) (half of that, rounded up, with BF_PLAN_COMPLEX_PACK),
+ * q < n_in = ceil(d_in/tile_D).  Rotations are automorphisms
  * followed by a key switch with one special prime (one prime per digit), each with its own
  * division by P.
  *   ct_in       device, n_in ciphertexts at full level, boundary layout
@@ -101,7 +118,8 @@ void bf_weights_free(bf_ctx* ctx, bf_weights* w);
  *   ct_out      device, n_out ciphertexts, full level, scale = scale(ct_in) * Delta; must not
  *               overlap ct_in
  * Slot (0, kappa, c) of ct_out[p] decrypts to the partial dot product of row p*tile_D + kappa over
- * column class c; the caller adds the tau partial sums.  Asynchronous on the context's stream,
+ * column class c (with BF_PLAN_COMPLEX_PACK: rows 2p*tile_D + kappa in the real part and
+ * (2p+1)*tile_D + kappa in the imaginary part); the caller adds the tau partial sums.  Asynchronous on the context's stream,
  * except that scratch memory may be grown (which synchronises) the first time a shape is seen.
  * Errors: INVALID_ARG, SHAPE, MISSING_KEY, OOM, RANGE (fallback path only), CUDA. */
 int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,

@@ -25,9 +25,14 @@ BF_ERR_TOO_LARGE = -9
 BF_ERR_TIMEOUT = -10
 
 
+BF_PLAN_COMPLEX_PACK = 1
+BF_PLAN_MODDOWN_PER_OUTPUT = 2
+
+
 class bf_plan(ctypes.Structure):
+    """bf_plan(tile_D, tau, bsgs_b, bsgs_g[, flags]); flags = BF_PLAN_* bits, 0 by default."""
     _fields_ = [("tile_D", ctypes.c_uint32), ("tau", ctypes.c_uint32),
-                ("bsgs_b", ctypes.c_uint32), ("bsgs_g", ctypes.c_uint32)]
+                ("bsgs_b", ctypes.c_uint32), ("bsgs_g", ctypes.c_uint32), ("flags", ctypes.c_uint32)]
 
 
 class BifrostError(RuntimeError):

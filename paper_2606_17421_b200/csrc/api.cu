@@ -105,9 +105,10 @@ struct bf_ctx {
     std::map<u32, int> key_of_steps;
     u64* keys = nullptr;
     u32* perms = nullptr;            // [n_keys][N] pinv: where position n goes under the key's automorphism
+    u32* perms_fwd = nullptr;        // [n_keys][N] perm: rotated[n] = unrotated[perm[n]] (per-output division by P)
     u32 n_keys = 0;
     // scratch (grow-only)
-    DevBuf X, Dig, U, Tc, Tn, Cc, A, Rres, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
+    DevBuf X, Dig, U, Ubig, Tc, Tn, Cc, A, Rres, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
     u64 cache_budget = 0, cache_used = 0;
     std::vector<bf_weights*> weights;
     std::string cuda_msg;
@@ -222,6 +223,8 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
         (u64)plan->bsgs_b * plan->bsgs_g != plan->tile_D / plan->tau)
         return BF_ERR_SHAPE;
     if (plan->bsgs_b - 1 > (u32)MAX_ROT_BATCH) return BF_ERR_SHAPE;
+    if (plan->flags & ~(u32)(BF_PLAN_COMPLEX_PACK | BF_PLAN_MODDOWN_PER_OUTPUT)) return BF_ERR_INVALID_ARG;
+    if ((plan->flags & BF_PLAN_MODDOWN_PER_OUTPUT) && plan->bsgs_g - 1 > (u32)MAX_ROT_BATCH) return BF_ERR_SHAPE;
 
     bf_ctx* ctx = new (std::nothrow) bf_ctx();
     if (!ctx) return BF_ERR_OOM;
@@ -399,7 +402,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
             delete w;
         }
     }
-    DevBuf* bufs[] = {&ctx->X, &ctx->Dig, &ctx->U, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres,
+    DevBuf* bufs[] = {&ctx->X, &ctx->Dig, &ctx->U, &ctx->Ubig, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres,
                       &ctx->fft, &ctx->coef, &ctx->ptnat, &ctx->ptjit, &ctx->stage_in, &ctx->stage_out, &ctx->nm_a, &ctx->nm_b};
     for (DevBuf* b : bufs) free_buf(*b);
     cudaFree(ctx->tw_fwd);
@@ -416,6 +419,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
     cudaFree(ctx->overflow_flag);
     cudaFree(ctx->keys);
     cudaFree(ctx->perms);
+    cudaFree(ctx->perms_fwd);
     for (cudaEvent_t& e : ctx->ev)
         if (e) cudaEventDestroy(e);
     for (auto& rec : ctx->prof.recs) { cudaEventDestroy(rec.a); cudaEventDestroy(rec.b); }
@@ -432,8 +436,10 @@ static void drop_eval_keys(bf_ctx* ctx) {
     ctx->epoch++;
     cudaFree(ctx->keys);
     cudaFree(ctx->perms);
+    cudaFree(ctx->perms_fwd);
     ctx->keys = nullptr;
     ctx->perms = nullptr;
+    ctx->perms_fwd = nullptr;
     ctx->key_of_steps.clear();
     ctx->n_keys = 0;
 }
@@ -499,11 +505,12 @@ extern "C" int bf_load_eval_keys(bf_ctx* ctx, const uint32_t* rot_steps, uint32_
     cudaError_t ne = ntt_forward_split(ctx->ring, B, n_keys * r * 2, LOAD_REDUCE, ctx->keys, perm_dev, 2 * r, ctx->stream);
     cudaError_t se = cudaStreamSynchronize(ctx->stream);
     cudaFree(stage);
-    cudaFree(perm_dev);
     if (ne != cudaSuccess || se != cudaSuccess) {
+        cudaFree(perm_dev);
         ctx->cuda_msg = std::string("key transform: ") + cudaGetErrorString(ne != cudaSuccess ? ne : se);
         return fail(BF_ERR_CUDA);
     }
+    ctx->perms_fwd = perm_dev;
     ctx->key_of_steps.swap(key_of_steps);
     ctx->n_keys = n_keys;
     ctx->epoch++;
@@ -520,9 +527,15 @@ extern "C" uint64_t bf_cache_bytes_used(const bf_ctx* ctx) { return ctx ? ctx->c
 
 static u32 cdiv(u32 a, u32 b) { return (u32)(((u64)a + b - 1) / b); }
 
+// output ciphertexts of a projection with d_out rows: one per row block of tile_D, or per pair of row blocks
+static u32 n_out_cts(const bf_ctx* ctx, u32 d_out) {
+    const u32 blocks = cdiv(d_out, ctx->plan.tile_D);
+    return (ctx->plan.flags & BF_PLAN_COMPLEX_PACK) ? cdiv(blocks, 2) : blocks;
+}
+
 extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
     if (!ctx) return 0;
-    const u32 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = cdiv(d_out, ctx->plan.tile_D);
+    const u32 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = n_out_cts(ctx, d_out);
     const TileLayout lay = mac_tile_layout(ctx->ring, n_out * ctx->plan.bsgs_g, n_in * ctx->plan.bsgs_b);
     return mac_tile_bytes(ctx->ring, lay);
 }
@@ -553,7 +566,8 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
         db.d_out = d_out;
         db.d_in = d_in;
         db.n_in = cdiv(d_in, ctx->plan.tile_D);
-        db.n_out = cdiv(d_out, ctx->plan.tile_D);
+        db.n_out = n_out_cts(ctx, d_out);
+        db.complex_pack = (ctx->plan.flags & BF_PLAN_COMPLEX_PACK) ? 1u : 0u;
         db.D = ctx->plan.tile_D;
         db.tau = ctx->plan.tau;
         db.b = ctx->plan.bsgs_b;
@@ -609,7 +623,7 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
     w->d_out = d_out;
     w->d_in = d_in;
     w->n_in = cdiv(d_in, ctx->plan.tile_D);
-    w->n_out = cdiv(d_out, ctx->plan.tile_D);
+    w->n_out = n_out_cts(ctx, d_out);
     w->bytes = bytes;
     w->lay = mac_tile_layout(ctx->ring, w->n_out * ctx->plan.bsgs_g, w->n_in * ctx->plan.bsgs_b);
     cudaError_t e = cudaMalloc(&w->pt, bytes);
@@ -719,6 +733,7 @@ static int moddown_batch(bf_ctx* ctx, const Lane& lane, const RotBatch& rb, cons
     B.mod_step = 1;
     B.lift_mod = ctx->ring.q[r];
     ModDownEpilogue epi;
+    memset(&epi, 0, sizeof(epi));
     epi.u = (const u64*)lane.U;
     epi.c0_base = c0_base;
     epi.c0_stride = c0_stride;
@@ -793,7 +808,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     if (!ctx || !ct_in || !ct_out || (!pt_weights && !W_raw) || !d_out || !d_in) return BF_ERR_INVALID_ARG;
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
     const u32 D = ctx->plan.tile_D, tau = ctx->plan.tau, b = ctx->plan.bsgs_b, g = ctx->plan.bsgs_g;
-    if (n_in != cdiv(d_in, D) || n_out != cdiv(d_out, D)) return BF_ERR_SHAPE;
+    if (n_in != cdiv(d_in, D) || n_out != n_out_cts(ctx, d_out)) return BF_ERR_SHAPE;
     if (pt_weights && (pt_weights->d_out != d_out || pt_weights->d_in != d_in)) return BF_ERR_SHAPE;
     const size_t ctw = (size_t)2 * r * N;                 // words per ciphertext
     // rotation keys the plan needs
@@ -832,9 +847,16 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     if (n_dig_sets < in_batch) n_dig_sets = in_batch;
     TRY(ensure(ctx, ctx->X, (size_t)n_in * b * ctw * 8));
     TRY(ensure(ctx, ctx->A, (size_t)n_out * g * ctw * 8));
-    TRY(ensure(ctx, ctx->Rres, (size_t)(n_giant ? n_giant : 1) * ctw * 8));
+    // one division by P per output: the inner products of all giant rotations stay alive until every chain is done
+    const bool per_output = (ctx->plan.flags & BF_PLAN_MODDOWN_PER_OUTPUT) && n_giant > 0;
+    TRY(ensure(ctx, ctx->Rres, (size_t)(per_output ? n_out : n_giant ? n_giant : 1) * ctw * 8));
     TRY(ensure(ctx, ctx->Cc, (size_t)n_dig_sets * r * N * 8));
-    TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_per_lane * (u32)lanes));
+    {
+        u32 rot_scratch = rot_per_lane * (u32)lanes;
+        if (per_output && rot_scratch < n_out) rot_scratch = n_out;     // Tc, Tn of the per-output division
+        TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_scratch));
+    }
+    if (per_output) TRY(ensure(ctx, ctx->Ubig, (size_t)n_giant * 2 * nb * N * 8));
     Lane lane[bf_ctx::MAX_LANES];
     for (int c = 0; c < lanes; ++c) {
         lane[c].s = c == 0 ? ctx->stream : ctx->side[c - 1];
@@ -954,11 +976,56 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
                     rb.c0[t] = (int)t;
                     rb.out[t] = (int)t;
                 }
+                if (per_output) {
+                    CK(launch_key_inner_product(ctx->ring, rb, lane[c].Dig, ctx->keys,
+                                                (u64*)ctx->Ubig.p + (size_t)rho0 * 2 * nb * N, ctx->device_error, lane[c].s));
+                    continue;
+                }
                 CK(launch_key_inner_product(ctx->ring, rb, lane[c].Dig, ctx->keys, lane[c].U, ctx->device_error, lane[c].s));
                 TRY(moddown_batch(ctx, lane[c], rb, Asrc, (long long)ctw, Rres + (size_t)rho0 * ctw, (long long)ctw));
             }
         }
         TRY(join_lanes(ctx, used));
+        if (per_output) {
+            // sum over the giant steps of each output in the extended basis (each term read through its rotation),
+            // then one division by P per output and component; the rotated c0 parts join in the same epilogue
+            RotBatch rb;
+            memset(&rb, 0, sizeof(rb));
+            rb.n = (int)(g - 1);
+            for (u32 j = 1; j < g; ++j) rb.key[j - 1] = giant_key[j];
+            ModDownEpilogue epi;
+            memset(&epi, 0, sizeof(epi));
+            epi.u = (const u64*)ctx->Ubig.p;
+            epi.c0_base = A + (size_t)n_out * ctw;              // ciphertexts with j >= 1, index (j - 1) * n_out + p
+            epi.c0_stride = (long long)ctw;
+            epi.pinv = ctx->perms;
+            epi.perm = ctx->perms_fwd;
+            epi.out_base = Rres;
+            epi.out_stride = (long long)ctw;
+            epi.n_sum = g - 1;
+            epi.n_out = n_out;
+            memset(&B, 0, sizeof(B));
+            B.src = (const u64*)ctx->Ubig.p;                    // (read through epi)
+            B.dst = (u64*)ctx->Tc.p;
+            B.dst_so = N;
+            B.n_m = 1;
+            B.mod0 = r;
+            B.mod_step = 0;
+            B.store_centred = 1;
+            CK(ntt_inverse_gathersum(ctx->ring, B, n_out * 2, rb, epi, ctx->stream));
+            memset(&B, 0, sizeof(B));
+            B.src = (const u64*)ctx->Tc.p;
+            B.dst = (u64*)ctx->Tn.p;
+            B.src_so = N;
+            B.src_sm = 0;
+            B.dst_so = (long long)r * N;
+            B.dst_sm = N;
+            B.n_m = r;
+            B.mod0 = 0;
+            B.mod_step = 1;
+            B.lift_mod = ctx->ring.q[r];
+            CK(ntt_forward_moddown(ctx->ring, B, n_out * 2, rb, epi, ctx->stream));
+        }
     }
     stamp(ctx, 3);
 
@@ -974,7 +1041,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     B.mod0 = 0;
     B.mod_step = 1;
     B.sum_src = Rres;
-    B.sum_terms = g - 1;
+    B.sum_terms = per_output ? 1 : g - 1;
     B.sum_stride = (long long)n_out * ctw;
     CK(ntt_inverse(ctx->ring, B, n_out, ctx->stream));
     stamp(ctx, 4);

@@ -236,6 +236,14 @@ struct RotBatch {                     // one key-switch launch over n rotations
 // (polynomial (o, m) = (rotation*2 + component, prime i)):  instead of storing t = NTT(lift),
 //   v = (u[o][i][n] - t) * P^{-1} + (component == 0 ? c0[c0(rot)][i][n] : 0)
 // is scattered to out[out(rot)][component][i][pinv[key(rot)][n]].
+//
+// Per-output form (n_sum > 0; one division by P per output ciphertext and component): polynomial (o, m) =
+// (output p * 2 + component, prime i).  The inner products of the n_sum giant rotations of output p sit in u at
+// rotation index jj * n_out + p (jj < n_sum, key rb.key[jj]), un-rotated; they are summed through each
+// rotation's permutation (rotated[n] = unrotated[perm[n]]), the inverse transform reads the P-residues that
+// way, and the forward transform's last store computes
+//   v[n] = (sum_jj u[jj][i][perm_jj[n]] - t[n]) * P^{-1} + (component == 0 ? sum_jj c0[jj][i][perm_jj[n]] : 0)
+// into out[p][component][i][n] (no scatter), with c0 of rotation index jj * n_out + p at c0_base + index * c0_stride.
 struct ModDownEpilogue {
     const u64* u;                 // [rot][2][r+1][N]
     const u64* c0_base;
@@ -243,6 +251,8 @@ struct ModDownEpilogue {
     const u32* pinv;              // [n_keys][N]
     u64* out_base;
     long long out_stride;
+    const u32* perm;              // [n_keys][N] (per-output form)
+    u32 n_sum, n_out;             // per-output form: giant steps summed per output, number of outputs
 };
 
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks

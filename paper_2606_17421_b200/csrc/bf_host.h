@@ -79,6 +79,9 @@ cudaError_t ntt_inverse(const RingHost& ring, const PolyBatch& B, u32 n_outer, c
 // Forward transform of the centred lifts of P-residues with the ModDown epilogue fused into its last store.
 cudaError_t ntt_forward_moddown(const RingHost& ring, const PolyBatch& B, u32 n_outer, const RotBatch& rb,
                                 const ModDownEpilogue& epi, cudaStream_t stream);
+// Inverse transform of the P-residues summed over the giant rotations of each output (per-output form of epi).
+cudaError_t ntt_inverse_gathersum(const RingHost& ring, const PolyBatch& B, u32 n_outer, const RotBatch& rb,
+                                  const ModDownEpilogue& epi, cudaStream_t stream);
 cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B, u32 n_outer, int load, u64* final_dst,
                               const u32* scatter, u32 scatter_div, cudaStream_t stream);
 
@@ -111,6 +114,7 @@ struct DiagBatch {                    // diagonals d0 .. d0+count-1 in [j][p][q]
     const float* W;
     u32 d_out, d_in, n_in, n_out, D, tau, b, g;
     u32 d0, count;
+    u32 complex_pack;                 // two row blocks per plaintext: block 2p in the real parts, 2p+1 in the imaginary
 };
 cudaError_t launch_encode(const RingHost& ring, const EncodeTables& tab, const DiagBatch& db, double2* fft_scratch,
                           i64* coeff_out, int* overflow_flag, cudaStream_t stream);

@@ -29,8 +29,10 @@ __device__ __forceinline__ double2 cmul_rn(double2 b, double2 w) {
 
 // Slot value of plaintext Pt[p][q][j][k] at slot s: generalised diagonal i = j*b + k of tile (p, q),
 // pre-rotated right by j*b*tau.  Slot s' = (rho*D + kappa)*tau + c holds
-// W[p*D + kappa][q*D + ((kappa + i + c*M) mod D)], zero outside the matrix.
-__device__ __forceinline__ double diag_value(const DiagBatch& db, u32 dd, u32 s, u32 n) {
+// W[p*D + kappa][q*D + ((kappa + i + c*M) mod D)], zero outside the matrix.  With complex packing output
+// ciphertext p carries two row blocks: W[2p*D + kappa][..] in the real part, W[(2p+1)*D + kappa][..] in
+// the imaginary part.
+__device__ __forceinline__ double2 diag_value(const DiagBatch& db, u32 dd, u32 s, u32 n) {
     const u32 k = dd % db.b;
     const u32 q = (dd / db.b) % db.n_in;
     const u32 p = (dd / (db.b * db.n_in)) % db.n_out;
@@ -39,10 +41,13 @@ __device__ __forceinline__ double diag_value(const DiagBatch& db, u32 dd, u32 s,
     const u32 c = sp % db.tau;
     const u32 kappa = (sp / db.tau) % db.D;
     const u32 M = db.D / db.tau;
-    const u32 row = p * db.D + kappa;
+    const u32 row = p * db.D * (db.complex_pack ? 2u : 1u) + kappa;
     const u32 col = q * db.D + ((kappa + j * db.b + k + c * M) % db.D);
-    if (row >= db.d_out || col >= db.d_in) return 0.0;
-    return (double)__ldg(&db.W[(size_t)row * db.d_in + col]);
+    double2 v = make_double2(0.0, 0.0);
+    if (col >= db.d_in) return v;
+    if (row < db.d_out) v.x = (double)__ldg(&db.W[(size_t)row * db.d_in + col]);
+    if (db.complex_pack && row + db.D < db.d_out) v.y = (double)__ldg(&db.W[(size_t)(row + db.D) * db.d_in + col]);
+    return v;
 }
 
 // One pass of the batched FFT.  CONTIG = the first pass (chunks of adjacent points, small butterfly
@@ -84,8 +89,7 @@ __global__ void __launch_bounds__(256) encode_fft_pass(const EncodeTables tab, c
                     if (g_first) {
                         const u32 gidx = CONTIG ? (u32)(lane0 + lane) * LEN + li : (u32)li * other + lane0 + lane;
                         if (CONTIG) {
-                            e[i].x = diag_value(db, db.d0 + diag, __ldg(&tab.slot_of_pos[gidx]), n);
-                            e[i].y = 0.0;
+                            e[i] = diag_value(db, db.d0 + diag, __ldg(&tab.slot_of_pos[gidx]), n);
                         } else {
                             e[i] = buf[gidx];
                         }
@@ -183,7 +187,7 @@ __device__ __forceinline__ DiagPos diag_pos(const DiagBatch& db, u32 dd) {
     const u32 p = (dd / (db.b * db.n_in)) % db.n_out;
     const u32 j = dd / (db.b * db.n_in * db.n_out);
     dp.rot = j * db.b * db.tau;
-    dp.row0 = p * db.D;
+    dp.row0 = p * db.D * (db.complex_pack ? 2u : 1u);
     dp.col0 = q * db.D;
     dp.ik = j * db.b + k;
     dp.log_tau = 31u - (u32)__clz(db.tau);
@@ -192,14 +196,17 @@ __device__ __forceinline__ DiagPos diag_pos(const DiagBatch& db, u32 dd) {
     dp.M = db.D >> dp.log_tau;
     return dp;
 }
-__device__ __forceinline__ double diag_value_at(const DiagBatch& db, const DiagPos& dp, u32 s, u32 n) {
+__device__ __forceinline__ double2 diag_value_at(const DiagBatch& db, const DiagPos& dp, u32 s, u32 n) {
     const u32 sp = (s - dp.rot) & (n - 1);
     const u32 c = sp & (dp.tau - 1);
     const u32 kappa = (sp >> dp.log_tau) & (dp.D - 1);
     const u32 row = dp.row0 + kappa;
     const u32 col = dp.col0 + ((kappa + dp.ik + c * dp.M) & (dp.D - 1));
-    if (row >= db.d_out || col >= db.d_in) return 0.0;
-    return (double)__ldg(&db.W[(size_t)row * db.d_in + col]);
+    double2 v = make_double2(0.0, 0.0);
+    if (col >= db.d_in) return v;
+    if (row < db.d_out) v.x = (double)__ldg(&db.W[(size_t)row * db.d_in + col]);
+    if (db.complex_pack && row + dp.D < db.d_out) v.y = (double)__ldg(&db.W[(size_t)(row + dp.D) * db.d_in + col]);
+    return v;
 }
 
 // Shared-memory slot of point li of chunk `lane` in the contiguous pass: 16-byte elements, eight to a row
@@ -235,8 +242,7 @@ __device__ __forceinline__ void fft_group(const EncodeTables& tab, const DiagBat
             if (FIRST) {
                 const u32 gidx = CONTIG ? ((u32)(lane0 + lane) << LOG_LEN) + li : ((u32)li << LOG_OTHER) + lane0 + lane;
                 if (CONTIG) {
-                    e[i].x = diag_value_at(db, dp, __ldg(&tab.slot_of_pos[gidx]), n);
-                    e[i].y = 0.0;
+                    e[i] = diag_value_at(db, dp, __ldg(&tab.slot_of_pos[gidx]), n);
                 } else {
                     e[i] = buf[gidx];
                 }

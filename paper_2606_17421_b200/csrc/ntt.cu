@@ -511,7 +511,9 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
 // Forward: second pass (final reduction to [0, q), then the store functors).  Inverse: first pass
 // (reads the batch source: plain residues, tiled/limb-split plaintexts, or a sum of arrays).
 // TILED: the transform-domain side of the batch lives in the tile-major plaintext cache (B.tile_ptr).
-template <bool FWD, bool EPI, bool FP, bool TILED>
+// EPI: 0 = none; 1 = division by P per rotation (scatter through the rotation's permutation); 2 = per output
+// (sum over the output's giant rotations, gathered through their permutations; see ModDownEpilogue).
+template <bool FWD, int EPI, bool FP, bool TILED>
 __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, u32 o, u32 m, u32 mod,
                                             u32 chunk, int lane, const RotBatch& rb, const ModDownEpilogue& epi) {
     typedef typename Elem<FP>::T T;
@@ -554,7 +556,23 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
             // the epilogue's operands do not depend on the transform: ask for them before the last butterflies
             u64 uu[4] = {0, 0, 0, 0}, cc[4] = {0, 0, 0, 0};
             u32 pp[4] = {0, 0, 0, 0};
-            if (EPI) {
+            if (EPI == 2) {
+                const u32 pp_out = o >> 1, comp = o & 1, ip = mod, nb = R.r + 1;
+                const size_t n = (size_t)chunk * LEN + 4 * s;
+                for (u32 jj = 0; jj < epi.n_sum; ++jj) {
+                    const uint4 pv = *(const uint4*)(epi.perm + (size_t)rb.key[jj] * R.N + n);
+                    const size_t rot = (size_t)jj * epi.n_out + pp_out;
+                    const u64* up = epi.u + ((rot * 2 + comp) * nb + ip) * R.N;
+                    uu[0] = add_mod(uu[0], __ldg(up + pv.x), q); uu[1] = add_mod(uu[1], __ldg(up + pv.y), q);
+                    uu[2] = add_mod(uu[2], __ldg(up + pv.z), q); uu[3] = add_mod(uu[3], __ldg(up + pv.w), q);
+                    if (comp == 0) {
+                        const u64* cp = epi.c0_base + rot * epi.c0_stride + (size_t)ip * R.N;
+                        cc[0] = add_mod(cc[0], __ldg(cp + pv.x), q); cc[1] = add_mod(cc[1], __ldg(cp + pv.y), q);
+                        cc[2] = add_mod(cc[2], __ldg(cp + pv.z), q); cc[3] = add_mod(cc[3], __ldg(cp + pv.w), q);
+                    }
+                }
+            }
+            if (EPI == 1) {
                 const u32 rot = o >> 1, comp = o & 1, ip = mod, nb = R.r + 1;
                 const size_t n = (size_t)chunk * LEN + 4 * s;
                 const u64* up = epi.u + ((size_t)o * nb + ip) * R.N + n;
@@ -587,7 +605,17 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                     v4[i] = v;
                 }
             }
-            if (EPI) {
+            if (EPI == 2) {
+                const u32 pp_out = o >> 1, comp = o & 1, ip = mod, r = R.r;
+                u64* op = epi.out_base + (size_t)pp_out * epi.out_stride + ((size_t)comp * r + ip) * R.N + (size_t)chunk * LEN + 4 * s;
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    v4[t] = add_mod(mul_shoup(sub_mod(uu[t], v4[t], q), R.pinv[ip], R.pinvs[ip], q), cc[t], q);
+                ((ulonglong2*)op)[0] = make_ulonglong2(v4[0], v4[1]);
+                ((ulonglong2*)op)[1] = make_ulonglong2(v4[2], v4[3]);
+                continue;
+            }
+            if (EPI == 1) {
                 const u32 rot = o >> 1, comp = o & 1, ip = mod, r = R.r;
                 u64* op = epi.out_base + (size_t)rb.out[rot] * epi.out_stride + ((size_t)comp * r + ip) * R.N;
 #pragma unroll
@@ -641,7 +669,17 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
         for (int it = 0; it < 2; ++it) {
             const int s = lane + 32 * it;
             u64 v4[4];
-            if constexpr (TILED) {  // read back from the tile-major plaintext cache
+            if constexpr (EPI == 2) {   // the residues of this output's giant rotations, each read through its rotation, summed
+                const u32 pp_out = o >> 1, comp = o & 1, nb = R.r + 1;
+                const size_t n = (size_t)chunk * LEN + 4 * s;
+                v4[0] = v4[1] = v4[2] = v4[3] = 0;
+                for (u32 jj = 0; jj < epi.n_sum; ++jj) {
+                    const uint4 pv = *(const uint4*)(epi.perm + (size_t)rb.key[jj] * R.N + n);
+                    const u64* up = epi.u + ((((size_t)jj * epi.n_out + pp_out) * 2 + comp) * nb + mod) * R.N;
+                    v4[0] = add_mod(v4[0], __ldg(up + pv.x), q); v4[1] = add_mod(v4[1], __ldg(up + pv.y), q);
+                    v4[2] = add_mod(v4[2], __ldg(up + pv.z), q); v4[3] = add_mod(v4[3], __ldg(up + pv.w), q);
+                }
+            } else if constexpr (TILED) {  // read back from the tile-major plaintext cache
                 const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
                 const u32 n = chunk * LEN + 4 * s;
                 const unsigned char* stage = (const unsigned char*)B.tile_ptr + tile_stage_of_word(B.tile, pj, term, mod, n);
@@ -717,7 +755,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
     }
 }
 
-template <bool FWD, bool EPI, bool TILED>
+template <bool FWD, int EPI, bool TILED>
 __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 8) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
@@ -826,17 +864,20 @@ static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n
     const u32 chunks = 1u << ring.geom.log_r;
     const u32 cpb = (u32)ring.geom.contig_lanes;
     dim3 grid(chunks / cpb, n_polys);
-    if (FWD && epi) {
-        launch_dependent(ring, ntt_contig<FWD, true, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
+    if (epi && epi->n_sum) {
+        launch_dependent(ring, ntt_contig<FWD, 2, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
+                         *epi);
+    } else if (FWD && epi) {
+        launch_dependent(ring, ntt_contig<FWD, 1, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
                          *epi);
     } else {
         static const RotBatch no_rb = {};
         static const ModDownEpilogue no_epi = {};
         if (B.tile_ptr)
-            launch_dependent(ring, ntt_contig<FWD, false, true>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
+            launch_dependent(ring, ntt_contig<FWD, 0, true>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
                              no_rb, no_epi);
         else
-            launch_dependent(ring, ntt_contig<FWD, false, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
+            launch_dependent(ring, ntt_contig<FWD, 0, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
                              no_rb, no_epi);
     }
     return cudaGetLastError();
@@ -877,6 +918,14 @@ cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B0, u32 n_o
     B.scatter_dst = final_dst;
     B.scatter_mont = 1;           // (the only permuted store is that of the rotation keys)
     return launch_contig<true>(ring, B, n_polys, stream);
+}
+
+cudaError_t ntt_inverse_gathersum(const RingHost& ring, const PolyBatch& B, u32 n_outer, const RotBatch& rb,
+                                  const ModDownEpilogue& epi, cudaStream_t stream) {
+    const u32 n_polys = n_outer * B.n_m;
+    cudaError_t e = launch_contig<false>(ring, B, n_polys, stream, &rb, &epi);
+    if (e != cudaSuccess) return e;
+    return launch_strided<false, LOAD_PLAIN>(ring, B, n_polys, stream);
 }
 
 cudaError_t ntt_inverse(const RingHost& ring, const PolyBatch& B, u32 n_outer, cudaStream_t stream) {

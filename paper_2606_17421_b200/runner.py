@@ -28,12 +28,16 @@ class WorkloadRunner:
 
     def __init__(self, name: str, seed: int = 0, device: str = "cuda:0", cache: bool = True,
                  cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None,
-                 fuse_shared_inputs: bool = True, fold_in_ciphertext: bool = False, compact_cache: bool = False):
+                 fuse_shared_inputs: bool = True, fold_in_ciphertext: bool = False, compact_cache: bool = False,
+                 pack: str | None = None, moddown: str | None = None):
         self.w = wl.WORKLOADS[name]
         ps = wl.PARAM_SETS[self.w.params]
         self.N, self.primes, self.P, self.scale = ps["N"], list(ps["primes"]), ps["special"], ps["scale"]
         self.r = len(self.primes)
         self.plan = self.w.plan
+        if pack or moddown:         # the workload's plan with another packing / key-switch variant
+            self.plan = wl.PlanSpec(self.plan.D, self.plan.tau, self.plan.b, self.plan.g,
+                                    pack or self.plan.pack, moddown or self.plan.moddown)
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         # a stream of our own: the legacy default stream cannot be captured, which would keep the
@@ -43,7 +47,9 @@ class WorkloadRunner:
         self.gen = torch.Generator(device=self.device)
         self.gen.manual_seed(seed)
         self.ctx = bf.bf_ctx_create(self.N, self.primes + [self.P], self.r, self.scale,
-                                    bf.bf_plan(self.plan.D, self.plan.tau, self.plan.b, self.plan.g),
+                                    bf.bf_plan(self.plan.D, self.plan.tau, self.plan.b, self.plan.g,
+                                               (bf.BF_PLAN_COMPLEX_PACK if self.plan.pack == "complex" else 0) |
+                                               (bf.BF_PLAN_MODDOWN_PER_OUTPUT if self.plan.moddown == "per_output" else 0)),
                                     self.stream.cuda_stream)
         if compact_cache:           # narrower resident words per prime: 68 % of the cache for the 50 + 6 x 40-bit chain
             bf.bf_set_compact_cache(self.ctx, True)
@@ -79,7 +85,7 @@ class WorkloadRunner:
             members_of = {L.name: [L] for L in units}
         for rep in range(self.w.n_repeat):
             for L in units:
-                n_in, n_out = wl.ceil_div(L.d_in, D), wl.ceil_div(L.d_out, D)
+                n_in, n_out = wl.ceil_div(L.d_in, D), wl.ceil_div(L.d_out, self.plan.rows_per_ct)
                 W = torch.from_numpy(np.concatenate(
                     [wl.gen_weights(seed, f"{m.name}.{rep}", m.d_out, m.d_in) for m in members_of[L.name]], axis=0)
                 ).to(self.device)

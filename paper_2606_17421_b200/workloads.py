@@ -41,6 +41,12 @@ class PlanSpec:
     tau: int
     b: int
     g: int
+    pack: str = "real"                  # "complex": two output row blocks per plaintext (real and imaginary parts)
+    moddown: str = "per_rotation"       # "per_output": one division by the special prime per output ciphertext
+
+    @property
+    def rows_per_ct(self) -> int:
+        return self.D * (2 if self.pack == "complex" else 1)
 
 
 @dataclass(frozen=True)

@@ -28,7 +28,9 @@ class GpuSide:
         # replays captured launch sequences
         self.stream = torch.cuda.Stream(device=self.dev)
         torch.cuda.set_stream(self.stream)
-        p = bf.bf_plan(plan.D, plan.tau, plan.b, plan.g)
+        flags = (bf.BF_PLAN_COMPLEX_PACK if plan.pack == "complex" else 0) | \
+                (bf.BF_PLAN_MODDOWN_PER_OUTPUT if plan.moddown == "per_output" else 0)
+        p = bf.bf_plan(plan.D, plan.tau, plan.b, plan.g, flags)
         self.ctx = bf.bf_ctx_create(par.N, par.basis, par.r, par.scale, p,
                                     torch.cuda.current_stream().cuda_stream)
 
@@ -62,7 +64,7 @@ class GpuSide:
         return uniq
 
     def linear(self, cts, W, d_out, d_in, weights=None):
-        n_in, n_out = len(cts), -(-d_out // self.plan.D)
+        n_in, n_out = len(cts), self.plan.n_out(d_out)
         ct_in = self.to_dev(np.stack(cts))
         ct_out = self.empty_u64(n_out, 2, self.par.r, self.par.N)
         Wd = self.to_dev(np.ascontiguousarray(W, dtype=np.float32))

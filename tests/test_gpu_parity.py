@@ -47,17 +47,18 @@ ENCODE_CASES = [
 
 
 @pytest.mark.parametrize("compact", [False, True])
+@pytest.mark.parametrize("pack", ["real", "complex"])
 @pytest.mark.parametrize("pkey,plan_t,shape", ENCODE_CASES)
-def test_encode_weights_matches_oracle(pkey, plan_t, shape, compact):
+def test_encode_weights_matches_oracle(pkey, plan_t, shape, compact, pack):
     par = oracle_params(pkey)
-    plan = ckks.Plan(*plan_t)
+    plan = ckks.Plan(*plan_t, pack=pack)
     d_out, d_in = shape
     W = wl.gen_weights(1, f"enc{pkey}{plan_t}", d_out, d_in)
     g = GpuSide(par, plan)
     try:
         g.bf.bf_set_compact_cache(g.ctx, compact)
         w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in)
-        n_in, n_out = -(-d_in // plan.D), -(-d_out // plan.D)
+        n_in, n_out = -(-d_in // plan.D), plan.n_out(d_out)
         used = g.bf.bf_cache_bytes_used(g.ctx)
         assert used == g.bf.bf_weights_bytes(g.ctx, d_out, d_in)
         # every encoded word is resident once: 8 bytes, or in the compact cache the narrowest format its
@@ -76,7 +77,7 @@ def test_encode_weights_matches_oracle(pkey, plan_t, shape, compact):
             idx = [idx[i] for i in sorted(keep)]
         out = g.empty_u64(par.r, par.N)
         for (p, q, j, k) in idx:
-            z = ckks.bsgs_plain_slots(W, plan, p, q, j, k, par.n)
+            z = ckks.plain_slots(W, plan, p, q, j, k, par.n)
             expect = ckks.to_residues(ckks.encode_coeffs(z, par.N, par.scale), par.primes)
             g.bf.bf_weights_export(g.ctx, w, p, q, j, k, out)
             assert np.array_equal(g.to_host_u64(out), expect), (p, q, j, k)
@@ -155,7 +156,7 @@ def run_case(par, plan, d_out, d_in, seed, tol, tag, tight=1e-5):
     keys = ckks.make_rotation_keys(par, s, plan, seed)
     cts = ckks.encrypt_vector(par, plan, s, x, seed)
     expect = ckks.linear(par, plan, cts, W, keys)
-    n_out = -(-d_out // plan.D)
+    n_out = plan.n_out(d_out)
     g = GpuSide(par, plan)
     try:
         g.load_keys(keys)
@@ -197,7 +198,7 @@ def run_case(par, plan, d_out, d_in, seed, tol, tag, tight=1e-5):
         for p in range(n_out):
             assert np.array_equal(low[p], ckks.rescale(par, expect[p]))
             part = ckks.fold_output(ckks.decode(ckks.decrypt(par, s, low[p]), par.N, scale), plan, p, d_out)
-            y[p * plan.D:p * plan.D + len(part)] = part
+            y[p * plan.rows_per_ct:p * plan.rows_per_ct + len(part)] = part
         err = np.abs(y - W.astype(np.float64) @ x).max()
         assert err < tol, err
         assert err < tight         # far inside the stated tolerance; catches scale bookkeeping slips
@@ -232,6 +233,60 @@ def test_linear_small_ring_plans(plan_t, shape):
     run_case(par, ckks.Plan(*plan_t), shape[0], shape[1], 2, 1e-2, f"small{plan_t}")
 
 
+@pytest.mark.parametrize("plan_t,shape", [
+    ((64, 4, 4, 4), (100, 130)),      # two row blocks -> one output ciphertext, ragged second block
+    ((64, 4, 4, 4), (150, 64)),       # three row blocks -> two ciphertexts, the last one with an empty imaginary part
+    ((64, 1, 8, 8), (128, 64)),       # classical replicated layout, both parts full
+    ((32, 32, 1, 1), (70, 50)),       # no rotation at all
+    ((64, 4, 4, 4), (1920, 64)),      # 15 output ciphertexts
+])
+def test_linear_complex_packing_small_ring(plan_t, shape):
+    par = oracle_params("n12")
+    run_case(par, ckks.Plan(*plan_t, pack="complex"), shape[0], shape[1], 6, 1e-2, f"cplx{plan_t}")
+
+
+def test_linear_gpt2_qkv_complex_packing_bit_exact():
+    # the 768 -> 2304 projection with two row blocks per plaintext: 2 output ciphertexts instead of 3
+    w = wl.WORKLOADS["gpt2_qkv"]
+    par = oracle_params(w.params)
+    L = w.layers[0]
+    run_case(par, ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, pack="complex"), L.d_out, L.d_in, 0, 1e-3, L.name)
+
+
+@pytest.mark.parametrize("pack", ["real", "complex"])
+@pytest.mark.parametrize("plan_t,shape", [
+    ((64, 4, 4, 4), (100, 130)),      # three giant rotations per output, two or one output ciphertexts
+    ((64, 1, 8, 8), (128, 64)),       # seven giant rotations per output
+    ((64, 1, 2, 32), (64, 64)),       # 31 giant rotations summed before the one division
+    ((64, 32, 2, 1), (64, 64)),       # no giant step: nothing to merge
+    ((64, 4, 4, 4), (1920, 64)),      # 90 (45) giant rotations: several key-switch launches feed one division stage
+])
+def test_linear_one_division_by_P_per_output_small_ring(plan_t, shape, pack):
+    par = oracle_params("n12")
+    run_case(par, ckks.Plan(*plan_t, pack=pack, moddown="per_output"), shape[0], shape[1], 7, 1e-2, f"po{plan_t}")
+
+
+@pytest.mark.parametrize("pack", ["real", "complex"])
+def test_linear_gpt2_qkv_one_division_by_P_per_output_bit_exact(pack):
+    w = wl.WORKLOADS["gpt2_qkv"]
+    par = oracle_params(w.params)
+    L = w.layers[0]
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, pack=pack, moddown="per_output")
+    run_case(par, plan, L.d_out, L.d_in, 0, 1e-3, L.name)
+
+
+def test_per_output_division_refuses_more_giant_steps_than_it_can_sum():
+    from paper_2606_17421_b200 import bifrost as bf
+    ps = wl.PARAM_SETS["n12"]
+    basis = list(ps["primes"]) + [ps["special"]]
+    with pytest.raises(bf.BifrostError) as ei:          # g - 1 = 127 > 64
+        bf.bf_ctx_create(ps["N"], basis, 3, 2.0 ** 40, bf.bf_plan(128, 1, 1, 128, bf.BF_PLAN_MODDOWN_PER_OUTPUT))
+    assert ei.value.code == bf.BF_ERR_SHAPE
+    with pytest.raises(bf.BifrostError) as ei:          # unknown flag bit
+        bf.bf_ctx_create(ps["N"], basis, 3, 2.0 ** 40, bf.bf_plan(64, 1, 8, 8, 64))
+    assert ei.value.code == bf.BF_ERR_INVALID_ARG
+
+
 def test_linear_gpt2_qkv_config_bit_exact():
     w = wl.WORKLOADS["gpt2_qkv"]
     par = oracle_params(w.params)
@@ -261,7 +316,7 @@ def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=()):
                 cts = ckks.encrypt_vector(par, plan, s, x, seed)
                 inputs[d_in] = (x, cts, [ckks.baby_rotations(par, plan, ct, keys) for ct in cts])
             x, cts, X = inputs[d_in]
-            n_in, n_out = len(cts), -(-d_out // plan.D)
+            n_in, n_out = len(cts), plan.n_out(d_out)
             blocks = list(blocks_of(name, n_out))
             expect = ckks.linear(par, plan, cts, W, keys, blocks=blocks, X=X)
             w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in)
@@ -284,7 +339,7 @@ def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=()):
                 assert np.array_equal(got[p], expect[p]), (name, p)
                 assert np.array_equal(low[p], ckks.rescale(par, expect[p])), (name, p)
                 part = ckks.fold_output(ckks.decode(ckks.decrypt(par, s, low[p]), par.N, scale), plan, p, d_out)
-                err = np.abs(part - y_ref[p * plan.D:p * plan.D + len(part)]).max()
+                err = np.abs(part - y_ref[p * plan.rows_per_ct:p * plan.rows_per_ct + len(part)]).max()
                 assert err < 1e-3, (name, p, err)
     finally:
         g.close()
