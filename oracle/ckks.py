@@ -30,6 +30,10 @@ as BSGS objects, and Sec. 6.1 names the encoded-weight cache as the memory wall)
   moddown = "per_output"  the giant-step key switches of an output are summed in the extended basis
                         {q_0..q_L, P} and divided by P once per output ciphertext and component,
                         instead of once per rotation
+  hoist = "double"      the baby-step rotations are not divided by P either: X[q][k] stays in the extended
+                        basis as (P*phi_k(c0) + u0, u1), the plaintexts are reduced modulo P as well, the
+                        products are summed over the extended basis, and each inner sum A[p][j] is divided
+                        by P once (per output block and giant step instead of per input and baby step)
 
 Array conventions (all numpy, C order):
   ciphertext  uint64 [2][r][N]   component, prime, coefficient; coefficient domain, residues in [0, q_i)
@@ -154,6 +158,7 @@ class Plan:
     g: int
     pack: str = "real"                 # "real" | "complex": see the module docstring
     moddown: str = "per_rotation"      # "per_rotation" | "per_output"
+    hoist: str = "single"              # "single" | "double"
 
     @property
     def M(self) -> int:
@@ -172,6 +177,7 @@ class Plan:
         assert self.D * self.tau <= n and n % (self.D * self.tau) == 0
         assert self.D % self.tau == 0 and self.b * self.g == self.M
         assert self.pack in ("real", "complex") and self.moddown in ("per_rotation", "per_output")
+        assert self.hoist in ("single", "double")
 
 
 def galois_element(steps: int, N: int) -> int:
@@ -504,7 +510,8 @@ def plain_slots(W: np.ndarray, plan: Plan, p: int, q: int, j: int, k: int, n: in
 def encode_weights(params: Params, plan: Plan, W: np.ndarray, blocks=None) -> dict:
     """Encoded diagonals of a projection W[d_out][d_in] (Sec. 4.2: pre-encoded weight diagonals kept
     as BSGS objects).  Returns {(p, q, j, k): uint64 [r][N] coefficient-domain plaintext} for the
-    requested output ciphertexts p (all by default)."""
+    requested output ciphertexts p (all by default); with double hoisting the plaintexts are reduced
+    modulo the special prime too: [r+1][N] over the extended basis."""
     plan.check(params.n)
     d_out, d_in = W.shape
     n_in, n_out = -(-d_in // plan.D), plan.n_out(d_out)
@@ -519,9 +526,37 @@ def encode_weights(params: Params, plan: Plan, W: np.ndarray, blocks=None) -> di
             m = encode_complex_batch(z, params.N, params.scale)
         else:
             m = encode_real_batch(z, params.N, params.scale)
-        res = to_residues(m, params.primes)
+        res = to_residues(m, params.basis if plan.hoist == "double" else params.primes)
         for t, pt in zip(part, res):
             out[t] = pt
+    return out
+
+
+def baby_rotations_ext(params: Params, plan: Plan, ct: np.ndarray, keys: dict, ks=None) -> dict:
+    """Double hoisting: X[k] = rot(ct, k*tau) before its division by P, over the extended basis:
+    (P * phi_k(c0) + u0, u1) with (u0, u1) = key_switch_ext(c1); for k = 0 simply (P * c0, P * c1), whose
+    residue modulo P is zero.  Dividing X[k] by P (mod_down) gives exactly the rotated ciphertext.
+    Returns {k: uint64 [2][r+1][N]}, coefficient domain."""
+    N, r, basis = params.N, params.r, params.basis
+    ks = range(plan.b) if ks is None else ks
+    out = {}
+    for k in ks:
+        steps = k * plan.tau
+        X = np.zeros((2, r + 1, N), dtype=np.uint64)
+        if steps % params.n == 0:
+            parts, u = (ct[0], ct[1]), None
+        else:
+            g = galois_element(steps, N)
+            u = key_switch_ext(params, ct[1], g, keys[g])
+            parts = (np.stack([automorphism(ct[0, i], g, qi) for i, qi in enumerate(params.primes)]), None)
+        for comp in range(2):
+            for i, qi in enumerate(params.primes):
+                if parts[comp] is not None:
+                    mul_acc(X[comp, i], parts[comp][i], np.full(N, params.P % qi, dtype=np.uint64), [qi], N)
+            if u is not None:
+                for mi, m in enumerate(basis):
+                    X[comp, mi] = _add(X[comp, mi], u[comp, mi], m)
+        out[k] = X
     return out
 
 
@@ -534,16 +569,21 @@ def baby_rotations(params: Params, plan: Plan, ct: np.ndarray, keys: dict, ks=No
 def inner_sum(params: Params, plan: Plan, Xh: list, encoded: dict, p: int, j: int) -> np.ndarray:
     """A[p][j] = sum_q sum_{k<b} Pt[p][q][j][k] (*) X[q][k], both components, every ciphertext
     prime; Xh[q][k] are the baby-step ciphertexts in the evaluation domain.  Returns the
-    coefficient-domain ciphertext [2][r][N]."""
-    N, r, primes = params.N, params.r, params.primes
-    acc = np.zeros((2, r, N), dtype=np.uint64)
+    coefficient-domain ciphertext [2][r][N].  With double hoisting the sum runs over the extended
+    basis (Xh and the plaintexts carry the residue modulo P) and is divided by P once at the end."""
+    N, r = params.N, params.r
+    moduli = params.basis if plan.hoist == "double" else params.primes
+    acc = np.zeros((2, len(moduli), N), dtype=np.uint64)
     for q in range(len(Xh)):
         pts = np.stack([encoded[(p, q, j, k)] for k in range(plan.b)])
-        pth = ntt(pts, primes * plan.b, params)
+        pth = ntt(pts, moduli * plan.b, params)
         for k in range(plan.b):
             for comp in range(2):
-                mul_acc(acc[comp], pth[k], Xh[q][k][comp], primes, N)
-    return intt(acc, primes * 2, params)
+                mul_acc(acc[comp], pth[k], Xh[q][k][comp], moduli, N)
+    A = intt(acc, moduli * 2, params)
+    if plan.hoist == "double":
+        A = np.stack([mod_down(A[0], params), mod_down(A[1], params)])
+    return A
 
 
 def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blocks=None, encoded=None,
@@ -563,11 +603,14 @@ def linear(params: Params, plan: Plan, cts: list, W: np.ndarray, keys: dict, blo
     blocks = list(range(n_out) if blocks is None else blocks)
     if encoded is None:
         encoded = encode_weights(params, plan, W, blocks)
-    # baby steps: X[q][k] = rot(ct_q, k*tau), then to the evaluation domain for the products
+    # baby steps: X[q][k] = rot(ct_q, k*tau) (double hoisting: before its division by P, over the extended
+    # basis), then to the evaluation domain for the products
     if X is None:
-        X = [baby_rotations(params, plan, cts[q], keys) for q in range(n_in)]
+        rot_fn = baby_rotations_ext if plan.hoist == "double" else baby_rotations
+        X = [rot_fn(params, plan, cts[q], keys) for q in range(n_in)]
     assert len(X) == n_in
-    Xh = [[ntt(X[q][k], primes * 2, params) for k in range(plan.b)] for q in range(n_in)]
+    x_moduli = basis if plan.hoist == "double" else primes
+    Xh = [[ntt(X[q][k], x_moduli * 2, params) for k in range(plan.b)] for q in range(n_in)]
     out = {}
     for p in blocks:
         Y = np.zeros((2, r, N), dtype=np.uint64)

@@ -444,3 +444,43 @@ def test_per_output_moddown_differs_from_per_rotation_only_by_rounding():
     cts2 = ckks.encrypt_vector(par, plan_c, s2, x, 8)
     o_c, o_d = ckks.linear(par, plan_c, cts2, W, keys2), ckks.linear(par, plan_d, cts2, W, keys2)
     assert all(np.array_equal(o_c[p], o_d[p]) for p in o_c)
+
+
+# ------------------------------------------------------------------ double hoisting
+
+def test_extended_baby_rotation_divided_by_P_is_the_rotation(ring64):
+    # (P*phi(c0) + u0, u1) differs from (u0, u1) by an exact multiple of P, so its division by P is
+    # phi(c0) + ModDown(u0), ModDown(u1): exactly what the single-hoisted rotation produces
+    par, s = ring64
+    plan = Plan(8, 4, 4, 1)
+    rng = np.random.default_rng(41)
+    z = rng.normal(size=par.n)
+    ct = ckks.encrypt(par, s, ckks.encode_coeffs(z, par.N, par.scale), 42)
+    keys = ckks.make_rotation_keys(par, s, plan, 43)
+    ext = ckks.baby_rotations_ext(par, plan, ct, keys)
+    plain = ckks.baby_rotations(par, plan, ct, keys)
+    for k in range(plan.b):
+        assert ext[k].shape == (2, par.r + 1, par.N)
+        got = np.stack([ckks.mod_down(ext[k][0], par), ckks.mod_down(ext[k][1], par)])
+        assert np.array_equal(got, plain[k]), k
+    assert not ext[0][:, par.r].any()                    # k = 0: P * ct has residue zero modulo P
+
+
+@pytest.mark.parametrize("pack,moddown", [("real", "per_rotation"), ("complex", "per_output")])
+def test_end_to_end_double_hoisting_small_ring(pack, moddown):
+    N = 256
+    primes, P = ckks.prime_chain(N, 2)
+    par = Params(N, primes, P, 2.0 ** 40)
+    W = wl.gen_weights(0, "dh", 37, 41)
+    x = wl.gen_activation(0, "dh", 41)
+    for plan_t in ((16, 4, 2, 2), (16, 1, 4, 4), (16, 8, 2, 1), (16, 1, 1, 16)):
+        plan = Plan(*plan_t, pack=pack, moddown=moddown, hoist="double")
+        out, s, keys, cts = run_linear_modes(par, plan, W, x, 1, 1e-6)
+        single = ckks.linear(par, Plan(*plan_t, pack=pack, moddown=moddown), cts, W, keys)
+        if plan.b > 1:            # the division by P moved: residues differ (the decrypted values do not, see above)
+            assert any(not np.array_equal(out[p], single[p]) for p in out)
+        else:                     # no baby rotation: only P * ct, whose division by P is exact
+            assert all(np.array_equal(out[p], single[p]) for p in out)
+    # the plaintexts carry the residue modulo P
+    enc = ckks.encode_weights(par, Plan(16, 4, 2, 2, hoist="double"), W, blocks=[0])
+    assert enc[(0, 0, 0, 0)].shape == (par.r + 1, N)
