@@ -108,7 +108,8 @@ MIN_REGION_S = 0.5      # every timed region lasts at least this long (steps are
 # overflow layers take the on-the-fly path), on_the_fly (budget of one byte: nothing is cached), compact
 # (compact cache format), fold (in-ciphertext fold of the tau partial sums), complex (two output row blocks per
 # plaintext, in the real and imaginary parts of the slots), per_output (one division by the special prime per
-# output ciphertext instead of one per giant rotation).
+# output ciphertext instead of one per giant rotation), double_hoist (baby-step rotations kept in the extended basis,
+# one division per inner sum).
 # The headline is the largest single-GPU configuration under the fastest plan variant that is parity-tested; the same
 # step under the plain plan, and the other configurations under both, follow as extras.
 BEST = "complex,per_output"
@@ -135,6 +136,8 @@ def parse_spec(spec: str):
             kw["pack"] = "complex"
         elif o == "per_output":
             kw["moddown"] = "per_output"
+        elif o == "double_hoist":
+            kw["hoist"] = "double"
         else:
             raise ValueError(f"unknown workload option {o!r}")
     return name, kw
@@ -172,9 +175,8 @@ def transform_counts(runner) -> dict:
         sets = (n_in if b > 1 else 0) + n_giant            # ModUp digit sets
         rots = n_in * (b - 1) + n_giant                    # key switches
         # divisions by P: one per rotation and component, or (per_output) one per baby rotation and per output
-        n_lift = 2 * rots
-        if runner.plan.moddown == "per_output" and n_giant:
-            n_lift = 2 * (n_in * (b - 1) + n_out)
+        n_baby_lift = 2 * n_out * g if runner.plan.hoist == "double" else 2 * n_in * (b - 1)
+        n_lift = n_baby_lift + 2 * (n_out if runner.plan.moddown == "per_output" and n_giant else n_giant)
         for i in range(r):
             fwd[i] += 2 * n_in + sets * (r - 1) + n_lift   # inputs; digits of the other primes; lifted P-residues
             inv[i] += n_giant + 2 * n_out                  # c1 of the giant-step inputs; outputs
@@ -182,7 +184,7 @@ def transform_counts(runner) -> dict:
         inv[r] += n_lift                                   # P-residues of the inner products
         if not e["handle"]:                                # on-the-fly path: every diagonal is transformed on each call
             n_diag = n_in * n_out * b * g
-            for i in range(r):
+            for i in range(r + (1 if runner.plan.hoist == "double" else 0)):
                 fwd[i] += n_diag
     def summary(cnt):
         return {"polys": sum(cnt), "fp64_polys": sum(c for c, f in zip(cnt, fp) if f),
@@ -335,7 +337,7 @@ class Measurement:
         return {"layers": len(R.layers), "unit_of_work": "decode token (all linear layers)" if whole_step else "one projection call",
                 "ring_N": R.N, "ct_primes": R.r,
                 "plan": {"D": R.plan.D, "tau": R.plan.tau, "b": R.plan.b, "g": R.plan.g, "pack": R.plan.pack,
-                         "moddown": R.plan.moddown},
+                         "moddown": R.plan.moddown, "hoist": R.plan.hoist},
                 "ciphertexts_in": sum(e["n_in"] for e in R.layers), "ciphertexts_out": sum(e["n_out"] for e in R.layers),
                 "boundary_bytes": h2d + d2h, "rotation_keys": len(R.rot_steps), "fallback_layers": R.n_fallback_layers(),
                 "encoded_weight_bytes_cached": R.cached_pt_bytes(), "encoded_weight_bytes_total": R.total_pt_bytes()}
@@ -482,7 +484,7 @@ class OracleSample:
         self.w = w
         self.par = ckks.Params(ps["N"], list(ps["primes"]), ps["special"], ps["scale"])
         self.plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, pack=kw.get("pack", w.plan.pack),
-                              moddown=kw.get("moddown", w.plan.moddown))
+                              moddown=kw.get("moddown", w.plan.moddown), hoist=kw.get("hoist", w.plan.hoist))
         self.L = w.layers[0]
         self.W = wl.gen_weights(0, self.L.name, self.L.d_out, self.L.d_in)
         x = wl.gen_activation(0, self.L.name, self.L.d_in)
@@ -514,16 +516,23 @@ class OracleSample:
                 for k in range(plan.b):
                     if (p, q, j, k) not in self.encoded:
                         z = ck.plain_slots(self.W, plan, p, q, j, k, par.n)
-                        self.encoded[(p, q, j, k)] = ck.to_residues(ck.encode_coeffs(z, par.N, par.scale), par.primes)
-        # evaluation-domain inputs for the sampled inner sums (unrotated stand-ins keep this bounded)
-        self.Xh = [[ck.ntt(self.cts[q], par.primes * 2, par) for _ in range(plan.b)] for q in range(self.n_in)]
+                        self.encoded[(p, q, j, k)] = ck.to_residues(ck.encode_coeffs(z, par.N, par.scale),
+                                                                    par.basis if plan.hoist == "double" else par.primes)
+        # evaluation-domain inputs for the sampled inner sums (unrotated stand-ins keep this bounded); with double
+        # hoisting they carry a residue modulo the special prime as well
+        if plan.hoist == "double":
+            ext = [self.np.concatenate([ct, ct[:, :1] % self.np.uint64(par.P)], axis=1) for ct in self.cts]
+            self.Xh = [[ck.ntt(ext[q], par.basis * 2, par) for _ in range(plan.b)] for q in range(self.n_in)]
+        else:
+            self.Xh = [[ck.ntt(self.cts[q], par.primes * 2, par) for _ in range(plan.b)] for q in range(self.n_in)]
 
     def step(self) -> dict:
         """One sampled step; returns seconds per part and the unit counts they cover."""
         ck, plan, par = self.ckks, self.plan, self.par
         t = {"baby": 0.0, "inner": 0.0, "giant": 0.0, "rescale": 0.0}
         t0 = time.perf_counter()
-        ck.baby_rotations(par, plan, self.cts[0], self.keys, ks=self.baby_ks)
+        (ck.baby_rotations_ext if plan.hoist == "double" else ck.baby_rotations)(par, plan, self.cts[0], self.keys,
+                                                                                  ks=self.baby_ks)
         t["baby"] = time.perf_counter() - t0
         n_giant = 0
         A = u = None
@@ -581,7 +590,7 @@ class OracleSample:
         self.prepare(n_baby, n_groups)
 
     def describe(self) -> str:
-        return (f"plan pack={self.plan.pack} moddown={self.plan.moddown}; layer {self.L.name}: {len(self.baby_ks)} of {self.plan.b - 1} baby rotations of one input and "
+        return (f"plan pack={self.plan.pack} moddown={self.plan.moddown} hoist={self.plan.hoist}; layer {self.L.name}: {len(self.baby_ks)} of {self.plan.b - 1} baby rotations of one input and "
                 f"{len(self.groups)} of {self.n_out * self.plan.g} (block, giant-step) groups (inner sum, giant "
                 f"rotation) plus one rescale per step, scaled by unit counts to every layer of the workload")
 

@@ -60,10 +60,16 @@ typedef struct bf_weights bf_weights;  /* device-resident encoded diagonals of o
  *   BF_PLAN_MODDOWN_PER_OUTPUT the key-switch results of an output's giant rotations are summed in
  *       the extended basis {q_i, P} and divided by P once per output ciphertext and component
  *       instead of once per rotation (Sec. 4.2 leaves the key-switching primitive open).  Needs
- *       bsgs_g - 1 <= 64. */
+ *       bsgs_g - 1 <= 64.
+ *   BF_PLAN_DOUBLE_HOIST       the baby-step rotations are not divided by P: they stay in the extended
+ *       basis as (P*phi_k(c0) + u0, u1), the encoded weights are held modulo P as well (one more
+ *       60-bit residue per coefficient: (r+1)/r of the cache), the products are summed over the
+ *       extended basis, and each inner sum is divided by P once, i.e. n_out * bsgs_g divisions per
+ *       call instead of n_in * (bsgs_b - 1). */
 enum {
     BF_PLAN_COMPLEX_PACK = 1,
-    BF_PLAN_MODDOWN_PER_OUTPUT = 2
+    BF_PLAN_MODDOWN_PER_OUTPUT = 2,
+    BF_PLAN_DOUBLE_HOIST = 4
 };
 typedef struct {
     uint32_t tile_D, tau, bsgs_b, bsgs_g;

@@ -27,6 +27,7 @@ BF_ERR_TIMEOUT = -10
 
 BF_PLAN_COMPLEX_PACK = 1
 BF_PLAN_MODDOWN_PER_OUTPUT = 2
+BF_PLAN_DOUBLE_HOIST = 4
 
 
 class bf_plan(ctypes.Structure):

@@ -108,7 +108,7 @@ struct bf_ctx {
     u32* perms_fwd = nullptr;        // [n_keys][N] perm: rotated[n] = unrotated[perm[n]] (per-output division by P)
     u32 n_keys = 0;
     // scratch (grow-only)
-    DevBuf X, Dig, U, Ubig, Tc, Tn, Cc, A, Rres, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
+    DevBuf X, X0, Aext, Dig, U, Ubig, Tc, Tn, Cc, A, Rres, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
     u64 cache_budget = 0, cache_used = 0;
     std::vector<bf_weights*> weights;
     std::string cuda_msg;
@@ -223,7 +223,7 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
         (u64)plan->bsgs_b * plan->bsgs_g != plan->tile_D / plan->tau)
         return BF_ERR_SHAPE;
     if (plan->bsgs_b - 1 > (u32)MAX_ROT_BATCH) return BF_ERR_SHAPE;
-    if (plan->flags & ~(u32)(BF_PLAN_COMPLEX_PACK | BF_PLAN_MODDOWN_PER_OUTPUT)) return BF_ERR_INVALID_ARG;
+    if (plan->flags & ~(u32)(BF_PLAN_COMPLEX_PACK | BF_PLAN_MODDOWN_PER_OUTPUT | BF_PLAN_DOUBLE_HOIST)) return BF_ERR_INVALID_ARG;
     if ((plan->flags & BF_PLAN_MODDOWN_PER_OUTPUT) && plan->bsgs_g - 1 > (u32)MAX_ROT_BATCH) return BF_ERR_SHAPE;
 
     bf_ctx* ctx = new (std::nothrow) bf_ctx();
@@ -402,7 +402,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
             delete w;
         }
     }
-    DevBuf* bufs[] = {&ctx->X, &ctx->Dig, &ctx->U, &ctx->Ubig, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres,
+    DevBuf* bufs[] = {&ctx->X, &ctx->X0, &ctx->Aext, &ctx->Dig, &ctx->U, &ctx->Ubig, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres,
                       &ctx->fft, &ctx->coef, &ctx->ptnat, &ctx->ptjit, &ctx->stage_in, &ctx->stage_out, &ctx->nm_a, &ctx->nm_b};
     for (DevBuf* b : bufs) free_buf(*b);
     cudaFree(ctx->tw_fwd);
@@ -527,6 +527,9 @@ extern "C" uint64_t bf_cache_bytes_used(const bf_ctx* ctx) { return ctx ? ctx->c
 
 static u32 cdiv(u32 a, u32 b) { return (u32)(((u64)a + b - 1) / b); }
 
+// primes the encoded plaintexts are held in: with double hoisting the special prime as well
+static u32 mac_primes(const bf_ctx* ctx) { return ctx->r + ((ctx->plan.flags & BF_PLAN_DOUBLE_HOIST) ? 1u : 0u); }
+
 // output ciphertexts of a projection with d_out rows: one per row block of tile_D, or per pair of row blocks
 static u32 n_out_cts(const bf_ctx* ctx, u32 d_out) {
     const u32 blocks = cdiv(d_out, ctx->plan.tile_D);
@@ -536,7 +539,7 @@ static u32 n_out_cts(const bf_ctx* ctx, u32 d_out) {
 extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
     if (!ctx) return 0;
     const u32 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = n_out_cts(ctx, d_out);
-    const TileLayout lay = mac_tile_layout(ctx->ring, n_out * ctx->plan.bsgs_g, n_in * ctx->plan.bsgs_b);
+    const TileLayout lay = mac_tile_layout(ctx->ring, n_out * ctx->plan.bsgs_g, n_in * ctx->plan.bsgs_b, mac_primes(ctx));
     return mac_tile_bytes(ctx->ring, lay);
 }
 
@@ -544,7 +547,7 @@ extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t
 // into dst in the tile-major layout `lay`, whose group 0 is group pj0 of W.
 static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0, u32 count, u64* dst,
                         const TileLayout& lay, u32 pj0) {
-    const u32 N = ctx->N, r = ctx->r, n = N / 2;
+    const u32 N = ctx->N, r = lay.n_primes, n = N / 2;       // (r: primes each diagonal is reduced into)
     // diagonals per pass: the encoder and the transforms gain from large batches (measured: 32 -> 128 per
     // pass takes 6 to 8 % off a call that encodes on the fly); the scratch of a pass is held to about 0.5 GB
     u32 chunk = (u32)(((size_t)512 << 20) / ((size_t)r * N * sizeof(u64))) & ~7u;
@@ -625,7 +628,7 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
     w->n_in = cdiv(d_in, ctx->plan.tile_D);
     w->n_out = n_out_cts(ctx, d_out);
     w->bytes = bytes;
-    w->lay = mac_tile_layout(ctx->ring, w->n_out * ctx->plan.bsgs_g, w->n_in * ctx->plan.bsgs_b);
+    w->lay = mac_tile_layout(ctx->ring, w->n_out * ctx->plan.bsgs_g, w->n_in * ctx->plan.bsgs_b, mac_primes(ctx));
     cudaError_t e = cudaMalloc(&w->pt, bytes);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -845,7 +848,15 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     const u32 rot_per_lane = baby_per_lane > giant_per_lane ? baby_per_lane : giant_per_lane;
     u32 n_dig_sets = giant_per_lane * (u32)lanes;       // digit sets alive at once
     if (n_dig_sets < in_batch) n_dig_sets = in_batch;
-    TRY(ensure(ctx, ctx->X, (size_t)n_in * b * ctw * 8));
+    // double hoisting: the rotated inputs and the inner sums live in the extended basis {q_i, P}
+    const bool dh = (ctx->plan.flags & BF_PLAN_DOUBLE_HOIST) != 0;
+    const u32 nmp = mac_primes(ctx);                      // primes of X, of the plaintexts and of the inner sums
+    const size_t xw = (size_t)2 * nmp * N;                // words per term of X / per inner sum
+    TRY(ensure(ctx, ctx->X, (size_t)n_in * b * xw * 8));
+    if (dh) {
+        TRY(ensure(ctx, ctx->X0, (size_t)n_in * ctw * 8));
+        TRY(ensure(ctx, ctx->Aext, (size_t)n_out * g * xw * 8));
+    }
     TRY(ensure(ctx, ctx->A, (size_t)n_out * g * ctw * 8));
     // one division by P per output: the inner products of all giant rotations stay alive until every chain is done
     const bool per_output = (ctx->plan.flags & BF_PLAN_MODDOWN_PER_OUTPUT) && n_giant > 0;
@@ -854,6 +865,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     {
         u32 rot_scratch = rot_per_lane * (u32)lanes;
         if (per_output && rot_scratch < n_out) rot_scratch = n_out;     // Tc, Tn of the per-output division
+        if (dh && rot_scratch < n_out * g) rot_scratch = n_out * g;     // Tc, Tn of the division of the inner sums
         TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_scratch));
     }
     if (per_output) TRY(ensure(ctx, ctx->Ubig, (size_t)n_giant * 2 * nb * N * 8));
@@ -880,21 +892,26 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     // ---- ingest, hoisted ModUp and baby steps, batched over the input ciphertexts
     PolyBatch B;
     memset(&B, 0, sizeof(B));
-    B.src = ct_in;                                       // X[q][0] = NTT(ct_q): polynomial (q, component*r + prime)
-    B.dst = X;
+    // X[q][0] = NTT(ct_q): polynomial (q, component*r + prime).  Double hoisting keeps it apart (X0: the hoisted ModUp
+    // copies its c1 part) and puts P * NTT(ct_q), zero modulo P, into X
+    u64* X0 = dh ? (u64*)ctx->X0.p : X;
+    const long long x0_stride = dh ? (long long)ctw : (long long)b * ctw;
+    B.src = ct_in;
+    B.dst = X0;
     B.src_so = (long long)ctw;
-    B.dst_so = (long long)b * ctw;
+    B.dst_so = x0_stride;
     B.src_sm = B.dst_sm = N;
     B.n_m = 2 * r;
     B.mod_wrap = r;
     B.mod0 = 0;
     B.mod_step = 1;
     CK(ntt_forward(ctx->ring, B, n_in, LOAD_PLAIN, ctx->stream));
+    if (dh) CK(launch_lift_times_p(ctx->ring, X0, (long long)ctw, X, (long long)b * xw, n_in, ctx->stream));
     if (b > 1) {
         for (u32 q0 = 0; q0 < n_in; q0 += in_batch) {
             const u32 qn = (n_in - q0 < in_batch) ? n_in - q0 : in_batch;
             TRY(modup(ctx, ctx->stream, ct_in + (size_t)q0 * ctw + (size_t)r * N, (long long)ctw, qn, Dig,
-                      X + (size_t)q0 * b * ctw + (size_t)r * N, (long long)b * ctw));
+                      X0 + (size_t)q0 * x0_stride + (size_t)r * N, x0_stride));
             // the rotations of the batch, dealt out to the lanes in contiguous runs
             const u32 n_rot = qn * (b - 1);
             const u32 per = cdiv(n_rot, (u32)lanes_baby);
@@ -912,6 +929,11 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
                     rb.c0[i] = (int)((q0 + q) * b);
                     rb.out[i] = (int)((q0 + q) * b + k);
                 }
+                if (dh) {       // no division by P: the inner product's last step assembles the rotated input in X
+                    CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, nullptr, ctx->device_error, lane[c].s, X,
+                                                ctx->perms));
+                    continue;
+                }
                 CK(launch_key_inner_product(ctx->ring, rb, Dig, ctx->keys, lane[c].U, ctx->device_error, lane[c].s));
                 TRY(moddown_batch(ctx, lane[c], rb, X, (long long)ctw, X, (long long)ctw));
             }
@@ -920,24 +942,60 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     }
     stamp(ctx, 1);
 
-    // ---- multiply-accumulate over the encoded diagonals
+    // ---- multiply-accumulate over the encoded diagonals (double hoisting: over the extended basis, into Aext)
     const u32 n_terms = n_in * b, n_pj = n_out * g;
+    u64* mac_out = dh ? (u64*)ctx->Aext.p : A;
     if (pt_weights) {
-        CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, A, n_pj, n_terms, true, ctx->device_error, ctx->stream));
+        CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, mac_out, n_pj, n_terms, true, ctx->device_error, ctx->stream));
     } else {
         // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them
-        const size_t group_bytes = (size_t)n_terms * r * N * 8;
+        const size_t group_bytes = (size_t)n_terms * nmp * N * 8;
         const size_t fit = ctx->encode_scratch_bytes / group_bytes;
         const u32 groups = fit < 1 ? 1u : fit > (size_t)n_pj ? n_pj : (u32)fit;
-        const TileLayout jl = mac_tile_layout(ctx->ring, groups, n_terms);
+        const TileLayout jl = mac_tile_layout(ctx->ring, groups, n_terms, nmp);
         TRY(ensure(ctx, ctx->ptjit, mac_tile_bytes(ctx->ring, jl)));
         for (u32 pj0 = 0; pj0 < n_pj; pj0 += groups) {
             const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
-            const TileLayout cl = mac_tile_layout(ctx->ring, cnt, n_terms);
+            const TileLayout cl = mac_tile_layout(ctx->ring, cnt, n_terms, nmp);
             TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p, cl, pj0));
-            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, cl, X, A + (size_t)pj0 * ctw, cnt, n_terms, false,
+            CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, cl, X, mac_out + (size_t)pj0 * xw, cnt, n_terms, false,
                           ctx->device_error, ctx->stream));
         }
+    }
+    if (dh) {
+        // one division by P per inner sum and component: A[pj][comp][i] = (Aext[pj][comp][i] - t) * P^{-1}, t the
+        // centred lift of the residue modulo P
+        const u64* Aext = (const u64*)ctx->Aext.p;
+        memset(&B, 0, sizeof(B));
+        B.src = Aext + (size_t)r * N;
+        B.dst = (u64*)ctx->Tc.p;
+        B.src_so = (long long)nb * N;
+        B.dst_so = N;
+        B.n_m = 1;
+        B.mod0 = r;
+        B.mod_step = 0;
+        B.store_centred = 1;
+        CK(ntt_inverse(ctx->ring, B, n_pj * 2, ctx->stream));
+        memset(&B, 0, sizeof(B));
+        B.src = (const u64*)ctx->Tc.p;
+        B.dst = (u64*)ctx->Tn.p;
+        B.src_so = N;
+        B.src_sm = 0;
+        B.dst_so = (long long)r * N;
+        B.dst_sm = N;
+        B.n_m = r;
+        B.mod0 = 0;
+        B.mod_step = 1;
+        B.lift_mod = ctx->ring.q[r];
+        RotBatch no_rb;
+        memset(&no_rb, 0, sizeof(no_rb));
+        ModDownEpilogue epi;
+        memset(&epi, 0, sizeof(epi));
+        epi.u = Aext;
+        epi.out_base = A;
+        epi.out_stride = (long long)r * N;
+        epi.plain = 1;
+        CK(ntt_forward_moddown(ctx->ring, B, n_pj * 2, no_rb, epi, ctx->stream));
     }
     stamp(ctx, 2);
 

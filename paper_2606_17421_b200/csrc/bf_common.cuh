@@ -253,6 +253,9 @@ struct ModDownEpilogue {
     long long out_stride;
     const u32* perm;              // [n_keys][N] (per-output form)
     u32 n_sum, n_out;             // per-output form: giant steps summed per output, number of outputs
+    u32 plain;                    // division by P of inner sums kept in the extended basis (double hoisting):
+                                  //   polynomial (o, i): out_base[o*out_stride + i*N + n] = (u[o][i][n] - t[n]) * P^{-1},
+                                  //   no rotation, nothing added
 };
 
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks
@@ -268,7 +271,9 @@ struct ModDownEpilogue {
 enum TileFormat : u32 { TILE_W64 = 0, TILE_W40 = 1, TILE_W32 = 2 };
 struct TileLayout {
     u32 log_tn, n_terms, n_pj, G, C, ntiles;
-    u32 fmt_bits;                           // TileFormat of ciphertext prime i in bits 2i, 2i+1
+    u32 fmt_bits;                           // TileFormat of prime i in bits 2i, 2i+1
+    u32 n_primes;                           // primes the plaintexts are held in: r, or r + 1 with double hoisting
+                                            //   (the special prime last, always in 8-byte whole words)
 };
 constexpr u32 TILE_TS = 8;
 constexpr u32 TILE_STAGE_WORDS = 2048;

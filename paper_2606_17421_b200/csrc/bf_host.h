@@ -90,11 +90,21 @@ cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B, u32 n_ou
 cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* b, u64* out, u32 n_polys, u32 n_m,
                                  u32 mod0, cudaStream_t stream);
 // u'[rot][comp][m][n] = sum_j dig[dig(rot)][j][m][n] * key'[key(rot)][j][comp][m][n]  (keys pre-permuted)
+// xext non-null (double hoisting): rotation `rot` is not stored to u but finished as a rotated input in the
+// extended basis: xext[rb.out[rot]][comp][m][pinv[rb.key[rot]][n]] = u'[comp][m][n] + (comp == 0 ?
+// xext[rb.c0[rot]][0][m][n] : 0), terms of [2][r+1][N] words (term rb.c0[rot] holds P times the un-rotated input).
 cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
-                                     int* error_flag, cudaStream_t stream);
+                                     int* error_flag, cudaStream_t stream, u64* xext = nullptr, const u32* pinv = nullptr);
+// dst[t][comp][i][n] = src[t][comp][i][n] * P mod q_i (i < r), dst[t][comp][r][n] = 0: the un-rotated inputs lifted to
+// the extended basis; src ciphertexts of [2][r][N] at src_stride, dst terms of [2][r+1][N] at dst_stride (words)
+cudaError_t launch_lift_times_p(const RingHost& ring, const u64* src, long long src_stride, u64* dst, long long dst_stride,
+                                u32 n_ct, cudaStream_t stream);
 u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintext format (0 = whole words)
-TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms);   // layout of n_pj groups of n_terms diagonals
+// layout of n_pj groups of n_terms diagonals held in n_primes primes (0 = the r ciphertext primes)
+TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms, u32 n_primes = 0);
 size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t);           // bytes that layout occupies
+// x: [n_terms][2][lay.n_primes][N], a: [n_pj][2][lay.n_primes][N]; every prime of the layout is processed (the special
+// prime, when present, by a launch of its own on whole words)
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
                        u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream);
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,

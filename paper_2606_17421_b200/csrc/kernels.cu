@@ -117,7 +117,7 @@ template <bool KARA, int LOG_TN, bool COMPACT>
 __global__ void __launch_bounds__(MAC_THREADS, 3)
 mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, const u64* __restrict__ x,
            u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, u32 early_weights,
-           u32 n_whole, u32 tail_split, int* __restrict__ error_flag) {
+           u32 n_whole, u32 tail_split, u32 prime0, u32 n_launch_primes, int* __restrict__ error_flag) {
     extern __shared__ __align__(128) unsigned char mac_smem[];
     asm volatile("griddepcontrol.launch_dependents;");
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
@@ -128,7 +128,8 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
     // Work units (tile, prime, slice of the output groups) are numbered tile-fastest.  The first n_whole
     // blocks take one unit each; the units after them (the part that would be a thin last wave) are each
     // cut into tail_split blocks over their output groups, so that the last wave is short instead.
-    const u32 N = R.N, r = R.r;
+    const u32 N = R.N;
+    const u32 r = lay.n_primes;                                    // primes per (term, component) of x and a
     const u32 tid = threadIdx.x;
     u32 unit = blockIdx.x, sub = 0, n_sub = 1;
     if (unit >= n_whole) {
@@ -137,9 +138,9 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         n_sub = tail_split;
     }
     const u32 tile_x = unit % (N >> LOG_TN);
-    const u32 i = (unit / (N >> LOG_TN)) % r;
+    const u32 i = prime0 + (unit / (N >> LOG_TN)) % n_launch_primes;   // this launch covers primes prime0 .. + n_launch_primes - 1
     const u32 n0 = tile_x << LOG_TN;
-    u32 pj_begin = (unit / (N >> LOG_TN) / r) * pj_per_block;
+    u32 pj_begin = (unit / (N >> LOG_TN) / n_launch_primes) * pj_per_block;
     u32 pj_end = min(n_pj, pj_begin + pj_per_block);
     if (n_sub > 1) {
         const u32 groups = (pj_end - pj_begin + PL - 1) / PL;
@@ -382,7 +383,7 @@ static u32 mac_log_tn(u32 n_terms) {
     return log_tn;
 }
 
-TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms) {
+TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms, u32 n_primes) {
     TileLayout t;
     memset(&t, 0, sizeof(t));
     t.log_tn = mac_log_tn(n_terms);
@@ -392,15 +393,16 @@ TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms) {
     t.G = (n_pj + PL - 1) / PL;
     t.C = (n_terms + TILE_TS - 1) / TILE_TS;
     t.ntiles = ring.dev.N >> t.log_tn;
-    for (u32 i = 0; i < ring.dev.r; ++i) {
-        const u32 f = !ring.compact_cache ? TILE_W64
+    t.n_primes = n_primes ? n_primes : ring.dev.r;
+    for (u32 i = 0; i < t.n_primes; ++i) {
+        const u32 f = !ring.compact_cache || i >= ring.dev.r ? TILE_W64
                     : ring.q[i] < (1ull << 32) ? TILE_W32 : ring.q[i] < (1ull << 40) ? TILE_W40 : TILE_W64;
         t.fmt_bits |= f << (2 * i);
     }
     return t;
 }
 
-size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t) { return tile_prime_base(t, ring.dev.r); }
+size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t) { (void)ring; return tile_prime_base(t, t.n_primes); }
 
 u32 mac_split_bits(const RingHost& ring) {
     u64 qmax = 0;
@@ -410,8 +412,8 @@ u32 mac_split_bits(const RingHost& ring) {
 
 template <bool KARA, int LOG_TN, bool COMPACT>
 static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a,
-                                u32 n_pj, u32 n_terms, u32 lazy, u32 early_weights, int* error_flag,
-                                cudaStream_t stream) {
+                                u32 n_pj, u32 n_terms, u32 lazy, u32 early_weights, u32 prime0, u32 n_launch_primes,
+                                int* error_flag, cudaStream_t stream) {
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     const size_t smem = (size_t)MAC_RING_BYTES + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_MAX_STAGES + 1) * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
@@ -424,7 +426,7 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
         attr_set[ds] = true;
     }
     // slices over output groups: enough blocks to fill the machine several times over
-    const u32 tiles = (ring.dev.N >> LOG_TN) * ring.dev.r;
+    const u32 tiles = (ring.dev.N >> LOG_TN) * n_launch_primes;
     u32 slices = (148u * 2 * 6 + tiles - 1) / tiles;
     const u32 max_slices = (n_pj + PL - 1) / PL;
     if (slices > max_slices) slices = max_slices;
@@ -460,18 +462,19 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     const u32 n_whole = tail_split > 1 ? units - rem : units;
     dim3 grid(n_whole + (units - n_whole) * tail_split);
     return launch_dependent(ring, mac_kernel<KARA, LOG_TN, COMPACT>, grid, dim3(MAC_THREADS), smem, stream, ring.dev, pt, lay, x, a,
-                            n_terms, n_pj, pj_per_block, lazy, early_weights, n_whole, tail_split, error_flag);
+                            n_terms, n_pj, pj_per_block, lazy, early_weights, n_whole, tail_split, prime0, n_launch_primes,
+                            error_flag);
 }
 
-cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
-                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream) {
-    if (n_pj == 0) return cudaSuccess;
-    if (lay.n_pj != n_pj || lay.n_terms != n_terms) return cudaErrorInvalidValue;
+// One launch over primes prime0 .. prime0 + n_launch_primes - 1 of the layout; kara: Karatsuba on 25-bit limbs
+// (those primes are all below 2^50), else whole words.
+static cudaError_t launch_mac_primes(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a,
+                                     u32 n_pj, u32 n_terms, bool weights_static, u32 prime0, u32 n_launch_primes, bool kara,
+                                     int* error_flag, cudaStream_t stream) {
     ProfScope prof(ring.prof, CAT_MAC, stream);
     u64 qmax = 0;
-    for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
+    for (u32 i = prime0; i < prime0 + n_launch_primes; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
     const u32 log_tn = lay.log_tn;
-    const bool kara = mac_split_bits(ring) != 0;
     // terms a lazy sum can take: Karatsuba's middle sum grows by < 2^52 per term; the whole-word
     // path is limited by its high partial sum and by the total staying below q * 2^64
     u32 lazy = 128u;
@@ -484,10 +487,10 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
     }
     const u32 early = weights_static ? 1u : 0u;
     bool compact = false;
-    for (u32 i = 0; i < ring.dev.r; ++i) compact = compact || tile_format(lay, i) != TILE_W64;
+    for (u32 i = prime0; i < prime0 + n_launch_primes; ++i) compact = compact || tile_format(lay, i) != TILE_W64;
 #define BF_MAC(S, L)                                                                                             \
-    (compact ? launch_mac_t<S, L, true>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, error_flag, stream)     \
-             : launch_mac_t<S, L, false>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, error_flag, stream))
+    (compact ? launch_mac_t<S, L, true>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, prime0, n_launch_primes, error_flag, stream)     \
+             : launch_mac_t<S, L, false>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, prime0, n_launch_primes, error_flag, stream))
     if (kara) {
         switch (log_tn) {
             case 8: return BF_MAC(true, 8);
@@ -505,6 +508,18 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
         default: return BF_MAC(false, 4);
     }
 #undef BF_MAC
+}
+
+cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
+                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream) {
+    if (n_pj == 0) return cudaSuccess;
+    if (lay.n_pj != n_pj || lay.n_terms != n_terms) return cudaErrorInvalidValue;
+    const u32 r = ring.dev.r;
+    const bool kara = mac_split_bits(ring) != 0;
+    cudaError_t e = launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, 0, r, kara, error_flag, stream);
+    if (e != cudaSuccess || lay.n_primes <= r) return e;
+    // double hoisting: the residues modulo the 60-bit special prime, on whole words
+    return launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, r, lay.n_primes - r, false, error_flag, stream);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -530,7 +545,8 @@ constexpr int KI_TILE = 128;
 __global__ void __launch_bounds__(KI_TILE, 10) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
                                                                     const u64* __restrict__ dig,
                                                                     const u64* __restrict__ keys, u64* __restrict__ u,
-                                                                    u32 small_ok, int* __restrict__ error_flag) {
+                                                                    u32 small_ok, int* __restrict__ error_flag,
+                                                                    u64* __restrict__ xext, const u32* __restrict__ pinv) {
     extern __shared__ __align__(128) unsigned char ki_smem[];
     const u32 rot = blockIdx.x, m = blockIdx.z;
     const u32 N = R.N, r = R.r, nb = r + 1;
@@ -563,7 +579,7 @@ __global__ void __launch_bounds__(KI_TILE, 10) key_inner_bulk_kernel(const RingD
     mbar_wait(bar, 0, error_flag);
     const u64 q = R.q[m];
     const u32 qneg32 = (u32)R.qneg[m];
-    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
+    u64 v0, v1;
     if (m < r && small_ok) {
         LimbAcc<true> a0, a1;
         for (u32 j = 0; j < r; ++j) {
@@ -571,8 +587,8 @@ __global__ void __launch_bounds__(KI_TILE, 10) key_inner_bulk_kernel(const RingD
             a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
             a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
         }
-        up[0] = a0.reduce_mont32(q, qneg32);             // the keys carry a factor 2^64
-        up[(size_t)nb * N] = a1.reduce_mont32(q, qneg32);
+        v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
+        v1 = a1.reduce_mont32(q, qneg32);
     } else {
         LimbAcc<false> a0, a1;
         for (u32 j = 0; j < r; ++j) {
@@ -580,13 +596,52 @@ __global__ void __launch_bounds__(KI_TILE, 10) key_inner_bulk_kernel(const RingD
             a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
             a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
         }
-        up[0] = a0.reduce_mont32(q, qneg32);             // the keys carry a factor 2^64
-        up[(size_t)nb * N] = a1.reduce_mont32(q, qneg32);
+        v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
+        v1 = a1.reduce_mont32(q, qneg32);
     }
+    if (xext) {
+        // double hoisting: no division by P; the rotated input in the extended basis is (P*c0 + u0, u1) moved
+        // through the rotation's permutation; P*c0 (zero modulo P) was stored as the un-rotated term
+        const size_t term_words = (size_t)2 * nb * N;
+        const u32 n = n0 + tid;
+        v0 = add_mod(v0, xext[(size_t)rb.c0[rot] * term_words + (size_t)m * N + n], q);
+        u64* xp = xext + (size_t)rb.out[rot] * term_words + (size_t)m * N + __ldg(&pinv[(size_t)rb.key[rot] * N + n]);
+        xp[0] = v0;
+        xp[(size_t)nb * N] = v1;
+        return;
+    }
+    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
+    up[0] = v0;
+    up[(size_t)nb * N] = v1;
+}
+
+// The un-rotated inputs lifted to the extended basis for double hoisting: times P modulo every ciphertext prime,
+// zero modulo P.  grid: x = coefficients / 256, y = ciphertext, z = component * (r + 1) + prime.
+__global__ void __launch_bounds__(256) lift_times_p_kernel(const RingDev R, const u64* __restrict__ src, long long src_stride,
+                                                           u64* __restrict__ dst, long long dst_stride) {
+    grid_dependency_enter();
+    const u32 N = R.N, r = R.r, nb = r + 1;
+    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
+    const u32 ct = blockIdx.y, comp = blockIdx.z / nb, m = blockIdx.z % nb;
+    u64 v = 0;
+    if (m < r) {
+        u64 hi = 0, lo = 0;
+        mac128(hi, lo, src[(size_t)ct * src_stride + ((size_t)comp * r + m) * N + n], R.pmod[m]);
+        v = reduce128(hi, lo, R.q[m], R.mu[m], R.c64[m], R.c64s[m]);
+    }
+    dst[(size_t)ct * dst_stride + ((size_t)comp * nb + m) * N + n] = v;
+}
+
+cudaError_t launch_lift_times_p(const RingHost& ring, const u64* src, long long src_stride, u64* dst, long long dst_stride,
+                                u32 n_ct, cudaStream_t stream) {
+    if (n_ct == 0) return cudaSuccess;
+    ProfScope prof(ring.prof, CAT_POINTWISE, stream);
+    dim3 grid(ring.dev.N / 256, n_ct, 2 * (ring.dev.r + 1));
+    return launch_dependent(ring, lift_times_p_kernel, grid, dim3(256), 0, stream, ring.dev, src, src_stride, dst, dst_stride);
 }
 
 cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
-                                     int* error_flag, cudaStream_t stream) {
+                                     int* error_flag, cudaStream_t stream, u64* xext, const u32* pinv) {
     if (rb.n == 0) return cudaSuccess;
     u64 qmax = 0;
     for (u32 i = 0; i < ring.dev.r; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
@@ -614,7 +669,7 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
     }
     dim3 grid(rb.n, ring.dev.N / KI_TILE, r + 1);
     return launch_dependent(ring, key_inner_bulk_kernel, grid, dim3(KI_TILE), smem, stream, ring.dev, rb, dig, keys, u,
-                            small_ok, error_flag);
+                            small_ok, error_flag, xext, pinv);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -578,13 +578,15 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 const u64* up = epi.u + ((size_t)o * nb + ip) * R.N + n;
                 const ulonglong2 u0 = *(const ulonglong2*)up, u1 = *(const ulonglong2*)(up + 2);
                 uu[0] = u0.x; uu[1] = u0.y; uu[2] = u1.x; uu[3] = u1.y;
-                if (comp == 0) {
+                if (comp == 0 && !epi.plain) {
                     const u64* cp = epi.c0_base + (size_t)rb.c0[rot] * epi.c0_stride + (size_t)ip * R.N + n;
                     const ulonglong2 c0 = *(const ulonglong2*)cp, c1 = *(const ulonglong2*)(cp + 2);
                     cc[0] = c0.x; cc[1] = c0.y; cc[2] = c1.x; cc[3] = c1.y;
                 }
-                const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
-                pp[0] = pv.x; pp[1] = pv.y; pp[2] = pv.z; pp[3] = pv.w;
+                if (!epi.plain) {
+                    const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
+                    pp[0] = pv.x; pp[1] = pv.y; pp[2] = pv.z; pp[3] = pv.w;
+                }
             }
             set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, qd);
             u64 v4[4];
@@ -615,6 +617,14 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 ((ulonglong2*)op)[1] = make_ulonglong2(v4[2], v4[3]);
                 continue;
             }
+            if (EPI == 1 && epi.plain) {
+                u64* op = epi.out_base + (size_t)o * epi.out_stride + (size_t)mod * R.N + (size_t)chunk * LEN + 4 * s;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) v4[t] = mul_shoup(sub_mod(uu[t], v4[t], q), R.pinv[mod], R.pinvs[mod], q);
+                ((ulonglong2*)op)[0] = make_ulonglong2(v4[0], v4[1]);
+                ((ulonglong2*)op)[1] = make_ulonglong2(v4[2], v4[3]);
+                continue;
+            }
             if (EPI == 1) {
                 const u32 rot = o >> 1, comp = o & 1, ip = mod, r = R.r;
                 u64* op = epi.out_base + (size_t)rb.out[rot] * epi.out_stride + ((size_t)comp * r + ip) * R.N;
@@ -633,7 +643,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 const u32 at = tile_word_index(B.tile, pj, term, n);
                 const u32 fmt = tile_format(B.tile, mod);
                 if (fmt == TILE_W64) {
-                    if (B.split_bits) {
+                    if (B.split_bits && !(q >> 50)) {     // (the special prime of double hoisting stays in whole words)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) v4[i] = limb_split(v4[i], B.split_bits);
                     }
@@ -689,7 +699,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                     const ulonglong2* gp = (const ulonglong2*)(stage + (size_t)at * 8);
                     const ulonglong2 a = gp[0], b = gp[1];
                     v4[0] = a.x; v4[1] = a.y; v4[2] = b.x; v4[3] = b.y;
-                    if (B.split_bits) {
+                    if (B.split_bits && !(q >> 50)) {
 #pragma unroll
                         for (int i = 0; i < 4; ++i) v4[i] = limb_join(v4[i], B.split_bits);
                     }

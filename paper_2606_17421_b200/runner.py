@@ -29,15 +29,15 @@ class WorkloadRunner:
     def __init__(self, name: str, seed: int = 0, device: str = "cuda:0", cache: bool = True,
                  cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None,
                  fuse_shared_inputs: bool = True, fold_in_ciphertext: bool = False, compact_cache: bool = False,
-                 pack: str | None = None, moddown: str | None = None):
+                 pack: str | None = None, moddown: str | None = None, hoist: str | None = None):
         self.w = wl.WORKLOADS[name]
         ps = wl.PARAM_SETS[self.w.params]
         self.N, self.primes, self.P, self.scale = ps["N"], list(ps["primes"]), ps["special"], ps["scale"]
         self.r = len(self.primes)
         self.plan = self.w.plan
-        if pack or moddown:         # the workload's plan with another packing / key-switch variant
+        if pack or moddown or hoist:         # the workload's plan with another packing / key-switch variant
             self.plan = wl.PlanSpec(self.plan.D, self.plan.tau, self.plan.b, self.plan.g,
-                                    pack or self.plan.pack, moddown or self.plan.moddown)
+                                    pack or self.plan.pack, moddown or self.plan.moddown, hoist or self.plan.hoist)
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         # a stream of our own: the legacy default stream cannot be captured, which would keep the
@@ -49,13 +49,16 @@ class WorkloadRunner:
         self.ctx = bf.bf_ctx_create(self.N, self.primes + [self.P], self.r, self.scale,
                                     bf.bf_plan(self.plan.D, self.plan.tau, self.plan.b, self.plan.g,
                                                (bf.BF_PLAN_COMPLEX_PACK if self.plan.pack == "complex" else 0) |
-                                               (bf.BF_PLAN_MODDOWN_PER_OUTPUT if self.plan.moddown == "per_output" else 0)),
+                                               (bf.BF_PLAN_MODDOWN_PER_OUTPUT if self.plan.moddown == "per_output" else 0) |
+                                               (bf.BF_PLAN_DOUBLE_HOIST if self.plan.hoist == "double" else 0)),
                                     self.stream.cuda_stream)
         if compact_cache:           # narrower resident words per prime: 68 % of the cache for the 50 + 6 x 40-bit chain
             bf.bf_set_compact_cache(self.ctx, True)
         self.compact_cache = compact_cache
         # resident bytes per encoded coefficient over all primes (8 each, or 4 / 5 / 8 by prime size when compact)
         self.word_bytes = sum((4 if q < 2 ** 32 else 5 if q < 2 ** 40 else 8) if compact_cache else 8 for q in self.primes)
+        if self.plan.hoist == "double":     # the residue modulo the special prime is kept too, always in 8 bytes
+            self.word_bytes += 8
         budget = cache_budget_bytes if cache_budget_bytes is not None else self.w.cache_budget_bytes
         if budget:
             bf.bf_set_cache_budget(self.ctx, int(budget))

@@ -43,6 +43,7 @@ class PlanSpec:
     g: int
     pack: str = "real"                  # "complex": two output row blocks per plaintext (real and imaginary parts)
     moddown: str = "per_rotation"       # "per_output": one division by the special prime per output ciphertext
+    hoist: str = "single"               # "double": baby-step rotations stay in the extended basis, one division per inner sum
 
     @property
     def rows_per_ct(self) -> int:

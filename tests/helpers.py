@@ -29,7 +29,8 @@ class GpuSide:
         self.stream = torch.cuda.Stream(device=self.dev)
         torch.cuda.set_stream(self.stream)
         flags = (bf.BF_PLAN_COMPLEX_PACK if plan.pack == "complex" else 0) | \
-                (bf.BF_PLAN_MODDOWN_PER_OUTPUT if plan.moddown == "per_output" else 0)
+                (bf.BF_PLAN_MODDOWN_PER_OUTPUT if plan.moddown == "per_output" else 0) | \
+                (bf.BF_PLAN_DOUBLE_HOIST if plan.hoist == "double" else 0)
         p = bf.bf_plan(plan.D, plan.tau, plan.b, plan.g, flags)
         self.ctx = bf.bf_ctx_create(par.N, par.basis, par.r, par.scale, p,
                                     torch.cuda.current_stream().cuda_stream)

@@ -275,6 +275,37 @@ def test_linear_gpt2_qkv_one_division_by_P_per_output_bit_exact(pack):
     run_case(par, plan, L.d_out, L.d_in, 0, 1e-3, L.name)
 
 
+@pytest.mark.parametrize("pack,moddown", [("real", "per_rotation"), ("complex", "per_output")])
+@pytest.mark.parametrize("plan_t,shape", [
+    ((64, 4, 4, 4), (100, 130)),      # three input ciphertexts, ragged
+    ((64, 1, 8, 8), (128, 64)),       # classical layout, seven baby rotations
+    ((64, 32, 2, 1), (64, 64)),       # no giant step
+    ((128, 1, 1, 128), (128, 128)),   # no baby step: only P * ct, whose division by P is exact
+    ((64, 4, 16, 1), (150, 64)),      # 16 terms per group, half-filled last stage
+    ((64, 4, 4, 4), (64, 1472)),      # 23 input ciphertexts: their baby rotations span two key-switch batches
+])
+def test_linear_double_hoisting_small_ring(plan_t, shape, pack, moddown):
+    if plan_t[3] - 1 > 64 and moddown == "per_output":
+        pytest.skip("per-output division sums at most 64 giant steps")
+    par = oracle_params("n12")
+    run_case(par, ckks.Plan(*plan_t, pack=pack, moddown=moddown, hoist="double"), shape[0], shape[1], 8, 1e-2, f"dh{plan_t}")
+
+
+@pytest.mark.parametrize("pack,moddown", [("real", "per_rotation"), ("complex", "per_output")])
+def test_linear_gpt2_qkv_double_hoisting_bit_exact(pack, moddown):
+    w = wl.WORKLOADS["gpt2_qkv"]
+    par = oracle_params(w.params)
+    L = w.layers[0]
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, pack=pack, moddown=moddown, hoist="double")
+    run_case(par, plan, L.d_out, L.d_in, 0, 1e-3, L.name)
+
+
+def test_linear_double_hoisting_with_the_papers_own_parameter_set():
+    # a 60-bit ciphertext prime next to the 60-bit special prime: whole-word accumulation for every prime
+    par = oracle_params("paper_n13")
+    run_case(par, ckks.Plan(256, 16, 4, 4, hoist="double"), 300, 520, 4, 1e-2, "paper_n13_dh", tight=1e-3)
+
+
 def test_per_output_division_refuses_more_giant_steps_than_it_can_sum():
     from paper_2606_17421_b200 import bifrost as bf
     ps = wl.PARAM_SETS["n12"]
