@@ -108,6 +108,7 @@ struct bf_ctx {
     u32* perms_fwd = nullptr;        // [n_keys][N] perm: rotated[n] = unrotated[perm[n]] (per-output division by P)
     u32 n_keys = 0;
     // scratch (grow-only)
+    size_t dig_half = 0;            // words from a digit set in Dig to its staging twin
     DevBuf X, X0, Aext, Dig, U, Ubig, Tc, Tn, Cc, A, Rres, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
     u64 cache_budget = 0, cache_used = 0;
     std::vector<bf_weights*> weights;
@@ -749,7 +750,10 @@ static int moddown_batch(bf_ctx* ctx, const Lane& lane, const RotBatch& rb, cons
 
 static int ensure_rot_scratch(bf_ctx* ctx, u32 n_dig_sets, u32 n_rot) {
     const size_t N = ctx->N, r = ctx->r, nb = r + 1;
-    TRY(ensure(ctx, ctx->Dig, (size_t)n_dig_sets * r * nb * N * 8));
+    // digit sets, tile-major for the inner product, and behind them a staging area of the same size for the
+    // intermediate of their transforms (natural order)
+    TRY(ensure(ctx, ctx->Dig, (size_t)2 * n_dig_sets * r * nb * N * 8));
+    ctx->dig_half = ctx->Dig.cap / 16;
     TRY(ensure(ctx, ctx->U, (size_t)n_rot * 2 * nb * N * 8));
     TRY(ensure(ctx, ctx->Tc, (size_t)n_rot * 2 * N * 8));
     TRY(ensure(ctx, ctx->Tn, (size_t)n_rot * 2 * r * N * 8));
@@ -780,7 +784,9 @@ static int modup(bf_ctx* ctx, cudaStream_t stream, const u64* c1_coeff, long lon
     B.src_so2 = set_stride;
     B.src_so = N;
     B.src_sm = 0;
-    B.dst = dig;
+    B.dst = dig + ctx->dig_half;         // staging between the two passes; the result goes to dig, tile-major
+    B.dtile_ptr = dig;
+    B.dtile_div = r;
     B.dst_so = (long long)nb * N;
     B.dst_sm = N;
     B.skip_diag = 1;
@@ -912,7 +918,9 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             const u32 qn = (n_in - q0 < in_batch) ? n_in - q0 : in_batch;
             TRY(modup(ctx, ctx->stream, ct_in + (size_t)q0 * ctw + (size_t)r * N, (long long)ctw, qn, Dig,
                       X0 + (size_t)q0 * x0_stride + (size_t)r * N, x0_stride));
-            // the rotations of the batch, dealt out to the lanes in contiguous runs
+            // the rotations of the batch, key-major (rotation t = (k - 1) * qn + q: those that share a key follow one
+            // another, so that an inner-product block loads the key once for all of them), dealt out to the lanes
+            // in contiguous runs
             const u32 n_rot = qn * (b - 1);
             const u32 per = cdiv(n_rot, (u32)lanes_baby);
             const int used = (int)cdiv(n_rot, per);
@@ -922,7 +930,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
                 memset(&rb, 0, sizeof(rb));
                 const u32 t_end = (u32)(c + 1) * per < n_rot ? (u32)(c + 1) * per : n_rot;
                 for (u32 t = (u32)c * per; t < t_end; ++t) {
-                    const u32 q = t / (b - 1), k = t % (b - 1) + 1;
+                    const u32 q = t % qn, k = t / qn + 1;
                     const int i = rb.n++;
                     rb.key[i] = baby_key[k];
                     rb.dig[i] = (int)q;

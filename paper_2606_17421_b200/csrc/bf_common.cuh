@@ -230,6 +230,10 @@ struct RotBatch {                     // one key-switch launch over n rotations
     int dig[MAX_ROT_BATCH];           // which digit set the rotation reads
     int c0[MAX_ROT_BATCH];            // which source ciphertext is being rotated (its c0 is added)
     int out[MAX_ROT_BATCH];           // which output ciphertext slot receives the result
+    // runs of consecutive rotations that use the same key (filled in by the inner-product launcher): a block of the
+    // inner product takes one run, loads the key once and walks the run's digit sets
+    int n_groups;
+    unsigned char grp_first[MAX_ROT_BATCH], grp_cnt[MAX_ROT_BATCH];
 };
 
 // Epilogue of the division by P, fused into the forward transform of the lifted P-residue
@@ -339,7 +343,19 @@ struct PolyBatch {
                                   //   product ends in a Montgomery reduction)
     u32 split_bits;               // L > 0: the NTT-domain side of the transform is stored as two L-bit-aligned
                                   // limbs per word, (v >> L) << 32 | (v & (2^L - 1)); forward writes, inverse reads it
+    u64* dtile_ptr;               // forward only, non-null: the final result goes there instead of dst, tile-major in tiles
+    u32 dtile_div;                //   of KS_TILE coefficients (see ks_tile_index); with `scatter` the store is permuted
 };
+
+// Operands of the key-switch inner product (digit sets and rotation keys) are kept tile-major, so that what a block
+// needs of one (outer index / div, modulus, tile) is contiguous and arrives by one bulk copy:
+//   polynomial (o, m), coefficient n  ->  ((((o / div) * n_m + m) * (N / KS_TILE) + n / KS_TILE) * div + o % div) * KS_TILE + n % KS_TILE
+// digits: o = set * r + digit, div = r (a block reads the r digit segments of a set, modulus and tile);
+// keys: o = (key * r + digit) * 2 + component, div = 2r.
+constexpr u32 KS_TILE = 128;
+__host__ __device__ __forceinline__ size_t ks_tile_index(u32 N, u32 n_m, u32 div, u32 o, u32 m, u32 n) {
+    return ((((size_t)(o / div) * n_m + m) * (N / KS_TILE) + n / KS_TILE) * div + o % div) * KS_TILE + n % KS_TILE;
+}
 
 __device__ __forceinline__ u64 limb_split(u64 v, u32 L) { return ((v >> L) << 32) | (v & ((1ull << L) - 1)); }
 __device__ __forceinline__ u64 limb_join(u64 s, u32 L) { return ((s >> 32) << L) | (s & 0xffffffffull); }

@@ -528,91 +528,112 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 // un-rotated index space with fully coalesced operands:
 //   u'[rot][comp][m][n] = sum_j dig[dig(rot)][j][m][n] * key'[key(rot)][j][comp][m][n]
 // and the automorphism is applied once, as a scatter, when the rotated ciphertext is assembled.
-// The key stream is read once per rotation; products accumulate as 32-bit limb partial sums
-// (with carry counters where the 60-bit special prime needs them), one reduction per output word.
-// grid: x = rotation (fastest, so that rotations sharing a key or a digit set run side by side and
-// meet in L2), y = tile, z = modulus of the extended basis.
+// Products accumulate as 32-bit limb partial sums (with carry counters where the 60-bit special prime needs
+// them), one reduction per output word.
 //
-// Bulk-copy version: a block owns one (rotation, modulus, tile of 128 coefficients).  Its 3r operand
-// segments (digit, key.b, key.a for every digit j; 1 KB each) are fetched by asynchronous bulk
-// copies into shared memory in one go, so the number of bytes in flight does not depend on
-// registers; ten blocks per SM overlap one block's arithmetic with the others' copies (measured: 128-coefficient
-// tiles beat 256 by 3 %, 64 lose 2 to 4 %).  The keys are resident in Montgomery form (times 2^64 mod q), so the
-// sum of the r products ends in the two-round 32-bit Montgomery reduction: r * max digit < 2^64 keeps it below
-// q * 2^64.
-constexpr int KI_TILE = 128;
+// A block owns one (run of rotations that share a key, modulus, tile of 128 coefficients): the baby rotations
+// of several input ciphertexts by the same amount, or the giant rotations of several output blocks by the same
+// amount.  The key's 2r segments of the tile (1 KB each) are fetched once by asynchronous bulk copies and stay
+// in shared memory, so that the key stream crosses HBM (and L2) once per run instead of once per rotation; the
+// r digit segments of each rotation of the run follow through two buffers, the next rotation's copies in flight
+// while the current one is multiplied.  The keys are resident in Montgomery form (times 2^64 mod q), so the sum
+// of the r products ends in the two-round 32-bit Montgomery reduction: r * max digit < 2^64 keeps it below
+// q * 2^64.  With double hoisting the block also finishes the rotated input (see launch_key_inner_product).
+// grid: x = run, y = tile, z = modulus of the extended basis.
+constexpr int KI_TILE = (int)KS_TILE;
 
-__global__ void __launch_bounds__(KI_TILE, 10) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
-                                                                    const u64* __restrict__ dig,
-                                                                    const u64* __restrict__ keys, u64* __restrict__ u,
-                                                                    u32 small_ok, int* __restrict__ error_flag,
-                                                                    u64* __restrict__ xext, const u32* __restrict__ pinv) {
+__global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
+                                                                   const u64* __restrict__ dig,
+                                                                   const u64* __restrict__ keys, u64* __restrict__ u,
+                                                                   u32 small_ok, int* __restrict__ error_flag,
+                                                                   u64* __restrict__ xext, const u32* __restrict__ pinv) {
     extern __shared__ __align__(128) unsigned char ki_smem[];
-    const u32 rot = blockIdx.x, m = blockIdx.z;
+    const u32 grp = blockIdx.x, m = blockIdx.z;
+    const u32 first = rb.grp_first[grp], cnt = rb.grp_cnt[grp];      // this block's run of rotations: one key
     const u32 N = R.N, r = R.r, nb = r + 1;
     const u32 n0 = blockIdx.y * KI_TILE;
-    u64* sd = (u64*)ki_smem;                        // [r][KI_TILE] digits
-    u64* sk = sd + (size_t)r * KI_TILE;             // [r][2][KI_TILE] key components
-    u64* bar = sk + (size_t)2 * r * KI_TILE;
+    u64* sk = (u64*)ki_smem;                        // [r][2][KI_TILE] key components
+    u64* sd = sk + (size_t)2 * r * KI_TILE;         // [2][r][KI_TILE] digits of the current and the next rotation
+    u64* kbar = sd + (size_t)2 * r * KI_TILE;
+    u64* dbar = kbar + 1;                           // [2]
     const u32 tid = threadIdx.x;
     asm volatile("griddepcontrol.launch_dependents;");
     if (tid == 0) {
-        mbar_init(bar, 1);
+        mbar_init(kbar, 1);
+        mbar_init(&dbar[0], 1);
+        mbar_init(&dbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (tid < 32) {
-        if (tid == 0) mbar_expect_tx(bar, 3 * r * KI_TILE * 8);
+    // digit segments of rotation `first + it` into buffer it & 1
+    auto fetch_digits = [&](u32 it) {
+        u64* buf = sd + (size_t)(it & 1) * r * KI_TILE;
+        if (tid == 0) mbar_expect_tx(&dbar[it & 1], r * KI_TILE * 8);
         __syncwarp();
-        const u64* dp = dig + ((size_t)rb.dig[rot] * r * nb + m) * N + n0;
-        const u64* kp = keys + ((size_t)rb.key[rot] * r * 2 * nb + m) * N + n0;
+        // the r digit segments of this set, modulus and tile are contiguous (see ks_tile_index): one copy
+        if (tid == 0)
+            bulk_g2s(buf, dig + ks_tile_index(N, nb, r, (u32)rb.dig[first + it] * r, m, n0), r * KI_TILE * 8, &dbar[it & 1]);
+    };
+    if (tid < 32) {
+        if (tid == 0) mbar_expect_tx(kbar, 2 * r * KI_TILE * 8);
+        __syncwarp();
         // the keys do not depend on the previous kernel: fetch them before waiting for it, the digits after
         const u64 stream_policy = l2_evict_first_policy();      // keys stream through; digits and outputs stay in L2
-        for (u32 e = tid; e < 2 * r; e += 32)
-            bulk_g2s_stream(sk + (size_t)e * KI_TILE, kp + (size_t)e * nb * N, KI_TILE * 8, bar, stream_policy);
+        if (tid == 0)       // the 2r key segments of this key, modulus and tile: one contiguous block
+            bulk_g2s_stream(sk, keys + ks_tile_index(N, nb, 2 * r, (u32)rb.key[first] * 2 * r, m, n0), 2 * r * KI_TILE * 8, kbar,
+                            stream_policy);
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        for (u32 j = tid; j < r; j += 32)
-            bulk_g2s(sd + (size_t)j * KI_TILE, dp + (size_t)j * nb * N, KI_TILE * 8, bar);
+        fetch_digits(0);
+        if (cnt > 1) fetch_digits(1);
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
-    mbar_wait(bar, 0, error_flag);
+    mbar_wait(kbar, 0, error_flag);
     const u64 q = R.q[m];
     const u32 qneg32 = (u32)R.qneg[m];
-    u64 v0, v1;
-    if (m < r && small_ok) {
-        LimbAcc<true> a0, a1;
-        for (u32 j = 0; j < r; ++j) {
-            const u64 d = sd[j * KI_TILE + tid];
-            a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
-            a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+    for (u32 it = 0; it < cnt; ++it) {
+        const u32 rot = first + it;
+        const u64* sdc = sd + (size_t)(it & 1) * r * KI_TILE;
+        mbar_wait(&dbar[it & 1], (it >> 1) & 1, error_flag);
+        u64 v0, v1;
+        if (m < r && small_ok) {
+            LimbAcc<true> a0, a1;
+            for (u32 j = 0; j < r; ++j) {
+                const u64 d = sdc[j * KI_TILE + tid];
+                a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
+                a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+            }
+            v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
+            v1 = a1.reduce_mont32(q, qneg32);
+        } else {
+            LimbAcc<false> a0, a1;
+            for (u32 j = 0; j < r; ++j) {
+                const u64 d = sdc[j * KI_TILE + tid];
+                a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
+                a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+            }
+            v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
+            v1 = a1.reduce_mont32(q, qneg32);
         }
-        v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
-        v1 = a1.reduce_mont32(q, qneg32);
-    } else {
-        LimbAcc<false> a0, a1;
-        for (u32 j = 0; j < r; ++j) {
-            const u64 d = sd[j * KI_TILE + tid];
-            a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
-            a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+        if (it + 2 < cnt) {                                  // the buffer is free once every thread has read it
+            __syncthreads();
+            if (tid < 32) fetch_digits(it + 2);
         }
-        v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
-        v1 = a1.reduce_mont32(q, qneg32);
+        if (xext) {
+            // double hoisting: no division by P; the rotated input in the extended basis is (P*c0 + u0, u1) moved
+            // through the rotation's permutation; P*c0 (zero modulo P) was stored as the un-rotated term
+            const size_t term_words = (size_t)2 * nb * N;
+            const u32 n = n0 + tid;
+            v0 = add_mod(v0, xext[(size_t)rb.c0[rot] * term_words + (size_t)m * N + n], q);
+            u64* xp = xext + (size_t)rb.out[rot] * term_words + (size_t)m * N + __ldg(&pinv[(size_t)rb.key[rot] * N + n]);
+            xp[0] = v0;
+            xp[(size_t)nb * N] = v1;
+        } else {
+            u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
+            up[0] = v0;
+            up[(size_t)nb * N] = v1;
+        }
     }
-    if (xext) {
-        // double hoisting: no division by P; the rotated input in the extended basis is (P*c0 + u0, u1) moved
-        // through the rotation's permutation; P*c0 (zero modulo P) was stored as the un-rotated term
-        const size_t term_words = (size_t)2 * nb * N;
-        const u32 n = n0 + tid;
-        v0 = add_mod(v0, xext[(size_t)rb.c0[rot] * term_words + (size_t)m * N + n], q);
-        u64* xp = xext + (size_t)rb.out[rot] * term_words + (size_t)m * N + __ldg(&pinv[(size_t)rb.key[rot] * N + n]);
-        xp[0] = v0;
-        xp[(size_t)nb * N] = v1;
-        return;
-    }
-    u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
-    up[0] = v0;
-    up[(size_t)nb * N] = v1;
 }
 
 // The un-rotated inputs lifted to the extended basis for double hoisting: times P modulo every ciphertext prime,
@@ -660,15 +681,27 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
         ring.prof->key_bytes_distinct += distinct * key_bytes;
         ring.prof->key_bytes_per_rotation += (u64)rb.n * key_bytes;
     }
-    const size_t smem = (size_t)3 * r * KI_TILE * 8 + 16;
+    const size_t smem = (size_t)4 * r * KI_TILE * 8 + 32;
+    // runs of consecutive rotations with the same key: one block per run, tile and modulus
+    RotBatch rbg = rb;
+    rbg.n_groups = 0;
+    for (int t = 0; t < rb.n; ++t) {
+        if (t > 0 && rb.key[t] == rb.key[t - 1]) {
+            rbg.grp_cnt[rbg.n_groups - 1]++;
+        } else {
+            rbg.grp_first[rbg.n_groups] = (unsigned char)t;
+            rbg.grp_cnt[rbg.n_groups] = 1;
+            rbg.n_groups++;
+        }
+    }
     static bool attr_set[MAX_DEVICES] = {false};     // per device: the attribute belongs to the device's copy of the kernel
     if (!attr_set[device_slot(ring)]) {
         cudaError_t e = cudaFuncSetAttribute(key_inner_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
         if (e != cudaSuccess) return e;
         attr_set[device_slot(ring)] = true;
     }
-    dim3 grid(rb.n, ring.dev.N / KI_TILE, r + 1);
-    return launch_dependent(ring, key_inner_bulk_kernel, grid, dim3(KI_TILE), smem, stream, ring.dev, rb, dig, keys, u,
+    dim3 grid(rbg.n_groups, ring.dev.N / KI_TILE, r + 1);
+    return launch_dependent(ring, key_inner_bulk_kernel, grid, dim3(KI_TILE), smem, stream, ring.dev, rbg, dig, keys, u,
                             small_ok, error_flag, xext, pinv);
 }
 

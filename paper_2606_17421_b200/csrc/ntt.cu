@@ -454,7 +454,8 @@ ntt_strided(const RingDev R, const PolyBatch B) {
         u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
         for (int w = threadIdx.x; w < (1 << (LOG_R + LOG_LANES)); w += blockDim.x) {
             const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * (1 << LOG_LANES) + (w & ((1 << LOG_LANES) - 1));
-            dd[gidx] = ds[gidx];
+            if (B.dtile_ptr) B.dtile_ptr[ks_tile_index(R.N, B.n_m, B.dtile_div, o, m, (u32)gidx)] = ds[gidx];
+            else dd[gidx] = ds[gidx];
         }
         return;
     }
@@ -495,7 +496,8 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
             u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
             for (int w = threadIdx.x; w < POINTS; w += blockDim.x) {
                 const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1));
-                dd[gidx] = ds[gidx];
+                if (B.dtile_ptr) B.dtile_ptr[ks_tile_index(R.N, B.n_m, B.dtile_div, o, m, (u32)gidx)] = ds[gidx];
+                else dd[gidx] = ds[gidx];
             }
             continue;
         }
@@ -661,6 +663,20 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
             if (B.split_bits) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) v4[i] = limb_split(v4[i], B.split_bits);
+            }
+            if (B.dtile_ptr) {  // operands of the key-switch inner product: tile-major (keys also permuted, times 2^64)
+                if (B.scatter) {
+                    const u32* sc = B.scatter + (size_t)(o / B.scatter_div) * R.N + chunk * LEN + 4 * s;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        B.dtile_ptr[ks_tile_index(R.N, B.n_m, B.dtile_div, o, m, sc[i])] =
+                            B.scatter_mont ? mul_shoup(v4[i], R.c64[mod], R.c64s[mod], q) : v4[i];
+                } else {
+                    ulonglong2* gp = (ulonglong2*)(B.dtile_ptr + ks_tile_index(R.N, B.n_m, B.dtile_div, o, m, chunk * LEN + 4 * s));
+                    gp[0] = make_ulonglong2(v4[0], v4[1]);
+                    gp[1] = make_ulonglong2(v4[2], v4[3]);
+                }
+                continue;
             }
             if (B.scatter) {    // permuted store (keys are kept pre-permuted by their automorphism)
                 const u32* sc = B.scatter + (size_t)(o / B.scatter_div) * R.N + chunk * LEN + 4 * s;
@@ -927,6 +943,8 @@ cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B0, u32 n_o
     B.scatter_div = scatter_div;
     B.scatter_dst = final_dst;
     B.scatter_mont = 1;           // (the only permuted store is that of the rotation keys)
+    B.dtile_ptr = final_dst;      // tile-major: o = (key * r + digit) * 2 + component
+    B.dtile_div = scatter_div;
     return launch_contig<true>(ring, B, n_polys, stream);
 }
 

@@ -111,6 +111,9 @@ for _D, _tau, _b, _g in ((1024, 16, 16, 4), (512, 32, 4, 4), (256, 64, 2, 2), (1
 # The GPT-2 QKV projection under the prototype's own CKKS parameters (Sec. 4.2): N = 8192, 4096 slots.
 WORKLOADS["gpt2_qkv_paper_params"] = Workload("gpt2_qkv_paper_params", "paper_n13", PlanSpec(1024, 4, 16, 16),
                                               (GPT2_LAYER[0],))
+# One transformer layer of the GPT-2 step (1.2 GB of encoded weights): small enough for profiler captures that need
+# several passes, with the call shapes of the whole step (one and three input ciphertexts, one and three output blocks).
+WORKLOADS["gpt2_layer"] = Workload("gpt2_layer", "n15", PlanSpec(1024, 16, 16, 4), GPT2_LAYER)
 CONFIG_ORDER = ["tiny", "gpt2_qkv", "gpt2_step", "qwen3_step", "llama3_layer"]
 
 
