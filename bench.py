@@ -109,13 +109,14 @@ MIN_REGION_S = 0.5      # every timed region lasts at least this long (steps are
 # (compact cache format), fold (in-ciphertext fold of the tau partial sums), complex (two output row blocks per
 # plaintext, in the real and imaginary parts of the slots), per_output (one division by the special prime per
 # output ciphertext instead of one per giant rotation), double_hoist (baby-step rotations kept in the extended basis,
-# one division per inner sum).
+# one division per inner sum), coeff64 / coeff32 (cached weights kept as rounded integer coefficients and transformed
+# on every call).
 # The headline is the largest single-GPU configuration under the fastest plan variant that is parity-tested; the same
 # step under the plain plan, and the other configurations under both, follow as extras.
-BEST = "complex,per_output"
+BEST = "complex,per_output,double_hoist"
 DEFAULT_WORKLOAD = "qwen3_step@budget=60," + BEST
 DEFAULT_EXTRA = ",".join([
-    "qwen3_step@budget=60", "qwen3_step@budget=40.5", "qwen3_step@budget=40.5,compact",
+    "qwen3_step@budget=60", "qwen3_step@budget=40.5", "qwen3_step@budget=40.5,compact", "qwen3_step@coeff32," + BEST,
     "gpt2_qkv", "gpt2_qkv@" + BEST, "gpt2_step", "gpt2_step@" + BEST,
     "llama3_layer", "llama3_layer@" + BEST, "llama3_layer@on_the_fly", "llama3_layer@on_the_fly," + BEST, "tiny"])
 
@@ -138,6 +139,8 @@ def parse_spec(spec: str):
             kw["moddown"] = "per_output"
         elif o == "double_hoist":
             kw["hoist"] = "double"
+        elif o in ("coeff64", "coeff32"):
+            kw["coef_bits"] = int(o[5:])
         else:
             raise ValueError(f"unknown workload option {o!r}")
     return name, kw
@@ -182,7 +185,7 @@ def transform_counts(runner) -> dict:
             inv[i] += n_giant + 2 * n_out                  # c1 of the giant-step inputs; outputs
         fwd[r] += sets * r
         inv[r] += n_lift                                   # P-residues of the inner products
-        if not e["handle"]:                                # on-the-fly path: every diagonal is transformed on each call
+        if runner.transforms_weights_per_call(e):          # on the fly or kept as coefficients: every diagonal is transformed on each call
             n_diag = n_in * n_out * b * g
             for i in range(r + (1 if runner.plan.hoist == "double" else 0)):
                 fwd[i] += n_diag
@@ -340,7 +343,8 @@ class Measurement:
                          "moddown": R.plan.moddown, "hoist": R.plan.hoist},
                 "ciphertexts_in": sum(e["n_in"] for e in R.layers), "ciphertexts_out": sum(e["n_out"] for e in R.layers),
                 "boundary_bytes": h2d + d2h, "rotation_keys": len(R.rot_steps), "fallback_layers": R.n_fallback_layers(),
-                "encoded_weight_bytes_cached": R.cached_pt_bytes(), "encoded_weight_bytes_total": R.total_pt_bytes()}
+                "encoded_weight_bytes_cached": R.cached_pt_bytes(), "encoded_weight_bytes_total": R.total_pt_bytes(),
+                "resident_weight_bytes": R.resident_bytes()}
 
     def close(self):
         import torch

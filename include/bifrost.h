@@ -141,6 +141,16 @@ int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weight
  * the gain is capacity).  bf_weights_bytes reports sizes for the current setting. */
 int bf_set_compact_cache(bf_ctx* ctx, int on);
 
+/* Coefficient form of the cache (the other answer to the memory wall of Sec. 6.1): with
+ * bf_set_coefficient_cache(ctx, 64 or 32) every weight encoded afterwards is kept as the rounded
+ * integer coefficients of its diagonals, one 64- or 32-bit word per coefficient whatever the number
+ * of primes (1/r or 1/(2r) of the transform-domain cache), and bf_linear reduces them per prime and
+ * transforms them on every call: the fallback path without its encoder.  Results are identical.
+ * 32 bits hold |coefficient| < 2^31: bf_encode_weights returns BF_ERR_RANGE when the weights and the
+ * scale give more.  bits = 0 (default) switches back to transform-domain residues; handles of all
+ * kinds can be used side by side.  bf_weights_bytes reports sizes for the current setting. */
+int bf_set_coefficient_cache(bf_ctx* ctx, int bits);
+
 /* Fallback path of bf_linear (W_raw given, Sec. 4.2 "fallback encode"): output groups are encoded
  * in rounds into a scratch buffer and consumed by the multiply-accumulate; `bytes` bounds that
  * buffer (default 4 GiB; one output group, n_in * b encoded diagonals, is the minimum whatever the

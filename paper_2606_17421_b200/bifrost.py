@@ -63,6 +63,7 @@ _SIGNATURES = {
     "bf_set_dependent_launch": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_set_lanes": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_set_compact_cache": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "bf_set_coefficient_cache": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_set_encode_scratch": (ctypes.c_int, [_vp, _u64]),
     "bf_rescale": (ctypes.c_int, [_vp, _vp, _vp, _u32, _u32, ctypes.POINTER(ctypes.c_double)]),
     "bf_fold": (ctypes.c_int, [_vp, _vp, _u32]),
@@ -186,6 +187,10 @@ def bf_set_graph_replay(ctx, on: bool):
 
 def bf_set_compact_cache(ctx, on: bool):
     _check(load().bf_set_compact_cache(ctx, 1 if on else 0), "bf_set_compact_cache", ctx)
+
+
+def bf_set_coefficient_cache(ctx, bits: int):
+    _check(load().bf_set_coefficient_cache(ctx, bits), "bf_set_coefficient_cache", ctx)
 
 
 def bf_set_encode_scratch(ctx, n_bytes: int):

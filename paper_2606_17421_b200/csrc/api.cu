@@ -81,6 +81,10 @@ struct bf_weights {
                         // NTT domain, Montgomery form (times 2^64 mod q_i), limbs split when the primes allow
     TileLayout lay;
     size_t bytes;
+    // coefficient form (bf_set_coefficient_cache): pt is null and the rounded integer coefficients of the diagonals
+    // are kept instead, [diagonal][N] in the order [j][p][q][k], 64- or 32-bit; every call transforms them
+    void* coef = nullptr;
+    u32 coef_bits = 0;
 };
 
 struct bf_ctx {
@@ -99,6 +103,7 @@ struct bf_ctx {
     // multiply-accumulate (at least one group is always held).  Measured on a LLaMA-3-8B layer: 1 GiB 78 ms,
     // 2 GiB 73 ms, 4 GiB 70 ms, 8 GiB 69 ms: the rotated inputs are re-read once per round
     size_t encode_scratch_bytes = (size_t)4 << 30;
+    u32 coef_cache_bits = 0;        // 64 / 32: weights encoded from now on are kept as rounded coefficients
     int* overflow_flag = nullptr;   // [0]: encoder range overflow; [1]: a bounded device-side wait gave up
     int* device_error = nullptr;
     // rotation keys
@@ -400,6 +405,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
     for (bf_weights* w : ctx->weights) {
         if (w) {
             cudaFree(w->pt);
+            cudaFree(w->coef);
             delete w;
         }
     }
@@ -540,14 +546,18 @@ static u32 n_out_cts(const bf_ctx* ctx, u32 d_out) {
 extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
     if (!ctx) return 0;
     const u32 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = n_out_cts(ctx, d_out);
+    if (ctx->coef_cache_bits)       // one rounded coefficient per diagonal and ring position, whatever the primes
+        return (u64)n_in * n_out * (ctx->plan.tile_D / ctx->plan.tau) * ctx->N * (ctx->coef_cache_bits / 8);
     const TileLayout lay = mac_tile_layout(ctx->ring, n_out * ctx->plan.bsgs_g, n_in * ctx->plan.bsgs_b, mac_primes(ctx));
     return mac_tile_bytes(ctx->ring, lay);
 }
 
 // Encode diagonals [d0, d0 + count) of W (order [j][p][q][k], i.e. group pj = d / n_terms, term d % n_terms)
 // into dst in the tile-major layout `lay`, whose group 0 is group pj0 of W.
+// The coefficients come from the encoder (W), or from a handle that keeps them (stored; W is then unused); coef_out
+// non-null: only encode, leaving the 64-bit coefficients of diagonal d0 + i at coef_out + i*N (no transform).
 static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0, u32 count, u64* dst,
-                        const TileLayout& lay, u32 pj0) {
+                        const TileLayout& lay, u32 pj0, const bf_weights* stored = nullptr, i64* coef_out = nullptr) {
     const u32 N = ctx->N, r = lay.n_primes, n = N / 2;       // (r: primes each diagonal is reduced into)
     // diagonals per pass: the encoder and the transforms gain from large batches (measured: 32 -> 128 per
     // pass takes 6 to 8 % off a call that encodes on the fly); the scratch of a pass is held to about 0.5 GB
@@ -555,9 +565,9 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
     if (chunk > 256) chunk = 256;
     if (chunk < 32) chunk = 32;
     if (chunk > count) chunk = count > 0 ? count : 1;
-    TRY(ensure(ctx, ctx->fft, (size_t)chunk * n * sizeof(double2)));
-    TRY(ensure(ctx, ctx->coef, (size_t)chunk * N * sizeof(i64)));
-    TRY(ensure(ctx, ctx->ptnat, (size_t)chunk * r * N * sizeof(u64)));
+    if (!stored) TRY(ensure(ctx, ctx->fft, (size_t)chunk * n * sizeof(double2)));
+    if (!coef_out && !(stored && stored->coef_bits == 64)) TRY(ensure(ctx, ctx->coef, (size_t)chunk * N * sizeof(i64)));
+    if (!coef_out) TRY(ensure(ctx, ctx->ptnat, (size_t)chunk * r * N * sizeof(u64)));
     EncodeTables tab;
     tab.slot_of_pos = ctx->slot_of_pos;
     tab.T = ctx->T;
@@ -578,10 +588,20 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
         db.g = ctx->plan.bsgs_g;
         db.d0 = d0 + lo;
         db.count = cnt;
-        CK(launch_encode(ctx->ring, tab, db, (double2*)ctx->fft.p, (i64*)ctx->coef.p, ctx->overflow_flag, ctx->stream));
+        const void* coef_src = ctx->coef.p;
+        if (stored && stored->coef_bits == 64) {
+            coef_src = (const i64*)stored->coef + (size_t)(d0 + lo) * N;
+        } else if (stored) {
+            CK(launch_widen_i32(ctx->ring, (const int*)stored->coef + (size_t)(d0 + lo) * N, (i64*)ctx->coef.p, (size_t)cnt * N,
+                                ctx->stream));
+        } else {
+            i64* into = coef_out ? coef_out + (size_t)lo * N : (i64*)ctx->coef.p;
+            CK(launch_encode(ctx->ring, tab, db, (double2*)ctx->fft.p, into, ctx->overflow_flag, ctx->stream));
+            if (coef_out) continue;
+        }
         PolyBatch B;
         memset(&B, 0, sizeof(B));
-        B.src = ctx->coef.p;
+        B.src = coef_src;
         B.dst = (u64*)ctx->ptnat.p;                 // first pass lands here; the second writes the tiles
         B.src_so = N;
         B.src_sm = 0;
@@ -630,23 +650,47 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
     w->n_out = n_out_cts(ctx, d_out);
     w->bytes = bytes;
     w->lay = mac_tile_layout(ctx->ring, w->n_out * ctx->plan.bsgs_g, w->n_in * ctx->plan.bsgs_b, mac_primes(ctx));
-    cudaError_t e = cudaMalloc(&w->pt, bytes);
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        delete w;
-        return BF_ERR_OOM;
-    }
     const u32 n_diag = w->n_in * w->n_out * (ctx->plan.tile_D / ctx->plan.tau);
     int s = BF_OK;
-    {   // padding words of the layout are never read, but keep the allocation defined
-        cudaError_t me = cudaMemsetAsync(w->pt, 0, bytes, ctx->stream);
-        if (me != cudaSuccess) s = BF_ERR_CUDA;
+    if (ctx->coef_cache_bits) {
+        // coefficient form: run the encoder only; 32-bit storage goes through a 64-bit staging area in pieces and
+        // is refused (BF_ERR_RANGE) when a coefficient does not fit
+        w->coef_bits = ctx->coef_cache_bits;
+        w->pt = nullptr;
+        if (cudaMalloc(&w->coef, bytes) != cudaSuccess) {
+            cudaGetLastError();
+            delete w;
+            return BF_ERR_OOM;
+        }
+        if (w->coef_bits == 64) {
+            s = encode_range(ctx, W, d_out, d_in, 0, n_diag, nullptr, w->lay, 0, nullptr, (i64*)w->coef);
+        } else {
+            const u32 piece = 256;
+            s = ensure(ctx, ctx->coef, (size_t)piece * ctx->N * sizeof(i64));
+            for (u32 d0 = 0; d0 < n_diag && s == BF_OK; d0 += piece) {
+                const u32 cnt = n_diag - d0 < piece ? n_diag - d0 : piece;
+                s = encode_range(ctx, W, d_out, d_in, d0, cnt, nullptr, w->lay, 0, nullptr, (i64*)ctx->coef.p);
+                if (s == BF_OK && launch_narrow_i64(ctx->ring, (const i64*)ctx->coef.p, (int*)w->coef + (size_t)d0 * ctx->N,
+                                                    (size_t)cnt * ctx->N, ctx->overflow_flag, ctx->stream) != cudaSuccess)
+                    s = BF_ERR_CUDA;
+            }
+        }
+    } else {
+        if (cudaMalloc(&w->pt, bytes) != cudaSuccess) {
+            cudaGetLastError();
+            delete w;
+            return BF_ERR_OOM;
+        }
+        // padding words of the layout are never read, but keep the allocation defined
+        if (cudaMemsetAsync(w->pt, 0, bytes, ctx->stream) != cudaSuccess) s = BF_ERR_CUDA;
+        if (s == BF_OK) s = encode_range(ctx, W, d_out, d_in, 0, n_diag, w->pt, w->lay, 0);
     }
-    if (s == BF_OK) s = encode_range(ctx, W, d_out, d_in, 0, n_diag, w->pt, w->lay, 0);
     if (s == BF_OK) s = check_overflow(ctx);
     if (s != BF_OK) {
         cudaStreamSynchronize(ctx->stream);
         cudaFree(w->pt);
+        cudaFree(w->coef);
+        cudaGetLastError();
         delete w;
         return s;
     }
@@ -662,6 +706,7 @@ extern "C" void bf_weights_free(bf_ctx* ctx, bf_weights* w) {
         if (ctx->weights[i] == w) {
             cudaStreamSynchronize(ctx->stream);
             cudaFree(w->pt);
+            cudaFree(w->coef);
             ctx->cache_used -= w->bytes;
             ctx->epoch++;
             delete w;
@@ -953,10 +998,11 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     // ---- multiply-accumulate over the encoded diagonals (double hoisting: over the extended basis, into Aext)
     const u32 n_terms = n_in * b, n_pj = n_out * g;
     u64* mac_out = dh ? (u64*)ctx->Aext.p : A;
-    if (pt_weights) {
+    if (pt_weights && pt_weights->pt) {
         CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, mac_out, n_pj, n_terms, true, ctx->device_error, ctx->stream));
     } else {
-        // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them
+        // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them (weights kept as
+        // coefficients: the same without the encoder, only their transforms)
         const size_t group_bytes = (size_t)n_terms * nmp * N * 8;
         const size_t fit = ctx->encode_scratch_bytes / group_bytes;
         const u32 groups = fit < 1 ? 1u : fit > (size_t)n_pj ? n_pj : (u32)fit;
@@ -965,7 +1011,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
         for (u32 pj0 = 0; pj0 < n_pj; pj0 += groups) {
             const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
             const TileLayout cl = mac_tile_layout(ctx->ring, cnt, n_terms, nmp);
-            TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p, cl, pj0));
+            TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p, cl, pj0, pt_weights));
             CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, cl, X, mac_out + (size_t)pj0 * xw, cnt, n_terms, false,
                           ctx->device_error, ctx->stream));
         }
@@ -1220,6 +1266,12 @@ extern "C" int bf_set_encode_scratch(bf_ctx* ctx, uint64_t bytes) {
     return BF_OK;
 }
 
+extern "C" int bf_set_coefficient_cache(bf_ctx* ctx, int bits) {
+    if (!ctx || (bits != 0 && bits != 32 && bits != 64)) return BF_ERR_INVALID_ARG;
+    ctx->coef_cache_bits = (u32)bits;
+    return BF_OK;
+}
+
 extern "C" int bf_set_compact_cache(bf_ctx* ctx, int on) {
     if (!ctx) return BF_ERR_INVALID_ARG;
     ctx->ring.compact_cache = on != 0;     // weights encoded from now on (and the fallback path's scratch) use it
@@ -1418,6 +1470,28 @@ extern "C" int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, u
     const size_t d = (((size_t)j * w->n_out + p) * w->n_in + q) * ctx->plan.bsgs_b + k;
     PolyBatch B;
     memset(&B, 0, sizeof(B));
+    if (w->coef) {      // coefficient form: reduce the stored integers per prime (through a transform and back)
+        const void* src = (const i64*)w->coef + d * N;
+        if (w->coef_bits == 32) {
+            TRY(ensure(ctx, ctx->coef, (size_t)N * sizeof(i64)));
+            CK(launch_widen_i32(ctx->ring, (const int*)w->coef + d * N, (i64*)ctx->coef.p, N, ctx->stream));
+            src = ctx->coef.p;
+        }
+        B.src = src;
+        B.dst = out;
+        B.src_so = 0;
+        B.src_sm = 0;
+        B.dst_so = (long long)r * N;
+        B.dst_sm = N;
+        B.n_m = r;
+        B.mod_step = 1;
+        CK(ntt_forward(ctx->ring, B, 1, LOAD_I64, ctx->stream));
+        B.src = out;
+        B.src_so = (long long)r * N;
+        B.src_sm = N;
+        CK(ntt_inverse(ctx->ring, B, 1, ctx->stream));
+        return BF_OK;
+    }
     B.src = out;                                 // unused: the first pass reads the tiles
     B.dst = out;
     B.src_so = B.dst_so = (long long)r * N;

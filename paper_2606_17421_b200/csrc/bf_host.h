@@ -110,6 +110,11 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
                            const u64* invs, const u64* qlmod, cudaStream_t stream);
 
+// 32-bit <-> 64-bit signed coefficients (the coefficient form of cached weights); narrowing sets *overflow_flag when a
+// value does not fit
+cudaError_t launch_widen_i32(const RingHost& ring, const int* src, i64* dst, size_t count, cudaStream_t stream);
+cudaError_t launch_narrow_i64(const RingHost& ring, const i64* src, int* dst, size_t count, int* overflow_flag,
+                              cudaStream_t stream);
 cudaError_t launch_imad_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream);   // 64 mad.wide per iteration and thread
 cudaError_t launch_fma64_probe(u64* sink, u32 blocks, u32 iters, cudaStream_t stream);  // 64 fma.rn.f64 per iteration and thread
 

@@ -784,6 +784,36 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
 }
 
 // ------------------------------------------------------------------------------------------------
+// Width changes of the rounded integer coefficients (the coefficient form of cached weights).
+__global__ void __launch_bounds__(256) widen_i32_kernel(const int* __restrict__ src, i64* __restrict__ dst, size_t count) {
+    grid_dependency_enter();
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = (i64)src[i];
+}
+__global__ void __launch_bounds__(256) narrow_i64_kernel(const i64* __restrict__ src, int* __restrict__ dst, size_t count,
+                                                         int* __restrict__ overflow) {
+    grid_dependency_enter();
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
+        const i64 v = src[i];
+        if (v != (i64)(int)v) atomicExch(overflow, 1);
+        dst[i] = (int)v;
+    }
+}
+cudaError_t launch_widen_i32(const RingHost& ring, const int* src, i64* dst, size_t count, cudaStream_t stream) {
+    if (!count) return cudaSuccess;
+    ProfScope prof(ring.prof, CAT_POINTWISE, stream);
+    const u32 blocks = (u32)((count + 1023) / 1024 < 148 * 16 ? (count + 1023) / 1024 : 148 * 16);
+    return launch_dependent(ring, widen_i32_kernel, dim3(blocks), dim3(256), 0, stream, src, dst, count);
+}
+cudaError_t launch_narrow_i64(const RingHost& ring, const i64* src, int* dst, size_t count, int* overflow_flag,
+                              cudaStream_t stream) {
+    if (!count) return cudaSuccess;
+    ProfScope prof(ring.prof, CAT_POINTWISE, stream);
+    const u32 blocks = (u32)((count + 1023) / 1024 < 148 * 16 ? (count + 1023) / 1024 : 148 * 16);
+    return launch_dependent(ring, narrow_i64_kernel, dim3(blocks), dim3(256), 0, stream, src, dst, count, overflow_flag);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Throughput probe for the 32x32+64-bit integer multiply-add the modular arithmetic is made of:
 // every thread runs 8 independent mad.wide.u32 chains.  Gives the measured denominator for the
 // integer-bound kernels (NTT, key switch).

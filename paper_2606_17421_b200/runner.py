@@ -29,7 +29,7 @@ class WorkloadRunner:
     def __init__(self, name: str, seed: int = 0, device: str = "cuda:0", cache: bool = True,
                  cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None,
                  fuse_shared_inputs: bool = True, fold_in_ciphertext: bool = False, compact_cache: bool = False,
-                 pack: str | None = None, moddown: str | None = None, hoist: str | None = None):
+                 pack: str | None = None, moddown: str | None = None, hoist: str | None = None, coef_bits: int = 0):
         self.w = wl.WORKLOADS[name]
         ps = wl.PARAM_SETS[self.w.params]
         self.N, self.primes, self.P, self.scale = ps["N"], list(ps["primes"]), ps["special"], ps["scale"]
@@ -55,6 +55,9 @@ class WorkloadRunner:
         if compact_cache:           # narrower resident words per prime: 68 % of the cache for the 50 + 6 x 40-bit chain
             bf.bf_set_compact_cache(self.ctx, True)
         self.compact_cache = compact_cache
+        if coef_bits:               # weights resident as rounded 64- or 32-bit coefficients, transformed on every call
+            bf.bf_set_coefficient_cache(self.ctx, coef_bits)
+        self.coef_bits = coef_bits
         # resident bytes per encoded coefficient over all primes (8 each, or 4 / 5 / 8 by prime size when compact)
         self.word_bytes = sum((4 if q < 2 ** 32 else 5 if q < 2 ** 40 else 8) if compact_cache else 8 for q in self.primes)
         if self.plan.hoist == "double":     # the residue modulo the special prime is kept too, always in 8 bytes
@@ -104,7 +107,9 @@ class WorkloadRunner:
                 ct_low = torch.empty((n_out, 2, self.r - 1, self.N), dtype=torch.int64, device=self.device)
                 self.layers.append(dict(layer=L, rep=rep, n_in=n_in, n_out=n_out, W=W, handle=handle,
                                         ct_in=ct_in, ct_out=ct_out, ct_low=ct_low,
-                                        pt_bytes=n_in * n_out * (D // self.plan.tau) * self.N * self.word_bytes))
+                                        pt_bytes=n_in * n_out * (D // self.plan.tau) * self.N * self.word_bytes,
+                                        resident_bytes=n_in * n_out * (D // self.plan.tau) * self.N *
+                                        (coef_bits // 8 if coef_bits else self.word_bytes) if handle else 0))
         torch.cuda.synchronize()
 
     # ------------------------------------------------------------------ one decode token
@@ -138,11 +143,19 @@ class WorkloadRunner:
     def cached_pt_bytes(self):
         return sum(e["pt_bytes"] for e in self.layers if e["handle"])
 
+    def resident_bytes(self):
+        """Bytes the cached weights occupy (differs from the streamed bytes when they are kept as coefficients)."""
+        return sum(e["resident_bytes"] for e in self.layers)
+
     def total_pt_bytes(self):
         return sum(e["pt_bytes"] for e in self.layers)
 
     def n_fallback_layers(self):
         return sum(1 for e in self.layers if not e["handle"])
+
+    def transforms_weights_per_call(self, e) -> bool:
+        """The call of layer entry e transforms its weights (encoded on the fly, or kept as coefficients)."""
+        return not e["handle"] or bool(self.coef_bits)
 
     def close(self):
         bf.bf_ctx_destroy(self.ctx)

@@ -9,6 +9,10 @@ from tests.helpers import GpuSide, custom_params, oracle_params
 
 pytestmark = pytest.mark.gpu
 
+# the plan variant the benchmark's headline runs: two row blocks per plaintext, one division by P per output
+# ciphertext, baby-step rotations kept in the extended basis
+BEST = dict(pack="complex", moddown="per_output", hoist="double")
+
 
 # ------------------------------------------------------------------ transforms
 
@@ -306,6 +310,65 @@ def test_linear_double_hoisting_with_the_papers_own_parameter_set():
     run_case(par, ckks.Plan(256, 16, 4, 4, hoist="double"), 300, 520, 4, 1e-2, "paper_n13_dh", tight=1e-3)
 
 
+@pytest.mark.parametrize("bits", [64, 32])
+@pytest.mark.parametrize("modes", [{}, BEST], ids=["plain", "best"])
+def test_weights_kept_as_coefficients_give_the_same_ciphertexts(bits, modes):
+    # the coefficient form of the cache: rounded integer coefficients are resident, reduced per prime and
+    # transformed on every call; residues must not change, and the handle is 1/r (1/2r) of the usual size
+    par = oracle_params("n12")
+    plan = ckks.Plan(64, 4, 4, 4, **modes)
+    d_out, d_in = 150, 130
+    s = ckks.keygen(par, 61)
+    keys = ckks.make_rotation_keys(par, s, plan, 61)
+    W = wl.gen_weights(61, "coef", d_out, d_in)
+    if bits == 32:      # on this small ring the slot vectors repeat eight times, which concentrates the coefficients:
+        W = W / 32      # keep them inside 32 bits (the full-size rings have no replication and fit as they are)
+    cts = ckks.encrypt_vector(par, plan, s, wl.gen_activation(61, "coef", d_in), 61)
+    expect = ckks.linear(par, plan, cts, W, keys)
+    n_out, n_in = plan.n_out(d_out), 3
+    g = GpuSide(par, plan)
+    try:
+        g.load_keys(keys)
+        Wd = g.to_dev(W)
+        full_bytes = g.bf.bf_weights_bytes(g.ctx, d_out, d_in)
+        g.bf.bf_set_coefficient_cache(g.ctx, bits)
+        w = g.bf.bf_encode_weights(g.ctx, Wd, d_out, d_in)
+        used = g.bf.bf_cache_bytes_used(g.ctx)
+        assert used == n_in * n_out * plan.M * par.N * bits // 8 == g.bf.bf_weights_bytes(g.ctx, d_out, d_in)
+        assert used * par.r * (64 // bits) <= full_bytes
+        ct_in = g.to_dev(np.stack(cts))
+        ct_out = g.empty_u64(n_out, 2, par.r, par.N)
+        for call in range(4):                       # direct, captured, replayed
+            ct_out.zero_()
+            g.bf.bf_linear(g.ctx, ct_in, n_in, w, None, d_out, d_in, ct_out, n_out)
+            got = g.to_host_u64(ct_out)
+            for p in range(n_out):
+                assert np.array_equal(got[p], expect[p]), (call, p)
+        out = g.empty_u64(par.r, par.N)
+        for (p, q, j, k) in ((0, 0, 0, 0), (n_out - 1, 2, 3, 1), (0, 1, 2, 3)):
+            z = ckks.plain_slots(W, plan, p, q, j, k, par.n)
+            g.bf.bf_weights_export(g.ctx, w, p, q, j, k, out)
+            assert np.array_equal(g.to_host_u64(out), ckks.to_residues(ckks.encode_coeffs(z, par.N, par.scale), par.primes))
+        # a transform-domain handle made afterwards works beside it
+        g.bf.bf_set_coefficient_cache(g.ctx, 0)
+        w2 = g.bf.bf_encode_weights(g.ctx, Wd, d_out, d_in)
+        got = g.to_host_u64(g.linear(cts, W, d_out, d_in, weights=w2))
+        assert all(np.array_equal(got[p], expect[p]) for p in range(n_out))
+        g.bf.bf_weights_free(g.ctx, w)
+        g.bf.bf_weights_free(g.ctx, w2)
+        assert g.bf.bf_cache_bytes_used(g.ctx) == 0
+        if bits == 32:      # coefficients beyond 32 bits are refused at encoding time
+            g.bf.bf_set_coefficient_cache(g.ctx, 32)
+            with pytest.raises(g.bf.BifrostError) as ei:
+                g.bf.bf_encode_weights(g.ctx, g.to_dev(W * 1024), d_out, d_in)
+            assert ei.value.code == g.bf.BF_ERR_RANGE
+            assert g.bf.bf_cache_bytes_used(g.ctx) == 0
+        with pytest.raises(g.bf.BifrostError):
+            g.bf.bf_set_coefficient_cache(g.ctx, 16)
+    finally:
+        g.close()
+
+
 def test_per_output_division_refuses_more_giant_steps_than_it_can_sum():
     from paper_2606_17421_b200 import bifrost as bf
     ps = wl.PARAM_SETS["n12"]
@@ -345,7 +408,8 @@ def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=()):
             if d_in not in inputs:
                 x = wl.gen_activation(seed, f"x{d_in}", d_in)
                 cts = ckks.encrypt_vector(par, plan, s, x, seed)
-                inputs[d_in] = (x, cts, [ckks.baby_rotations(par, plan, ct, keys) for ct in cts])
+                rot_fn = ckks.baby_rotations_ext if plan.hoist == "double" else ckks.baby_rotations
+                inputs[d_in] = (x, cts, [rot_fn(par, plan, ct, keys) for ct in cts])
             x, cts, X = inputs[d_in]
             n_in, n_out = len(cts), plan.n_out(d_out)
             blocks = list(blocks_of(name, n_out))
@@ -376,38 +440,49 @@ def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=()):
         g.close()
 
 
-def test_gpt2_step_one_whole_layer_every_block():
-    # config 2: one transformer layer of the GPT-2 decode step, all four calls, every output block
-    # (qkv 3 blocks, out_proj 1, ffn_up 3, ffn_down 1 with three input ciphertexts)
+@pytest.mark.parametrize("modes", [{}, BEST], ids=["plain", "best"])
+def test_gpt2_step_one_whole_layer_every_block(modes):
+    # config 2: one transformer layer of the GPT-2 decode step, all four calls, every output ciphertext
+    # (qkv 3 row blocks, out_proj 1, ffn_up 3, ffn_down 1 with three input ciphertexts)
     w = wl.WORKLOADS["gpt2_step"]
     par = oracle_params(w.params)
-    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, **modes)
     check_blocks(par, plan, w.layers, lambda name, n_out: range(n_out), 11)
 
 
-def test_qwen3_step_the_calls_of_one_layer():
+@pytest.mark.parametrize("modes", [{}, BEST], ids=["plain", "best"])
+def test_qwen3_step_the_calls_of_one_layer(modes):
     # config 3: the four calls the runner issues per layer.  q+k+v (1024 -> 4096) in full; o (2048 -> 1024, two
     # input ciphertexts) in full, also on the fly; gate+up (1024 -> 6144): its 18 giant rotations run as two
     # chains of 9 -- blocks 0 and 2 lie in the first chain for j = 1, 2 and in the second for j = 3, blocks 3
-    # and 5 in the first for j = 1 and in the second for j = 2, 3; down (3072 -> 1024) in full
+    # and 5 in the first for j = 1 and in the second for j = 2, 3; down (3072 -> 1024) in full.  With two row
+    # blocks per ciphertext: every output ciphertext of every call
     w = wl.WORKLOADS["qwen3_step"]
     par = oracle_params(w.params)
-    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, **modes)
     pick = {"q+k+v": [0, 1, 2, 3], "o": [0], "gate+up": [0, 2, 3, 5], "down": [0]}
-    check_blocks(par, plan, w.layers, lambda name, n_out: pick[name], 12, on_the_fly=("o",))
+    blocks_of = (lambda name, n_out: range(n_out)) if modes else (lambda name, n_out: pick[name])
+    check_blocks(par, plan, w.layers, blocks_of, 12, on_the_fly=("o",))
 
 
-def test_llama3_layer_the_calls_the_benchmark_times():
+@pytest.mark.parametrize("modes", [{}, BEST], ids=["plain", "best"])
+def test_llama3_layer_the_calls_the_benchmark_times(modes):
     # config 4 at N = 2^16: q+k+v (4096 -> 6144): first block, the k block and the v block; o (4096 -> 4096):
     # first and last; gate+up (4096 -> 28672): 84 giant rotations in four launches of 22, 22, 22 and 18 --
     # rotation (j - 1) * 28 + p of block p, so block 0 meets launches 1, 2, 3; block 14 (first of up) 1, 2, 4;
     # blocks 21 and 22 the end of launch 1 and the start of launch 2; block 27 launches 2, 3 and the very last
     # rotation; down (14336 -> 4096): 14 input ciphertexts whose 98 baby rotations share two hoisted ModUps
-    # (9 + 5 ciphertexts), every output block, and once more with the weights encoded on the fly
+    # (9 + 5 ciphertexts), every output block, and once more with the weights encoded on the fly.
+    # With two row blocks per ciphertext gate+up has 14 outputs and 42 giant rotations in launches of 22 and 20:
+    # rotation (j - 1) * 14 + p, so ciphertext 0 meets launch 1 twice and launch 2, ciphertexts 7 and 8 the end of
+    # launch 1 and the start of launch 2, ciphertext 13 the very last rotation
     w = wl.WORKLOADS["llama3_layer"]
     par = oracle_params(w.params)
-    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g)
-    pick = {"q+k+v": [0, 4, 5], "o": [0, 3], "gate+up": [0, 14, 21, 22, 27], "down": [0, 1, 2, 3]}
+    plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, **modes)
+    if modes:
+        pick = {"q+k+v": [0, 2], "o": [0, 1], "gate+up": [0, 7, 8, 13], "down": [0, 1]}
+    else:
+        pick = {"q+k+v": [0, 4, 5], "o": [0, 3], "gate+up": [0, 14, 21, 22, 27], "down": [0, 1, 2, 3]}
     check_blocks(par, plan, w.layers, lambda name, n_out: pick[name], 13, on_the_fly=("down",))
 
 
