@@ -890,7 +890,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     const int lanes_giant = (lanes > 1 && n_giant >= 6 && n_giant * ring_weight <= 20) ? lanes : 1;
     const int lanes_baby = (lanes > 1 && in_batch * (b - 1) * ring_weight <= 24) ? lanes : 1;
     const u32 baby_rots = in_batch * (b - 1);
-    const u32 baby_per_lane = cdiv(baby_rots > 0 ? baby_rots : 1, (u32)lanes);
+    const u32 baby_per_lane = b > 1 ? cdiv(b - 1, (u32)lanes) * in_batch : 1u;     // (a lane takes whole keys)
     u32 giant_per_lane = cdiv(n_giant > 0 ? n_giant : 1, (u32)lanes);     // rotations a lane holds at once
     // (rounded down: a single chain uses the buffers of all lanes, giant_per_lane * lanes rotations per launch,
     // and a launch takes at most MAX_ROT_BATCH)
@@ -967,7 +967,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             // another, so that an inner-product block loads the key once for all of them), dealt out to the lanes
             // in contiguous runs
             const u32 n_rot = qn * (b - 1);
-            const u32 per = cdiv(n_rot, (u32)lanes_baby);
+            const u32 per = cdiv(b - 1, (u32)lanes_baby) * qn;           // whole keys per lane: no key is streamed by two lanes
             const int used = (int)cdiv(n_rot, per);
             TRY(fork_lanes(ctx, used));
             for (int c = 0; c < used; ++c) {
@@ -999,7 +999,13 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     const u32 n_terms = n_in * b, n_pj = n_out * g;
     u64* mac_out = dh ? (u64*)ctx->Aext.p : A;
     if (pt_weights && pt_weights->pt) {
-        CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, mac_out, n_pj, n_terms, true, ctx->device_error, ctx->stream));
+        // double hoisting: the launch for the special prime (one eighth of the words, on whole-word arithmetic) runs
+        // beside the launch for the ciphertext primes
+        const bool beside = dh && lanes > 1;
+        if (beside) TRY(fork_lanes(ctx, 2));
+        CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, mac_out, n_pj, n_terms, true, ctx->device_error, ctx->stream,
+                      beside ? ctx->side[0] : nullptr));
+        if (beside) TRY(join_lanes(ctx, 2));
     } else {
         // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them (weights kept as
         // coefficients: the same without the encoder, only their transforms)

@@ -105,8 +105,11 @@ TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms, u32 n_pr
 size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t);           // bytes that layout occupies
 // x: [n_terms][2][lay.n_primes][N], a: [n_pj][2][lay.n_primes][N]; every prime of the layout is processed (the special
 // prime, when present, by a launch of its own on whole words)
+// special_stream non-null: the launch for the special prime goes there (the caller has ordered that stream after
+// everything the launch reads and joins it afterwards), beside the launch for the ciphertext primes on `stream`
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
-                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream);
+                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream,
+                       cudaStream_t special_stream = nullptr);
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
                            const u64* invs, const u64* qlmod, cudaStream_t stream);
 

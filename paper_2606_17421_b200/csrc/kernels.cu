@@ -511,7 +511,7 @@ static cudaError_t launch_mac_primes(const RingHost& ring, const u64* pt, const 
 }
 
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
-                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream) {
+                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream, cudaStream_t special_stream) {
     if (n_pj == 0) return cudaSuccess;
     if (lay.n_pj != n_pj || lay.n_terms != n_terms) return cudaErrorInvalidValue;
     const u32 r = ring.dev.r;
@@ -519,7 +519,8 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
     cudaError_t e = launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, 0, r, kara, error_flag, stream);
     if (e != cudaSuccess || lay.n_primes <= r) return e;
     // double hoisting: the residues modulo the 60-bit special prime, on whole words
-    return launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, r, lay.n_primes - r, false, error_flag, stream);
+    return launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, r, lay.n_primes - r, false, error_flag,
+                             special_stream ? special_stream : stream);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -588,12 +589,23 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
-    mbar_wait(kbar, 0, error_flag);
     const u64 q = R.q[m];
     const u32 qneg32 = (u32)R.qneg[m];
+    const size_t term_words = (size_t)2 * nb * N;
+    // double hoisting: what the last step of a rotation reads from global memory (where the coefficient goes under the
+    // rotation, and P*c0) is requested before the wait for the operands, so that it is not a second round trip
+    u32 dest = 0;
+    u64 pc0 = 0;
+    if (xext) {
+        dest = __ldg(&pinv[(size_t)rb.key[first] * N + n0 + tid]);          // (the same for every rotation of the run)
+        pc0 = xext[(size_t)rb.c0[first] * term_words + (size_t)m * N + n0 + tid];
+    }
+    mbar_wait(kbar, 0, error_flag);
     for (u32 it = 0; it < cnt; ++it) {
         const u32 rot = first + it;
         const u64* sdc = sd + (size_t)(it & 1) * r * KI_TILE;
+        u64 pc0_next = 0;
+        if (xext && it + 1 < cnt) pc0_next = xext[(size_t)rb.c0[rot + 1] * term_words + (size_t)m * N + n0 + tid];
         mbar_wait(&dbar[it & 1], (it >> 1) & 1, error_flag);
         u64 v0, v1;
         if (m < r && small_ok) {
@@ -622,12 +634,11 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
         if (xext) {
             // double hoisting: no division by P; the rotated input in the extended basis is (P*c0 + u0, u1) moved
             // through the rotation's permutation; P*c0 (zero modulo P) was stored as the un-rotated term
-            const size_t term_words = (size_t)2 * nb * N;
-            const u32 n = n0 + tid;
-            v0 = add_mod(v0, xext[(size_t)rb.c0[rot] * term_words + (size_t)m * N + n], q);
-            u64* xp = xext + (size_t)rb.out[rot] * term_words + (size_t)m * N + __ldg(&pinv[(size_t)rb.key[rot] * N + n]);
+            v0 = add_mod(v0, pc0, q);
+            u64* xp = xext + (size_t)rb.out[rot] * term_words + (size_t)m * N + dest;
             xp[0] = v0;
             xp[(size_t)nb * N] = v1;
+            pc0 = pc0_next;
         } else {
             u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
             up[0] = v0;
