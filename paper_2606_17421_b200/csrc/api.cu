@@ -889,7 +889,6 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     const u32 ring_weight = N > (1u << 15) ? N >> 15 : 1u;
     const int lanes_giant = (lanes > 1 && n_giant >= 6 && n_giant * ring_weight <= 20) ? lanes : 1;
     const int lanes_baby = (lanes > 1 && in_batch * (b - 1) * ring_weight <= 24) ? lanes : 1;
-    const u32 baby_rots = in_batch * (b - 1);
     const u32 baby_per_lane = b > 1 ? cdiv(b - 1, (u32)lanes) * in_batch : 1u;     // (a lane takes whole keys)
     u32 giant_per_lane = cdiv(n_giant > 0 ? n_giant : 1, (u32)lanes);     // rotations a lane holds at once
     // (rounded down: a single chain uses the buffers of all lanes, giant_per_lane * lanes rotations per launch,
@@ -956,8 +955,11 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     B.mod_wrap = r;
     B.mod0 = 0;
     B.mod_step = 1;
+    if (dh) {                   // the transform's last store also writes P * NTT(ct_q) as term q*b of X
+        B.lift_ptr = X;
+        B.lift_so = (long long)b * (long long)xw;
+    }
     CK(ntt_forward(ctx->ring, B, n_in, LOAD_PLAIN, ctx->stream));
-    if (dh) CK(launch_lift_times_p(ctx->ring, X0, (long long)ctw, X, (long long)b * xw, n_in, ctx->stream));
     if (b > 1) {
         for (u32 q0 = 0; q0 < n_in; q0 += in_batch) {
             const u32 qn = (n_in - q0 < in_batch) ? n_in - q0 : in_batch;

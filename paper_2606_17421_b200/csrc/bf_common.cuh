@@ -343,6 +343,9 @@ struct PolyBatch {
                                   //   product ends in a Montgomery reduction)
     u32 split_bits;               // L > 0: the NTT-domain side of the transform is stored as two L-bit-aligned
                                   // limbs per word, (v >> L) << 32 | (v & (2^L - 1)); forward writes, inverse reads it
+    u64* lift_ptr;                // forward only, non-null (double hoisting): polynomial (o, m = comp * mod_wrap + i) is also
+    long long lift_so;            //   stored times P mod q_i at lift_ptr + o*lift_so + (comp*(r+1) + i)*N, and zeros as the
+                                  //   residue modulo P: the un-rotated input lifted to the extended basis
     u64* dtile_ptr;               // forward only, non-null: the final result goes there instead of dst, tile-major in tiles
     u32 dtile_div;                //   of KS_TILE coefficients (see ks_tile_index); with `scatter` the store is permuted
 };

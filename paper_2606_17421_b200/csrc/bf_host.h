@@ -95,10 +95,6 @@ cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* 
 // xext[rb.c0[rot]][0][m][n] : 0), terms of [2][r+1][N] words (term rb.c0[rot] holds P times the un-rotated input).
 cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
                                      int* error_flag, cudaStream_t stream, u64* xext = nullptr, const u32* pinv = nullptr);
-// dst[t][comp][i][n] = src[t][comp][i][n] * P mod q_i (i < r), dst[t][comp][r][n] = 0: the un-rotated inputs lifted to
-// the extended basis; src ciphertexts of [2][r][N] at src_stride, dst terms of [2][r+1][N] at dst_stride (words)
-cudaError_t launch_lift_times_p(const RingHost& ring, const u64* src, long long src_stride, u64* dst, long long dst_stride,
-                                u32 n_ct, cudaStream_t stream);
 u32 mac_split_bits(const RingHost& ring);   // limb width of the cached plaintext format (0 = whole words)
 // layout of n_pj groups of n_terms diagonals held in n_primes primes (0 = the r ciphertext primes)
 TileLayout mac_tile_layout(const RingHost& ring, u32 n_pj, u32 n_terms, u32 n_primes = 0);

@@ -647,31 +647,6 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
     }
 }
 
-// The un-rotated inputs lifted to the extended basis for double hoisting: times P modulo every ciphertext prime,
-// zero modulo P.  grid: x = coefficients / 256, y = ciphertext, z = component * (r + 1) + prime.
-__global__ void __launch_bounds__(256) lift_times_p_kernel(const RingDev R, const u64* __restrict__ src, long long src_stride,
-                                                           u64* __restrict__ dst, long long dst_stride) {
-    grid_dependency_enter();
-    const u32 N = R.N, r = R.r, nb = r + 1;
-    const u32 n = blockIdx.x * blockDim.x + threadIdx.x;
-    const u32 ct = blockIdx.y, comp = blockIdx.z / nb, m = blockIdx.z % nb;
-    u64 v = 0;
-    if (m < r) {
-        u64 hi = 0, lo = 0;
-        mac128(hi, lo, src[(size_t)ct * src_stride + ((size_t)comp * r + m) * N + n], R.pmod[m]);
-        v = reduce128(hi, lo, R.q[m], R.mu[m], R.c64[m], R.c64s[m]);
-    }
-    dst[(size_t)ct * dst_stride + ((size_t)comp * nb + m) * N + n] = v;
-}
-
-cudaError_t launch_lift_times_p(const RingHost& ring, const u64* src, long long src_stride, u64* dst, long long dst_stride,
-                                u32 n_ct, cudaStream_t stream) {
-    if (n_ct == 0) return cudaSuccess;
-    ProfScope prof(ring.prof, CAT_POINTWISE, stream);
-    dim3 grid(ring.dev.N / 256, n_ct, 2 * (ring.dev.r + 1));
-    return launch_dependent(ring, lift_times_p_kernel, grid, dim3(256), 0, stream, ring.dev, src, src_stride, dst, dst_stride);
-}
-
 cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, const u64* dig, const u64* keys, u64* u,
                                      int* error_flag, cudaStream_t stream, u64* xext, const u32* pinv) {
     if (rb.n == 0) return cudaSuccess;

@@ -660,6 +660,24 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 }
                 continue;
             }
+            if (B.lift_ptr) {   // P times the value, into the extended-basis copy of the un-rotated inputs
+                const u32 comp = B.mod_wrap ? m / B.mod_wrap : 0u, nbp = R.r + 1;
+                u64* xp = B.lift_ptr + (size_t)o * B.lift_so + ((size_t)comp * nbp + mod) * R.N + (size_t)chunk * LEN + 4 * s;
+                u64 p4[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    u64 hi = 0, lo = 0;
+                    mac128(hi, lo, v4[i], R.pmod[mod]);
+                    p4[i] = reduce128(hi, lo, q, R.mu[mod], R.c64[mod], R.c64s[mod]);
+                }
+                ((ulonglong2*)xp)[0] = make_ulonglong2(p4[0], p4[1]);
+                ((ulonglong2*)xp)[1] = make_ulonglong2(p4[2], p4[3]);
+                if (mod == 0) {     // the residue modulo P of P * ct is zero
+                    u64* zp = B.lift_ptr + (size_t)o * B.lift_so + ((size_t)comp * nbp + R.r) * R.N + (size_t)chunk * LEN + 4 * s;
+                    ((ulonglong2*)zp)[0] = make_ulonglong2(0, 0);
+                    ((ulonglong2*)zp)[1] = make_ulonglong2(0, 0);
+                }
+            }
             if (B.split_bits) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) v4[i] = limb_split(v4[i], B.split_bits);
