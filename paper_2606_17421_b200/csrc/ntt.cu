@@ -514,7 +514,7 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
 // (reads the batch source: plain residues, tiled/limb-split plaintexts, or a sum of arrays).
 // TILED: the transform-domain side of the batch lives in the tile-major plaintext cache (B.tile_ptr).
 // EPI: 0 = none; 1 = division by P per rotation (scatter through the rotation's permutation); 2 = per output
-// (sum over the output's giant rotations, gathered through their permutations; see ModDownEpilogue).
+// (sum over the output's giant rotations, gathered through their permutations); 3 = plain (see ModDownEpilogue).
 template <bool FWD, int EPI, bool FP, bool TILED>
 __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, u32 o, u32 m, u32 mod,
                                             u32 chunk, int lane, const RotBatch& rb, const ModDownEpilogue& epi) {
@@ -574,21 +574,24 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                     }
                 }
             }
+            if (EPI == 3) {         // plain division: only the inner sum's residue is needed
+                const u64* up = epi.u + ((size_t)o * (R.r + 1) + mod) * R.N + (size_t)chunk * LEN + 4 * s;
+                const ulonglong2 u0 = *(const ulonglong2*)up, u1 = *(const ulonglong2*)(up + 2);
+                uu[0] = u0.x; uu[1] = u0.y; uu[2] = u1.x; uu[3] = u1.y;
+            }
             if (EPI == 1) {
                 const u32 rot = o >> 1, comp = o & 1, ip = mod, nb = R.r + 1;
                 const size_t n = (size_t)chunk * LEN + 4 * s;
                 const u64* up = epi.u + ((size_t)o * nb + ip) * R.N + n;
                 const ulonglong2 u0 = *(const ulonglong2*)up, u1 = *(const ulonglong2*)(up + 2);
                 uu[0] = u0.x; uu[1] = u0.y; uu[2] = u1.x; uu[3] = u1.y;
-                if (comp == 0 && !epi.plain) {
+                if (comp == 0) {
                     const u64* cp = epi.c0_base + (size_t)rb.c0[rot] * epi.c0_stride + (size_t)ip * R.N + n;
                     const ulonglong2 c0 = *(const ulonglong2*)cp, c1 = *(const ulonglong2*)(cp + 2);
                     cc[0] = c0.x; cc[1] = c0.y; cc[2] = c1.x; cc[3] = c1.y;
                 }
-                if (!epi.plain) {
-                    const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
-                    pp[0] = pv.x; pp[1] = pv.y; pp[2] = pv.z; pp[3] = pv.w;
-                }
+                const uint4 pv = *(const uint4*)(epi.pinv + (size_t)rb.key[rot] * R.N + n);
+                pp[0] = pv.x; pp[1] = pv.y; pp[2] = pv.z; pp[3] = pv.w;
             }
             set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, qd);
             u64 v4[4];
@@ -619,7 +622,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 ((ulonglong2*)op)[1] = make_ulonglong2(v4[2], v4[3]);
                 continue;
             }
-            if (EPI == 1 && epi.plain) {
+            if (EPI == 3) {
                 u64* op = epi.out_base + (size_t)o * epi.out_stride + (size_t)mod * R.N + (size_t)chunk * LEN + 4 * s;
 #pragma unroll
                 for (int t = 0; t < 4; ++t) v4[t] = mul_shoup(sub_mod(uu[t], v4[t], q), R.pinv[mod], R.pinvs[mod], q);
@@ -908,7 +911,10 @@ static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n
     const u32 chunks = 1u << ring.geom.log_r;
     const u32 cpb = (u32)ring.geom.contig_lanes;
     dim3 grid(chunks / cpb, n_polys);
-    if (epi && epi->n_sum) {
+    if (FWD && epi && epi->plain) {
+        launch_dependent(ring, ntt_contig<FWD, 3, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
+                         *epi);
+    } else if (epi && epi->n_sum) {
         launch_dependent(ring, ntt_contig<FWD, 2, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
                          *epi);
     } else if (FWD && epi) {
