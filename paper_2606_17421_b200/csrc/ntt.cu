@@ -561,16 +561,35 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
             if (EPI == 2) {
                 const u32 pp_out = o >> 1, comp = o & 1, ip = mod, nb = R.r + 1;
                 const size_t n = (size_t)chunk * LEN + 4 * s;
-                for (u32 jj = 0; jj < epi.n_sum; ++jj) {
-                    const uint4 pv = *(const uint4*)(epi.perm + (size_t)rb.key[jj] * R.N + n);
-                    const size_t rot = (size_t)jj * epi.n_out + pp_out;
-                    const u64* up = epi.u + ((rot * 2 + comp) * nb + ip) * R.N;
-                    uu[0] = add_mod(uu[0], __ldg(up + pv.x), q); uu[1] = add_mod(uu[1], __ldg(up + pv.y), q);
-                    uu[2] = add_mod(uu[2], __ldg(up + pv.z), q); uu[3] = add_mod(uu[3], __ldg(up + pv.w), q);
-                    if (comp == 0) {
-                        const u64* cp = epi.c0_base + rot * epi.c0_stride + (size_t)ip * R.N;
-                        cc[0] = add_mod(cc[0], __ldg(cp + pv.x), q); cc[1] = add_mod(cc[1], __ldg(cp + pv.y), q);
-                        cc[2] = add_mod(cc[2], __ldg(cp + pv.z), q); cc[3] = add_mod(cc[3], __ldg(cp + pv.w), q);
+                // three rotations at a time: their permutation entries are requested together, then all the words they
+                // point at, so that a group costs two round trips instead of two per rotation
+                for (u32 j0 = 0; j0 < epi.n_sum; j0 += 3) {
+                    uint4 pv[3];
+                    u64 uv[3][4], cv[3][4];
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t)
+                        if (j0 + t < epi.n_sum) pv[t] = *(const uint4*)(epi.perm + (size_t)rb.key[j0 + t] * R.N + n);
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t) {
+                        if (j0 + t >= epi.n_sum) continue;
+                        const size_t rot = (size_t)(j0 + t) * epi.n_out + pp_out;
+                        const u64* up = epi.u + ((rot * 2 + comp) * nb + ip) * R.N;
+                        uv[t][0] = __ldg(up + pv[t].x); uv[t][1] = __ldg(up + pv[t].y);
+                        uv[t][2] = __ldg(up + pv[t].z); uv[t][3] = __ldg(up + pv[t].w);
+                        if (comp == 0) {
+                            const u64* cp = epi.c0_base + rot * epi.c0_stride + (size_t)ip * R.N;
+                            cv[t][0] = __ldg(cp + pv[t].x); cv[t][1] = __ldg(cp + pv[t].y);
+                            cv[t][2] = __ldg(cp + pv[t].z); cv[t][3] = __ldg(cp + pv[t].w);
+                        }
+                    }
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t) {
+                        if (j0 + t >= epi.n_sum) continue;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            uu[w] = add_mod(uu[w], uv[t][w], q);
+                            if (comp == 0) cc[w] = add_mod(cc[w], cv[t][w], q);
+                        }
                     }
                 }
             }
@@ -720,11 +739,28 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 const u32 pp_out = o >> 1, comp = o & 1, nb = R.r + 1;
                 const size_t n = (size_t)chunk * LEN + 4 * s;
                 v4[0] = v4[1] = v4[2] = v4[3] = 0;
-                for (u32 jj = 0; jj < epi.n_sum; ++jj) {
-                    const uint4 pv = *(const uint4*)(epi.perm + (size_t)rb.key[jj] * R.N + n);
-                    const u64* up = epi.u + ((((size_t)jj * epi.n_out + pp_out) * 2 + comp) * nb + mod) * R.N;
-                    v4[0] = add_mod(v4[0], __ldg(up + pv.x), q); v4[1] = add_mod(v4[1], __ldg(up + pv.y), q);
-                    v4[2] = add_mod(v4[2], __ldg(up + pv.z), q); v4[3] = add_mod(v4[3], __ldg(up + pv.w), q);
+                // three rotations at a time: their permutation entries are requested together, then all the words they
+                // point at, so that a group costs two round trips instead of two per rotation (these launches are a few
+                // polynomials only: latency is all they cost)
+                for (u32 j0 = 0; j0 < epi.n_sum; j0 += 3) {
+                    uint4 pv[3];
+                    u64 uv[3][4];
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t)
+                        if (j0 + t < epi.n_sum) pv[t] = *(const uint4*)(epi.perm + (size_t)rb.key[j0 + t] * R.N + n);
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t) {
+                        if (j0 + t >= epi.n_sum) continue;
+                        const u64* up = epi.u + ((((size_t)(j0 + t) * epi.n_out + pp_out) * 2 + comp) * nb + mod) * R.N;
+                        uv[t][0] = __ldg(up + pv[t].x); uv[t][1] = __ldg(up + pv[t].y);
+                        uv[t][2] = __ldg(up + pv[t].z); uv[t][3] = __ldg(up + pv[t].w);
+                    }
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t) {
+                        if (j0 + t >= epi.n_sum) continue;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) v4[w] = add_mod(v4[w], uv[t][w], q);
+                    }
                 }
             } else if constexpr (TILED) {  // read back from the tile-major plaintext cache
                 const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
@@ -802,8 +838,10 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
     }
 }
 
+// (the per-output forms run on a few polynomials per launch and hold the operands of three rotations at once: they
+// trade resident blocks for registers)
 template <bool FWD, int EPI, bool TILED>
-__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, 8) ntt_contig(const RingDev R, const PolyBatch B,
+__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, EPI == 2 ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
     __shared__ __align__(128) u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
