@@ -534,10 +534,11 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 //
 // A block owns one (run of rotations that share a key, modulus, tile of 128 coefficients): the baby rotations
 // of several input ciphertexts by the same amount, or the giant rotations of several output blocks by the same
-// amount.  The key's 2r segments of the tile (1 KB each) are fetched once by asynchronous bulk copies and stay
-// in shared memory, so that the key stream crosses HBM (and L2) once per run instead of once per rotation; the
-// r digit segments of each rotation of the run follow through two buffers, the next rotation's copies in flight
-// while the current one is multiplied.  The keys are resident in Montgomery form (times 2^64 mod q), so the sum
+// amount.  Keys and digit sets are kept tile-major (see ks_tile_index): the key's 2r segments of the tile are one
+// contiguous block, fetched once by one asynchronous bulk copy, and stay in shared memory, so that the key stream
+// crosses HBM (and L2) once per run instead of once per rotation; the r digit segments of each rotation of the run
+// (one contiguous block as well) follow through two buffers, the next rotation's copy in flight while the current
+// one is multiplied.  The keys are resident in Montgomery form (times 2^64 mod q), so the sum
 // of the r products ends in the two-round 32-bit Montgomery reduction: r * max digit < 2^64 keeps it below
 // q * 2^64.  With double hoisting the block also finishes the rotated input (see launch_key_inner_product).
 // grid: x = run, y = tile, z = modulus of the extended basis.
