@@ -144,6 +144,8 @@ def parse_spec(spec: str):
             kw["hoist"] = "double"
         elif o in ("coeff64", "coeff32"):
             kw["coef_bits"] = int(o[5:])
+        elif o.startswith("lanes="):
+            kw["lanes"] = int(o[6:])
         else:
             raise ValueError(f"unknown workload option {o!r}")
     return name, kw

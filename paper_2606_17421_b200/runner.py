@@ -29,7 +29,8 @@ class WorkloadRunner:
     def __init__(self, name: str, seed: int = 0, device: str = "cuda:0", cache: bool = True,
                  cache_budget_bytes: int | None = None, stream: torch.cuda.Stream | None = None,
                  fuse_shared_inputs: bool = True, fold_in_ciphertext: bool = False, compact_cache: bool = False,
-                 pack: str | None = None, moddown: str | None = None, hoist: str | None = None, coef_bits: int = 0):
+                 pack: str | None = None, moddown: str | None = None, hoist: str | None = None, coef_bits: int = 0,
+                 lanes: int | None = None):
         self.w = wl.WORKLOADS[name]
         ps = wl.PARAM_SETS[self.w.params]
         self.N, self.primes, self.P, self.scale = ps["N"], list(ps["primes"]), ps["special"], ps["scale"]
@@ -55,6 +56,8 @@ class WorkloadRunner:
         if compact_cache:           # narrower resident words per prime: 68 % of the cache for the 50 + 6 x 40-bit chain
             bf.bf_set_compact_cache(self.ctx, True)
         self.compact_cache = compact_cache
+        if lanes:                   # concurrent key-switch chains (the library's default otherwise)
+            bf.bf_set_lanes(self.ctx, lanes)
         if coef_bits:               # weights resident as rounded 64- or 32-bit coefficients, transformed on every call
             bf.bf_set_coefficient_cache(self.ctx, coef_bits)
         self.coef_bits = coef_bits
