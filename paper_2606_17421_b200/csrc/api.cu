@@ -816,8 +816,11 @@ static int find_key(bf_ctx* ctx, u32 steps, int* key) {
 // of the extended basis and transformed: dig[set][j][m] = NTT_m( c1_j mod m ).  The digit in its own
 // prime is the transform of c1 itself, which the caller already has (c1_ntt + s*c1_ntt_stride, [r][N]):
 // it is copied, not recomputed.
+// div_t non-null: c1_coeff holds residues of polynomials of the extended basis and div_t + s*set_stride their
+// residues modulo P (centred): the digits are those of the polynomial divided by P (then c1_ntt is not used: no
+// transform of the quotient exists yet).
 static int modup(bf_ctx* ctx, cudaStream_t stream, const u64* c1_coeff, long long set_stride, u32 n_sets, u64* dig,
-                 const u64* c1_ntt, long long c1_ntt_stride) {
+                 const u64* c1_ntt, long long c1_ntt_stride, const u64* div_t = nullptr) {
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
     PolyBatch B;
     memset(&B, 0, sizeof(B));
@@ -834,10 +837,12 @@ static int modup(bf_ctx* ctx, cudaStream_t stream, const u64* c1_coeff, long lon
     B.dtile_div = r;
     B.dst_so = (long long)nb * N;
     B.dst_sm = N;
-    B.skip_diag = 1;
+    B.skip_diag = div_t ? 0 : 1;
     B.src_digits = 1;
     B.diag_src = c1_ntt;
     B.diag_so = c1_ntt_stride;
+    B.div_t = div_t;
+    B.div_so = set_stride;
     CK(ntt_forward(ctx->ring, B, n_sets * r, LOAD_REDUCE, stream));
     return BF_OK;
 }
@@ -911,11 +916,16 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     // one division by P per output: the inner products of all giant rotations stay alive until every chain is done
     const bool per_output = (ctx->plan.flags & BF_PLAN_MODDOWN_PER_OUTPUT) && n_giant > 0;
     TRY(ensure(ctx, ctx->Rres, (size_t)(per_output ? n_out : n_giant ? n_giant : 1) * ctw * 8));
-    TRY(ensure(ctx, ctx->Cc, (size_t)n_dig_sets * r * N * 8));
+    // double hoisting with one division per output: the giant steps' inputs are never divided in the transform domain
+    // (see below); their coefficient forms keep the residue modulo P
+    const bool assemble = dh && per_output;
+    const u32 cc_primes = assemble ? nb : r;
+    TRY(ensure(ctx, ctx->Cc, (size_t)n_dig_sets * cc_primes * N * 8));
     {
         u32 rot_scratch = rot_per_lane * (u32)lanes;
         if (per_output && rot_scratch < n_out) rot_scratch = n_out;     // Tc, Tn of the per-output division
         if (dh && rot_scratch < n_out * g) rot_scratch = n_out * g;     // Tc, Tn of the division of the inner sums
+        if (assemble && rot_scratch * 2 < n_out * (g + 3)) rot_scratch = cdiv(n_out * (g + 3), 2u);   // Tc of the output assembly
         TRY(ensure_rot_scratch(ctx, n_dig_sets, rot_scratch));
     }
     if (per_output) TRY(ensure(ctx, ctx->Ubig, (size_t)n_giant * 2 * nb * N * 8));
@@ -926,7 +936,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
         lane[c].U = (u64*)ctx->U.p + (size_t)c * rot_per_lane * 2 * nb * N;
         lane[c].Tc = (u64*)ctx->Tc.p + (size_t)c * rot_per_lane * 2 * N;
         lane[c].Tn = (u64*)ctx->Tn.p + (size_t)c * rot_per_lane * 2 * r * N;
-        lane[c].Cc = (u64*)ctx->Cc.p + (size_t)c * giant_per_lane * r * N;
+        lane[c].Cc = (u64*)ctx->Cc.p + (size_t)c * giant_per_lane * cc_primes * N;
     }
     u64* X = (u64*)ctx->X.p;
     u64* A = (u64*)ctx->A.p;
@@ -1024,7 +1034,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
                           ctx->device_error, ctx->stream));
         }
     }
-    if (dh) {
+    if (dh && !assemble) {
         // one division by P per inner sum and component: A[pj][comp][i] = (Aext[pj][comp][i] - t) * P^{-1}, t the
         // centred lift of the residue modulo P
         const u64* Aext = (const u64*)ctx->Aext.p;
@@ -1073,6 +1083,39 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             for (u32 rho0 = (u32)c * per; rho0 < lane_end; rho0 += giant_chunk) {
                 const u32 cnt = (lane_end - rho0 < giant_chunk) ? lane_end - rho0 : giant_chunk;
                 if (cnt > (u32)MAX_ROT_BATCH) return BF_ERR_INVALID_ARG;   // (cannot happen: see giant_per_lane)
+                if (assemble) {
+                    // The inner sums stay in the extended basis.  A giant step needs the digits of c1 / P: both happen
+                    // in the coefficient domain, where the division is element-wise, so one inverse transform over all
+                    // r + 1 primes feeds the hoisted ModUp, whose first load divides (no transform of the lift of the
+                    // P-residue, none of the quotient back and forth)
+                    const u64* Esrc = (const u64*)ctx->Aext.p + (size_t)(n_out + rho0) * xw + (size_t)nmp * N;   // c1 of each
+                    memset(&B, 0, sizeof(B));
+                    B.src = Esrc;
+                    B.dst = lane[c].Cc;
+                    B.src_so = (long long)xw;
+                    B.src_sm = N;
+                    B.dst_so = (long long)nb * N;
+                    B.dst_sm = N;
+                    B.n_m = nb;
+                    B.mod0 = 0;
+                    B.mod_step = 1;
+                    B.store_centred = 2;
+                    CK(ntt_inverse(ctx->ring, B, cnt, lane[c].s));
+                    TRY(modup(ctx, lane[c].s, lane[c].Cc, (long long)nb * N, cnt, lane[c].Dig, nullptr, 0,
+                              lane[c].Cc + (size_t)r * N));
+                    RotBatch rb;
+                    memset(&rb, 0, sizeof(rb));
+                    rb.n = (int)cnt;
+                    for (u32 t = 0; t < cnt; ++t) {
+                        rb.key[t] = giant_key[(rho0 + t) / n_out + 1];
+                        rb.dig[t] = (int)t;
+                        rb.c0[t] = (int)t;
+                        rb.out[t] = (int)t;
+                    }
+                    CK(launch_key_inner_product(ctx->ring, rb, lane[c].Dig, ctx->keys,
+                                                (u64*)ctx->Ubig.p + (size_t)rho0 * 2 * nb * N, ctx->device_error, lane[c].s));
+                    continue;
+                }
                 const u64* Asrc = A + (size_t)(n_out + rho0) * ctw;      // ciphertexts with j >= 1 are contiguous
                 memset(&B, 0, sizeof(B));
                 B.src = Asrc + (size_t)r * N;                            // c1 of each
@@ -1106,6 +1149,56 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             }
         }
         TRY(join_lanes(ctx, used));
+        if (assemble) {
+            // Output p, component by component, is a sum of terms of the extended basis, each divided by P by itself
+            // (the inner sum of giant step 0, the rotated c0 parts of the other inner sums) or once for their sum (the
+            // key-switch results).  The result is wanted in the coefficient domain, where the division is element-
+            // wise: so the terms' residues modulo the q_i are summed in the load of one inverse transform, their
+            // residues modulo P are transformed apart, and one element-wise kernel divides.  Same values as dividing
+            // each term in the transform domain (the transform is linear, the rotation commutes with the centred lift).
+            RotBatch rb;
+            memset(&rb, 0, sizeof(rb));
+            rb.n = (int)(g - 1);
+            for (u32 j = 1; j < g; ++j) rb.key[j - 1] = giant_key[j];
+            ModDownEpilogue epi;
+            memset(&epi, 0, sizeof(epi));
+            epi.u = (const u64*)ctx->Ubig.p;
+            epi.aext = (const u64*)ctx->Aext.p;
+            epi.aext_stride = (long long)xw;
+            epi.perm = ctx->perms_fwd;
+            epi.n_sum = g - 1;
+            epi.n_out = n_out;
+            epi.assemble = 1;
+            const u32 n_t = g + 3;
+            const bool beside = lanes > 1;
+            if (beside) TRY(fork_lanes(ctx, 2));
+            memset(&B, 0, sizeof(B));
+            B.src = epi.aext;                                   // (read through epi)
+            B.dst = (u64*)ctx->Tc.p;
+            B.dst_so = (long long)n_t * N;
+            B.dst_sm = N;
+            B.n_m = n_t;
+            B.mod0 = r;
+            B.mod_step = 0;
+            B.store_centred = 1;
+            CK(ntt_inverse_gathersum(ctx->ring, B, n_out, rb, epi, beside ? ctx->side[0] : ctx->stream));
+            memset(&B, 0, sizeof(B));
+            B.src = epi.aext;
+            B.dst = ct_out;
+            B.dst_so = (long long)ctw;
+            B.dst_sm = N;
+            B.n_m = 2 * r;
+            B.mod_wrap = r;
+            B.mod0 = 0;
+            B.mod_step = 1;
+            CK(ntt_inverse_gathersum(ctx->ring, B, n_out, rb, epi, ctx->stream));
+            if (beside) TRY(join_lanes(ctx, 2));
+            CK(finish_division(ctx->ring, ct_out, (long long)ctw, (const u64*)ctx->Tc.p, n_t, n_out, ctx->stream));
+            stamp(ctx, 3);
+            stamp(ctx, 4);
+            if (!pt_weights) TRY(check_overflow(ctx));
+            return BF_OK;
+        }
         if (per_output) {
             // sum over the giant steps of each output in the extended basis (each term read through its rotation),
             // then one division by P per output and component; the rotated c0 parts join in the same epilogue

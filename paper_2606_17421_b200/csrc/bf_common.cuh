@@ -260,6 +260,17 @@ struct ModDownEpilogue {
     u32 plain;                    // division by P of inner sums kept in the extended basis (double hoisting):
                                   //   polynomial (o, i): out_base[o*out_stride + i*N + n] = (u[o][i][n] - t[n]) * P^{-1},
                                   //   no rotation, nothing added
+    // Output assembly in the extended basis (double hoisting with one division per output; inverse transforms only).
+    // aext[(j*n_out + p)][comp][r+1][N] are the inner sums, u[((j-1)*n_out + p)*2 + comp][r+1][N] the key-switch
+    // results of the giant steps j >= 1, both read through rotation j's permutation.  Polynomial (o = p, m):
+    //   modulus i < r, m = comp*r + i:  aext[p][comp][i] + sum_j u[j][p][comp][i] + (comp == 0) sum_j aext[j*n_out+p][0][i]
+    //   modulus P, m = 0, 1:            sum_j u[j][p][comp = m][P]
+    //               m = 2, 3:            aext[p][comp = m - 2][P]
+    //               m = 3 + j:           aext[j*n_out + p][0][P]
+    // (the residues modulo P stay apart because each of those terms is divided by P, i.e. rounded, by itself)
+    const u64* aext;
+    long long aext_stride;
+    u32 assemble;
 };
 
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks
@@ -328,7 +339,8 @@ struct PolyBatch {
     u64 lift_mod;                 // LOAD_CENTRED: the modulus M the source residues live in
     u32 src_digits;               // LOAD_REDUCE: the source of outer index o is a residue modulo prime o % r
     u32 store_centred;            // inverse transform: store the centred lift of each coefficient plus 2^59
-                                  //   (the form LOAD_CENTRED reads) instead of the residue in [0, q)
+                                  //   (the form LOAD_CENTRED reads) instead of the residue in [0, q); 2: only for the
+                                  //   polynomials modulo the special prime
     u32 from_mont;                // inverse transform only: input is in Montgomery form, output is not
     u64* tile_ptr;                // non-null: the NTT-domain side lives there in the tile-major layout `tile`
     TileLayout tile;              //   (forward writes its final result there, inverse reads its input there);
@@ -348,6 +360,10 @@ struct PolyBatch {
                                   //   residue modulo P: the un-rotated input lifted to the extended basis
     u64* dtile_ptr;               // forward only, non-null: the final result goes there instead of dst, tile-major in tiles
     u32 dtile_div;                //   of KS_TILE coefficients (see ks_tile_index); with `scatter` the store is permuted
+    const u64* div_t;             // forward from a shared source, non-null (double hoisting): the source of digit
+    long long div_so;             //   i = o % o_div of set s = o / o_div is the residue modulo q_i of a polynomial in the
+                                  //   extended basis, coefficient domain, and t = div_t + s*div_so holds its residue
+                                  //   modulo P as a centred lift plus 2^59: the digit is (source - t) * P^{-1} mod q_i
 };
 
 // Operands of the key-switch inner product (digit sets and rotation keys) are kept tile-major, so that what a block

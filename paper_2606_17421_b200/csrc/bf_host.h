@@ -82,6 +82,10 @@ cudaError_t ntt_forward_moddown(const RingHost& ring, const PolyBatch& B, u32 n_
 // Inverse transform of the P-residues summed over the giant rotations of each output (per-output form of epi).
 cudaError_t ntt_inverse_gathersum(const RingHost& ring, const PolyBatch& B, u32 n_outer, const RotBatch& rb,
                                   const ModDownEpilogue& epi, cudaStream_t stream);
+// ct[p][comp][i] = (ct[p][comp][i] - sum of the centred P-residues T[p][.]) * P^{-1}: the division that ends the output
+// assembly in the extended basis (ModDownEpilogue::assemble names the n_t polynomials of T per output)
+cudaError_t finish_division(const RingHost& ring, u64* ct, long long ct_stride, const u64* T, u32 n_t, u32 n_out,
+                            cudaStream_t stream);
 cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B, u32 n_outer, int load, u64* final_dst,
                               const u32* scatter, u32 scatter_div, cudaStream_t stream);
 

@@ -426,7 +426,8 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
                         } else {
                             out = mul_shoup(e[i], mont ? R.ninv_m[mod] : R.ninv[mod], mont ? R.ninv_ms[mod] : R.ninvs[mod], q);
                         }
-                        if (B.store_centred) out = (out > (q - 1) / 2 ? out - q : out) + (1ull << 59);
+                        if (B.store_centred == 1 || (B.store_centred == 2 && mod == R.r))
+                            out = (out > (q - 1) / 2 ? out - q : out) + (1ull << 59);
                         dst[gidx] = out;
                     }
                 } else {
@@ -484,8 +485,26 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
         const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
                                        : (size_t)o * B.src_so;
         const u64* src = (const u64*)B.src + src_off;
-        for (int w = threadIdx.x; w < POINTS; w += blockDim.x)
-            staged[w] = src[((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1))];
+        if (B.div_t) {
+            // the digit is a division by P away: (source - t) * P^{-1} modulo the digit's own prime, t the centred lift
+            // of the polynomial's residue modulo P (exact: same value as dividing in the transform domain)
+            const u32 i = o % B.o_div;
+            LoadConsts dc;
+            dc.q = R.q[i];
+            dc.mu = R.mu[i];
+            dc.lift_mod = R.q[R.r];
+            dc.lift_red = barrett64(dc.lift_mod, dc.q, dc.mu);
+            const u64* tp = B.div_t + (size_t)(o / B.o_div) * B.div_so;
+            const u64 pinv = R.pinv[i], pinvs = R.pinvs[i];
+            for (int w = threadIdx.x; w < POINTS; w += blockDim.x) {
+                const size_t idx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1));
+                const u64 t = load_src<LOAD_CENTRED>(tp, idx, dc);
+                staged[w] = mul_shoup(sub_mod(src[idx], t, dc.q), pinv, pinvs, dc.q);
+            }
+        } else {
+            for (int w = threadIdx.x; w < POINTS; w += blockDim.x)
+                staged[w] = src[((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1))];
+        }
     }
     __syncthreads();
     for (u32 m = m_begin; m < m_end; ++m) {
@@ -762,6 +781,56 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                         for (int w = 0; w < 4; ++w) v4[w] = add_mod(v4[w], uv[t][w], q);
                     }
                 }
+            } else if constexpr (EPI == 4) {   // output assembly in the extended basis (see ModDownEpilogue::assemble)
+                const u32 nb = R.r + 1, g1 = epi.n_sum;
+                const size_t n = (size_t)chunk * LEN + 4 * s;
+                u32 comp = 0, ju = 0, jc_lo = 1, jc_hi = 0;    // u-terms of giant steps 1..ju, rotated c0 parts of jc_lo..jc_hi
+                bool ident = false;
+                if (mod < R.r) { comp = m / R.r; ident = true; ju = g1; if (comp == 0) jc_hi = g1; }
+                else if (m < 2) { comp = m; ju = g1; }
+                else if (m < 4) { comp = m - 2; ident = true; }
+                else { jc_lo = jc_hi = m - 3; }
+                v4[0] = v4[1] = v4[2] = v4[3] = 0;
+                if (ident) {
+                    const u64* ap = epi.aext + (size_t)o * epi.aext_stride + ((size_t)comp * nb + mod) * R.N + n;
+                    const ulonglong2 a = *(const ulonglong2*)ap, b = *(const ulonglong2*)(ap + 2);
+                    v4[0] = a.x; v4[1] = a.y; v4[2] = b.x; v4[3] = b.y;
+                }
+                const u32 j_first = ju ? 1u : jc_lo, j_last = ju ? g1 : jc_hi;
+                // three rotations at a time: their permutation entries are requested together, then all the words they
+                // point at (these launches are a few polynomials only: latency is all they cost)
+                for (u32 j0 = j_first; j0 <= j_last; j0 += 3) {
+                    uint4 pv[3];
+                    u64 uv[3][4], cv[3][4];
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t)
+                        if (j0 + t <= j_last) pv[t] = *(const uint4*)(epi.perm + (size_t)rb.key[j0 + t - 1] * R.N + n);
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t) {
+                        const u32 j = j0 + t;
+                        if (j > j_last) continue;
+                        if (j <= ju) {
+                            const u64* up = epi.u + ((((size_t)(j - 1) * epi.n_out + o) * 2 + comp) * nb + mod) * R.N;
+                            uv[t][0] = __ldg(up + pv[t].x); uv[t][1] = __ldg(up + pv[t].y);
+                            uv[t][2] = __ldg(up + pv[t].z); uv[t][3] = __ldg(up + pv[t].w);
+                        }
+                        if (j >= jc_lo && j <= jc_hi) {
+                            const u64* cp = epi.aext + ((size_t)j * epi.n_out + o) * epi.aext_stride + (size_t)mod * R.N;
+                            cv[t][0] = __ldg(cp + pv[t].x); cv[t][1] = __ldg(cp + pv[t].y);
+                            cv[t][2] = __ldg(cp + pv[t].z); cv[t][3] = __ldg(cp + pv[t].w);
+                        }
+                    }
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t) {
+                        const u32 j = j0 + t;
+                        if (j > j_last) continue;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            if (j <= ju) v4[w] = add_mod(v4[w], uv[t][w], q);
+                            if (j >= jc_lo && j <= jc_hi) v4[w] = add_mod(v4[w], cv[t][w], q);
+                        }
+                    }
+                }
             } else if constexpr (TILED) {  // read back from the tile-major plaintext cache
                 const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
                 const u32 n = chunk * LEN + 4 * s;
@@ -841,7 +910,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 // (the per-output forms run on a few polynomials per launch and hold the operands of three rotations at once: they
 // trade resident blocks for registers)
 template <bool FWD, int EPI, bool TILED>
-__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, EPI == 2 ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
+__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, (EPI == 2 || EPI == 4) ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
     __shared__ __align__(128) u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
@@ -952,6 +1021,9 @@ static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n
     if (FWD && epi && epi->plain) {
         launch_dependent(ring, ntt_contig<FWD, 3, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
                          *epi);
+    } else if (!FWD && epi && epi->assemble) {
+        launch_dependent(ring, ntt_contig<false, 4, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
+                         *epi);
     } else if (epi && epi->n_sum) {
         launch_dependent(ring, ntt_contig<FWD, 2, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
                          *epi);
@@ -1016,6 +1088,41 @@ cudaError_t ntt_inverse_gathersum(const RingHost& ring, const PolyBatch& B, u32 
     cudaError_t e = launch_contig<false>(ring, B, n_polys, stream, &rb, &epi);
     if (e != cudaSuccess) return e;
     return launch_strided<false, LOAD_PLAIN>(ring, B, n_polys, stream);
+}
+
+// Last step of the output assembly in the extended basis: the inverse transforms above left, per output p and
+// component, the sum of all terms modulo every q_i (in ct) and each separately rounded term's residue modulo P as a
+// centred lift plus 2^59 (in T, n_t polynomials per output, indexed as ModDownEpilogue::assemble lists them):
+//   ct[p][comp][i][n] = (ct[p][comp][i][n] - sum_terms t_term[n]) * P^{-1}  (mod q_i)
+__global__ void __launch_bounds__(256) finish_division_kernel(const RingDev R, u64* __restrict__ ct, long long ct_stride,
+                                                              const u64* __restrict__ T, u32 n_t) {
+    grid_dependency_enter();
+    const u32 n = blockIdx.x * 256 + threadIdx.x;
+    const u32 p = blockIdx.y >> 1, comp = blockIdx.y & 1;
+    const u64* tp = T + (size_t)p * n_t * R.N + n;
+    u64* cp = ct + (size_t)p * ct_stride + (size_t)comp * R.r * R.N + n;
+    const u64 P = R.q[R.r];
+    for (u32 i = 0; i < R.r; ++i) {
+        LoadConsts dc;
+        dc.q = R.q[i];
+        dc.mu = R.mu[i];
+        dc.lift_mod = P;
+        dc.lift_red = barrett64(P, dc.q, dc.mu);
+        u64 acc = add_mod(load_src<LOAD_CENTRED>(tp, (size_t)comp * R.N, dc),
+                          load_src<LOAD_CENTRED>(tp, (size_t)(comp + 2) * R.N, dc), dc.q);
+        if (comp == 0)
+            for (u32 m = 4; m < n_t; ++m) acc = add_mod(acc, load_src<LOAD_CENTRED>(tp, (size_t)m * R.N, dc), dc.q);
+        u64* w = cp + (size_t)i * R.N;
+        *w = mul_shoup(sub_mod(*w, acc, dc.q), R.pinv[i], R.pinvs[i], dc.q);
+    }
+}
+
+cudaError_t finish_division(const RingHost& ring, u64* ct, long long ct_stride, const u64* T, u32 n_t, u32 n_out,
+                            cudaStream_t stream) {
+    ProfScope prof(ring.prof, CAT_NTT_INV_STRIDED, stream);
+    launch_dependent(ring, finish_division_kernel, dim3(ring.dev.N / 256, n_out * 2), dim3(256), 0, stream, ring.dev, ct,
+                     ct_stride, T, n_t);
+    return cudaGetLastError();
 }
 
 cudaError_t ntt_inverse(const RingHost& ring, const PolyBatch& B, u32 n_outer, cudaStream_t stream) {
