@@ -1010,13 +1010,20 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     // ---- multiply-accumulate over the encoded diagonals (double hoisting: over the extended basis, into Aext)
     const u32 n_terms = n_in * b, n_pj = n_out * g;
     u64* mac_out = dh ? (u64*)ctx->Aext.p : A;
+    MacScatter msc;
+    memset(&msc, 0, sizeof(msc));
+    if (assemble) {         // component 0 of the inner sums with j >= 1 is stored rotated (only the output assembly reads it)
+        msc.pinv = ctx->perms;
+        msc.n_out = n_out;
+        for (u32 j = 1; j < g; ++j) msc.key[j] = giant_key[j];
+    }
     if (pt_weights && pt_weights->pt) {
         // double hoisting: the launch for the special prime (one eighth of the words, on whole-word arithmetic) runs
         // beside the launch for the ciphertext primes
         const bool beside = dh && lanes > 1;
         if (beside) TRY(fork_lanes(ctx, 2));
         CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, mac_out, n_pj, n_terms, true, ctx->device_error, ctx->stream,
-                      beside ? ctx->side[0] : nullptr));
+                      beside ? ctx->side[0] : nullptr, &msc));
         if (beside) TRY(join_lanes(ctx, 2));
     } else {
         // fallback: encode groups of (j, p) just in time into a scratch ring, then consume them (weights kept as
@@ -1030,8 +1037,9 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             const u32 cnt = (n_pj - pj0 < groups) ? n_pj - pj0 : groups;
             const TileLayout cl = mac_tile_layout(ctx->ring, cnt, n_terms, nmp);
             TRY(encode_range(ctx, W_raw, d_out, d_in, pj0 * n_terms, cnt * n_terms, (u64*)ctx->ptjit.p, cl, pj0, pt_weights));
+            msc.pj0 = pj0;
             CK(launch_mac(ctx->ring, (const u64*)ctx->ptjit.p, cl, X, mac_out + (size_t)pj0 * xw, cnt, n_terms, false,
-                          ctx->device_error, ctx->stream));
+                          ctx->device_error, ctx->stream, nullptr, &msc));
         }
     }
     if (dh && !assemble) {
@@ -1112,8 +1120,10 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
                         rb.c0[t] = (int)t;
                         rb.out[t] = (int)t;
                     }
+                    // (stored through the rotation: the output assembly reads plain sums)
                     CK(launch_key_inner_product(ctx->ring, rb, lane[c].Dig, ctx->keys,
-                                                (u64*)ctx->Ubig.p + (size_t)rho0 * 2 * nb * N, ctx->device_error, lane[c].s));
+                                                (u64*)ctx->Ubig.p + (size_t)rho0 * 2 * nb * N, ctx->device_error, lane[c].s,
+                                                nullptr, ctx->perms));
                     continue;
                 }
                 const u64* Asrc = A + (size_t)(n_out + rho0) * ctw;      // ciphertexts with j >= 1 are contiguous
@@ -1165,7 +1175,6 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             epi.u = (const u64*)ctx->Ubig.p;
             epi.aext = (const u64*)ctx->Aext.p;
             epi.aext_stride = (long long)xw;
-            epi.perm = ctx->perms_fwd;
             epi.n_sum = g - 1;
             epi.n_out = n_out;
             epi.assemble = 1;

@@ -262,7 +262,8 @@ struct ModDownEpilogue {
                                   //   no rotation, nothing added
     // Output assembly in the extended basis (double hoisting with one division per output; inverse transforms only).
     // aext[(j*n_out + p)][comp][r+1][N] are the inner sums, u[((j-1)*n_out + p)*2 + comp][r+1][N] the key-switch
-    // results of the giant steps j >= 1, both read through rotation j's permutation.  Polynomial (o = p, m):
+    // results of the giant steps j >= 1; what is rotated (u, and component 0 of the inner sums with j >= 1) was stored
+    // through rotation j's permutation by its producer.  Polynomial (o = p, m):
     //   modulus i < r, m = comp*r + i:  aext[p][comp][i] + sum_j u[j][p][comp][i] + (comp == 0) sum_j aext[j*n_out+p][0][i]
     //   modulus P, m = 0, 1:            sum_j u[j][p][comp = m][P]
     //               m = 2, 3:            aext[p][comp = m - 2][P]
@@ -271,6 +272,15 @@ struct ModDownEpilogue {
     const u64* aext;
     long long aext_stride;
     u32 assemble;
+};
+
+// Double hoisting with one division per output: component 0 of inner sum (j, p), j >= 1, is only ever used rotated
+// by giant step j, so the multiply-accumulate stores it through that rotation's permutation (group pj0 + pj has
+// j = (pj0 + pj) / n_out; pinv = null: plain stores).
+struct MacScatter {
+    const u32* pinv;              // [n_keys][N]
+    u32 n_out, pj0;
+    int key[MAX_ROT_BATCH + 1];   // key (permutation table) of giant step j
 };
 
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks

@@ -94,6 +94,7 @@ cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B, u32 n_ou
 cudaError_t launch_pointwise_mul(const RingHost& ring, const u64* a, const u64* b, u64* out, u32 n_polys, u32 n_m,
                                  u32 mod0, cudaStream_t stream);
 // u'[rot][comp][m][n] = sum_j dig[dig(rot)][j][m][n] * key'[key(rot)][j][comp][m][n]  (keys pre-permuted)
+// pinv non-null, xext null: u'[rot][comp][m] is stored through the rotation's permutation, at pinv[rb.key[rot]][n].
 // xext non-null (double hoisting): rotation `rot` is not stored to u but finished as a rotated input in the
 // extended basis: xext[rb.out[rot]][comp][m][pinv[rb.key[rot]][n]] = u'[comp][m][n] + (comp == 0 ?
 // xext[rb.c0[rot]][0][m][n] : 0), terms of [2][r+1][N] words (term rb.c0[rot] holds P times the un-rotated input).
@@ -109,7 +110,7 @@ size_t mac_tile_bytes(const RingHost& ring, const TileLayout& t);           // b
 // everything the launch reads and joins it afterwards), beside the launch for the ciphertext primes on `stream`
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
                        u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream,
-                       cudaStream_t special_stream = nullptr);
+                       cudaStream_t special_stream = nullptr, const MacScatter* scatter = nullptr);
 cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_ct, u32 level, const u64* inv,
                            const u64* invs, const u64* qlmod, cudaStream_t stream);
 

@@ -117,7 +117,7 @@ template <bool KARA, int LOG_TN, bool COMPACT>
 __global__ void __launch_bounds__(MAC_THREADS, 3)
 mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, const u64* __restrict__ x,
            u64* __restrict__ a, u32 n_terms, u32 n_pj, u32 pj_per_block, u32 lazy_terms, u32 early_weights,
-           u32 n_whole, u32 tail_split, u32 prime0, u32 n_launch_primes, int* __restrict__ error_flag) {
+           u32 n_whole, u32 tail_split, u32 prime0, u32 n_launch_primes, int* __restrict__ error_flag, const MacScatter sc) {
     extern __shared__ __align__(128) unsigned char mac_smem[];
     asm volatile("griddepcontrol.launch_dependents;");
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
@@ -343,18 +343,20 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         if (pj < pj_end) {
             since_flush += cnt;
             if (ch + 1 == n_chunks) {
-                u64* ap = a + ((size_t)pj * 2 * r + i) * N + n0 + c;
+                u64* ap = a + ((size_t)pj * 2 * r + i) * N;
+                u32 at0 = n0 + c;                                       // where component 0 goes (see MacScatter)
+                if (sc.pinv && sc.pj0 + pj >= sc.n_out) at0 = __ldg(sc.pinv + (size_t)sc.key[(sc.pj0 + pj) / sc.n_out] * N + n0 + c);
                 if (KARA) {
                     u64 H, L;
                     k0.value(KARA_L, H, L);
-                    ap[0] = redc_2x32(H, L, q, qneg32);
+                    ap[at0] = redc_2x32(H, L, q, qneg32);
                     k1.value(KARA_L, H, L);
-                    ap[(size_t)r * N] = redc_2x32(H, L, q, qneg32);
+                    ap[(size_t)r * N + n0 + c] = redc_2x32(H, L, q, qneg32);
                     k0 = KaraAcc();
                     k1 = KaraAcc();
                 } else {
-                    ap[0] = a0.reduce_mont(q, R.qneg[i]);
-                    ap[(size_t)r * N] = a1.reduce_mont(q, R.qneg[i]);
+                    ap[at0] = a0.reduce_mont(q, R.qneg[i]);
+                    ap[(size_t)r * N + n0 + c] = a1.reduce_mont(q, R.qneg[i]);
                     a0.reset_to(0);
                     a1.reset_to(0);
                 }
@@ -413,7 +415,7 @@ u32 mac_split_bits(const RingHost& ring) {
 template <bool KARA, int LOG_TN, bool COMPACT>
 static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a,
                                 u32 n_pj, u32 n_terms, u32 lazy, u32 early_weights, u32 prime0, u32 n_launch_primes,
-                                int* error_flag, cudaStream_t stream) {
+                                int* error_flag, cudaStream_t stream, const MacScatter& sc) {
     constexpr u32 TN = 1u << LOG_TN, PL = MAC_CONSUMERS >> LOG_TN;
     const size_t smem = (size_t)MAC_RING_BYTES + (size_t)n_terms * 2 * TN * 8 + (2 * MAC_MAX_STAGES + 1) * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
@@ -463,14 +465,14 @@ static cudaError_t launch_mac_t(const RingHost& ring, const u64* pt, const TileL
     dim3 grid(n_whole + (units - n_whole) * tail_split);
     return launch_dependent(ring, mac_kernel<KARA, LOG_TN, COMPACT>, grid, dim3(MAC_THREADS), smem, stream, ring.dev, pt, lay, x, a,
                             n_terms, n_pj, pj_per_block, lazy, early_weights, n_whole, tail_split, prime0, n_launch_primes,
-                            error_flag);
+                            error_flag, sc);
 }
 
 // One launch over primes prime0 .. prime0 + n_launch_primes - 1 of the layout; kara: Karatsuba on 25-bit limbs
 // (those primes are all below 2^50), else whole words.
 static cudaError_t launch_mac_primes(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a,
                                      u32 n_pj, u32 n_terms, bool weights_static, u32 prime0, u32 n_launch_primes, bool kara,
-                                     int* error_flag, cudaStream_t stream) {
+                                     int* error_flag, cudaStream_t stream, const MacScatter& sc) {
     ProfScope prof(ring.prof, CAT_MAC, stream);
     u64 qmax = 0;
     for (u32 i = prime0; i < prime0 + n_launch_primes; ++i) qmax = ring.q[i] > qmax ? ring.q[i] : qmax;
@@ -489,8 +491,8 @@ static cudaError_t launch_mac_primes(const RingHost& ring, const u64* pt, const 
     bool compact = false;
     for (u32 i = prime0; i < prime0 + n_launch_primes; ++i) compact = compact || tile_format(lay, i) != TILE_W64;
 #define BF_MAC(S, L)                                                                                             \
-    (compact ? launch_mac_t<S, L, true>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, prime0, n_launch_primes, error_flag, stream)     \
-             : launch_mac_t<S, L, false>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, prime0, n_launch_primes, error_flag, stream))
+    (compact ? launch_mac_t<S, L, true>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, prime0, n_launch_primes, error_flag, stream, sc) \
+             : launch_mac_t<S, L, false>(ring, pt, lay, x, a, n_pj, n_terms, lazy, early, prime0, n_launch_primes, error_flag, stream, sc))
     if (kara) {
         switch (log_tn) {
             case 8: return BF_MAC(true, 8);
@@ -511,16 +513,20 @@ static cudaError_t launch_mac_primes(const RingHost& ring, const u64* pt, const 
 }
 
 cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& lay, const u64* x, u64* a, u32 n_pj,
-                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream, cudaStream_t special_stream) {
+                       u32 n_terms, bool weights_static, int* error_flag, cudaStream_t stream, cudaStream_t special_stream,
+                       const MacScatter* scatter) {
     if (n_pj == 0) return cudaSuccess;
     if (lay.n_pj != n_pj || lay.n_terms != n_terms) return cudaErrorInvalidValue;
     const u32 r = ring.dev.r;
     const bool kara = mac_split_bits(ring) != 0;
-    cudaError_t e = launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, 0, r, kara, error_flag, stream);
+    MacScatter sc;
+    if (scatter) sc = *scatter;
+    else memset(&sc, 0, sizeof(sc));
+    cudaError_t e = launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, 0, r, kara, error_flag, stream, sc);
     if (e != cudaSuccess || lay.n_primes <= r) return e;
     // double hoisting: the residues modulo the 60-bit special prime, on whole words
     return launch_mac_primes(ring, pt, lay, x, a, n_pj, n_terms, weights_static, r, lay.n_primes - r, false, error_flag,
-                             special_stream ? special_stream : stream);
+                             special_stream ? special_stream : stream, sc);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -597,10 +603,8 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
     // rotation, and P*c0) is requested before the wait for the operands, so that it is not a second round trip
     u32 dest = 0;
     u64 pc0 = 0;
-    if (xext) {
-        dest = __ldg(&pinv[(size_t)rb.key[first] * N + n0 + tid]);          // (the same for every rotation of the run)
-        pc0 = xext[(size_t)rb.c0[first] * term_words + (size_t)m * N + n0 + tid];
-    }
+    if (pinv) dest = __ldg(&pinv[(size_t)rb.key[first] * N + n0 + tid]);    // (the same for every rotation of the run)
+    if (xext) pc0 = xext[(size_t)rb.c0[first] * term_words + (size_t)m * N + n0 + tid];
     mbar_wait(kbar, 0, error_flag);
     for (u32 it = 0; it < cnt; ++it) {
         const u32 rot = first + it;
@@ -641,7 +645,8 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
             xp[(size_t)nb * N] = v1;
             pc0 = pc0_next;
         } else {
-            u64* up = u + ((size_t)rot * 2 * nb + m) * N + n0 + tid;
+            // (pinv without xext: the plain result, stored through the rotation's permutation)
+            u64* up = u + ((size_t)rot * 2 * nb + m) * N + (pinv ? dest : n0 + tid);
             up[0] = v0;
             up[(size_t)nb * N] = v1;
         }

@@ -796,40 +796,43 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                     const ulonglong2 a = *(const ulonglong2*)ap, b = *(const ulonglong2*)(ap + 2);
                     v4[0] = a.x; v4[1] = a.y; v4[2] = b.x; v4[3] = b.y;
                 }
-                const u32 j_first = ju ? 1u : jc_lo, j_last = ju ? g1 : jc_hi;
-                // three rotations at a time: their permutation entries are requested together, then all the words they
-                // point at (these launches are a few polynomials only: latency is all they cost)
-                for (u32 j0 = j_first; j0 <= j_last; j0 += 3) {
-                    uint4 pv[3];
-                    u64 uv[3][4], cv[3][4];
+                // (the producers stored every rotated term through its rotation already: plain loads; the words of
+                // three giant steps are requested together)
+                const u64* ub = epi.u + (((size_t)o * 2 + comp) * nb + mod) * R.N + n;          // giant step 1
+                const size_t u_step = (size_t)epi.n_out * 2 * nb * R.N;
+                for (u32 j0 = 1; j0 <= ju; j0 += 3) {
+                    ulonglong2 a2[3], b2[3];
 #pragma unroll
                     for (u32 t = 0; t < 3; ++t)
-                        if (j0 + t <= j_last) pv[t] = *(const uint4*)(epi.perm + (size_t)rb.key[j0 + t - 1] * R.N + n);
-#pragma unroll
-                    for (u32 t = 0; t < 3; ++t) {
-                        const u32 j = j0 + t;
-                        if (j > j_last) continue;
-                        if (j <= ju) {
-                            const u64* up = epi.u + ((((size_t)(j - 1) * epi.n_out + o) * 2 + comp) * nb + mod) * R.N;
-                            uv[t][0] = __ldg(up + pv[t].x); uv[t][1] = __ldg(up + pv[t].y);
-                            uv[t][2] = __ldg(up + pv[t].z); uv[t][3] = __ldg(up + pv[t].w);
+                        if (j0 + t <= ju) {
+                            const u64* up = ub + (size_t)(j0 + t - 1) * u_step;
+                            a2[t] = *(const ulonglong2*)up;
+                            b2[t] = *(const ulonglong2*)(up + 2);
                         }
-                        if (j >= jc_lo && j <= jc_hi) {
-                            const u64* cp = epi.aext + ((size_t)j * epi.n_out + o) * epi.aext_stride + (size_t)mod * R.N;
-                            cv[t][0] = __ldg(cp + pv[t].x); cv[t][1] = __ldg(cp + pv[t].y);
-                            cv[t][2] = __ldg(cp + pv[t].z); cv[t][3] = __ldg(cp + pv[t].w);
-                        }
-                    }
 #pragma unroll
-                    for (u32 t = 0; t < 3; ++t) {
-                        const u32 j = j0 + t;
-                        if (j > j_last) continue;
-#pragma unroll
-                        for (int w = 0; w < 4; ++w) {
-                            if (j <= ju) v4[w] = add_mod(v4[w], uv[t][w], q);
-                            if (j >= jc_lo && j <= jc_hi) v4[w] = add_mod(v4[w], cv[t][w], q);
+                    for (u32 t = 0; t < 3; ++t)
+                        if (j0 + t <= ju) {
+                            v4[0] = add_mod(v4[0], a2[t].x, q); v4[1] = add_mod(v4[1], a2[t].y, q);
+                            v4[2] = add_mod(v4[2], b2[t].x, q); v4[3] = add_mod(v4[3], b2[t].y, q);
                         }
-                    }
+                }
+                const u64* cb = epi.aext + (size_t)o * epi.aext_stride + (size_t)mod * R.N + n;  // inner sum (0, p), c0
+                const size_t c_step = (size_t)epi.n_out * epi.aext_stride;
+                for (u32 j0 = jc_lo; j0 <= jc_hi; j0 += 3) {
+                    ulonglong2 a2[3], b2[3];
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t)
+                        if (j0 + t <= jc_hi) {
+                            const u64* cp = cb + (size_t)(j0 + t) * c_step;
+                            a2[t] = *(const ulonglong2*)cp;
+                            b2[t] = *(const ulonglong2*)(cp + 2);
+                        }
+#pragma unroll
+                    for (u32 t = 0; t < 3; ++t)
+                        if (j0 + t <= jc_hi) {
+                            v4[0] = add_mod(v4[0], a2[t].x, q); v4[1] = add_mod(v4[1], a2[t].y, q);
+                            v4[2] = add_mod(v4[2], b2[t].x, q); v4[3] = add_mod(v4[3], b2[t].y, q);
+                        }
                 }
             } else if constexpr (TILED) {  // read back from the tile-major plaintext cache
                 const u32 pj = (B.o_base + o) / B.tile.n_terms - B.tile_pj0, term = (B.o_base + o) % B.tile.n_terms;
@@ -910,7 +913,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 // (the per-output forms run on a few polynomials per launch and hold the operands of three rotations at once: they
 // trade resident blocks for registers)
 template <bool FWD, int EPI, bool TILED>
-__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, (EPI == 2 || EPI == 4) ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
+__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, EPI == 2 ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
     __shared__ __align__(128) u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
@@ -1101,20 +1104,32 @@ __global__ void __launch_bounds__(256) finish_division_kernel(const RingDev R, u
     const u32 p = blockIdx.y >> 1, comp = blockIdx.y & 1;
     const u64* tp = T + (size_t)p * n_t * R.N + n;
     u64* cp = ct + (size_t)p * ct_stride + (size_t)comp * R.r * R.N + n;
-    const u64 P = R.q[R.r];
-    for (u32 i = 0; i < R.r; ++i) {
-        LoadConsts dc;
-        dc.q = R.q[i];
-        dc.mu = R.mu[i];
-        dc.lift_mod = P;
-        dc.lift_red = barrett64(P, dc.q, dc.mu);
-        u64 acc = add_mod(load_src<LOAD_CENTRED>(tp, (size_t)comp * R.N, dc),
-                          load_src<LOAD_CENTRED>(tp, (size_t)(comp + 2) * R.N, dc), dc.q);
-        if (comp == 0)
-            for (u32 m = 4; m < n_t; ++m) acc = add_mod(acc, load_src<LOAD_CENTRED>(tp, (size_t)m * R.N, dc), dc.q);
-        u64* w = cp + (size_t)i * R.N;
-        *w = mul_shoup(sub_mod(*w, acc, dc.q), R.pinv[i], R.pinvs[i], dc.q);
+    u64 v[MAX_MODULI];
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i)
+        if ((u32)i < R.r) v[i] = cp[(size_t)i * R.N];
+    // this component's terms: polynomials comp, comp + 2 and, for component 0, 4 .. n_t - 1.  Their centred values are
+    // added as integers, eight at a time (each is below 2^59 in magnitude), and the sum is reduced once per prime
+    const u32 nt = comp == 0 ? n_t - 2 : 2u;
+    for (u32 k0 = 0; k0 < nt; k0 += 8) {
+        i64 S = 0;
+        for (u32 k = k0; k < nt && k < k0 + 8; ++k) {
+            const u32 m = k < 2 ? comp + 2 * k : k + 2;
+            S += (i64)(tp[(size_t)m * R.N] - (1ull << 59));
+        }
+        const bool neg = S < 0;
+        const u64 a = neg ? (u64)(-S) : (u64)S;
+#pragma unroll
+        for (int i = 0; i < MAX_MODULI; ++i)
+            if ((u32)i < R.r) {
+                u64 t = barrett64(a, R.q[i], R.mu[i]);
+                if (neg && t) t = R.q[i] - t;
+                v[i] = sub_mod(v[i], t, R.q[i]);
+            }
     }
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i)
+        if ((u32)i < R.r) cp[(size_t)i * R.N] = mul_shoup(v[i], R.pinv[i], R.pinvs[i], R.q[i]);
 }
 
 cudaError_t finish_division(const RingHost& ring, u64* ct, long long ct_stride, const u64* T, u32 n_t, u32 n_out,
