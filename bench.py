@@ -185,11 +185,22 @@ def transform_counts(runner) -> dict:
         # divisions by P: one per rotation and component, or (per_output) one per baby rotation and per output
         n_baby_lift = 2 * n_out * g if runner.plan.hoist == "double" else 2 * n_in * (b - 1)
         n_lift = n_baby_lift + 2 * (n_out if runner.plan.moddown == "per_output" and n_giant else n_giant)
-        for i in range(r):
-            fwd[i] += 2 * n_in + sets * (r - 1) + n_lift   # inputs; digits of the other primes; lifted P-residues
-            inv[i] += n_giant + 2 * n_out                  # c1 of the giant-step inputs; outputs
-        fwd[r] += sets * r
-        inv[r] += n_lift                                   # P-residues of the inner products
+        if runner.plan.hoist == "double" and runner.plan.moddown == "per_output" and n_giant:
+            # inner sums stay in the extended basis: no lifted P-residue is transformed; the giant steps' ModUp divides in
+            # its first load (and transforms each digit in its own prime too); the outputs are assembled by one inverse
+            # transform per residue, g + 3 of them modulo P per output
+            baby_sets = n_in if b > 1 else 0
+            for i in range(r):
+                fwd[i] += 2 * n_in + baby_sets * (r - 1) + n_giant * r
+                inv[i] += n_giant + 2 * n_out
+            fwd[r] += sets * r
+            inv[r] += n_giant + n_out * (g + 3)
+        else:
+            for i in range(r):
+                fwd[i] += 2 * n_in + sets * (r - 1) + n_lift   # inputs; digits of the other primes; lifted P-residues
+                inv[i] += n_giant + 2 * n_out                  # c1 of the giant-step inputs; outputs
+            fwd[r] += sets * r
+            inv[r] += n_lift                                   # P-residues of the inner products
         if runner.transforms_weights_per_call(e):          # on the fly or kept as coefficients: every diagonal is transformed on each call
             n_diag = n_in * n_out * b * g
             for i in range(r + (1 if runner.plan.hoist == "double" else 0)):

@@ -1644,7 +1644,7 @@ extern "C" int bf_kernel_categories(void) { return (int)CAT_COUNT; }
 extern "C" const char* bf_kernel_category_name(int cat) {
     static const char* names[CAT_COUNT] = {"ntt_fwd_strided", "ntt_fwd_contig", "ntt_inv_contig", "ntt_inv_strided",
                                            "key_inner_product", "mac", "rescale",
-                                           "encode_fft_a", "encode_fft_b", "pointwise_mul"};
+                                           "encode_fft_a", "encode_fft_b", "pointwise_mul", "divide_by_p"};
     return (cat >= 0 && cat < (int)CAT_COUNT) ? names[cat] : "";
 }
 

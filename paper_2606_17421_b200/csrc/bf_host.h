@@ -19,7 +19,7 @@ struct NttGeometry {
 enum KernelCat : int {
     CAT_NTT_FWD_STRIDED = 0, CAT_NTT_FWD_CONTIG, CAT_NTT_INV_CONTIG, CAT_NTT_INV_STRIDED,
     CAT_KEY_INNER, CAT_MAC, CAT_RESCALE,
-    CAT_ENCODE_FFT_A, CAT_ENCODE_FFT_B, CAT_POINTWISE, CAT_COUNT
+    CAT_ENCODE_FFT_A, CAT_ENCODE_FFT_B, CAT_POINTWISE, CAT_DIVIDE, CAT_COUNT
 };
 
 struct Profiler {

@@ -1134,7 +1134,7 @@ __global__ void __launch_bounds__(256) finish_division_kernel(const RingDev R, u
 
 cudaError_t finish_division(const RingHost& ring, u64* ct, long long ct_stride, const u64* T, u32 n_t, u32 n_out,
                             cudaStream_t stream) {
-    ProfScope prof(ring.prof, CAT_NTT_INV_STRIDED, stream);
+    ProfScope prof(ring.prof, CAT_DIVIDE, stream);
     launch_dependent(ring, finish_division_kernel, dim3(ring.dev.N / 256, n_out * 2), dim3(256), 0, stream, ring.dev, ct,
                      ct_stride, T, n_t);
     return cudaGetLastError();
