@@ -170,7 +170,6 @@ def transform_counts(runner) -> dict:
     (at least 10 32-bit multiply-adds per butterfly)."""
     import math
     r, N = runner.r, runner.N
-    b, g = runner.plan.b, runner.plan.g
     per = (N // 2) * int(math.log2(N))
     moduli = list(runner.primes) + [runner.P]
     cost = [8 if q < (1 << 41) else 12 if q < (1 << 50) else 10 for q in moduli]
@@ -178,7 +177,7 @@ def transform_counts(runner) -> dict:
     fwd = [0] * (r + 1)
     inv = [0] * (r + 1)
     for e in runner.layers:
-        n_in, n_out = e["n_in"], e["n_out"]
+        n_in, n_out, b, g = e["n_in"], e["n_out"], e["b"], e["g"]
         n_giant = (g - 1) * n_out
         sets = (n_in if b > 1 else 0) + n_giant            # ModUp digit sets
         rots = n_in * (b - 1) + n_giant                    # key switches
@@ -358,7 +357,9 @@ class Measurement:
         return {"layers": len(R.layers), "unit_of_work": "decode token (all linear layers)" if whole_step else "one projection call",
                 "ring_N": R.N, "ct_primes": R.r,
                 "plan": {"D": R.plan.D, "tau": R.plan.tau, "b": R.plan.b, "g": R.plan.g, "pack": R.plan.pack,
-                         "moddown": R.plan.moddown, "hoist": R.plan.hoist},
+                         "moddown": R.plan.moddown, "hoist": R.plan.hoist,
+                         "splits_per_call": {k: f"{b}x{g}" for k, (b, g) in R.splits.items()
+                                             if (b, g) != (R.plan.b, R.plan.g)}},
                 "ciphertexts_in": sum(e["n_in"] for e in R.layers), "ciphertexts_out": sum(e["n_out"] for e in R.layers),
                 "boundary_bytes": h2d + d2h, "rotation_keys": len(R.rot_steps), "fallback_layers": R.n_fallback_layers(),
                 "encoded_weight_bytes_cached": R.cached_pt_bytes(), "encoded_weight_bytes_total": R.total_pt_bytes(),

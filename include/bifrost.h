@@ -110,6 +110,13 @@ uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in);
  * allocating when the cache budget would be exceeded: the caller then passes W itself to bf_linear.
  * Synchronises. */
 int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, uint32_t d_in, bf_weights** out);
+/* The same with a baby/giant split of its own for this projection (Sec. 4.2 "BSGS matrix-vector multiply": the
+ * split trades hoisted baby rotations of the inputs against full key switches of the outputs, and the best trade
+ * depends on n_in and n_out).  bsgs_b * bsgs_g = tile_D / tau as for the plan, both powers of two,
+ * bsgs_b - 1 <= 64 (and bsgs_g - 1 <= 64 with BF_PLAN_MODDOWN_PER_OUTPUT), else BF_ERR_SHAPE.  bf_linear with this handle
+ * needs the rotation keys of this split: k*tau for k < bsgs_b and j*bsgs_b*tau for j < bsgs_g. */
+int bf_encode_weights_split(bf_ctx* ctx, const float* W, uint32_t d_out, uint32_t d_in, uint32_t bsgs_b, uint32_t bsgs_g,
+                            bf_weights** out);
 void bf_weights_free(bf_ctx* ctx, bf_weights* w);
 
 /* FHE_Linear (Alg. 3, decode loop; Sec. 4.2 "BSGS matrix-vector multiply"):
@@ -119,7 +126,7 @@ void bf_weights_free(bf_ctx* ctx, bf_weights* w);
  * followed by a key switch with one special prime (one prime per digit), each with its own
  * division by P.
  *   ct_in       device, n_in ciphertexts at full level, boundary layout
- *   pt_weights  handle from bf_encode_weights for this (d_out, d_in); or NULL, in which case
+ *   pt_weights  handle from bf_encode_weights for this (d_out, d_in) (b and g are then the handle's); or NULL, in which case
  *   W_raw       device fp32 [d_out][d_in] is encoded on the fly (fallback path)
  *   ct_out      device, n_out ciphertexts, full level, scale = scale(ct_in) * Delta; must not
  *               overlap ct_in

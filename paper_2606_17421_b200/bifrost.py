@@ -56,6 +56,7 @@ _SIGNATURES = {
     "bf_cache_bytes_used": (_u64, [_vp]),
     "bf_weights_bytes": (_u64, [_vp, _u32, _u32]),
     "bf_encode_weights": (ctypes.c_int, [_vp, _vp, _u32, _u32, ctypes.POINTER(_vp)]),
+    "bf_encode_weights_split": (ctypes.c_int, [_vp, _vp, _u32, _u32, _u32, _u32, ctypes.POINTER(_vp)]),
     "bf_weights_free": (None, [_vp, _vp]),
     "bf_linear": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
     "bf_device_status": (ctypes.c_int, [_vp]),
@@ -164,6 +165,13 @@ def bf_weights_bytes(ctx, d_out: int, d_in: int) -> int:
 def bf_encode_weights(ctx, W, d_out: int, d_in: int):
     out = _vp()
     _check(load().bf_encode_weights(ctx, _ptr(W), d_out, d_in, ctypes.byref(out)), "bf_encode_weights", ctx)
+    return out
+
+
+def bf_encode_weights_split(ctx, W, d_out: int, d_in: int, bsgs_b: int, bsgs_g: int):
+    out = _vp()
+    _check(load().bf_encode_weights_split(ctx, _ptr(W), d_out, d_in, bsgs_b, bsgs_g, ctypes.byref(out)),
+           "bf_encode_weights_split", ctx)
     return out
 
 

@@ -77,6 +77,7 @@ struct DevBuf {
 
 struct bf_weights {
     u32 d_out, d_in, n_in, n_out;
+    u32 b, g;           // baby/giant split the diagonals are grouped by (the plan's unless bf_encode_weights_split chose)
     u64* pt;            // groups pj = j*n_out + p of terms t = q*b + k in the tile-major layout `lay`;
                         // NTT domain, Montgomery form (times 2^64 mod q_i), limbs split when the primes allow
     TileLayout lay;
@@ -543,13 +544,24 @@ static u32 n_out_cts(const bf_ctx* ctx, u32 d_out) {
     return (ctx->plan.flags & BF_PLAN_COMPLEX_PACK) ? cdiv(blocks, 2) : blocks;
 }
 
-extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
-    if (!ctx) return 0;
+static u64 weights_bytes(const bf_ctx* ctx, u32 d_out, u32 d_in, u32 b, u32 g) {
     const u32 n_in = cdiv(d_in, ctx->plan.tile_D), n_out = n_out_cts(ctx, d_out);
     if (ctx->coef_cache_bits)       // one rounded coefficient per diagonal and ring position, whatever the primes
         return (u64)n_in * n_out * (ctx->plan.tile_D / ctx->plan.tau) * ctx->N * (ctx->coef_cache_bits / 8);
-    const TileLayout lay = mac_tile_layout(ctx->ring, n_out * ctx->plan.bsgs_g, n_in * ctx->plan.bsgs_b, mac_primes(ctx));
+    const TileLayout lay = mac_tile_layout(ctx->ring, n_out * g, n_in * b, mac_primes(ctx));
     return mac_tile_bytes(ctx->ring, lay);
+}
+
+extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t d_in) {
+    if (!ctx) return 0;
+    return weights_bytes(ctx, d_out, d_in, ctx->plan.bsgs_b, ctx->plan.bsgs_g);
+}
+
+// a baby/giant split the context's plan admits
+static bool split_ok(const bf_ctx* ctx, u32 b, u32 g) {
+    if (!b || !g || (b & (b - 1)) || (g & (g - 1))) return false;
+    if ((u64)b * g != ctx->plan.tile_D / ctx->plan.tau || b - 1 > (u32)MAX_ROT_BATCH) return false;
+    return !((ctx->plan.flags & BF_PLAN_MODDOWN_PER_OUTPUT) && g - 1 > (u32)MAX_ROT_BATCH);
 }
 
 // Encode diagonals [d0, d0 + count) of W (order [j][p][q][k], i.e. group pj = d / n_terms, term d % n_terms)
@@ -557,7 +569,8 @@ extern "C" uint64_t bf_weights_bytes(const bf_ctx* ctx, uint32_t d_out, uint32_t
 // The coefficients come from the encoder (W), or from a handle that keeps them (stored; W is then unused); coef_out
 // non-null: only encode, leaving the 64-bit coefficients of diagonal d0 + i at coef_out + i*N (no transform).
 static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0, u32 count, u64* dst,
-                        const TileLayout& lay, u32 pj0, const bf_weights* stored = nullptr, i64* coef_out = nullptr) {
+                        const TileLayout& lay, u32 pj0, const bf_weights* stored = nullptr, i64* coef_out = nullptr,
+                        u32 split_b = 0, u32 split_g = 0) {
     const u32 N = ctx->N, r = lay.n_primes, n = N / 2;       // (r: primes each diagonal is reduced into)
     // diagonals per pass: the encoder and the transforms gain from large batches (measured: 32 -> 128 per
     // pass takes 6 to 8 % off a call that encodes on the fly); the scratch of a pass is held to about 0.5 GB
@@ -584,8 +597,8 @@ static int encode_range(bf_ctx* ctx, const float* W, u32 d_out, u32 d_in, u32 d0
         db.complex_pack = (ctx->plan.flags & BF_PLAN_COMPLEX_PACK) ? 1u : 0u;
         db.D = ctx->plan.tile_D;
         db.tau = ctx->plan.tau;
-        db.b = ctx->plan.bsgs_b;
-        db.g = ctx->plan.bsgs_g;
+        db.b = split_b ? split_b : stored ? stored->b : ctx->plan.bsgs_b;
+        db.g = split_g ? split_g : stored ? stored->g : ctx->plan.bsgs_g;
         db.d0 = d0 + lo;
         db.count = cnt;
         const void* coef_src = ctx->coef.p;
@@ -638,9 +651,16 @@ extern "C" int bf_device_status(bf_ctx* ctx) {
 }
 
 extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, uint32_t d_in, bf_weights** out) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    return bf_encode_weights_split(ctx, W, d_out, d_in, ctx->plan.bsgs_b, ctx->plan.bsgs_g, out);
+}
+
+extern "C" int bf_encode_weights_split(bf_ctx* ctx, const float* W, uint32_t d_out, uint32_t d_in, uint32_t bsgs_b,
+                                       uint32_t bsgs_g, bf_weights** out) {
     if (!ctx || !W || !out || !d_out || !d_in) return BF_ERR_INVALID_ARG;
     *out = nullptr;
-    const u64 bytes = bf_weights_bytes(ctx, d_out, d_in);
+    if (!split_ok(ctx, bsgs_b, bsgs_g)) return BF_ERR_SHAPE;
+    const u64 bytes = weights_bytes(ctx, d_out, d_in, bsgs_b, bsgs_g);
     if (ctx->cache_budget && ctx->cache_used + bytes > ctx->cache_budget) return BF_ERR_OOM;
     bf_weights* w = new (std::nothrow) bf_weights();
     if (!w) return BF_ERR_OOM;
@@ -649,7 +669,9 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
     w->n_in = cdiv(d_in, ctx->plan.tile_D);
     w->n_out = n_out_cts(ctx, d_out);
     w->bytes = bytes;
-    w->lay = mac_tile_layout(ctx->ring, w->n_out * ctx->plan.bsgs_g, w->n_in * ctx->plan.bsgs_b, mac_primes(ctx));
+    w->b = bsgs_b;
+    w->g = bsgs_g;
+    w->lay = mac_tile_layout(ctx->ring, w->n_out * bsgs_g, w->n_in * bsgs_b, mac_primes(ctx));
     const u32 n_diag = w->n_in * w->n_out * (ctx->plan.tile_D / ctx->plan.tau);
     int s = BF_OK;
     if (ctx->coef_cache_bits) {
@@ -663,13 +685,13 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
             return BF_ERR_OOM;
         }
         if (w->coef_bits == 64) {
-            s = encode_range(ctx, W, d_out, d_in, 0, n_diag, nullptr, w->lay, 0, nullptr, (i64*)w->coef);
+            s = encode_range(ctx, W, d_out, d_in, 0, n_diag, nullptr, w->lay, 0, nullptr, (i64*)w->coef, bsgs_b, bsgs_g);
         } else {
             const u32 piece = 256;
             s = ensure(ctx, ctx->coef, (size_t)piece * ctx->N * sizeof(i64));
             for (u32 d0 = 0; d0 < n_diag && s == BF_OK; d0 += piece) {
                 const u32 cnt = n_diag - d0 < piece ? n_diag - d0 : piece;
-                s = encode_range(ctx, W, d_out, d_in, d0, cnt, nullptr, w->lay, 0, nullptr, (i64*)ctx->coef.p);
+                s = encode_range(ctx, W, d_out, d_in, d0, cnt, nullptr, w->lay, 0, nullptr, (i64*)ctx->coef.p, bsgs_b, bsgs_g);
                 if (s == BF_OK && launch_narrow_i64(ctx->ring, (const i64*)ctx->coef.p, (int*)w->coef + (size_t)d0 * ctx->N,
                                                     (size_t)cnt * ctx->N, ctx->overflow_flag, ctx->stream) != cudaSuccess)
                     s = BF_ERR_CUDA;
@@ -683,7 +705,7 @@ extern "C" int bf_encode_weights(bf_ctx* ctx, const float* W, uint32_t d_out, ui
         }
         // padding words of the layout are never read, but keep the allocation defined
         if (cudaMemsetAsync(w->pt, 0, bytes, ctx->stream) != cudaSuccess) s = BF_ERR_CUDA;
-        if (s == BF_OK) s = encode_range(ctx, W, d_out, d_in, 0, n_diag, w->pt, w->lay, 0);
+        if (s == BF_OK) s = encode_range(ctx, W, d_out, d_in, 0, n_diag, w->pt, w->lay, 0, nullptr, nullptr, bsgs_b, bsgs_g);
     }
     if (s == BF_OK) s = check_overflow(ctx);
     if (s != BF_OK) {
@@ -866,7 +888,8 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
                           const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out) {
     if (!ctx || !ct_in || !ct_out || (!pt_weights && !W_raw) || !d_out || !d_in) return BF_ERR_INVALID_ARG;
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
-    const u32 D = ctx->plan.tile_D, tau = ctx->plan.tau, b = ctx->plan.bsgs_b, g = ctx->plan.bsgs_g;
+    const u32 D = ctx->plan.tile_D, tau = ctx->plan.tau;
+    const u32 b = pt_weights ? pt_weights->b : ctx->plan.bsgs_b, g = pt_weights ? pt_weights->g : ctx->plan.bsgs_g;
     if (n_in != cdiv(d_in, D) || n_out != n_out_cts(ctx, d_out)) return BF_ERR_SHAPE;
     if (pt_weights && (pt_weights->d_out != d_out || pt_weights->d_in != d_in)) return BF_ERR_SHAPE;
     const size_t ctw = (size_t)2 * r * N;                 // words per ciphertext
@@ -1575,9 +1598,9 @@ extern "C" int bf_negacyclic_mul(bf_ctx* ctx, const uint64_t* a, const uint64_t*
 extern "C" int bf_weights_export(bf_ctx* ctx, const bf_weights* w, uint32_t p, uint32_t q, uint32_t j, uint32_t k,
                                  uint64_t* out) {
     if (!ctx || !w || !out) return BF_ERR_INVALID_ARG;
-    if (p >= w->n_out || q >= w->n_in || j >= ctx->plan.bsgs_g || k >= ctx->plan.bsgs_b) return BF_ERR_SHAPE;
+    if (p >= w->n_out || q >= w->n_in || j >= w->g || k >= w->b) return BF_ERR_SHAPE;
     const u32 N = ctx->N, r = ctx->r;
-    const size_t d = (((size_t)j * w->n_out + p) * w->n_in + q) * ctx->plan.bsgs_b + k;
+    const size_t d = (((size_t)j * w->n_out + p) * w->n_in + q) * w->b + k;
     PolyBatch B;
     memset(&B, 0, sizeof(B));
     if (w->coef) {      // coefficient form: reduce the stored integers per prime (through a transform and back)

@@ -68,9 +68,20 @@ class WorkloadRunner:
         budget = cache_budget_bytes if cache_budget_bytes is not None else self.w.cache_budget_bytes
         if budget:
             bf.bf_set_cache_budget(self.ctx, int(budget))
-        # rotation keys: uniform residues over the extended basis
-        steps = [k * self.plan.tau for k in range(1, self.plan.b)] + \
-                [j * self.plan.b * self.plan.tau for j in range(1, self.plan.g)]
+        # calls: projections that read the same activation stacked into one (q/k/v, gate/up), each with its baby/giant split
+        D = self.plan.D
+        if fuse_shared_inputs:
+            fused = wl.fuse_shared_inputs(self.w.layers, D)
+            units = [wl.Layer(nm, d_in, sum(m.d_out for m in members)) for nm, d_in, members in fused]
+            members_of = {nm: members for nm, _, members in fused}
+        else:
+            units = list(self.w.layers)
+            members_of = {L.name: [L] for L in units}
+        self.splits = {L.name: self.w.split_of(L.name, self.plan) for L in units}
+        # rotation keys for every split in use: uniform residues over the extended basis
+        steps = []
+        for b, g in sorted(set(self.splits.values()) | {(self.plan.b, self.plan.g)}):
+            steps += [k * self.plan.tau for k in range(1, b)] + [j * b * self.plan.tau for j in range(1, g)]
         self.fold_in_ciphertext = fold_in_ciphertext
         if fold_in_ciphertext:      # the variant that sums the tau partial results on the device
             steps += [1 << i for i in range(self.plan.tau.bit_length() - 1)]
@@ -84,14 +95,6 @@ class WorkloadRunner:
         self.key_bytes = len(self.rot_steps) * self.r * 2 * (self.r + 1) * self.N * 8
         # layers
         self.layers = []
-        D = self.plan.D
-        if fuse_shared_inputs:      # q/k/v and gate/up read the same activation: one call over the stacked matrix
-            units = [wl.Layer(nm, d_in, sum(m.d_out for m in members)) for nm, d_in, members in
-                     wl.fuse_shared_inputs(self.w.layers, D)]
-            members_of = {nm: members for nm, _, members in wl.fuse_shared_inputs(self.w.layers, D)}
-        else:
-            units = list(self.w.layers)
-            members_of = {L.name: [L] for L in units}
         for rep in range(self.w.n_repeat):
             for L in units:
                 n_in, n_out = wl.ceil_div(L.d_in, D), wl.ceil_div(L.d_out, self.plan.rows_per_ct)
@@ -99,16 +102,19 @@ class WorkloadRunner:
                     [wl.gen_weights(seed, f"{m.name}.{rep}", m.d_out, m.d_in) for m in members_of[L.name]], axis=0)
                 ).to(self.device)
                 handle = None
+                b, g = self.splits[L.name]
                 if cache:
                     try:
-                        handle = bf.bf_encode_weights(self.ctx, W, L.d_out, L.d_in)
+                        handle = bf.bf_encode_weights_split(self.ctx, W, L.d_out, L.d_in, b, g)
                     except bf.BifrostError as e:
                         if e.code != bf.BF_ERR_OOM:
                             raise
+                if handle is None:      # the on-the-fly path runs under the plan's own split
+                    b, g = self.plan.b, self.plan.g
                 ct_in = _uniform_residues(self.gen, self.primes, (n_in, 2), self.N, self.device)
                 ct_out = torch.empty((n_out, 2, self.r, self.N), dtype=torch.int64, device=self.device)
                 ct_low = torch.empty((n_out, 2, self.r - 1, self.N), dtype=torch.int64, device=self.device)
-                self.layers.append(dict(layer=L, rep=rep, n_in=n_in, n_out=n_out, W=W, handle=handle,
+                self.layers.append(dict(layer=L, rep=rep, n_in=n_in, n_out=n_out, b=b, g=g, W=W, handle=handle,
                                         ct_in=ct_in, ct_out=ct_out, ct_low=ct_low,
                                         pt_bytes=n_in * n_out * (D // self.plan.tau) * self.N * self.word_bytes,
                                         resident_bytes=n_in * n_out * (D // self.plan.tau) * self.N *

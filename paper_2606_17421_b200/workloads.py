@@ -68,6 +68,15 @@ class Workload:
     layers: tuple               # the distinct projections of one transformer layer
     n_repeat: int = 1           # number of transformer layers in a decode step
     cache_budget_bytes: int | None = None
+    # baby/giant splits (b, g) of single calls (by the name of the call, stacked projections joined with "+") that differ
+    # from the plan's: measured per call shape on B200 under double hoisting with one division per output, and used
+    # under that plan variant only.  Many input ciphertexts favour fewer baby steps, many outputs fewer giant steps.
+    splits: dict = field(default_factory=dict)
+
+    def split_of(self, call: str, plan: PlanSpec):
+        if plan.hoist == "double" and plan.moddown == "per_output":
+            return self.splits.get(call, (plan.b, plan.g))
+        return (plan.b, plan.g)
 
 
 GPT2_LAYER = (Layer("qkv", 768, 2304), Layer("out_proj", 768, 768),
@@ -98,10 +107,17 @@ WORKLOADS = {
     # M = 64 diagonals per tile split as 16 baby x 4 giant steps: measured fastest on B200 (fewer full
     # key switches than 8 x 8 at the price of four more rotation keys)
     "gpt2_qkv": Workload("gpt2_qkv", "n15", PlanSpec(1024, 16, 16, 4), (GPT2_LAYER[0],)),
-    "gpt2_step": Workload("gpt2_step", "n15", PlanSpec(1024, 16, 16, 4), GPT2_LAYER, n_repeat=12),
+    # (per call, ms on B200 for 16x4 / 32x2 / 8x8: ffn_down 0.547 / 0.932 / 0.525; the other three are fastest at 16x4)
+    "gpt2_step": Workload("gpt2_step", "n15", PlanSpec(1024, 16, 16, 4), GPT2_LAYER, n_repeat=12,
+                          splits={"ffn_down": (8, 8)}),
+    # (16x4 / 32x2 / 8x8: q+k+v 0.405 / 0.418 / 0.562, o 0.417 / 0.580 / 0.430, gate+up 0.505 / 0.471 / 0.766,
+    # down 0.548 / 0.926 / 0.520)
     "qwen3_step": Workload("qwen3_step", "n15", PlanSpec(1024, 16, 16, 4), QWEN3_LAYER, n_repeat=28,
-                           cache_budget_bytes=60 * 10 ** 9),
-    "llama3_layer": Workload("llama3_layer", "n16", PlanSpec(1024, 32, 8, 4), LLAMA3_8B_LAYER),
+                           cache_budget_bytes=60 * 10 ** 9, splits={"gate+up": (32, 2), "down": (8, 8)}),
+    # (8x4 / 16x2 / 4x8: q+k+v 1.85 / 1.90 / 2.58, o 1.48 / 1.67 / 1.91, gate+up 6.07 / 4.33 / 10.25 (32x1: 4.57),
+    # down 4.00 / 6.65 / 3.55 (2x16: 4.51))
+    "llama3_layer": Workload("llama3_layer", "n16", PlanSpec(1024, 32, 8, 4), LLAMA3_8B_LAYER,
+                             splits={"gate+up": (16, 2), "down": (4, 8)}),
 }
 # Tile-size study (the paper's Sec. 5.3 experiment on a 1024 x 1024 product): smaller tiles need fewer or no
 # rotations but send more ciphertexts across the TEE boundary (1024/D in, 1024/D out).
@@ -113,7 +129,8 @@ WORKLOADS["gpt2_qkv_paper_params"] = Workload("gpt2_qkv_paper_params", "paper_n1
                                               (GPT2_LAYER[0],))
 # One transformer layer of the GPT-2 step (1.2 GB of encoded weights): small enough for profiler captures that need
 # several passes, with the call shapes of the whole step (one and three input ciphertexts, one and three output blocks).
-WORKLOADS["gpt2_layer"] = Workload("gpt2_layer", "n15", PlanSpec(1024, 16, 16, 4), GPT2_LAYER)
+WORKLOADS["gpt2_layer"] = Workload("gpt2_layer", "n15", PlanSpec(1024, 16, 16, 4), GPT2_LAYER,
+                                   splits={"ffn_down": (8, 8)})
 CONFIG_ORDER = ["tiny", "gpt2_qkv", "gpt2_step", "qwen3_step", "llama3_layer"]
 
 

@@ -381,6 +381,57 @@ def test_per_output_division_refuses_more_giant_steps_than_it_can_sum():
     assert ei.value.code == bf.BF_ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("modes", [{}, BEST, dict(hoist="double")], ids=["plain", "best", "double_hoist"])
+def test_weights_with_a_split_of_their_own(modes):
+    # one context (plan 8 x 4), three handles for the same matrix with the splits 8 x 4, 16 x 2 and 2 x 16, and a
+    # coefficient-form handle with 4 x 8: every call matches the oracle run under that split; what the context
+    # refuses: a split whose product is not D / tau, one that is not a power of two, a missing key
+    from paper_2606_17421_b200 import bifrost as bf
+    par = oracle_params("n12")
+    base = ckks.Plan(64, 2, 8, 4, **modes)
+    d_out, d_in, seed = 150, 100, 21
+    W = wl.gen_weights(seed, "split", d_out, d_in)
+    x = wl.gen_activation(seed, "split", d_in)
+    s = ckks.keygen(par, seed)
+    variants = [(8, 4), (16, 2), (2, 16), (4, 8)]
+    plans = [ckks.Plan(base.D, base.tau, b, g, base.pack, base.moddown, base.hoist) for b, g in variants]
+    extra = sorted({st for pl in plans for st in ckks.required_rotations(pl)})
+    keys = ckks.make_rotation_keys(par, s, base, seed, extra_steps=extra)
+    cts = ckks.encrypt_vector(par, base, s, x, seed)
+    g = GpuSide(par, base)
+    try:
+        Wd = g.to_dev(W)
+        g.load_keys(keys)                            # the keys of the plan's own split only
+        w = g.bf.bf_encode_weights_split(g.ctx, Wd, d_out, d_in, 16, 2)
+        with pytest.raises(bf.BifrostError) as ei:
+            g.linear(cts, W, d_out, d_in, weights=w)
+        assert ei.value.code == bf.BF_ERR_MISSING_KEY
+        g.bf.bf_weights_free(g.ctx, w)
+        g.load_keys(keys, extra_steps=extra)
+        for bad in ((8, 8), (3, 11), (0, 32), (32, 0)):
+            with pytest.raises(bf.BifrostError) as ei:
+                g.bf.bf_encode_weights_split(g.ctx, Wd, d_out, d_in, *bad)
+            assert ei.value.code == bf.BF_ERR_SHAPE, bad
+        for (b, gg), plan in zip(variants, plans):
+            expect = ckks.linear(par, plan, cts, W, keys)
+            if (b, gg) == (4, 8):
+                g.bf.bf_set_coefficient_cache(g.ctx, 64)
+            w = g.bf.bf_encode_weights_split(g.ctx, Wd, d_out, d_in, b, gg)
+            g.bf.bf_set_coefficient_cache(g.ctx, 0)
+            n_out = plan.n_out(d_out)
+            ct_in = g.to_dev(np.stack(cts))
+            out = g.empty_u64(n_out, 2, par.r, par.N)
+            for call in range(3):               # direct, captured, replayed
+                out.zero_()
+                g.bf.bf_linear(g.ctx, ct_in, len(cts), w, None, d_out, d_in, out, n_out)
+            got = g.to_host_u64(out)
+            for p in range(n_out):
+                assert np.array_equal(got[p], expect[p]), (b, gg, p)
+            g.bf.bf_weights_free(g.ctx, w)
+    finally:
+        g.close()
+
+
 def test_linear_gpt2_qkv_config_bit_exact():
     w = wl.WORKLOADS["gpt2_qkv"]
     par = oracle_params(w.params)
@@ -388,33 +439,45 @@ def test_linear_gpt2_qkv_config_bit_exact():
     run_case(par, ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g), L.d_out, L.d_in, 0, 1e-3, L.name)
 
 
-def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=()):
+def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=(), splits=None):
     """Full-size calls exactly as the benchmark's runner issues them (projections that read the same
     activation stacked row-wise into one call, repeated on the same buffers so that the third call is the
     replayed graph with its concurrent key-switch chains): the device computes every output block, the
     oracle the listed ones; those must agree on every residue, before and after the rescale, and decrypt
     to the fp64 product.  Calls with the same d_in share one set of input ciphertexts, so that the
-    oracle rotates them only once."""
+    oracle rotates them only once.  splits: {call name: (b, g)}, the calls whose weights are encoded with a
+    baby/giant split of their own (as the runner does under the headline plan)."""
+    splits = splits or {}
+    assert not set(splits) & set(on_the_fly)        # the on-the-fly path runs under the plan's own split
+    base = plan
+    plans = {name: ckks.Plan(base.D, base.tau, b, g, base.pack, base.moddown, base.hoist) for name, (b, g) in splits.items()}
+    extra = sorted({st for pl in plans.values() for st in ckks.required_rotations(pl)})
     s = ckks.keygen(par, seed)
-    keys = ckks.make_rotation_keys(par, s, plan, seed)
-    units = wl.fuse_shared_inputs(layers, plan.D)
-    inputs = {}                      # d_in -> (x, ciphertexts, the oracle's baby rotations)
-    g = GpuSide(par, plan)
+    keys = ckks.make_rotation_keys(par, s, base, seed, extra_steps=extra)
+    units = wl.fuse_shared_inputs(layers, base.D)
+    inputs, rotated = {}, {}         # d_in -> (x, ciphertexts); (d_in, b) -> the oracle's baby rotations
+    g = GpuSide(par, base)
     try:
-        g.load_keys(keys)
+        g.load_keys(keys, extra_steps=extra)
         for name, d_in, members in units:
+            plan = plans.get(name, base)
             d_out = sum(m.d_out for m in members)
             W = np.concatenate([wl.gen_weights(seed, m.name, m.d_out, m.d_in) for m in members], axis=0)
             if d_in not in inputs:
                 x = wl.gen_activation(seed, f"x{d_in}", d_in)
-                cts = ckks.encrypt_vector(par, plan, s, x, seed)
+                inputs[d_in] = (x, ckks.encrypt_vector(par, base, s, x, seed))
+            x, cts = inputs[d_in]
+            if (d_in, plan.b) not in rotated:
                 rot_fn = ckks.baby_rotations_ext if plan.hoist == "double" else ckks.baby_rotations
-                inputs[d_in] = (x, cts, [rot_fn(par, plan, ct, keys) for ct in cts])
-            x, cts, X = inputs[d_in]
+                rotated[(d_in, plan.b)] = [rot_fn(par, plan, ct, keys) for ct in cts]
+            X = rotated[(d_in, plan.b)]
             n_in, n_out = len(cts), plan.n_out(d_out)
             blocks = list(blocks_of(name, n_out))
             expect = ckks.linear(par, plan, cts, W, keys, blocks=blocks, X=X)
-            w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in)
+            if name in splits:
+                w = g.bf.bf_encode_weights_split(g.ctx, g.to_dev(W), d_out, d_in, plan.b, plan.g)
+            else:
+                w = g.bf.bf_encode_weights(g.ctx, g.to_dev(W), d_out, d_in)
             ct_in = g.to_dev(np.stack(cts))
             out = g.empty_u64(n_out, 2, par.r, par.N)
             for call in range(3):               # direct, captured, replayed
@@ -447,7 +510,7 @@ def test_gpt2_step_one_whole_layer_every_block(modes):
     w = wl.WORKLOADS["gpt2_step"]
     par = oracle_params(w.params)
     plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, **modes)
-    check_blocks(par, plan, w.layers, lambda name, n_out: range(n_out), 11)
+    check_blocks(par, plan, w.layers, lambda name, n_out: range(n_out), 11, splits=w.splits if modes else None)
 
 
 @pytest.mark.parametrize("modes", [{}, BEST], ids=["plain", "best"])
@@ -462,7 +525,7 @@ def test_qwen3_step_the_calls_of_one_layer(modes):
     plan = ckks.Plan(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, **modes)
     pick = {"q+k+v": [0, 1, 2, 3], "o": [0], "gate+up": [0, 2, 3, 5], "down": [0]}
     blocks_of = (lambda name, n_out: range(n_out)) if modes else (lambda name, n_out: pick[name])
-    check_blocks(par, plan, w.layers, blocks_of, 12, on_the_fly=("o",))
+    check_blocks(par, plan, w.layers, blocks_of, 12, on_the_fly=("o",), splits=w.splits if modes else None)
 
 
 @pytest.mark.parametrize("modes", [{}, BEST], ids=["plain", "best"])
@@ -483,7 +546,10 @@ def test_llama3_layer_the_calls_the_benchmark_times(modes):
         pick = {"q+k+v": [0, 2], "o": [0, 1], "gate+up": [0, 7, 8, 13], "down": [0, 1]}
     else:
         pick = {"q+k+v": [0, 4, 5], "o": [0, 3], "gate+up": [0, 14, 21, 22, 27], "down": [0, 1, 2, 3]}
-    check_blocks(par, plan, w.layers, lambda name, n_out: pick[name], 13, on_the_fly=("down",))
+    # (under the headline plan gate+up and down run with splits of their own, 16 x 2 and 4 x 8; o is then the call
+    # that is also checked with its weights encoded on the fly)
+    check_blocks(par, plan, w.layers, lambda name, n_out: pick[name], 13, on_the_fly=("o",) if modes else ("down",),
+                 splits=w.splits if modes else None)
 
 
 def test_linear_with_the_papers_own_parameter_set():
