@@ -302,6 +302,8 @@ extern "C" int bf_ctx_create(bf_ctx** out, uint32_t N, const uint64_t* primes, u
         R.c30_d[m] = (double)((1ull << 30) % q);
         R.c30_q[m] = R.c30_d[m] / (double)q;
         R.k59_d[m] = (double)(2 * q - (1ull << 59) % q);
+        R.pinv_d[m] = m < n_ct_primes ? (double)R.pinv[m] : 0.0;
+        R.pinv_q[m] = m < n_ct_primes ? (double)R.pinv[m] / (double)q : 0.0;
         {   // constants of the encoder's fp64 load (see RingDev::enc_consts)
             const u64 c96 = h_mulmod(R.c64[m], (1ull << 32) % q, q);
             const u64 c127 = h_mulmod(R.c64[m], (1ull << 63) % q, q);

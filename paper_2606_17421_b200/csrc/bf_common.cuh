@@ -38,6 +38,7 @@ struct RingDev {
     double ninvm_d[MAX_MODULI], ninvm_q[MAX_MODULI];   // the same for N^{-1} * 2^{-64} (leaving Montgomery form)
     double c30_d[MAX_MODULI], c30_q[MAX_MODULI];       // (double)(2^30 mod q) and that over q
     double k59_d[MAX_MODULI];    // 2q - (2^59 mod q): undoes the offset of a stored centred lift, keeps it positive
+    double pinv_d[MAX_MODULI], pinv_q[MAX_MODULI];     // (double)(P^{-1} mod q_i) and that over q_i (i < r)
     // encoder output (signed 64-bit coefficients) into Montgomery form on the fp64 path: the word is
     // (hi' - 2^31) 2^32 + lo, so times 2^64 it is  hi' (2^96 mod q) + lo (2^64 mod q) - (2^127 mod q).
     // Five doubles per prime, in device memory (kernel parameters stay small): (double)(2^96 mod q), that

@@ -493,13 +493,34 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
             dc.q = R.q[i];
             dc.mu = R.mu[i];
             dc.lift_mod = R.q[R.r];
-            dc.lift_red = barrett64(dc.lift_mod, dc.q, dc.mu);
             const u64* tp = B.div_t + (size_t)(o / B.o_div) * B.div_so;
-            const u64 pinv = R.pinv[i], pinvs = R.pinvs[i];
-            for (int w = threadIdx.x; w < POINTS; w += blockDim.x) {
-                const size_t idx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1));
-                const u64 t = load_src<LOAD_CENTRED>(tp, idx, dc);
-                staged[w] = mul_shoup(sub_mod(src[idx], t, dc.q), pinv, pinvs, dc.q);
+            if (R.fp_ok[i]) {
+                // in fp64 (every value an exact integer): t lazily reduced by the load functor, the difference times
+                // P^{-1} as a centred product, brought to [0, q) -- the digit must be the canonical residue, since it is
+                // reduced into the other primes next
+                const double qd = R.qd[i], pv = R.pinv_d[i], pq = R.pinv_q[i];
+                dc.qd = qd;
+                dc.c30 = R.c30_d[i];
+                dc.c30q = R.c30_q[i];
+                dc.wide = (dc.q >> 41) != 0;
+                dc.k59 = dc.wide ? R.k59_d[i] : __dsub_rn(R.k59_d[i], __dadd_rn(qd, qd));
+                const double q3 = __dadd_rn(__dadd_rn(qd, qd), qd);
+                for (int w = threadIdx.x; w < POINTS; w += blockDim.x) {
+                    const size_t idx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1));
+                    const double t = load_src_fp<LOAD_CENTRED>(tp, idx, dc);       // (-1.75q, 0.76q), or (0.25q, 2.76q) when wide
+                    const double x = __dsub_rn(u2d(src[idx]), t);
+                    double s2 = dc.wide ? fp_mul_centred(__dadd_rn(x, q3), pv, pq, qd) : fp_mul_centred_signed(x, pv, pq, qd);
+                    if (s2 < 0.0) s2 = __dadd_rn(s2, qd);
+                    staged[w] = d2u(s2);
+                }
+            } else {
+                dc.lift_red = barrett64(dc.lift_mod, dc.q, dc.mu);
+                const u64 pinv = R.pinv[i], pinvs = R.pinvs[i];
+                for (int w = threadIdx.x; w < POINTS; w += blockDim.x) {
+                    const size_t idx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1));
+                    const u64 t = load_src<LOAD_CENTRED>(tp, idx, dc);
+                    staged[w] = mul_shoup(sub_mod(src[idx], t, dc.q), pinv, pinvs, dc.q);
+                }
             }
         } else {
             for (int w = threadIdx.x; w < POINTS; w += blockDim.x)
