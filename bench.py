@@ -34,16 +34,18 @@ UNIT = "ms"
 # the device), so the figures come from one GPT-2 layer under the same plan (same kernels, same call shapes), whose
 # traffic grows in proportion to the streamed bytes; `traffic` in the line = this ratio x the algorithmic bytes of a launch.
 NCU_TRAFFIC_RATIO = {
-    "mac": 1.12,                  # 293.6 MB read + 7.3 MB written for 268.4 MB of cached words (X tiles and outputs on top)
-    "key_inner_product": 1.28,    # eight captured launches: 1954.9 MB for 52 distinct keys of 29.36 MB (digit sets, outputs)
+    "mac": 1.32,                  # eight captured launches (four calls): 1417 MB for 1074 MB of cached words (rotated inputs, outputs)
+    "key_inner_product": 1.40,    # eight captured launches: 1352 MB for 33 distinct keys of 29.36 MB (digit sets, outputs)
 }
+# (ncu flushes the caches before every captured launch: rotated inputs and digit sets that a step finds in L2 count as
+# DRAM traffic in these ratios)
 # Executed warp instructions per butterfly by pipe, from the same captures (profiles/gpt2_layer_headline_plan_kernels_ncu.md),
 # to set beside the modelled 8 / 12 / 10 operations: the large fp64-path batches of each direction.
 NCU_PIPE_INSTR = {
-    "ntt_forward": {"all": 25.2, "fp64": 7.7, "alu": 7.0, "fma_integer": 5.7, "lsu": 2.3,
-                    "from": "giant ModUp of 21 rotations, both passes"},
+    "ntt_forward": {"all": 27.2, "fp64": 8.2, "alu": 7.4, "fma_integer": 6.1, "lsu": 2.4,
+                    "from": "hoisted ModUp of three inputs (147 transforms), both passes"},
     "ntt_inverse": {"all": 21.0, "fp64": 10.3, "alu": 3.9, "fma_integer": 2.0, "lsu": 2.3,
-                    "from": "c1 of 3 giant rotations x 7 primes, both passes"},
+                    "from": "c1 of 3 giant rotations x 7 primes, both passes (an earlier capture of the same kernels)"},
 }
 
 
