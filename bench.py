@@ -313,6 +313,9 @@ class Measurement:
                          "frac": round(ach / hbm_peak, 4), "of": peak_kind, "traffic": traffic_of("mac", mac_bytes),
                          "launches_per_step": mac_n, "avg_ms": round(mac_ms, 5),
                          "bytes_per_launch": round(mac_bytes), "frac_of_nominal_8000": round(ach / 8000.0, 4)}
+            if R.plan.hoist == "double":
+                rl["mac"]["note"] = ("a call's two launches (ciphertext primes; the special prime beside it on a second "
+                                     "stream) are timed as one span, the way they run; avg_ms = that span / 2")
         # key-switch inner product: algorithmic bytes = every distinct key of a launch once
         ki_ms, ki_n = avg_ms("key_inner_product")
         if ki_ms:

@@ -756,7 +756,8 @@ static Lane main_lane(bf_ctx* ctx) {
 
 static int ensure_lanes(bf_ctx* ctx) {
     if (!ctx->ev_fork) CK(cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
-    for (int i = 0; i + 1 < ctx->n_lanes; ++i) {
+    const int n_side = ctx->n_lanes > 2 ? ctx->n_lanes - 1 : 1;       // (one side stream at least: the special prime's MAC)
+    for (int i = 0; i < n_side && i + 1 < bf_ctx::MAX_LANES; ++i) {
         if (!ctx->side[i]) CK(cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking));
         if (!ctx->ev_join[i]) CK(cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming));
     }
@@ -1045,7 +1046,10 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     if (pt_weights && pt_weights->pt) {
         // double hoisting: the launch for the special prime (one eighth of the words, on whole-word arithmetic) runs
         // beside the launch for the ciphertext primes
-        const bool beside = dh && lanes > 1;
+        // (also while single launches are being timed, chains serialised: the pair is then timed as one span, the way
+        // it runs)
+        const bool beside = dh && (lanes > 1 || ctx->prof.timing);
+        ProfSpan span(beside ? &ctx->prof : nullptr, CAT_MAC, ctx->stream);
         if (beside) TRY(fork_lanes(ctx, 2));
         CK(launch_mac(ctx->ring, pt_weights->pt, pt_weights->lay, X, mac_out, n_pj, n_terms, true, ctx->device_error, ctx->stream,
                       beside ? ctx->side[0] : nullptr, &msc));

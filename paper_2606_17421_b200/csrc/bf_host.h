@@ -31,6 +31,7 @@ struct Profiler {
     struct Rec { int cat; cudaEvent_t a, b; };
     std::vector<Rec> recs;            // event pairs recorded since the last collection
     std::vector<cudaEvent_t> pool;    // idle events
+    bool span_open = false;           // a ProfSpan is timing the launches inside it as one
     cudaEvent_t get();
 };
 
@@ -39,6 +40,14 @@ struct ProfScope {
     Profiler* p; int cat; cudaStream_t s; cudaEvent_t a = nullptr;
     ProfScope(Profiler* prof, int c, cudaStream_t st);
     ~ProfScope();
+};
+
+// Times a group of launches that run side by side as one span on stream st (from everything before the group to
+// everything after its join); the launches inside are still counted by their own ProfScope, but not timed singly.
+struct ProfSpan {
+    Profiler* p; int cat; cudaStream_t s; cudaEvent_t a = nullptr;
+    ProfSpan(Profiler* prof, int c, cudaStream_t st);
+    ~ProfSpan();
 };
 
 struct RingHost {

@@ -29,7 +29,7 @@ cudaEvent_t Profiler::get() {
 ProfScope::ProfScope(Profiler* prof, int c, cudaStream_t st) : p(prof), cat(c), s(st) {
     if (!p) return;
     p->launches[cat]++;
-    if (p->timing) {
+    if (p->timing && !p->span_open) {
         a = p->get();
         cudaEventRecord(a, s);
     }
@@ -40,6 +40,21 @@ ProfScope::~ProfScope() {
     cudaEvent_t b = p->get();
     cudaEventRecord(b, s);
     p->recs.push_back({cat, a, b});
+}
+
+ProfSpan::ProfSpan(Profiler* prof, int c, cudaStream_t st) : p(prof), cat(c), s(st) {
+    if (!p || !p->timing) return;
+    a = p->get();
+    cudaEventRecord(a, s);
+    p->span_open = true;
+}
+
+ProfSpan::~ProfSpan() {
+    if (!p || !a) return;
+    cudaEvent_t b = p->get();
+    cudaEventRecord(b, s);
+    p->recs.push_back({cat, a, b});
+    p->span_open = false;
 }
 
 struct LoadConsts {
