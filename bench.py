@@ -5,8 +5,8 @@ timed beside it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload qwen3_step@budget=60] [--impl reference]
 
-A step = one decode token's worth of the workload: bf_linear + bf_rescale for every linear layer
-of the workload, cached encoded weights streamed from HBM (49 GB per step for the Qwen3-0.6B-shaped
+A step = one decode token's worth of the workload: the encrypted product and its rescale
+(bf_linear_rescaled: bf_linear + bf_rescale as one call) for every linear layer of the workload, cached encoded weights streamed from HBM (49 GB per step for the Qwen3-0.6B-shaped
 default, 352 MB for the single GPT-2 projection: always larger than L2, so consecutive steps cannot
 be served from cache).  The other configurations are timed after the main one and reported under
 "other_workloads", each with its own rooflines.  Inputs are seeded and synthetic.

@@ -138,6 +138,15 @@ void bf_weights_free(bf_ctx* ctx, bf_weights* w);
 int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
               const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out);
 
+/* bf_linear followed by bf_rescale from the full level (Sec. 2.1 rescaling; the decode loop of Alg. 3 rescales every
+ * product), as one call: ct_low receives n_out ciphertexts of r-1 primes, boundary layout [2][r-1][N], the same residues
+ * as the two calls in turn.  Where the plan ends the product in an element-wise kernel (double hoisting with one
+ * division per output) the rescale happens inside it; the full-level result then never reaches memory the caller sees.
+ * scale_inout (host, may be NULL) is divided by the dropped prime.  Same errors as bf_linear; BF_ERR_LEVEL if r < 2. */
+int bf_linear_rescaled(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
+                       const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_low, uint32_t n_out,
+                       double* scale_inout);
+
 /* Cache compression (Sec. 6.1 names the encoded-weight cache as the memory wall).  With
  * bf_set_compact_cache(ctx, 1) every weight encoded afterwards, cached or on the fallback path, is
  * held in the narrowest word format its prime allows: 4 bytes per word for primes below 2^32, 5

@@ -59,6 +59,7 @@ _SIGNATURES = {
     "bf_encode_weights_split": (ctypes.c_int, [_vp, _vp, _u32, _u32, _u32, _u32, ctypes.POINTER(_vp)]),
     "bf_weights_free": (None, [_vp, _vp]),
     "bf_linear": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32]),
+    "bf_linear_rescaled": (ctypes.c_int, [_vp, _vp, _u32, _vp, _vp, _u32, _u32, _vp, _u32, ctypes.POINTER(ctypes.c_double)]),
     "bf_device_status": (ctypes.c_int, [_vp]),
     "bf_set_graph_replay": (ctypes.c_int, [_vp, ctypes.c_int]),
     "bf_set_dependent_launch": (ctypes.c_int, [_vp, ctypes.c_int]),
@@ -218,6 +219,15 @@ def bf_rescale(ctx, ct_in, ct_out, n_ct: int, level: int, scale: float | None = 
     s = ctypes.c_double(scale if scale is not None else 0.0)
     _check(load().bf_rescale(ctx, _ptr(ct_in), _ptr(ct_out), n_ct, level,
                              ctypes.byref(s) if scale is not None else None), "bf_rescale", ctx)
+    return s.value if scale is not None else None
+
+
+def bf_linear_rescaled(ctx, ct_in, n_in: int, pt_weights, W_raw, d_out: int, d_in: int, ct_low, n_out: int,
+                       scale: float | None = None):
+    """Returns the new scale when `scale` is given."""
+    s = ctypes.c_double(scale if scale is not None else 0.0)
+    _check(load().bf_linear_rescaled(ctx, _ptr(ct_in), n_in, pt_weights, _ptr(W_raw), d_out, d_in, _ptr(ct_low), n_out,
+                                     ctypes.byref(s) if scale is not None else None), "bf_linear_rescaled", ctx)
     return s.value if scale is not None else None
 
 

@@ -115,7 +115,7 @@ struct bf_ctx {
     u32 n_keys = 0;
     // scratch (grow-only)
     size_t dig_half = 0;            // words from a digit set in Dig to its staging twin
-    DevBuf X, X0, Aext, Dig, U, Ubig, Tc, Tn, Cc, A, Rres, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
+    DevBuf X, X0, Aext, Dig, U, Ubig, Tc, Tn, Cc, A, Rres, Lfull, fft, coef, ptnat, ptjit, stage_in, stage_out, nm_a, nm_b;
     u64 cache_budget = 0, cache_used = 0;
     std::vector<bf_weights*> weights;
     std::string cuda_msg;
@@ -131,7 +131,9 @@ struct bf_ctx {
     struct GraphKey {
         const void *ct_in, *weights, *ct_out;
         u32 d_out, d_in;
+        bool rescaled;
         bool operator<(const GraphKey& o) const {
+            if (rescaled != o.rescaled) return rescaled < o.rescaled;
             if (ct_in != o.ct_in) return ct_in < o.ct_in;
             if (weights != o.weights) return weights < o.weights;
             if (ct_out != o.ct_out) return ct_out < o.ct_out;
@@ -412,7 +414,7 @@ extern "C" void bf_ctx_destroy(bf_ctx* ctx) {
             delete w;
         }
     }
-    DevBuf* bufs[] = {&ctx->X, &ctx->X0, &ctx->Aext, &ctx->Dig, &ctx->U, &ctx->Ubig, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres,
+    DevBuf* bufs[] = {&ctx->X, &ctx->X0, &ctx->Aext, &ctx->Dig, &ctx->U, &ctx->Ubig, &ctx->Tc, &ctx->Tn, &ctx->Cc, &ctx->A, &ctx->Rres, &ctx->Lfull,
                       &ctx->fft, &ctx->coef, &ctx->ptnat, &ctx->ptjit, &ctx->stage_in, &ctx->stage_out, &ctx->nm_a, &ctx->nm_b};
     for (DevBuf* b : bufs) free_buf(*b);
     cudaFree(ctx->tw_fwd);
@@ -887,9 +889,23 @@ static u32 giant_batch(const bf_ctx* ctx) {
     return (u32)nrot;
 }
 
+static void rescale_consts(const bf_ctx* ctx, u32 level, RescaleConsts& rc) {
+    memset(&rc, 0, sizeof(rc));
+    const u64 qL = ctx->ring.q[level - 1];
+    for (u32 i = 0; i + 1 < level; ++i) {
+        const u64 q = ctx->ring.q[i];
+        rc.inv[i] = h_invmod(qL % q, q);
+        rc.invs[i] = h_shoup(rc.inv[i], q);
+        rc.qlmod[i] = qL % q;
+    }
+}
+
+// ct_low non-null: the result is rescaled on the way ([n_out][2][r-1][N] at ct_low; ct_out is not used): fused into the
+// last kernel where the plan ends in an element-wise kernel, else as the rescale kernel behind the call.
 static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
-                          const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out) {
-    if (!ctx || !ct_in || !ct_out || (!pt_weights && !W_raw) || !d_out || !d_in) return BF_ERR_INVALID_ARG;
+                          const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out,
+                          uint64_t* ct_low = nullptr) {
+    if (!ctx || !ct_in || (!ct_out && !ct_low) || (!pt_weights && !W_raw) || !d_out || !d_in) return BF_ERR_INVALID_ARG;
     const u32 N = ctx->N, r = ctx->r, nb = r + 1;
     const u32 D = ctx->plan.tile_D, tau = ctx->plan.tau;
     const u32 b = pt_weights ? pt_weights->b : ctx->plan.bsgs_b, g = pt_weights ? pt_weights->g : ctx->plan.bsgs_g;
@@ -939,6 +955,12 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
         TRY(ensure(ctx, ctx->Aext, (size_t)n_out * g * xw * 8));
     }
     TRY(ensure(ctx, ctx->A, (size_t)n_out * g * ctw * 8));
+    if (ct_low) {                   // the full-level result is an intermediate
+        TRY(ensure(ctx, ctx->Lfull, (size_t)n_out * ctw * 8));
+        ct_out = (u64*)ctx->Lfull.p;
+    }
+    RescaleConsts rcs;
+    if (ct_low) rescale_consts(ctx, r, rcs);
     // one division by P per output: the inner products of all giant rotations stay alive until every chain is done
     const bool per_output = (ctx->plan.flags & BF_PLAN_MODDOWN_PER_OUTPUT) && n_giant > 0;
     TRY(ensure(ctx, ctx->Rres, (size_t)(per_output ? n_out : n_giant ? n_giant : 1) * ctw * 8));
@@ -1231,7 +1253,8 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
             B.mod_step = 1;
             CK(ntt_inverse_gathersum(ctx->ring, B, n_out, rb, epi, ctx->stream));
             if (beside) TRY(join_lanes(ctx, 2));
-            CK(finish_division(ctx->ring, ct_out, (long long)ctw, (const u64*)ctx->Tc.p, n_t, n_out, ctx->stream));
+            CK(finish_division(ctx->ring, ct_out, (long long)ctw, (const u64*)ctx->Tc.p, n_t, n_out, ctx->stream,
+                               ct_low ? &rcs : nullptr, ct_low));
             stamp(ctx, 3);
             stamp(ctx, 4);
             if (!pt_weights) TRY(check_overflow(ctx));
@@ -1295,6 +1318,7 @@ static int linear_enqueue(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, con
     B.sum_terms = per_output ? 1 : g - 1;
     B.sum_stride = (long long)n_out * ctw;
     CK(ntt_inverse(ctx->ring, B, n_out, ctx->stream));
+    if (ct_low) CK(launch_rescale(ctx->ring, ct_out, ct_low, n_out, r, rcs.inv, rcs.invs, rcs.qlmod, ctx->stream));
     stamp(ctx, 4);
     if (!pt_weights) TRY(check_overflow(ctx));
     (void)nb;
@@ -1312,8 +1336,27 @@ static void destroy_graphs(bf_ctx* ctx) {
 // 20-odd dependent launches then cost one submission and lose their launch gaps.  Not used on the
 // fallback path (it synchronises to read the encoder's range flag), while per-launch or per-stage
 // timing is on, or when the caller's stream is itself being captured.
+static int linear_call(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
+                       const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out, bool rescaled);
+
 extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
                          const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out) {
+    return linear_call(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out, false);
+}
+
+extern "C" int bf_linear_rescaled(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
+                                  const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_low, uint32_t n_out,
+                                  double* scale_inout) {
+    if (!ctx) return BF_ERR_INVALID_ARG;
+    if (ctx->r < 2) return BF_ERR_LEVEL;
+    TRY(linear_call(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_low, n_out, true));
+    if (scale_inout) *scale_inout /= (double)ctx->ring.q[ctx->r - 1];
+    return BF_OK;
+}
+
+// (out: ct_out of bf_linear, or ct_low of bf_linear_rescaled)
+static int linear_call(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, const bf_weights* pt_weights,
+                       const float* W_raw, uint32_t d_out, uint32_t d_in, uint64_t* ct_out, uint32_t n_out, bool rescaled) {
     if (!ctx) return BF_ERR_INVALID_ARG;
     bool eligible = ctx->use_graphs && pt_weights && !ctx->timing && !ctx->prof.timing && ct_in && ct_out;
     if (eligible) {
@@ -1323,9 +1366,9 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
             eligible = false;
         }
     }
-    if (!eligible) return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
+    if (!eligible) return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, rescaled ? nullptr : ct_out, n_out, rescaled ? ct_out : nullptr);
     if (ctx->graphs.size() > 4096) destroy_graphs(ctx);
-    bf_ctx::GraphKey key{ct_in, pt_weights, ct_out, d_out, d_in};
+    bf_ctx::GraphKey key{ct_in, pt_weights, ct_out, d_out, d_in, rescaled};
     bf_ctx::GraphEntry& ge = ctx->graphs[key];
     if (ge.exec && ge.epoch == ctx->epoch) {
         CK(cudaGraphLaunch(ge.exec, ctx->stream));
@@ -1342,7 +1385,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     if (ge.unusable || ge.seen == 0 || ge.epoch != ctx->epoch) {
         // first call with these arguments (or first since a change): run directly, which also grows
         // whatever scratch the shape needs
-        const int rc = linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
+        const int rc = linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, rescaled ? nullptr : ct_out, n_out, rescaled ? ct_out : nullptr);
         if (rc == BF_OK) { ge.seen = 1; ge.epoch = ctx->epoch; }
         return rc;
     }
@@ -1353,12 +1396,12 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
     if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         cudaGetLastError();
         ge.unusable = true;
-        return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
+        return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, rescaled ? nullptr : ct_out, n_out, rescaled ? ct_out : nullptr);
     }
     // measured: inside a replayed graph plain edges are as fast as programmatic ones, so capture those
     const bool dependent = ctx->ring.dependent_launch;
     ctx->ring.dependent_launch = false;
-    const int rc = linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
+    const int rc = linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, rescaled ? nullptr : ct_out, n_out, rescaled ? ct_out : nullptr);
     ctx->ring.dependent_launch = dependent;
     cudaGraph_t graph = nullptr;
     const cudaError_t ec = cudaStreamEndCapture(ctx->stream, &graph);
@@ -1370,7 +1413,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         ctx->prof.key_bytes_per_rotation = kr_before;
         ge.unusable = true;
         if (rc != BF_OK) return rc;      // argument errors are reported as usual
-        return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
+        return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, rescaled ? nullptr : ct_out, n_out, rescaled ? ct_out : nullptr);
     }
     cudaGraphExec_t exec = nullptr;
     const cudaError_t ei = cudaGraphInstantiate(&exec, graph, 0);
@@ -1381,7 +1424,7 @@ extern "C" int bf_linear(bf_ctx* ctx, const uint64_t* ct_in, uint32_t n_in, cons
         ctx->prof.key_bytes_distinct = kd_before;
         ctx->prof.key_bytes_per_rotation = kr_before;
         ge.unusable = true;
-        return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, ct_out, n_out);
+        return linear_enqueue(ctx, ct_in, n_in, pt_weights, W_raw, d_out, d_in, rescaled ? nullptr : ct_out, n_out, rescaled ? ct_out : nullptr);
     }
     for (int c = 0; c < (int)CAT_COUNT; ++c) ge.launches[c] = ctx->prof.launches[c] - before[c];
     ge.key_bytes_distinct = ctx->prof.key_bytes_distinct - kd_before;
@@ -1436,14 +1479,9 @@ extern "C" int bf_rescale(bf_ctx* ctx, const uint64_t* ct_in, uint64_t* ct_out, 
     if (!ctx || !ct_in || !ct_out || !n_ct) return BF_ERR_INVALID_ARG;
     if (level < 2 || level > ctx->r) return BF_ERR_LEVEL;
     const u64 qL = ctx->ring.q[level - 1];
-    u64 inv[MAX_MODULI], invs[MAX_MODULI], qlmod[MAX_MODULI];
-    for (u32 i = 0; i + 1 < level; ++i) {
-        const u64 q = ctx->ring.q[i];
-        inv[i] = h_invmod(qL % q, q);
-        invs[i] = h_shoup(inv[i], q);
-        qlmod[i] = qL % q;
-    }
-    CK(launch_rescale(ctx->ring, ct_in, ct_out, n_ct, level, inv, invs, qlmod, ctx->stream));
+    RescaleConsts rc;
+    rescale_consts(ctx, level, rc);
+    CK(launch_rescale(ctx->ring, ct_in, ct_out, n_ct, level, rc.inv, rc.invs, rc.qlmod, ctx->stream));
     if (scale_inout) *scale_inout /= (double)qL;
     return BF_OK;
 }
@@ -1456,8 +1494,8 @@ extern "C" int bf_linear_host(bf_ctx* ctx, const uint64_t* host_ct_in, uint32_t 
     TRY(ensure(ctx, ctx->stage_in, (size_t)n_in * ctw * 8));
     TRY(ensure(ctx, ctx->stage_out, (size_t)n_out * ctw * 8));
     CK(cudaMemcpyAsync(ctx->stage_in.p, host_ct_in, (size_t)n_in * ctw * 8, cudaMemcpyHostToDevice, ctx->stream));
-    TRY(bf_linear(ctx, (const u64*)ctx->stage_in.p, n_in, pt_weights, W_raw, d_out, d_in, (u64*)ctx->stage_out.p, n_out));
-    TRY(bf_rescale(ctx, (const u64*)ctx->stage_out.p, (u64*)ctx->stage_out.p, n_out, ctx->r, nullptr));
+    TRY(bf_linear_rescaled(ctx, (const u64*)ctx->stage_in.p, n_in, pt_weights, W_raw, d_out, d_in, (u64*)ctx->stage_out.p,
+                           n_out, nullptr));
     const size_t out_bytes = (size_t)n_out * 2 * (ctx->r - 1) * ctx->N * 8;
     CK(cudaMemcpyAsync(host_ct_out, ctx->stage_out.p, out_bytes, cudaMemcpyDeviceToHost, ctx->stream));
     return check_overflow(ctx);          // synchronises; reports a device-side wait that gave up

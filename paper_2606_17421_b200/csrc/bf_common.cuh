@@ -284,6 +284,11 @@ struct MacScatter {
     int key[MAX_ROT_BATCH + 1];   // key (permutation table) of giant step j
 };
 
+// Constants of a rescale from `level` primes: q_L^{-1} mod q_i with its Shoup companion, and q_L mod q_i (i < level - 1).
+struct RescaleConsts {
+    u64 inv[MAX_MODULI], invs[MAX_MODULI], qlmod[MAX_MODULI];
+};
+
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks
 // each stream one contiguous region:  word (group pj, term t, prime i, coefficient n) has index
 //   ((pj%PL)*TS + t%TS)*TN + n%TN   inside stage   ((i, n/TN), pj/PL, t/TS)

@@ -93,8 +93,9 @@ cudaError_t ntt_inverse_gathersum(const RingHost& ring, const PolyBatch& B, u32 
                                   const ModDownEpilogue& epi, cudaStream_t stream);
 // ct[p][comp][i] = (ct[p][comp][i] - sum of the centred P-residues T[p][.]) * P^{-1}: the division that ends the output
 // assembly in the extended basis (ModDownEpilogue::assemble names the n_t polynomials of T per output)
+// rc, low non-null: the rescale from r primes follows in the same kernel; the result goes to low ([n_out][2][r-1][N])
 cudaError_t finish_division(const RingHost& ring, u64* ct, long long ct_stride, const u64* T, u32 n_t, u32 n_out,
-                            cudaStream_t stream);
+                            cudaStream_t stream, const RescaleConsts* rc = nullptr, u64* low = nullptr);
 cudaError_t ntt_forward_split(const RingHost& ring, const PolyBatch& B, u32 n_outer, int load, u64* final_dst,
                               const u32* scatter, u32 scatter_div, cudaStream_t stream);
 

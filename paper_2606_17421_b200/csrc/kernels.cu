@@ -703,9 +703,6 @@ cudaError_t launch_key_inner_product(const RingHost& ring, const RotBatch& rb, c
 // Every address a thread touches is congruent to its coefficient index modulo N, and it reads all
 // residues of that coefficient before writing, so one ciphertext can be rescaled in place even
 // though the output is packed more tightly ([2][level-1][N]).
-struct RescaleConsts {
-    u64 inv[MAX_MODULI], invs[MAX_MODULI], qlmod[MAX_MODULI];
-};
 
 // `in` and `out` may alias, hence no __restrict__.  When they do and several ciphertexts are
 // rescaled, the launch uses one thread per coefficient that walks the ciphertexts in order

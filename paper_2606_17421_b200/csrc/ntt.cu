@@ -1133,8 +1133,11 @@ cudaError_t ntt_inverse_gathersum(const RingHost& ring, const PolyBatch& B, u32 
 // component, the sum of all terms modulo every q_i (in ct) and each separately rounded term's residue modulo P as a
 // centred lift plus 2^59 (in T, n_t polynomials per output, indexed as ModDownEpilogue::assemble lists them):
 //   ct[p][comp][i][n] = (ct[p][comp][i][n] - sum_terms t_term[n]) * P^{-1}  (mod q_i)
+// low non-null: the rescale (Sec. 2.1) follows in the same thread, which holds all residues of its coefficient: the
+// result goes to low[p][comp][r-1][N] as c'_i = (c_i - centred(c_{r-1})) * q_{r-1}^{-1} and ct only held the sums.
 __global__ void __launch_bounds__(256) finish_division_kernel(const RingDev R, u64* __restrict__ ct, long long ct_stride,
-                                                              const u64* __restrict__ T, u32 n_t) {
+                                                              const u64* __restrict__ T, u32 n_t, const RescaleConsts rc,
+                                                              u64* __restrict__ low) {
     grid_dependency_enter();
     const u32 n = blockIdx.x * 256 + threadIdx.x;
     const u32 p = blockIdx.y >> 1, comp = blockIdx.y & 1;
@@ -1165,14 +1168,36 @@ __global__ void __launch_bounds__(256) finish_division_kernel(const RingDev R, u
     }
 #pragma unroll
     for (int i = 0; i < MAX_MODULI; ++i)
-        if ((u32)i < R.r) cp[(size_t)i * R.N] = mul_shoup(v[i], R.pinv[i], R.pinvs[i], R.q[i]);
+        if ((u32)i < R.r) v[i] = mul_shoup(v[i], R.pinv[i], R.pinvs[i], R.q[i]);
+    if (!low) {
+#pragma unroll
+        for (int i = 0; i < MAX_MODULI; ++i)
+            if ((u32)i < R.r) cp[(size_t)i * R.N] = v[i];
+        return;
+    }
+    u64 t = 0;                      // the residue that is dropped
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i)
+        if ((u32)i == R.r - 1) t = v[i];
+    const bool high = t > (R.q[R.r - 1] - 1) / 2;
+    u64* lp = low + ((size_t)p * 2 + comp) * (R.r - 1) * R.N + n;
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i)
+        if ((u32)i + 1 < R.r) {
+            const u64 q = R.q[i];
+            u64 tq = barrett64(t, q, R.mu[i]);
+            if (high) tq = sub_mod(tq, rc.qlmod[i], q);
+            lp[(size_t)i * R.N] = mul_shoup(sub_mod(v[i], tq, q), rc.inv[i], rc.invs[i], q);
+        }
 }
 
 cudaError_t finish_division(const RingHost& ring, u64* ct, long long ct_stride, const u64* T, u32 n_t, u32 n_out,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, const RescaleConsts* rc, u64* low) {
     ProfScope prof(ring.prof, CAT_DIVIDE, stream);
+    RescaleConsts none;
+    memset(&none, 0, sizeof(none));
     launch_dependent(ring, finish_division_kernel, dim3(ring.dev.N / 256, n_out * 2), dim3(256), 0, stream, ring.dev, ct,
-                     ct_stride, T, n_t);
+                     ct_stride, T, n_t, rc ? *rc : none, rc ? low : (u64*)nullptr);
     return cudaGetLastError();
 }
 

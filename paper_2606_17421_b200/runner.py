@@ -123,13 +123,17 @@ class WorkloadRunner:
 
     # ------------------------------------------------------------------ one decode token
     def step(self):
-        """All linear layers of the workload once: bf_linear + bf_rescale per layer (device buffers)."""
+        """All linear layers of the workload once: the product and its rescale per layer (device buffers), as the one
+        call that does both unless the in-ciphertext fold sits between them."""
         for e in self.layers:
             L = e["layer"]
+            if not self.fold_in_ciphertext:
+                bf.bf_linear_rescaled(self.ctx, e["ct_in"], e["n_in"], e["handle"], None if e["handle"] else e["W"],
+                                      L.d_out, L.d_in, e["ct_low"], e["n_out"])
+                continue
             bf.bf_linear(self.ctx, e["ct_in"], e["n_in"], e["handle"], None if e["handle"] else e["W"],
                          L.d_out, L.d_in, e["ct_out"], e["n_out"])
-            if self.fold_in_ciphertext:
-                bf.bf_fold(self.ctx, e["ct_out"], e["n_out"])
+            bf.bf_fold(self.ctx, e["ct_out"], e["n_out"])
             bf.bf_rescale(self.ctx, e["ct_out"], e["ct_low"], e["n_out"], self.r)
 
     def make_host_buffers(self):

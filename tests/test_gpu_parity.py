@@ -212,6 +212,16 @@ def run_case(par, plan, d_out, d_in, seed, tol, tag, tight=1e-5):
         h_out = torch.empty((n_out, 2, par.r - 1, par.N), dtype=torch.int64).pin_memory()
         g.bf.bf_linear_host(g.ctx, h_in, len(cts), w, None, d_out, d_in, h_out, n_out)
         assert np.array_equal(h_out.numpy().view(np.uint64), low)
+        # product and rescale as one call: cached (direct, captured, replayed) and on the fly
+        low_fused = g.empty_u64(n_out, 2, par.r - 1, par.N)
+        for call in range(3):
+            low_fused.zero_()
+            assert g.bf.bf_linear_rescaled(g.ctx, ct_in, len(cts), w, None, d_out, d_in, low_fused, n_out,
+                                           par.scale * par.scale) == scale
+        assert np.array_equal(g.to_host_u64(low_fused), low)
+        low_fused.zero_()
+        g.bf.bf_linear_rescaled(g.ctx, ct_in, len(cts), None, Wd, d_out, d_in, low_fused, n_out)
+        assert np.array_equal(g.to_host_u64(low_fused), low)
     finally:
         g.close()
 
@@ -490,7 +500,15 @@ def check_blocks(par, plan, layers, blocks_of, seed, on_the_fly=(), splits=None)
                 del fly
             low = g.empty_u64(n_out, 2, par.r - 1, par.N)
             scale = g.bf.bf_rescale(g.ctx, out, low, n_out, par.r, par.scale * par.scale)
-            got, low = g.to_host_u64(out), g.to_host_u64(low)
+            # the call the runner makes: product and rescale in one (direct, captured, replayed)
+            low_fused = g.empty_u64(n_out, 2, par.r - 1, par.N)
+            for call in range(3):
+                low_fused.zero_()
+                scale_fused = g.bf.bf_linear_rescaled(g.ctx, ct_in, n_in, w, None, d_out, d_in, low_fused, n_out,
+                                                      par.scale * par.scale)
+            assert scale_fused == scale
+            got, low, low_fused = g.to_host_u64(out), g.to_host_u64(low), g.to_host_u64(low_fused)
+            assert np.array_equal(low_fused, low), name       # every output ciphertext
             g.bf.bf_weights_free(g.ctx, w)
             y_ref = W.astype(np.float64) @ x
             for p in blocks:
