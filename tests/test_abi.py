@@ -38,3 +38,20 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(bifrost, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libbifrost.so"))
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         bifrost.load()
+
+
+def test_workload_splits_name_calls_and_factor_the_diagonals():
+    # the per-call baby/giant splits of the workloads: every name is a call the runner issues (projections that
+    # share an input joined with "+"), b and g are powers of two with b * g = D / tau, within what one launch holds,
+    # and only the plan variant they were measured under takes them
+    from paper_2606_17421_b200 import workloads as wl
+    for name, w in wl.WORKLOADS.items():
+        calls = {nm for nm, _, _ in wl.fuse_shared_inputs(w.layers, w.plan.D)}
+        for call, (b, g) in w.splits.items():
+            assert call in calls, (name, call)
+            assert b * g == w.plan.D // w.plan.tau, (name, call)
+            assert b & (b - 1) == 0 and g & (g - 1) == 0 and 1 <= b - 1 <= 64 and g - 1 <= 64, (name, call)
+        headline = wl.PlanSpec(w.plan.D, w.plan.tau, w.plan.b, w.plan.g, "complex", "per_output", "double")
+        for call in calls:
+            assert w.split_of(call, w.plan) == (w.plan.b, w.plan.g)
+            assert w.split_of(call, headline) == w.splits.get(call, (w.plan.b, w.plan.g))

@@ -222,6 +222,21 @@ def run_case(par, plan, d_out, d_in, seed, tol, tag, tight=1e-5):
         low_fused.zero_()
         g.bf.bf_linear_rescaled(g.ctx, ct_in, len(cts), None, Wd, d_out, d_in, low_fused, n_out)
         assert np.array_equal(g.to_host_u64(low_fused), low)
+        # the two entry points on the SAME output address (replayed launch sequences are keyed by the arguments):
+        # a full-level result, then a rescaled one, then a full-level one again, each repeated into its replay
+        shared = g.empty_u64(n_out, 2, par.r, par.N)
+        shared_low = shared.view(-1)[:n_out * 2 * (par.r - 1) * par.N].view(n_out, 2, par.r - 1, par.N)
+        for kind in ("full", "rescaled", "full"):
+            for call in range(3):
+                shared.zero_()
+                if kind == "full":
+                    g.bf.bf_linear(g.ctx, ct_in, len(cts), w, None, d_out, d_in, shared, n_out)
+                else:
+                    g.bf.bf_linear_rescaled(g.ctx, ct_in, len(cts), w, None, d_out, d_in, shared_low, n_out)
+            if kind == "full":
+                assert np.array_equal(g.to_host_u64(shared), got_cached), kind
+            else:
+                assert np.array_equal(g.to_host_u64(shared_low), low), kind
     finally:
         g.close()
 
