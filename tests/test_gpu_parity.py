@@ -689,12 +689,14 @@ def test_unloading_keys_invalidates_replayed_launch_sequences():
         g.close()
 
 
+@pytest.mark.parametrize("modes", [{}, dict(moddown="per_output", hoist="double")], ids=["plain", "extended"])
 @pytest.mark.parametrize("lanes", [3, 4])
-def test_more_giant_rotations_than_one_launch_holds_with_three_and_four_lanes(lanes):
+def test_more_giant_rotations_than_one_launch_holds_with_three_and_four_lanes(lanes, modes):
     # 30 output blocks x 3 giant steps = 90 rotations: as one chain they go in launches of lanes * floor(64 / lanes)
-    # rotations, which must not exceed the 64 a launch holds (with 3 lanes: 63)
+    # rotations, which must not exceed the 64 a launch holds (with 3 lanes: 63); also with the inner sums kept in the
+    # extended basis (30 outputs assembled from 90 key-switch results)
     par = oracle_params("n12")
-    plan = ckks.Plan(64, 4, 4, 4)
+    plan = ckks.Plan(64, 4, 4, 4, **modes)
     d_out, d_in = 1920, 64
     s = ckks.keygen(par, 52)
     keys = ckks.make_rotation_keys(par, s, plan, 52)
@@ -791,11 +793,13 @@ def test_fold_of_more_ciphertexts_than_one_key_switch_batch():
         g.close()
 
 
-def test_fallback_path_in_several_rounds_of_its_scratch():
+@pytest.mark.parametrize("modes", [{}, BEST], ids=["plain", "best"])
+def test_fallback_path_in_several_rounds_of_its_scratch(modes):
     # the on-the-fly path encodes output groups in rounds bounded by a scratch size: one group per round,
     # two per round with a ragged last round, and everything in one round must give the oracle's residues
+    # (headline plan: rounds that start in the middle of a giant step, whose rotated parts are stored permuted)
     par = oracle_params("n12")
-    plan = ckks.Plan(64, 4, 4, 4)
+    plan = ckks.Plan(64, 4, 4, 4, **modes)
     d_out, d_in = 150, 130                        # 3 output blocks x 4 giant steps = 12 groups of 3 x 4 terms
     s = ckks.keygen(par, 31)
     keys = ckks.make_rotation_keys(par, s, plan, 31)
@@ -803,14 +807,14 @@ def test_fallback_path_in_several_rounds_of_its_scratch():
     x = wl.gen_activation(31, "rounds", d_in)
     cts = ckks.encrypt_vector(par, plan, s, x, 31)
     expect = ckks.linear(par, plan, cts, W, keys)
-    group_bytes = 3 * 4 * par.r * par.N * 8
+    group_bytes = 3 * 4 * (par.r + (1 if modes else 0)) * par.N * 8
     g = GpuSide(par, plan)
     try:
         g.load_keys(keys)
-        for bound in (1, 5 * group_bytes + 17, 2 * group_bytes, 1 << 32):
+        for bound in (1, 5 * group_bytes + 17, 2 * group_bytes, 3 * group_bytes, 1 << 32):
             g.bf.bf_set_encode_scratch(g.ctx, bound)
             got = g.to_host_u64(g.linear(cts, W, d_out, d_in))
-            for p in range(3):
+            for p in range(plan.n_out(d_out)):
                 assert np.array_equal(got[p], expect[p]), (bound, p)
         with pytest.raises(g.bf.BifrostError):
             g.bf.bf_set_encode_scratch(g.ctx, 0)
