@@ -376,6 +376,9 @@ struct PolyBatch {
                                   //   residue modulo P: the un-rotated input lifted to the extended basis
     u64* dtile_ptr;               // forward only, non-null: the final result goes there instead of dst, tile-major in tiles
     u32 dtile_div;                //   of KS_TILE coefficients (see ks_tile_index); with `scatter` the store is permuted
+    u32 grid3;                    // set by the launchers: the grid is (x, m, o) and no index has to be divided out
+    u32 o_div_magic, dtile_magic; // ceil(2^32 / o_div), ceil(2^32 / dtile_div): o / d = umulhi(o, magic) for o < 2^16
+                                  //   (set by the launchers with grid3; 0 = divide)
     const u64* div_t;             // forward from a shared source, non-null (double hoisting): the source of digit
     long long div_so;             //   i = o % o_div of set s = o / o_div is the residue modulo q_i of a polynomial in the
                                   //   extended basis, coefficient domain, and t = div_t + s*div_so holds its residue
@@ -390,6 +393,17 @@ struct PolyBatch {
 constexpr u32 KS_TILE = 128;
 __host__ __device__ __forceinline__ size_t ks_tile_index(u32 N, u32 n_m, u32 div, u32 o, u32 m, u32 n) {
     return ((((size_t)(o / div) * n_m + m) * (N / KS_TILE) + n / KS_TILE) * div + o % div) * KS_TILE + n % KS_TILE;
+}
+
+// o / d and o % d with a host-made reciprocal (see PolyBatch::grid3); magic = 0 divides
+__device__ __forceinline__ void split_index(u32 o, u32 d, u32 magic, u32& hi, u32& lo) {
+    hi = magic ? __umulhi(o, magic) : o / d;
+    lo = o - hi * d;
+}
+// ks_tile_index of coefficient 0 of polynomial (o = o_hi * div + o_lo, m); coefficient n then sits at
+// base + (n / KS_TILE) * div * KS_TILE + n % KS_TILE
+__device__ __forceinline__ size_t ks_tile_base(u32 N, u32 n_m, u32 div, u32 o_hi, u32 o_lo, u32 m) {
+    return (((size_t)o_hi * n_m + m) * (N / KS_TILE) * div + o_lo) * KS_TILE;
 }
 
 __device__ __forceinline__ u64 limb_split(u64 v, u32 L) { return ((v >> L) << 32) | (v & ((1ull << L) - 1)); }

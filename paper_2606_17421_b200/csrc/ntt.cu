@@ -337,9 +337,13 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
     ulonglong2 tw_mine = make_ulonglong2(0, 0);
     if (threadIdx.x < LEN) tw_mine = __ldg(&tw_global[threadIdx.x]);
     u64* dst = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
-    const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
-                                   : (size_t)o * B.src_so;
-    const char* src = (const char*)B.src + (src_off + (size_t)m * B.src_sm) * 8;
+    const char* src = nullptr;
+    if constexpr (!STAGED) {
+        u32 o_hi = 0, o_lo = o;
+        if (B.o_div) split_index(o, B.o_div, B.o_div_magic, o_hi, o_lo);
+        const size_t src_off = B.o_div ? (size_t)o_hi * B.src_so2 + (size_t)o_lo * B.src_so : (size_t)o * B.src_so;
+        src = (const char*)B.src + (src_off + (size_t)m * B.src_sm) * 8;
+    }
     LoadConsts lc;
     lc.q = q;
     lc.mu = mu;
@@ -454,6 +458,27 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
     }
 }
 
+// Polynomial (o, m) of a block and its modulus: straight from the grid (x, m, o) when the launcher could lay it out
+// so, else divided out of blockIdx.y.  (n_m <= 2 * mod_wrap in every batch that wraps.)
+__device__ __forceinline__ void block_poly(const PolyBatch& B, u32& o, u32& m, u32& mod) {
+    if (B.grid3) {
+        m = blockIdx.y;
+        o = blockIdx.z;
+    } else {
+        o = blockIdx.y / B.n_m;
+        m = blockIdx.y - o * B.n_m;
+    }
+    const u32 mm = (B.mod_wrap && m >= B.mod_wrap) ? m - B.mod_wrap : m;
+    mod = B.mod0 + mm * B.mod_step;
+}
+// a digit in its own prime (o = set * r + digit with digit == mod), which ModUp copies instead of transforming
+__device__ __forceinline__ bool own_prime(const RingDev& R, const PolyBatch& B, u32 o, u32 mod) {
+    if (!B.skip_diag || mod >= R.r) return false;
+    u32 hi, lo;
+    split_index(o, R.r, B.o_div == R.r ? B.o_div_magic : 0u, hi, lo);
+    return lo == mod;
+}
+
 template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
 __global__ void __launch_bounds__(((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8),
                                   ((1 << (LOG_R + LOG_LANES)) / 8) >= 512 ? 2 : ((1 << (LOG_R + LOG_LANES)) / 8) >= 256 ? 4 : 8)
@@ -461,10 +486,9 @@ ntt_strided(const RingDev R, const PolyBatch B) {
     __shared__ u64 sm[1 << (LOG_R + LOG_LANES)];
     __shared__ ulonglong2 tws[1 << LOG_R];
     grid_dependency_enter();
-    const u32 poly = blockIdx.y;
-    const u32 o = poly / B.n_m, m = poly % B.n_m;
-    const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
-    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) {
+    u32 o, m, mod;
+    block_poly(B, o, m, mod);
+    if (FWD && own_prime(R, B, o, mod)) {
         // this digit's transform in its own prime exists already: copy the tile instead
         const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
         u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
@@ -497,18 +521,19 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
     const u32 m_begin = blockIdx.z * m_per_block;
     const u32 m_end = min(B.n_m, m_begin + m_per_block);
     {
-        const size_t src_off = B.o_div ? (size_t)(o / B.o_div) * B.src_so2 + (size_t)(o % B.o_div) * B.src_so
-                                       : (size_t)o * B.src_so;
+        u32 o_hi = 0, o_lo = o;
+        if (B.o_div) split_index(o, B.o_div, B.o_div_magic, o_hi, o_lo);
+        const size_t src_off = B.o_div ? (size_t)o_hi * B.src_so2 + (size_t)o_lo * B.src_so : (size_t)o * B.src_so;
         const u64* src = (const u64*)B.src + src_off;
         if (B.div_t) {
             // the digit is a division by P away: (source - t) * P^{-1} modulo the digit's own prime, t the centred lift
             // of the polynomial's residue modulo P (exact: same value as dividing in the transform domain)
-            const u32 i = o % B.o_div;
+            const u32 i = o_lo;
             LoadConsts dc;
             dc.q = R.q[i];
             dc.mu = R.mu[i];
             dc.lift_mod = R.q[R.r];
-            const u64* tp = B.div_t + (size_t)(o / B.o_div) * B.div_so;
+            const u64* tp = B.div_t + (size_t)o_hi * B.div_so;
             if (R.fp_ok[i]) {
                 // in fp64 (every value an exact integer): t lazily reduced by the load functor, the difference times
                 // P^{-1} as a centred product, brought to [0, q) -- the digit must be the canonical residue, since it is
@@ -544,8 +569,8 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
     }
     __syncthreads();
     for (u32 m = m_begin; m < m_end; ++m) {
-        const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
-        if (B.skip_diag && mod < R.r && o % R.r == mod) {
+        const u32 mod = B.mod0 + ((B.mod_wrap && m >= B.mod_wrap) ? m - B.mod_wrap : m) * B.mod_step;
+        if (own_prime(R, B, o, mod)) {
             // this digit's transform in its own prime exists already: copy the tile instead
             const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
             u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
@@ -570,7 +595,9 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
 // TILED: the transform-domain side of the batch lives in the tile-major plaintext cache (B.tile_ptr).
 // EPI: 0 = none; 1 = division by P per rotation (scatter through the rotation's permutation); 2 = per output
 // (sum over the output's giant rotations, gathered through their permutations); 3 = plain (see ModDownEpilogue).
-template <bool FWD, int EPI, bool FP, bool TILED>
+// DTILE: the forward result goes to the tile-major operand array of the inner product and nowhere else (ModUp: the
+// hot case; its index arithmetic is hoisted out of the store loop and none of the other store functors is compiled in).
+template <bool FWD, int EPI, bool FP, bool TILED, bool DTILE = false>
 __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B, u64* sm_raw, u32 o, u32 m, u32 mod,
                                             u32 chunk, int lane, const RotBatch& rb, const ModDownEpilogue& epi) {
     typedef typename Elem<FP>::T T;
@@ -590,6 +617,13 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
     const u32 a_mid = slice + 8u * (u32)swz((lane >> 2) * 32 + (lane & 3));           // points base + 4 i
     const u32 a_near = slice + 8u * (u32)swz(4 * lane);                               // points 4 (lane + 32 it) + i
     T e[8];
+    size_t dtile_base = 0;
+    if constexpr (DTILE) {
+        u32 o_hi, o_lo;
+        split_index(o, B.dtile_div, B.dtile_magic, o_hi, o_lo);
+        dtile_base = ks_tile_base(R.N, B.n_m, B.dtile_div, o_hi, o_lo, m);
+    }
+    (void)dtile_base;
     if (FWD) {
         // group 0: K = 3, spacing 32
 #pragma unroll
@@ -669,22 +703,33 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
             }
             set_butterflies<2, true>(e, tw, 64u * mult, (u32)s, q, qd);
             u64 v4[4];
+            if (FP && (q >> 41)) {          // final reduction to [0, q)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {   // final reduction to [0, q)
-                if (FP) {
-                    if (q >> 41) {
-                        v4[i] = d2u(fp_reduce(*(double*)&e[i], qd, R.qinv_d[mod]));
-                    } else {
-                        double v = fp_centre(*(double*)&e[i], qd, R.qinv_d[mod]);
-                        if (v < 0.0) v = __dadd_rn(v, qd);
-                        v4[i] = d2u(v);
-                    }
-                } else {
+                for (int i = 0; i < 4; ++i) v4[i] = d2u(fp_reduce(*(double*)&e[i], qd, R.qinv_d[mod]));
+            } else if (FP) {
+                const double qi = R.qinv_d[mod];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    double v = fp_centre(*(double*)&e[i], qd, qi);
+                    if (v < 0.0) v = __dadd_rn(v, qd);
+                    v4[i] = d2u(v);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
                     u64 v = *(u64*)&e[i];
                     if (v >= 2 * q) v -= 2 * q;
                     if (v >= q) v -= q;
                     v4[i] = v;
                 }
+            }
+            if constexpr (DTILE) {
+                // (4 adjacent coefficients never straddle a tile of 128)
+                const u32 n = chunk * LEN + 4 * s;
+                ulonglong2* gp = (ulonglong2*)(B.dtile_ptr + dtile_base + (size_t)(n / KS_TILE) * B.dtile_div * KS_TILE + n % KS_TILE);
+                gp[0] = make_ulonglong2(v4[0], v4[1]);
+                gp[1] = make_ulonglong2(v4[2], v4[3]);
+                continue;
             }
             if (EPI == 2) {
                 const u32 pp_out = o >> 1, comp = o & 1, ip = mod, r = R.r;
@@ -738,7 +783,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
                 continue;
             }
             if (B.lift_ptr) {   // P times the value, into the extended-basis copy of the un-rotated inputs
-                const u32 comp = B.mod_wrap ? m / B.mod_wrap : 0u, nbp = R.r + 1;
+                const u32 comp = (B.mod_wrap && m >= B.mod_wrap) ? 1u : 0u, nbp = R.r + 1;    // (n_m <= 2 * mod_wrap)
                 u64* xp = B.lift_ptr + (size_t)o * B.lift_so + ((size_t)comp * nbp + mod) * R.N + (size_t)chunk * LEN + 4 * s;
                 u64 p4[4];
 #pragma unroll
@@ -948,22 +993,21 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 
 // (the per-output forms run on a few polynomials per launch and hold the operands of three rotations at once: they
 // trade resident blocks for registers)
-template <bool FWD, int EPI, bool TILED>
+template <bool FWD, int EPI, bool TILED, bool DTILE = false>
 __global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, EPI == 2 ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
     __shared__ __align__(128) u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
     grid_dependency_enter();
-    const u32 poly = blockIdx.y;
-    const u32 o = poly / B.n_m, m = poly % B.n_m;
-    const u32 mod = B.mod0 + (B.mod_wrap ? m % B.mod_wrap : m) * B.mod_step;
-    if (FWD && B.skip_diag && mod < R.r && o % R.r == mod) return;
+    u32 o, m, mod;
+    block_poly(B, o, m, mod);
+    if (FWD && own_prime(R, B, o, mod)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if ((u32)warp >= chunks_per_block) return;
     const u32 chunk = blockIdx.x * chunks_per_block + warp;
     u64* sm = sm_all + (warp << LOG_C);
-    if (R.fp_ok[mod]) contig_body<FWD, EPI, true, TILED>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
-    else contig_body<FWD, EPI, false, TILED>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
+    if (R.fp_ok[mod]) contig_body<FWD, EPI, true, TILED, DTILE>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
+    else contig_body<FWD, EPI, false, TILED, DTILE>(R, B, sm, o, m, mod, chunk, lane, rb, epi);
 }
 
 NttGeometry ntt_geometry(u32 logN) {
@@ -982,15 +1026,33 @@ NttGeometry ntt_geometry(u32 logN) {
     return g;
 }
 
+// Grid of a batch of n_polys = n_outer * n_m polynomials with x_blocks blocks each: (x, m, o) with the reciprocals
+// the kernels use instead of divisions, when the outer count fits the grid's z extent; else (x, o * n_m + m).
+static dim3 poly_grid(PolyBatch& B, u32 x_blocks, u32 n_polys) {
+    const u32 n_outer = n_polys / B.n_m;
+    B.grid3 = 0;
+    B.o_div_magic = B.dtile_magic = 0;
+    if (n_outer * B.n_m != n_polys || n_outer > 65535u || B.n_m > 65535u) return dim3(x_blocks, n_polys);
+    B.grid3 = 1;
+    if (B.o_div) B.o_div_magic = (u32)((((u64)1 << 32) + B.o_div - 1) / B.o_div);
+    if (B.dtile_div) B.dtile_magic = (u32)((((u64)1 << 32) + B.dtile_div - 1) / B.dtile_div);
+    return dim3(x_blocks, B.n_m, n_outer);
+}
+
 template <bool FWD, int LOAD, int LOG_R, int LOG_LANES>
-static void launch_strided_t(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream) {
+static void launch_strided_t(const RingHost& ring, const PolyBatch& B_in, u32 n_polys, cudaStream_t stream) {
     constexpr int NT = ((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8);
-    dim3 grid((1u << LOG_C) >> LOG_LANES, n_polys);
+    PolyBatch B = B_in;
+    const dim3 grid = poly_grid(B, (1u << LOG_C) >> LOG_LANES, n_polys);
     launch_dependent(ring, ntt_strided<FWD, LOAD, LOG_R, LOG_LANES>, grid, dim3(NT), 0, stream, ring.dev, B);
 }
 
 template <int LOAD, int LOG_R, int LOG_LANES>
-static void launch_shared_src_t(const RingHost& ring, const PolyBatch& B, u32 n_outer, cudaStream_t stream) {
+static void launch_shared_src_t(const RingHost& ring, const PolyBatch& B_in, u32 n_outer, cudaStream_t stream) {
+    PolyBatch B = B_in;             // (its grid is (tile, o, slice of the targets): o is never divided out)
+    B.grid3 = 0;
+    B.dtile_magic = B.dtile_div ? (u32)((((u64)1 << 32) + B.dtile_div - 1) / B.dtile_div) : 0u;
+    B.o_div_magic = B.o_div ? (u32)((((u64)1 << 32) + B.o_div - 1) / B.o_div) : 0u;
     constexpr int NT = ((1 << (LOG_R + LOG_LANES)) / 8) < 32 ? 32 : ((1 << (LOG_R + LOG_LANES)) / 8);
     constexpr u32 S = (1u << LOG_C) >> LOG_LANES;
     // targets per block: fewer blocks share the source better but quantise into waves; cost model =
@@ -1050,13 +1112,14 @@ static cudaError_t launch_strided(const RingHost& ring, const PolyBatch& B, u32 
 }
 
 template <bool FWD>
-static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n_polys, cudaStream_t stream,
+static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B_in, u32 n_polys, cudaStream_t stream,
                                  const RotBatch* rb = nullptr, const ModDownEpilogue* epi = nullptr) {
     if (n_polys == 0) return cudaSuccess;
     ProfScope prof(ring.prof, FWD ? CAT_NTT_FWD_CONTIG : CAT_NTT_INV_CONTIG, stream);
     const u32 chunks = 1u << ring.geom.log_r;
     const u32 cpb = (u32)ring.geom.contig_lanes;
-    dim3 grid(chunks / cpb, n_polys);
+    PolyBatch B = B_in;
+    const dim3 grid = poly_grid(B, chunks / cpb, n_polys);
     if (FWD && epi && epi->plain) {
         launch_dependent(ring, ntt_contig<FWD, 3, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb, *rb,
                          *epi);
@@ -1075,6 +1138,9 @@ static cudaError_t launch_contig(const RingHost& ring, const PolyBatch& B, u32 n
         if (B.tile_ptr)
             launch_dependent(ring, ntt_contig<FWD, 0, true>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
                              no_rb, no_epi);
+        else if (FWD && B.dtile_ptr && !B.scatter && !B.lift_ptr && !B.split_bits)
+            launch_dependent(ring, ntt_contig<true, 0, false, true>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B,
+                             cpb, no_rb, no_epi);
         else
             launch_dependent(ring, ntt_contig<FWD, 0, false>, grid, dim3(32 * CHUNKS_PER_BLOCK), 0, stream, ring.dev, B, cpb,
                              no_rb, no_epi);
