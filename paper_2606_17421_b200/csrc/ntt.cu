@@ -366,7 +366,12 @@ __device__ __forceinline__ void strided_body(const RingDev& R, const PolyBatch& 
         lc.k59 = __ldg(ec + 4);
     }
     {
-        const u64 qs = (LOAD == LOAD_REDUCE && B.src_digits) ? R.q[o % R.r] : ~(u64)0;
+        u64 qs = ~(u64)0;
+        if (LOAD == LOAD_REDUCE && B.src_digits) {      // the prime the source digit belongs to
+            u32 s_hi, s_lo;
+            split_index(o, R.r, B.o_div == R.r ? B.o_div_magic : 0u, s_hi, s_lo);
+            qs = R.q[s_lo];
+        }
         lc.src_small = qs <= q + (q >> 1);
         lc.src_fp = qs < (1ull << 51);
     }
