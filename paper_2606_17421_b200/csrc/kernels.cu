@@ -580,7 +580,8 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
         __syncwarp();
         // the r digit segments of this set, modulus and tile are contiguous (see ks_tile_index): one copy
         if (tid == 0)
-            bulk_g2s(buf, dig + ks_tile_index(N, nb, r, (u32)rb.dig[first + it] * r, m, n0), r * KI_TILE * 8, &dbar[it & 1]);
+            bulk_g2s(buf, dig + ks_tile_base(N, nb, r, (u32)rb.dig[first + it], 0u, m) + (size_t)blockIdx.y * r * KI_TILE,
+                     r * KI_TILE * 8, &dbar[it & 1]);
     };
     if (tid < 32) {
         if (tid == 0) mbar_expect_tx(kbar, 2 * r * KI_TILE * 8);
@@ -588,8 +589,8 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
         // the keys do not depend on the previous kernel: fetch them before waiting for it, the digits after
         const u64 stream_policy = l2_evict_first_policy();      // keys stream through; digits and outputs stay in L2
         if (tid == 0)       // the 2r key segments of this key, modulus and tile: one contiguous block
-            bulk_g2s_stream(sk, keys + ks_tile_index(N, nb, 2 * r, (u32)rb.key[first] * 2 * r, m, n0), 2 * r * KI_TILE * 8, kbar,
-                            stream_policy);
+            bulk_g2s_stream(sk, keys + ks_tile_base(N, nb, 2 * r, (u32)rb.key[first], 0u, m) + (size_t)blockIdx.y * 2 * r * KI_TILE,
+                            2 * r * KI_TILE * 8, kbar, stream_policy);
         asm volatile("griddepcontrol.wait;" ::: "memory");
         fetch_digits(0);
         if (cnt > 1) fetch_digits(1);

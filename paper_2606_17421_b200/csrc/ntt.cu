@@ -497,9 +497,15 @@ ntt_strided(const RingDev R, const PolyBatch B) {
         // this digit's transform in its own prime exists already: copy the tile instead
         const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
         u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
+        size_t tbase = 0;
+        if (B.dtile_ptr) {
+            u32 t_hi, t_lo;
+            split_index(o, B.dtile_div, B.dtile_magic, t_hi, t_lo);
+            tbase = ks_tile_base(R.N, B.n_m, B.dtile_div, t_hi, t_lo, m);
+        }
         for (int w = threadIdx.x; w < (1 << (LOG_R + LOG_LANES)); w += blockDim.x) {
             const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * (1 << LOG_LANES) + (w & ((1 << LOG_LANES) - 1));
-            if (B.dtile_ptr) B.dtile_ptr[ks_tile_index(R.N, B.n_m, B.dtile_div, o, m, (u32)gidx)] = ds[gidx];
+            if (B.dtile_ptr) B.dtile_ptr[tbase + (gidx / KS_TILE) * B.dtile_div * KS_TILE + gidx % KS_TILE] = ds[gidx];
             else dd[gidx] = ds[gidx];
         }
         return;
@@ -579,9 +585,15 @@ ntt_strided_shared_src(const RingDev R, const PolyBatch B, u32 m_per_block) {
             // this digit's transform in its own prime exists already: copy the tile instead
             const u64* ds = B.diag_src + (size_t)(o / R.r) * B.diag_so + (size_t)mod * R.N;
             u64* dd = B.dst + (size_t)o * B.dst_so + (size_t)m * B.dst_sm;
+            size_t tbase = 0;
+            if (B.dtile_ptr) {
+                u32 t_hi, t_lo;
+                split_index(o, B.dtile_div, B.dtile_magic, t_hi, t_lo);
+                tbase = ks_tile_base(R.N, B.n_m, B.dtile_div, t_hi, t_lo, m);
+            }
             for (int w = threadIdx.x; w < POINTS; w += blockDim.x) {
                 const size_t gidx = ((size_t)(w >> LOG_LANES) << LOG_C) + blockIdx.x * LANES + (w & (LANES - 1));
-                if (B.dtile_ptr) B.dtile_ptr[ks_tile_index(R.N, B.n_m, B.dtile_div, o, m, (u32)gidx)] = ds[gidx];
+                if (B.dtile_ptr) B.dtile_ptr[tbase + (gidx / KS_TILE) * B.dtile_div * KS_TILE + gidx % KS_TILE] = ds[gidx];
                 else dd[gidx] = ds[gidx];
             }
             continue;
