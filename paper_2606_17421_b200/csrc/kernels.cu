@@ -137,10 +137,13 @@ mac_kernel(const RingDev R, const u64* __restrict__ pt, const TileLayout lay, co
         unit = n_whole + (unit - n_whole) / tail_split;
         n_sub = tail_split;
     }
-    const u32 tile_x = unit % (N >> LOG_TN);
-    const u32 i = prime0 + (unit / (N >> LOG_TN)) % n_launch_primes;   // this launch covers primes prime0 .. + n_launch_primes - 1
+    // (N / TN is a power of two; the remaining quotient by the number of primes of the launch is one division)
+    const u32 tiles_log = R.logN - LOG_TN;
+    const u32 tile_x = unit & ((1u << tiles_log) - 1u);
+    const u32 rest = unit >> tiles_log, slice = rest / n_launch_primes;
+    const u32 i = prime0 + (rest - slice * n_launch_primes);          // this launch covers primes prime0 .. + n_launch_primes - 1
     const u32 n0 = tile_x << LOG_TN;
-    u32 pj_begin = (unit / (N >> LOG_TN) / n_launch_primes) * pj_per_block;
+    u32 pj_begin = slice * pj_per_block;
     u32 pj_end = min(n_pj, pj_begin + pj_per_block);
     if (n_sub > 1) {
         const u32 groups = (pj_end - pj_begin + PL - 1) / PL;
