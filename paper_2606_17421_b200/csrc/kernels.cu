@@ -553,6 +553,28 @@ cudaError_t launch_mac(const RingHost& ring, const u64* pt, const TileLayout& la
 // grid: x = run, y = tile, z = modulus of the extended basis.
 constexpr int KI_TILE = (int)KS_TILE;
 
+// sum over the r digits of digit x key for both key components, reduced (the keys carry a factor 2^64); RC > 0: r == RC
+template <bool SMALL, int RC>
+__device__ __forceinline__ void ki_products(const u64* sdc, const u64* sk, u32 r, u32 tid, u64 q, u32 qneg32, u64& v0, u64& v1) {
+    LimbAcc<SMALL> a0, a1;
+    if constexpr (RC > 0) {
+#pragma unroll
+        for (int j = 0; j < RC; ++j) {
+            const u64 d = sdc[j * KI_TILE + tid];
+            a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
+            a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+        }
+    } else {
+        for (u32 j = 0; j < r; ++j) {
+            const u64 d = sdc[j * KI_TILE + tid];
+            a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
+            a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
+        }
+    }
+    v0 = a0.reduce_mont32(q, qneg32);
+    v1 = a1.reduce_mont32(q, qneg32);
+}
+
 __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDev R, const RotBatch rb,
                                                                    const u64* __restrict__ dig,
                                                                    const u64* __restrict__ keys, u64* __restrict__ u,
@@ -618,23 +640,15 @@ __global__ void __launch_bounds__(KI_TILE, 8) key_inner_bulk_kernel(const RingDe
         mbar_wait(&dbar[it & 1], (it >> 1) & 1, error_flag);
         u64 v0, v1;
         if (m < r && small_ok) {
-            LimbAcc<true> a0, a1;
-            for (u32 j = 0; j < r; ++j) {
-                const u64 d = sdc[j * KI_TILE + tid];
-                a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
-                a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
-            }
-            v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
-            v1 = a1.reduce_mont32(q, qneg32);
+            // (digit counts of the shipped parameter sets with the loop unrolled: the launches where several rotations
+            // share a key are bound by instruction issue)
+            if (r == 7) ki_products<true, 7>(sdc, sk, r, tid, q, qneg32, v0, v1);
+            else if (r == 9) ki_products<true, 9>(sdc, sk, r, tid, q, qneg32, v0, v1);
+            else ki_products<true, 0>(sdc, sk, r, tid, q, qneg32, v0, v1);
         } else {
-            LimbAcc<false> a0, a1;
-            for (u32 j = 0; j < r; ++j) {
-                const u64 d = sdc[j * KI_TILE + tid];
-                a0.mac(d, sk[(j * 2) * KI_TILE + tid]);
-                a1.mac(d, sk[(j * 2 + 1) * KI_TILE + tid]);
-            }
-            v0 = a0.reduce_mont32(q, qneg32);                // the keys carry a factor 2^64
-            v1 = a1.reduce_mont32(q, qneg32);
+            if (r == 7) ki_products<false, 7>(sdc, sk, r, tid, q, qneg32, v0, v1);
+            else if (r == 9) ki_products<false, 9>(sdc, sk, r, tid, q, qneg32, v0, v1);
+            else ki_products<false, 0>(sdc, sk, r, tid, q, qneg32, v0, v1);
         }
         if (it + 2 < cnt) {                                  // the buffer is free once every thread has read it
             __syncthreads();
