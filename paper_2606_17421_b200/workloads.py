@@ -107,15 +107,15 @@ WORKLOADS = {
     # M = 64 diagonals per tile split as 16 baby x 4 giant steps: measured fastest on B200 (fewer full
     # key switches than 8 x 8 at the price of four more rotation keys)
     "gpt2_qkv": Workload("gpt2_qkv", "n15", PlanSpec(1024, 16, 16, 4), (GPT2_LAYER[0],)),
-    # (per call, ms on B200 for 16x4 / 32x2 / 8x8: ffn_down 0.547 / 0.932 / 0.525; the other three are fastest at 16x4)
+    # (per call, ms on B200 for 16x4 / 32x2 / 8x8: ffn_down 0.507 / 0.872 / 0.490; the other three are fastest at 16x4)
     "gpt2_step": Workload("gpt2_step", "n15", PlanSpec(1024, 16, 16, 4), GPT2_LAYER, n_repeat=12,
                           splits={"ffn_down": (8, 8)}),
-    # (16x4 / 32x2 / 8x8: q+k+v 0.405 / 0.418 / 0.562, o 0.417 / 0.580 / 0.430, gate+up 0.505 / 0.471 / 0.766,
-    # down 0.548 / 0.926 / 0.520)
+    # (16x4 / 32x2 / 8x8: q+k+v 0.380 / 0.395 / 0.534, o 0.384 / 0.535 / 0.401, gate+up 0.483 / 0.454 / 0.729,
+    # down 0.507 / 0.872 / 0.490)
     "qwen3_step": Workload("qwen3_step", "n15", PlanSpec(1024, 16, 16, 4), QWEN3_LAYER, n_repeat=28,
                            cache_budget_bytes=60 * 10 ** 9, splits={"gate+up": (32, 2), "down": (8, 8)}),
-    # (8x4 / 16x2 / 4x8: q+k+v 1.85 / 1.90 / 2.58, o 1.48 / 1.67 / 1.91, gate+up 6.07 / 4.33 / 10.25 (32x1: 4.57),
-    # down 4.00 / 6.65 / 3.55 (2x16: 4.51))
+    # (8x4 / 16x2 / 4x8: q+k+v 1.79 / 1.79 / 2.49, o 1.43 / 1.56 / 1.84, gate+up 5.88 / 4.25 / 9.86,
+    # down 3.78 / 6.29 / 3.44)
     "llama3_layer": Workload("llama3_layer", "n16", PlanSpec(1024, 32, 8, 4), LLAMA3_8B_LAYER,
                              splits={"gate+up": (16, 2), "down": (4, 8)}),
 }
