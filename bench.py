@@ -42,8 +42,9 @@ NCU_TRAFFIC_RATIO = {
 # Executed warp instructions per butterfly by pipe, from the same captures (profiles/gpt2_layer_headline_plan_kernels_ncu.md),
 # to set beside the modelled 8 / 12 / 10 operations: the large fp64-path batches of each direction.
 NCU_PIPE_INSTR = {
-    "ntt_forward": {"all": 27.2, "fp64": 8.2, "alu": 7.4, "fma_integer": 6.1, "lsu": 2.4,
-                    "from": "hoisted ModUp of three inputs (147 transforms), both passes"},
+    "ntt_forward": {"all": 24.7, "fp64": 8.3, "alu": 6.3, "fma_integer": 5.4, "lsu": 2.4,
+                    "from": "hoisted ModUp of three inputs (147 transforms: six primes on the 8-operation fp64 path, one "
+                            "on the 12-operation one, one on the 60-bit integer path), both passes"},
     "ntt_inverse": {"all": 21.0, "fp64": 10.3, "alu": 3.9, "fma_integer": 2.0, "lsu": 2.3,
                     "from": "c1 of 3 giant rotations x 7 primes, both passes (an earlier capture of the same kernels)"},
 }
