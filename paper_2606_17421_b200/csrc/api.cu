@@ -897,6 +897,9 @@ static void rescale_consts(const bf_ctx* ctx, u32 level, RescaleConsts& rc) {
         rc.inv[i] = h_invmod(qL % q, q);
         rc.invs[i] = h_shoup(rc.inv[i], q);
         rc.qlmod[i] = qL % q;
+        rc.inv_d[i] = (double)rc.inv[i];
+        rc.inv_q[i] = (double)rc.inv[i] / (double)q;
+        rc.qlmod_d[i] = (double)rc.qlmod[i];
     }
 }
 

@@ -287,6 +287,7 @@ struct MacScatter {
 // Constants of a rescale from `level` primes: q_L^{-1} mod q_i with its Shoup companion, and q_L mod q_i (i < level - 1).
 struct RescaleConsts {
     u64 inv[MAX_MODULI], invs[MAX_MODULI], qlmod[MAX_MODULI];
+    double inv_d[MAX_MODULI], inv_q[MAX_MODULI], qlmod_d[MAX_MODULI];   // the same as doubles; inv_q = inv / q_i
 };
 
 // Tile-major layout of cached plaintexts, chosen so that the multiply-accumulate kernel's blocks

@@ -775,6 +775,7 @@ cudaError_t launch_rescale(const RingHost& ring, const u64* in, u64* out, u32 n_
                            const u64* invs, const u64* qlmod, cudaStream_t stream) {
     if (n_ct == 0) return cudaSuccess;
     RescaleConsts rc;
+    memset(&rc, 0, sizeof(rc));
     for (u32 i = 0; i + 1 < level; ++i) { rc.inv[i] = inv[i]; rc.invs[i] = invs[i]; rc.qlmod[i] = qlmod[i]; }
     ProfScope prof(ring.prof, CAT_RESCALE, stream);
     if (in == out && n_ct > 1) {

@@ -1260,8 +1260,11 @@ __global__ void __launch_bounds__(256) finish_division_kernel(const RingDev R, u
     }
     u64 t = 0;                      // the residue that is dropped
 #pragma unroll
-    for (int i = 0; i < MAX_MODULI; ++i)
-        if ((u32)i == R.r - 1) t = v[i];
+    for (int i = 0; i < MAX_MODULI; ++i) {
+        u64 vi = v[i];
+        asm volatile("" : "+l"(vi));    // (keeps the selection a chain of moves: as an indexed read it would put v in local memory)
+        if ((u32)i == R.r - 1) t = vi;
+    }
     const bool high = t > (R.q[R.r - 1] - 1) / 2;
     u64* lp = low + ((size_t)p * 2 + comp) * (R.r - 1) * R.N + n;
 #pragma unroll
@@ -1274,11 +1277,91 @@ __global__ void __launch_bounds__(256) finish_division_kernel(const RingDev R, u
         }
 }
 
+// The same in fp64 (every value an exact integer below 2^53), for rings whose ciphertext primes are all on the fp64
+// path: a 64-bit modular product costs about twenty integer instructions, an exact fp64 one six on a pipe that is
+// otherwise idle here.  Each term sum S = s_hi 2^30 + s_lo is reduced as s_hi (2^30 mod q) + s_lo; products come back
+// centred and are brought to [0, q) only where a canonical residue is needed (the stored words, the dropped residue).
+__device__ __forceinline__ double fp_times_const(double x, bool wide, double w, double wq, double q, double qinv) {
+    // x an integer of magnitude below 2^50 (any sign): x * w mod q in [0, q)
+    double s2;
+    if (wide) s2 = fp_mul_centred(__dadd_rn(fp_centre(x, q, qinv), q), w, wq, q);     // operand in (0.5q, 1.5q)
+    else s2 = fp_mul_centred_signed(x, w, wq, q);
+    return s2 < 0.0 ? __dadd_rn(s2, q) : s2;
+}
+
+__global__ void __launch_bounds__(256) finish_division_fp_kernel(const RingDev R, u64* __restrict__ ct, long long ct_stride,
+                                                                 const u64* __restrict__ T, u32 n_t, const RescaleConsts rc,
+                                                                 u64* __restrict__ low) {
+    grid_dependency_enter();
+    const u32 n = blockIdx.x * 256 + threadIdx.x;
+    const u32 p = blockIdx.y >> 1, comp = blockIdx.y & 1;
+    const u64* tp = T + (size_t)p * n_t * R.N + n;
+    u64* cp = ct + (size_t)p * ct_stride + (size_t)comp * R.r * R.N + n;
+    double v[MAX_MODULI];
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i)
+        if ((u32)i < R.r) v[i] = u2d(cp[(size_t)i * R.N]);
+    const u32 nt = comp == 0 ? n_t - 2 : 2u;
+    for (u32 k0 = 0; k0 < nt; k0 += 8) {
+        i64 S = 0;
+        for (u32 k = k0; k < nt && k < k0 + 8; ++k) {
+            const u32 m = k < 2 ? comp + 2 * k : k + 2;
+            S += (i64)(tp[(size_t)m * R.N] - (1ull << 59));
+        }
+        const i64 s_hi = S >> 30;                               // |s_hi| < 2^33
+        const double lo = u2d((u64)(S & ((1ll << 30) - 1)));
+        const bool sneg = s_hi < 0;
+        const double ah = u2d((u64)(sneg ? -s_hi : s_hi));
+#pragma unroll
+        for (int i = 0; i < MAX_MODULI; ++i)
+            if ((u32)i < R.r) {
+                const double sm = fp_mul_centred(ah, R.c30_d[i], R.c30_q[i], R.qd[i]);      // within 0.75 q
+                const double x = __dsub_rn(__dsub_rn(v[i], sneg ? -sm : sm), lo);
+                v[i] = fp_centre(x, R.qd[i], R.qinv_d[i]);
+            }
+    }
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i)
+        if ((u32)i < R.r) v[i] = fp_times_const(v[i], (R.q[i] >> 41) != 0, R.pinv_d[i], R.pinv_q[i], R.qd[i], R.qinv_d[i]);
+    if (!low) {
+#pragma unroll
+        for (int i = 0; i < MAX_MODULI; ++i)
+            if ((u32)i < R.r) cp[(size_t)i * R.N] = d2u(v[i]);
+        return;
+    }
+    double t = 0.0;                 // the residue that is dropped (below 2^46: the launcher checked)
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i) {
+        double vi = v[i];
+        asm volatile("" : "+d"(vi));    // (keeps the selection a chain of moves: as an indexed read it would put v in local memory)
+        if ((u32)i == R.r - 1) t = vi;
+    }
+    const bool high = d2u(t) > (R.q[R.r - 1] - 1) / 2;
+    u64* lp = low + ((size_t)p * 2 + comp) * (R.r - 1) * R.N + n;
+#pragma unroll
+    for (int i = 0; i < MAX_MODULI; ++i)
+        if ((u32)i + 1 < R.r) {
+            double tq = fp_reduce(t, R.qd[i], R.qinv_d[i]);
+            if (high) tq = __dsub_rn(tq, rc.qlmod_d[i]);
+            const double y = fp_times_const(__dsub_rn(v[i], tq), (R.q[i] >> 41) != 0, rc.inv_d[i], rc.inv_q[i], R.qd[i],
+                                            R.qinv_d[i]);
+            lp[(size_t)i * R.N] = d2u(y);
+        }
+}
+
 cudaError_t finish_division(const RingHost& ring, u64* ct, long long ct_stride, const u64* T, u32 n_t, u32 n_out,
                             cudaStream_t stream, const RescaleConsts* rc, u64* low) {
     ProfScope prof(ring.prof, CAT_DIVIDE, stream);
     RescaleConsts none;
     memset(&none, 0, sizeof(none));
+    bool fp = true;
+    for (u32 i = 0; i < ring.dev.r; ++i) fp = fp && ring.dev.fp_ok[i];
+    if (rc && ring.q[ring.dev.r - 1] >= (1ull << 46)) fp = false;
+    if (fp) {
+        launch_dependent(ring, finish_division_fp_kernel, dim3(ring.dev.N / 256, n_out * 2), dim3(256), 0, stream, ring.dev,
+                         ct, ct_stride, T, n_t, rc ? *rc : none, rc ? low : (u64*)nullptr);
+        return cudaGetLastError();
+    }
     launch_dependent(ring, finish_division_kernel, dim3(ring.dev.N / 256, n_out * 2), dim3(256), 0, stream, ring.dev, ct,
                      ct_stride, T, n_t, rc ? *rc : none, rc ? low : (u64*)nullptr);
     return cudaGetLastError();
