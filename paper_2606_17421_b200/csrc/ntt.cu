@@ -1011,7 +1011,7 @@ __device__ __forceinline__ void contig_body(const RingDev& R, const PolyBatch& B
 // (the per-output forms run on a few polynomials per launch and hold the operands of three rotations at once: they
 // trade resident blocks for registers)
 template <bool FWD, int EPI, bool TILED, bool DTILE = false>
-__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, EPI == 2 ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
+__global__ void __launch_bounds__(32 * CHUNKS_PER_BLOCK, (EPI == 2 || EPI == 4) ? 5 : 8) ntt_contig(const RingDev R, const PolyBatch B,
                                                                        u32 chunks_per_block, const RotBatch rb,
                                                                        const ModDownEpilogue epi) {
     __shared__ __align__(128) u64 sm_all[CHUNKS_PER_BLOCK << LOG_C];
