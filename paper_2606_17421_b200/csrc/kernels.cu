@@ -734,7 +734,9 @@ __global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const Res
   for (u32 ct = blockIdx.y; ct < blockIdx.y + n_seq; ++ct) {
     const u64* ip = in + (size_t)ct * 2 * level * N + n;
     u64* op = out + (size_t)ct * 2 * (level - 1) * N + n;
-    u64 res[2][MAX_MODULI];
+    // In place the packed output of residue (comp, i) lands where residue (comp, i) (component 0) or (comp, i - 1)
+    // (component 1) was read, and the dropped residues are read before anything of their component is written: so
+    // each residue is read, then its slot (or an earlier one) written, in order, with nothing held back.
 #pragma unroll
     for (int comp = 0; comp < 2; ++comp) {
         const u64 t = ip[((size_t)comp * level + (level - 1)) * N];
@@ -744,12 +746,9 @@ __global__ void __launch_bounds__(256) rescale_kernel(const RingDev R, const Res
             u64 tq = barrett64(t, q, R.mu[i]);
             if (high) tq = sub_mod(tq, rc.qlmod[i], q);
             const u64 c = ip[((size_t)comp * level + i) * N];
-            res[comp][i] = mul_shoup(sub_mod(c, tq, q), rc.inv[i], rc.invs[i], q);
+            op[((size_t)comp * (level - 1) + i) * N] = mul_shoup(sub_mod(c, tq, q), rc.inv[i], rc.invs[i], q);
         }
     }
-#pragma unroll
-    for (int comp = 0; comp < 2; ++comp)
-        for (u32 i = 0; i + 1 < level; ++i) op[((size_t)comp * (level - 1) + i) * N] = res[comp][i];
   }
 }
 
