@@ -600,11 +600,15 @@ class OracleSample:
         per_inner = t["inner"] / t["n_inner"]
         per_giant = t["giant"] / t["n_giant"]
         total = 0.0
-        for L in self.w.layers:
-            n_in, n_out = wl.ceil_div(L.d_in, plan.D), plan.n_out(L.d_out)
-            total += n_in * (plan.b - 1) * per_baby
-            total += n_out * plan.g * per_inner * (n_in / self.n_in)
-            total += n_out * (plan.g - 1) * per_giant
+        spec = wl.PlanSpec(plan.D, plan.tau, plan.b, plan.g, plan.pack, plan.moddown, plan.hoist)
+        # the calls the runner issues: projections that share an input stacked, each under its baby/giant split (an
+        # inner sum has n_in * b terms: its sampled cost is scaled by both)
+        for name, d_in, members in wl.fuse_shared_inputs(self.w.layers, plan.D):
+            b, g = self.w.split_of(name, spec)
+            n_in, n_out = wl.ceil_div(d_in, plan.D), plan.n_out(sum(m.d_out for m in members))
+            total += n_in * (b - 1) * per_baby
+            total += n_out * g * per_inner * (n_in / self.n_in) * (b / plan.b)
+            total += n_out * (g - 1) * per_giant
             total += n_out * t["rescale"]
         return total * self.w.n_repeat * 1e3
 
@@ -621,7 +625,7 @@ class OracleSample:
     def describe(self) -> str:
         return (f"plan pack={self.plan.pack} moddown={self.plan.moddown} hoist={self.plan.hoist}; layer {self.L.name}: {len(self.baby_ks)} of {self.plan.b - 1} baby rotations of one input and "
                 f"{len(self.groups)} of {self.n_out * self.plan.g} (block, giant-step) groups (inner sum, giant "
-                f"rotation) plus one rescale per step, scaled by unit counts to every layer of the workload")
+                f"rotation) plus one rescale per step, scaled by unit counts to every call of the workload (stacked projections, per-call splits)")
 
 
 def cpu_baseline(workload: str, budget_s: float) -> dict:
