@@ -899,9 +899,25 @@ def test_error_paths_do_not_touch_the_device():
         with pytest.raises(bf.BifrostError) as ei:          # wrong number of input ciphertexts
             bf.bf_linear(ctx, ct, 2, None, W, 64, 64, ct.clone(), 1)
         assert ei.value.code == bf.BF_ERR_SHAPE
+        low = torch.zeros((1, 2, 2, ps["N"]), dtype=torch.int64, device="cuda")
+        with pytest.raises(bf.BifrostError) as ei:          # the fused call reports the same errors
+            bf.bf_linear_rescaled(ctx, ct, 1, None, W, 64, 64, low, 1)
+        assert ei.value.code == bf.BF_ERR_MISSING_KEY
+        with pytest.raises(bf.BifrostError) as ei:
+            bf.bf_linear_rescaled(ctx, ct, 2, None, W, 64, 64, low, 1)
+        assert ei.value.code == bf.BF_ERR_SHAPE
+        with pytest.raises(bf.BifrostError) as ei:          # no output buffer
+            bf.bf_linear_rescaled(ctx, ct, 1, None, W, 64, 64, None, 1)
+        assert ei.value.code == bf.BF_ERR_INVALID_ARG
         bf.bf_set_cache_budget(ctx, 1000)
         with pytest.raises(bf.BifrostError) as ei:
             bf.bf_encode_weights(ctx, W, 64, 64)
         assert ei.value.code == bf.BF_ERR_OOM
+        with pytest.raises(bf.BifrostError) as ei:          # (the budget is checked after the split)
+            bf.bf_encode_weights_split(ctx, W, 64, 64, 16, 4)
+        assert ei.value.code == bf.BF_ERR_OOM
+        with pytest.raises(bf.BifrostError) as ei:
+            bf.bf_encode_weights_split(ctx, W, 64, 64, 16, 8)
+        assert ei.value.code == bf.BF_ERR_SHAPE
     finally:
         bf.bf_ctx_destroy(ctx)
