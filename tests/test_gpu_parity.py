@@ -457,6 +457,61 @@ def test_weights_with_a_split_of_their_own(modes):
         g.close()
 
 
+@pytest.mark.parametrize("case", range(32))
+def test_random_small_ring_cases(case):
+    # seeded random draws over what the other cases fix by hand: tile side, replica split, baby/giant split of the plan
+    # and of the handle, the three plan flags, ragged shapes with one to three input and output blocks; the cached
+    # call, the replayed call and the fused product + rescale must all match the oracle
+    rng = np.random.default_rng(1000 + case)
+    par = oracle_params("n12")
+    D = int(rng.choice([32, 64, 128]))
+    tau = int(rng.choice([t for t in (1, 2, 4, 8, 16) if D * t <= par.n and D // t >= 2]))
+    M = D // tau
+    splits = [(b, M // b) for b in (1, 2, 4, 8, 16, 32, 64) if b <= M and M % b == 0 and b - 1 <= 64 and M // b - 1 <= 64]
+    b, g_ = splits[int(rng.integers(len(splits)))]
+    hb, hg = splits[int(rng.integers(len(splits)))]
+    modes = dict(pack=str(rng.choice(["real", "complex"])), moddown=str(rng.choice(["per_rotation", "per_output"])),
+                 hoist=str(rng.choice(["single", "double"])))
+    d_in = int(rng.integers(1, 3 * D + 1))
+    d_out = int(rng.integers(1, 3 * D + 1))
+    base = ckks.Plan(D, tau, b, g_, **modes)
+    hplan = ckks.Plan(D, tau, hb, hg, **modes)
+    seed = 2000 + case
+    W = wl.gen_weights(seed, "rand", d_out, d_in)
+    x = wl.gen_activation(seed, "rand", d_in)
+    s = ckks.keygen(par, seed)
+    extra = ckks.required_rotations(hplan)
+    keys = ckks.make_rotation_keys(par, s, base, seed, extra_steps=extra)
+    cts = ckks.encrypt_vector(par, base, s, x, seed)
+    expect_base = ckks.linear(par, base, cts, W, keys)
+    expect_h = ckks.linear(par, hplan, cts, W, keys)
+    n_out = base.n_out(d_out)
+    g = GpuSide(par, base)
+    try:
+        g.load_keys(keys, extra_steps=extra)
+        Wd = g.to_dev(W)
+        ct_in = g.to_dev(np.stack(cts))
+        for plan, expect, w in ((base, expect_base, g.bf.bf_encode_weights(g.ctx, Wd, d_out, d_in)),
+                                (hplan, expect_h, g.bf.bf_encode_weights_split(g.ctx, Wd, d_out, d_in, hb, hg))):
+            out = g.empty_u64(n_out, 2, par.r, par.N)
+            low = g.empty_u64(n_out, 2, par.r - 1, par.N)
+            for call in range(3):
+                out.zero_()
+                low.zero_()
+                g.bf.bf_linear(g.ctx, ct_in, len(cts), w, None, d_out, d_in, out, n_out)
+                g.bf.bf_linear_rescaled(g.ctx, ct_in, len(cts), w, None, d_out, d_in, low, n_out)
+            got, got_low = g.to_host_u64(out), g.to_host_u64(low)
+            for p in range(n_out):
+                assert np.array_equal(got[p], expect[p]), (case, plan, p)
+                assert np.array_equal(got_low[p], ckks.rescale(par, expect[p])), (case, plan, p, "rescaled")
+            g.bf.bf_weights_free(g.ctx, w)
+        fly = g.to_host_u64(g.linear(cts, W, d_out, d_in))          # on the fly: the plan's own split
+        for p in range(n_out):
+            assert np.array_equal(fly[p], expect_base[p]), (case, p, "on the fly")
+    finally:
+        g.close()
+
+
 def test_linear_gpt2_qkv_config_bit_exact():
     w = wl.WORKLOADS["gpt2_qkv"]
     par = oracle_params(w.params)
